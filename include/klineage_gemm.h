@@ -1,0 +1,156 @@
+/*
+ * klineage_gemm.h - C ABI of the B200 (sm_100a) bf16 GEMM lineage.
+ *
+ * The library computes  C <- A . B  for bf16 A and B with fp32 accumulation and
+ * an fp32 or bf16 C, for arbitrary (unaligned) M, N, K and leading dimensions.
+ * It offers the same product through five separately selectable kernels that
+ * form a forward lineage in the sense of the paper's Method section (a lineage
+ * L = (K_0, tau_1, ..., K_n) from a naive kernel K_0 to an expert kernel K_n):
+ * each rung adds one of the optimization intents the paper's Introduction and
+ * Table 1 name, together with the precondition that makes it valid.
+ *
+ * C99, no C++ types, no exceptions cross this boundary.  All pointers named
+ * "device" are device pointers on the handle's GPU; everything else is host
+ * memory.  There is no CPU fallback and no cross-rung fallback: a variant
+ * either runs its own kernel or the call returns an error (the paper's
+ * harness notes, Appendix B, describe how wrappers that silently fall back to
+ * a reference fake correctness).
+ */
+#ifndef KLINEAGE_GEMM_H
+#define KLINEAGE_GEMM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Opaque handle, owned by the library, released by klineage_gemm_destroy. */
+typedef struct klineage_gemm_s* klineage_gemm_t;
+
+typedef enum {
+    KLINEAGE_OK = 0,
+    KLINEAGE_ERR_INVALID_ARG = 1,        /* null pointer, negative size, ld too small, aliasing ... */
+    KLINEAGE_ERR_BAD_VARIANT = 2,        /* variant outside 0..4                                      */
+    KLINEAGE_ERR_UNSUPPORTED_DEVICE = 3, /* the rung needs sm_100 hardware the device lacks          */
+    KLINEAGE_ERR_ALLOC = 4,              /* device or host allocation failed in create                */
+    KLINEAGE_ERR_LAUNCH = 5,             /* the CUDA runtime rejected a launch or a tensor map        */
+    KLINEAGE_ERR_TIMEOUT = 6,            /* a bounded device-side wait gave up (see get_device_status) */
+    KLINEAGE_ERR_INTERNAL = 7
+} klineage_status_t;
+
+/* Storage of B (K x N).  A is always row-major M x K, C always row-major M x N. */
+typedef enum {
+    KLINEAGE_B_ROW_MAJOR = 0, /* element (k, j) at B[k * ldb + j]  (N contiguous) */
+    KLINEAGE_B_COL_MAJOR = 1  /* element (k, j) at B[j * ldb + k]  (K contiguous) */
+} klineage_layout_t;
+
+typedef enum {
+    KLINEAGE_C_F32 = 0, /* C holds the fp32 accumulator                                  */
+    KLINEAGE_C_BF16 = 1 /* C holds the accumulator rounded to bf16, round-to-nearest-even */
+} klineage_ctype_t;
+
+/*
+ * The lineage rungs (paper: Introduction, "tiling, shared-memory staging,
+ * vectorized loads, software pipelining, or hardware intrinsics"; Table 1).
+ */
+typedef enum {
+    KLINEAGE_NAIVE = 0,      /* K_0: one thread per C element, K-loop over global memory                     */
+    KLINEAGE_TILED = 1,      /* Table 1 "tile / sm_stage": block tile staged in shared memory, register tile */
+    KLINEAGE_VECTORIZED = 2, /* Table 1 "vectorize_global": 128-bit accesses when aligned, masked tail,
+                                scalar fallback when base or leading dimension is not 16-byte aligned        */
+    KLINEAGE_PIPELINED = 3,  /* Table 1 "cp.async + pipeline" / "tma_load": multi-stage ring fed by TMA with
+                                full/empty mbarriers; producer threads when TMA's alignment rules fail       */
+    KLINEAGE_TCGEN05 = 4     /* Table 1 "warp_specialize" + matrix intrinsics: tcgen05.mma into TMEM (the
+                                sm_100 successor of the table's wgmma), producer / MMA / epilogue warps,
+                                persistent tile scheduler, swizzled shared-memory epilogue, split-K          */
+} klineage_variant_t;
+
+/* Create-time configuration (host memory, read during create only). */
+typedef struct {
+    int device;             /* CUDA device ordinal the handle is bound to                              */
+    int b_layout;           /* klineage_layout_t                                                       */
+    int c_dtype;            /* klineage_ctype_t                                                        */
+    size_t workspace_bytes; /* device scratch for split-K partial sums; 0 selects the default (32 MiB) */
+    unsigned flags;         /* reserved, must be 0                                                     */
+} klineage_gemm_config_t;
+
+/*
+ * Creates a handle bound to cfg->device with the given B layout and C dtype
+ * (the paper's GEMM workload, Evaluation Table 2, fixes neither; they are
+ * properties of the handle so that klineage_gemm_run keeps the BLAS-like
+ * argument list).  Allocates the device workspace and status block (this is the
+ * only allocating call besides destroy).  out and cfg are host pointers.
+ * Errors: INVALID_ARG (null, bad enum, flags != 0, no such device), ALLOC.
+ */
+klineage_status_t klineage_gemm_create(klineage_gemm_t* out, const klineage_gemm_config_t* cfg);
+
+/*
+ * Enqueues C <- A . B on `stream` (a cudaStream_t, may be NULL for the default
+ * stream) using exactly the rung `variant`; returns after the enqueue, performs
+ * no device synchronisation and no allocation.
+ *
+ *   M, N, K   sizes, 0 <= value < 2^31.  M*N == 0: nothing is launched, OK.
+ *             K == 0: C is set to zero.
+ *   A         device, bf16 bits, row-major M x K, lda >= K  (elements)
+ *   B         device, bf16 bits, K x N in the handle's layout,
+ *             ldb >= N (row-major) or ldb >= K (column-major)
+ *   C         device, fp32 or bf16 per the handle, row-major, ldc >= N; write-only
+ *             (previous contents, NaN included, are ignored); padding between N and
+ *             ldc is never written.  A and B must not overlap C.
+ *   Pointers need only element alignment (2 bytes bf16, 4 bytes fp32); wider
+ *   alignment is detected per call and selects the vector / TMA sub-paths
+ *   (paper, Introduction: "vectorized loads require alignment and valid tail
+ *   handling").  Buffers stay owned by the caller.
+ *
+ * Errors: INVALID_ARG, BAD_VARIANT, UNSUPPORTED_DEVICE (variant 3 or 4 on a
+ * device without sm_100 TMA/tcgen05), LAUNCH.  Device-side give-ups (a bounded
+ * barrier wait that expired) are reported by klineage_gemm_get_device_status.
+ * One handle must not be used from two host threads at once.
+ */
+klineage_status_t klineage_gemm_run(klineage_gemm_t h, int64_t M, int64_t N, int64_t K,
+                                    const void* A, int64_t lda, const void* B, int64_t ldb,
+                                    void* C, int64_t ldc, int variant, void* stream);
+
+/*
+ * The host-side argument checks of klineage_gemm_run, callable without a handle
+ * or a device (pointers are only compared, never dereferenced).  Returns what
+ * run would return for these arguments before touching the GPU: OK,
+ * INVALID_ARG or BAD_VARIANT.  The paper states the principle (Introduction):
+ * an optimization applied outside its precondition yields a wrong or failing
+ * kernel, so preconditions are checked, not assumed.
+ */
+klineage_status_t klineage_gemm_check_args(int b_layout, int c_dtype, int64_t M, int64_t N, int64_t K,
+                                           const void* A, int64_t lda, const void* B, int64_t ldb,
+                                           const void* C, int64_t ldc, int variant);
+
+/* Releases the handle, its workspace and status block.  NULL is accepted. */
+klineage_status_t klineage_gemm_destroy(klineage_gemm_t h);
+
+/*
+ * Reads the device status block (synchronous copy; call after synchronising
+ * the stream).  *code_out receives KLINEAGE_OK or KLINEAGE_ERR_TIMEOUT;
+ * *kernel_id_out (may be NULL) receives the id the last finished kernel wrote
+ * on the device, which identifies rung and sub-path (see
+ * klineage_gemm_last_kernel_id).  The error code is cleared by the read.
+ * The paper's gate (Method: compile, correctness, profile) is what this serves.
+ */
+klineage_status_t klineage_gemm_get_device_status(klineage_gemm_t h, int* code_out, int* kernel_id_out);
+
+/*
+ * Host-side record of the kernel the last successful run enqueued:
+ *   0 naive | 100 tiled | 200 + 1*(A vector) + 2*(B vector) + 4*(C vector)
+ *   300 TMA pipeline, 301 producer-thread pipeline
+ *   400 + 1*(generic-proxy producer) + 2*(direct epilogue) + 4*(split-K)
+ *   900 zero fill (K == 0); -1 before the first run or after a no-op.
+ */
+int klineage_gemm_last_kernel_id(klineage_gemm_t h);
+
+const char* klineage_status_string(int status);
+const char* klineage_variant_name(int variant);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KLINEAGE_GEMM_H */

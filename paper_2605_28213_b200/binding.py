@@ -1,0 +1,187 @@
+"""ctypes face of ``libklineage_gemm.so``: argument marshalling only.
+
+Names mirror the C ABI (``include/klineage_gemm.h``).  PyTorch appears only as
+the owner of device memory and streams.  There is no fallback of any kind: if
+the CUDA library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional
+
+PKG = Path(__file__).resolve().parent
+LIB_PATH = PKG / "libklineage_gemm.so"
+
+KLINEAGE_OK = 0
+KLINEAGE_ERR_INVALID_ARG = 1
+KLINEAGE_ERR_BAD_VARIANT = 2
+KLINEAGE_ERR_UNSUPPORTED_DEVICE = 3
+KLINEAGE_ERR_ALLOC = 4
+KLINEAGE_ERR_LAUNCH = 5
+KLINEAGE_ERR_TIMEOUT = 6
+KLINEAGE_ERR_INTERNAL = 7
+
+KLINEAGE_B_ROW_MAJOR, KLINEAGE_B_COL_MAJOR = 0, 1
+KLINEAGE_C_F32, KLINEAGE_C_BF16 = 0, 1
+KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELINED, KLINEAGE_TCGEN05 = range(5)
+VARIANTS = (KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELINED, KLINEAGE_TCGEN05)
+
+EXPORTED_SYMBOLS = (
+    "klineage_gemm_create", "klineage_gemm_run", "klineage_gemm_destroy", "klineage_gemm_check_args",
+    "klineage_gemm_get_device_status", "klineage_gemm_last_kernel_id", "klineage_status_string",
+    "klineage_variant_name",
+)
+
+
+class klineage_gemm_config_t(ctypes.Structure):
+    _fields_ = [("device", ctypes.c_int), ("b_layout", ctypes.c_int), ("c_dtype", ctypes.c_int),
+                ("workspace_bytes", ctypes.c_size_t), ("flags", ctypes.c_uint)]
+
+
+class KlineageError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {klineage_status_string(status)} (status {status})")
+
+
+if not LIB_PATH.exists():
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2605_28213_b200.build` "
+        "(nvcc, sm_100a).  This package has no CPU or PyTorch fallback.")
+
+_lib = ctypes.CDLL(str(LIB_PATH))
+_i64, _p, _int = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
+
+_lib.klineage_gemm_create.restype = _int
+_lib.klineage_gemm_create.argtypes = [ctypes.POINTER(_p), ctypes.POINTER(klineage_gemm_config_t)]
+_lib.klineage_gemm_run.restype = _int
+_lib.klineage_gemm_run.argtypes = [_p, _i64, _i64, _i64, _p, _i64, _p, _i64, _p, _i64, _int, _p]
+_lib.klineage_gemm_destroy.restype = _int
+_lib.klineage_gemm_destroy.argtypes = [_p]
+_lib.klineage_gemm_check_args.restype = _int
+_lib.klineage_gemm_check_args.argtypes = [_int, _int, _i64, _i64, _i64, _p, _i64, _p, _i64, _p, _i64, _int]
+_lib.klineage_gemm_get_device_status.restype = _int
+_lib.klineage_gemm_get_device_status.argtypes = [_p, ctypes.POINTER(_int), ctypes.POINTER(_int)]
+_lib.klineage_gemm_last_kernel_id.restype = _int
+_lib.klineage_gemm_last_kernel_id.argtypes = [_p]
+_lib.klineage_status_string.restype = ctypes.c_char_p
+_lib.klineage_status_string.argtypes = [_int]
+_lib.klineage_variant_name.restype = ctypes.c_char_p
+_lib.klineage_variant_name.argtypes = [_int]
+
+
+def klineage_status_string(status: int) -> str:
+    return _lib.klineage_status_string(int(status)).decode()
+
+
+def klineage_variant_name(variant: int) -> str:
+    return _lib.klineage_variant_name(int(variant)).decode()
+
+
+def klineage_gemm_check_args(b_layout, c_dtype, M, N, K, A, lda, B, ldb, C, ldc, variant) -> int:
+    """Raw status of the host-side argument checks (pointers are integers or None)."""
+    return _lib.klineage_gemm_check_args(b_layout, c_dtype, M, N, K, A, lda, B, ldb, C, ldc, variant)
+
+
+def klineage_gemm_create(device: int, b_layout: int, c_dtype: int, workspace_bytes: int = 0,
+                         flags: int = 0) -> int:
+    """Returns the opaque handle (an integer); raises KlineageError on failure."""
+    cfg = klineage_gemm_config_t(device, b_layout, c_dtype, workspace_bytes, flags)
+    h = _p()
+    st = _lib.klineage_gemm_create(ctypes.byref(h), ctypes.byref(cfg))
+    if st != KLINEAGE_OK:
+        raise KlineageError(st, "klineage_gemm_create")
+    return h.value
+
+
+def klineage_gemm_run_raw(h, M, N, K, A, lda, B, ldb, C, ldc, variant, stream) -> int:
+    """Raw status code; pointers are integers (device addresses) or None."""
+    return _lib.klineage_gemm_run(h, M, N, K, A, lda, B, ldb, C, ldc, variant, stream)
+
+
+def klineage_gemm_run(h, M, N, K, A, lda, B, ldb, C, ldc, variant, stream=None) -> None:
+    st = klineage_gemm_run_raw(h, M, N, K, A, lda, B, ldb, C, ldc, variant, stream)
+    if st != KLINEAGE_OK:
+        raise KlineageError(st, "klineage_gemm_run")
+
+
+def klineage_gemm_destroy(h) -> None:
+    _lib.klineage_gemm_destroy(h)
+
+
+def klineage_gemm_get_device_status(h):
+    """(status code, id of the kernel that last ran on the device)."""
+    code, kid = _int(0), _int(0)
+    st = _lib.klineage_gemm_get_device_status(h, ctypes.byref(code), ctypes.byref(kid))
+    if st != KLINEAGE_OK:
+        raise KlineageError(st, "klineage_gemm_get_device_status")
+    return code.value, kid.value
+
+
+def klineage_gemm_last_kernel_id(h) -> int:
+    return _lib.klineage_gemm_last_kernel_id(h)
+
+
+class Gemm:
+    """Handle wrapper: ``Gemm(device, b_col_major, c_bf16).run(A, B, C, M, N, K, lda, ldb, ldc, variant)``.
+
+    ``A``, ``B``, ``C`` are torch CUDA tensors (any shape; only ``data_ptr()`` is
+    used) or integer device addresses.  The launch goes to torch's current stream
+    unless ``stream`` (a ``torch.cuda.Stream`` or raw pointer) is given.
+    """
+
+    def __init__(self, device: int = 0, b_col_major: bool = False, c_bf16: bool = False,
+                 workspace_bytes: int = 0):
+        self.device = int(device)
+        self.b_col_major = bool(b_col_major)
+        self.c_bf16 = bool(c_bf16)
+        self._h: Optional[int] = klineage_gemm_create(
+            self.device, KLINEAGE_B_COL_MAJOR if b_col_major else KLINEAGE_B_ROW_MAJOR,
+            KLINEAGE_C_BF16 if c_bf16 else KLINEAGE_C_F32, workspace_bytes)
+
+    @staticmethod
+    def _ptr(x):
+        if x is None or isinstance(x, int):
+            return x
+        return x.data_ptr()
+
+    @staticmethod
+    def _stream(stream):
+        if stream is None:
+            import torch
+            return torch.cuda.current_stream().cuda_stream
+        if isinstance(stream, int):
+            return stream
+        return stream.cuda_stream
+
+    def run(self, A, B, C, M, N, K, lda, ldb, ldc, variant, stream=None) -> None:
+        klineage_gemm_run(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(C), ldc,
+                          int(variant), self._stream(stream))
+
+    def run_raw(self, A, B, C, M, N, K, lda, ldb, ldc, variant, stream=None) -> int:
+        return klineage_gemm_run_raw(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(C),
+                                     ldc, int(variant), self._stream(stream))
+
+    def device_status(self):
+        return klineage_gemm_get_device_status(self._h)
+
+    def last_kernel_id(self) -> int:
+        return klineage_gemm_last_kernel_id(self._h)
+
+    def close(self) -> None:
+        if self._h is not None:
+            klineage_gemm_destroy(self._h)
+            self._h = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,128 @@
+// Shared declarations of the GEMM lineage kernels: the argument block every
+// rung receives, device-side status codes, bf16 helpers and the tile raster.
+#pragma once
+#include <cstdint>
+#include <cuda.h>          // CUtensorMap and its enums only; libcuda is never linked
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+namespace klin {
+
+// Problem description handed to every rung.  A is row-major M x K; B is K x N,
+// row-major (b_col == 0: element (k,j) at B[k*ldb + j]) or column-major
+// (b_col == 1: element (k,j) at B[j*ldb + k]); C is row-major M x N, fp32 or
+// bf16.  Leading dimensions are in elements.  status points at the handle's
+// device status block: status[0] = first device-side error code (0 = none),
+// status[1] = id of the kernel that ran last, status[2..3] = error detail.
+struct GemmArgs {
+    int M, N, K;
+    const uint16_t* A;
+    int64_t lda;
+    const uint16_t* B;
+    int64_t ldb;
+    void* C;
+    int64_t ldc;
+    int b_col;
+    int c_bf16;
+    unsigned* status;
+};
+
+// Device-side error codes written to status[0].
+enum DeviceError : unsigned {
+    kDevOk = 0,
+    kDevBarrierTimeout = 1,   // a bounded mbarrier wait gave up
+};
+
+// Kernel ids written to status[1] and reported by klineage_gemm_last_kernel_id().
+enum KernelId : int {
+    kIdNaive = 0,
+    kIdTiled = 100,
+    kIdVectorized = 200,      // + 1 (A vector loads) + 2 (B vector loads) + 4 (C vector stores)
+    kIdPipelined = 300,       // + 1 when the producer-thread path replaces TMA
+    kIdTcgen05 = 400,         // + 1 generic-proxy producer, + 2 direct epilogue, + 4 split-K
+    kIdZeroFill = 900,
+};
+
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t h)
+{
+    return __uint_as_float(static_cast<uint32_t>(h) << 16);
+}
+// Low / high half of a packed pair of bf16 values.
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+__device__ __forceinline__ uint16_t float_to_bf16_bits(float f)
+{
+    return __bfloat16_as_ushort(__float2bfloat16_rn(f));
+}
+// Two floats -> packed bf16x2 (lo in bits 0..15), round to nearest even.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    return static_cast<uint32_t>(float_to_bf16_bits(lo)) | (static_cast<uint32_t>(float_to_bf16_bits(hi)) << 16);
+}
+
+__device__ __forceinline__ void store_c(void* C, int c_bf16, int64_t idx, float v)
+{
+    if (c_bf16)
+        static_cast<uint16_t*>(C)[idx] = float_to_bf16_bits(v);
+    else
+        static_cast<float*>(C)[idx] = v;
+}
+
+__device__ __forceinline__ void report_error(unsigned* status, unsigned code, unsigned d0, unsigned d1)
+{
+    if (atomicCAS(&status[0], 0u, code) == 0u) {
+        status[2] = d0;
+        status[3] = d1;
+    }
+}
+
+// Tile raster shared by the tiled rungs: linear tile index -> (tile_m, tile_n),
+// walking groups of kGroupM tile-rows column by column so that the tiles in
+// flight together share A row-panels and B column-panels in L2.
+constexpr int kGroupM = 8;
+__host__ __device__ __forceinline__ void raster_tile(int64_t t, int tiles_m, int tiles_n, int& tm, int& tn)
+{
+    const int64_t per_group = static_cast<int64_t>(kGroupM) * tiles_n;
+    const int g = static_cast<int>(t / per_group);
+    const int first_m = g * kGroupM;
+    const int rows = (tiles_m - first_m < kGroupM) ? (tiles_m - first_m) : kGroupM;
+    const int64_t r = t - static_cast<int64_t>(g) * per_group;
+    tm = first_m + static_cast<int>(r % rows);
+    tn = static_cast<int>(r / rows);
+}
+
+// Per-rung launchers (defined one per translation unit).  Each enqueues its
+// kernel(s) on `stream`, returns the launch error and reports the kernel id.
+typedef CUresult (*TensorMapEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                           const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                           CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                           CUtensorMapFloatOOBfill);
+
+// Host-side state of a handle that the TMA rungs need.
+struct RunContext {
+    int device = 0;
+    int sm_count = 0;
+    int cc_major = 0, cc_minor = 0;
+    int max_smem_optin = 0;
+    TensorMapEncodeTiledFn encode_tiled = nullptr;   // from cudaGetDriverEntryPoint
+    void* workspace = nullptr;                       // split-K partial sums (fp32)
+    size_t workspace_bytes = 0;
+    unsigned* tile_counters = nullptr;               // split-K arrival counters, zero between calls
+    int n_tile_counters = 0;
+    unsigned flags = 0;
+};
+
+// Encodes a 2-D tiled tensor map (dims/strides innermost first; stride of the
+// outer dimension in bytes).  Returns false when the driver rejects it.
+bool encode_map_2d(const RunContext& ctx, CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t dim0,
+                   uint64_t dim1, uint64_t stride1_bytes, uint32_t box0, uint32_t box1, CUtensorMapSwizzle swz);
+
+cudaError_t launch_r0_naive(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
+cudaError_t launch_r1_tiled(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
+cudaError_t launch_r2_vectorized(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
+cudaError_t launch_r3_pipelined(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id);
+cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id);
+cudaError_t launch_zero_fill(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
+
+}  // namespace klin

@@ -1,0 +1,264 @@
+// Host runtime and C ABI of the GEMM lineage: handle, argument validation,
+// alignment classification, tensor-map encoding, rung dispatch, status block.
+// No rung ever substitutes for another, and nothing here computes on the CPU.
+#include "../../include/klineage_gemm.h"
+#include "common.cuh"
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+using namespace klin;
+
+struct klineage_gemm_s {
+    RunContext ctx;
+    int b_layout = 0;
+    int c_dtype = 0;
+    unsigned* status = nullptr;   // device: 4 words (error, kernel id, detail0, detail1)
+    int last_kernel_id = -1;
+};
+
+namespace klin {
+
+bool encode_map_2d(const RunContext& ctx, CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t dim0,
+                   uint64_t dim1, uint64_t stride1_bytes, uint32_t box0, uint32_t box1, CUtensorMapSwizzle swz)
+{
+    if (!ctx.encode_tiled) return false;
+    const cuuint64_t dims[2] = {dim0, dim1};
+    const cuuint64_t strides[1] = {stride1_bytes};
+    const cuuint32_t box[2] = {box0, box1};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = ctx.encode_tiled(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
+                                        CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+}  // namespace klin
+
+namespace {
+
+constexpr size_t kDefaultWorkspace = 32u << 20;
+constexpr int kTileCounters = 4096;
+
+// Restores the caller's current device on scope exit.
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        ok = (prev == dev) || (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard()
+    {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+bool ranges_overlap(const void* a, size_t a_bytes, const void* b, size_t b_bytes)
+{
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + b_bytes && b0 < a0 + a_bytes;
+}
+
+}  // namespace
+
+extern "C" {
+
+klineage_status_t klineage_gemm_create(klineage_gemm_t* out, const klineage_gemm_config_t* cfg)
+{
+    if (!out) return KLINEAGE_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!cfg) return KLINEAGE_ERR_INVALID_ARG;
+    if (cfg->b_layout != KLINEAGE_B_ROW_MAJOR && cfg->b_layout != KLINEAGE_B_COL_MAJOR) return KLINEAGE_ERR_INVALID_ARG;
+    if (cfg->c_dtype != KLINEAGE_C_F32 && cfg->c_dtype != KLINEAGE_C_BF16) return KLINEAGE_ERR_INVALID_ARG;
+    if (cfg->flags != 0) return KLINEAGE_ERR_INVALID_ARG;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev) {
+        cudaGetLastError();
+        return KLINEAGE_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(cfg->device);
+    if (!guard.ok) return KLINEAGE_ERR_INVALID_ARG;
+
+    klineage_gemm_s* h = new (std::nothrow) klineage_gemm_s();
+    if (!h) return KLINEAGE_ERR_ALLOC;
+    h->b_layout = cfg->b_layout;
+    h->c_dtype = cfg->c_dtype;
+    RunContext& c = h->ctx;
+    c.device = cfg->device;
+    cudaDeviceGetAttribute(&c.sm_count, cudaDevAttrMultiProcessorCount, c.device);
+    cudaDeviceGetAttribute(&c.cc_major, cudaDevAttrComputeCapabilityMajor, c.device);
+    cudaDeviceGetAttribute(&c.cc_minor, cudaDevAttrComputeCapabilityMinor, c.device);
+    cudaDeviceGetAttribute(&c.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, c.device);
+
+    // cuTensorMapEncodeTiled comes from the driver at run time, so the library
+    // has no link-time dependency on libcuda.
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+        c.encode_tiled = reinterpret_cast<TensorMapEncodeTiledFn>(fn);
+    else
+        cudaGetLastError();
+
+    c.workspace_bytes = cfg->workspace_bytes ? cfg->workspace_bytes : kDefaultWorkspace;
+    c.n_tile_counters = kTileCounters;
+    bool ok = cudaMalloc(&c.workspace, c.workspace_bytes) == cudaSuccess;
+    ok = ok && cudaMalloc(reinterpret_cast<void**>(&c.tile_counters), sizeof(unsigned) * kTileCounters) == cudaSuccess;
+    ok = ok && cudaMalloc(reinterpret_cast<void**>(&h->status), 4 * sizeof(unsigned)) == cudaSuccess;
+    ok = ok && cudaMemset(c.tile_counters, 0, sizeof(unsigned) * kTileCounters) == cudaSuccess;
+    ok = ok && cudaMemset(h->status, 0, 4 * sizeof(unsigned)) == cudaSuccess;
+    ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        klineage_gemm_destroy(h);
+        return KLINEAGE_ERR_ALLOC;
+    }
+    *out = h;
+    return KLINEAGE_OK;
+}
+
+klineage_status_t klineage_gemm_destroy(klineage_gemm_t h)
+{
+    if (!h) return KLINEAGE_OK;
+    {
+        DeviceGuard guard(h->ctx.device);
+        if (h->ctx.workspace) cudaFree(h->ctx.workspace);
+        if (h->ctx.tile_counters) cudaFree(h->ctx.tile_counters);
+        if (h->status) cudaFree(h->status);
+    }
+    delete h;
+    return KLINEAGE_OK;
+}
+
+klineage_status_t klineage_gemm_check_args(int b_layout, int c_dtype, int64_t M, int64_t N, int64_t K, const void* A,
+                                           int64_t lda, const void* B, int64_t ldb, const void* C, int64_t ldc,
+                                           int variant)
+{
+    if (b_layout != KLINEAGE_B_ROW_MAJOR && b_layout != KLINEAGE_B_COL_MAJOR) return KLINEAGE_ERR_INVALID_ARG;
+    if (c_dtype != KLINEAGE_C_F32 && c_dtype != KLINEAGE_C_BF16) return KLINEAGE_ERR_INVALID_ARG;
+    if (variant < KLINEAGE_NAIVE || variant > KLINEAGE_TCGEN05) return KLINEAGE_ERR_BAD_VARIANT;
+    const int64_t lim = int64_t(1) << 31;
+    if (M < 0 || N < 0 || K < 0 || M >= lim || N >= lim || K >= lim) return KLINEAGE_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return KLINEAGE_OK;
+    const bool bcol = b_layout == KLINEAGE_B_COL_MAJOR;
+    const size_t celt = c_dtype == KLINEAGE_C_BF16 ? 2 : 4;
+    if (!C || ldc < N) return KLINEAGE_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(C) % celt) return KLINEAGE_ERR_INVALID_ARG;
+    if (K > 0) {
+        if (!A || !B) return KLINEAGE_ERR_INVALID_ARG;
+        if (lda < K || ldb < (bcol ? K : N)) return KLINEAGE_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(A) % 2 || reinterpret_cast<uintptr_t>(B) % 2) return KLINEAGE_ERR_INVALID_ARG;
+        const size_t a_bytes = (size_t(M - 1) * lda + K) * 2;
+        const size_t b_bytes = (size_t((bcol ? N : K) - 1) * ldb + (bcol ? K : N)) * 2;
+        const size_t c_bytes = (size_t(M - 1) * ldc + N) * celt;
+        if (ranges_overlap(A, a_bytes, C, c_bytes) || ranges_overlap(B, b_bytes, C, c_bytes))
+            return KLINEAGE_ERR_INVALID_ARG;
+    }
+    return KLINEAGE_OK;
+}
+
+klineage_status_t klineage_gemm_run(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                    const void* B, int64_t ldb, void* C, int64_t ldc, int variant, void* stream)
+{
+    if (!h) return KLINEAGE_ERR_INVALID_ARG;
+    const klineage_status_t chk = klineage_gemm_check_args(h->b_layout, h->c_dtype, M, N, K, A, lda, B, ldb, C, ldc, variant);
+    if (chk != KLINEAGE_OK) return chk;
+    if (M == 0 || N == 0) {
+        h->last_kernel_id = -1;
+        return KLINEAGE_OK;
+    }
+    const bool bcol = h->b_layout == KLINEAGE_B_COL_MAJOR;
+    if ((variant == KLINEAGE_PIPELINED || variant == KLINEAGE_TCGEN05) && h->ctx.cc_major != 10)
+        return KLINEAGE_ERR_UNSUPPORTED_DEVICE;
+
+    DeviceGuard guard(h->ctx.device);
+    if (!guard.ok) return KLINEAGE_ERR_LAUNCH;
+
+    GemmArgs g;
+    g.M = static_cast<int>(M);
+    g.N = static_cast<int>(N);
+    g.K = static_cast<int>(K);
+    g.A = static_cast<const uint16_t*>(A);
+    g.lda = lda;
+    g.B = static_cast<const uint16_t*>(B);
+    g.ldb = ldb;
+    g.C = C;
+    g.ldc = ldc;
+    g.b_col = bcol ? 1 : 0;
+    g.c_bf16 = h->c_dtype == KLINEAGE_C_BF16 ? 1 : 0;
+    g.status = h->status;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int kid = -1;
+    cudaError_t e;
+    if (K == 0) {
+        e = launch_zero_fill(g, s, &kid);
+    } else {
+        switch (variant) {
+            case KLINEAGE_NAIVE: e = launch_r0_naive(g, s, &kid); break;
+            case KLINEAGE_TILED: e = launch_r1_tiled(g, s, &kid); break;
+            case KLINEAGE_VECTORIZED: e = launch_r2_vectorized(g, s, &kid); break;
+            case KLINEAGE_PIPELINED: e = launch_r3_pipelined(g, h->ctx, s, &kid); break;
+            default: e = launch_r4_tcgen05(g, h->ctx, s, &kid); break;
+        }
+    }
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return KLINEAGE_ERR_LAUNCH;
+    }
+    h->last_kernel_id = kid;
+    return KLINEAGE_OK;
+}
+
+klineage_status_t klineage_gemm_get_device_status(klineage_gemm_t h, int* code_out, int* kernel_id_out)
+{
+    if (!h || !code_out) return KLINEAGE_ERR_INVALID_ARG;
+    DeviceGuard guard(h->ctx.device);
+    unsigned w[4] = {0, 0, 0, 0};
+    if (cudaMemcpy(w, h->status, sizeof w, cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return KLINEAGE_ERR_INTERNAL;
+    }
+    *code_out = (w[0] == kDevOk) ? KLINEAGE_OK : KLINEAGE_ERR_TIMEOUT;
+    if (kernel_id_out) *kernel_id_out = static_cast<int>(w[1]);
+    if (w[0] != kDevOk) {
+        fprintf(stderr, "klineage_gemm: device-side give-up code=%u block=%u where=0x%x\n", w[0], w[2], w[3]);
+        if (cudaMemset(h->status, 0, sizeof(unsigned)) != cudaSuccess) cudaGetLastError();
+    }
+    return KLINEAGE_OK;
+}
+
+int klineage_gemm_last_kernel_id(klineage_gemm_t h) { return h ? h->last_kernel_id : -1; }
+
+const char* klineage_status_string(int status)
+{
+    switch (status) {
+        case KLINEAGE_OK: return "ok";
+        case KLINEAGE_ERR_INVALID_ARG: return "invalid argument";
+        case KLINEAGE_ERR_BAD_VARIANT: return "bad variant";
+        case KLINEAGE_ERR_UNSUPPORTED_DEVICE: return "unsupported device";
+        case KLINEAGE_ERR_ALLOC: return "allocation failed";
+        case KLINEAGE_ERR_LAUNCH: return "launch failed";
+        case KLINEAGE_ERR_TIMEOUT: return "device-side wait timed out";
+        case KLINEAGE_ERR_INTERNAL: return "internal error";
+        default: return "unknown status";
+    }
+}
+
+const char* klineage_variant_name(int variant)
+{
+    switch (variant) {
+        case KLINEAGE_NAIVE: return "naive";
+        case KLINEAGE_TILED: return "tiled";
+        case KLINEAGE_VECTORIZED: return "vectorized";
+        case KLINEAGE_PIPELINED: return "pipelined";
+        case KLINEAGE_TCGEN05: return "tcgen05";
+        default: return "unknown";
+    }
+}
+
+}  // extern "C"

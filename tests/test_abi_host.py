@@ -1,0 +1,105 @@
+"""Host-only checks of the C ABI: the library loads without a GPU, exports every
+symbol the header declares, and validates arguments before touching a device."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def kb():
+    from paper_2605_28213_b200 import build
+    build.build()
+    from paper_2605_28213_b200 import binding
+    return binding
+
+
+def declared_functions():
+    names = set()
+    for hdr in (ROOT / "include").glob("*.h"):
+        text = re.sub(r"/\*.*?\*/", "", hdr.read_text(), flags=re.S)
+        names |= set(re.findall(r"\b(klineage_[a-z0-9_]+)\s*\(", text))
+    return names
+
+
+def test_library_exports_every_declared_symbol(kb):
+    decl = declared_functions()
+    assert {"klineage_gemm_create", "klineage_gemm_run", "klineage_gemm_destroy"} <= decl
+    lib = ctypes.CDLL(str(kb.LIB_PATH))
+    for name in decl:
+        assert hasattr(lib, name), f"{name} declared in include/ but not exported"
+    assert decl == set(kb.EXPORTED_SYMBOLS) | {n for n in decl if n not in kb.EXPORTED_SYMBOLS}
+    for name in kb.EXPORTED_SYMBOLS:
+        assert name in decl or name.startswith("klineage_"), name
+
+
+def test_status_and_variant_names(kb):
+    assert kb.klineage_status_string(0) == "ok"
+    assert kb.klineage_status_string(kb.KLINEAGE_ERR_BAD_VARIANT) == "bad variant"
+    assert kb.klineage_status_string(12345) == "unknown status"
+    assert [kb.klineage_variant_name(v) for v in range(5)] == ["naive", "tiled", "vectorized", "pipelined", "tcgen05"]
+    assert kb.klineage_variant_name(5) == "unknown"
+
+
+def test_check_args_rules(kb):
+    chk = kb.klineage_gemm_check_args
+    A, B, C = 0x10000, 0x20000, 0x40000
+    ok = lambda **kw: chk(**{**dict(b_layout=0, c_dtype=0, M=8, N=9, K=10, A=A, lda=10, B=B, ldb=9, C=C, ldc=9,
+                                    variant=0), **kw})
+    assert ok() == kb.KLINEAGE_OK
+    assert ok(variant=5) == kb.KLINEAGE_ERR_BAD_VARIANT and ok(variant=-1) == kb.KLINEAGE_ERR_BAD_VARIANT
+    assert ok(b_layout=2) == kb.KLINEAGE_ERR_INVALID_ARG and ok(c_dtype=3) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert ok(M=-1) == kb.KLINEAGE_ERR_INVALID_ARG and ok(K=1 << 31) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert ok(lda=9) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert ok(ldb=8) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert ok(ldc=8) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert ok(b_layout=1, ldb=9) == kb.KLINEAGE_ERR_INVALID_ARG      # column-major needs ldb >= K
+    assert ok(b_layout=1, ldb=10) == kb.KLINEAGE_OK
+    assert ok(A=None) == kb.KLINEAGE_ERR_INVALID_ARG and ok(C=None) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert ok(A=A + 1) == kb.KLINEAGE_ERR_INVALID_ARG                # bf16 needs 2-byte alignment
+    assert ok(C=C + 2) == kb.KLINEAGE_ERR_INVALID_ARG                # fp32 C needs 4-byte alignment
+    assert ok(C=C + 2, c_dtype=1) == kb.KLINEAGE_OK                  # bf16 C needs only 2
+    assert ok(C=A + 4) == kb.KLINEAGE_ERR_INVALID_ARG                # C overlaps A
+    assert ok(C=B) == kb.KLINEAGE_ERR_INVALID_ARG                    # C overlaps B
+    assert ok(M=0, A=None, C=None) == kb.KLINEAGE_OK                 # empty product: nothing is read
+    assert ok(K=0, A=None, B=None) == kb.KLINEAGE_OK                 # K == 0 only writes C
+    assert ok(A=A + 2, B=B + 2, lda=11) == kb.KLINEAGE_OK            # element alignment suffices
+
+
+def test_no_handle_and_no_device_paths(kb):
+    assert kb.klineage_gemm_run_raw(None, 1, 1, 1, 16, 1, 32, 1, 64, 1, 0, None) == kb.KLINEAGE_ERR_INVALID_ARG
+    kb.klineage_gemm_destroy(None)
+    assert kb.klineage_gemm_last_kernel_id(None) == -1
+    import torch
+    if not torch.cuda.is_available():
+        with pytest.raises(kb.KlineageError) as e:
+            kb.klineage_gemm_create(0, 0, 0)
+        assert e.value.status == kb.KLINEAGE_ERR_INVALID_ARG
+
+
+def test_binding_refuses_to_import_without_the_library(tmp_path, monkeypatch):
+    """No fallback: with the shared library absent the binding must raise, not degrade."""
+    import importlib.util
+    src = (ROOT / "paper_2605_28213_b200" / "binding.py").read_text()
+    fake = tmp_path / "binding_copy.py"
+    fake.write_text(src)
+    spec = importlib.util.spec_from_file_location("binding_copy", fake)
+    mod = importlib.util.module_from_spec(spec)
+    with pytest.raises(ImportError):
+        spec.loader.exec_module(mod)
+
+
+def test_product_never_imports_the_oracle():
+    """The product and the oracle share no code and neither imports the other."""
+    imp = re.compile(r"^\s*(from|import)\s+oracle\b|liboracle|oracle_gemm|gemm_oracle|oracle/", re.M)
+    for py in (ROOT / "paper_2605_28213_b200").rglob("*.py"):
+        assert not imp.search(py.read_text()), f"{py} reaches into the oracle"
+    for src in (ROOT / "paper_2605_28213_b200" / "csrc").glob("*.cu*"):
+        assert not imp.search(src.read_text()), f"{src} reaches into the oracle"
+    back = re.compile(r"^\s*(from|import)\s+paper_2605_28213_b200|klineage_gemm|csrc", re.M)
+    for f in (ROOT / "oracle").glob("*"):
+        if f.suffix in (".py", ".c"):
+            assert not back.search(f.read_text()), f"{f} reaches into the product"

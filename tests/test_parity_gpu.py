@@ -1,0 +1,234 @@
+"""GPU parity: every lineage rung, through the C ABI, against the CPU oracle.
+
+Bit-exact on integer-valued inputs; within K * 2^-23 * (|A|.|B|)_ij on random
+bf16 inputs (fp32 C), widened by one bf16 rounding for bf16 C.  The paper's own
+gate is "correctness at three random seeds" (Evaluation, Setup); seeds 1..3 are
+used on the small configurations.
+"""
+import numpy as np
+import pytest
+
+from paper_2605_28213_b200 import inputs as gen
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+VARIANT_NAMES = ["naive", "tiled", "vectorized", "pipelined", "tcgen05"]
+VARIANTS = list(range(5))
+
+
+@pytest.fixture(scope="module")
+def kb():
+    from paper_2605_28213_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def handles(kb):
+    """One handle per (B layout, C dtype)."""
+    hs = {(col, bf): kb.Gemm(0, b_col_major=col, c_bf16=bf) for col in (False, True) for bf in (False, True)}
+    yield hs
+    for h in hs.values():
+        h.close()
+
+
+def run_and_check(handles, case, variant, C_ref=None, S=None, rows=None, exact=False, offsets=(0, 0, 0)):
+    dev = P.DeviceCase(case, *offsets)
+    dev.run(handles[(case.b_col_major, case.c_bf16)], variant)
+    vals, bits = dev.result()
+    if C_ref is None:
+        rows = np.arange(case.M)
+        C_ref, S = P.oracle_rows(case, rows)
+    P.assert_matches_oracle(case, vals[rows], bits[rows], C_ref, S, exact,
+                            f"{case.name} {VARIANT_NAMES[variant]}")
+    return vals, bits
+
+
+# ------------------------------------------------------------------ the five configurations
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_NAMES)
+@pytest.mark.parametrize("name,seeds", [("c1", (1, 2, 3)), ("c2", (1, 2, 3)), ("c2pad", (1,)), ("c5", (1,)),
+                                        ("c3", (1,)), ("c4", (1,))])
+def test_config_random_within_bound(handles, variant, name, seeds):
+    for seed in seeds:
+        case, rows, C_ref, S = P.cached_reference(name, seed, False)
+        run_and_check(handles, case, variant, C_ref, S, rows)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_NAMES)
+@pytest.mark.parametrize("name", ["c1", "c2", "c2pad", "c5", "c3", "c4"])
+def test_config_integer_bit_exact(handles, variant, name):
+    case, rows, C_ref, S = P.cached_reference(name, 2, True)
+    vals_a, _ = run_and_check(handles, case, variant, C_ref, S, rows, exact=True)
+    # the other output dtype, plus the full-matrix checksum on whichever result is fp32
+    import dataclasses
+    other = dataclasses.replace(case, c_bf16=not case.c_bf16)
+    vals_b, _ = run_and_check(handles, other, variant, C_ref, S, rows, exact=True)
+    f32_vals = vals_b if case.c_bf16 else vals_a
+    assert P.integer_checksums_match(case, f32_vals), "row/column checksums of the full matrix differ"
+
+
+# ------------------------------------------------------------------ adversarial shapes
+EDGE = [1, 2, 7, 8, 9, 15, 16, 17, 63, 64, 65, 127, 128, 129, 255, 257]
+ADVERSARIAL = [(1, 1, 1), (1, 1, 257), (2, 7, 8), (7, 2, 9), (8, 9, 15), (9, 8, 16), (15, 17, 17), (16, 16, 63),
+               (17, 15, 64), (63, 65, 65), (64, 64, 127), (65, 63, 128), (127, 129, 129), (128, 128, 255),
+               (129, 127, 257), (255, 257, 1), (257, 255, 2), (1, 257, 129), (257, 1, 127), (130, 260, 70),
+               (300, 520, 200), (16, 700, 1030), (5, 33, 4100)]
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_NAMES)
+@pytest.mark.parametrize("col", [False, True], ids=["Brow", "Bcol"])
+def test_adversarial_shapes(handles, variant, col):
+    assert all(d in EDGE or d > 257 for s in ADVERSARIAL[:19] for d in s)
+    for idx, (M, N, K) in enumerate(ADVERSARIAL):
+        for bf in (False, True):
+            # integer values: bit-exact, catches any dropped / duplicated / mis-indexed product
+            ci = gen.make_case(M, N, K, seed=idx, dist_a="integer", dist_b="integer", b_col_major=col, c_bf16=bf,
+                               name=f"adv{M}x{N}x{K}-int")
+            run_and_check(handles, ci, variant, exact=True)
+        cr = gen.make_case(M, N, K, seed=idx, dist_a="normal", dist_b="uniform", b_col_major=col, c_bf16=False,
+                           name=f"adv{M}x{N}x{K}")
+        run_and_check(handles, cr, variant)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_NAMES)
+@pytest.mark.parametrize("col", [False, True], ids=["Brow", "Bcol"])
+def test_unaligned_bases_and_padded_leading_dimensions(handles, variant, col):
+    shapes = [(130, 136, 72), (67, 250, 129), (256, 264, 64)]
+    for idx, (M, N, K) in enumerate(shapes):
+        for (pa, pb, pc), offs in [((0, 0, 0), (1, 1, 1)), ((8, 8, 8), (0, 0, 0)), ((3, 5, 7), (1, 3, 1)),
+                                   ((8, 16, 4), (8, 8, 4)), ((8, 8, 8), (0, 1, 0)), ((8, 8, 8), (0, 0, 1))]:
+            for bf in (False, True):
+                case = gen.make_case(M, N, K, seed=100 + idx, dist_a="integer", dist_b="integer", lda=K + pa,
+                                     ldb=(K if col else N) + pb, ldc=N + pc, b_col_major=col, c_bf16=bf,
+                                     name=f"ld{M}x{N}x{K}+{pa},{pb},{pc}@{offs}")
+                run_and_check(handles, case, variant, exact=True, offsets=offs)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_NAMES)
+def test_random_small_shapes(handles, variant):
+    rng = np.random.default_rng(1234 + variant)
+    for it in range(24):
+        M, N, K = (int(rng.integers(1, 400)) for _ in range(3))
+        col, bf = bool(rng.integers(2)), bool(rng.integers(2))
+        pa, pb, pc = (int(rng.integers(0, 9)) for _ in range(3))
+        case = gen.make_case(M, N, K, seed=it, dist_a="uniform", dist_b="normal", lda=K + pa,
+                             ldb=(K if col else N) + pb, ldc=N + pc, b_col_major=col, c_bf16=bf, name=f"rnd{it}")
+        run_and_check(handles, case, variant, offsets=tuple(int(rng.integers(0, 3)) for _ in range(3)))
+
+
+# ------------------------------------------------------------------ degenerate sizes
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_NAMES)
+def test_degenerate_sizes(handles, kb, variant):
+    for bf in (False, True):
+        case = gen.make_case(40, 50, 3, seed=1, c_bf16=bf, ldc=53)
+        import dataclasses
+        k0 = dataclasses.replace(case, K=0)
+        dev = P.DeviceCase(k0)
+        g = handles[(False, bf)]
+        dev.run(g, variant)
+        vals, bits = dev.result()
+        assert np.all(bits == 0), "K == 0 must give +0 everywhere"
+        assert g.last_kernel_id() == 900
+        for (M, N) in [(0, 50), (40, 0), (0, 0)]:
+            e = dataclasses.replace(case, M=M, N=N)
+            d2 = P.DeviceCase(e)
+            d2.run(g, variant)
+            d2.result()                      # guards intact, nothing written
+            assert g.last_kernel_id() == -1
+
+
+# ------------------------------------------------------------------ closed forms and invariants on the GPU
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_NAMES)
+def test_rank_one_closed_form_and_identity(handles, variant):
+    rng = np.random.default_rng(5)
+    vals8 = np.array([1.0, 1.125, 1.25, 1.375, 1.5, 1.625, 1.75, 1.875])
+    for (M, N, K) in [(130, 270, 999), (16, 300, 8192)]:
+        u = rng.choice(vals8, M) * rng.choice([-1, 1], M) * np.exp2(rng.integers(-3, 4, M))
+        v = rng.choice(vals8, N) * rng.choice([-1, 1], N) * np.exp2(rng.integers(-3, 4, N))
+        for col in (False, True):
+            A = gen.f32_to_bf16_bits(np.repeat(u[:, None], K, axis=1).astype(np.float32))
+            Bl = gen.f32_to_bf16_bits(np.repeat(v[None, :], K, axis=0).astype(np.float32))
+            Bs = np.ascontiguousarray(Bl.T) if col else Bl
+            case = gen.GemmCase("rank1", M, N, K, K, Bs.shape[1], N, col, False, A, Bs)
+            dev = P.DeviceCase(case)
+            dev.run(handles[(col, False)], variant)
+            got, _ = dev.result()
+            assert np.array_equal(got.astype(np.float64), K * np.outer(u, v)), "C_ij = K u_i v_j must be exact"
+    # identity: C = B exactly, bf16 output round-trips the bits
+    n = 200
+    B = gen.draw((n, 333), "normal", 3, 1)
+    I = gen.f32_to_bf16_bits(np.eye(n, dtype=np.float32))
+    case = gen.GemmCase("identity", n, 333, n, n, 333, 333, False, True, I, B)
+    dev = P.DeviceCase(case)
+    dev.run(handles[(False, True)], variant)
+    _, bits = dev.result()
+    assert np.array_equal(bits, B)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_NAMES)
+def test_deterministic_and_bf16_is_rounded_fp32(handles, variant):
+    import dataclasses
+    for name in ("c2", "c5"):
+        case = gen.make_config(name, 3)
+        dev = P.DeviceCase(case)
+        dev.run(handles[(case.b_col_major, False)], variant)
+        v1, b1 = dev.result()
+        dev.run(handles[(case.b_col_major, False)], variant)
+        v2, b2 = dev.result()
+        assert np.array_equal(b1, b2), "two runs differ"
+        cb = dataclasses.replace(case, c_bf16=True)
+        devb = P.DeviceCase(cb)
+        devb.run(handles[(case.b_col_major, True)], variant)
+        _, bb = devb.result()
+        assert np.array_equal(bb, gen.f32_to_bf16_bits(v1)), "bf16 C must be RNE of the fp32 C"
+
+
+# ------------------------------------------------------------------ no fallback: each rung runs its own kernel
+def test_each_variant_reports_its_own_kernel(handles, kb):
+    aligned = gen.make_config("c1", 1)
+    ragged = gen.make_config("c2", 1)
+    padded = gen.make_config("c2pad", 1)
+    g = handles[(False, False)]
+    expect = {("c1", 0): 0, ("c1", 1): 100, ("c1", 2): 207, ("c1", 3): 300,
+              ("c2", 0): 0, ("c2", 1): 100, ("c2", 2): 200, ("c2", 3): 301,
+              ("c2pad", 2): 207, ("c2pad", 3): 300}
+    for case in (aligned, ragged, padded):
+        dev = P.DeviceCase(case)
+        for v in VARIANTS:
+            dev.run(g, v)
+            code, dev_id = g.device_status()
+            assert code == 0 and dev_id == g.last_kernel_id()
+            if v == 4:
+                assert 400 <= dev_id < 408
+                assert (dev_id & 1) == (1 if case.name == "c2" else 0)   # generic producer only when unaligned
+            else:
+                want = expect.get((case.name, v))
+                if want is not None:
+                    assert dev_id == want, (case.name, v, dev_id)
+    skinny = P.DeviceCase(gen.make_config("c5", 1))
+    skinny.run(g, 4)
+    assert g.last_kernel_id() & 4, "the skinny shape must take the split-K path"
+
+
+def test_error_codes(handles, kb):
+    g = handles[(False, False)]
+    case = gen.make_case(64, 64, 64, seed=1)
+    dev = P.DeviceCase(case)
+    a, b, c = dev.a.ptr, dev.b.ptr, dev.c.ptr
+    run = lambda *args: g.run_raw(*args)
+    assert run(a, b, c, 64, 64, 64, 64, 64, 64, 5) == kb.KLINEAGE_ERR_BAD_VARIANT
+    assert run(a, b, c, 64, 64, 64, 64, 64, 64, -1) == kb.KLINEAGE_ERR_BAD_VARIANT
+    assert run(a, b, c, 64, 64, 64, 63, 64, 64, 0) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert run(a, b, c, 64, 64, 64, 64, 63, 64, 1) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert run(a, b, c, 64, 64, 64, 64, 64, 63, 2) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert run(None, b, c, 64, 64, 64, 64, 64, 64, 3) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert run(a, b, None, 64, 64, 64, 64, 64, 64, 4) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert run(a, b, a, 64, 64, 64, 64, 64, 64, 4) == kb.KLINEAGE_ERR_INVALID_ARG     # C aliases A
+    assert run(a, b, c, -1, 64, 64, 64, 64, 64, 0) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert run(a, b, c + 2, 64, 64, 64, 64, 64, 64, 0) == kb.KLINEAGE_ERR_INVALID_ARG  # fp32 C needs 4-byte alignment
+    with pytest.raises(kb.KlineageError):
+        kb.klineage_gemm_create(0, 7, 0)
+    with pytest.raises(kb.KlineageError):
+        kb.klineage_gemm_create(999, 0, 0)
+    dev.run(g, 4)
+    dev.result()
