@@ -1,0 +1,371 @@
+#!/usr/bin/env python
+"""Benchmark of the bf16 GEMM lineage on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-extras]
+
+A "step" is one pass of the hot path: one C <- A.B at the headline workload
+(8192^3, row-major bf16 A and B, fp32 accumulation, bf16 C - the compute-bound
+configuration) through the top lineage rung (tcgen05), called through the C ABI.
+Inputs are seeded synthetic data already resident in HBM; A+B+C (384 MiB) exceed
+the L2, so no flush is needed between iterations.  One JSON line is printed by
+rank 0.  With N > 1 every rank runs an independent GEMM (weak scaling, no
+data-path collective); timing is the max over ranks of CUDA-event time.
+
+`--impl reference` times the CPU oracle (plain fp64 triple loop) on a bounded
+row slab of the same workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+METRIC = "bf16 GEMM TFLOP/s per lineage rung and % of B200 BF16 peak (or HBM GB/s)"
+WORKLOAD = "c4: M=N=K=8192, row-major A and B, N(0,1/sqrt(K)) bf16, fp32 accumulate, bf16 C"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one tcgen05-rung launch at 8192^3
+# (ncu capture summarised in profiles/); None until a capture exists.
+R4_C4_DRAM_TRAFFIC_BYTES = None
+VARIANT_NAMES = ["naive", "tiled", "vectorized", "pipelined", "tcgen05"]
+
+
+def load_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            d = json.loads(p.read_text())
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ---------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.004)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------- reference arm (CPU oracle)
+def oracle_sample_seconds(case, rows: int, repeat: int = 1):
+    """Seconds the oracle needs for the first `rows` rows of C (C only, all host cores)."""
+    import numpy as np
+    from oracle import gemm_oracle as orc
+    A_sub = np.ascontiguousarray(case.A[:rows])
+    best = None
+    for _ in range(repeat):
+        t0 = time.perf_counter()
+        orc.gemm(rows, case.N, case.K, A_sub, case.lda, case.B, case.ldb, case.b_col_major, want_S=False)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return best
+
+
+def cpu_baseline(case, budget_s: float = 12.0):
+    """Times the oracle, as it stands, on a bounded row slab sized for ~budget_s of CPU work."""
+    from oracle import gemm_oracle as orc
+    probe_rows = min(case.M, 16)
+    t_probe = oracle_sample_seconds(case, probe_rows)
+    rows = int(max(probe_rows, min(case.M, budget_s / max(t_probe, 1e-6) * probe_rows)))
+    rows = max(16, (rows // 16) * 16) if case.M >= 16 else case.M
+    t = oracle_sample_seconds(case, rows)
+    flops = 2.0 * rows * case.N * case.K
+    return {"value": flops / t / 1e12, "unit": "TFLOP/s", "cores": orc.host_threads(), "kind": "oracle",
+            "sample": f"first {rows} of {case.M} rows of C at the full N={case.N}, K={case.K} "
+                      f"(fp64 triple loop, {t:.2f} s)", "seconds": t, "rows": rows}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_2605_28213_b200 import inputs as gen
+    from oracle import gemm_oracle as orc
+    case = gen.make_config("c4", 1)
+    # one step = a slab sized so that warmup + steps stay within a few minutes
+    t_probe = oracle_sample_seconds(case, 16)
+    total_steps = max(1, args.steps + args.warmup)
+    per_step_budget = min(10.0, 150.0 / total_steps)
+    rows = int(max(16, min(case.M, per_step_budget / max(t_probe, 1e-6) * 16)) // 16 * 16)
+    for _ in range(args.warmup):
+        oracle_sample_seconds(case, rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_sample_seconds(case, rows)
+    dt = (time.perf_counter() - t0) / max(1, args.steps)
+    value = 2.0 * rows * case.N * case.K / dt / 1e12
+    sample = f"each step = first {rows} of {case.M} rows of C at the full N and K (fp64 triple loop)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": orc.host_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ---------------------------------------------------------------------------- GPU arm
+class DeviceProblem:
+    """A configuration resident in HBM plus its handle."""
+
+    def __init__(self, case, kb, torch, device):
+        self.case, self.torch = case, torch
+        self.A = torch.from_numpy(case.A.view("int16")).to(device)
+        self.B = torch.from_numpy(case.B.view("int16")).to(device)
+        self.C = torch.empty((case.M, case.ldc), dtype=torch.int16 if case.c_bf16 else torch.float32, device=device)
+        self.gemm = kb.Gemm(device.index, b_col_major=case.b_col_major, c_bf16=case.c_bf16)
+
+    def run(self, variant, B=None):
+        c = self.case
+        self.gemm.run(self.A, self.B if B is None else B, self.C, c.M, c.N, c.K, c.lda, c.ldb, c.ldc, variant)
+
+    def time(self, variant, reps, warmup, flush=None, rotate=None):
+        """Median and min milliseconds of single launches (events around each launch)."""
+        torch = self.torch
+        for i in range(warmup):
+            self.run(variant, None if not rotate else rotate[i % len(rotate)])
+        torch.cuda.synchronize()
+        times = []
+        for i in range(reps):
+            if flush is not None:
+                flush.fill_(i)                      # evict L2 outside the timed interval
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            self.run(variant, None if not rotate else rotate[i % len(rotate)])
+            e1.record()
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1))
+        return statistics.median(times), min(times)
+
+
+def smoke_check(prob, variant):
+    """Sampled parity of the timed configuration against the oracle before any number is reported."""
+    import numpy as np
+    from oracle import gemm_oracle as orc
+    from paper_2605_28213_b200 import inputs as gen
+    c = prob.case
+    rows = np.array(sorted({(r * 977 + 13) % c.M for r in range(8)}))
+    C_ref, S = orc.gemm(len(rows), c.N, c.K, np.ascontiguousarray(c.A[rows]), c.lda, c.B, c.ldb, c.b_col_major)
+    prob.run(variant)
+    prob.torch.cuda.synchronize()
+    got = prob.C[rows.tolist()][:, :c.N].cpu().numpy()
+    vals = gen.bf16_bits_to_f32(got.view(np.uint16)).astype(np.float64) if c.c_bf16 else got.astype(np.float64)
+    bound = orc.bound_bf16(c.K, S, C_ref) if c.c_bf16 else orc.bound_f32(c.K, S)
+    return bool(np.all(np.abs(vals - C_ref) <= bound))
+
+
+def run_gpu(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2605_28213_b200 import binding as kb
+    from paper_2605_28213_b200 import inputs as gen
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    peaks, peak_kind = load_peaks()
+
+    case = gen.make_config("c4", 1 + rank)
+    prob = DeviceProblem(case, kb, torch, device)
+    V = kb.KLINEAGE_TCGEN05
+    parity_ok = smoke_check(prob, V) if rank == 0 else True
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        prob.run(V)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        e0.record()
+        for _ in range(args.steps):
+            prob.run(V)
+        e1.record()
+        barrier()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    code, kid = prob.gemm.device_status()
+    ms_per_step = ms / args.steps
+    tflops = case.flops * world / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end: pinned host buffers, H2D of A and B, GEMM, D2H of C, every step
+    hA = torch.from_numpy(case.A.view("int16")).pin_memory()
+    hB = torch.from_numpy(case.B.view("int16")).pin_memory()
+    hC = torch.empty((case.M, case.ldc), dtype=torch.int16).pin_memory()
+    e2e_steps = max(2, min(args.steps, 5))
+
+    def e2e_step():
+        prob.A.copy_(hA, non_blocking=True)
+        prob.B.copy_(hB, non_blocking=True)
+        prob.run(V)
+        hC.copy_(prob.C, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_s], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = {"value": case.flops * world / e2e_s / 1e12, "unit": "TFLOP/s",
+           "h2d_bytes_per_step": int(hA.numel() * 2 + hB.numel() * 2), "d2h_bytes_per_step": int(hC.numel() * 2),
+           "steps": e2e_steps}
+
+    line = {
+        "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 inputs, fp32 accumulate (tcgen05.mma kind::f16), bf16 C",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "variant": "tcgen05 (rung 4)", "parallelism": f"{world} independent GEMMs",
+                   "l2": "A+B+C = 384 MiB exceed the 126 MB L2; no flush between iterations"},
+        "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": args.steps,
+        "parity_checked": parity_ok, "device_status": code, "kernel_id": kid,
+    }
+    per_gpu = tflops / world
+    line["roofline"] = {"bound": "tensor", "achieved": per_gpu, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                        "frac": per_gpu / peaks["bf16_tflops"], "traffic": R4_C4_DRAM_TRAFFIC_BYTES,
+                        "peak_source": f"{peak_kind} (burst cuBLAS bf16)",
+                        "frac_of_sustained": per_gpu / peaks["bf16_tflops_sustained"],
+                        "frac_of_nominal_2250": per_gpu / 2250.0, "kernel": "r4_tcgen05_kernel",
+                        "flops_per_launch": case.flops}
+
+    if rank == 0 and world == 1 and not args.no_extras:
+        line["lineage"] = lineage_table(prob, kb, gen, torch, device, peaks)
+        line["cpu_baseline"] = cpu_baseline(case)
+    if world > 1:
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    return 0 if (parity_ok and code == 0) else 1
+
+
+def lineage_table(prob_c4, kb, gen, torch, device, peaks):
+    """Per-rung throughput at 8192^3 and 4096^3, and the HBM-bound skinny shape for every rung."""
+    out = {}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    reps = {0: (1, 2), 1: (2, 5), 2: (2, 5), 3: (2, 5), 4: (5, 30)}          # (warmup, reps)
+    c4 = prob_c4.case
+    rows = {}
+    for v in range(5):
+        w, r = reps[v]
+        med, mn = prob_c4.time(v, r, w)
+        rows[VARIANT_NAMES[v]] = {"ms_median": med, "ms_min": mn, "tflops": c4.flops / (med * 1e-3) / 1e12,
+                                  "frac_bf16_peak": c4.flops / (med * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                  "kernel_id": prob_c4.gemm.last_kernel_id()}
+    out["c4_8192^3"] = rows
+
+    c3 = gen.make_config("c3", 1)
+    p3 = DeviceProblem(c3, kb, torch, device)
+    rows = {}
+    for v in range(5):
+        w, r = reps[v]
+        med, mn = p3.time(v, r * 2, w, flush=flush)
+        rows[VARIANT_NAMES[v]] = {"ms_median": med, "ms_min": mn, "tflops": c3.flops / (med * 1e-3) / 1e12,
+                                  "frac_bf16_peak": c3.flops / (med * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                  "kernel_id": p3.gemm.last_kernel_id()}
+    out["c3_4096^3_Bcol"] = rows
+    del p3
+
+    c5 = gen.make_config("c5", 1)
+    p5 = DeviceProblem(c5, kb, torch, device)
+    rot = [p5.B] + [p5.B.clone() for _ in range(3)]          # distinct weight buffers: no warm-L2 replay
+    rows = {}
+    for v in range(5):
+        w, r = reps[v]
+        med, mn = p5.time(v, r * 4, w + 2, flush=flush, rotate=rot)
+        gbs = c5.algorithmic_bytes / (med * 1e-3) / 1e9
+        rows[VARIANT_NAMES[v]] = {"us_median": med * 1e3, "us_min": mn * 1e3, "gbs": gbs,
+                                  "frac_hbm": gbs / peaks["hbm_gbs"], "tflops": c5.flops / (med * 1e-3) / 1e12,
+                                  "kernel_id": p5.gemm.last_kernel_id()}
+    out["c5_16x8192x8192"] = rows
+    out["note"] = ("single launches timed with CUDA events after a 256 MiB L2 flush (c3, c5; c5 also rotates 4 weight "
+                   "buffers); c4 operands exceed L2")
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="klineage", choices=["klineage", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the per-rung table and the CPU baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

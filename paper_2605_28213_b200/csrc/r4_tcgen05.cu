@@ -1,4 +1,522 @@
+// Rung 4 - the expert kernel K_n of the lineage: "warp_specialize" plus matrix
+// intrinsics (paper, Table 1; Introduction: "matrix intrinsics require
+// compatible tile shapes, layouts, and hardware support").  On sm_100a the
+// intrinsic is tcgen05.mma with the accumulator in tensor memory (TMEM); the
+// table's wgmma does not exist on this architecture.
+//
+// One persistent CTA per SM walks a static schedule of work units
+// (128 x 256 output tile, optional K split).  Warp roles:
+//   warp 0      TMA producer: per k-block (64 deep) loads the A box and the B
+//               box(es) into a 4-stage shared-memory ring, 128-byte swizzled
+//   warp 1      MMA issuer: owns TMEM (512 columns = two 128x256 fp32
+//               accumulators); one lane issues 4 tcgen05.mma (K = 16 each) per
+//               k-block and commits to the stage's "empty" barrier; after the
+//               last k-block commits to the accumulator's "full" barrier
+//   warps 2..5  epilogue: tcgen05.ld the accumulator (each warp its 32 TMEM
+//               lanes), round to bf16 if asked, stage 32-row x 128-byte blocks
+//               in swizzled shared memory, then TMA-store them (aligned C) or
+//               copy them out with coalesced masked stores (any C); the double
+//               buffered accumulator lets this overlap the next tile's MMAs
+//   warps 6..9  only when A or B breaks TMA's alignment rules: generic-proxy
+//               producers that gather the operands with masked loads into the
+//               same swizzled layout and fence them towards the async proxy
+// Split-K (few tiles, long K - the skinny decode shape): each unit writes an
+// fp32 partial tile to the workspace; the last unit to arrive per 32-row block
+// adds the partials in split order (deterministic) and writes C.
+//
+// Every barrier wait is bounded; on expiry the CTA records an error, stops
+// issuing work, lets its copies drain, frees TMEM and returns.
 #include "common.cuh"
+#include "ptx.cuh"
+#include <cstring>
+
 namespace klin {
-cudaError_t launch_r4_tcgen05(const GemmArgs&, RunContext&, cudaStream_t, int*) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int kABytes = BM * BK * 2;              // 16 KiB
+constexpr int kBBytes = BN * BK * 2;              // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytes;    // 48 KiB
+constexpr int kEpiBufBytes = 32 * 128;            // one 32-row x 128-byte staging block
+constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;   // 4 warps x 2 buffers
+constexpr int kBarBytes = 256;
+constexpr int kSmemBytes = 1024 + STAGES * kStageBytes + kEpiBytes + kBarBytes;
+constexpr int kTmemCols = 512;
+constexpr int kThreadsTma = 6 * 32, kThreadsGeneric = 10 * 32;
+constexpr int kProducerThreads = 128;
+
+struct R4Params {
+    int tiles_m, tiles_n;
+    int splits, kb_per_split, nkb;
+    int epi_tma;            // 1: TMA-store epilogue, 0: coalesced masked stores
+    int kid;
+    float* ws;              // split-K partials [split][M][ldw]
+    int64_t ldw;
+    unsigned* counters;     // [tile * 4 + row block], zero between launches
+    uint32_t idesc;
+    uint32_t b_desc_hi, b_desc_lbo, b_kstep;   // B operand descriptor pieces (depend on the layout of B)
+};
+
+// 64-bit shared-memory matrix descriptor: start address, leading / stride byte
+// offsets (all >> 4), descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    const uint32_t lo = ((smem_addr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+    const uint32_t hi = ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
+    return (static_cast<uint64_t>(hi) << 32) | lo;
 }
+
+// 8 consecutive bf16 starting at p, `valid` of them in range, as one 16-byte chunk.
+__device__ __forceinline__ uint4 gather8(const uint16_t* p, int valid)
+{
+    if (valid >= 8 && (reinterpret_cast<uintptr_t>(p) & 15) == 0) return __ldg(reinterpret_cast<const uint4*>(p));
+    uint16_t v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = (e < valid) ? __ldg(p + e) : uint16_t(0);
+    uint4 r;
+    r.x = v[0] | (uint32_t(v[1]) << 16);
+    r.y = v[2] | (uint32_t(v[3]) << 16);
+    r.z = v[4] | (uint32_t(v[5]) << 16);
+    r.w = v[6] | (uint32_t(v[7]) << 16);
+    return r;
+}
+
+template <bool BCOL, bool GENERIC>
+__global__ void __launch_bounds__(GENERIC ? kThreadsGeneric : kThreadsTma, 1)
+r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  const __grid_constant__ CUtensorMap map_c, R4Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* epi_smem = smem + STAGES * kStageBytes;
+    uint64_t* full = reinterpret_cast<uint64_t*>(epi_smem + kEpiBytes);
+    uint64_t* empty = full + STAGES;
+    uint64_t* acc_full = empty + STAGES;
+    uint64_t* acc_empty = acc_full + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile uint32_t* abort_flag = tmem_slot + 1;   // [0] raised on give-up, [1] stays 0
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (blockIdx.x == 0 && threadIdx.x == 0) g.status[1] = p.kid;
+
+    if (warp == 0 && lane == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(&full[s], GENERIC ? kProducerThreads : 1);
+            ptx::mbar_init(&empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(&acc_full[b], 1);
+            ptx::mbar_init(&acc_empty[b], 4);
+        }
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;
+        ptx::fence_barrier_init();
+        if (!GENERIC) {
+            ptx::prefetch_tensormap(&map_a);
+            ptx::prefetch_tensormap(&map_b);
+        }
+        if (p.epi_tma) ptx::prefetch_tensormap(&map_c);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(tmem_slot, kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int64_t total_units = static_cast<int64_t>(p.tiles_m) * p.tiles_n * p.splits;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (!GENERIC && lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+                int tm, tn;
+                raster_tile(u / p.splits, p.tiles_m, p.tiles_n, tm, tn);
+                const int split = static_cast<int>(u % p.splits);
+                const int kb0 = split * p.kb_per_split, kb1 = min(p.nkb, kb0 + p.kb_per_split);
+                const int m0 = tm * BM, n0 = tn * BN;
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
+                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x400u | s);
+                        abort_flag[0] = 1;
+                        ok = false;
+                        break;
+                    }
+                    uint8_t* sa = smem + s * kStageBytes;
+                    uint8_t* sb = sa + kABytes;
+                    ptx::mbar_arrive_expect_tx(&full[s], kStageBytes);
+                    ptx::tma_load_2d(sa, &map_a, kb * BK, m0, &full[s]);
+                    if (BCOL) {
+                        ptx::tma_load_2d(sb, &map_b, kb * BK, n0, &full[s]);
+                    } else {
+#pragma unroll
+                        for (int cb = 0; cb < BN / 64; ++cb)
+                            ptx::tma_load_2d(sb + cb * (64 * BK * 2), &map_b, n0 + cb * 64, kb * BK, &full[s]);
+                    }
+                }
+            }
+            // Drain: every load issued must have landed before shared memory is released.
+            const uint32_t first = it > STAGES ? it - STAGES : 0;
+            for (uint32_t j = first; j < it; ++j) ptx::mbar_wait(&full[j % STAGES], (j / STAGES) & 1, abort_flag + 1);
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t it = 0, t = 0;
+            bool ok = true;
+            for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++t) {
+                const int split = static_cast<int>(u % p.splits);
+                const int kb0 = split * p.kb_per_split, kb1 = min(p.nkb, kb0 + p.kb_per_split);
+                const uint32_t buf = t & 1;
+                if (!ptx::mbar_wait(&acc_empty[buf], ((t >> 1) & 1) ^ 1, abort_flag)) {
+                    report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x410u | buf);
+                    abort_flag[0] = 1;
+                    break;
+                }
+                ptx::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!ptx::mbar_wait(&full[s], (it / STAGES) & 1, abort_flag)) {
+                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x420u | s);
+                        abort_flag[0] = 1;
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t sa = ptx::smem_u32(smem + s * kStageBytes);
+                    const uint32_t sb = sa + kABytes;
+                    const uint64_t a_desc = make_desc(sa, 16, 1024);
+                    const uint64_t b_desc = (static_cast<uint64_t>(p.b_desc_hi) << 32) |
+                                            (((sb >> 4) & 0x3FFFu) | (p.b_desc_lbo << 16));
+#pragma unroll
+                    for (int k4 = 0; k4 < BK / 16; ++k4) {
+                        // K-major operand: +32 bytes per 16 k inside the 128-byte swizzle row.
+                        ptx::umma_f16(d_tmem, a_desc + static_cast<uint64_t>(k4 * 2),
+                                      b_desc + static_cast<uint64_t>(k4 * p.b_kstep), p.idesc,
+                                      (kb > kb0 || k4 > 0) ? 1u : 0u);
+                    }
+                    ptx::umma_commit(&empty[s]);
+                }
+                if (ok) ptx::umma_commit(&acc_full[buf]);
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------------------ epilogue
+        const int q = warp & 3;                              // TMEM lane quarter this warp may read
+        uint8_t* stg = epi_smem + (warp - 2) * 2 * kEpiBufBytes;
+        uint32_t t = 0;
+        uint32_t nstaged = 0;                                // staging blocks written so far (buffer = parity)
+        bool ok = true;
+        for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++t) {
+            int tm, tn;
+            const int64_t tile = u / p.splits;
+            raster_tile(tile, p.tiles_m, p.tiles_n, tm, tn);
+            const int split = static_cast<int>(u % p.splits);
+            const int m0 = tm * BM, n0 = tn * BN;
+            const uint32_t buf = t & 1;
+            if (!ptx::mbar_wait(&acc_full[buf], (t >> 1) & 1, abort_flag)) {
+                if (lane == 0) report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x430u | buf);
+                abort_flag[0] = 1;
+                ok = false;
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            const int row0 = m0 + q * 32;
+            if (row0 < g.M) {
+                const bool partial = p.splits > 1;
+                const bool out_bf16 = g.c_bf16 && !partial;
+                const bool use_tma = p.epi_tma && !partial;
+                const int cpc = out_bf16 ? 64 : 32;           // columns per 128-byte staging row
+                float* dst_f = partial ? p.ws + static_cast<int64_t>(split) * g.M * p.ldw : static_cast<float*>(g.C);
+                uint16_t* dst_h = static_cast<uint16_t*>(g.C);
+                const int64_t ld = partial ? p.ldw : g.ldc;
+                const int rows = min(32, g.M - row0);
+                for (int c = 0; c * cpc < BN; ++c) {
+                    const int col0 = n0 + c * cpc;
+                    if (col0 >= g.N) break;
+                    uint32_t v[32], w[32];
+                    const uint32_t taddr = tmem_base + buf * BN + c * cpc + (static_cast<uint32_t>(q * 32) << 16);
+                    ptx::tmem_ld_32x32b_x32(taddr, v);
+                    if (out_bf16) {
+                        uint32_t v2[32];
+                        ptx::tmem_ld_32x32b_x32(taddr + 32, v2);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            w[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+                            w[16 + i] = pack_bf16x2(__uint_as_float(v2[2 * i]), __uint_as_float(v2[2 * i + 1]));
+                        }
+                    } else {
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) w[i] = v[i];
+                    }
+                    uint8_t* b = stg + (nstaged++ & 1) * kEpiBufBytes;
+                    if (use_tma) {
+                        if (lane == 0) ptx::tma_store_wait_read<1>();   // the store that last read this buffer
+                        __syncwarp();
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<uint4*>(b + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                            make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                    if (use_tma) {
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            ptx::tma_store_2d(&map_c, col0, row0, b);
+                            ptx::tma_store_commit();
+                        }
+                    } else {
+                        __syncwarp();
+                        // lane l owns 32-bit word l of every staged row: coalesced 128-byte rows.
+                        for (int rr = 0; rr < rows; ++rr) {
+                            const uint32_t word =
+                                *reinterpret_cast<const uint32_t*>(b + rr * 128 + (((lane >> 2) ^ (rr & 7)) << 4) +
+                                                                   (lane & 3) * 4);
+                            const int64_t row = row0 + rr;
+                            if (out_bf16) {
+                                const int col = col0 + 2 * lane;
+                                uint16_t* d = dst_h + row * ld + col;
+                                if (col + 1 < g.N && (reinterpret_cast<uintptr_t>(d) & 3) == 0) {
+                                    *reinterpret_cast<uint32_t*>(d) = word;
+                                } else {
+                                    if (col < g.N) d[0] = static_cast<uint16_t>(word & 0xFFFFu);
+                                    if (col + 1 < g.N) d[1] = static_cast<uint16_t>(word >> 16);
+                                }
+                            } else {
+                                const int col = col0 + lane;
+                                if (col < g.N) dst_f[row * ld + col] = __uint_as_float(word);
+                            }
+                        }
+                        __syncwarp();
+                    }
+                }
+            }
+            // TMEM reads of this tile are done: hand the accumulator back.
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
+
+            if (p.splits > 1 && row0 < g.M) {
+                // Arrival per (tile, 32-row block); the last arriver adds the partials in split order.
+                __threadfence();
+                __syncwarp();
+                unsigned old = 0;
+                unsigned* cnt = p.counters + tile * 4 + q;
+                if (lane == 0) old = atomicAdd(cnt, 1u);
+                old = __shfl_sync(0xFFFFFFFFu, old, 0);
+                if (old == static_cast<unsigned>(p.splits - 1)) {
+                    __threadfence();
+                    const int rows = min(32, g.M - row0);
+                    const int64_t plane = static_cast<int64_t>(g.M) * p.ldw;
+                    for (int rr = 0; rr < rows; ++rr) {
+                        const int64_t row = row0 + rr;
+                        for (int cc = lane * 4; cc < BN; cc += 128) {
+                            const int col = n0 + cc;
+                            if (col >= g.N) break;
+                            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                            const float* src = p.ws + row * p.ldw + col;   // ldw % 4 == 0: 16-byte aligned
+                            for (int sp = 0; sp < p.splits; ++sp) {
+                                const float4 x = __ldcg(reinterpret_cast<const float4*>(src + sp * plane));
+                                acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+                            }
+                            const float o[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                if (col + e < g.N) store_c(g.C, g.c_bf16, row * g.ldc + col + e, o[e]);
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) *cnt = 0;   // ready for the next launch
+                }
+            }
+        }
+        if (p.epi_tma && lane == 0) ptx::tma_store_wait_all<0>();
+    } else if (GENERIC) {
+        // ------------------------------------------------------------ generic-proxy producers
+        const int pt = threadIdx.x - 6 * 32;                 // 0..127
+        uint32_t it = 0;
+        bool ok = true;
+        for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+            int tm, tn;
+            raster_tile(u / p.splits, p.tiles_m, p.tiles_n, tm, tn);
+            const int split = static_cast<int>(u % p.splits);
+            const int kb0 = split * p.kb_per_split, kb1 = min(p.nkb, kb0 + p.kb_per_split);
+            const int m0 = tm * BM, n0 = tn * BN;
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                const int s = it % STAGES;
+                if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
+                    if (pt == 0) report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x440u | s);
+                    abort_flag[0] = 1;
+                    ok = false;
+                    break;
+                }
+                uint8_t* sa = smem + s * kStageBytes;
+                uint8_t* sb = sa + kABytes;
+                const int k0 = kb * BK;
+                // A: 128 rows x 8 chunks of 8 k (K-major, 128-byte swizzle)
+#pragma unroll 4
+                for (int c = pt; c < BM * 8; c += kProducerThreads) {
+                    const int r = c >> 3, kc = c & 7;
+                    const int64_t gm = m0 + r;
+                    const int gk = k0 + kc * 8;
+                    const int valid = (gm < g.M) ? min(8, max(0, g.K - gk)) : 0;
+                    *reinterpret_cast<uint4*>(sa + r * 128 + ((kc ^ (r & 7)) << 4)) =
+                        gather8(g.A + gm * g.lda + gk, valid);
+                }
+                if (BCOL) {
+                    // B column-major: 256 n-rows x 8 chunks of 8 k (K-major)
+#pragma unroll 4
+                    for (int c = pt; c < BN * 8; c += kProducerThreads) {
+                        const int n = c >> 3, kc = c & 7;
+                        const int64_t gn = n0 + n;
+                        const int gk = k0 + kc * 8;
+                        const int valid = (gn < g.N) ? min(8, max(0, g.K - gk)) : 0;
+                        *reinterpret_cast<uint4*>(sb + n * 128 + ((kc ^ (n & 7)) << 4)) =
+                            gather8(g.B + gn * g.ldb + gk, valid);
+                    }
+                } else {
+                    // B row-major: 64 k-rows x 32 chunks of 8 n (MN-major): 64-column blocks of
+                    // 64 k-rows x 128 bytes, chunk index swizzled with the k-row.
+#pragma unroll 4
+                    for (int c = pt; c < BK * 32; c += kProducerThreads) {
+                        const int k = c >> 5, nc = c & 31;
+                        const int64_t gk = k0 + k;
+                        const int gn = n0 + nc * 8;
+                        const int valid = (gk < g.K) ? min(8, max(0, g.N - gn)) : 0;
+                        *reinterpret_cast<uint4*>(sb + (nc >> 3) * (64 * BK * 2) + k * 128 + (((nc & 7) ^ (k & 7)) << 4)) =
+                            gather8(g.B + gk * g.ldb + gn, valid);
+                    }
+                }
+                ptx::fence_proxy_async_smem();
+                ptx::mbar_arrive(&full[s]);
+            }
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+bool tma_ok(const void* base, int64_t ld_elems, int elt)
+{
+    return reinterpret_cast<uintptr_t>(base) % 16 == 0 && (ld_elems * elt) % 16 == 0 &&
+           ld_elems * elt < (int64_t(1) << 40);
+}
+
+// Chooses the number of K splits: minimise waves x (k-blocks per unit + fixed
+// per-unit cost), within the workspace and counter budgets.
+int choose_splits(int64_t tiles, int nkb, int sm, int64_t M, int64_t ldw, const RunContext& ctx)
+{
+    if (tiles * 2 > sm || nkb < 8 || tiles * 4 > ctx.n_tile_counters) return 1;
+    const int kFixed = 6;
+    int best = 1;
+    int64_t best_cost = ((tiles + sm - 1) / sm) * (nkb + kFixed);
+    for (int s = 2; s <= 32 && s * 4 <= nkb; ++s) {
+        const int per = (nkb + s - 1) / s;
+        const int eff = (nkb + per - 1) / per;        // splits that actually get work
+        if (eff != s) continue;
+        if (static_cast<size_t>(s) * M * ldw * sizeof(float) > ctx.workspace_bytes) break;
+        const int64_t cost = ((tiles * s + sm - 1) / sm) * (per + kFixed);
+        if (cost < best_cost) {
+            best_cost = cost;
+            best = s;
+        }
+    }
+    return best;
+}
+
+template <bool BCOL, bool GENERIC>
+cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
+                   const R4Params& p, unsigned grid, int device, cudaStream_t stream)
+{
+    auto kern = r4_tcgen05_kernel<BCOL, GENERIC>;
+    static bool attr_set[64] = {};
+    if (device < 0 || device >= 64 || !attr_set[device]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        if (device >= 0 && device < 64) attr_set[device] = true;
+    }
+    kern<<<grid, GENERIC ? kThreadsGeneric : kThreadsTma, kSmemBytes, stream>>>(g, ma, mb, mc, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
+{
+    if (ctx.max_smem_optin < kSmemBytes) return cudaErrorInvalidConfiguration;
+    const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN;
+    const int64_t tiles = tiles_m * tiles_n;
+    if (tiles > 0x3FFFFFFFll) return cudaErrorInvalidConfiguration;
+
+    R4Params p;
+    memset(&p, 0, sizeof p);
+    p.tiles_m = static_cast<int>(tiles_m);
+    p.tiles_n = static_cast<int>(tiles_n);
+    p.nkb = (g.K + BK - 1) / BK;
+    p.ldw = (static_cast<int64_t>(g.N) + 3) & ~int64_t(3);
+    p.splits = choose_splits(tiles, p.nkb, ctx.sm_count, g.M, p.ldw, ctx);
+    p.kb_per_split = (p.nkb + p.splits - 1) / p.splits;
+    p.ws = static_cast<float*>(ctx.workspace);
+    p.counters = ctx.tile_counters;
+
+    const bool generic = !(ctx.encode_tiled && tma_ok(g.A, g.lda, 2) && tma_ok(g.B, g.ldb, 2));
+    const int celt = g.c_bf16 ? 2 : 4;
+    p.epi_tma = (p.splits == 1 && ctx.encode_tiled && tma_ok(g.C, g.ldc, celt)) ? 1 : 0;
+
+    // Instruction descriptor: fp32 accumulator, bf16 A and B, A K-major, B K-major
+    // (column-major B) or MN-major (row-major B), N = 256, M = 128.
+    p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((g.b_col ? 0u : 1u) << 16) | (static_cast<uint32_t>(BN >> 3) << 17) |
+              (static_cast<uint32_t>(BM >> 4) << 24);
+    // Shared-memory descriptor of B (version 1, 128-byte swizzle):
+    //   K-major : 8-row groups 1024 bytes apart; +32 bytes per 16 k
+    //   MN-major: 64-column blocks 8192 bytes apart (leading offset), 8-k groups 1024 bytes
+    //             apart (stride offset); +2048 bytes per 16 k
+    p.b_desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    p.b_desc_lbo = g.b_col ? 1u : ((64u * BK * 2u) >> 4);
+    p.b_kstep = g.b_col ? 2u : (2048u >> 4);
+
+    CUtensorMap ma, mb, mc;
+    memset(&ma, 0, sizeof ma);
+    memset(&mb, 0, sizeof mb);
+    memset(&mc, 0, sizeof mc);
+    bool ok = true;
+    if (!generic) {
+        ok = encode_map_2d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, BM,
+                           CU_TENSOR_MAP_SWIZZLE_128B);
+        if (g.b_col)
+            ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, BN,
+                                     CU_TENSOR_MAP_SWIZZLE_128B);
+        else
+            ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, g.ldb * 2, 64, BK,
+                                     CU_TENSOR_MAP_SWIZZLE_128B);
+    }
+    if (p.epi_tma)
+        ok = ok && encode_map_2d(ctx, &mc, g.c_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                                 g.C, g.N, g.M, g.ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!ok) return cudaErrorInvalidValue;
+
+    p.kid = kIdTcgen05 + (generic ? 1 : 0) + (p.epi_tma ? 0 : 2) + (p.splits > 1 ? 4 : 0);
+    *kernel_id = p.kid;
+    const int64_t units = tiles * p.splits;
+    const unsigned grid = static_cast<unsigned>(units < ctx.sm_count ? units : ctx.sm_count);
+    if (g.b_col)
+        return generic ? launch<true, true>(g, ma, mb, mc, p, grid, ctx.device, stream)
+                       : launch<true, false>(g, ma, mb, mc, p, grid, ctx.device, stream);
+    return generic ? launch<false, true>(g, ma, mb, mc, p, grid, ctx.device, stream)
+                   : launch<false, false>(g, ma, mb, mc, p, grid, ctx.device, stream);
+}
+
+}  // namespace klin
