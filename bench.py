@@ -158,6 +158,23 @@ def run_reference(args):
     return 0
 
 
+# ---------------------------------------------------------------------------- multi-rank helpers
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """MAX all-reduce of a per-rank scalar (elapsed time); identity for one rank."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(flops_per_rank: float, world: int, seconds_per_step: float) -> float:
+    """Aggregate over all ranks: every rank does flops_per_rank of work per step (weak scaling)."""
+    return flops_per_rank * world / seconds_per_step / 1e12
+
+
 # ---------------------------------------------------------------------------- GPU arm
 class DeviceProblem:
     """A configuration resident in HBM plus its handle."""
@@ -246,14 +263,10 @@ def run_gpu(args):
             prob.run(V)
         e1.record()
         barrier()
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), world, device)
     code, kid = prob.gemm.device_status()
     ms_per_step = ms / args.steps
-    tflops = case.flops * world / (ms_per_step * 1e-3) / 1e12
+    tflops = whole_job_tflops(case.flops, world, ms_per_step * 1e-3)
 
     # ---- end to end: pinned host buffers, H2D of A and B, GEMM, D2H of C, every step
     hA = torch.from_numpy(case.A.view("int16")).pin_memory()
@@ -273,12 +286,8 @@ def run_gpu(args):
     for _ in range(e2e_steps):
         e2e_step()
     barrier()
-    e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_s], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e = {"value": case.flops * world / e2e_s / 1e12, "unit": "TFLOP/s",
+    e2e_s = max_over_ranks((time.perf_counter() - t0) / e2e_steps, world, device)
+    e2e = {"value": whole_job_tflops(case.flops, world, e2e_s), "unit": "TFLOP/s",
            "h2d_bytes_per_step": int(hA.numel() * 2 + hB.numel() * 2), "d2h_bytes_per_step": int(hC.numel() * 2),
            "steps": e2e_steps}
 
