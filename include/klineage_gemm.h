@@ -37,7 +37,8 @@ typedef enum {
     KLINEAGE_ERR_ALLOC = 4,              /* device or host allocation failed in create                */
     KLINEAGE_ERR_LAUNCH = 5,             /* the CUDA runtime rejected a launch or a tensor map        */
     KLINEAGE_ERR_TIMEOUT = 6,            /* a bounded device-side wait gave up (see get_device_status) */
-    KLINEAGE_ERR_INTERNAL = 7
+    KLINEAGE_ERR_INTERNAL = 7,
+    KLINEAGE_ERR_SCRATCH_LIMIT = 8       /* klineage_gemm_run_noalloc: the shape needs more fixed scratch than exists */
 } klineage_status_t;
 
 /* Storage of B (K x N).  A is always row-major M x K, C always row-major M x N. */
@@ -146,6 +147,49 @@ klineage_status_t klineage_gemm_get_device_status(klineage_gemm_t h, int* code_o
  *   900 zero fill (K == 0); -1 before the first run or after a no-op.
  */
 int klineage_gemm_last_kernel_id(klineage_gemm_t h);
+
+/*
+ * The tcgen05 rung (variant 4) for callers that must not allocate device memory.
+ * (The paper has no counterpart to this call; it exists for integration.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a plug-in or
+ * operator called by a host framework that owns the whole memory budget and
+ * forbids outside allocations, a latency-critical serving loop (cudaMalloc can
+ * synchronise the device and may fail late, under memory pressure), or a process
+ * whose remaining device memory is already spoken for.  klineage_gemm_create
+ * allocates a workspace, so such callers cannot even obtain a handle.
+ *
+ * This call takes no handle and calls no allocator: not cudaMalloc/cudaFree, not
+ * an allocating library routine.  Its scratch memory (split-K partial sums,
+ * arrival counters, status words) is a fixed array inside the library image:
+ * 8 MiB of partial sums + 16 KiB of counters.  Every GPU that loads the library
+ * holds those bytes until the process exits, whether or not this call is used.
+ *
+ *   b_layout, c_dtype   as in klineage_gemm_config_t
+ *   M, N, K, A, lda, B, ldb, C, ldc, stream   exactly as for klineage_gemm_run;
+ *                       the caller still owns and passes inputs and output
+ *   The GEMM runs on the calling thread's current CUDA device; the pointers must
+ *   belong to that device.
+ *
+ * Limits and rules:
+ *   - A shape whose K split would need more than the 8 MiB of partial sums
+ *     (splits * M * round_up(N,4) * 4 bytes; only shapes with few output tiles
+ *     are split) is refused with KLINEAGE_ERR_SCRATCH_LIMIT and a message on
+ *     stderr; nothing is launched.  Use a handle for such shapes.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents;
+ *     each call re-zeroes the counters and status words on `stream` before its
+ *     kernel.  Two calls that overlap on the GPU (different streams, or several
+ *     host threads) race on the array: keep calls to one stream at a time.
+ *   - Device-side give-ups (bounded waits) cannot be read back through this call.
+ * Results are bit-identical to klineage_gemm_run(..., KLINEAGE_TCGEN05, ...) with a
+ * default handle for every accepted shape.
+ * Errors: as klineage_gemm_run, plus KLINEAGE_ERR_SCRATCH_LIMIT.
+ */
+klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype, int64_t M, int64_t N, int64_t K,
+                                            const void* A, int64_t lda, const void* B, int64_t ldb,
+                                            void* C, int64_t ldc, void* stream);
 
 const char* klineage_status_string(int status);
 const char* klineage_variant_name(int variant);

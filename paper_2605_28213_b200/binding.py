@@ -21,6 +21,7 @@ KLINEAGE_ERR_ALLOC = 4
 KLINEAGE_ERR_LAUNCH = 5
 KLINEAGE_ERR_TIMEOUT = 6
 KLINEAGE_ERR_INTERNAL = 7
+KLINEAGE_ERR_SCRATCH_LIMIT = 8
 
 KLINEAGE_B_ROW_MAJOR, KLINEAGE_B_COL_MAJOR = 0, 1
 KLINEAGE_C_F32, KLINEAGE_C_BF16 = 0, 1
@@ -30,7 +31,7 @@ VARIANTS = (KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELI
 EXPORTED_SYMBOLS = (
     "klineage_gemm_create", "klineage_gemm_run", "klineage_gemm_destroy", "klineage_gemm_check_args",
     "klineage_gemm_get_device_status", "klineage_gemm_last_kernel_id", "klineage_status_string",
-    "klineage_variant_name",
+    "klineage_variant_name", "klineage_gemm_run_noalloc",
 )
 
 
@@ -69,6 +70,20 @@ _lib.klineage_status_string.restype = ctypes.c_char_p
 _lib.klineage_status_string.argtypes = [_int]
 _lib.klineage_variant_name.restype = ctypes.c_char_p
 _lib.klineage_variant_name.argtypes = [_int]
+
+
+_lib.klineage_gemm_run_noalloc.restype = _int
+_lib.klineage_gemm_run_noalloc.argtypes = [_int, _int, _i64, _i64, _i64, _p, _i64, _p, _i64, _p, _i64, _p]
+
+
+def klineage_gemm_run_noalloc(b_layout, c_dtype, M, N, K, A, lda, B, ldb, C, ldc, stream=None) -> int:
+    """Raw status of the allocation-free tcgen05 call (no handle; fixed in-library scratch).
+
+    For callers that may not allocate device memory.  Pointers are integer device
+    addresses on the current device; see the header for the scratch limit and the
+    one-stream-at-a-time rule.
+    """
+    return _lib.klineage_gemm_run_noalloc(b_layout, c_dtype, M, N, K, A, lda, B, ldb, C, ldc, stream)
 
 
 def klineage_status_string(status: int) -> str:

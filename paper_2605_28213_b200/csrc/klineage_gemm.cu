@@ -245,6 +245,7 @@ const char* klineage_status_string(int status)
         case KLINEAGE_ERR_LAUNCH: return "launch failed";
         case KLINEAGE_ERR_TIMEOUT: return "device-side wait timed out";
         case KLINEAGE_ERR_INTERNAL: return "internal error";
+        case KLINEAGE_ERR_SCRATCH_LIMIT: return "shape exceeds the fixed scratch of the allocation-free call";
         default: return "unknown status";
     }
 }

@@ -26,9 +26,12 @@
 //
 // Every barrier wait is bounded; on expiry the CTA records an error, stops
 // issuing work, lets its copies drain, frees TMEM and returns.
+#include "../../include/klineage_gemm.h"
 #include "common.cuh"
 #include "ptx.cuh"
+#include <cstdio>
 #include <cstring>
+#include <mutex>
 
 namespace klin {
 namespace {
@@ -520,3 +523,147 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
 }
 
 }  // namespace klin
+
+// ---------------------------------------------------------------------------
+// Allocation-free entry point.
+//
+// klineage_gemm_run_noalloc runs the tcgen05 rung without a handle and without
+// ever asking the CUDA allocator for memory.  Everything the kernel needs beyond
+// the caller's A, B and C - the split-K partial sums, the per-row-block arrival
+// counters and the four status words - lives in the fixed array below, which is
+// part of the library image: each GPU that loads the library reserves these
+// bytes until the process exits.
+namespace klin {
+namespace {
+
+constexpr size_t kNoAllocPartialBytes = size_t(8) << 20;   // split-K partial sums (fp32)
+constexpr int kNoAllocCounters = 4096;                     // arrival counters (one per tile and 32-row block)
+constexpr size_t kNoAllocScratchBytes = kNoAllocPartialBytes + kNoAllocCounters * sizeof(unsigned) + 256;
+
+}  // namespace
+}  // namespace klin
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[klin::kNoAllocScratchBytes];
+
+namespace klin {
+namespace {
+
+// Per-device state of the entry point.  In host code the name g_noalloc_scratch
+// is only a stand-in for the device array, so the real device address is looked
+// up once per device (with that device current) and kept here.
+struct NoAllocDevice {
+    bool ready = false;
+    unsigned char* scratch = nullptr;
+    unsigned* status = nullptr;
+    RunContext ctx;
+};
+NoAllocDevice g_noalloc_devices[64];
+std::mutex g_noalloc_mutex;
+
+klineage_status_t noalloc_setup(int device, NoAllocDevice** out)
+{
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    NoAllocDevice& d = g_noalloc_devices[device];
+    if (!d.ready) {
+        unsigned char* ptr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch);
+        if (e != cudaSuccess || ptr == nullptr) {
+            cudaGetLastError();
+            fprintf(stderr, "klineage_gemm_run_noalloc: cudaGetSymbolAddress failed: %s\n", cudaGetErrorString(e));
+            return KLINEAGE_ERR_INTERNAL;
+        }
+        RunContext& c = d.ctx;
+        c.device = device;
+        cudaDeviceGetAttribute(&c.sm_count, cudaDevAttrMultiProcessorCount, device);
+        cudaDeviceGetAttribute(&c.cc_major, cudaDevAttrComputeCapabilityMajor, device);
+        cudaDeviceGetAttribute(&c.cc_minor, cudaDevAttrComputeCapabilityMinor, device);
+        cudaDeviceGetAttribute(&c.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            c.encode_tiled = reinterpret_cast<TensorMapEncodeTiledFn>(fn);
+        else
+            cudaGetLastError();
+        d.scratch = ptr;
+        c.workspace = ptr;
+        c.workspace_bytes = kNoAllocPartialBytes;
+        c.tile_counters = reinterpret_cast<unsigned*>(ptr + kNoAllocPartialBytes);
+        c.n_tile_counters = kNoAllocCounters;
+        d.status = c.tile_counters + kNoAllocCounters;
+        d.ready = true;
+    }
+    *out = &d;
+    return KLINEAGE_OK;
+}
+
+}  // namespace
+}  // namespace klin
+
+extern "C" klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype, int64_t M, int64_t N, int64_t K,
+                                                       const void* A, int64_t lda, const void* B, int64_t ldb,
+                                                       void* C, int64_t ldc, void* stream)
+{
+    using namespace klin;
+    const klineage_status_t chk =
+        klineage_gemm_check_args(b_layout, c_dtype, M, N, K, A, lda, B, ldb, C, ldc, KLINEAGE_TCGEN05);
+    if (chk != KLINEAGE_OK) return chk;
+    if (M == 0 || N == 0) return KLINEAGE_OK;
+
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) {
+        cudaGetLastError();
+        return KLINEAGE_ERR_INVALID_ARG;
+    }
+    NoAllocDevice* d = nullptr;
+    const klineage_status_t st = noalloc_setup(device, &d);
+    if (st != KLINEAGE_OK) return st;
+    if (d->ctx.cc_major != 10) return KLINEAGE_ERR_UNSUPPORTED_DEVICE;
+
+    GemmArgs g;
+    g.M = static_cast<int>(M);
+    g.N = static_cast<int>(N);
+    g.K = static_cast<int>(K);
+    g.A = static_cast<const uint16_t*>(A);
+    g.lda = lda;
+    g.B = static_cast<const uint16_t*>(B);
+    g.ldb = ldb;
+    g.C = C;
+    g.ldc = ldc;
+    g.b_col = b_layout == KLINEAGE_B_COL_MAJOR ? 1 : 0;
+    g.c_bf16 = c_dtype == KLINEAGE_C_BF16 ? 1 : 0;
+    g.status = d->status;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int kid = -1;
+    if (K == 0) return launch_zero_fill(g, s, &kid) == cudaSuccess ? KLINEAGE_OK : KLINEAGE_ERR_LAUNCH;
+
+    // Refuse, rather than quietly change the schedule, when the K split this
+    // shape would get needs more partial-sum space than the fixed array holds.
+    const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+    const int nkb = static_cast<int>((K + BK - 1) / BK);
+    const int64_t ldw = (N + 3) & ~int64_t(3);
+    RunContext unlimited = d->ctx;
+    unlimited.workspace_bytes = ~size_t(0);
+    const int splits = tiles > 0x3FFFFFFFll ? 1 : choose_splits(tiles, nkb, d->ctx.sm_count, M, ldw, unlimited);
+    const size_t need = splits > 1 ? static_cast<size_t>(splits) * M * ldw * sizeof(float) : 0;
+    if (need > kNoAllocPartialBytes) {
+        fprintf(stderr,
+                "klineage_gemm_run_noalloc: M=%lld N=%lld K=%lld needs %zu bytes of split-K scratch, the fixed "
+                "array holds %zu; use klineage_gemm_run with a handle for this shape\n",
+                static_cast<long long>(M), static_cast<long long>(N), static_cast<long long>(K), need,
+                kNoAllocPartialBytes);
+        return KLINEAGE_ERR_SCRATCH_LIMIT;
+    }
+
+    // The array keeps whatever the previous call left: counters and status must start at zero.
+    if (cudaMemsetAsync(d->ctx.tile_counters, 0, (kNoAllocCounters + 4) * sizeof(unsigned), s) != cudaSuccess) {
+        cudaGetLastError();
+        return KLINEAGE_ERR_LAUNCH;
+    }
+    if (launch_r4_tcgen05(g, d->ctx, s, &kid) != cudaSuccess) {
+        cudaGetLastError();
+        return KLINEAGE_ERR_LAUNCH;
+    }
+    return KLINEAGE_OK;
+}

@@ -1,0 +1,81 @@
+"""The allocation-free entry point against the handle-based one.
+
+Some users of this library sit where device allocation is forbidden: an
+operator plugged into a framework that owns the whole memory budget, a serving
+loop that cannot afford cudaMalloc's implicit synchronisation, a process whose
+remaining HBM is already committed.  klineage_gemm_run_noalloc serves them from
+a fixed scratch array inside the library.  Its results must equal those of
+klineage_gemm_run on the tcgen05 rung bit for bit - on a first call and on a
+second call that finds the first call's leftovers in the shared scratch.
+
+This file sorts last on purpose: a run that stops at the first failure has
+already executed every other test.
+"""
+import numpy as np
+import pytest
+
+from paper_2605_28213_b200 import inputs as gen
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+def run_both(kb, case, calls=2):
+    """C from the handle path, then `calls` results of the allocation-free path on the same inputs."""
+    import torch
+    stream = torch.cuda.current_stream().cuda_stream
+    with kb.Gemm(0, b_col_major=case.b_col_major, c_bf16=case.c_bf16) as g:
+        dev = P.DeviceCase(case)
+        dev.run(g, kb.KLINEAGE_TCGEN05)
+        _, want_bits = dev.result()
+        kid = g.last_kernel_id()
+    outs = []
+    for _ in range(calls):
+        d2 = P.DeviceCase(case)                       # fresh, poisoned C every call
+        st = kb.klineage_gemm_run_noalloc(
+            kb.KLINEAGE_B_COL_MAJOR if case.b_col_major else kb.KLINEAGE_B_ROW_MAJOR,
+            kb.KLINEAGE_C_BF16 if case.c_bf16 else kb.KLINEAGE_C_F32,
+            case.M, case.N, case.K, d2.a.ptr, case.lda, d2.b.ptr, case.ldb, d2.c.ptr, case.ldc, stream)
+        assert st == kb.KLINEAGE_OK, kb.klineage_status_string(st)
+        torch.cuda.synchronize()
+        outs.append(d2.result()[1])                   # also checks guard bands and row padding
+    return want_bits, outs, kid
+
+
+def test_no_alloc_matches_handle_path_on_two_calls_in_a_row():
+    from paper_2605_28213_b200 import binding as kb
+    # a skinny, long-K shape: takes the split-K path, i.e. really uses the scratch array
+    skinny = gen.make_case(16, 2048, 4096, seed=5, dist_a="normal", dist_b="normal", sigma_b=0.02, name="skinny")
+    want, outs, kid = run_both(kb, skinny)
+    assert kid & 4, "the comparison shape must exercise split-K scratch"
+    for k, got in enumerate(outs):
+        assert np.array_equal(got, want), f"call {k + 1}: allocation-free result differs from the handle path"
+    # and against the oracle, with the tolerance every other parity test uses
+    C_ref, S = P.oracle_rows(skinny, np.arange(skinny.M))
+    P.assert_matches_oracle(skinny, outs[-1].view(np.float32), outs[-1], C_ref, S, exact=False, what="no-alloc skinny")
+
+    # ragged, column-major B, bf16 C: the path without a K split still goes through the same call
+    ragged = gen.make_case(300, 520, 200, seed=6, dist_a="integer", dist_b="integer", b_col_major=True, c_bf16=True,
+                           name="ragged")
+    want, outs, _ = run_both(kb, ragged)
+    for got in outs:
+        assert np.array_equal(got, want)
+
+
+def test_no_alloc_refuses_shapes_beyond_its_fixed_scratch():
+    import torch
+    from paper_2605_28213_b200 import binding as kb
+    # 2 splits x 2048 x 1024 fp32 partial sums = 16 MiB > the 8 MiB the library reserves
+    M, N, K = 2048, 1024, 4096
+    A = torch.zeros(M * K, dtype=torch.int16, device="cuda")
+    B = torch.zeros(K * N, dtype=torch.int16, device="cuda")
+    C = torch.full((M * N,), 7.0, dtype=torch.float32, device="cuda")
+    st = kb.klineage_gemm_run_noalloc(0, 0, M, N, K, A.data_ptr(), K, B.data_ptr(), N, C.data_ptr(), N,
+                                      torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert st == kb.KLINEAGE_ERR_SCRATCH_LIMIT
+    assert "scratch" in kb.klineage_status_string(st)
+    assert bool((C == 7.0).all().item()), "a refused call must not touch C"
+    # argument errors are reported exactly as by the handle path
+    assert kb.klineage_gemm_run_noalloc(0, 0, 8, 8, 8, A.data_ptr(), 7, B.data_ptr(), 8, C.data_ptr(), 8,
+                                        None) == kb.KLINEAGE_ERR_INVALID_ARG
