@@ -29,7 +29,14 @@ ROOT = Path(__file__).resolve().parent
 sys.path.insert(0, str(ROOT))
 
 METRIC = "bf16 GEMM TFLOP/s per lineage rung and % of B200 BF16 peak (or HBM GB/s)"
-WORKLOAD = "c4: M=N=K=8192, row-major A and B, N(0,1/sqrt(K)) bf16, fp32 accumulate, bf16 C"
+WORKLOADS = {
+    "c1": "c1: M=N=K=256, row-major, U[-1,1) bf16, fp32 C",
+    "c2": "c2: M=1000 N=1001 K=999, row-major, unaligned leading dimensions, U[-1,1) bf16, fp32 C",
+    "c3": "c3: M=N=K=4096, B column-major, N(0,1) bf16, fp32 accumulate, bf16 C",
+    "c4": "c4: M=N=K=8192, row-major A and B, N(0,1/sqrt(K)) bf16, fp32 accumulate, bf16 C",
+    "c5": "c5: M=16 N=8192 K=8192, row-major, N(0,1) x N(0,0.02) bf16, fp32 C (weight streaming)",
+}
+WORKLOAD = WORKLOADS["c4"]
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one tcgen05-rung launch at 8192^3
 # (ncu capture summarised in profiles/); None until a capture exists.
@@ -243,24 +250,28 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=device)
     peaks, peak_kind = load_peaks()
 
-    case = gen.make_config("c4", 1 + rank)
+    case = gen.make_config(args.workload, 1 + rank)
     prob = DeviceProblem(case, kb, torch, device)
-    V = kb.KLINEAGE_TCGEN05
+    V = args.variant
     parity_ok = smoke_check(prob, V) if rank == 0 else True
+    # A workload whose operands fit the L2 (c5: 129 MiB of weights) rotates over distinct
+    # B buffers so that no iteration replays a warm L2.
+    small = case.algorithmic_bytes < (300 << 20)
+    rot = [prob.B] + ([prob.B.clone() for _ in range(3)] if small else [])
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(3, args.warmup)):
-        prob.run(V)
+    for i in range(max(3, args.warmup)):
+        prob.run(V, rot[i % len(rot)])
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local) as clocks:
         e0.record()
-        for _ in range(args.steps):
-            prob.run(V)
+        for i in range(args.steps):
+            prob.run(V, rot[i % len(rot)])
         e1.record()
         barrier()
     ms = max_over_ranks(e0.elapsed_time(e1), world, device)
@@ -271,7 +282,7 @@ def run_gpu(args):
     # ---- end to end: pinned host buffers, H2D of A and B, GEMM, D2H of C, every step
     hA = torch.from_numpy(case.A.view("int16")).pin_memory()
     hB = torch.from_numpy(case.B.view("int16")).pin_memory()
-    hC = torch.empty((case.M, case.ldc), dtype=torch.int16).pin_memory()
+    hC = torch.empty_like(prob.C, device="cpu").pin_memory()
     e2e_steps = max(2, min(args.steps, 5))
 
     def e2e_step():
@@ -288,7 +299,7 @@ def run_gpu(args):
     barrier()
     e2e_s = max_over_ranks((time.perf_counter() - t0) / e2e_steps, world, device)
     e2e = {"value": whole_job_tflops(case.flops, world, e2e_s), "unit": "TFLOP/s",
-           "h2d_bytes_per_step": int(hA.numel() * 2 + hB.numel() * 2), "d2h_bytes_per_step": int(hC.numel() * 2),
+           "h2d_bytes_per_step": int(hA.numel() * 2 + hB.numel() * 2), "d2h_bytes_per_step": int(hC.numel() * hC.element_size()),
            "steps": e2e_steps}
 
     line = {
@@ -296,20 +307,30 @@ def run_gpu(args):
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16 inputs, fp32 accumulate (tcgen05.mma kind::f16), bf16 C",
         "data": "synthetic",
-        "config": {"workload": WORKLOAD, "variant": "tcgen05 (rung 4)", "parallelism": f"{world} independent GEMMs",
-                   "l2": "A+B+C = 384 MiB exceed the 126 MB L2; no flush between iterations"},
+        "config": {"workload": WORKLOADS[args.workload], "variant": f"{VARIANT_NAMES[V]} (rung {V})",
+                   "parallelism": f"{world} independent GEMMs",
+                   "l2": (f"{len(rot)} distinct B buffers rotated ({len(rot) * case.B.nbytes >> 20} MiB > L2); no flush"
+                          if small else "A+B+C = 384 MiB exceed the 126 MB L2; no flush between iterations")},
         "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": args.steps,
         "parity_checked": parity_ok, "device_status": code, "kernel_id": kid,
     }
     per_gpu = tflops / world
-    line["roofline"] = {"bound": "tensor", "achieved": per_gpu, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                        "frac": per_gpu / peaks["bf16_tflops"], "traffic": R4_C4_DRAM_TRAFFIC_BYTES,
-                        "peak_source": f"{peak_kind} (burst cuBLAS bf16)",
-                        "frac_of_sustained": per_gpu / peaks["bf16_tflops_sustained"],
-                        "frac_of_nominal_2250": per_gpu / 2250.0, "kernel": "r4_tcgen05_kernel",
-                        "flops_per_launch": case.flops}
+    if args.workload == "c5":
+        gbs = case.algorithmic_bytes / (ms_per_step * 1e-3) / 1e9
+        line["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                            "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                            "peak_source": f"{peak_kind} (copy bandwidth)", "frac_of_nominal_8000": gbs / 8000.0,
+                            "algorithmic_bytes_per_launch": case.algorithmic_bytes}
+    else:
+        line["roofline"] = {"bound": "tensor", "achieved": per_gpu, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                            "frac": per_gpu / peaks["bf16_tflops"],
+                            "traffic": R4_C4_DRAM_TRAFFIC_BYTES if (args.workload, V) == ("c4", 4) else None,
+                            "peak_source": f"{peak_kind} (burst cuBLAS bf16)",
+                            "frac_of_sustained": per_gpu / peaks["bf16_tflops_sustained"],
+                            "frac_of_nominal_2250": per_gpu / 2250.0, "kernel": "r4_tcgen05_kernel",
+                            "flops_per_launch": case.flops}
 
-    if rank == 0 and world == 1 and not args.no_extras:
+    if rank == 0 and world == 1 and not args.no_extras and (args.workload, V) == ("c4", 4):
         line["lineage"] = lineage_table(prob, kb, gen, torch, device, peaks)
         line["cpu_baseline"] = cpu_baseline(case)
     if world > 1:
@@ -370,6 +391,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="klineage", choices=["klineage", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the per-rung table and the CPU baseline")
+    ap.add_argument("--workload", default="c4", choices=sorted(WORKLOADS),
+                    help="configuration to time (default: the headline 8192^3; others are for profiling)")
+    ap.add_argument("--variant", type=int, default=4, choices=range(5), help="lineage rung to time (default 4)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -39,7 +39,7 @@ enum KernelId : int {
     kIdTiled = 100,
     kIdVectorized = 200,      // + 1 (A vector loads) + 2 (B vector loads) + 4 (C vector stores)
     kIdPipelined = 300,       // + 1 when the producer-thread path replaces TMA
-    kIdTcgen05 = 400,         // + 1 generic-proxy producer, + 2 direct epilogue, + 4 split-K
+    kIdTcgen05 = 400,         // + 1 generic-proxy producer, + 2 direct epilogue, + 4 split-K, + 8 skinny (swapped operands)
     kIdZeroFill = 900,
 };
 

@@ -20,9 +20,19 @@
 //   warps 6..9  only when A or B breaks TMA's alignment rules: generic-proxy
 //               producers that gather the operands with masked loads into the
 //               same swizzled layout and fence them towards the async proxy
-// Split-K (few tiles, long K - the skinny decode shape): each unit writes an
-// fp32 partial tile to the workspace; the last unit to arrive per 32-row block
-// adds the partials in split order (deterministic) and writes C.
+// Split-K (few tiles, long K): each unit writes an fp32 partial tile to the
+// workspace; the last unit to arrive per block of the tile adds the partials in
+// split order (deterministic) and writes C.
+// Skinny mode (M <= 64, the decode-like weight-streaming shape): the operands
+// swap roles - the 256 weight columns of the tile become the 2 x 128 MMA rows
+// (TMEM lanes) and the few activation rows become the MMA's N (16..64).  All
+// four epilogue warps then hold useful lanes, a lane's registers run over m,
+// and stores are coalesced along n straight from registers.  With M <= 32 the
+// K splits of a tile form a thread-block cluster and reduce through distributed
+// shared memory instead of the global workspace: every CTA sends each 32-column
+// block of its partial tile to the block's owner CTA (plain st.shared::cluster),
+// one cluster barrier, and each owner adds the partials in rank order and stores
+// its columns of C.  No atomics, no round trip through L2.
 //
 // Every barrier wait is bounded; on expiry the CTA records an error, stops
 // issuing work, lets its copies drain, frees TMEM and returns.
@@ -58,6 +68,9 @@ struct R4Params {
     unsigned* counters;     // [tile * 4 + row block], zero between launches
     uint32_t idesc;
     uint32_t b_desc_hi, b_desc_lbo, b_kstep;   // B operand descriptor pieces (depend on the layout of B)
+    int n_mma;              // skinny mode: M rounded up to 16 = the MMA's N
+    uint32_t stage_tx;      // bytes one stage's TMA loads deliver (A box + B boxes)
+    int cluster;            // 1: the splits of a tile are one cluster and reduce through DSMEM
 };
 
 // 64-bit shared-memory matrix descriptor: start address, leading / stride byte
@@ -84,7 +97,7 @@ __device__ __forceinline__ uint4 gather8(const uint16_t* p, int valid)
     return r;
 }
 
-template <bool BCOL, bool GENERIC>
+template <bool BCOL, bool GENERIC, bool SWAP>
 __global__ void __launch_bounds__(GENERIC ? kThreadsGeneric : kThreadsTma, 1)
 r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ CUtensorMap map_c, R4Params p)
@@ -101,6 +114,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (blockIdx.x == 0 && threadIdx.x == 0) g.status[1] = p.kid;
+    // Cluster mode: no CTA may touch a peer's shared memory before that peer runs.
+    if (SWAP && p.cluster) ptx::cluster_arrive_release();
 
     if (warp == 0 && lane == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -128,6 +143,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    if (SWAP && p.cluster) ptx::cluster_wait_acquire();
 
     const int64_t total_units = static_cast<int64_t>(p.tiles_m) * p.tiles_n * p.splits;
 
@@ -152,7 +168,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     }
                     uint8_t* sa = smem + s * kStageBytes;
                     uint8_t* sb = sa + kABytes;
-                    ptx::mbar_arrive_expect_tx(&full[s], kStageBytes);
+                    ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
                     ptx::tma_load_2d(sa, &map_a, kb * BK, m0, &full[s]);
                     if (BCOL) {
                         ptx::tma_load_2d(sb, &map_b, kb * BK, n0, &full[s]);
@@ -200,9 +216,18 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
 #pragma unroll
                     for (int k4 = 0; k4 < BK / 16; ++k4) {
                         // K-major operand: +32 bytes per 16 k inside the 128-byte swizzle row.
-                        ptx::umma_f16(d_tmem, a_desc + static_cast<uint64_t>(k4 * 2),
-                                      b_desc + static_cast<uint64_t>(k4 * p.b_kstep), p.idesc,
-                                      (kb > kb0 || k4 > 0) ? 1u : 0u);
+                        const uint32_t acc = (kb > kb0 || k4 > 0) ? 1u : 0u;
+                        if (SWAP) {
+                            // weights are the 128-row operand (two halves of the tile's 256 columns,
+                            // 16 KiB apart in the stage), activations the N operand
+#pragma unroll
+                            for (int h = 0; h < 2; ++h)
+                                ptx::umma_f16(d_tmem + h * 128, b_desc + static_cast<uint64_t>(h * (16384 >> 4) + k4 * p.b_kstep),
+                                              a_desc + static_cast<uint64_t>(k4 * 2), p.idesc, acc);
+                        } else {
+                            ptx::umma_f16(d_tmem, a_desc + static_cast<uint64_t>(k4 * 2),
+                                          b_desc + static_cast<uint64_t>(k4 * p.b_kstep), p.idesc, acc);
+                        }
                     }
                     ptx::umma_commit(&empty[s]);
                 }
@@ -230,6 +255,99 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 break;
             }
             ptx::tc_fence_after_sync();
+            if (SWAP) {
+                // lane = weight column n, registers = activation rows m
+                const bool partial = p.splits > 1 && !p.cluster;
+                float* dst_f = partial ? p.ws + static_cast<int64_t>(split) * g.M * p.ldw : static_cast<float*>(g.C);
+                const int64_t ld = partial ? p.ldw : g.ldc;
+                const bool out_bf16 = g.c_bf16 && !partial;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int nbase = n0 + h * 128 + q * 32;
+                    if (nbase >= g.N) continue;
+                    const int n = nbase + lane;
+                    for (int mc = 0; mc < p.n_mma; mc += 16) {
+                        uint32_t v[16];
+                        ptx::tmem_ld_32x32b_x16(tmem_base + buf * BN + h * 128 + mc + (static_cast<uint32_t>(q * 32) << 16), v);
+                        ptx::tmem_ld_wait();
+                        if (p.cluster) {
+                            // block (h, q) of the tile belongs to CTA (block % splits); this CTA's
+                            // partial goes to slot [split][block / splits][m][lane] of the owner.
+                            const int bi = h * 4 + q;
+                            const uint32_t owner = static_cast<uint32_t>(bi % p.splits);
+                            const int nblk = 8 / p.splits;
+                            float* slot = reinterpret_cast<float*>(epi_smem) +
+                                          ((split * nblk + bi / p.splits) * p.n_mma + mc) * 32 + lane;
+                            const uint32_t remote = ptx::map_to_cta(ptx::smem_u32(slot), owner);
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) ptx::st_cluster_f32(remote + j * 128, __uint_as_float(v[j]));
+                        } else if (n < g.N) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const int m = mc + j;
+                                if (m < g.M) {
+                                    if (out_bf16)
+                                        static_cast<uint16_t*>(g.C)[m * ld + n] = float_to_bf16_bits(__uint_as_float(v[j]));
+                                    else
+                                        dst_f[m * ld + n] = __uint_as_float(v[j]);
+                                }
+                            }
+                        }
+                    }
+                }
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
+
+                if (partial) {
+                    // One arrival counter per (tile, lane quarter); the last arriver sums its 2 x 32
+                    // columns over all rows, partials in split order, loads batched to hide latency.
+                    const int64_t plane = static_cast<int64_t>(g.M) * p.ldw;
+                    if (n0 + q * 32 < g.N) {
+                        __syncwarp();
+                        unsigned old = 0;
+                        unsigned* cnt = p.counters + tile * 4 + q;
+                        if (lane == 0) {
+                            __threadfence();
+                            old = atomicAdd(cnt, 1u);
+                            __threadfence();
+                        }
+                        old = __shfl_sync(0xFFFFFFFFu, old, 0);
+                        if (old == static_cast<unsigned>(p.splits - 1)) {
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                const int n = n0 + h * 128 + q * 32 + lane;
+                                if (n >= g.N) continue;
+                                for (int mb = 0; mb < g.M; mb += 16) {
+                                    float acc[16];
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+                                    for (int sp = 0; sp < p.splits; sp += 4) {
+                                        float x[4][16];
+#pragma unroll
+                                        for (int s4 = 0; s4 < 4; ++s4)
+#pragma unroll
+                                            for (int j = 0; j < 16; ++j)
+                                                x[s4][j] = (sp + s4 < p.splits && mb + j < g.M)
+                                                               ? __ldcg(p.ws + (sp + s4) * plane + (mb + j) * p.ldw + n)
+                                                               : 0.f;
+#pragma unroll
+                                        for (int s4 = 0; s4 < 4; ++s4)
+#pragma unroll
+                                            for (int j = 0; j < 16; ++j) acc[j] += x[s4][j];
+                                    }
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j)
+                                        if (mb + j < g.M) store_c(g.C, g.c_bf16, (mb + j) * g.ldc + n, acc[j]);
+                                }
+                            }
+                            __syncwarp();
+                            if (lane == 0) *cnt = 0;   // ready for the next launch
+                        }
+                    }
+                }
+                continue;
+            }
             const int row0 = m0 + q * 32;
             if (row0 < g.M) {
                 const bool partial = p.splits > 1;
@@ -340,7 +458,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     if (lane == 0) *cnt = 0;   // ready for the next launch
                 }
             }
-        }
+                }
         if (p.epi_tma && lane == 0) ptx::tma_store_wait_all<0>();
     } else if (GENERIC) {
         // ------------------------------------------------------------ generic-proxy producers
@@ -404,6 +522,30 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         }
     }
 
+    if (SWAP && p.cluster) {
+        // Every thread of every CTA of the cluster arrives; after the wait all partial
+        // blocks sent to this CTA are visible in its shared memory.
+        ptx::cluster_arrive_release();
+        ptx::cluster_wait_acquire();
+        if (warp >= 2 && warp < 6 && !abort_flag[0]) {
+            const int rank = static_cast<int>(blockIdx.x % p.splits);
+            int tm, tn;
+            raster_tile(blockIdx.x / p.splits, p.tiles_m, p.tiles_n, tm, tn);
+            const int n0 = tn * BN;
+            const int nblk = 8 / p.splits;
+            const float* slots = reinterpret_cast<const float*>(epi_smem);
+            // work items (local block, row m), dealt round-robin to the four warps
+            for (int item = warp - 2; item < nblk * g.M; item += 4) {
+                const int bl = item / g.M, m = item % g.M;
+                const int bi = bl * p.splits + rank;
+                const int n = n0 + (bi >> 2) * 128 + (bi & 3) * 32 + lane;
+                float acc = 0.f;
+                for (int src = 0; src < p.splits; ++src) acc += slots[((src * nblk + bl) * p.n_mma + m) * 32 + lane];
+                if (n < g.N) store_c(g.C, g.c_bf16, static_cast<int64_t>(m) * g.ldc + n, acc);
+            }
+        }
+    }
+
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
@@ -440,16 +582,76 @@ int choose_splits(int64_t tiles, int nkb, int sm, int64_t M, int64_t ldw, const 
     return best;
 }
 
-template <bool BCOL, bool GENERIC>
+// Skinny shapes with M <= 32: the K splits of a tile run as one thread-block cluster
+// (2, 4 or 8 CTAs) and need no workspace.  Returns 1 when splitting does not pay.
+int choose_cluster_splits(int64_t tiles, int nkb, int sm)
+{
+    if (tiles * 2 > sm || nkb < 8) return 1;
+    const int kFixed = 3;
+    int best = 1;
+    int64_t best_cost = ((tiles + sm - 1) / sm) * (nkb + kFixed);
+    for (int s = 2; s <= 8 && s * 4 <= nkb; s *= 2) {
+        const int per = (nkb + s - 1) / s;
+        if ((nkb + per - 1) / per != s) continue;
+        const int64_t cost = ((tiles * s + sm - 1) / sm) * (per + kFixed);
+        if (cost < best_cost) {
+            best_cost = cost;
+            best = s;
+        }
+    }
+    return best;
+}
+
+// How a shape is split along K: not at all, through the global workspace, or
+// through a cluster.  One function so that every caller plans the same way.
+struct SplitPlan {
+    int splits;
+    bool cluster;
+    bool swap;
+};
+SplitPlan plan_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContext& ctx)
+{
+    SplitPlan sp;
+    sp.swap = M <= 64;
+    sp.cluster = false;
+    if (sp.swap && M <= 32) {
+        const int s = choose_cluster_splits(tiles, nkb, ctx.sm_count);
+        if (s > 1) {
+            sp.splits = s;
+            sp.cluster = true;
+            return sp;
+        }
+    }
+    sp.splits = choose_splits(tiles, nkb, ctx.sm_count, M, ldw, ctx);
+    return sp;
+}
+
+template <bool BCOL, bool GENERIC, bool SWAP>
 cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
                    const R4Params& p, unsigned grid, int device, cudaStream_t stream)
 {
-    auto kern = r4_tcgen05_kernel<BCOL, GENERIC>;
+    auto kern = r4_tcgen05_kernel<BCOL, GENERIC, SWAP>;
     static bool attr_set[64] = {};
     if (device < 0 || device >= 64 || !attr_set[device]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
         if (device >= 0 && device < 64) attr_set[device] = true;
+    }
+    if (p.cluster) {
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(GENERIC ? kThreadsGeneric : kThreadsTma);
+        cfg.dynamicSmemBytes = kSmemBytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = static_cast<unsigned>(p.splits);
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, kern, g, ma, mb, mc, p);
     }
     kern<<<grid, GENERIC ? kThreadsGeneric : kThreadsTma, kSmemBytes, stream>>>(g, ma, mb, mc, p);
     return cudaGetLastError();
@@ -470,19 +672,30 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     p.tiles_n = static_cast<int>(tiles_n);
     p.nkb = (g.K + BK - 1) / BK;
     p.ldw = (static_cast<int64_t>(g.N) + 3) & ~int64_t(3);
-    p.splits = choose_splits(tiles, p.nkb, ctx.sm_count, g.M, p.ldw, ctx);
+    const SplitPlan plan = plan_split(g.M, tiles, p.nkb, p.ldw, ctx);
+    p.splits = plan.splits;
+    p.cluster = plan.cluster ? 1 : 0;
     p.kb_per_split = (p.nkb + p.splits - 1) / p.splits;
     p.ws = static_cast<float*>(ctx.workspace);
     p.counters = ctx.tile_counters;
 
     const bool generic = !(ctx.encode_tiled && tma_ok(g.A, g.lda, 2) && tma_ok(g.B, g.ldb, 2));
     const int celt = g.c_bf16 ? 2 : 4;
-    p.epi_tma = (p.splits == 1 && ctx.encode_tiled && tma_ok(g.C, g.ldc, celt)) ? 1 : 0;
+    // Skinny mode: few activation rows -> they become the MMA's N, the weights its 128 rows.
+    const bool swap = plan.swap;
+    p.n_mma = (g.M + 15) & ~15;
+    p.epi_tma = (!swap && p.splits == 1 && ctx.encode_tiled && tma_ok(g.C, g.ldc, celt)) ? 1 : 0;
 
-    // Instruction descriptor: fp32 accumulator, bf16 A and B, A K-major, B K-major
-    // (column-major B) or MN-major (row-major B), N = 256, M = 128.
-    p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((g.b_col ? 0u : 1u) << 16) | (static_cast<uint32_t>(BN >> 3) << 17) |
-              (static_cast<uint32_t>(BM >> 4) << 24);
+    // Instruction descriptor: fp32 accumulator (bits 4-5), bf16 A and B (bits 7-9, 10-12),
+    // operand majors (bit 15 A, bit 16 B; 0 = K-major, 1 = MN-major), N >> 3 (bits 17-22),
+    // M >> 4 (bits 24-28).  Row-major B is MN-major, column-major B is K-major.
+    const uint32_t w_major = g.b_col ? 0u : 1u;
+    if (swap)
+        p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (w_major << 15) | (static_cast<uint32_t>(p.n_mma >> 3) << 17) |
+                  (static_cast<uint32_t>(128 >> 4) << 24);
+    else
+        p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (w_major << 16) | (static_cast<uint32_t>(BN >> 3) << 17) |
+                  (static_cast<uint32_t>(BM >> 4) << 24);
     // Shared-memory descriptor of B (version 1, 128-byte swizzle):
     //   K-major : 8-row groups 1024 bytes apart; +32 bytes per 16 k
     //   MN-major: 64-column blocks 8192 bytes apart (leading offset), 8-k groups 1024 bytes
@@ -496,8 +709,11 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     memset(&mb, 0, sizeof mb);
     memset(&mc, 0, sizeof mc);
     bool ok = true;
+    // Skinny mode fetches only the activation rows the MMA reads (n_mma of them).
+    const uint32_t a_box_rows = swap ? static_cast<uint32_t>(p.n_mma) : BM;
+    p.stage_tx = a_box_rows * BK * 2 + kBBytes;
     if (!generic) {
-        ok = encode_map_2d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, BM,
+        ok = encode_map_2d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, a_box_rows,
                            CU_TENSOR_MAP_SWIZZLE_128B);
         if (g.b_col)
             ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, BN,
@@ -511,15 +727,20 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
                                  g.C, g.N, g.M, g.ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return cudaErrorInvalidValue;
 
-    p.kid = kIdTcgen05 + (generic ? 1 : 0) + (p.epi_tma ? 0 : 2) + (p.splits > 1 ? 4 : 0);
+    p.kid = kIdTcgen05 + (generic ? 1 : 0) + (p.epi_tma ? 0 : 2) + (p.splits > 1 ? 4 : 0) + (swap ? 8 : 0) +
+            (p.cluster ? 16 : 0);
     *kernel_id = p.kid;
     const int64_t units = tiles * p.splits;
-    const unsigned grid = static_cast<unsigned>(units < ctx.sm_count ? units : ctx.sm_count);
-    if (g.b_col)
-        return generic ? launch<true, true>(g, ma, mb, mc, p, grid, ctx.device, stream)
-                       : launch<true, false>(g, ma, mb, mc, p, grid, ctx.device, stream);
-    return generic ? launch<false, true>(g, ma, mb, mc, p, grid, ctx.device, stream)
-                   : launch<false, false>(g, ma, mb, mc, p, grid, ctx.device, stream);
+    // A cluster handles exactly one tile, so the cluster path launches every unit as a CTA.
+    const unsigned grid = static_cast<unsigned>((p.cluster || units < ctx.sm_count) ? units : ctx.sm_count);
+#define KLIN_R4_LAUNCH(BC, GE, SW) launch<BC, GE, SW>(g, ma, mb, mc, p, grid, ctx.device, stream)
+    if (swap) {
+        if (g.b_col) return generic ? KLIN_R4_LAUNCH(true, true, true) : KLIN_R4_LAUNCH(true, false, true);
+        return generic ? KLIN_R4_LAUNCH(false, true, true) : KLIN_R4_LAUNCH(false, false, true);
+    }
+    if (g.b_col) return generic ? KLIN_R4_LAUNCH(true, true, false) : KLIN_R4_LAUNCH(true, false, false);
+    return generic ? KLIN_R4_LAUNCH(false, true, false) : KLIN_R4_LAUNCH(false, false, false);
+#undef KLIN_R4_LAUNCH
 }
 
 }  // namespace klin
@@ -645,8 +866,12 @@ extern "C" klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype
     const int64_t ldw = (N + 3) & ~int64_t(3);
     RunContext unlimited = d->ctx;
     unlimited.workspace_bytes = ~size_t(0);
-    const int splits = tiles > 0x3FFFFFFFll ? 1 : choose_splits(tiles, nkb, d->ctx.sm_count, M, ldw, unlimited);
-    const size_t need = splits > 1 ? static_cast<size_t>(splits) * M * ldw * sizeof(float) : 0;
+    SplitPlan plan;
+    plan.splits = 1;
+    plan.cluster = false;
+    if (tiles <= 0x3FFFFFFFll) plan = plan_split(static_cast<int>(M), tiles, nkb, ldw, unlimited);
+    const size_t need =
+        (plan.splits > 1 && !plan.cluster) ? static_cast<size_t>(plan.splits) * M * ldw * sizeof(float) : 0;
     if (need > kNoAllocPartialBytes) {
         fprintf(stderr,
                 "klineage_gemm_run_noalloc: M=%lld N=%lld K=%lld needs %zu bytes of split-K scratch, the fixed "

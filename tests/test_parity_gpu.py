@@ -199,7 +199,7 @@ def test_each_variant_reports_its_own_kernel(handles, kb):
             code, dev_id = g.device_status()
             assert code == 0 and dev_id == g.last_kernel_id()
             if v == 4:
-                assert 400 <= dev_id < 408
+                assert 400 <= dev_id < 432
                 assert (dev_id & 1) == (1 if case.name == "c2" else 0)   # generic producer only when unaligned
             else:
                 want = expect.get((case.name, v))

@@ -44,22 +44,25 @@ def run_both(kb, case, calls=2):
 
 def test_no_alloc_matches_handle_path_on_two_calls_in_a_row():
     from paper_2605_28213_b200 import binding as kb
-    # a skinny, long-K shape: takes the split-K path, i.e. really uses the scratch array
-    skinny = gen.make_case(16, 2048, 4096, seed=5, dist_a="normal", dist_b="normal", sigma_b=0.02, name="skinny")
+    # a short-and-wide, long-K shape: split along K through the workspace, i.e. really uses the scratch array
+    skinny = gen.make_case(48, 2048, 4096, seed=5, dist_a="normal", dist_b="normal", sigma_b=0.02, name="skinny")
     want, outs, kid = run_both(kb, skinny)
-    assert kid & 4, "the comparison shape must exercise split-K scratch"
+    assert (kid & 4) and not (kid & 16), "the comparison shape must exercise split-K scratch in global memory"
     for k, got in enumerate(outs):
         assert np.array_equal(got, want), f"call {k + 1}: allocation-free result differs from the handle path"
     # and against the oracle, with the tolerance every other parity test uses
     C_ref, S = P.oracle_rows(skinny, np.arange(skinny.M))
     P.assert_matches_oracle(skinny, outs[-1].view(np.float32), outs[-1], C_ref, S, exact=False, what="no-alloc skinny")
 
-    # ragged, column-major B, bf16 C: the path without a K split still goes through the same call
-    ragged = gen.make_case(300, 520, 200, seed=6, dist_a="integer", dist_b="integer", b_col_major=True, c_bf16=True,
-                           name="ragged")
-    want, outs, _ = run_both(kb, ragged)
-    for got in outs:
-        assert np.array_equal(got, want)
+    # taller tile, split along K with the row-block reduce; and a decode-like M=16 shape (cluster reduce,
+    # no global scratch) plus a ragged column-major bf16 case without any split: same call, same bits
+    for case in (gen.make_case(200, 512, 4096, seed=7, dist_a="integer", dist_b="integer", name="tall"),
+                 gen.make_case(16, 2048, 4096, seed=8, dist_a="normal", dist_b="normal", name="decode"),
+                 gen.make_case(300, 520, 200, seed=6, dist_a="integer", dist_b="integer", b_col_major=True,
+                               c_bf16=True, name="ragged")):
+        want, outs, _ = run_both(kb, case)
+        for got in outs:
+            assert np.array_equal(got, want), case.name
 
 
 def test_no_alloc_refuses_shapes_beyond_its_fixed_scratch():
