@@ -109,6 +109,19 @@ __device__ __forceinline__ void tma_store_wait_all()
     asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// ------------------------------------------- programmatic dependent launch
+// Blocks until every grid this one depends on has completed and its memory
+// operations are visible (a no-op for a launch without the attribute).
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+// Lets the next grid in the stream start its own prologue.
+__device__ __forceinline__ void grid_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ------------------------------------------------------- thread-block cluster
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {

@@ -113,9 +113,57 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     volatile uint32_t* abort_flag = tmem_slot + 1;   // [0] raised on give-up, [1] stays 0
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (blockIdx.x == 0 && threadIdx.x == 0) g.status[1] = p.kid;
     // Cluster mode: no CTA may touch a peer's shared memory before that peer runs.
     if (SWAP && p.cluster) ptx::cluster_arrive_release();
+    const int64_t total_units = static_cast<int64_t>(p.tiles_m) * p.tiles_n * p.splits;
+
+    // TMA producer state (used by warp 0, lane 0 only): position in the static schedule.
+    struct {
+        int64_t u;
+        int kb, kb1, m0, n0;
+        uint32_t it;
+        bool live;
+    } prod = {static_cast<int64_t>(blockIdx.x), 0, 0, 0, 0, 0u, false};
+    auto prod_enter_unit = [&]() {
+        prod.live = prod.u < total_units;
+        if (!prod.live) return;
+        int tm, tn;
+        raster_tile(prod.u / p.splits, p.tiles_m, p.tiles_n, tm, tn);
+        const int split = static_cast<int>(prod.u % p.splits);
+        prod.kb = split * p.kb_per_split;
+        prod.kb1 = min(p.nkb, prod.kb + p.kb_per_split);
+        prod.m0 = tm * BM;
+        prod.n0 = tn * BN;
+    };
+    // Issues loads until `limit` k-blocks have been issued in total or the schedule ends.
+    auto produce = [&](uint32_t limit) {
+        while (prod.live && prod.it < limit) {
+            const uint32_t it = prod.it;
+            const int s = it % STAGES;
+            if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
+                report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x400u | s);
+                abort_flag[0] = 1;
+                prod.live = false;
+                break;
+            }
+            uint8_t* sa = smem + s * kStageBytes;
+            uint8_t* sb = sa + kABytes;
+            ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
+            ptx::tma_load_2d(sa, &map_a, prod.kb * BK, prod.m0, &full[s]);
+            if (BCOL) {
+                ptx::tma_load_2d(sb, &map_b, prod.kb * BK, prod.n0, &full[s]);
+            } else {
+#pragma unroll
+                for (int cb = 0; cb < BN / 64; ++cb)
+                    ptx::tma_load_2d(sb + cb * (64 * BK * 2), &map_b, prod.n0 + cb * 64, prod.kb * BK, &full[s]);
+            }
+            ++prod.it;
+            if (++prod.kb == prod.kb1) {
+                prod.u += gridDim.x;
+                prod_enter_unit();
+            }
+        }
+    };
 
     if (warp == 0 && lane == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -134,6 +182,17 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             ptx::prefetch_tensormap(&map_b);
         }
         if (p.epi_tma) ptx::prefetch_tensormap(&map_c);
+        // The launch is a programmatic dependent one: everything above (and the TMEM
+        // allocation in warp 1) may overlap the tail of the previous kernel in the stream;
+        // nothing below the wait touches global memory before that kernel has completed.
+        if (!GENERIC) prod_enter_unit();           // schedule arithmetic only
+        ptx::grid_dependency_wait();
+        if (!GENERIC) {
+            // The first ring fill needs nothing from the other warps: start it before the
+            // set-up barrier so that TMEM allocation hides behind the first loads' latency.
+            produce(STAGES);
+        }
+        if (blockIdx.x == 0) g.status[1] = p.kid;
     }
     if (warp == 1) {
         ptx::tmem_alloc(tmem_slot, kTmemCols);
@@ -143,43 +202,16 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
     if (SWAP && p.cluster) ptx::cluster_wait_acquire();
-
-    const int64_t total_units = static_cast<int64_t>(p.tiles_m) * p.tiles_n * p.splits;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (!GENERIC && lane == 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
-                int tm, tn;
-                raster_tile(u / p.splits, p.tiles_m, p.tiles_n, tm, tn);
-                const int split = static_cast<int>(u % p.splits);
-                const int kb0 = split * p.kb_per_split, kb1 = min(p.nkb, kb0 + p.kb_per_split);
-                const int m0 = tm * BM, n0 = tn * BN;
-                for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
-                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x400u | s);
-                        abort_flag[0] = 1;
-                        ok = false;
-                        break;
-                    }
-                    uint8_t* sa = smem + s * kStageBytes;
-                    uint8_t* sb = sa + kABytes;
-                    ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
-                    ptx::tma_load_2d(sa, &map_a, kb * BK, m0, &full[s]);
-                    if (BCOL) {
-                        ptx::tma_load_2d(sb, &map_b, kb * BK, n0, &full[s]);
-                    } else {
-#pragma unroll
-                        for (int cb = 0; cb < BN / 64; ++cb)
-                            ptx::tma_load_2d(sb + cb * (64 * BK * 2), &map_b, n0 + cb * 64, kb * BK, &full[s]);
-                    }
-                }
-            }
+            produce(0xFFFFFFFFu);
             // Drain: every load issued must have landed before shared memory is released.
+            const uint32_t it = prod.it;
             const uint32_t first = it > STAGES ? it - STAGES : 0;
             for (uint32_t j = first; j < it; ++j) ptx::mbar_wait(&full[j % STAGES], (j / STAGES) & 1, abort_flag + 1);
         }
@@ -534,14 +566,24 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             const int n0 = tn * BN;
             const int nblk = 8 / p.splits;
             const float* slots = reinterpret_cast<const float*>(epi_smem);
-            // work items (local block, row m), dealt round-robin to the four warps
-            for (int item = warp - 2; item < nblk * g.M; item += 4) {
-                const int bl = item / g.M, m = item % g.M;
+            // each warp takes every fourth row m of every local block, four rows per step so
+            // that their shared-memory loads are in flight together; lanes run along n
+            for (int bl = 0; bl < nblk; ++bl) {
                 const int bi = bl * p.splits + rank;
                 const int n = n0 + (bi >> 2) * 128 + (bi & 3) * 32 + lane;
-                float acc = 0.f;
-                for (int src = 0; src < p.splits; ++src) acc += slots[((src * nblk + bl) * p.n_mma + m) * 32 + lane];
-                if (n < g.N) store_c(g.C, g.c_bf16, static_cast<int64_t>(m) * g.ldc + n, acc);
+                if (n >= g.N) continue;
+                for (int mb = warp - 2; mb < g.M; mb += 16) {
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                    for (int src = 0; src < p.splits; ++src) {
+                        const float* sl = slots + ((src * nblk + bl) * p.n_mma + mb) * 32 + lane;
+#pragma unroll
+                        for (int r = 0; r < 4; ++r)
+                            if (mb + 4 * r < g.M) acc[r] += sl[4 * r * 32];
+                    }
+#pragma unroll
+                    for (int r = 0; r < 4; ++r)
+                        if (mb + 4 * r < g.M) store_c(g.C, g.c_bf16, static_cast<int64_t>(mb + 4 * r) * g.ldc + n, acc[r]);
+                }
             }
         }
     }
@@ -637,24 +679,29 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
         if (e != cudaSuccess) return e;
         if (device >= 0 && device < 64) attr_set[device] = true;
     }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(GENERIC ? kThreadsGeneric : kThreadsTma);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attrs[2];
+    unsigned na = 0;
+    // Programmatic dependent launch: the kernel's set-up may overlap the previous kernel's
+    // tail; the kernel itself waits (griddepcontrol.wait) before it touches global memory.
+    attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
     if (p.cluster) {
-        cudaLaunchConfig_t cfg;
-        memset(&cfg, 0, sizeof cfg);
-        cfg.gridDim = dim3(grid);
-        cfg.blockDim = dim3(GENERIC ? kThreadsGeneric : kThreadsTma);
-        cfg.dynamicSmemBytes = kSmemBytes;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr;
-        attr.id = cudaLaunchAttributeClusterDimension;
-        attr.val.clusterDim.x = static_cast<unsigned>(p.splits);
-        attr.val.clusterDim.y = 1;
-        attr.val.clusterDim.z = 1;
-        cfg.attrs = &attr;
-        cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, kern, g, ma, mb, mc, p);
+        attrs[na].id = cudaLaunchAttributeClusterDimension;
+        attrs[na].val.clusterDim.x = static_cast<unsigned>(p.splits);
+        attrs[na].val.clusterDim.y = 1;
+        attrs[na].val.clusterDim.z = 1;
+        ++na;
     }
-    kern<<<grid, GENERIC ? kThreadsGeneric : kThreadsTma, kSmemBytes, stream>>>(g, ma, mb, mc, p);
-    return cudaGetLastError();
+    cfg.attrs = attrs;
+    cfg.numAttrs = na;
+    return cudaLaunchKernelEx(&cfg, kern, g, ma, mb, mc, p);
 }
 
 }  // namespace
