@@ -5,7 +5,10 @@
 // 128 x 128 x 32 tiles, a ring of 4 shared-memory stages holding RAW bf16, a
 // full/empty mbarrier pair per stage with phase parity.  Loads for k-block
 // kb+3 are in flight while k-block kb is multiplied (fp32 FMA on CUDA cores,
-// bf16 -> fp32 widening when a value is read from shared memory).
+// bf16 -> fp32 widening when a value is read from shared memory).  With no
+// global loads or shared-memory stores left in the issue stream, the multiply
+// uses sm_100's packed fma.rn.f32x2 (two independent fp32 FMAs per instruction,
+// same rounding as scalar fmaf), which leaves issue slots for the widening.
 //
 //   TMA path (A, B 16-byte aligned with 16-byte-multiple row pitch): one
 //   thread issues cp.async.bulk.tensor loads that complete on the stage's
@@ -151,11 +154,11 @@ r3_pipelined_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
         }
     }
 
-    float acc[8][8];
+    float2 acc2[8][4];   // acc2[i][jp] = accumulators of columns 2*jp and 2*jp+1 of row i
 #pragma unroll
     for (int i = 0; i < 8; ++i)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+        for (int jp = 0; jp < 4; ++jp) acc2[i][jp] = make_float2(0.f, 0.f);
 
     for (int kb = 0; kb < nkb && ok; ++kb) {
         const int s = kb % STAGES;
@@ -202,27 +205,32 @@ r3_pipelined_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
                 }
 #pragma unroll
                 for (int k8 = 0; k8 < 8; ++k8) {
-                    float b[8];
+                    float2 b2[4];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) b[j] = (k8 & 1) ? bf16_hi(bw[j][k8 >> 1]) : bf16_lo(bw[j][k8 >> 1]);
+                    for (int jp = 0; jp < 4; ++jp) {
+                        b2[jp].x = (k8 & 1) ? bf16_hi(bw[2 * jp][k8 >> 1]) : bf16_lo(bw[2 * jp][k8 >> 1]);
+                        b2[jp].y = (k8 & 1) ? bf16_hi(bw[2 * jp + 1][k8 >> 1]) : bf16_lo(bw[2 * jp + 1][k8 >> 1]);
+                    }
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const float a = (k8 & 1) ? bf16_hi(aw[i][k8 >> 1]) : bf16_lo(aw[i][k8 >> 1]);
+                        const float2 a2 = make_float2(a, a);
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a, b[j], acc[i][j]);
+                        for (int jp = 0; jp < 4; ++jp) acc2[i][jp] = __ffma2_rn(a2, b2[jp], acc2[i][jp]);
                     }
                 }
             } else {
 #pragma unroll
                 for (int k8 = 0; k8 < 8; ++k8) {
                     const uint4 v = *reinterpret_cast<const uint4*>(sb + (kk * 8 + k8) * 256 + tx * 16);
-                    const float b[8] = {bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y),
-                                        bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w)};
+                    const float2 b2[4] = {make_float2(bf16_lo(v.x), bf16_hi(v.x)), make_float2(bf16_lo(v.y), bf16_hi(v.y)),
+                                          make_float2(bf16_lo(v.z), bf16_hi(v.z)), make_float2(bf16_lo(v.w), bf16_hi(v.w))};
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const float a = (k8 & 1) ? bf16_hi(aw[i][k8 >> 1]) : bf16_lo(aw[i][k8 >> 1]);
+                        const float2 a2 = make_float2(a, a);
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a, b[j], acc[i][j]);
+                        for (int jp = 0; jp < 4; ++jp) acc2[i][jp] = __ffma2_rn(a2, b2[jp], acc2[i][jp]);
                     }
                 }
             }
@@ -253,6 +261,14 @@ r3_pipelined_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
     }
 
     // Epilogue: rows ty + 16 i; columns tx*8 + j (row-major B) or tx + 16 j.
+    float acc[8][8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int jp = 0; jp < 4; ++jp) {
+            acc[i][2 * jp] = acc2[i][jp].x;
+            acc[i][2 * jp + 1] = acc2[i][jp].y;
+        }
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int64_t gm = m0 + ty + 16 * i;

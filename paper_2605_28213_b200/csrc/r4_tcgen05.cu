@@ -687,11 +687,16 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
     cfg.stream = stream;
     cudaLaunchAttribute attrs[2];
     unsigned na = 0;
-    // Programmatic dependent launch: the kernel's set-up may overlap the previous kernel's
-    // tail; the kernel itself waits (griddepcontrol.wait) before it touches global memory.
-    attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attrs[na].val.programmaticStreamSerializationAllowed = 1;
-    ++na;
+    // Programmatic dependent launch for single-wave launches (short kernels, where the gap
+    // between back-to-back launches is a visible share of the time): the kernel's set-up may
+    // overlap the previous kernel's tail; the kernel itself waits (griddepcontrol.wait) before
+    // it touches global memory.  Multi-wave launches measured slower with it and do without.
+    const int64_t units = static_cast<int64_t>(p.tiles_m) * p.tiles_n * p.splits;
+    if (units <= static_cast<int64_t>(grid)) {
+        attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attrs[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
     if (p.cluster) {
         attrs[na].id = cudaLaunchAttributeClusterDimension;
         attrs[na].val.clusterDim.x = static_cast<unsigned>(p.splits);

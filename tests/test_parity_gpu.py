@@ -116,6 +116,39 @@ def test_random_small_shapes(handles, variant):
         run_and_check(handles, case, variant, offsets=tuple(int(rng.integers(0, 3)) for _ in range(3)))
 
 
+# ------------------------------------------------------------------ skinny shapes of the top rung
+SKINNY = [  # (M, N, K, expected flags of kernel id - 400: 4 split-K, 8 swapped operands, 16 cluster reduce)
+    (16, 1024, 8192, 4 | 8 | 16),      # 4 tiles: cluster of 8
+    (16, 16384, 1024, 4 | 8 | 16),     # 64 tiles: cluster of 2
+    (8, 2048, 2048, 4 | 8 | 16),       # cluster of 4, M below one MMA N step
+    (32, 1000, 4096, 4 | 8 | 16),      # M = 32: largest cluster-reduced M, ragged N
+    (33, 1000, 4096, 4 | 8),           # M = 33: swapped, split through the global workspace
+    (64, 520, 2048, 4 | 8),            # M = 64: last swapped M
+    (65, 520, 2048, 4),                # M = 65: regular orientation, split-K with row-block reduce
+    (16, 256, 64, 8),                  # one tile, one k-block: no split
+    (1, 8192, 8192, 4 | 8 | 16),       # GEMV
+]
+
+
+@pytest.mark.parametrize("col", [False, True], ids=["Brow", "Bcol"])
+def test_tcgen05_skinny_modes(handles, col):
+    for idx, (M, N, K, flags) in enumerate(SKINNY):
+        for bf in (False, True):
+            case = gen.make_case(M, N, K, seed=40 + idx, dist_a="integer", dist_b="integer", b_col_major=col,
+                                 c_bf16=bf, name=f"skinny{M}x{N}x{K}-int")
+            run_and_check(handles, case, 4, exact=True)
+            got = handles[(col, bf)].last_kernel_id() - 400
+            assert got & ~3 == flags, (M, N, K, got, flags)
+        case = gen.make_case(M, N, K, seed=40 + idx, dist_a="normal", dist_b="normal", sigma_b=0.02, b_col_major=col,
+                             name=f"skinny{M}x{N}x{K}")
+        run_and_check(handles, case, 4)
+    # unaligned operands: the generic-proxy producers feed the swapped and the cluster paths too
+    case = gen.make_case(16, 1001, 4099, seed=77, dist_a="integer", dist_b="integer", b_col_major=col, lda=4101,
+                         ldb=(4099 if col else 1001) + 2, ldc=1003, name="skinny-unaligned")
+    run_and_check(handles, case, 4, exact=True, offsets=(1, 1, 1))
+    assert (handles[(col, False)].last_kernel_id() - 400) & 1
+
+
 # ------------------------------------------------------------------ degenerate sizes
 @pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_NAMES)
 def test_degenerate_sizes(handles, kb, variant):
@@ -200,14 +233,15 @@ def test_each_variant_reports_its_own_kernel(handles, kb):
             assert code == 0 and dev_id == g.last_kernel_id()
             if v == 4:
                 assert 400 <= dev_id < 432
-                assert (dev_id & 1) == (1 if case.name == "c2" else 0)   # generic producer only when unaligned
+                assert ((dev_id - 400) & 1) == (1 if case.name == "c2" else 0)   # generic producer only when unaligned
             else:
                 want = expect.get((case.name, v))
                 if want is not None:
                     assert dev_id == want, (case.name, v, dev_id)
     skinny = P.DeviceCase(gen.make_config("c5", 1))
     skinny.run(g, 4)
-    assert g.last_kernel_id() & 4, "the skinny shape must take the split-K path"
+    flags = g.last_kernel_id() - 400
+    assert (flags & 4) and (flags & 8) and (flags & 16), "the skinny shape must run swapped, split along K, cluster-reduced"
 
 
 def test_error_codes(handles, kb):
