@@ -39,8 +39,10 @@ WORKLOADS = {
 WORKLOAD = WORKLOADS["c4"]
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one tcgen05-rung launch at 8192^3
-# (ncu capture summarised in profiles/); None until a capture exists.
-R4_C4_DRAM_TRAFFIC_BYTES = None
+# (ncu capture summarised in profiles/r4_tcgen05_c4_8192.md): 1.369 GB read + 0.127 GB written.
+R4_C4_DRAM_TRAFFIC_BYTES = 1.496e9
+# the same for the skinny shape (profiles/r4_tcgen05_c5_skinny.md): 134.6 MB read + 4.1 MB written.
+R4_C5_DRAM_TRAFFIC_BYTES = 1.387e8
 VARIANT_NAMES = ["naive", "tiled", "vectorized", "pipelined", "tcgen05"]
 
 
@@ -318,7 +320,7 @@ def run_gpu(args):
     if args.workload == "c5":
         gbs = case.algorithmic_bytes / (ms_per_step * 1e-3) / 1e9
         line["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                            "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                            "frac": gbs / peaks["hbm_gbs"], "traffic": R4_C5_DRAM_TRAFFIC_BYTES if V == 4 else None,
                             "peak_source": f"{peak_kind} (copy bandwidth)", "frac_of_nominal_8000": gbs / 8000.0,
                             "algorithmic_bytes_per_launch": case.algorithmic_bytes}
     else:
