@@ -81,12 +81,13 @@ __device__ __forceinline__ void report_error(unsigned* status, unsigned code, un
 // walking groups of kGroupM tile-rows column by column so that the tiles in
 // flight together share A row-panels and B column-panels in L2.
 constexpr int kGroupM = 8;
-__host__ __device__ __forceinline__ void raster_tile(int64_t t, int tiles_m, int tiles_n, int& tm, int& tn)
+__host__ __device__ __forceinline__ void raster_tile(int64_t t, int tiles_m, int tiles_n, int& tm, int& tn,
+                                                     int group_m = kGroupM)
 {
-    const int64_t per_group = static_cast<int64_t>(kGroupM) * tiles_n;
+    const int64_t per_group = static_cast<int64_t>(group_m) * tiles_n;
     const int g = static_cast<int>(t / per_group);
-    const int first_m = g * kGroupM;
-    const int rows = (tiles_m - first_m < kGroupM) ? (tiles_m - first_m) : kGroupM;
+    const int first_m = g * group_m;
+    const int rows = (tiles_m - first_m < group_m) ? (tiles_m - first_m) : group_m;
     const int64_t r = t - static_cast<int64_t>(g) * per_group;
     tm = first_m + static_cast<int>(r % rows);
     tn = static_cast<int>(r / rows);

@@ -71,7 +71,46 @@ struct R4Params {
     int n_mma;              // skinny mode: M rounded up to 16 = the MMA's N
     uint32_t stage_tx;      // bytes one stage's TMA loads deliver (A box + B boxes)
     int cluster;            // 1: the splits of a tile are one cluster and reduce through DSMEM
+    int group_m;            // tile raster: tile-rows per group
+    int64_t full_units;     // units [0, full_units) are whole tiles; later ones are 128-column half tiles
+    int64_t total_units;
+    uint32_t idesc_half;    // instruction descriptor for a half tile (N = 128)
 };
+
+// One entry of the static schedule.
+struct Unit {
+    int64_t tile;
+    int m0, n0;             // first row / column of C it computes
+    int ncols;              // 256, or 128 for the half tiles that fill the last wave
+    int split, kb0, kb1;    // K split index and k-block range
+};
+__device__ __forceinline__ Unit decode_unit(int64_t u, const R4Params& p)
+{
+    Unit x;
+    int half = 0;
+    x.ncols = BN;
+    if (p.splits > 1) {
+        x.tile = u / p.splits;
+        x.split = static_cast<int>(u % p.splits);
+    } else {
+        x.split = 0;
+        if (u < p.full_units) {
+            x.tile = u;
+        } else {
+            const int64_t v = u - p.full_units;
+            x.tile = p.full_units + (v >> 1);
+            half = static_cast<int>(v & 1);
+            x.ncols = BN / 2;
+        }
+    }
+    int tm, tn;
+    raster_tile(x.tile, p.tiles_m, p.tiles_n, tm, tn, p.group_m);
+    x.m0 = tm * BM;
+    x.n0 = tn * BN + half * (BN / 2);
+    x.kb0 = x.split * p.kb_per_split;
+    x.kb1 = min(p.nkb, x.kb0 + p.kb_per_split);
+    return x;
+}
 
 // 64-bit shared-memory matrix descriptor: start address, leading / stride byte
 // offsets (all >> 4), descriptor version 1, 128-byte swizzle.
@@ -115,7 +154,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Cluster mode: no CTA may touch a peer's shared memory before that peer runs.
     if (SWAP && p.cluster) ptx::cluster_arrive_release();
-    const int64_t total_units = static_cast<int64_t>(p.tiles_m) * p.tiles_n * p.splits;
+    const int64_t total_units = p.total_units;
 
     // TMA producer state (used by warp 0, lane 0 only): position in the static schedule.
     struct {
@@ -127,13 +166,11 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     auto prod_enter_unit = [&]() {
         prod.live = prod.u < total_units;
         if (!prod.live) return;
-        int tm, tn;
-        raster_tile(prod.u / p.splits, p.tiles_m, p.tiles_n, tm, tn);
-        const int split = static_cast<int>(prod.u % p.splits);
-        prod.kb = split * p.kb_per_split;
-        prod.kb1 = min(p.nkb, prod.kb + p.kb_per_split);
-        prod.m0 = tm * BM;
-        prod.n0 = tn * BN;
+        const Unit x = decode_unit(prod.u, p);
+        prod.kb = x.kb0;
+        prod.kb1 = x.kb1;
+        prod.m0 = x.m0;
+        prod.n0 = x.n0;     // a half tile still loads 256 columns from n0; its MMA reads the first 128
     };
     // Issues loads until `limit` k-blocks have been issued in total or the schedule ends.
     auto produce = [&](uint32_t limit) {
@@ -221,8 +258,9 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             uint32_t it = 0, t = 0;
             bool ok = true;
             for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++t) {
-                const int split = static_cast<int>(u % p.splits);
-                const int kb0 = split * p.kb_per_split, kb1 = min(p.nkb, kb0 + p.kb_per_split);
+                const Unit x = decode_unit(u, p);
+                const int kb0 = x.kb0, kb1 = x.kb1;
+                const uint32_t idesc = (x.ncols == BN) ? p.idesc : p.idesc_half;
                 const uint32_t buf = t & 1;
                 if (!ptx::mbar_wait(&acc_empty[buf], ((t >> 1) & 1) ^ 1, abort_flag)) {
                     report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x410u | buf);
@@ -255,10 +293,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
 #pragma unroll
                             for (int h = 0; h < 2; ++h)
                                 ptx::umma_f16(d_tmem + h * 128, b_desc + static_cast<uint64_t>(h * (16384 >> 4) + k4 * p.b_kstep),
-                                              a_desc + static_cast<uint64_t>(k4 * 2), p.idesc, acc);
+                                              a_desc + static_cast<uint64_t>(k4 * 2), idesc, acc);
                         } else {
                             ptx::umma_f16(d_tmem, a_desc + static_cast<uint64_t>(k4 * 2),
-                                          b_desc + static_cast<uint64_t>(k4 * p.b_kstep), p.idesc, acc);
+                                          b_desc + static_cast<uint64_t>(k4 * p.b_kstep), idesc, acc);
                         }
                     }
                     ptx::umma_commit(&empty[s]);
@@ -274,11 +312,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         uint32_t nstaged = 0;                                // staging blocks written so far (buffer = parity)
         bool ok = true;
         for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++t) {
-            int tm, tn;
-            const int64_t tile = u / p.splits;
-            raster_tile(tile, p.tiles_m, p.tiles_n, tm, tn);
-            const int split = static_cast<int>(u % p.splits);
-            const int m0 = tm * BM, n0 = tn * BN;
+            const Unit x = decode_unit(u, p);
+            const int64_t tile = x.tile;
+            const int split = x.split;
+            const int m0 = x.m0, n0 = x.n0;
             const uint32_t buf = t & 1;
             if (!ptx::mbar_wait(&acc_full[buf], (t >> 1) & 1, abort_flag)) {
                 if (lane == 0) report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x430u | buf);
@@ -390,7 +427,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 uint16_t* dst_h = static_cast<uint16_t*>(g.C);
                 const int64_t ld = partial ? p.ldw : g.ldc;
                 const int rows = min(32, g.M - row0);
-                for (int c = 0; c * cpc < BN; ++c) {
+                for (int c = 0; c * cpc < x.ncols; ++c) {
                     const int col0 = n0 + c * cpc;
                     if (col0 >= g.N) break;
                     uint32_t v[32], w[32];
@@ -498,11 +535,9 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         uint32_t it = 0;
         bool ok = true;
         for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
-            int tm, tn;
-            raster_tile(u / p.splits, p.tiles_m, p.tiles_n, tm, tn);
-            const int split = static_cast<int>(u % p.splits);
-            const int kb0 = split * p.kb_per_split, kb1 = min(p.nkb, kb0 + p.kb_per_split);
-            const int m0 = tm * BM, n0 = tn * BN;
+            const Unit x = decode_unit(u, p);
+            const int kb0 = x.kb0, kb1 = x.kb1;
+            const int m0 = x.m0, n0 = x.n0;
             for (int kb = kb0; kb < kb1; ++kb, ++it) {
                 const int s = it % STAGES;
                 if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
@@ -561,9 +596,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         ptx::cluster_wait_acquire();
         if (warp >= 2 && warp < 6 && !abort_flag[0]) {
             const int rank = static_cast<int>(blockIdx.x % p.splits);
-            int tm, tn;
-            raster_tile(blockIdx.x / p.splits, p.tiles_m, p.tiles_n, tm, tn);
-            const int n0 = tn * BN;
+            const int n0 = decode_unit(blockIdx.x, p).n0;
             const int nblk = 8 / p.splits;
             const float* slots = reinterpret_cast<const float*>(epi_smem);
             // each warp takes every fourth row m of every local block, four rows per step so
@@ -691,8 +724,7 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
     // between back-to-back launches is a visible share of the time): the kernel's set-up may
     // overlap the previous kernel's tail; the kernel itself waits (griddepcontrol.wait) before
     // it touches global memory.  Multi-wave launches measured slower with it and do without.
-    const int64_t units = static_cast<int64_t>(p.tiles_m) * p.tiles_n * p.splits;
-    if (units <= static_cast<int64_t>(grid)) {
+    if (p.total_units <= static_cast<int64_t>(grid)) {
         attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attrs[na].val.programmaticStreamSerializationAllowed = 1;
         ++na;
@@ -782,7 +814,17 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     p.kid = kIdTcgen05 + (generic ? 1 : 0) + (p.epi_tma ? 0 : 2) + (p.splits > 1 ? 4 : 0) + (swap ? 8 : 0) +
             (p.cluster ? 16 : 0);
     *kernel_id = p.kid;
-    const int64_t units = tiles * p.splits;
+    // Static schedule.  Without a K split, a last wave that would leave at least half of the
+    // SMs idle is cut into 128-column half tiles (twice as many units, half as long).
+    p.group_m = 16;   // measured: 16 tile-rows per raster group re-read least from HBM at 8192^3
+    p.full_units = tiles;
+    if (p.splits == 1 && !swap) {
+        const int64_t tail = tiles % ctx.sm_count;
+        if (tail != 0 && 2 * tail <= ctx.sm_count && g.N > BN / 2) p.full_units = tiles - tail;
+    }
+    p.total_units = p.splits > 1 ? tiles * p.splits : p.full_units + 2 * (tiles - p.full_units);
+    p.idesc_half = (p.idesc & ~(0x3Fu << 17)) | (static_cast<uint32_t>((BN / 2) >> 3) << 17);
+    const int64_t units = p.total_units;
     // A cluster handles exactly one tile, so the cluster path launches every unit as a CTA.
     const unsigned grid = static_cast<unsigned>((p.cluster || units < ctx.sm_count) ? units : ctx.sm_count);
 #define KLIN_R4_LAUNCH(BC, GE, SW) launch<BC, GE, SW>(g, ma, mb, mc, p, grid, ctx.device, stream)
