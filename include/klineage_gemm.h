@@ -144,6 +144,7 @@ klineage_status_t klineage_gemm_get_device_status(klineage_gemm_t h, int* code_o
  *   0 naive | 100 tiled | 200 + 1*(A vector) + 2*(B vector) + 4*(C vector)
  *   300 TMA pipeline, 301 producer-thread pipeline
  *   400 + 1*(generic-proxy producer) + 2*(direct epilogue) + 4*(split-K) + 8*(skinny mode)
+ *       + 16*(cluster reduce) + 32*(CTA-pair MMA)
  *   900 zero fill (K == 0); -1 before the first run or after a no-op.
  */
 int klineage_gemm_last_kernel_id(klineage_gemm_t h);

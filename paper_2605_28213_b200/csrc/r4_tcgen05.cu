@@ -763,6 +763,9 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     p.ws = static_cast<float*>(ctx.workspace);
     p.counters = ctx.tile_counters;
 
+    // Large aligned problems run on the CTA-pair kernel (tcgen05.mma.cta_group::2).
+    if (!plan.swap && plan.splits == 1 && r4_pair_applicable(g, ctx)) return launch_r4_tcgen05_pair(g, ctx, stream, kernel_id);
+
     const bool generic = !(ctx.encode_tiled && tma_ok(g.A, g.lda, 2) && tma_ok(g.B, g.ldb, 2));
     const int celt = g.c_bf16 ? 2 : 4;
     // Skinny mode: few activation rows -> they become the MMA's N, the weights its 128 rows.

@@ -1,0 +1,454 @@
+// Rung 4, CTA-pair form: tcgen05.mma.cta_group::2.
+//
+// Two CTAs on neighbouring SMs (a cluster of 2) share one 512 x 256 output
+// tile, computed as two 256-row MMA blocks.  Each CTA holds its own 2 x 128 rows
+// of A and ONE HALF (128 columns) of the B block in shared memory; the MMAs,
+// issued by one thread of the pair's even CTA, feed both SMs' tensor cores,
+// which fetch the other half of B from the peer's shared memory.  Per k-block a
+// CTA loads 48 KiB for 256 x 256 x 64 multiply-adds (half the bytes per flop of
+// the single-CTA 128 x 256 tile).  The two row blocks have separate fp32
+// accumulators in TMEM (2 x 256 columns) and their MMAs ALTERNATE: measured on
+// B200, back-to-back tcgen05.mma into the same accumulator run at 159 clocks
+// per 128 x 256 x 16 instruction, alternating accumulators at the full 128.
+//
+//   warp 0      TMA producer (each CTA loads its own A box and its half of B;
+//               no multicast: every byte is fetched by exactly one CTA).  Both
+//               CTAs' loads complete on the EVEN CTA's "full" barrier
+//               (cp.async.bulk.tensor ... .cta_group::2 lets the barrier live in
+//               the partner), which expects the bytes of both
+//   warp 1      even CTA: MMA issuer; idle in the odd CTA
+//   warps 2..5  epilogue of the CTA's own 128 rows (same staging + TMA store /
+//               masked-store code path as the single-CTA kernel)
+// "Stage free" and "accumulator ready" reach both CTAs through two plain
+// tcgen05.commit instructions (own barrier, peer's barrier), never the
+// multicast form.  All waits are bounded; both CTAs pass a cluster barrier
+// before exit so that no remote arrive can hit shared memory of a finished CTA.
+//
+// Preconditions (paper, Introduction: intrinsics "require compatible tile
+// shapes, layouts, and hardware support"): A, B TMA-loadable (16-byte aligned
+// base and pitch), no K split, not the skinny orientation.  Everything else
+// runs on the single-CTA kernel of r4_tcgen05.cu.
+#include "common.cuh"
+#include "ptx.cuh"
+#include <cstring>
+
+namespace klin {
+namespace {
+
+constexpr int PM = 128;            // rows per CTA and MMA block; a pair tile has 2 blocks x 2 CTAs x 128 = 512 rows
+constexpr int TILE_M = 4 * PM;
+constexpr int PN = 256;            // columns of C per pair
+constexpr int BK = 64;
+constexpr int STAGES = 4;
+constexpr int kABlockBytes = PM * BK * 2;      // 16 KiB per row block
+constexpr int kABytes = 2 * kABlockBytes;      // 32 KiB
+constexpr int kBHalfBytes = (PN / 2) * BK * 2; // 16 KiB
+constexpr int kStageBytes = kABytes + kBHalfBytes;
+constexpr int kEpiBufBytes = 32 * 128;
+constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;
+constexpr int kSmemBytes = 1024 + STAGES * kStageBytes + kEpiBytes + 512;
+constexpr int kTmemCols = 512;
+constexpr int kThreads = 6 * 32;
+
+struct PairParams {
+    int tiles_m2, tiles_n;      // 512-row x 256-column tiles
+    int nkb;
+    int epi_tma;
+    int kid;
+    int group_m;
+    int64_t total_tiles;
+    uint32_t idesc;
+    uint32_t b_desc_hi, b_desc_lbo, b_kstep;
+};
+
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(ptx::smem_u32(smem_dst)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_f16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                              uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Plain commit of the pair's MMAs onto a barrier given by its shared::cluster
+// address (own CTA or the peer).
+__device__ __forceinline__ void umma_commit_pair(uint32_t cluster_bar_addr)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_bar_addr)
+                 : "memory");
+}
+// 2-D tiled load whose completion is counted on a barrier that may live in the
+// partner CTA (shared::cluster address); the data lands in this CTA.
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const void* tmap, int x, int y, uint32_t cluster_bar_addr)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, "
+        "%3}], [%4];"
+        ::"r"(ptx::smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(cluster_bar_addr)
+        : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar_addr) : "memory");
+}
+
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_field, uint32_t hi)
+{
+    const uint32_t lo = ((smem_addr >> 4) & 0x3FFFu) | (lbo_field << 16);
+    return (static_cast<uint64_t>(hi) << 32) | lo;
+}
+
+template <bool BCOL>
+__global__ void __launch_bounds__(kThreads, 1)
+r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_c, PairParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* epi_smem = smem + STAGES * kStageBytes;
+    uint64_t* full = reinterpret_cast<uint64_t*>(epi_smem + kEpiBytes);   // even CTA: both CTAs' loads landed
+    uint64_t* empty = full + STAGES;                                      // the pair's MMAs are done with the stage
+    uint64_t* acc_full = empty + STAGES;                                  // [0]: the tile's accumulators are complete
+    uint64_t* acc_empty = acc_full + 2;                                   // [0]: even CTA, both epilogues drained
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();          // 0 = even CTA (issues the MMAs), 1 = odd CTA
+    const int64_t pair_id = blockIdx.x >> 1;
+    const int64_t n_pairs = gridDim.x >> 1;
+
+    if (warp == 0 && lane == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(&full[s], 1);
+            ptx::mbar_init(&empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(&acc_full[b], 1);
+            ptx::mbar_init(&acc_empty[b], 8);              // 4 epilogue warps of each CTA
+        }
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;
+        ptx::fence_barrier_init();
+        ptx::prefetch_tensormap(&map_a);
+        ptx::prefetch_tensormap(&map_b);
+        if (p.epi_tma) ptx::prefetch_tensormap(&map_c);
+        if (blockIdx.x == 0) g.status[1] = p.kid;
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_slot, kTmemCols);
+        tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    // Both CTAs' barriers exist before anyone signals across the pair.
+    ptx::cluster_arrive_release();
+    ptx::cluster_wait_acquire();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    auto tile_origin = [&](int64_t t, int& m0, int& n0) {
+        int tm, tn;
+        raster_tile(t, p.tiles_m2, p.tiles_n, tm, tn, p.group_m);
+        m0 = tm * TILE_M + static_cast<int>(rank) * PM;     // this CTA's rows: m0 + [0,128) and m0 + 256 + [0,128)
+        n0 = tn * PN;
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t t = pair_id; t < p.total_tiles && ok; t += n_pairs) {
+                int m0, n0;
+                tile_origin(t, m0, n0);
+                const int nb = n0 + static_cast<int>(rank) * (PN / 2);      // this CTA's half of B
+                for (int kb = 0; kb < p.nkb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
+                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x500u | s);
+                        abort_flag[0] = 1;
+                        ok = false;
+                        break;
+                    }
+                    uint8_t* sa = smem + s * kStageBytes;
+                    uint8_t* sb = sa + kABytes;
+                    // The even CTA's barrier counts the bytes of both CTAs' loads of this stage.
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(&full[s], 2 * kStageBytes);
+                    const uint32_t bar = ptx::map_to_cta(ptx::smem_u32(&full[s]), 0);
+                    tma_load_2d_pair(sa, &map_a, kb * BK, m0, bar);
+                    tma_load_2d_pair(sa + kABlockBytes, &map_a, kb * BK, m0 + 2 * PM, bar);
+                    if (BCOL) {
+                        tma_load_2d_pair(sb, &map_b, kb * BK, nb, bar);
+                    } else {
+                        tma_load_2d_pair(sb, &map_b, nb, kb * BK, bar);
+                        tma_load_2d_pair(sb + 64 * BK * 2, &map_b, nb + 64, kb * BK, bar);
+                    }
+                }
+            }
+            // Drain: in the even CTA wait for the last fills; the odd CTA's loads are covered by
+            // the same barriers (the MMAs that consumed them have completed before the epilogue ends).
+            if (rank == 0) {
+                const uint32_t first = it > STAGES ? it - STAGES : 0;
+                for (uint32_t j = first; j < it; ++j)
+                    ptx::mbar_wait(&full[j % STAGES], (j / STAGES) & 1, abort_flag + 1);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            // -------------------------------------------------------- MMA issuer (even CTA)
+            uint32_t it = 0, tcount = 0;
+            bool ok = true;
+            for (int64_t t = pair_id; t < p.total_tiles && ok; t += n_pairs, ++tcount) {
+                // Both accumulators are rewritten: wait until both CTAs' epilogues drained the last tile.
+                if (!ptx::mbar_wait(&acc_empty[0], (tcount & 1) ^ 1, abort_flag)) {
+                    report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x520u);
+                    abort_flag[0] = 1;
+                    break;
+                }
+                ptx::tc_fence_after_sync();
+                for (int kb = 0; kb < p.nkb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t par = (it / STAGES) & 1;
+                    if (!ptx::mbar_wait(&full[s], par, abort_flag)) {
+                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x530u | s);
+                        abort_flag[0] = 1;
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t sa = ptx::smem_u32(smem + s * kStageBytes);
+                    const uint32_t sb = sa + kABytes;
+                    const uint64_t a_desc = make_desc(sa, 1, (1024u >> 4) | (1u << 14) | (2u << 29));
+                    const uint64_t b_desc = make_desc(sb, p.b_desc_lbo, p.b_desc_hi);
+#pragma unroll
+                    for (int k4 = 0; k4 < BK / 16; ++k4) {
+                        const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
+                        // alternate the two row blocks: consecutive MMAs never share an accumulator
+                        umma_f16_pair(tmem_base, a_desc + static_cast<uint64_t>(k4 * 2),
+                                      b_desc + static_cast<uint64_t>(k4 * p.b_kstep), p.idesc, acc);
+                        umma_f16_pair(tmem_base + PN, a_desc + static_cast<uint64_t>((kABlockBytes >> 4) + k4 * 2),
+                                      b_desc + static_cast<uint64_t>(k4 * p.b_kstep), p.idesc, acc);
+                    }
+                    umma_commit_pair(ptx::smem_u32(&empty[s]));
+                    umma_commit_pair(ptx::map_to_cta(ptx::smem_u32(&empty[s]), 1));
+                }
+                if (ok) {
+                    umma_commit_pair(ptx::smem_u32(&acc_full[0]));
+                    umma_commit_pair(ptx::map_to_cta(ptx::smem_u32(&acc_full[0]), 1));
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (own 128 rows)
+        const int q = warp & 3;
+        uint8_t* stg = epi_smem + (warp - 2) * 2 * kEpiBufBytes;
+        uint32_t tcount = 0, nstaged = 0;
+        bool ok = true;
+        for (int64_t t = pair_id; t < p.total_tiles && ok; t += n_pairs, ++tcount) {
+            int m0, n0;
+            tile_origin(t, m0, n0);
+            if (!ptx::mbar_wait(&acc_full[0], tcount & 1, abort_flag)) {
+                if (lane == 0) report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x540u);
+                abort_flag[0] = 1;
+                ok = false;
+                break;
+            }
+            ptx::tc_fence_after_sync();
+#pragma unroll 1
+            for (int mb = 0; mb < 2; ++mb) {
+            const int row0 = m0 + mb * 2 * PM + q * 32;
+            if (row0 < g.M) {
+                const bool out_bf16 = g.c_bf16 != 0;
+                const int cpc = out_bf16 ? 64 : 32;
+                float* dst_f = static_cast<float*>(g.C);
+                uint16_t* dst_h = static_cast<uint16_t*>(g.C);
+                const int rows = min(32, g.M - row0);
+                for (int c = 0; c * cpc < PN; ++c) {
+                    const int col0 = n0 + c * cpc;
+                    if (col0 >= g.N) break;
+                    uint32_t v[32], w[32];
+                    const uint32_t taddr = tmem_base + mb * PN + c * cpc + (static_cast<uint32_t>(q * 32) << 16);
+                    ptx::tmem_ld_32x32b_x32(taddr, v);
+                    if (out_bf16) {
+                        uint32_t v2[32];
+                        ptx::tmem_ld_32x32b_x32(taddr + 32, v2);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            w[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+                            w[16 + i] = pack_bf16x2(__uint_as_float(v2[2 * i]), __uint_as_float(v2[2 * i + 1]));
+                        }
+                    } else {
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) w[i] = v[i];
+                    }
+                    uint8_t* b = stg + (nstaged++ & 1) * kEpiBufBytes;
+                    if (p.epi_tma) {
+                        if (lane == 0) ptx::tma_store_wait_read<1>();
+                        __syncwarp();
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<uint4*>(b + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                            make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                    if (p.epi_tma) {
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            ptx::tma_store_2d(&map_c, col0, row0, b);
+                            ptx::tma_store_commit();
+                        }
+                    } else {
+                        __syncwarp();
+                        for (int rr = 0; rr < rows; ++rr) {
+                            const uint32_t word =
+                                *reinterpret_cast<const uint32_t*>(b + rr * 128 + (((lane >> 2) ^ (rr & 7)) << 4) +
+                                                                   (lane & 3) * 4);
+                            const int64_t row = row0 + rr;
+                            if (out_bf16) {
+                                const int col = col0 + 2 * lane;
+                                uint16_t* d = dst_h + row * g.ldc + col;
+                                if (col + 1 < g.N && (reinterpret_cast<uintptr_t>(d) & 3) == 0) {
+                                    *reinterpret_cast<uint32_t*>(d) = word;
+                                } else {
+                                    if (col < g.N) d[0] = static_cast<uint16_t>(word & 0xFFFFu);
+                                    if (col + 1 < g.N) d[1] = static_cast<uint16_t>(word >> 16);
+                                }
+                            } else {
+                                const int col = col0 + lane;
+                                if (col < g.N) dst_f[row * g.ldc + col] = __uint_as_float(word);
+                            }
+                        }
+                        __syncwarp();
+                    }
+                }
+            }
+            }
+            // Hand the accumulators back to the MMA issuer in the even CTA.
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&acc_empty[0]), 0));
+        }
+        if (p.epi_tma && lane == 0) ptx::tma_store_wait_all<0>();
+    }
+
+    // No CTA leaves while its partner may still signal into its shared memory.
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_arrive_release();
+    ptx::cluster_wait_acquire();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
+template <bool BCOL>
+cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
+                   const PairParams& p, unsigned grid, int device, cudaStream_t stream)
+{
+    auto kern = r4_pair_kernel<BCOL>;
+    static bool attr_set[64] = {};
+    if (device < 0 || device >= 64 || !attr_set[device]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        if (device >= 0 && device < 64) attr_set[device] = true;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, g, ma, mb, mc, p);
+}
+
+}  // namespace
+
+bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx)
+{
+    auto ok2 = [](const void* base, int64_t ld) {
+        return reinterpret_cast<uintptr_t>(base) % 16 == 0 && (ld * 2) % 16 == 0 && ld * 2 < (int64_t(1) << 40);
+    };
+    if (!ctx.encode_tiled || ctx.max_smem_optin < kSmemBytes) return false;
+    if (!ok2(g.A, g.lda) || !ok2(g.B, g.ldb)) return false;
+    // worthwhile only when the pairs fill the machine: at least one 512 x 256 tile per SM pair
+    const int64_t tiles = static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * ((g.N + PN - 1) / PN);
+    return g.M > 2 * PM && tiles >= ctx.sm_count / 2;
+}
+
+cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
+{
+    PairParams p;
+    memset(&p, 0, sizeof p);
+    p.tiles_m2 = (g.M + TILE_M - 1) / TILE_M;
+    p.tiles_n = (g.N + PN - 1) / PN;
+    p.total_tiles = static_cast<int64_t>(p.tiles_m2) * p.tiles_n;
+    p.nkb = (g.K + BK - 1) / BK;
+    p.group_m = 4;                                  // 4 x 512 rows per raster group
+    const int celt = g.c_bf16 ? 2 : 4;
+    p.epi_tma = (reinterpret_cast<uintptr_t>(g.C) % 16 == 0 && (g.ldc * celt) % 16 == 0 &&
+                 g.ldc * celt < (int64_t(1) << 40))
+                    ? 1
+                    : 0;
+    // Instruction descriptor: fp32 accumulator, bf16 A/B, A K-major, B K-major (column-major B) or
+    // MN-major (row-major B), N = 256, M = 256 (128 rows in each CTA of the pair).
+    const uint32_t w_major = g.b_col ? 0u : 1u;
+    p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (w_major << 16) | (static_cast<uint32_t>(PN >> 3) << 17) |
+              (static_cast<uint32_t>((2 * PM) >> 4) << 24);
+    // B half in shared memory: 128 columns.  K-major: 128 rows of 128 bytes; MN-major: two
+    // 64-column blocks 8192 bytes apart, 8-k groups 1024 bytes apart.
+    p.b_desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    p.b_desc_lbo = g.b_col ? 1u : ((64u * BK * 2u) >> 4);
+    p.b_kstep = g.b_col ? 2u : (2048u >> 4);
+
+    CUtensorMap ma, mb, mc;
+    memset(&ma, 0, sizeof ma);
+    memset(&mb, 0, sizeof mb);
+    memset(&mc, 0, sizeof mc);
+    bool ok = encode_map_2d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, PM,
+                            CU_TENSOR_MAP_SWIZZLE_128B);
+    if (g.b_col)
+        ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, PN / 2,
+                                 CU_TENSOR_MAP_SWIZZLE_128B);
+    else
+        ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, g.ldb * 2, 64, BK,
+                                 CU_TENSOR_MAP_SWIZZLE_128B);
+    if (p.epi_tma)
+        ok = ok && encode_map_2d(ctx, &mc, g.c_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                                 g.C, g.N, g.M, g.ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!ok) return cudaErrorInvalidValue;
+
+    p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + 32;
+    *kernel_id = p.kid;
+    const int64_t max_pairs = ctx.sm_count / 2;
+    const unsigned grid = 2u * static_cast<unsigned>(p.total_tiles < max_pairs ? p.total_tiles : max_pairs);
+    return g.b_col ? launch<true>(g, ma, mb, mc, p, grid, ctx.device, stream)
+                   : launch<false>(g, ma, mb, mc, p, grid, ctx.device, stream);
+}
+
+}  // namespace klin

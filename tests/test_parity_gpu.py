@@ -149,6 +149,27 @@ def test_tcgen05_skinny_modes(handles, col):
     assert (handles[(col, False)].last_kernel_id() - 400) & 1
 
 
+# ------------------------------------------------------------------ CTA-pair form of the top rung
+@pytest.mark.parametrize("col", [False, True], ids=["Brow", "Bcol"])
+def test_tcgen05_cta_pair_ragged(handles, col):
+    """Large aligned shapes run on tcgen05.mma.cta_group::2 (512 x 256 pair tiles); tails in M, N and K."""
+    for idx, (M, N, K) in enumerate([(5000, 5200, 1000), (4608, 4352, 72)]):
+        for bf in (False, True):
+            case = gen.make_case(M, N, K, seed=60 + idx, dist_a="integer", dist_b="integer", b_col_major=col,
+                                 c_bf16=bf, name=f"pair{M}x{N}x{K}-int")
+            rows = P.sample_rows(M)
+            C_ref, S = P.oracle_rows(case, rows)
+            vals, _ = run_and_check(handles, case, 4, C_ref, S, rows, exact=True)
+            assert (handles[(col, bf)].last_kernel_id() - 400) & 32, "expected the CTA-pair kernel"
+            if not bf:
+                assert P.integer_checksums_match(case, vals)
+        case = gen.make_case(M, N, K, seed=60 + idx, dist_a="normal", dist_b="uniform", b_col_major=col,
+                             name=f"pair{M}x{N}x{K}")
+        rows = P.sample_rows(M)
+        C_ref, S = P.oracle_rows(case, rows)
+        run_and_check(handles, case, 4, C_ref, S, rows)
+
+
 # ------------------------------------------------------------------ degenerate sizes
 @pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_NAMES)
 def test_degenerate_sizes(handles, kb, variant):
@@ -232,7 +253,7 @@ def test_each_variant_reports_its_own_kernel(handles, kb):
             code, dev_id = g.device_status()
             assert code == 0 and dev_id == g.last_kernel_id()
             if v == 4:
-                assert 400 <= dev_id < 432
+                assert 400 <= dev_id < 464
                 assert ((dev_id - 400) & 1) == (1 if case.name == "c2" else 0)   # generic producer only when unaligned
             else:
                 want = expect.get((case.name, v))
