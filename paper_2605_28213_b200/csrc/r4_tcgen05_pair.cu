@@ -17,8 +17,9 @@
 //               (cp.async.bulk.tensor ... .cta_group::2 lets the barrier live in
 //               the partner), which expects the bytes of both
 //   warp 1      even CTA: MMA issuer; idle in the odd CTA
-//   warps 2..5  epilogue of the CTA's own 128 rows (same staging + TMA store /
-//               masked-store code path as the single-CTA kernel)
+//   warps 2..9  epilogue: four warps per row block drain its accumulator (TMEM
+//               loads software-pipelined against convert / stage / TMA store or
+//               masked stores) and hand it back right after the last load
 // "Stage free" and "accumulator ready" reach both CTAs through two plain
 // tcgen05.commit instructions (own barrier, peer's barrier), never the
 // multicast form.  All waits are bounded; both CTAs pass a cluster barrier
@@ -45,10 +46,10 @@ constexpr int kABytes = 2 * kABlockBytes;      // 32 KiB
 constexpr int kBHalfBytes = (PN / 2) * BK * 2; // 16 KiB
 constexpr int kStageBytes = kABytes + kBHalfBytes;
 constexpr int kEpiBufBytes = 32 * 128;
-constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;
+constexpr int kEpiBytes = 8 * kEpiBufBytes;       // one staging block per epilogue warp
 constexpr int kSmemBytes = 1024 + STAGES * kStageBytes + kEpiBytes + 512;
 constexpr int kTmemCols = 512;
-constexpr int kThreads = 6 * 32;
+constexpr int kThreads = 10 * 32;                // producer, MMA issuer, 2 x 4 epilogue warps
 
 struct PairParams {
     int tiles_m2, tiles_n;      // 512-row x 256-column tiles
@@ -140,7 +141,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(&acc_full[b], 1);
-            ptx::mbar_init(&acc_empty[b], 8);              // 4 epilogue warps of each CTA
+            ptx::mbar_init(&acc_empty[b], 16);             // 8 epilogue warps of each CTA
         }
         abort_flag[0] = 0;
         abort_flag[1] = 0;
@@ -255,10 +256,19 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (own 128 rows)
+        // ------------------------------------------------------------ epilogue
+        // Warps 2..5 drain the first row block's accumulator, warps 6..9 the second; a warp
+        // reads the TMEM lane quarter (warp & 3).  TMEM loads of the next 128-byte unit are in
+        // flight while the current one is converted, staged and stored, and the accumulator is
+        // handed back as soon as its last load has landed.
         const int q = warp & 3;
-        uint8_t* stg = epi_smem + (warp - 2) * 2 * kEpiBufBytes;
-        uint32_t tcount = 0, nstaged = 0;
+        const int mb = (warp - 2) >> 2;
+        uint8_t* b = epi_smem + (warp - 2) * kEpiBufBytes;
+        const bool out_bf16 = g.c_bf16 != 0;
+        const int cpc = out_bf16 ? 64 : 32;                   // columns per 128-byte staging row
+        float* dst_f = static_cast<float*>(g.C);
+        uint16_t* dst_h = static_cast<uint16_t*>(g.C);
+        uint32_t tcount = 0;
         bool ok = true;
         for (int64_t t = pair_id; t < p.total_tiles && ok; t += n_pairs, ++tcount) {
             int m0, n0;
@@ -270,81 +280,88 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 break;
             }
             ptx::tc_fence_after_sync();
-#pragma unroll 1
-            for (int mb = 0; mb < 2; ++mb) {
             const int row0 = m0 + mb * 2 * PM + q * 32;
-            if (row0 < g.M) {
-                const bool out_bf16 = g.c_bf16 != 0;
-                const int cpc = out_bf16 ? 64 : 32;
-                float* dst_f = static_cast<float*>(g.C);
-                uint16_t* dst_h = static_cast<uint16_t*>(g.C);
-                const int rows = min(32, g.M - row0);
-                for (int c = 0; c * cpc < PN; ++c) {
-                    const int col0 = n0 + c * cpc;
-                    if (col0 >= g.N) break;
-                    uint32_t v[32], w[32];
-                    const uint32_t taddr = tmem_base + mb * PN + c * cpc + (static_cast<uint32_t>(q * 32) << 16);
-                    ptx::tmem_ld_32x32b_x32(taddr, v);
-                    if (out_bf16) {
-                        uint32_t v2[32];
-                        ptx::tmem_ld_32x32b_x32(taddr + 32, v2);
-                        ptx::tmem_ld_wait();
+            const int rows = min(32, g.M - row0);
+            const int nunits = (row0 < g.M) ? (min(PN, g.N - n0) + cpc - 1) / cpc : 0;
+            const uint32_t tbase = tmem_base + mb * PN + (static_cast<uint32_t>(q * 32) << 16);
+
+            auto release = [&]() {
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&acc_empty[0]), 0));
+            };
+            auto issue = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32]) {
+                ptx::tmem_ld_32x32b_x32(tbase + u * cpc, r0);
+                if (out_bf16) ptx::tmem_ld_32x32b_x32(tbase + u * cpc + 32, r1);
+            };
+            auto finish = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32]) {
+                const int col0 = n0 + u * cpc;
+                uint32_t w[32];
+                if (out_bf16) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            w[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-                            w[16 + i] = pack_bf16x2(__uint_as_float(v2[2 * i]), __uint_as_float(v2[2 * i + 1]));
-                        }
-                    } else {
-                        ptx::tmem_ld_wait();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) w[i] = v[i];
+                    for (int i = 0; i < 16; ++i) {
+                        w[i] = pack_bf16x2(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
+                        w[16 + i] = pack_bf16x2(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]));
                     }
-                    uint8_t* b = stg + (nstaged++ & 1) * kEpiBufBytes;
-                    if (p.epi_tma) {
-                        if (lane == 0) ptx::tma_store_wait_read<1>();
-                        __syncwarp();
-                    }
+                } else {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        *reinterpret_cast<uint4*>(b + lane * 128 + ((j ^ (lane & 7)) << 4)) =
-                            make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-                    if (p.epi_tma) {
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) {
-                            ptx::tma_store_2d(&map_c, col0, row0, b);
-                            ptx::tma_store_commit();
-                        }
-                    } else {
-                        __syncwarp();
-                        for (int rr = 0; rr < rows; ++rr) {
-                            const uint32_t word =
-                                *reinterpret_cast<const uint32_t*>(b + rr * 128 + (((lane >> 2) ^ (rr & 7)) << 4) +
-                                                                   (lane & 3) * 4);
-                            const int64_t row = row0 + rr;
-                            if (out_bf16) {
-                                const int col = col0 + 2 * lane;
-                                uint16_t* d = dst_h + row * g.ldc + col;
-                                if (col + 1 < g.N && (reinterpret_cast<uintptr_t>(d) & 3) == 0) {
-                                    *reinterpret_cast<uint32_t*>(d) = word;
-                                } else {
-                                    if (col < g.N) d[0] = static_cast<uint16_t>(word & 0xFFFFu);
-                                    if (col + 1 < g.N) d[1] = static_cast<uint16_t>(word >> 16);
-                                }
+                    for (int i = 0; i < 32; ++i) w[i] = r0[i];
+                }
+                if (p.epi_tma) {
+                    if (lane == 0) ptx::tma_store_wait_read<0>();   // the previous store has read the buffer
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    *reinterpret_cast<uint4*>(b + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                        make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                if (p.epi_tma) {
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::tma_store_2d(&map_c, col0, row0, b);
+                        ptx::tma_store_commit();
+                    }
+                } else {
+                    __syncwarp();
+                    for (int rr = 0; rr < rows; ++rr) {
+                        const uint32_t word = *reinterpret_cast<const uint32_t*>(
+                            b + rr * 128 + (((lane >> 2) ^ (rr & 7)) << 4) + (lane & 3) * 4);
+                        const int64_t row = row0 + rr;
+                        if (out_bf16) {
+                            const int col = col0 + 2 * lane;
+                            uint16_t* d = dst_h + row * g.ldc + col;
+                            if (col + 1 < g.N && (reinterpret_cast<uintptr_t>(d) & 3) == 0) {
+                                *reinterpret_cast<uint32_t*>(d) = word;
                             } else {
-                                const int col = col0 + lane;
-                                if (col < g.N) dst_f[row * g.ldc + col] = __uint_as_float(word);
+                                if (col < g.N) d[0] = static_cast<uint16_t>(word & 0xFFFFu);
+                                if (col + 1 < g.N) d[1] = static_cast<uint16_t>(word >> 16);
                             }
+                        } else {
+                            const int col = col0 + lane;
+                            if (col < g.N) dst_f[row * g.ldc + col] = __uint_as_float(word);
                         }
-                        __syncwarp();
                     }
+                    __syncwarp();
+                }
+            };
+
+            if (nunits == 0) {
+                release();
+                continue;
+            }
+            uint32_t a0[32], a1[32], c0[32], c1[32];
+            issue(0, a0, a1);
+            for (int u = 0; u < nunits; u += 2) {
+                ptx::tmem_ld_wait();
+                if (u + 1 < nunits) issue(u + 1, c0, c1); else release();
+                finish(u, a0, a1);
+                if (u + 1 < nunits) {
+                    ptx::tmem_ld_wait();
+                    if (u + 2 < nunits) issue(u + 2, a0, a1); else release();
+                    finish(u + 1, c0, c1);
                 }
             }
-            }
-            // Hand the accumulators back to the MMA issuer in the even CTA.
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&acc_empty[0]), 0));
         }
         if (p.epi_tma && lane == 0) ptx::tma_store_wait_all<0>();
     }
