@@ -39,8 +39,8 @@ WORKLOADS = {
 WORKLOAD = WORKLOADS["c4"]
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one tcgen05-rung launch at 8192^3
-# (ncu capture summarised in profiles/r4_tcgen05_c4_8192.md): 1.369 GB read + 0.127 GB written.
-R4_C4_DRAM_TRAFFIC_BYTES = 1.496e9
+# (ncu capture summarised in profiles/r4_tcgen05_c4_8192.md): 0.961 GB read + 0.132 GB written.
+R4_C4_DRAM_TRAFFIC_BYTES = 1.093e9
 # the same for the skinny shape (profiles/r4_tcgen05_c5_skinny.md): 134.6 MB read + 4.1 MB written.
 R4_C5_DRAM_TRAFFIC_BYTES = 1.387e8
 VARIANT_NAMES = ["naive", "tiled", "vectorized", "pipelined", "tcgen05"]
@@ -329,7 +329,8 @@ def run_gpu(args):
                             "traffic": R4_C4_DRAM_TRAFFIC_BYTES if (args.workload, V) == ("c4", 4) else None,
                             "peak_source": f"{peak_kind} (burst cuBLAS bf16)",
                             "frac_of_sustained": per_gpu / peaks["bf16_tflops_sustained"],
-                            "frac_of_nominal_2250": per_gpu / 2250.0, "kernel": "r4_tcgen05_kernel",
+                            "frac_of_nominal_2250": per_gpu / 2250.0,
+                            "kernel": "r4_pair_kernel" if (kid - 400) & 32 else VARIANT_NAMES[V],
                             "flops_per_launch": case.flops}
 
     if rank == 0 and world == 1 and not args.no_extras and (args.workload, V) == ("c4", 4):
