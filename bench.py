@@ -43,7 +43,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 R4_C4_DRAM_TRAFFIC_BYTES = 1.093e9
 # the same for the skinny shape (profiles/r4_tcgen05_c5_skinny.md): 134.6 MB read + 4.1 MB written.
 R4_C5_DRAM_TRAFFIC_BYTES = 1.387e8
-VARIANT_NAMES = ["naive", "tiled", "vectorized", "pipelined", "tcgen05"]
+VARIANT_NAMES = ["naive", "tiled", "vectorized", "pipelined", "tcgen05", "mma_sync"]
+LINEAGE_ORDER = [0, 1, 2, 3, 5, 4]     # rung 3.5 (mma.sync, variant id 5) sits between rungs 3 and 4
 
 
 def load_peaks():
@@ -347,10 +348,10 @@ def lineage_table(prob_c4, kb, gen, torch, device, peaks):
     """Per-rung throughput at 8192^3 and 4096^3, and the HBM-bound skinny shape for every rung."""
     out = {}
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
-    reps = {0: (1, 2), 1: (2, 5), 2: (2, 5), 3: (2, 5), 4: (5, 30)}          # (warmup, reps)
+    reps = {0: (1, 2), 1: (2, 5), 2: (2, 5), 3: (2, 5), 5: (3, 10), 4: (5, 30)}          # (warmup, reps)
     c4 = prob_c4.case
     rows = {}
-    for v in range(5):
+    for v in LINEAGE_ORDER:
         w, r = reps[v]
         med, mn = prob_c4.time(v, r, w)
         rows[VARIANT_NAMES[v]] = {"ms_median": med, "ms_min": mn, "tflops": c4.flops / (med * 1e-3) / 1e12,
@@ -361,7 +362,7 @@ def lineage_table(prob_c4, kb, gen, torch, device, peaks):
     c3 = gen.make_config("c3", 1)
     p3 = DeviceProblem(c3, kb, torch, device)
     rows = {}
-    for v in range(5):
+    for v in LINEAGE_ORDER:
         w, r = reps[v]
         med, mn = p3.time(v, r * 2, w, flush=flush)
         rows[VARIANT_NAMES[v]] = {"ms_median": med, "ms_min": mn, "tflops": c3.flops / (med * 1e-3) / 1e12,
@@ -374,8 +375,8 @@ def lineage_table(prob_c4, kb, gen, torch, device, peaks):
     p5 = DeviceProblem(c5, kb, torch, device)
     rot = [p5.B] + [p5.B.clone() for _ in range(3)]          # 4 x 128 MiB of weights: no warm-L2 replay
     rows = {}
-    for v in range(5):
-        loops, per_loop = (3, 4) if v < 4 else (9, 40)
+    for v in LINEAGE_ORDER:
+        loops, per_loop = (3, 4) if v != 4 else (9, 40)
         best = []
         for _ in range(loops):
             for i in range(4):
@@ -408,7 +409,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the per-rung table and the CPU baseline")
     ap.add_argument("--workload", default="c4", choices=sorted(WORKLOADS),
                     help="configuration to time (default: the headline 8192^3; others are for profiling)")
-    ap.add_argument("--variant", type=int, default=4, choices=range(5), help="lineage rung to time (default 4)")
+    ap.add_argument("--variant", type=int, default=4, choices=range(6),
+                    help="lineage rung to time (default 4 = tcgen05; 5 = the mma.sync rung 3.5)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -32,7 +32,7 @@ typedef struct klineage_gemm_s* klineage_gemm_t;
 typedef enum {
     KLINEAGE_OK = 0,
     KLINEAGE_ERR_INVALID_ARG = 1,        /* null pointer, negative size, ld too small, aliasing ... */
-    KLINEAGE_ERR_BAD_VARIANT = 2,        /* variant outside 0..4                                      */
+    KLINEAGE_ERR_BAD_VARIANT = 2,        /* variant outside 0..5                                      */
     KLINEAGE_ERR_UNSUPPORTED_DEVICE = 3, /* the rung needs sm_100 hardware the device lacks          */
     KLINEAGE_ERR_ALLOC = 4,              /* device or host allocation failed in create                */
     KLINEAGE_ERR_LAUNCH = 5,             /* the CUDA runtime rejected a launch or a tensor map        */
@@ -63,9 +63,12 @@ typedef enum {
                                 scalar fallback when base or leading dimension is not 16-byte aligned        */
     KLINEAGE_PIPELINED = 3,  /* Table 1 "cp.async + pipeline" / "tma_load": multi-stage ring fed by TMA with
                                 full/empty mbarriers; producer threads when TMA's alignment rules fail       */
-    KLINEAGE_TCGEN05 = 4     /* Table 1 "warp_specialize" + matrix intrinsics: tcgen05.mma into TMEM (the
+    KLINEAGE_TCGEN05 = 4,    /* Table 1 "warp_specialize" + matrix intrinsics: tcgen05.mma into TMEM (the
                                 sm_100 successor of the table's wgmma), producer / MMA / epilogue warps,
                                 persistent tile scheduler, swizzled shared-memory epilogue, split-K          */
+    KLINEAGE_MMA_SYNC = 5    /* "rung 3.5", outside the five-step ladder: Table 1 "ldmatrix.swizzle" + "mma
+                                (m16n8k16)", the legacy warp-level tensor-core path on rung 3's TMA ring; it
+                                sits between rungs 3 and 4 in speed and completes the table's vocabulary       */
 } klineage_variant_t;
 
 /* Create-time configuration (host memory, read during create only). */
@@ -89,7 +92,7 @@ klineage_status_t klineage_gemm_create(klineage_gemm_t* out, const klineage_gemm
 
 /*
  * Enqueues C <- A . B on `stream` (a cudaStream_t, may be NULL for the default
- * stream) using exactly the rung `variant`; returns after the enqueue, performs
+ * stream) using exactly the rung `variant` (0..5); returns after the enqueue, performs
  * no device synchronisation and no allocation.
  *
  *   M, N, K   sizes, 0 <= value < 2^31.  M*N == 0: nothing is launched, OK.
@@ -105,7 +108,7 @@ klineage_status_t klineage_gemm_create(klineage_gemm_t* out, const klineage_gemm
  *   (paper, Introduction: "vectorized loads require alignment and valid tail
  *   handling").  Buffers stay owned by the caller.
  *
- * Errors: INVALID_ARG, BAD_VARIANT, UNSUPPORTED_DEVICE (variant 3 or 4 on a
+ * Errors: INVALID_ARG, BAD_VARIANT, UNSUPPORTED_DEVICE (variant 3, 4 or 5 on a
  * device without sm_100 TMA/tcgen05), LAUNCH.  Device-side give-ups (a bounded
  * barrier wait that expired) are reported by klineage_gemm_get_device_status.
  * One handle must not be used from two host threads at once.
@@ -145,6 +148,7 @@ klineage_status_t klineage_gemm_get_device_status(klineage_gemm_t h, int* code_o
  *   300 TMA pipeline, 301 producer-thread pipeline
  *   400 + 1*(generic-proxy producer) + 2*(direct epilogue) + 4*(split-K) + 8*(skinny mode)
  *       + 16*(cluster reduce) + 32*(CTA-pair MMA)
+ *   500 mma.sync rung on the TMA ring, 501 on producer threads
  *   900 zero fill (K == 0); -1 before the first run or after a no-op.
  */
 int klineage_gemm_last_kernel_id(klineage_gemm_t h);

@@ -25,8 +25,10 @@ KLINEAGE_ERR_SCRATCH_LIMIT = 8
 
 KLINEAGE_B_ROW_MAJOR, KLINEAGE_B_COL_MAJOR = 0, 1
 KLINEAGE_C_F32, KLINEAGE_C_BF16 = 0, 1
-KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELINED, KLINEAGE_TCGEN05 = range(5)
-VARIANTS = (KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELINED, KLINEAGE_TCGEN05)
+KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELINED, KLINEAGE_TCGEN05, KLINEAGE_MMA_SYNC = range(6)
+# the five-step ladder, then the intermediate legacy tensor-core rung ("3.5")
+VARIANTS = (KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELINED, KLINEAGE_TCGEN05,
+            KLINEAGE_MMA_SYNC)
 
 EXPORTED_SYMBOLS = (
     "klineage_gemm_create", "klineage_gemm_run", "klineage_gemm_destroy", "klineage_gemm_check_args",

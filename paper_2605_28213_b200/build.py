@@ -10,7 +10,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libklineage_gemm.so"
-SOURCES = ["klineage_gemm.cu", "r0_naive.cu", "r1_tiled.cu", "r2_vectorized.cu", "r3_pipelined.cu",
+SOURCES = ["klineage_gemm.cu", "r0_naive.cu", "r1_tiled.cu", "r2_vectorized.cu", "r3_pipelined.cu", "r35_mma_sync.cu",
            "r4_tcgen05.cu", "r4_tcgen05_pair.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]

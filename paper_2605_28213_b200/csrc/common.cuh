@@ -40,6 +40,7 @@ enum KernelId : int {
     kIdVectorized = 200,      // + 1 (A vector loads) + 2 (B vector loads) + 4 (C vector stores)
     kIdPipelined = 300,       // + 1 when the producer-thread path replaces TMA
     kIdTcgen05 = 400,         // + 1 generic-proxy producer, + 2 direct epilogue, + 4 split-K, + 8 skinny (swapped operands), + 16 cluster reduce, + 32 CTA pair
+    kIdMmaSync = 500,         // rung 3.5 (mma.sync); + 1 when the producer-thread path replaces TMA
     kIdZeroFill = 900,
 };
 
@@ -124,6 +125,7 @@ cudaError_t launch_r1_tiled(const GemmArgs& g, cudaStream_t stream, int* kernel_
 cudaError_t launch_r2_vectorized(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
 cudaError_t launch_r3_pipelined(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id);
 cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id);
+cudaError_t launch_r35_mma_sync(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id);
 cudaError_t launch_zero_fill(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
 // CTA-pair (cta_group::2) form of rung 4 and the test of its preconditions.
 bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx);

@@ -140,7 +140,7 @@ klineage_status_t klineage_gemm_check_args(int b_layout, int c_dtype, int64_t M,
 {
     if (b_layout != KLINEAGE_B_ROW_MAJOR && b_layout != KLINEAGE_B_COL_MAJOR) return KLINEAGE_ERR_INVALID_ARG;
     if (c_dtype != KLINEAGE_C_F32 && c_dtype != KLINEAGE_C_BF16) return KLINEAGE_ERR_INVALID_ARG;
-    if (variant < KLINEAGE_NAIVE || variant > KLINEAGE_TCGEN05) return KLINEAGE_ERR_BAD_VARIANT;
+    if (variant < KLINEAGE_NAIVE || variant > KLINEAGE_MMA_SYNC) return KLINEAGE_ERR_BAD_VARIANT;
     const int64_t lim = int64_t(1) << 31;
     if (M < 0 || N < 0 || K < 0 || M >= lim || N >= lim || K >= lim) return KLINEAGE_ERR_INVALID_ARG;
     if (M == 0 || N == 0) return KLINEAGE_OK;
@@ -172,7 +172,8 @@ klineage_status_t klineage_gemm_run(klineage_gemm_t h, int64_t M, int64_t N, int
         return KLINEAGE_OK;
     }
     const bool bcol = h->b_layout == KLINEAGE_B_COL_MAJOR;
-    if ((variant == KLINEAGE_PIPELINED || variant == KLINEAGE_TCGEN05) && h->ctx.cc_major != 10)
+    if ((variant == KLINEAGE_PIPELINED || variant == KLINEAGE_TCGEN05 || variant == KLINEAGE_MMA_SYNC) &&
+        h->ctx.cc_major != 10)
         return KLINEAGE_ERR_UNSUPPORTED_DEVICE;
 
     DeviceGuard guard(h->ctx.device);
@@ -203,6 +204,7 @@ klineage_status_t klineage_gemm_run(klineage_gemm_t h, int64_t M, int64_t N, int
             case KLINEAGE_TILED: e = launch_r1_tiled(g, s, &kid); break;
             case KLINEAGE_VECTORIZED: e = launch_r2_vectorized(g, s, &kid); break;
             case KLINEAGE_PIPELINED: e = launch_r3_pipelined(g, h->ctx, s, &kid); break;
+            case KLINEAGE_MMA_SYNC: e = launch_r35_mma_sync(g, h->ctx, s, &kid); break;
             default: e = launch_r4_tcgen05(g, h->ctx, s, &kid); break;
         }
     }
@@ -258,6 +260,7 @@ const char* klineage_variant_name(int variant)
         case KLINEAGE_VECTORIZED: return "vectorized";
         case KLINEAGE_PIPELINED: return "pipelined";
         case KLINEAGE_TCGEN05: return "tcgen05";
+        case KLINEAGE_MMA_SYNC: return "mma_sync";
         default: return "unknown";
     }
 }

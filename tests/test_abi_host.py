@@ -40,8 +40,9 @@ def test_status_and_variant_names(kb):
     assert kb.klineage_status_string(0) == "ok"
     assert kb.klineage_status_string(kb.KLINEAGE_ERR_BAD_VARIANT) == "bad variant"
     assert kb.klineage_status_string(12345) == "unknown status"
-    assert [kb.klineage_variant_name(v) for v in range(5)] == ["naive", "tiled", "vectorized", "pipelined", "tcgen05"]
-    assert kb.klineage_variant_name(5) == "unknown"
+    assert [kb.klineage_variant_name(v) for v in range(6)] == ["naive", "tiled", "vectorized", "pipelined", "tcgen05",
+                                                                "mma_sync"]
+    assert kb.klineage_variant_name(6) == "unknown"
 
 
 def test_check_args_rules(kb):
@@ -50,7 +51,8 @@ def test_check_args_rules(kb):
     ok = lambda **kw: chk(**{**dict(b_layout=0, c_dtype=0, M=8, N=9, K=10, A=A, lda=10, B=B, ldb=9, C=C, ldc=9,
                                     variant=0), **kw})
     assert ok() == kb.KLINEAGE_OK
-    assert ok(variant=5) == kb.KLINEAGE_ERR_BAD_VARIANT and ok(variant=-1) == kb.KLINEAGE_ERR_BAD_VARIANT
+    assert ok(variant=6) == kb.KLINEAGE_ERR_BAD_VARIANT and ok(variant=-1) == kb.KLINEAGE_ERR_BAD_VARIANT
+    assert ok(variant=5) == kb.KLINEAGE_OK
     assert ok(b_layout=2) == kb.KLINEAGE_ERR_INVALID_ARG and ok(c_dtype=3) == kb.KLINEAGE_ERR_INVALID_ARG
     assert ok(M=-1) == kb.KLINEAGE_ERR_INVALID_ARG and ok(K=1 << 31) == kb.KLINEAGE_ERR_INVALID_ARG
     assert ok(lda=9) == kb.KLINEAGE_ERR_INVALID_ARG

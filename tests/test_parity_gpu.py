@@ -13,8 +13,8 @@ from tests import parity as P
 
 pytestmark = pytest.mark.gpu
 
-VARIANT_NAMES = ["naive", "tiled", "vectorized", "pipelined", "tcgen05"]
-VARIANTS = list(range(5))
+VARIANT_NAMES = ["naive", "tiled", "vectorized", "pipelined", "tcgen05", "mma_sync"]
+VARIANTS = list(range(6))
 
 
 @pytest.fixture(scope="module")
@@ -243,9 +243,9 @@ def test_each_variant_reports_its_own_kernel(handles, kb):
     ragged = gen.make_config("c2", 1)
     padded = gen.make_config("c2pad", 1)
     g = handles[(False, False)]
-    expect = {("c1", 0): 0, ("c1", 1): 100, ("c1", 2): 207, ("c1", 3): 300,
-              ("c2", 0): 0, ("c2", 1): 100, ("c2", 2): 200, ("c2", 3): 301,
-              ("c2pad", 2): 207, ("c2pad", 3): 300}
+    expect = {("c1", 0): 0, ("c1", 1): 100, ("c1", 2): 207, ("c1", 3): 300, ("c1", 5): 500,
+              ("c2", 0): 0, ("c2", 1): 100, ("c2", 2): 200, ("c2", 3): 301, ("c2", 5): 501,
+              ("c2pad", 2): 207, ("c2pad", 3): 300, ("c2pad", 5): 500}
     for case in (aligned, ragged, padded):
         dev = P.DeviceCase(case)
         for v in VARIANTS:
@@ -271,7 +271,7 @@ def test_error_codes(handles, kb):
     dev = P.DeviceCase(case)
     a, b, c = dev.a.ptr, dev.b.ptr, dev.c.ptr
     run = lambda *args: g.run_raw(*args)
-    assert run(a, b, c, 64, 64, 64, 64, 64, 64, 5) == kb.KLINEAGE_ERR_BAD_VARIANT
+    assert run(a, b, c, 64, 64, 64, 64, 64, 64, 6) == kb.KLINEAGE_ERR_BAD_VARIANT
     assert run(a, b, c, 64, 64, 64, 64, 64, 64, -1) == kb.KLINEAGE_ERR_BAD_VARIANT
     assert run(a, b, c, 64, 64, 64, 63, 64, 64, 0) == kb.KLINEAGE_ERR_INVALID_ARG
     assert run(a, b, c, 64, 64, 64, 64, 63, 64, 1) == kb.KLINEAGE_ERR_INVALID_ARG
