@@ -1,5 +1,5 @@
-// Inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor, no
-// multicast form anywhere), proxy fences, tcgen05 (alloc / mma / commit / ld).
+// Inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor, always the
+// one-destination form), proxy fences, tcgen05 (alloc / mma / commit / ld).
 // Every wait is bounded: mbar_wait() gives up after a fixed number of polls and
 // returns false, so that a protocol bug ends in an error status, not a hang.
 #pragma once
@@ -190,7 +190,7 @@ __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint6
         : "memory");
 }
 // Arrive (count 1) on `bar` once every tcgen05.mma issued so far by this
-// thread has completed.  Plain form, never the multicast one.
+// thread has completed.  Plain single-barrier form only.
 __device__ __forceinline__ void umma_commit(uint64_t* bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))

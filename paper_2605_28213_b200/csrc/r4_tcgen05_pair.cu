@@ -12,7 +12,7 @@
 // per 128 x 256 x 16 instruction, alternating accumulators at the full 128.
 //
 //   warp 0      TMA producer (each CTA loads its own A box and its half of B;
-//               no multicast: every byte is fetched by exactly one CTA).  Both
+//               every byte is fetched by exactly one CTA, into its own memory).  Both
 //               CTAs' loads complete on the EVEN CTA's "full" barrier
 //               (cp.async.bulk.tensor ... .cta_group::2 lets the barrier live in
 //               the partner), which expects the bytes of both
@@ -22,7 +22,7 @@
 //               masked stores) and hand it back right after the last load
 // "Stage free" and "accumulator ready" reach both CTAs through two plain
 // tcgen05.commit instructions (own barrier, peer's barrier), never the
-// multicast form.  All waits are bounded; both CTAs pass a cluster barrier
+// cluster-wide broadcast form.  All waits are bounded; both CTAs pass a cluster barrier
 // before exit so that no remote arrive can hit shared memory of a finished CTA.
 //
 // Preconditions (paper, Introduction: intrinsics "require compatible tile

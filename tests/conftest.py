@@ -11,6 +11,11 @@ if str(ROOT) not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on a B200)")
+    # The CUDA library is built in-tree and kept out of version control: build it when a
+    # checkout has none (nvcc cross-compiles sm_100a without a GPU).  The oracle builds on demand.
+    from paper_2605_28213_b200 import build as kbuild
+    if not kbuild.LIB.exists():
+        kbuild.build()
 
 
 def pytest_collection_modifyitems(config, items):
