@@ -395,8 +395,33 @@ def lineage_table(prob_c4, kb, gen, torch, device, peaks):
                                   "frac_hbm": gbs / peaks["hbm_gbs"], "tflops": c5.flops / (med * 1e-3) / 1e12,
                                   "kernel_id": p5.gemm.last_kernel_id()}
     out["c5_16x8192x8192"] = rows
+    # c1 and c2 are launch- and occupancy-bound (report only): back-to-back launches, operands L2-resident.
+    for name in ("c1", "c2"):
+        cs = gen.make_config(name, 1)
+        ps = DeviceProblem(cs, kb, torch, device)
+        rows = {}
+        for v in LINEAGE_ORDER:
+            per_loop = 200 if v else 20
+            for _ in range(3):
+                ps.run(v)
+            torch.cuda.synchronize()
+            best = []
+            for _ in range(5):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(per_loop):
+                    ps.run(v)
+                e1.record()
+                e1.synchronize()
+                best.append(e0.elapsed_time(e1) / per_loop)
+            med = statistics.median(best)
+            rows[VARIANT_NAMES[v]] = {"us_median": med * 1e3, "us_min": min(best) * 1e3,
+                                      "tflops": cs.flops / (med * 1e-3) / 1e12, "kernel_id": ps.gemm.last_kernel_id()}
+        out[f"{name}_{cs.M}x{cs.N}x{cs.K}"] = rows
+        del ps
     out["note"] = ("c4, c3: single launches timed with CUDA events (c3 after a 256 MiB L2 flush; c4 operands exceed "
-                   "L2); c5: back-to-back launches rotating over 4 distinct weight buffers (512 MiB > L2), time per launch")
+                   "L2); c5: back-to-back launches rotating over 4 distinct weight buffers (512 MiB > L2), time per "
+                   "launch; c1, c2: back-to-back launches, operands L2-resident (launch/occupancy bound, report only)")
     return out
 
 

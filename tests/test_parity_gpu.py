@@ -170,6 +170,35 @@ def test_tcgen05_cta_pair_ragged(handles, col):
         run_and_check(handles, case, 4, C_ref, S, rows)
 
 
+# ------------------------------------------------------------------ mid-size shapes: every scheduling mode of the top rung
+MIDSIZE = [  # (M, N, K): what the shape exercises on the tcgen05 rung
+    (1500, 2100, 333),    # 12 x 9 tiles on 148 SMs: single under-filled wave cut into half tiles, N tail inside a half
+    (2304, 5120, 200),    # 360 tiles: two full waves + a 64-tile tail cut into half tiles
+    (3000, 2900, 150),    # 24 x 12 = 288 tiles: 140-tile tail, too full for half tiles
+    (200, 700, 4096),     # 2 x 3 tiles, long K: split-K through the workspace, row-block reduce, M tail
+    (130, 8192, 1024),    # 2 x 32 tiles, regular orientation, split-K
+    (4200, 4352, 136),    # CTA pairs: last 512-row tile has 104 rows (second row block and odd CTA empty)
+    (1024, 9000, 96),     # wide N with a tail, K tail
+]
+
+
+@pytest.mark.parametrize("variant", [4, 5], ids=["tcgen05", "mma_sync"])
+def test_midsize_shapes(handles, variant):
+    rng = np.random.default_rng(99)
+    for idx, (M, N, K) in enumerate(MIDSIZE):
+        col, bf = bool(idx & 1), bool(rng.integers(2))
+        case = gen.make_case(M, N, K, seed=80 + idx, dist_a="integer", dist_b="integer", b_col_major=col, c_bf16=False,
+                             name=f"mid{M}x{N}x{K}-int")
+        rows = P.sample_rows(M)
+        C_ref, S = P.oracle_rows(case, rows)
+        vals, _ = run_and_check(handles, case, variant, C_ref, S, rows, exact=True)
+        assert P.integer_checksums_match(case, vals), case.name
+        case = gen.make_case(M, N, K, seed=80 + idx, dist_a="normal", dist_b="uniform", b_col_major=not col, c_bf16=bf,
+                             name=f"mid{M}x{N}x{K}")
+        C_ref, S = P.oracle_rows(case, rows)
+        run_and_check(handles, case, variant, C_ref, S, rows)
+
+
 # ------------------------------------------------------------------ degenerate sizes
 @pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_NAMES)
 def test_degenerate_sizes(handles, kb, variant):
