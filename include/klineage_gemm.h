@@ -76,7 +76,8 @@ typedef struct {
     int device;             /* CUDA device ordinal the handle is bound to                              */
     int b_layout;           /* klineage_layout_t                                                       */
     int c_dtype;            /* klineage_ctype_t                                                        */
-    size_t workspace_bytes; /* device scratch for split-K partial sums; 0 selects the default (32 MiB) */
+    size_t workspace_bytes; /* device scratch: split-K partial sums and aligned copies of unaligned operands
+                               (rung 4); 0 selects the default (32 MiB)                                */
     unsigned flags;         /* reserved, must be 0                                                     */
 } klineage_gemm_config_t;
 
@@ -147,7 +148,7 @@ klineage_status_t klineage_gemm_get_device_status(klineage_gemm_t h, int* code_o
  *   0 naive | 100 tiled | 200 + 1*(A vector) + 2*(B vector) + 4*(C vector)
  *   300 TMA pipeline, 301 producer-thread pipeline
  *   400 + 1*(generic-proxy producer) + 2*(direct epilogue) + 4*(split-K) + 8*(skinny mode)
- *       + 16*(cluster reduce) + 32*(CTA-pair MMA)
+ *       + 16*(cluster reduce) + 32*(CTA-pair MMA) + 64*(unaligned operands repacked into the workspace)
  *   500 mma.sync rung on the TMA ring, 501 on producer threads
  *   900 zero fill (K == 0); -1 before the first run or after a no-op.
  */

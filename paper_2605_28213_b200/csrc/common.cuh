@@ -39,7 +39,8 @@ enum KernelId : int {
     kIdTiled = 100,
     kIdVectorized = 200,      // + 1 (A vector loads) + 2 (B vector loads) + 4 (C vector stores)
     kIdPipelined = 300,       // + 1 when the producer-thread path replaces TMA
-    kIdTcgen05 = 400,         // + 1 generic-proxy producer, + 2 direct epilogue, + 4 split-K, + 8 skinny (swapped operands), + 16 cluster reduce, + 32 CTA pair
+    kIdTcgen05 = 400,         // + 1 generic-proxy producer, + 2 direct epilogue, + 4 split-K, + 8 skinny (swapped operands), + 16 cluster reduce, + 32 CTA pair,
+                              // + 64 unaligned operands repacked into the workspace first
     kIdMmaSync = 500,         // rung 3.5 (mma.sync); + 1 when the producer-thread path replaces TMA
     kIdZeroFill = 900,
 };
@@ -113,6 +114,8 @@ struct RunContext {
     unsigned* tile_counters = nullptr;               // split-K arrival counters, zero between calls
     int n_tile_counters = 0;
     unsigned flags = 0;
+    bool allow_repack = true;   // rung 4 may copy unaligned operands into the workspace (needs scratch)
+    int kid_flags = 0;          // added to the kernel id a rung-4 launch reports (64 = operands repacked)
 };
 
 // Encodes a 2-D tiled tensor map (dims/strides innermost first; stride of the

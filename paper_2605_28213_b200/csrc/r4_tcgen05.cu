@@ -637,12 +637,16 @@ bool tma_ok(const void* base, int64_t ld_elems, int elt)
 
 // Chooses the number of K splits: minimise waves x (k-blocks per unit + fixed
 // per-unit cost), within the workspace and counter budgets.
-int choose_splits(int64_t tiles, int nkb, int sm, int64_t M, int64_t ldw, const RunContext& ctx)
+// `fixed` is the per-unit cost of splitting in k-block times: small for the skinny orientation
+// (coalesced partial stores, batched reduce), large for 128-row tiles, whose last arriver
+// re-reads splits x 32 x 256 floats per warp (measured: ~45 us at 1000^3, i.e. splitting
+// only pays for very long K).
+int choose_splits(int64_t tiles, int nkb, int sm, int64_t M, int64_t ldw, const RunContext& ctx, int fixed)
 {
     if (tiles * 2 > sm || nkb < 8 || tiles * 4 > ctx.n_tile_counters) return 1;
-    const int kFixed = 6;
+    const int kFixed = fixed;
     int best = 1;
-    int64_t best_cost = ((tiles + sm - 1) / sm) * (nkb + kFixed);
+    int64_t best_cost = ((tiles + sm - 1) / sm) * static_cast<int64_t>(nkb);
     for (int s = 2; s <= 32 && s * 4 <= nkb; ++s) {
         const int per = (nkb + s - 1) / s;
         const int eff = (nkb + per - 1) / per;        // splits that actually get work
@@ -697,7 +701,7 @@ SplitPlan plan_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContex
             return sp;
         }
     }
-    sp.splits = choose_splits(tiles, nkb, ctx.sm_count, M, ldw, ctx);
+    sp.splits = choose_splits(tiles, nkb, ctx.sm_count, M, ldw, ctx, sp.swap ? 6 : 100);
     return sp;
 }
 
@@ -743,7 +747,87 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
 
 }  // namespace
 
+namespace {
+
+// Copies a rows x cols bf16 matrix with an arbitrary (element-aligned) base and pitch into a
+// buffer whose pitch is a multiple of 8 elements, zero-filling the pitch padding: the
+// precondition repair that lets an unaligned operand use the TMA / tcgen05 path.  One
+// 16-byte store per thread; consecutive threads take consecutive 8-element groups.
+__global__ void __launch_bounds__(256) repack_rows_kernel(const uint16_t* __restrict__ src, int64_t ld_src,
+                                                          uint16_t* __restrict__ dst, int64_t ld_dst, int64_t rows,
+                                                          int cols)
+{
+    const int64_t groups_per_row = ld_dst >> 3;
+    const int64_t total = rows * groups_per_row;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t r = i / groups_per_row;
+        const int c0 = static_cast<int>(i - r * groups_per_row) * 8;
+        const uint16_t* s = src + r * ld_src + c0;
+        uint16_t v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = (c0 + e < cols) ? __ldg(s + e) : uint16_t(0);
+        uint4 o;
+        o.x = v[0] | (uint32_t(v[1]) << 16);
+        o.y = v[2] | (uint32_t(v[3]) << 16);
+        o.z = v[4] | (uint32_t(v[5]) << 16);
+        o.w = v[6] | (uint32_t(v[7]) << 16);
+        *reinterpret_cast<uint4*>(dst + r * ld_dst + c0) = o;
+    }
+}
+
+cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id);
+
+}  // namespace
+
+// Entry of rung 4.  Operands that break TMA's alignment rules (base not 16-byte aligned or
+// pitch not a multiple of 16 bytes) are first copied into the handle's workspace with an
+// aligned pitch when they fit there - one streaming pass over the operand, after which the
+// aligned kernels apply; otherwise the generic-proxy producers gather them tile by tile.
 cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
+{
+    const bool bad_a = !tma_ok(g.A, g.lda, 2), bad_b = !tma_ok(g.B, g.ldb, 2);
+    if (!(bad_a || bad_b) || !ctx.allow_repack || !ctx.encode_tiled) return launch_r4_planned(g, ctx, stream, kernel_id);
+    const int64_t b_rows = g.b_col ? g.N : g.K, b_cols = g.b_col ? g.K : g.N;
+    const int64_t lda2 = (static_cast<int64_t>(g.K) + 7) & ~int64_t(7), ldb2 = (b_cols + 7) & ~int64_t(7);
+    const size_t bytes_a = bad_a ? static_cast<size_t>(g.M) * lda2 * 2 : 0;
+    const size_t bytes_b = bad_b ? static_cast<size_t>(b_rows) * ldb2 * 2 : 0;
+    const size_t used = ((bytes_a + 255) & ~size_t(255)) + ((bytes_b + 255) & ~size_t(255));
+    // keep at least half of the workspace for split-K partial sums
+    if (used > ctx.workspace_bytes / 2) return launch_r4_planned(g, ctx, stream, kernel_id);
+
+    GemmArgs g2 = g;
+    uint8_t* ws = static_cast<uint8_t*>(ctx.workspace);
+    auto repack = [&](const uint16_t* src, int64_t ld_src, uint16_t* dst, int64_t ld_dst, int64_t rows, int cols) {
+        const int64_t groups = rows * (ld_dst >> 3);
+        const int64_t blocks = (groups + 255) / 256;
+        repack_rows_kernel<<<static_cast<unsigned>(blocks < 8 * 148 ? blocks : 8 * 148), 256, 0, stream>>>(
+            src, ld_src, dst, ld_dst, rows, cols);
+        return cudaGetLastError();
+    };
+    if (bad_a) {
+        cudaError_t e = repack(g.A, g.lda, reinterpret_cast<uint16_t*>(ws), lda2, g.M, g.K);
+        if (e != cudaSuccess) return e;
+        g2.A = reinterpret_cast<const uint16_t*>(ws);
+        g2.lda = lda2;
+    }
+    if (bad_b) {
+        uint16_t* dst = reinterpret_cast<uint16_t*>(ws + ((bytes_a + 255) & ~size_t(255)));
+        cudaError_t e = repack(g.B, g.ldb, dst, ldb2, b_rows, static_cast<int>(b_cols));
+        if (e != cudaSuccess) return e;
+        g2.B = dst;
+        g2.ldb = ldb2;
+    }
+    RunContext c2 = ctx;
+    c2.workspace = ws + used;
+    c2.workspace_bytes = ctx.workspace_bytes - used;
+    c2.kid_flags = 64;
+    return launch_r4_planned(g2, c2, stream, kernel_id);
+}
+
+namespace {
+
+cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
 {
     if (ctx.max_smem_optin < kSmemBytes) return cudaErrorInvalidConfiguration;
     const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN;
@@ -771,7 +855,13 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     // Skinny mode: few activation rows -> they become the MMA's N, the weights its 128 rows.
     const bool swap = plan.swap;
     p.n_mma = (g.M + 15) & ~15;
-    p.epi_tma = (!swap && p.splits == 1 && ctx.encode_tiled && tma_ok(g.C, g.ldc, celt)) ? 1 : 0;
+    // TMA store needs C 16-byte aligned with a 16-byte-multiple pitch, and a row length that is a
+    // multiple of 16 bytes: measured on B200, a store box that ends inside a 16-byte unit at the
+    // right edge of the tensor writes that whole unit, i.e. up to 12 bytes of row padding.
+    p.epi_tma = (!swap && p.splits == 1 && ctx.encode_tiled && tma_ok(g.C, g.ldc, celt) &&
+                 (static_cast<int64_t>(g.N) * celt) % 16 == 0)
+                    ? 1
+                    : 0;
 
     // Instruction descriptor: fp32 accumulator (bits 4-5), bf16 A and B (bits 7-9, 10-12),
     // operand majors (bit 15 A, bit 16 B; 0 = K-major, 1 = MN-major), N >> 3 (bits 17-22),
@@ -815,7 +905,7 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     if (!ok) return cudaErrorInvalidValue;
 
     p.kid = kIdTcgen05 + (generic ? 1 : 0) + (p.epi_tma ? 0 : 2) + (p.splits > 1 ? 4 : 0) + (swap ? 8 : 0) +
-            (p.cluster ? 16 : 0);
+            (p.cluster ? 16 : 0) + ctx.kid_flags;
     *kernel_id = p.kid;
     // Static schedule.  Without a K split, a last wave that would leave at least half of the
     // SMs idle is cut into 128-column half tiles (twice as many units, half as long).
@@ -839,6 +929,8 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     return generic ? KLIN_R4_LAUNCH(false, true, false) : KLIN_R4_LAUNCH(false, false, false);
 #undef KLIN_R4_LAUNCH
 }
+
+}  // namespace
 
 }  // namespace klin
 
@@ -909,6 +1001,7 @@ klineage_status_t noalloc_setup(int device, NoAllocDevice** out)
         c.tile_counters = reinterpret_cast<unsigned*>(ptr + kNoAllocPartialBytes);
         c.n_tile_counters = kNoAllocCounters;
         d.status = c.tile_counters + kNoAllocCounters;
+        c.allow_repack = false;   // its fixed scratch is reserved for split-K partial sums
         d.ready = true;
     }
     *out = &d;

@@ -428,8 +428,10 @@ cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStrea
     p.nkb = (g.K + BK - 1) / BK;
     p.group_m = 4;                                  // 4 x 512 rows per raster group
     const int celt = g.c_bf16 ? 2 : 4;
+    // (row length a multiple of 16 bytes too: a store box ending inside a 16-byte unit at the tensor's
+    // right edge writes the whole unit)
     p.epi_tma = (reinterpret_cast<uintptr_t>(g.C) % 16 == 0 && (g.ldc * celt) % 16 == 0 &&
-                 g.ldc * celt < (int64_t(1) << 40))
+                 (static_cast<int64_t>(g.N) * celt) % 16 == 0 && g.ldc * celt < (int64_t(1) << 40))
                     ? 1
                     : 0;
     // Instruction descriptor: fp32 accumulator, bf16 A/B, A K-major, B K-major (column-major B) or
@@ -460,7 +462,7 @@ cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStrea
                                  g.C, g.N, g.M, g.ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return cudaErrorInvalidValue;
 
-    p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + 32;
+    p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + 32 + ctx.kid_flags;
     *kernel_id = p.kid;
     const int64_t max_pairs = ctx.sm_count / 2;
     const unsigned grid = 2u * static_cast<unsigned>(p.total_tiles < max_pairs ? p.total_tiles : max_pairs);

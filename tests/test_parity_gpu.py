@@ -32,6 +32,17 @@ def handles(kb):
         h.close()
 
 
+@pytest.fixture(scope="module")
+def handles_tiny_ws(kb):
+    """Handles whose workspace is too small for operand repacking or split-K partials: on the tcgen05 rung
+    unaligned operands then go through the generic-proxy producers."""
+    hs = {(col, bf): kb.Gemm(0, b_col_major=col, c_bf16=bf, workspace_bytes=4096)
+          for col in (False, True) for bf in (False, True)}
+    yield hs
+    for h in hs.values():
+        h.close()
+
+
 def run_and_check(handles, case, variant, C_ref=None, S=None, rows=None, exact=False, offsets=(0, 0, 0)):
     dev = P.DeviceCase(case, *offsets)
     dev.run(handles[(case.b_col_major, case.c_bf16)], variant)
@@ -116,6 +127,26 @@ def test_random_small_shapes(handles, variant):
         run_and_check(handles, case, variant, offsets=tuple(int(rng.integers(0, 3)) for _ in range(3)))
 
 
+# ------------------------------------------------------------------ generic-proxy producers of the top rung
+@pytest.mark.parametrize("col", [False, True], ids=["Brow", "Bcol"])
+def test_tcgen05_generic_producers(handles_tiny_ws, col):
+    """With no room to repack, unaligned operands are gathered tile by tile into the swizzled layout."""
+    shapes = [(1000, 1001, 999, (0, 0, 0)), (130, 270, 100, (1, 1, 1)), (16, 1001, 2051, (1, 0, 1)),
+              (300, 520, 200, (1, 1, 0)), (64, 64, 64, (1, 1, 1)), (257, 513, 129, (0, 1, 0))]
+    for idx, (M, N, K, offs) in enumerate(shapes):
+        for bf in (False, True):
+            case = gen.make_case(M, N, K, seed=120 + idx, dist_a="integer", dist_b="integer", b_col_major=col,
+                                 c_bf16=bf, lda=K + (K % 2 == 0), ldb=(K if col else N) + ((K if col else N) % 2 == 0),
+                                 ldc=N + 1, name=f"generic{M}x{N}x{K}-int")
+            run_and_check(handles_tiny_ws, case, 4, exact=True, offsets=offs)
+            flags = handles_tiny_ws[(col, bf)].last_kernel_id() - 400
+            assert (flags & 1) and not (flags & 64), (M, N, K, flags)
+        case = gen.make_case(M, N, K, seed=120 + idx, dist_a="normal", dist_b="uniform", b_col_major=col,
+                             lda=K + (K % 2 == 0), ldb=(K if col else N) + ((K if col else N) % 2 == 0),
+                             name=f"generic{M}x{N}x{K}")
+        run_and_check(handles_tiny_ws, case, 4, offsets=offs)
+
+
 # ------------------------------------------------------------------ skinny shapes of the top rung
 SKINNY = [  # (M, N, K, expected flags of kernel id - 400: 4 split-K, 8 swapped operands, 16 cluster reduce)
     (16, 1024, 8192, 4 | 8 | 16),      # 4 tiles: cluster of 8
@@ -124,7 +155,7 @@ SKINNY = [  # (M, N, K, expected flags of kernel id - 400: 4 split-K, 8 swapped 
     (32, 1000, 4096, 4 | 8 | 16),      # M = 32: largest cluster-reduced M, ragged N
     (33, 1000, 4096, 4 | 8),           # M = 33: swapped, split through the global workspace
     (64, 520, 2048, 4 | 8),            # M = 64: last swapped M
-    (65, 520, 2048, 4),                # M = 65: regular orientation, split-K with row-block reduce
+    (65, 520, 32768, 4),               # M = 65: regular orientation, K long enough for split-K with row-block reduce
     (16, 256, 64, 8),                  # one tile, one k-block: no split
     (1, 8192, 8192, 4 | 8 | 16),       # GEMV
 ]
@@ -146,13 +177,21 @@ def test_tcgen05_skinny_modes(handles, col):
     case = gen.make_case(16, 1001, 4099, seed=77, dist_a="integer", dist_b="integer", b_col_major=col, lda=4101,
                          ldb=(4099 if col else 1001) + 2, ldc=1003, name="skinny-unaligned")
     run_and_check(handles, case, 4, exact=True, offsets=(1, 1, 1))
-    assert (handles[(col, False)].last_kernel_id() - 400) & 1
+    assert (handles[(col, False)].last_kernel_id() - 400) & 64, "unaligned operands that fit are repacked"
 
 
 # ------------------------------------------------------------------ CTA-pair form of the top rung
 @pytest.mark.parametrize("col", [False, True], ids=["Brow", "Bcol"])
 def test_tcgen05_cta_pair_ragged(handles, col):
     """Large aligned shapes run on tcgen05.mma.cta_group::2 (512 x 256 pair tiles); tails in M, N and K."""
+    # aligned pitch but a row length that ends inside a 16-byte unit: C padding must stay untouched
+    for bf in (False, True):
+        case = gen.make_case(4608, 4350 + (0 if bf else 1), 64, seed=59, dist_a="integer", dist_b="integer",
+                             b_col_major=col, c_bf16=bf, lda=64, ldb=(64 if col else 4352), ldc=4352,
+                             name="pair-ragged-row-end")
+        rows = P.sample_rows(case.M)
+        C_ref, S = P.oracle_rows(case, rows)
+        run_and_check(handles, case, 4, C_ref, S, rows, exact=True)
     for idx, (M, N, K) in enumerate([(5000, 5200, 1000), (4608, 4352, 72)]):
         for bf in (False, True):
             case = gen.make_case(M, N, K, seed=60 + idx, dist_a="integer", dist_b="integer", b_col_major=col,
@@ -175,8 +214,8 @@ MIDSIZE = [  # (M, N, K): what the shape exercises on the tcgen05 rung
     (1500, 2100, 333),    # 12 x 9 tiles on 148 SMs: single under-filled wave cut into half tiles, N tail inside a half
     (2304, 5120, 200),    # 360 tiles: two full waves + a 64-tile tail cut into half tiles
     (3000, 2900, 150),    # 24 x 12 = 288 tiles: 140-tile tail, too full for half tiles
-    (200, 700, 4096),     # 2 x 3 tiles, long K: split-K through the workspace, row-block reduce, M tail
-    (130, 8192, 1024),    # 2 x 32 tiles, regular orientation, split-K
+    (200, 700, 30000),    # 2 x 3 tiles, very long K: split-K through the workspace, row-block reduce, M tail
+    (130, 8192, 1024),    # 2 x 32 tiles of 128 rows, half tiles
     (4200, 4352, 136),    # CTA pairs: last 512-row tile has 104 rows (second row block and odd CTA empty)
     (1024, 9000, 96),     # wide N with a tail, K tail
 ]
@@ -282,8 +321,9 @@ def test_each_variant_reports_its_own_kernel(handles, kb):
             code, dev_id = g.device_status()
             assert code == 0 and dev_id == g.last_kernel_id()
             if v == 4:
-                assert 400 <= dev_id < 464
-                assert ((dev_id - 400) & 1) == (1 if case.name == "c2" else 0)   # generic producer only when unaligned
+                assert 400 <= dev_id < 528
+                # unaligned operands are repacked into the workspace (flag 64), never gathered, when they fit
+                assert ((dev_id - 400) & 1) == 0 and bool((dev_id - 400) & 64) == (case.name == "c2")
             else:
                 want = expect.get((case.name, v))
                 if want is not None:

@@ -57,7 +57,7 @@ def test_no_alloc_matches_handle_path_on_two_calls_in_a_row():
 
     # taller tile, split along K with the row-block reduce; and a decode-like M=16 shape (cluster reduce,
     # no global scratch) plus a ragged column-major bf16 case without any split: same call, same bits
-    for case in (gen.make_case(200, 512, 4096, seed=7, dist_a="integer", dist_b="integer", name="tall"),
+    for case in (gen.make_case(200, 256, 30016, seed=7, dist_a="integer", dist_b="integer", name="tall"),
                  gen.make_case(16, 2048, 4096, seed=8, dist_a="normal", dist_b="normal", name="decode"),
                  gen.make_case(300, 520, 200, seed=6, dist_a="integer", dist_b="integer", b_col_major=True,
                                c_bf16=True, name="ragged")):
@@ -69,8 +69,8 @@ def test_no_alloc_matches_handle_path_on_two_calls_in_a_row():
 def test_no_alloc_refuses_shapes_beyond_its_fixed_scratch():
     import torch
     from paper_2605_28213_b200 import binding as kb
-    # 2 splits x 2048 x 1024 fp32 partial sums = 16 MiB > the 8 MiB the library reserves
-    M, N, K = 2048, 1024, 4096
+    # a K long enough to be split, and splits x 2048 x 1024 fp32 partial sums >= 16 MiB > the 8 MiB reserved
+    M, N, K = 2048, 1024, 65536
     A = torch.zeros(M * K, dtype=torch.int16, device="cuda")
     B = torch.zeros(K * N, dtype=torch.int16, device="cuda")
     C = torch.full((M * N,), 7.0, dtype=torch.float32, device="cuda")
