@@ -77,7 +77,7 @@ typedef struct {
     int b_layout;           /* klineage_layout_t                                                       */
     int c_dtype;            /* klineage_ctype_t                                                        */
     size_t workspace_bytes; /* device scratch: split-K partial sums and aligned copies of unaligned operands
-                               (rung 4); 0 selects the default (32 MiB)                                */
+                               (rung 4); 0 selects the default (64 MiB)                                */
     unsigned flags;         /* reserved, must be 0                                                     */
 } klineage_gemm_config_t;
 

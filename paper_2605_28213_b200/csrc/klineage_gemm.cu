@@ -38,7 +38,7 @@ bool encode_map_2d(const RunContext& ctx, CUtensorMap* map, CUtensorMapDataType 
 
 namespace {
 
-constexpr size_t kDefaultWorkspace = 32u << 20;
+constexpr size_t kDefaultWorkspace = 64u << 20;
 constexpr int kTileCounters = 4096;
 
 // Restores the caller's current device on scope exit.
