@@ -305,6 +305,12 @@ def run_gpu(args):
            "h2d_bytes_per_step": int(hA.numel() * 2 + hB.numel() * 2), "d2h_bytes_per_step": int(hC.numel() * hC.element_size()),
            "steps": e2e_steps}
 
+    # kernels of this library per step: the GEMM kernel, plus one repack kernel per operand that
+    # breaks TMA's alignment rules when the tcgen05 rung copies it into the workspace (kernel-id flag 64)
+    launches_per_step = 1
+    if V == 4 and (kid - 400) & 64:
+        launches_per_step += int(prob.A.data_ptr() % 16 != 0 or case.lda % 8 != 0)
+        launches_per_step += int(prob.B.data_ptr() % 16 != 0 or case.ldb % 8 != 0)
     line = {
         "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -314,7 +320,7 @@ def run_gpu(args):
                    "parallelism": f"{world} independent GEMMs",
                    "l2": (f"{len(rot)} distinct B buffers rotated ({len(rot) * case.B.nbytes >> 20} MiB > L2); no flush"
                           if small else "A+B+C = 384 MiB exceed the 126 MB L2; no flush between iterations")},
-        "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": args.steps,
+        "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": args.steps * launches_per_step,
         "parity_checked": parity_ok, "device_status": code, "kernel_id": kid,
     }
     per_gpu = tflops / world
