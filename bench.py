@@ -375,6 +375,24 @@ def lineage_table(prob_c4, kb, gen, torch, device, peaks):
                                   "frac_bf16_peak": c3.flops / (med * 1e-3) / 1e12 / peaks["bf16_tflops"],
                                   "kernel_id": p3.gemm.last_kernel_id()}
     out["c3_4096^3_Bcol"] = rows
+    # AddMM at the same shape (the paper's held-out AddMM instance is 4096^3): bias epilogue fused, top rungs only
+    bias = torch.from_numpy(gen.draw((1, c3.N), "normal", 1, 2)[0].view("int16")).to(device)
+    rows = {}
+    for v in (5, 4):
+        times = []
+        for i in range(13):
+            flush.fill_(i)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            p3.gemm.run_addmm(p3.A, p3.B, bias, p3.C, c3.M, c3.N, c3.K, c3.lda, c3.ldb, c3.ldc, v)
+            e1.record()
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1))
+        med = statistics.median(times[3:])
+        rows[VARIANT_NAMES[v]] = {"ms_median": med, "tflops": c3.flops / (med * 1e-3) / 1e12,
+                                  "frac_bf16_peak": c3.flops / (med * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                  "kernel_id": p3.gemm.last_kernel_id()}
+    out["addmm_4096^3_Bcol"] = rows
     del p3
 
     c5 = gen.make_config("c5", 1)

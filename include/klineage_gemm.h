@@ -119,6 +119,19 @@ klineage_status_t klineage_gemm_run(klineage_gemm_t h, int64_t M, int64_t N, int
                                     void* C, int64_t ldc, int variant, void* stream);
 
 /*
+ * AddMM:  C <- A . B + bias,  bias a vector of N bf16 values (device, 2-byte aligned,
+ * not overlapping C) added to every row - the bias-epilogue fusion of the paper's
+ * held-out plain-GEMM family (Appendix D, "Additional Held-out Verification": AddMM at
+ * 4096^3).  The bias is added to the fp32 accumulator before the rounding to bf16 (bf16 C);
+ * with a K split it is added once, by the final reduction.  K == 0 gives C[i][j] = bias[j].
+ * Every other argument, rule and error is that of klineage_gemm_run; bias == NULL with
+ * M*N > 0 is INVALID_ARG.
+ */
+klineage_status_t klineage_gemm_run_addmm(klineage_gemm_t h, int64_t M, int64_t N, int64_t K,
+                                          const void* A, int64_t lda, const void* B, int64_t ldb,
+                                          const void* bias, void* C, int64_t ldc, int variant, void* stream);
+
+/*
  * The host-side argument checks of klineage_gemm_run, callable without a handle
  * or a device (pointers are only compared, never dereferenced).  Returns what
  * run would return for these arguments before touching the GPU: OK,

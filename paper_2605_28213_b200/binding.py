@@ -33,7 +33,7 @@ VARIANTS = (KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELI
 EXPORTED_SYMBOLS = (
     "klineage_gemm_create", "klineage_gemm_run", "klineage_gemm_destroy", "klineage_gemm_check_args",
     "klineage_gemm_get_device_status", "klineage_gemm_last_kernel_id", "klineage_status_string",
-    "klineage_variant_name", "klineage_gemm_run_noalloc",
+    "klineage_variant_name", "klineage_gemm_run_noalloc", "klineage_gemm_run_addmm",
 )
 
 
@@ -86,6 +86,15 @@ def klineage_gemm_run_noalloc(b_layout, c_dtype, M, N, K, A, lda, B, ldb, C, ldc
     one-stream-at-a-time rule.
     """
     return _lib.klineage_gemm_run_noalloc(b_layout, c_dtype, M, N, K, A, lda, B, ldb, C, ldc, stream)
+
+
+_lib.klineage_gemm_run_addmm.restype = _int
+_lib.klineage_gemm_run_addmm.argtypes = [_p, _i64, _i64, _i64, _p, _i64, _p, _i64, _p, _p, _i64, _int, _p]
+
+
+def klineage_gemm_run_addmm_raw(h, M, N, K, A, lda, B, ldb, bias, C, ldc, variant, stream) -> int:
+    """Raw status of C <- A.B + bias (bias: N bf16 values on the device)."""
+    return _lib.klineage_gemm_run_addmm(h, M, N, K, A, lda, B, ldb, bias, C, ldc, variant, stream)
 
 
 def klineage_status_string(status: int) -> str:
@@ -175,6 +184,12 @@ class Gemm:
     def run(self, A, B, C, M, N, K, lda, ldb, ldc, variant, stream=None) -> None:
         klineage_gemm_run(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(C), ldc,
                           int(variant), self._stream(stream))
+
+    def run_addmm(self, A, B, bias, C, M, N, K, lda, ldb, ldc, variant, stream=None) -> None:
+        st = klineage_gemm_run_addmm_raw(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(bias),
+                                         self._ptr(C), ldc, int(variant), self._stream(stream))
+        if st != KLINEAGE_OK:
+            raise KlineageError(st, "klineage_gemm_run_addmm")
 
     def run_raw(self, A, B, C, M, N, K, lda, ldb, ldc, variant, stream=None) -> int:
         return klineage_gemm_run_raw(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(C),

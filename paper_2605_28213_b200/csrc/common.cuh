@@ -25,6 +25,7 @@ struct GemmArgs {
     int b_col;
     int c_bf16;
     unsigned* status;
+    const uint16_t* bias;   // optional: N bf16 values added to every row of A.B (AddMM); nullptr = plain GEMM
 };
 
 // Device-side error codes written to status[0].
@@ -61,6 +62,12 @@ __device__ __forceinline__ uint16_t float_to_bf16_bits(float f)
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     return static_cast<uint32_t>(float_to_bf16_bits(lo)) | (static_cast<uint32_t>(float_to_bf16_bits(hi)) << 16);
+}
+
+// The bias of column `col` (0 when the call has none); col must be < N.
+__device__ __forceinline__ float bias_at(const GemmArgs& g, int64_t col)
+{
+    return g.bias ? bf16_bits_to_float(__ldg(g.bias + col)) : 0.f;
 }
 
 __device__ __forceinline__ void store_c(void* C, int c_bf16, int64_t idx, float v)

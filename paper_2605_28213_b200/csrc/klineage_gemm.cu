@@ -161,8 +161,12 @@ klineage_status_t klineage_gemm_check_args(int b_layout, int c_dtype, int64_t M,
     return KLINEAGE_OK;
 }
 
-klineage_status_t klineage_gemm_run(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
-                                    const void* B, int64_t ldb, void* C, int64_t ldc, int variant, void* stream)
+}  // extern "C"
+
+// Shared body of klineage_gemm_run (bias == nullptr) and klineage_gemm_run_addmm.
+static klineage_status_t run_impl(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                  const void* B, int64_t ldb, const void* bias, void* C, int64_t ldc, int variant,
+                                  void* stream)
 {
     if (!h) return KLINEAGE_ERR_INVALID_ARG;
     const klineage_status_t chk = klineage_gemm_check_args(h->b_layout, h->c_dtype, M, N, K, A, lda, B, ldb, C, ldc, variant);
@@ -192,6 +196,7 @@ klineage_status_t klineage_gemm_run(klineage_gemm_t h, int64_t M, int64_t N, int
     g.b_col = bcol ? 1 : 0;
     g.c_bf16 = h->c_dtype == KLINEAGE_C_BF16 ? 1 : 0;
     g.status = h->status;
+    g.bias = static_cast<const uint16_t*>(bias);
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int kid = -1;
@@ -214,6 +219,30 @@ klineage_status_t klineage_gemm_run(klineage_gemm_t h, int64_t M, int64_t N, int
     }
     h->last_kernel_id = kid;
     return KLINEAGE_OK;
+}
+
+extern "C" {
+
+klineage_status_t klineage_gemm_run(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                    const void* B, int64_t ldb, void* C, int64_t ldc, int variant, void* stream)
+{
+    return run_impl(h, M, N, K, A, lda, B, ldb, nullptr, C, ldc, variant, stream);
+}
+
+klineage_status_t klineage_gemm_run_addmm(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A,
+                                          int64_t lda, const void* B, int64_t ldb, const void* bias, void* C,
+                                          int64_t ldc, int variant, void* stream)
+{
+    if (!h) return KLINEAGE_ERR_INVALID_ARG;
+    if (M > 0 && N > 0) {
+        if (!bias || reinterpret_cast<uintptr_t>(bias) % 2) return KLINEAGE_ERR_INVALID_ARG;
+        if (C && N > 0 && M > 0 && ldc >= N) {
+            const size_t celt = h->c_dtype == KLINEAGE_C_BF16 ? 2 : 4;
+            const size_t c_bytes = (size_t(M - 1) * ldc + N) * celt;
+            if (ranges_overlap(bias, size_t(N) * 2, C, c_bytes)) return KLINEAGE_ERR_INVALID_ARG;
+        }
+    }
+    return run_impl(h, M, N, K, A, lda, B, ldb, bias, C, ldc, variant, stream);
 }
 
 klineage_status_t klineage_gemm_get_device_status(klineage_gemm_t h, int* code_out, int* kernel_id_out)

@@ -25,7 +25,7 @@ __global__ void __launch_bounds__(kBx* kBy) r0_naive_kernel(GemmArgs g, int tile
             for (int k = 0; k < g.K; ++k)
                 acc = fmaf(bf16_bits_to_float(a[k]), bf16_bits_to_float(b[static_cast<int64_t>(k) * g.ldb]), acc);
         }
-        store_c(g.C, g.c_bf16, i * g.ldc + j, acc);
+        store_c(g.C, g.c_bf16, i * g.ldc + j, acc + bias_at(g, j));
     }
 }
 
@@ -35,7 +35,7 @@ __global__ void zero_fill_kernel(GemmArgs g)
     const int64_t total = static_cast<int64_t>(g.M) * g.N;
     for (int64_t e = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; e < total;
          e += static_cast<int64_t>(gridDim.x) * blockDim.x)
-        store_c(g.C, g.c_bf16, (e / g.N) * g.ldc + (e % g.N), 0.f);
+        store_c(g.C, g.c_bf16, (e / g.N) * g.ldc + (e % g.N), 0.f + bias_at(g, e % g.N));
 }
 
 }  // namespace

@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(NT) r1_tiled_kernel(GemmArgs g, int tiles_m, i
 #pragma unroll
         for (int j = 0; j < TN; ++j) {
             const int64_t gn = n0 + tx * TN + j;
-            if (gn < g.N) store_c(g.C, g.c_bf16, gm * g.ldc + gn, acc[i][j]);
+            if (gn < g.N) store_c(g.C, g.c_bf16, gm * g.ldc + gn, acc[i][j] + bias_at(g, gn));
         }
     }
 }

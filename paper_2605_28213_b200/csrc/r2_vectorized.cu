@@ -104,7 +104,9 @@ r2_vectorized_kernel(GemmArgs g, int tiles_m, int tiles_n, int a_vec, int b_vec,
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int gn = n0 + h * 64 + tx * 4;
-            const float* v = &acc[i][h * 4];
+            float v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = acc[i][h * 4 + j] + (gn + j < g.N ? bias_at(g, gn + j) : 0.f);
             if (c_vec && gn + 4 <= g.N) {
                 if (g.c_bf16) {
                     uint2 w = make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));

@@ -271,7 +271,8 @@ r35_mma_sync_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int gn = n0 + wn + j * 8 + (lane & 3) * 2;
-                const float v0 = acc[i][j][h * 2], v1 = acc[i][j][h * 2 + 1];
+                const float v0 = acc[i][j][h * 2] + (gn < g.N ? bias_at(g, gn) : 0.f);
+                const float v1 = acc[i][j][h * 2 + 1] + (gn + 1 < g.N ? bias_at(g, gn + 1) : 0.f);
                 if (g.c_bf16) {
                     uint16_t* d = static_cast<uint16_t*>(g.C) + gm * g.ldc + gn;
                     if (gn + 1 < g.N && (reinterpret_cast<uintptr_t>(d) & 3) == 0) {

@@ -269,6 +269,15 @@ r3_pipelined_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
             acc[i][2 * jp] = acc2[i][jp].x;
             acc[i][2 * jp + 1] = acc2[i][jp].y;
         }
+    if (g.bias) {   // AddMM: the bias of each of this thread's 8 columns
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int gn = n0 + (BCOL ? tx + 16 * j : tx * 8 + j);
+            const float b = gn < g.N ? bias_at(g, gn) : 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i][j] += b;
+        }
+    }
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int64_t gm = m0 + ty + 16 * i;

@@ -351,8 +351,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
 #pragma unroll
                             for (int j = 0; j < 16; ++j) ptx::st_cluster_f32(remote + j * 128, __uint_as_float(v[j]));
                         } else if (n < g.N) {
+                            const float bn = partial ? 0.f : bias_at(g, n);
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
+                                v[j] = __float_as_uint(__uint_as_float(v[j]) + bn);
                                 const int m = mc + j;
                                 if (m < g.M) {
                                     if (out_bf16)
@@ -407,7 +409,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                                     }
 #pragma unroll
                                     for (int j = 0; j < 16; ++j)
-                                        if (mb + j < g.M) store_c(g.C, g.c_bf16, (mb + j) * g.ldc + n, acc[j]);
+                                        if (mb + j < g.M) store_c(g.C, g.c_bf16, (mb + j) * g.ldc + n, acc[j] + bias_at(g, n));
                                 }
                             }
                             __syncwarp();
@@ -437,6 +439,14 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         uint32_t v2[32];
                         ptx::tmem_ld_32x32b_x32(taddr + 32, v2);
                         ptx::tmem_ld_wait();
+                        if (g.bias) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                v[i] = __float_as_uint(__uint_as_float(v[i]) + (col0 + i < g.N ? bias_at(g, col0 + i) : 0.f));
+                                v2[i] = __float_as_uint(__uint_as_float(v2[i]) +
+                                                        (col0 + 32 + i < g.N ? bias_at(g, col0 + 32 + i) : 0.f));
+                            }
+                        }
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             w[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
@@ -444,10 +454,15 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         }
                     } else {
                         ptx::tmem_ld_wait();
+                        if (g.bias && !partial) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                v[i] = __float_as_uint(__uint_as_float(v[i]) + (col0 + i < g.N ? bias_at(g, col0 + i) : 0.f));
+                        }
 #pragma unroll
                         for (int i = 0; i < 32; ++i) w[i] = v[i];
                     }
-                    uint8_t* b = stg + (nstaged++ & 1) * kEpiBufBytes;
+                    uint8_t* b = stg + (nstaged++ & 1) * kEpiBufBytes;   // (bias was added above)
                     if (use_tma) {
                         if (lane == 0) ptx::tma_store_wait_read<1>();   // the store that last read this buffer
                         __syncwarp();
@@ -520,7 +535,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                             const float o[4] = {acc.x, acc.y, acc.z, acc.w};
 #pragma unroll
                             for (int e = 0; e < 4; ++e)
-                                if (col + e < g.N) store_c(g.C, g.c_bf16, row * g.ldc + col + e, o[e]);
+                                if (col + e < g.N) store_c(g.C, g.c_bf16, row * g.ldc + col + e, o[e] + bias_at(g, col + e));
                         }
                     }
                     __syncwarp();
@@ -615,7 +630,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     }
 #pragma unroll
                     for (int r = 0; r < 4; ++r)
-                        if (mb + 4 * r < g.M) store_c(g.C, g.c_bf16, static_cast<int64_t>(mb + 4 * r) * g.ldc + n, acc[r]);
+                        if (mb + 4 * r < g.M)
+                            store_c(g.C, g.c_bf16, static_cast<int64_t>(mb + 4 * r) * g.ldc + n, acc[r] + bias_at(g, n));
                 }
             }
         }
@@ -1044,6 +1060,7 @@ extern "C" klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype
     g.b_col = b_layout == KLINEAGE_B_COL_MAJOR ? 1 : 0;
     g.c_bf16 = c_dtype == KLINEAGE_C_BF16 ? 1 : 0;
     g.status = d->status;
+    g.bias = nullptr;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int kid = -1;

@@ -119,6 +119,21 @@ def test_hand_worked_example():
         assert np.array_equal(got, rows["C_BF16"].astype(np.float32))
 
 
+def test_addmm_reference_is_product_plus_row_bias():
+    """The AddMM reference used by the GPU tests: oracle product + bias broadcast along rows, in fp64."""
+    rows = {}
+    for line in (GOLDEN / "hand_worked_2x3x2.txt").read_text().splitlines():
+        if line and not line.startswith("#"):
+            key, *vals = line.split()
+            rows[key] = np.array([float(v) for v in vals])
+    A, B = bits_of(rows["A"].reshape(2, 3)), bits_of(rows["B"].reshape(3, 2))
+    bias = bits_of([0.5, -2.0])
+    C, S = run_oracle(A, B)
+    got = C + orc.bf16_bits_to_f64(bias)[None, :]
+    # by hand: C = [[0, -4.71875], [-139.5, 3.5]]  ->  [[0.5, -6.71875], [-139, 1.5]]
+    assert np.array_equal(got, np.array([[0.5, -6.71875], [-139.0, 1.5]]))
+
+
 # ------------------------------------------------------------- index / layout
 def test_identity_left_and_right():
     B = gen.draw((37, 53), "normal", 5, 1)
