@@ -439,12 +439,13 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         uint32_t v2[32];
                         ptx::tmem_ld_32x32b_x32(taddr + 32, v2);
                         ptx::tmem_ld_wait();
-                        if (g.bias) {
+                        if (g.bias) {   // lane l fetches two columns' bias, shuffles hand them round
+                            const float b0 = (col0 + lane < g.N) ? bias_at(g, col0 + lane) : 0.f;
+                            const float b1 = (col0 + 32 + lane < g.N) ? bias_at(g, col0 + 32 + lane) : 0.f;
 #pragma unroll
                             for (int i = 0; i < 32; ++i) {
-                                v[i] = __float_as_uint(__uint_as_float(v[i]) + (col0 + i < g.N ? bias_at(g, col0 + i) : 0.f));
-                                v2[i] = __float_as_uint(__uint_as_float(v2[i]) +
-                                                        (col0 + 32 + i < g.N ? bias_at(g, col0 + 32 + i) : 0.f));
+                                v[i] = __float_as_uint(__uint_as_float(v[i]) + __shfl_sync(0xFFFFFFFFu, b0, i));
+                                v2[i] = __float_as_uint(__uint_as_float(v2[i]) + __shfl_sync(0xFFFFFFFFu, b1, i));
                             }
                         }
 #pragma unroll
@@ -455,9 +456,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     } else {
                         ptx::tmem_ld_wait();
                         if (g.bias && !partial) {
+                            const float b0 = (col0 + lane < g.N) ? bias_at(g, col0 + lane) : 0.f;
 #pragma unroll
                             for (int i = 0; i < 32; ++i)
-                                v[i] = __float_as_uint(__uint_as_float(v[i]) + (col0 + i < g.N ? bias_at(g, col0 + i) : 0.f));
+                                v[i] = __float_as_uint(__uint_as_float(v[i]) + __shfl_sync(0xFFFFFFFFu, b0, i));
                         }
 #pragma unroll
                         for (int i = 0; i < 32; ++i) w[i] = v[i];

@@ -297,12 +297,14 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             auto finish = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32]) {
                 const int col0 = n0 + u * cpc;
                 if (g.bias) {   // AddMM: this unit's columns get their bias in fp32, before any rounding
+                    // lane l fetches the bias of columns col0 + l and col0 + 32 + l; a shuffle hands column i's
+                    // value to every lane (every lane holds a different row of the same columns)
+                    const float b0 = (col0 + lane < g.N) ? bias_at(g, col0 + lane) : 0.f;
+                    const float b1 = (out_bf16 && col0 + 32 + lane < g.N) ? bias_at(g, col0 + 32 + lane) : 0.f;
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        r0[i] = __float_as_uint(__uint_as_float(r0[i]) + (col0 + i < g.N ? bias_at(g, col0 + i) : 0.f));
-                        if (out_bf16)
-                            r1[i] = __float_as_uint(__uint_as_float(r1[i]) +
-                                                    (col0 + 32 + i < g.N ? bias_at(g, col0 + 32 + i) : 0.f));
+                        r0[i] = __float_as_uint(__uint_as_float(r0[i]) + __shfl_sync(0xFFFFFFFFu, b0, i));
+                        if (out_bf16) r1[i] = __float_as_uint(__uint_as_float(r1[i]) + __shfl_sync(0xFFFFFFFFu, b1, i));
                     }
                 }
                 uint32_t w[32];
