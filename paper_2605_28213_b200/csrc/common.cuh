@@ -94,6 +94,18 @@ __host__ __device__ __forceinline__ void raster_tile(int64_t t, int tiles_m, int
                                                      int group_m = kGroupM)
 {
     const int64_t per_group = static_cast<int64_t>(group_m) * tiles_n;
+    if (t < 0x7FFFFFFFll && per_group < 0x7FFFFFFFll) {
+        // the common case in 32-bit arithmetic: a 64-bit division costs hundreds of cycles on the
+        // critical path of short kernels
+        const uint32_t t32 = static_cast<uint32_t>(t), pg = static_cast<uint32_t>(per_group);
+        const uint32_t g = t32 / pg;
+        const int first_m = static_cast<int>(g) * group_m;
+        const uint32_t rows = static_cast<uint32_t>((tiles_m - first_m < group_m) ? (tiles_m - first_m) : group_m);
+        const uint32_t r = t32 - g * pg;
+        tm = first_m + static_cast<int>(r % rows);
+        tn = static_cast<int>(r / rows);
+        return;
+    }
     const int g = static_cast<int>(t / per_group);
     const int first_m = g * group_m;
     const int rows = (tiles_m - first_m < group_m) ? (tiles_m - first_m) : group_m;

@@ -90,8 +90,14 @@ __device__ __forceinline__ Unit decode_unit(int64_t u, const R4Params& p)
     int half = 0;
     x.ncols = BN;
     if (p.splits > 1) {
-        x.tile = u / p.splits;
-        x.split = static_cast<int>(u % p.splits);
+        if (u < 0x7FFFFFFFll) {   // 32-bit division: this sits on the critical path of short kernels
+            const uint32_t u32 = static_cast<uint32_t>(u), sp = static_cast<uint32_t>(p.splits);
+            x.tile = u32 / sp;
+            x.split = static_cast<int>(u32 - static_cast<uint32_t>(x.tile) * sp);
+        } else {
+            x.tile = u / p.splits;
+            x.split = static_cast<int>(u % p.splits);
+        }
     } else {
         x.split = 0;
         if (u < p.full_units) {
