@@ -393,7 +393,25 @@ def lineage_table(prob_c4, kb, gen, torch, device, peaks):
                                   "frac_bf16_peak": c3.flops / (med * 1e-3) / 1e12 / peaks["bf16_tflops"],
                                   "kernel_id": p3.gemm.last_kernel_id()}
     out["addmm_4096^3_Bcol"] = rows
-    del p3
+    # Autotuner of the tcgen05 rung: every candidate plan timed on the operands (fresh handles, so that no
+    # pin leaks into the rows above and below), and the paper's held-out MM 2048^3 instance beside c3 and c4.
+    mm2k = gen.make_case(2048, 2048, 2048, seed=1, dist_a="normal", dist_b="normal", c_bf16=True, name="mm2048")
+    p2k = DeviceProblem(mm2k, kb, torch, device)
+    tune = {}
+    for name, pr in (("mm_2048^3", p2k), ("c3_4096^3_Bcol", p3), ("c4_8192^3", prob_c4)):
+        c = pr.case
+        time.sleep(1.0)     # let the power state settle: a sweep that starts hot times its first candidates low
+        with kb.Gemm(device.index, b_col_major=c.b_col_major, c_bf16=c.c_bf16) as tg:
+            n_cand = len(tg.plan_candidates(pr.A, pr.B, pr.C, c.M, c.N, c.K, c.lda, c.ldb, c.ldc))
+            plan, best_us, heur_us = tg.autotune(pr.A, pr.B, pr.C, c.M, c.N, c.K, c.lda, c.ldb, c.ldc, iters=10)
+        tune[name] = {"candidates": n_cand, "pinned_plan": dict(zip(("kernel", "splits", "split_via", "group_m",
+                                                                      "half_tail"), plan.as_tuple())),
+                      "us_pinned": best_us, "us_heuristic": heur_us,
+                      "tflops_pinned": c.flops / (best_us * 1e-6) / 1e12,
+                      "tflops_heuristic": c.flops / (heur_us * 1e-6) / 1e12}
+    tune["note"] = "microseconds per launch in back-to-back loops of 10 launches, minimum of two passes"
+    out["autotune"] = tune
+    del p3, p2k
 
     c5 = gen.make_config("c5", 1)
     p5 = DeviceProblem(c5, kb, torch, device)

@@ -210,6 +210,77 @@ klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype, int64_t M
                                             const void* A, int64_t lda, const void* B, int64_t ldb,
                                             void* C, int64_t ldc, void* stream);
 
+/* ---------------------------------------------------------------------------
+ * Launch plans and the autotuner of the tcgen05 rung.
+ *
+ * Paper, Table 1 (transition vocabulary: `templatize`, `autotune`) and Appendix D
+ * (the recipe parameters a skill carries - block size, stages, split - steered
+ * by a short sweep on top of a fixed kernel structure).  The tcgen05 rung leaves
+ * a few choices of its schedule open; each is a field of the plan below, 0 =
+ * "let the rung's heuristic decide":
+ *   kernel     1 single-CTA kernel (128 x 256 tiles), 2 CTA-pair kernel (512 x 256 tiles)
+ *   splits     number of K splits (1 = none)
+ *   split_via  with splits > 1: 1 partial sums through the global workspace,
+ *              2 through a thread-block cluster (M <= 32, splits 2 / 4 / 8)
+ *   group_m    tile-rows per raster group (L2 reuse pattern)
+ *   half_tail  1 cut the last wave into 128-column half tiles, 2 never
+ * Every plan computes the same C up to fp32 summation order (plans that differ
+ * only in kernel / group_m / half_tail are bit-identical; K splits change the
+ * order of the partial sums and stay within the parity bound).
+ *
+ * A plan is pinned per handle for one (M, N, K) and alignment class of the
+ * operands (16-byte alignment of base and pitch of A, B, C; the pointers are
+ * used for nothing else and no memory is touched).  Later klineage_gemm_run /
+ * klineage_gemm_run_addmm calls with variant KLINEAGE_TCGEN05 on that shape use
+ * it.  All host-side; not thread-safe per handle.
+ */
+typedef struct {
+    int kernel;
+    int splits;
+    int split_via;
+    int group_m;
+    int half_tail;
+} klineage_gemm_plan_t;
+
+#define KLINEAGE_MAX_PLANS 48
+
+/* Writes the candidate plans of a problem to out[0 .. min(cap, *count)) and their
+ * number to *count (at most KLINEAGE_MAX_PLANS); out[0] is the all-zero
+ * heuristic plan.  Host only.  Errors: as klineage_gemm_check_args. */
+klineage_status_t klineage_gemm_plan_candidates(klineage_gemm_t h, int64_t M, int64_t N, int64_t K,
+                                                const void* A, int64_t lda, const void* B, int64_t ldb,
+                                                const void* C, int64_t ldc,
+                                                klineage_gemm_plan_t* out, int cap, int* count);
+
+/* Pins `plan` for the shape (plan == NULL removes the pin).  A plan that cannot
+ * run the shape (e.g. the pair kernel with unaligned operands, more splits than
+ * k-blocks or than the workspace holds) is refused with KLINEAGE_ERR_INVALID_ARG
+ * and nothing changes. */
+klineage_status_t klineage_gemm_set_plan(klineage_gemm_t h, int64_t M, int64_t N, int64_t K,
+                                         const void* A, int64_t lda, const void* B, int64_t ldb,
+                                         const void* C, int64_t ldc, const klineage_gemm_plan_t* plan);
+
+/* Reads the pinned plan (*pinned_out = 1) or the all-zero plan (*pinned_out = 0). */
+klineage_status_t klineage_gemm_get_plan(klineage_gemm_t h, int64_t M, int64_t N, int64_t K,
+                                         const void* A, int64_t lda, const void* B, int64_t ldb,
+                                         const void* C, int64_t ldc,
+                                         klineage_gemm_plan_t* plan_out, int* pinned_out);
+
+/* Times every candidate plan on the caller's operands (device pointers, as for
+ * klineage_gemm_run; `iters` launches per measurement, <= 0 means 10, CUDA events
+ * on `stream`, two passes, minimum), pins the fastest - the heuristic plan unless
+ * another beats it by more than 1 % - and leaves C = A.B computed by it.
+ * Blocks the host until done (this call synchronises `stream`).  Candidates whose
+ * launch fails or that report a device-side give-up are skipped.
+ * best_out / best_us_out / heuristic_us_out (each optional): the pinned plan,
+ * its time per launch and the heuristic plan's, in microseconds.
+ * Errors: as klineage_gemm_run; KLINEAGE_ERR_LAUNCH when no candidate ran. */
+klineage_status_t klineage_gemm_autotune(klineage_gemm_t h, int64_t M, int64_t N, int64_t K,
+                                         const void* A, int64_t lda, const void* B, int64_t ldb,
+                                         void* C, int64_t ldc, int iters, void* stream,
+                                         klineage_gemm_plan_t* best_out, float* best_us_out,
+                                         float* heuristic_us_out);
+
 const char* klineage_status_string(int status);
 const char* klineage_variant_name(int variant);
 

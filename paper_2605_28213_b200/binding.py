@@ -34,6 +34,7 @@ EXPORTED_SYMBOLS = (
     "klineage_gemm_create", "klineage_gemm_run", "klineage_gemm_destroy", "klineage_gemm_check_args",
     "klineage_gemm_get_device_status", "klineage_gemm_last_kernel_id", "klineage_status_string",
     "klineage_variant_name", "klineage_gemm_run_noalloc", "klineage_gemm_run_addmm",
+    "klineage_gemm_plan_candidates", "klineage_gemm_set_plan", "klineage_gemm_get_plan", "klineage_gemm_autotune",
 )
 
 
@@ -95,6 +96,68 @@ _lib.klineage_gemm_run_addmm.argtypes = [_p, _i64, _i64, _i64, _p, _i64, _p, _i6
 def klineage_gemm_run_addmm_raw(h, M, N, K, A, lda, B, ldb, bias, C, ldc, variant, stream) -> int:
     """Raw status of C <- A.B + bias (bias: N bf16 values on the device)."""
     return _lib.klineage_gemm_run_addmm(h, M, N, K, A, lda, B, ldb, bias, C, ldc, variant, stream)
+
+
+class klineage_gemm_plan_t(ctypes.Structure):
+    """Launch plan of the tcgen05 rung (0 in a field = the rung's heuristic)."""
+    _fields_ = [("kernel", _int), ("splits", _int), ("split_via", _int), ("group_m", _int), ("half_tail", _int)]
+
+    def as_tuple(self):
+        return (self.kernel, self.splits, self.split_via, self.group_m, self.half_tail)
+
+    def __repr__(self):
+        return ("plan(kernel=%d, splits=%d, split_via=%d, group_m=%d, half_tail=%d)" % self.as_tuple())
+
+
+KLINEAGE_MAX_PLANS = 48
+_shape_args = [_p, _i64, _i64, _i64, _p, _i64, _p, _i64, _p, _i64]
+_lib.klineage_gemm_plan_candidates.restype = _int
+_lib.klineage_gemm_plan_candidates.argtypes = _shape_args + [ctypes.POINTER(klineage_gemm_plan_t), _int,
+                                                             ctypes.POINTER(_int)]
+_lib.klineage_gemm_set_plan.restype = _int
+_lib.klineage_gemm_set_plan.argtypes = _shape_args + [ctypes.POINTER(klineage_gemm_plan_t)]
+_lib.klineage_gemm_get_plan.restype = _int
+_lib.klineage_gemm_get_plan.argtypes = _shape_args + [ctypes.POINTER(klineage_gemm_plan_t), ctypes.POINTER(_int)]
+_lib.klineage_gemm_autotune.restype = _int
+_lib.klineage_gemm_autotune.argtypes = _shape_args + [_int, _p, ctypes.POINTER(klineage_gemm_plan_t),
+                                                      ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)]
+
+
+def klineage_gemm_plan_candidates(h, M, N, K, A, lda, B, ldb, C, ldc):
+    """List of candidate plans (klineage_gemm_plan_t); the first is the all-zero heuristic plan."""
+    arr = (klineage_gemm_plan_t * KLINEAGE_MAX_PLANS)()
+    n = _int(0)
+    st = _lib.klineage_gemm_plan_candidates(h, M, N, K, A, lda, B, ldb, C, ldc, arr, KLINEAGE_MAX_PLANS,
+                                            ctypes.byref(n))
+    if st != KLINEAGE_OK:
+        raise KlineageError(st, "klineage_gemm_plan_candidates")
+    return [klineage_gemm_plan_t(*arr[i].as_tuple()) for i in range(n.value)]
+
+
+def klineage_gemm_set_plan_raw(h, M, N, K, A, lda, B, ldb, C, ldc, plan) -> int:
+    """Raw status of pinning `plan` (None removes the pin)."""
+    ref = None if plan is None else ctypes.byref(plan)
+    return _lib.klineage_gemm_set_plan(h, M, N, K, A, lda, B, ldb, C, ldc, ref)
+
+
+def klineage_gemm_get_plan(h, M, N, K, A, lda, B, ldb, C, ldc):
+    """(plan, pinned?) for the shape."""
+    plan, pinned = klineage_gemm_plan_t(), _int(0)
+    st = _lib.klineage_gemm_get_plan(h, M, N, K, A, lda, B, ldb, C, ldc, ctypes.byref(plan), ctypes.byref(pinned))
+    if st != KLINEAGE_OK:
+        raise KlineageError(st, "klineage_gemm_get_plan")
+    return plan, bool(pinned.value)
+
+
+def klineage_gemm_autotune(h, M, N, K, A, lda, B, ldb, C, ldc, iters, stream):
+    """(pinned plan, its microseconds per launch, the heuristic plan's microseconds)."""
+    plan = klineage_gemm_plan_t()
+    best, heur = ctypes.c_float(0), ctypes.c_float(0)
+    st = _lib.klineage_gemm_autotune(h, M, N, K, A, lda, B, ldb, C, ldc, iters, stream, ctypes.byref(plan),
+                                     ctypes.byref(best), ctypes.byref(heur))
+    if st != KLINEAGE_OK:
+        raise KlineageError(st, "klineage_gemm_autotune")
+    return plan, best.value, heur.value
 
 
 def klineage_status_string(status: int) -> str:
@@ -194,6 +257,22 @@ class Gemm:
     def run_raw(self, A, B, C, M, N, K, lda, ldb, ldc, variant, stream=None) -> int:
         return klineage_gemm_run_raw(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(C),
                                      ldc, int(variant), self._stream(stream))
+
+    def plan_candidates(self, A, B, C, M, N, K, lda, ldb, ldc):
+        return klineage_gemm_plan_candidates(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(C), ldc)
+
+    def set_plan(self, plan, A, B, C, M, N, K, lda, ldb, ldc) -> None:
+        st = klineage_gemm_set_plan_raw(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(C), ldc,
+                                        plan)
+        if st != KLINEAGE_OK:
+            raise KlineageError(st, "klineage_gemm_set_plan")
+
+    def get_plan(self, A, B, C, M, N, K, lda, ldb, ldc):
+        return klineage_gemm_get_plan(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(C), ldc)
+
+    def autotune(self, A, B, C, M, N, K, lda, ldb, ldc, iters: int = 10, stream=None):
+        return klineage_gemm_autotune(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(C), ldc,
+                                      int(iters), self._stream(stream))
 
     def device_status(self):
         return klineage_gemm_get_device_status(self._h)

@@ -121,6 +121,17 @@ typedef CUresult (*TensorMapEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cu
                                            CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                            CUtensorMapFloatOOBfill);
 
+// Launch plan of the tcgen05 rung: the knobs its schedule leaves open.  Zero in a field
+// lets the rung's own heuristic decide; the autotuner times candidate plans and pins the
+// fastest per shape (paper, Table 1: `templatize` / `autotune` transitions).
+struct R4Plan {
+    int kernel = 0;      // 0 auto, 1 single-CTA kernel, 2 CTA-pair kernel
+    int splits = 0;      // 0 auto, 1 no K split, n > 1 K splits
+    int split_via = 0;   // with splits > 1: 0 auto, 1 global workspace, 2 cluster (distributed shared memory)
+    int group_m = 0;     // 0 auto, else tile-rows per raster group
+    int half_tail = 0;   // 0 auto, 1 cut the last wave into half tiles, 2 never
+};
+
 // Host-side state of a handle that the TMA rungs need.
 struct RunContext {
     int device = 0;
@@ -135,6 +146,7 @@ struct RunContext {
     unsigned flags = 0;
     bool allow_repack = true;   // rung 4 may copy unaligned operands into the workspace (needs scratch)
     int kid_flags = 0;          // added to the kernel id a rung-4 launch reports (64 = operands repacked)
+    R4Plan plan;                // pinned plan of this call's shape (all zero = heuristics)
 };
 
 // Encodes a 2-D tiled tensor map (dims/strides innermost first; stride of the
@@ -151,6 +163,12 @@ cudaError_t launch_r35_mma_sync(const GemmArgs& g, RunContext& ctx, cudaStream_t
 cudaError_t launch_zero_fill(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
 // CTA-pair (cta_group::2) form of rung 4 and the test of its preconditions.
 bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx);
+// Hard preconditions of the CTA-pair kernel only (operands TMA-loadable), without the size heuristic.
+bool r4_pair_possible(const GemmArgs& g, const RunContext& ctx);
+// True when `plan` can run this problem on the tcgen05 rung (the launcher refuses it otherwise).
+bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& plan);
+// Candidate plans of a problem, the all-zero heuristic plan first; returns how many were written.
+int r4_enumerate_plans(const GemmArgs& g, const RunContext& ctx, R4Plan* out, int cap);
 cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id);
 
 }  // namespace klin

@@ -4,11 +4,18 @@
 #include "../../include/klineage_gemm.h"
 #include "common.cuh"
 
+#include <array>
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <new>
 
 using namespace klin;
+
+// Key of a pinned plan: the shape and the alignment class of the three operands (the class
+// decides which sub-paths of the tcgen05 rung can run, so a plan tuned for one does not
+// carry over to another).
+typedef std::array<int64_t, 4> PlanKey;
 
 struct klineage_gemm_s {
     RunContext ctx;
@@ -16,6 +23,9 @@ struct klineage_gemm_s {
     int c_dtype = 0;
     unsigned* status = nullptr;   // device: 4 words (error, kernel id, detail0, detail1)
     int last_kernel_id = -1;
+    std::map<PlanKey, R4Plan> plans;   // pinned by klineage_gemm_set_plan / klineage_gemm_autotune
+    bool forcing = false;              // autotune in progress: run `forced` whatever is pinned
+    R4Plan forced;
 };
 
 namespace klin {
@@ -56,6 +66,61 @@ struct DeviceGuard {
         if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
     }
 };
+
+bool aligned16(const void* base, int64_t ld, int elt)
+{
+    return reinterpret_cast<uintptr_t>(base) % 16 == 0 && (ld * elt) % 16 == 0;
+}
+
+PlanKey plan_key(const klineage_gemm_s* h, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, const void* B,
+                 int64_t ldb, const void* C, int64_t ldc)
+{
+    const int celt = h->c_dtype == KLINEAGE_C_BF16 ? 2 : 4;
+    const int64_t cls = (aligned16(A, lda, 2) ? 1 : 0) | (aligned16(B, ldb, 2) ? 2 : 0) | (aligned16(C, ldc, celt) ? 4 : 0);
+    return PlanKey{M, N, K, cls};
+}
+
+GemmArgs make_args(const klineage_gemm_s* h, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, const void* B,
+                   int64_t ldb, const void* bias, void* C, int64_t ldc)
+{
+    GemmArgs g;
+    g.M = static_cast<int>(M);
+    g.N = static_cast<int>(N);
+    g.K = static_cast<int>(K);
+    g.A = static_cast<const uint16_t*>(A);
+    g.lda = lda;
+    g.B = static_cast<const uint16_t*>(B);
+    g.ldb = ldb;
+    g.C = C;
+    g.ldc = ldc;
+    g.b_col = h->b_layout == KLINEAGE_B_COL_MAJOR ? 1 : 0;
+    g.c_bf16 = h->c_dtype == KLINEAGE_C_BF16 ? 1 : 0;
+    g.status = h->status;
+    g.bias = static_cast<const uint16_t*>(bias);
+    return g;
+}
+
+klineage_gemm_plan_t to_public(const R4Plan& p)
+{
+    klineage_gemm_plan_t o;
+    o.kernel = p.kernel;
+    o.splits = p.splits;
+    o.split_via = p.split_via;
+    o.group_m = p.group_m;
+    o.half_tail = p.half_tail;
+    return o;
+}
+
+R4Plan from_public(const klineage_gemm_plan_t& p)
+{
+    R4Plan o;
+    o.kernel = p.kernel;
+    o.splits = p.splits;
+    o.split_via = p.split_via;
+    o.group_m = p.group_m;
+    o.half_tail = p.half_tail;
+    return o;
+}
 
 bool ranges_overlap(const void* a, size_t a_bytes, const void* b, size_t b_bytes)
 {
@@ -183,20 +248,8 @@ static klineage_status_t run_impl(klineage_gemm_t h, int64_t M, int64_t N, int64
     DeviceGuard guard(h->ctx.device);
     if (!guard.ok) return KLINEAGE_ERR_LAUNCH;
 
-    GemmArgs g;
-    g.M = static_cast<int>(M);
-    g.N = static_cast<int>(N);
-    g.K = static_cast<int>(K);
-    g.A = static_cast<const uint16_t*>(A);
-    g.lda = lda;
-    g.B = static_cast<const uint16_t*>(B);
-    g.ldb = ldb;
-    g.C = C;
-    g.ldc = ldc;
-    g.b_col = bcol ? 1 : 0;
-    g.c_bf16 = h->c_dtype == KLINEAGE_C_BF16 ? 1 : 0;
-    g.status = h->status;
-    g.bias = static_cast<const uint16_t*>(bias);
+    const GemmArgs g = make_args(h, M, N, K, A, lda, B, ldb, bias, C, ldc);
+    (void)bcol;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int kid = -1;
@@ -210,7 +263,18 @@ static klineage_status_t run_impl(klineage_gemm_t h, int64_t M, int64_t N, int64
             case KLINEAGE_VECTORIZED: e = launch_r2_vectorized(g, s, &kid); break;
             case KLINEAGE_PIPELINED: e = launch_r3_pipelined(g, h->ctx, s, &kid); break;
             case KLINEAGE_MMA_SYNC: e = launch_r35_mma_sync(g, h->ctx, s, &kid); break;
-            default: e = launch_r4_tcgen05(g, h->ctx, s, &kid); break;
+            default: {
+                // the plan pinned for this shape and alignment class, else the rung's heuristics
+                h->ctx.plan = R4Plan();
+                if (h->forcing) {
+                    h->ctx.plan = h->forced;
+                } else if (!h->plans.empty()) {
+                    const auto it = h->plans.find(plan_key(h, M, N, K, A, lda, B, ldb, C, ldc));
+                    if (it != h->plans.end()) h->ctx.plan = it->second;
+                }
+                e = launch_r4_tcgen05(g, h->ctx, s, &kid);
+                break;
+            }
         }
     }
     if (e != cudaSuccess) {
@@ -243,6 +307,150 @@ klineage_status_t klineage_gemm_run_addmm(klineage_gemm_t h, int64_t M, int64_t 
         }
     }
     return run_impl(h, M, N, K, A, lda, B, ldb, bias, C, ldc, variant, stream);
+}
+
+// ------------------------------------------------------------------ launch plans and the autotuner
+klineage_status_t klineage_gemm_plan_candidates(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A,
+                                                int64_t lda, const void* B, int64_t ldb, const void* C, int64_t ldc,
+                                                klineage_gemm_plan_t* out, int cap, int* count)
+{
+    if (!h || !count || cap < 0 || (cap > 0 && !out)) return KLINEAGE_ERR_INVALID_ARG;
+    const klineage_status_t chk =
+        klineage_gemm_check_args(h->b_layout, h->c_dtype, M, N, K, A, lda, B, ldb, C, ldc, KLINEAGE_TCGEN05);
+    if (chk != KLINEAGE_OK) return chk;
+    const GemmArgs g = make_args(h, M, N, K, A, lda, B, ldb, nullptr, const_cast<void*>(C), ldc);
+    R4Plan tmp[KLINEAGE_MAX_PLANS];
+    const int n = r4_enumerate_plans(g, h->ctx, tmp, KLINEAGE_MAX_PLANS);
+    *count = n;
+    for (int i = 0; i < n && i < cap; ++i) out[i] = to_public(tmp[i]);
+    return KLINEAGE_OK;
+}
+
+klineage_status_t klineage_gemm_set_plan(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                         const void* B, int64_t ldb, const void* C, int64_t ldc,
+                                         const klineage_gemm_plan_t* plan)
+{
+    if (!h) return KLINEAGE_ERR_INVALID_ARG;
+    const klineage_status_t chk =
+        klineage_gemm_check_args(h->b_layout, h->c_dtype, M, N, K, A, lda, B, ldb, C, ldc, KLINEAGE_TCGEN05);
+    if (chk != KLINEAGE_OK) return chk;
+    const PlanKey key = plan_key(h, M, N, K, A, lda, B, ldb, C, ldc);
+    if (!plan) {
+        h->plans.erase(key);
+        return KLINEAGE_OK;
+    }
+    const R4Plan pl = from_public(*plan);
+    const GemmArgs g = make_args(h, M, N, K, A, lda, B, ldb, nullptr, const_cast<void*>(C), ldc);
+    if (!r4_plan_valid(g, h->ctx, pl)) return KLINEAGE_ERR_INVALID_ARG;
+    h->plans[key] = pl;
+    return KLINEAGE_OK;
+}
+
+klineage_status_t klineage_gemm_get_plan(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                         const void* B, int64_t ldb, const void* C, int64_t ldc,
+                                         klineage_gemm_plan_t* plan_out, int* pinned_out)
+{
+    if (!h || !plan_out) return KLINEAGE_ERR_INVALID_ARG;
+    const auto it = h->plans.find(plan_key(h, M, N, K, A, lda, B, ldb, C, ldc));
+    const bool found = it != h->plans.end();
+    *plan_out = to_public(found ? it->second : R4Plan());
+    if (pinned_out) *pinned_out = found ? 1 : 0;
+    return KLINEAGE_OK;
+}
+
+klineage_status_t klineage_gemm_autotune(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                         const void* B, int64_t ldb, void* C, int64_t ldc, int iters, void* stream,
+                                         klineage_gemm_plan_t* best_out, float* best_us_out, float* heuristic_us_out)
+{
+    if (!h) return KLINEAGE_ERR_INVALID_ARG;
+    const klineage_status_t chk =
+        klineage_gemm_check_args(h->b_layout, h->c_dtype, M, N, K, A, lda, B, ldb, C, ldc, KLINEAGE_TCGEN05);
+    if (chk != KLINEAGE_OK) return chk;
+    if (M == 0 || N == 0 || K == 0) {
+        if (best_out) *best_out = to_public(R4Plan());
+        if (best_us_out) *best_us_out = 0.f;
+        if (heuristic_us_out) *heuristic_us_out = 0.f;
+        return KLINEAGE_OK;
+    }
+    if (iters <= 0) iters = 10;
+    DeviceGuard guard(h->ctx.device);
+    if (!guard.ok) return KLINEAGE_ERR_LAUNCH;
+    const GemmArgs g = make_args(h, M, N, K, A, lda, B, ldb, nullptr, C, ldc);
+    R4Plan cand[KLINEAGE_MAX_PLANS];
+    const int n = r4_enumerate_plans(g, h->ctx, cand, KLINEAGE_MAX_PLANS);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+        cudaGetLastError();
+        if (e0) cudaEventDestroy(e0);
+        return KLINEAGE_ERR_INTERNAL;
+    }
+    float best = -1.f, heur = -1.f;
+    int best_i = -1;
+    klineage_status_t fatal = KLINEAGE_OK;
+    // Two passes over the candidates, the minimum of each candidate's two averages: a pass
+    // sees every candidate under similar clocks, the minimum discards a disturbed one.
+    float t_min[KLINEAGE_MAX_PLANS];
+    for (int i = 0; i < n; ++i) t_min[i] = -1.f;
+    h->forcing = true;
+    for (int pass = 0; pass < 2 && fatal == KLINEAGE_OK; ++pass) {
+        for (int i = 0; i < n; ++i) {
+            if (pass == 1 && t_min[i] < 0.f) continue;   // failed in the first pass
+            h->forced = cand[i];
+            // one untimed launch (instruction cache, tensor maps), then the timed ones
+            klineage_status_t st = klineage_gemm_run(h, M, N, K, A, lda, B, ldb, C, ldc, KLINEAGE_TCGEN05, stream);
+            if (st == KLINEAGE_OK) {
+                cudaEventRecord(e0, s);
+                for (int r = 0; r < iters && st == KLINEAGE_OK; ++r)
+                    st = klineage_gemm_run(h, M, N, K, A, lda, B, ldb, C, ldc, KLINEAGE_TCGEN05, stream);
+                cudaEventRecord(e1, s);
+            }
+            if (cudaStreamSynchronize(s) != cudaSuccess) {
+                cudaGetLastError();
+                fatal = KLINEAGE_ERR_LAUNCH;
+                break;
+            }
+            int code = 0;
+            if (klineage_gemm_get_device_status(h, &code, nullptr) != KLINEAGE_OK) {
+                fatal = KLINEAGE_ERR_INTERNAL;
+                break;
+            }
+            if (st != KLINEAGE_OK || code != KLINEAGE_OK) {
+                t_min[i] = -1.f;
+                continue;
+            }
+            float ms = 0.f;
+            cudaEventElapsedTime(&ms, e0, e1);
+            const float us = ms * 1e3f / static_cast<float>(iters);
+            if (pass == 0 || us < t_min[i]) t_min[i] = us;
+        }
+    }
+    h->forcing = false;
+    h->forced = R4Plan();
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (fatal != KLINEAGE_OK) return fatal;
+    for (int i = 0; i < n; ++i) {
+        if (t_min[i] < 0.f) continue;
+        if (i == 0) heur = t_min[i];
+        if (best_i < 0 || t_min[i] < best) {
+            best = t_min[i];
+            best_i = i;
+        }
+    }
+    if (best_i < 0) return KLINEAGE_ERR_LAUNCH;
+    // keep the heuristic plan unless a candidate beats it by more than the timing noise (1 %)
+    if (heur > 0.f && best > 0.99f * heur) {
+        best_i = 0;
+        best = heur;
+    }
+    // leave C holding the product computed by the chosen plan
+    h->plans[plan_key(h, M, N, K, A, lda, B, ldb, C, ldc)] = cand[best_i];
+    const klineage_status_t st = klineage_gemm_run(h, M, N, K, A, lda, B, ldb, C, ldc, KLINEAGE_TCGEN05, stream);
+    if (best_out) *best_out = to_public(cand[best_i]);
+    if (best_us_out) *best_us_out = best;
+    if (heuristic_us_out) *heuristic_us_out = heur;
+    return st;
 }
 
 klineage_status_t klineage_gemm_get_device_status(klineage_gemm_t h, int* code_out, int* kernel_id_out)

@@ -729,6 +729,40 @@ SplitPlan plan_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContex
     return sp;
 }
 
+// Whether `splits` K splits can run: every split gets k-blocks, and the partial sums fit
+// the cluster (skinny orientation, M <= 32, 2 / 4 / 8 CTAs) or the workspace and counters.
+bool split_feasible(int M, int64_t tiles, int nkb, int64_t ldw, const RunContext& ctx, int splits, bool cluster)
+{
+    if (splits == 1) return !cluster;
+    if (splits < 1 || splits > 64 || splits > nkb) return false;
+    const int per = (nkb + splits - 1) / splits;
+    if ((nkb + per - 1) / per != splits) return false;
+    if (cluster) return M <= 32 && (splits == 2 || splits == 4 || splits == 8);
+    if (tiles * 4 > ctx.n_tile_counters) return false;
+    return static_cast<size_t>(splits) * M * ldw * sizeof(float) <= ctx.workspace_bytes;
+}
+
+// The heuristic plan with the pinned fields of `pl` applied; false when they cannot run.
+bool resolve_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContext& ctx, const R4Plan& pl, SplitPlan* out)
+{
+    SplitPlan sp = plan_split(M, tiles, nkb, ldw, ctx);
+    if (pl.splits > 0) {
+        sp.splits = pl.splits;
+        if (pl.splits == 1)
+            sp.cluster = false;
+        else if (pl.split_via == 2)
+            sp.cluster = true;
+        else if (pl.split_via == 1)
+            sp.cluster = false;
+        else
+            sp.cluster = sp.swap && M <= 32 && (pl.splits == 2 || pl.splits == 4 || pl.splits == 8);
+        if (sp.cluster && !sp.swap) return false;
+        if (!split_feasible(M, tiles, nkb, ldw, ctx, sp.splits, sp.cluster)) return false;
+    }
+    *out = sp;
+    return true;
+}
+
 template <bool BCOL, bool GENERIC, bool SWAP>
 cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
                    const R4Params& p, unsigned grid, int device, cudaStream_t stream)
@@ -864,7 +898,9 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     p.tiles_n = static_cast<int>(tiles_n);
     p.nkb = (g.K + BK - 1) / BK;
     p.ldw = (static_cast<int64_t>(g.N) + 3) & ~int64_t(3);
-    const SplitPlan plan = plan_split(g.M, tiles, p.nkb, p.ldw, ctx);
+    const R4Plan& pinned = ctx.plan;
+    SplitPlan plan;
+    if (!resolve_split(g.M, tiles, p.nkb, p.ldw, ctx, pinned, &plan)) return cudaErrorInvalidValue;
     p.splits = plan.splits;
     p.cluster = plan.cluster ? 1 : 0;
     p.kb_per_split = (p.nkb + p.splits - 1) / p.splits;
@@ -872,7 +908,9 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     p.counters = ctx.tile_counters;
 
     // Large aligned problems run on the CTA-pair kernel (tcgen05.mma.cta_group::2).
-    if (!plan.swap && plan.splits == 1 && r4_pair_applicable(g, ctx)) return launch_r4_tcgen05_pair(g, ctx, stream, kernel_id);
+    if (pinned.kernel == 2 && (plan.swap || plan.splits != 1 || !r4_pair_possible(g, ctx))) return cudaErrorInvalidValue;
+    const bool use_pair = pinned.kernel == 2 || (pinned.kernel == 0 && r4_pair_applicable(g, ctx));
+    if (!plan.swap && plan.splits == 1 && use_pair) return launch_r4_tcgen05_pair(g, ctx, stream, kernel_id);
 
     const bool generic = !(ctx.encode_tiled && tma_ok(g.A, g.lda, 2) && tma_ok(g.B, g.ldb, 2));
     const int celt = g.c_bf16 ? 2 : 4;
@@ -933,11 +971,12 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     *kernel_id = p.kid;
     // Static schedule.  Without a K split, a last wave that would leave at least half of the
     // SMs idle is cut into 128-column half tiles (twice as many units, half as long).
-    p.group_m = 16;   // measured: 16 tile-rows per raster group re-read least from HBM at 8192^3
+    p.group_m = pinned.group_m > 0 ? pinned.group_m : 16;   // measured: 16 tile-rows per group re-read least from HBM at 8192^3
     p.full_units = tiles;
-    if (p.splits == 1 && !swap) {
+    if (p.splits == 1 && !swap && pinned.half_tail != 2) {
         const int64_t tail = tiles % ctx.sm_count;
-        if (tail != 0 && 2 * tail <= ctx.sm_count && g.N > BN / 2) p.full_units = tiles - tail;
+        const bool pays = 2 * tail <= ctx.sm_count;
+        if (tail != 0 && (pays || pinned.half_tail == 1) && g.N > BN / 2) p.full_units = tiles - tail;
     }
     p.total_units = p.splits > 1 ? tiles * p.splits : p.full_units + 2 * (tiles - p.full_units);
     p.idesc_half = (p.idesc & ~(0x3Fu << 17)) | (static_cast<uint32_t>((BN / 2) >> 3) << 17);
@@ -955,6 +994,88 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
 }
 
 }  // namespace
+
+bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& pl)
+{
+    if (pl.kernel < 0 || pl.kernel > 2 || pl.splits < 0 || pl.split_via < 0 || pl.split_via > 2 || pl.group_m < 0 ||
+        pl.group_m > 1024 || pl.half_tail < 0 || pl.half_tail > 2)
+        return false;
+    if (g.M <= 0 || g.N <= 0 || g.K <= 0) return true;   // nothing to launch; any plan is moot
+    const int64_t tiles = static_cast<int64_t>((g.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
+    const int nkb = (g.K + BK - 1) / BK;
+    const int64_t ldw = (static_cast<int64_t>(g.N) + 3) & ~int64_t(3);
+    SplitPlan sp;
+    if (!resolve_split(g.M, tiles, nkb, ldw, ctx, pl, &sp)) return false;
+    if (pl.kernel == 2 && (sp.swap || sp.splits != 1 || !r4_pair_possible(g, ctx))) return false;
+    return true;
+}
+
+// Candidates: both kernels where the pair kernel can run, a few raster groups, the half-tile
+// tail on and off, and K splits around the heuristic's choice.  Unaligned operands are tuned
+// as they run (after the repack, aligned): the caller passes the problem it will run.
+int r4_enumerate_plans(const GemmArgs& g, const RunContext& ctx, R4Plan* out, int cap)
+{
+    int n = 0;
+    auto push = [&](const R4Plan& pl) {
+        if (n >= cap || !r4_plan_valid(g, ctx, pl)) return;
+        for (int i = 0; i < n; ++i)
+            if (out[i].kernel == pl.kernel && out[i].splits == pl.splits && out[i].split_via == pl.split_via &&
+                out[i].group_m == pl.group_m && out[i].half_tail == pl.half_tail)
+                return;
+        out[n++] = pl;
+    };
+    push(R4Plan());
+    if (g.M <= 0 || g.N <= 0 || g.K <= 0) return n;
+    const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN;
+    const int64_t tiles = tiles_m * tiles_n;
+    const int nkb = (g.K + BK - 1) / BK;
+    const bool swap = g.M <= 64;
+    if (!swap) {
+        if (r4_pair_possible(g, ctx) && g.M > BM)
+            for (int gm : {2, 4, 8, 16}) {
+                if (gm > 2 && gm / 2 >= (g.M + 511) / 512) continue;   // more rows per group than there are
+                R4Plan pl;
+                pl.kernel = 2;
+                pl.splits = 1;
+                pl.group_m = gm;
+                push(pl);
+            }
+        for (int gm : {4, 8, 16, 32}) {
+            if (gm > 4 && gm / 2 >= tiles_m) continue;
+            for (int ht : {1, 2}) {
+                if (ht == 1 && tiles % ctx.sm_count == 0) continue;
+                R4Plan pl;
+                pl.kernel = 1;
+                pl.splits = 1;
+                pl.group_m = gm;
+                pl.half_tail = ht;
+                push(pl);
+            }
+        }
+    }
+    // K splits: when the unsplit tiles leave SMs idle
+    if (tiles < ctx.sm_count) {
+        const int64_t want = ctx.sm_count / tiles;   // splits that fill one wave
+        for (int s : {2, 3, 4, 6, 8, 12, 16, 24, 32}) {
+            if (s > 2 * want + 1) continue;
+            R4Plan pl;
+            pl.kernel = 1;
+            pl.splits = s;
+            pl.split_via = 1;
+            push(pl);
+            if (swap && g.M <= 32 && (s == 2 || s == 4 || s == 8)) {
+                pl.split_via = 2;
+                push(pl);
+            }
+        }
+        R4Plan pl;
+        pl.kernel = 1;
+        pl.splits = 1;
+        push(pl);
+    }
+    (void)nkb;
+    return n;
+}
 
 }  // namespace klin
 

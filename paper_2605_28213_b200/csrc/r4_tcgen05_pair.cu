@@ -417,13 +417,18 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
 
 }  // namespace
 
-bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx)
+bool r4_pair_possible(const GemmArgs& g, const RunContext& ctx)
 {
     auto ok2 = [](const void* base, int64_t ld) {
         return reinterpret_cast<uintptr_t>(base) % 16 == 0 && (ld * 2) % 16 == 0 && ld * 2 < (int64_t(1) << 40);
     };
     if (!ctx.encode_tiled || ctx.max_smem_optin < kSmemBytes) return false;
-    if (!ok2(g.A, g.lda) || !ok2(g.B, g.ldb)) return false;
+    return ok2(g.A, g.lda) && ok2(g.B, g.ldb);
+}
+
+bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx)
+{
+    if (!r4_pair_possible(g, ctx)) return false;
     // worthwhile only when the pairs fill the machine: at least one 512 x 256 tile per SM pair
     const int64_t tiles = static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * ((g.N + PN - 1) / PN);
     return g.M > 2 * PM && tiles >= ctx.sm_count / 2;
@@ -437,7 +442,7 @@ cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStrea
     p.tiles_n = (g.N + PN - 1) / PN;
     p.total_tiles = static_cast<int64_t>(p.tiles_m2) * p.tiles_n;
     p.nkb = (g.K + BK - 1) / BK;
-    p.group_m = 4;                                  // 4 x 512 rows per raster group
+    p.group_m = ctx.plan.group_m > 0 ? ctx.plan.group_m : 4;   // default: 4 x 512 rows per raster group
     const int celt = g.c_bf16 ? 2 : 4;
     // (row length a multiple of 16 bytes too: a store box ending inside a 16-byte unit at the tensor's
     // right edge writes the whole unit)
