@@ -211,6 +211,51 @@ klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype, int64_t M
                                             void* C, int64_t ldc, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * Batched and grouped GEMM (paper, Appendix D: BMM at batch 16 x 2048^3 and
+ * batch 32 x 1024^3, GroupedGEMM at G = 4 and 8 are held-out members of the GEMM
+ * family; the paper prints no interface for them, this one follows the
+ * strided-batch and pointer-array conventions of BLAS libraries).
+ *
+ * klineage_gemm_run_batched: C_b <- A_b . B_b for b in [0, batch), every problem
+ * of the shape and layout of klineage_gemm_run; operand b starts stride_a /
+ * stride_b / stride_c ELEMENTS after operand b-1 (device memory).  stride_a or
+ * stride_b may be 0 (one matrix shared by all batches); the C matrices must not
+ * overlap (stride_c >= (M-1)*ldc + N when batch > 1) nor overlap A or B.
+ * batch <= 65535; batch == 0 is a no-op.
+ *
+ * klineage_gemm_run_grouped: C_i <- A_i . B_i for i in [0, groups), each group
+ * with its own M[i], N[i], K[i], pointers and pitches; all groups share the
+ * handle's B layout and C dtype.  The ten arrays are HOST arrays of `groups`
+ * entries, read before the call returns; the pointers in A, B, C are device
+ * pointers.  Groups with M*N == 0 are skipped, K == 0 zero-fills that C.  No C
+ * may overlap another group's C or any A or B.
+ *
+ * Execution: with variant KLINEAGE_TCGEN05, TMA-loadable operands (16-byte
+ * aligned bases, pitches and batch strides) and more than 256 rows per
+ * problem, ONE launch of the CTA-pair kernel walks the tiles of all problems
+ * (batched: the batch is the third dimension of the tensor maps; grouped: a
+ * table of per-group tensor maps and sizes, built in the handle's workspace
+ * and copied on `stream` ahead of the kernel; at most 256 groups per launch).
+ * Every other case - lower rungs, unaligned operands, small or skinny problems
+ * - runs the rung's ordinary path once per problem, in order, on `stream`.
+ * Results equal those of `batch` / `groups` separate klineage_gemm_run calls
+ * with the same variant, bit for bit unless such a call would split K.
+ * Errors: as klineage_gemm_run; everything is validated before the first launch.
+ */
+klineage_status_t klineage_gemm_run_batched(klineage_gemm_t h, int64_t batch, int64_t M, int64_t N, int64_t K,
+                                            const void* A, int64_t lda, int64_t stride_a,
+                                            const void* B, int64_t ldb, int64_t stride_b,
+                                            void* C, int64_t ldc, int64_t stride_c,
+                                            int variant, void* stream);
+
+klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups,
+                                            const int64_t* M, const int64_t* N, const int64_t* K,
+                                            const void* const* A, const int64_t* lda,
+                                            const void* const* B, const int64_t* ldb,
+                                            void* const* C, const int64_t* ldc,
+                                            int variant, void* stream);
+
+/* ---------------------------------------------------------------------------
  * Launch plans and the autotuner of the tcgen05 rung.
  *
  * Paper, Table 1 (transition vocabulary: `templatize`, `autotune`) and Appendix D

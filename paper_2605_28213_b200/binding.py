@@ -34,6 +34,7 @@ EXPORTED_SYMBOLS = (
     "klineage_gemm_create", "klineage_gemm_run", "klineage_gemm_destroy", "klineage_gemm_check_args",
     "klineage_gemm_get_device_status", "klineage_gemm_last_kernel_id", "klineage_status_string",
     "klineage_variant_name", "klineage_gemm_run_noalloc", "klineage_gemm_run_addmm",
+    "klineage_gemm_run_batched", "klineage_gemm_run_grouped",
     "klineage_gemm_plan_candidates", "klineage_gemm_set_plan", "klineage_gemm_get_plan", "klineage_gemm_autotune",
 )
 
@@ -96,6 +97,32 @@ _lib.klineage_gemm_run_addmm.argtypes = [_p, _i64, _i64, _i64, _p, _i64, _p, _i6
 def klineage_gemm_run_addmm_raw(h, M, N, K, A, lda, B, ldb, bias, C, ldc, variant, stream) -> int:
     """Raw status of C <- A.B + bias (bias: N bf16 values on the device)."""
     return _lib.klineage_gemm_run_addmm(h, M, N, K, A, lda, B, ldb, bias, C, ldc, variant, stream)
+
+
+_lib.klineage_gemm_run_batched.restype = _int
+_lib.klineage_gemm_run_batched.argtypes = [_p, _i64, _i64, _i64, _i64, _p, _i64, _i64, _p, _i64, _i64, _p, _i64, _i64,
+                                           _int, _p]
+_lib.klineage_gemm_run_grouped.restype = _int
+_lib.klineage_gemm_run_grouped.argtypes = [_p, _int] + [ctypes.POINTER(_i64)] * 3 + [
+    ctypes.POINTER(_p), ctypes.POINTER(_i64), ctypes.POINTER(_p), ctypes.POINTER(_i64), ctypes.POINTER(_p),
+    ctypes.POINTER(_i64), _int, _p]
+
+
+def klineage_gemm_run_batched_raw(h, batch, M, N, K, A, lda, stride_a, B, ldb, stride_b, C, ldc, stride_c, variant,
+                                  stream) -> int:
+    """Raw status of C_b <- A_b . B_b, b < batch (strides in elements)."""
+    return _lib.klineage_gemm_run_batched(h, batch, M, N, K, A, lda, stride_a, B, ldb, stride_b, C, ldc, stride_c,
+                                          variant, stream)
+
+
+def klineage_gemm_run_grouped_raw(h, M, N, K, A, lda, B, ldb, C, ldc, variant, stream) -> int:
+    """Raw status of C_i <- A_i . B_i over groups; every argument up to ldc is a sequence with one entry per group."""
+    n = len(M)
+    assert all(len(x) == n for x in (N, K, A, lda, B, ldb, C, ldc))
+    i64s = lambda xs: (_i64 * n)(*[int(x) for x in xs])
+    ptrs = lambda xs: (_p * n)(*[None if x is None else int(x) for x in xs])
+    return _lib.klineage_gemm_run_grouped(h, n, i64s(M), i64s(N), i64s(K), ptrs(A), i64s(lda), ptrs(B), i64s(ldb),
+                                          ptrs(C), i64s(ldc), variant, stream)
 
 
 class klineage_gemm_plan_t(ctypes.Structure):
@@ -253,6 +280,20 @@ class Gemm:
                                          self._ptr(C), ldc, int(variant), self._stream(stream))
         if st != KLINEAGE_OK:
             raise KlineageError(st, "klineage_gemm_run_addmm")
+
+    def run_batched(self, batch, A, B, C, M, N, K, lda, ldb, ldc, stride_a, stride_b, stride_c, variant,
+                    stream=None) -> None:
+        st = klineage_gemm_run_batched_raw(self._h, batch, M, N, K, self._ptr(A), lda, stride_a, self._ptr(B), ldb,
+                                           stride_b, self._ptr(C), ldc, stride_c, int(variant), self._stream(stream))
+        if st != KLINEAGE_OK:
+            raise KlineageError(st, "klineage_gemm_run_batched")
+
+    def run_grouped(self, A, B, C, M, N, K, lda, ldb, ldc, variant, stream=None) -> None:
+        st = klineage_gemm_run_grouped_raw(self._h, M, N, K, [self._ptr(x) for x in A], lda,
+                                           [self._ptr(x) for x in B], ldb, [self._ptr(x) for x in C], ldc,
+                                           int(variant), self._stream(stream))
+        if st != KLINEAGE_OK:
+            raise KlineageError(st, "klineage_gemm_run_grouped")
 
     def run_raw(self, A, B, C, M, N, K, lda, ldb, ldc, variant, stream=None) -> int:
         return klineage_gemm_run_raw(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(C),

@@ -154,6 +154,32 @@ struct RunContext {
 bool encode_map_2d(const RunContext& ctx, CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t dim0,
                    uint64_t dim1, uint64_t stride1_bytes, uint32_t box0, uint32_t box1, CUtensorMapSwizzle swz);
 
+// The same with a third, outermost dimension (the batch index of a batched GEMM): box 1 along it.
+bool encode_map_3d(const RunContext& ctx, CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t dim0,
+                   uint64_t dim1, uint64_t dim2, uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t box0,
+                   uint32_t box1, CUtensorMapSwizzle swz);
+
+// Several problems in one launch of the tcgen05 rung (paper, Appendix D: BMM and GroupedGEMM are
+// held-out members of the GEMM family).
+//   batched: `batch` problems of one shape, operand b at base + b * stride (elements); the tensor
+//            maps get the batch as a third dimension, the tile schedule runs over batch x tiles.
+//   grouped: problems of different shapes; one table entry per group in device memory holds
+//            the group's tensor maps, sizes and its first tile in the launch-wide schedule.
+struct BatchArgs {
+    int batch = 1;
+    int64_t stride_a = 0, stride_b = 0, stride_c = 0;   // elements
+};
+struct alignas(128) GroupEntry {
+    CUtensorMap map_a, map_b, map_c;    // 3 x 128 bytes
+    void* C;
+    int64_t ldc;
+    int M, N, K, nkb;
+    int tiles_m, tiles_n;               // in tiles of the kernel that runs the table
+    int tile_start;                     // first tile of this group in the launch-wide schedule
+    int epi_tma;                        // this group's C can take the TMA-store epilogue
+};
+constexpr int kMaxGroups = 256;         // groups per launch (the schedule's prefix sums live in shared memory)
+
 cudaError_t launch_r0_naive(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
 cudaError_t launch_r1_tiled(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
 cudaError_t launch_r2_vectorized(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
@@ -170,5 +196,14 @@ bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& plan)
 // Candidate plans of a problem, the all-zero heuristic plan first; returns how many were written.
 int r4_enumerate_plans(const GemmArgs& g, const RunContext& ctx, R4Plan* out, int cap);
 cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id);
+// Batched form on the CTA-pair kernel: one launch over batch x tiles.  `possible` tests the
+// preconditions (operands and batch strides TMA-loadable); shapes it refuses run batch by batch.
+bool r4_pair_batched_possible(const GemmArgs& g, const BatchArgs& b, const RunContext& ctx);
+cudaError_t launch_r4_pair_batched(const GemmArgs& g, const BatchArgs& b, RunContext& ctx, cudaStream_t stream,
+                                   int* kernel_id);
+// Grouped form: `groups` host descriptions (A, B, C, sizes, pitches in GemmArgs form; all with the
+// handle's B layout and C dtype).  The table is built in the handle's workspace on `stream`.
+bool r4_pair_grouped_possible(const GemmArgs* groups, int n, const RunContext& ctx);
+cudaError_t launch_r4_pair_grouped(const GemmArgs* groups, int n, RunContext& ctx, cudaStream_t stream, int* kernel_id);
 
 }  // namespace klin

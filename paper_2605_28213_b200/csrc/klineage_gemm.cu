@@ -44,6 +44,21 @@ bool encode_map_2d(const RunContext& ctx, CUtensorMap* map, CUtensorMapDataType 
     return r == CUDA_SUCCESS;
 }
 
+bool encode_map_3d(const RunContext& ctx, CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t dim0,
+                   uint64_t dim1, uint64_t dim2, uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t box0,
+                   uint32_t box1, CUtensorMapSwizzle swz)
+{
+    if (!ctx.encode_tiled) return false;
+    const cuuint64_t dims[3] = {dim0, dim1, dim2};
+    const cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
+    const cuuint32_t box[3] = {box0, box1, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = ctx.encode_tiled(map, dt, 3, const_cast<void*>(base), dims, strides, box, estr,
+                                        CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 }  // namespace klin
 
 namespace {
@@ -307,6 +322,139 @@ klineage_status_t klineage_gemm_run_addmm(klineage_gemm_t h, int64_t M, int64_t 
         }
     }
     return run_impl(h, M, N, K, A, lda, B, ldb, bias, C, ldc, variant, stream);
+}
+
+// ------------------------------------------------------------------ batched and grouped GEMM
+klineage_status_t klineage_gemm_run_batched(klineage_gemm_t h, int64_t batch, int64_t M, int64_t N, int64_t K,
+                                            const void* A, int64_t lda, int64_t stride_a, const void* B, int64_t ldb,
+                                            int64_t stride_b, void* C, int64_t ldc, int64_t stride_c, int variant,
+                                            void* stream)
+{
+    if (!h || batch < 0 || batch > 65535) return KLINEAGE_ERR_INVALID_ARG;
+    const klineage_status_t chk = klineage_gemm_check_args(h->b_layout, h->c_dtype, M, N, K, A, lda, B, ldb, C, ldc, variant);
+    if (chk != KLINEAGE_OK) return chk;
+    if (batch == 0 || M == 0 || N == 0) {
+        h->last_kernel_id = -1;
+        return KLINEAGE_OK;
+    }
+    const bool bcol = h->b_layout == KLINEAGE_B_COL_MAJOR;
+    const size_t celt = h->c_dtype == KLINEAGE_C_BF16 ? 2 : 4;
+    if (stride_a < 0 || stride_b < 0 || stride_c < 0) return KLINEAGE_ERR_INVALID_ARG;
+    // the C matrices of different batches must not overlap; A and B may be shared (stride 0)
+    const int64_t c_extent = (M - 1) * ldc + N;
+    if (batch > 1 && stride_c < c_extent) return KLINEAGE_ERR_INVALID_ARG;
+    if (K > 0) {
+        const size_t a_bytes = (size_t(batch - 1) * stride_a + size_t(M - 1) * lda + K) * 2;
+        const size_t b_bytes = (size_t(batch - 1) * stride_b + size_t((bcol ? N : K) - 1) * ldb + (bcol ? K : N)) * 2;
+        const size_t c_bytes = (size_t(batch - 1) * stride_c + size_t(c_extent)) * celt;
+        if (ranges_overlap(A, a_bytes, C, c_bytes) || ranges_overlap(B, b_bytes, C, c_bytes)) return KLINEAGE_ERR_INVALID_ARG;
+    }
+    const uint8_t* a8 = static_cast<const uint8_t*>(A);
+    const uint8_t* b8 = static_cast<const uint8_t*>(B);
+    uint8_t* c8 = static_cast<uint8_t*>(C);
+    if (variant == KLINEAGE_TCGEN05 && K > 0 && h->ctx.cc_major == 10) {
+        // one launch over batch x tiles on the CTA-pair kernel when the batch maps onto 3-D tensor maps
+        const GemmArgs g = make_args(h, M, N, K, A, lda, B, ldb, nullptr, C, ldc);
+        BatchArgs ba;
+        ba.batch = static_cast<int>(batch);
+        ba.stride_a = stride_a;
+        ba.stride_b = stride_b;
+        ba.stride_c = stride_c;
+        const int64_t pair_tiles = ((M + 511) / 512) * ((N + 255) / 256) * batch;
+        if (M > 256 && pair_tiles >= h->ctx.sm_count / 2 && r4_pair_batched_possible(g, ba, h->ctx)) {
+            DeviceGuard guard(h->ctx.device);
+            if (!guard.ok) return KLINEAGE_ERR_LAUNCH;
+            h->ctx.plan = R4Plan();
+            int kid = -1;
+            if (launch_r4_pair_batched(g, ba, h->ctx, static_cast<cudaStream_t>(stream), &kid) != cudaSuccess) {
+                cudaGetLastError();
+                return KLINEAGE_ERR_LAUNCH;
+            }
+            h->last_kernel_id = kid;
+            return KLINEAGE_OK;
+        }
+    }
+    // every other case: the rung's ordinary path, one launch per batch
+    for (int64_t b = 0; b < batch; ++b) {
+        const klineage_status_t st = run_impl(h, M, N, K, a8 ? a8 + b * stride_a * 2 : nullptr, lda,
+                                              b8 ? b8 + b * stride_b * 2 : nullptr, ldb, nullptr,
+                                              c8 + b * stride_c * celt, ldc, variant, stream);
+        if (st != KLINEAGE_OK) return st;
+    }
+    return KLINEAGE_OK;
+}
+
+klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups, const int64_t* M, const int64_t* N,
+                                            const int64_t* K, const void* const* A, const int64_t* lda,
+                                            const void* const* B, const int64_t* ldb, void* const* C, const int64_t* ldc,
+                                            int variant, void* stream)
+{
+    if (!h || groups < 0) return KLINEAGE_ERR_INVALID_ARG;
+    if (groups == 0) {
+        h->last_kernel_id = -1;
+        return KLINEAGE_OK;
+    }
+    if (!M || !N || !K || !A || !lda || !B || !ldb || !C || !ldc) return KLINEAGE_ERR_INVALID_ARG;
+    const bool bcol = h->b_layout == KLINEAGE_B_COL_MAJOR;
+    const size_t celt = h->c_dtype == KLINEAGE_C_BF16 ? 2 : 4;
+    // validate everything before anything is launched
+    for (int i = 0; i < groups; ++i) {
+        const klineage_status_t chk =
+            klineage_gemm_check_args(h->b_layout, h->c_dtype, M[i], N[i], K[i], A[i], lda[i], B[i], ldb[i], C[i], ldc[i], variant);
+        if (chk != KLINEAGE_OK) return chk;
+    }
+    // no group's C may overlap another group's C or any group's A or B
+    for (int i = 0; i < groups; ++i) {
+        if (M[i] == 0 || N[i] == 0) continue;
+        const size_t ci = (size_t(M[i] - 1) * ldc[i] + N[i]) * celt;
+        for (int j = 0; j < groups; ++j) {
+            if (M[j] == 0 || N[j] == 0) continue;
+            if (j != i && ranges_overlap(C[i], ci, C[j], (size_t(M[j] - 1) * ldc[j] + N[j]) * celt)) return KLINEAGE_ERR_INVALID_ARG;
+            if (K[j] == 0) continue;
+            const size_t aj = (size_t(M[j] - 1) * lda[j] + K[j]) * 2;
+            const size_t bj = (size_t((bcol ? N[j] : K[j]) - 1) * ldb[j] + (bcol ? K[j] : N[j])) * 2;
+            if (ranges_overlap(C[i], ci, A[j], aj) || ranges_overlap(C[i], ci, B[j], bj)) return KLINEAGE_ERR_INVALID_ARG;
+        }
+    }
+    h->last_kernel_id = -1;
+    if (variant == KLINEAGE_TCGEN05 && h->ctx.cc_major == 10) {
+        // one launch over the tiles of all groups when every non-empty group suits the CTA-pair kernel
+        GemmArgs* ga = new (std::nothrow) GemmArgs[groups];
+        if (!ga) return KLINEAGE_ERR_ALLOC;
+        int n = 0;
+        bool suits = true;
+        int64_t pair_tiles = 0;
+        for (int i = 0; i < groups; ++i) {
+            if (M[i] == 0 || N[i] == 0) continue;
+            if (K[i] == 0 || M[i] <= 256) {
+                suits = false;
+                break;
+            }
+            ga[n++] = make_args(h, M[i], N[i], K[i], A[i], lda[i], B[i], ldb[i], nullptr, C[i], ldc[i]);
+            pair_tiles += ((M[i] + 511) / 512) * ((N[i] + 255) / 256);
+        }
+        suits = suits && n >= 1 && n <= kMaxGroups && pair_tiles >= h->ctx.sm_count / 2 && r4_pair_grouped_possible(ga, n, h->ctx);
+        if (suits) {
+            DeviceGuard guard(h->ctx.device);
+            klineage_status_t st = guard.ok ? KLINEAGE_OK : KLINEAGE_ERR_LAUNCH;
+            int kid = -1;
+            h->ctx.plan = R4Plan();
+            if (st == KLINEAGE_OK && launch_r4_pair_grouped(ga, n, h->ctx, static_cast<cudaStream_t>(stream), &kid) != cudaSuccess) {
+                cudaGetLastError();
+                st = KLINEAGE_ERR_LAUNCH;
+            }
+            delete[] ga;
+            if (st == KLINEAGE_OK) h->last_kernel_id = kid;
+            return st;
+        }
+        delete[] ga;
+    }
+    // every other case: the rung's ordinary path, one launch per group
+    for (int i = 0; i < groups; ++i) {
+        const klineage_status_t st = run_impl(h, M[i], N[i], K[i], A[i], lda[i], B[i], ldb[i], nullptr, C[i], ldc[i], variant, stream);
+        if (st != KLINEAGE_OK) return st;
+    }
+    return KLINEAGE_OK;
 }
 
 // ------------------------------------------------------------------ launch plans and the autotuner

@@ -32,6 +32,7 @@
 #include "common.cuh"
 #include "ptx.cuh"
 #include <cstring>
+#include <new>
 
 namespace klin {
 namespace {
@@ -47,7 +48,8 @@ constexpr int kBHalfBytes = (PN / 2) * BK * 2; // 16 KiB
 constexpr int kStageBytes = kABytes + kBHalfBytes;
 constexpr int kEpiBufBytes = 32 * 128;
 constexpr int kEpiBytes = 8 * kEpiBufBytes;       // one staging block per epilogue warp
-constexpr int kSmemBytes = 1024 + STAGES * kStageBytes + kEpiBytes + 512;
+constexpr int kBarBytes = 1536;                 // barriers, TMEM slot, abort flag, grouped schedule (<= 257 ints)
+constexpr int kSmemBytes = 1024 + STAGES * kStageBytes + kEpiBytes + kBarBytes;
 constexpr int kTmemCols = 512;
 constexpr int kThreads = 10 * 32;                // producer, MMA issuer, 2 x 4 epilogue warps
 
@@ -60,6 +62,23 @@ struct PairParams {
     int64_t total_tiles;
     uint32_t idesc;
     uint32_t b_desc_hi, b_desc_lbo, b_kstep;
+    // batched launches (MODE 1): the schedule runs over batch x tiles_per_batch
+    int tiles_per_batch;
+    int64_t stride_c_bytes;
+    // grouped launches (MODE 2): table in device memory, one entry per group
+    const GroupEntry* groups;
+    int n_groups;
+};
+
+// What a role needs to know about one tile of the schedule.
+struct TileInfo {
+    int m0, n0;                 // first row of this CTA's first row block / first column of the pair tile
+    int M, N, nkb;              // extent of the problem the tile belongs to
+    int z;                      // batch index (third tensor-map coordinate), 0 otherwise
+    int epi_tma;
+    const CUtensorMap *ma, *mb, *mc;
+    uint8_t* C;                 // base of that problem's C
+    int64_t ldc;
 };
 
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_dst, uint32_t ncols)
@@ -103,6 +122,16 @@ __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const void* tma
         ::"r"(ptx::smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(cluster_bar_addr)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_3d_pair(void* smem_dst, const void* tmap, int x, int y, int z,
+                                                 uint32_t cluster_bar_addr)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, "
+        "%3, %4}], [%5];"
+        ::"r"(ptx::smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z),
+        "r"(cluster_bar_addr)
+        : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar_addr)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar_addr) : "memory");
@@ -114,7 +143,9 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_f
     return (static_cast<uint64_t>(hi) << 32) | lo;
 }
 
-template <bool BCOL>
+// MODE 0: one problem (tensor maps 2-D).  MODE 1: batched (3-D tensor maps, z = batch).
+// MODE 2: grouped (per-group tensor maps and sizes from a table in device memory).
+template <bool BCOL, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c, PairParams p)
@@ -128,6 +159,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
     uint64_t* acc_empty = acc_full + 2;                                   // [0]: even CTA, both epilogues drained
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile uint32_t* abort_flag = tmem_slot + 1;
+    int* gstart = reinterpret_cast<int*>(const_cast<uint32_t*>(abort_flag) + 2);   // MODE 2: first tile of every group
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();          // 0 = even CTA (issues the MMAs), 1 = odd CTA
@@ -146,10 +178,16 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         abort_flag[0] = 0;
         abort_flag[1] = 0;
         ptx::fence_barrier_init();
-        ptx::prefetch_tensormap(&map_a);
-        ptx::prefetch_tensormap(&map_b);
-        if (p.epi_tma) ptx::prefetch_tensormap(&map_c);
+        if (MODE != 2) {
+            ptx::prefetch_tensormap(&map_a);
+            ptx::prefetch_tensormap(&map_b);
+            if (p.epi_tma) ptx::prefetch_tensormap(&map_c);
+        }
         if (blockIdx.x == 0) g.status[1] = p.kid;
+    }
+    if (MODE == 2 && warp >= 2) {
+        for (int i = threadIdx.x - 64; i <= p.n_groups; i += kThreads - 64)
+            gstart[i] = (i < p.n_groups) ? p.groups[i].tile_start : static_cast<int>(p.total_tiles);
     }
     if (warp == 1) {
         tmem_alloc_pair(tmem_slot, kTmemCols);
@@ -163,11 +201,58 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    auto tile_origin = [&](int64_t t, int& m0, int& n0) {
+    int group_hint = 0;     // MODE 2: a thread's tiles come in increasing order, so its search resumes here
+    auto tile_info = [&](int64_t t) {
+        TileInfo x;
         int tm, tn;
-        raster_tile(t, p.tiles_m2, p.tiles_n, tm, tn, p.group_m);
-        m0 = tm * TILE_M + static_cast<int>(rank) * PM;     // this CTA's rows: m0 + [0,128) and m0 + 256 + [0,128)
-        n0 = tn * PN;
+        if (MODE == 2) {
+            const int ti = static_cast<int>(t);
+            int gi = group_hint;
+            while (gstart[gi + 1] <= ti) ++gi;              // gstart[n_groups] = total tiles > ti
+            group_hint = gi;
+            const GroupEntry* e = p.groups + gi;
+            x.M = e->M;
+            x.N = e->N;
+            x.nkb = e->nkb;
+            x.z = 0;
+            x.epi_tma = e->epi_tma;
+            x.ma = &e->map_a;
+            x.mb = &e->map_b;
+            x.mc = &e->map_c;
+            x.C = static_cast<uint8_t*>(e->C);
+            x.ldc = e->ldc;
+            raster_tile(ti - gstart[gi], e->tiles_m, e->tiles_n, tm, tn, p.group_m);
+        } else {
+            x.M = g.M;
+            x.N = g.N;
+            x.nkb = p.nkb;
+            x.epi_tma = p.epi_tma;
+            x.ma = &map_a;
+            x.mb = &map_b;
+            x.mc = &map_c;
+            x.ldc = g.ldc;
+            if (MODE == 1) {
+                const uint32_t t32 = static_cast<uint32_t>(t), tpb = static_cast<uint32_t>(p.tiles_per_batch);
+                const uint32_t b = t32 / tpb;
+                x.z = static_cast<int>(b);
+                x.C = static_cast<uint8_t*>(g.C) + static_cast<int64_t>(b) * p.stride_c_bytes;
+                raster_tile(t32 - b * tpb, p.tiles_m2, p.tiles_n, tm, tn, p.group_m);
+            } else {
+                x.z = 0;
+                x.C = static_cast<uint8_t*>(g.C);
+                raster_tile(t, p.tiles_m2, p.tiles_n, tm, tn, p.group_m);
+            }
+        }
+        x.m0 = tm * TILE_M + static_cast<int>(rank) * PM;   // this CTA's rows: m0 + [0,128) and m0 + 256 + [0,128)
+        x.n0 = tn * PN;
+        return x;
+    };
+    // One operand box of a stage; completion is counted on the even CTA's barrier.
+    auto load_box = [&](void* dst, const CUtensorMap* map, int c0, int c1, int z, uint32_t bar) {
+        if (MODE == 1)
+            tma_load_3d_pair(dst, map, c0, c1, z, bar);
+        else
+            tma_load_2d_pair(dst, map, c0, c1, bar);
     };
 
     if (warp == 0) {
@@ -176,10 +261,10 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             uint32_t it = 0;
             bool ok = true;
             for (int64_t t = pair_id; t < p.total_tiles && ok; t += n_pairs) {
-                int m0, n0;
-                tile_origin(t, m0, n0);
-                const int nb = n0 + static_cast<int>(rank) * (PN / 2);      // this CTA's half of B
-                for (int kb = 0; kb < p.nkb; ++kb, ++it) {
+                const TileInfo x = tile_info(t);
+                const int m0 = x.m0;
+                const int nb = x.n0 + static_cast<int>(rank) * (PN / 2);    // this CTA's half of B
+                for (int kb = 0; kb < x.nkb; ++kb, ++it) {
                     const int s = it % STAGES;
                     if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
                         report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x500u | s);
@@ -192,13 +277,13 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     // The even CTA's barrier counts the bytes of both CTAs' loads of this stage.
                     if (rank == 0) ptx::mbar_arrive_expect_tx(&full[s], 2 * kStageBytes);
                     const uint32_t bar = ptx::map_to_cta(ptx::smem_u32(&full[s]), 0);
-                    tma_load_2d_pair(sa, &map_a, kb * BK, m0, bar);
-                    tma_load_2d_pair(sa + kABlockBytes, &map_a, kb * BK, m0 + 2 * PM, bar);
+                    load_box(sa, x.ma, kb * BK, m0, x.z, bar);
+                    load_box(sa + kABlockBytes, x.ma, kb * BK, m0 + 2 * PM, x.z, bar);
                     if (BCOL) {
-                        tma_load_2d_pair(sb, &map_b, kb * BK, nb, bar);
+                        load_box(sb, x.mb, kb * BK, nb, x.z, bar);
                     } else {
-                        tma_load_2d_pair(sb, &map_b, nb, kb * BK, bar);
-                        tma_load_2d_pair(sb + 64 * BK * 2, &map_b, nb + 64, kb * BK, bar);
+                        load_box(sb, x.mb, nb, kb * BK, x.z, bar);
+                        load_box(sb + 64 * BK * 2, x.mb, nb + 64, kb * BK, x.z, bar);
                     }
                 }
             }
@@ -223,7 +308,8 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     break;
                 }
                 ptx::tc_fence_after_sync();
-                for (int kb = 0; kb < p.nkb; ++kb, ++it) {
+                const int nkb = (MODE == 2) ? tile_info(t).nkb : p.nkb;
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t par = (it / STAGES) & 1;
                     if (!ptx::mbar_wait(&full[s], par, abort_flag)) {
@@ -266,13 +352,13 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         uint8_t* b = epi_smem + (warp - 2) * kEpiBufBytes;
         const bool out_bf16 = g.c_bf16 != 0;
         const int cpc = out_bf16 ? 64 : 32;                   // columns per 128-byte staging row
-        float* dst_f = static_cast<float*>(g.C);
-        uint16_t* dst_h = static_cast<uint16_t*>(g.C);
         uint32_t tcount = 0;
         bool ok = true;
         for (int64_t t = pair_id; t < p.total_tiles && ok; t += n_pairs, ++tcount) {
-            int m0, n0;
-            tile_origin(t, m0, n0);
+            const TileInfo x = tile_info(t);
+            const int m0 = x.m0, n0 = x.n0;
+            float* dst_f = reinterpret_cast<float*>(x.C);
+            uint16_t* dst_h = reinterpret_cast<uint16_t*>(x.C);
             if (!ptx::mbar_wait(&acc_full[0], tcount & 1, abort_flag)) {
                 if (lane == 0) report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x540u);
                 abort_flag[0] = 1;
@@ -281,8 +367,8 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             }
             ptx::tc_fence_after_sync();
             const int row0 = m0 + mb * 2 * PM + q * 32;
-            const int rows = min(32, g.M - row0);
-            const int nunits = (row0 < g.M) ? (min(PN, g.N - n0) + cpc - 1) / cpc : 0;
+            const int rows = min(32, x.M - row0);
+            const int nunits = (row0 < x.M) ? (min(PN, x.N - n0) + cpc - 1) / cpc : 0;
             const uint32_t tbase = tmem_base + mb * PN + (static_cast<uint32_t>(q * 32) << 16);
 
             auto release = [&]() {
@@ -299,8 +385,8 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 if (g.bias) {   // AddMM: this unit's columns get their bias in fp32, before any rounding
                     // lane l fetches the bias of columns col0 + l and col0 + 32 + l; a shuffle hands column i's
                     // value to every lane (every lane holds a different row of the same columns)
-                    const float b0 = (col0 + lane < g.N) ? bias_at(g, col0 + lane) : 0.f;
-                    const float b1 = (out_bf16 && col0 + 32 + lane < g.N) ? bias_at(g, col0 + 32 + lane) : 0.f;
+                    const float b0 = (col0 + lane < x.N) ? bias_at(g, col0 + lane) : 0.f;
+                    const float b1 = (out_bf16 && col0 + 32 + lane < x.N) ? bias_at(g, col0 + 32 + lane) : 0.f;
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         r0[i] = __float_as_uint(__uint_as_float(r0[i]) + __shfl_sync(0xFFFFFFFFu, b0, i));
@@ -318,6 +404,8 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
 #pragma unroll
                     for (int i = 0; i < 32; ++i) w[i] = r0[i];
                 }
+                // (a warp's staging buffer may still be read by its previous TMA store, possibly of
+                // another group's tile: wait whenever any tile of the launch can take that path)
                 if (p.epi_tma) {
                     if (lane == 0) ptx::tma_store_wait_read<0>();   // the previous store has read the buffer
                     __syncwarp();
@@ -326,11 +414,14 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 for (int j = 0; j < 8; ++j)
                     *reinterpret_cast<uint4*>(b + lane * 128 + ((j ^ (lane & 7)) << 4)) =
                         make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-                if (p.epi_tma) {
+                if (x.epi_tma) {
                     ptx::fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        ptx::tma_store_2d(&map_c, col0, row0, b);
+                        if (MODE == 1)
+                            ptx::tma_store_3d(x.mc, col0, row0, x.z, b);
+                        else
+                            ptx::tma_store_2d(x.mc, col0, row0, b);
                         ptx::tma_store_commit();
                     }
                 } else {
@@ -341,16 +432,16 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                         const int64_t row = row0 + rr;
                         if (out_bf16) {
                             const int col = col0 + 2 * lane;
-                            uint16_t* d = dst_h + row * g.ldc + col;
-                            if (col + 1 < g.N && (reinterpret_cast<uintptr_t>(d) & 3) == 0) {
+                            uint16_t* d = dst_h + row * x.ldc + col;
+                            if (col + 1 < x.N && (reinterpret_cast<uintptr_t>(d) & 3) == 0) {
                                 *reinterpret_cast<uint32_t*>(d) = word;
                             } else {
-                                if (col < g.N) d[0] = static_cast<uint16_t>(word & 0xFFFFu);
-                                if (col + 1 < g.N) d[1] = static_cast<uint16_t>(word >> 16);
+                                if (col < x.N) d[0] = static_cast<uint16_t>(word & 0xFFFFu);
+                                if (col + 1 < x.N) d[1] = static_cast<uint16_t>(word >> 16);
                             }
                         } else {
                             const int col = col0 + lane;
-                            if (col < g.N) dst_f[row * g.ldc + col] = __uint_as_float(word);
+                            if (col < x.N) dst_f[row * x.ldc + col] = __uint_as_float(word);
                         }
                     }
                     __syncwarp();
@@ -388,11 +479,11 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
     }
 }
 
-template <bool BCOL>
+template <bool BCOL, int MODE>
 cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
                    const PairParams& p, unsigned grid, int device, cudaStream_t stream)
 {
-    auto kern = r4_pair_kernel<BCOL>;
+    auto kern = r4_pair_kernel<BCOL, MODE>;
     static bool attr_set[64] = {};
     if (device < 0 || device >= 64 || !attr_set[device]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
@@ -432,6 +523,166 @@ bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx)
     // worthwhile only when the pairs fill the machine: at least one 512 x 256 tile per SM pair
     const int64_t tiles = static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * ((g.N + PN - 1) / PN);
     return g.M > 2 * PM && tiles >= ctx.sm_count / 2;
+}
+
+namespace {
+
+bool tma2(const void* base, int64_t ld_elems, int elt)
+{
+    return reinterpret_cast<uintptr_t>(base) % 16 == 0 && (ld_elems * elt) % 16 == 0 &&
+           ld_elems * elt < (int64_t(1) << 40);
+}
+
+// The fields of PairParams that depend only on the operand layout.
+void fill_layout(PairParams& p, const GemmArgs& g, const RunContext& ctx)
+{
+    p.group_m = ctx.plan.group_m > 0 ? ctx.plan.group_m : 4;
+    const uint32_t w_major = g.b_col ? 0u : 1u;
+    p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (w_major << 16) | (static_cast<uint32_t>(PN >> 3) << 17) |
+              (static_cast<uint32_t>((2 * PM) >> 4) << 24);
+    p.b_desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    p.b_desc_lbo = g.b_col ? 1u : ((64u * BK * 2u) >> 4);
+    p.b_kstep = g.b_col ? 2u : (2048u >> 4);
+}
+
+bool c_takes_tma_store(const GemmArgs& g)
+{
+    const int celt = g.c_bf16 ? 2 : 4;
+    return tma2(g.C, g.ldc, celt) && (static_cast<int64_t>(g.N) * celt) % 16 == 0;
+}
+
+}  // namespace
+
+bool r4_pair_batched_possible(const GemmArgs& g, const BatchArgs& b, const RunContext& ctx)
+{
+    if (!r4_pair_possible(g, ctx) || b.batch < 1 || b.batch > 65535) return false;
+    // batch strides become tensor-map strides: multiples of 16 bytes, below 2^40
+    auto ok = [](int64_t stride_elems) {
+        return stride_elems > 0 && (stride_elems * 2) % 16 == 0 && stride_elems * 2 < (int64_t(1) << 40);
+    };
+    if (!ok(b.stride_a) || !ok(b.stride_b)) return false;
+    const int64_t tiles = static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * ((g.N + PN - 1) / PN);
+    return tiles * b.batch < 0x7FFFFFFFll;
+}
+
+cudaError_t launch_r4_pair_batched(const GemmArgs& g, const BatchArgs& b, RunContext& ctx, cudaStream_t stream,
+                                   int* kernel_id)
+{
+    if (!r4_pair_batched_possible(g, b, ctx)) return cudaErrorInvalidValue;
+    PairParams p;
+    memset(&p, 0, sizeof p);
+    fill_layout(p, g, ctx);
+    p.tiles_m2 = (g.M + TILE_M - 1) / TILE_M;
+    p.tiles_n = (g.N + PN - 1) / PN;
+    p.tiles_per_batch = p.tiles_m2 * p.tiles_n;
+    p.total_tiles = static_cast<int64_t>(p.tiles_per_batch) * b.batch;
+    p.nkb = (g.K + BK - 1) / BK;
+    const int celt = g.c_bf16 ? 2 : 4;
+    p.stride_c_bytes = b.stride_c * celt;
+    p.epi_tma = (c_takes_tma_store(g) && p.stride_c_bytes % 16 == 0 && p.stride_c_bytes > 0 &&
+                 p.stride_c_bytes < (int64_t(1) << 40))
+                    ? 1
+                    : 0;
+    CUtensorMap ma, mb, mc;
+    memset(&ma, 0, sizeof ma);
+    memset(&mb, 0, sizeof mb);
+    memset(&mc, 0, sizeof mc);
+    const uint64_t nb = static_cast<uint64_t>(b.batch);
+    bool ok = encode_map_3d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, nb, g.lda * 2, b.stride_a * 2, BK,
+                            PM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (g.b_col)
+        ok = ok && encode_map_3d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, nb, g.ldb * 2, b.stride_b * 2,
+                                 BK, PN / 2, CU_TENSOR_MAP_SWIZZLE_128B);
+    else
+        ok = ok && encode_map_3d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, nb, g.ldb * 2, b.stride_b * 2,
+                                 64, BK, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (p.epi_tma)
+        ok = ok && encode_map_3d(ctx, &mc, g.c_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                                 g.C, g.N, g.M, nb, g.ldc * celt, static_cast<uint64_t>(p.stride_c_bytes),
+                                 g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!ok) return cudaErrorInvalidValue;
+    p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + 32 + ctx.kid_flags;
+    *kernel_id = p.kid;
+    const int64_t max_pairs = ctx.sm_count / 2;
+    const unsigned grid = 2u * static_cast<unsigned>(p.total_tiles < max_pairs ? p.total_tiles : max_pairs);
+    return g.b_col ? launch<true, 1>(g, ma, mb, mc, p, grid, ctx.device, stream)
+                   : launch<false, 1>(g, ma, mb, mc, p, grid, ctx.device, stream);
+}
+
+bool r4_pair_grouped_possible(const GemmArgs* groups, int n, const RunContext& ctx)
+{
+    if (n < 1 || n > kMaxGroups || ctx.workspace_bytes < static_cast<size_t>(n) * sizeof(GroupEntry)) return false;
+    int64_t tiles = 0;
+    for (int i = 0; i < n; ++i) {
+        const GemmArgs& g = groups[i];
+        if (g.M <= 0 || g.N <= 0 || g.K <= 0) return false;          // the caller drops empty groups
+        if (!r4_pair_possible(g, ctx)) return false;
+        tiles += static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * ((g.N + PN - 1) / PN);
+    }
+    return tiles < 0x7FFFFFFFll;
+}
+
+cudaError_t launch_r4_pair_grouped(const GemmArgs* groups, int n, RunContext& ctx, cudaStream_t stream, int* kernel_id)
+{
+    if (!r4_pair_grouped_possible(groups, n, ctx)) return cudaErrorInvalidValue;
+    static_assert(sizeof(GroupEntry) % 128 == 0, "table entries keep their tensor maps 128-byte aligned");
+    GroupEntry* table = new (std::nothrow) GroupEntry[n];
+    if (!table) return cudaErrorMemoryAllocation;
+    memset(table, 0, sizeof(GroupEntry) * n);
+    PairParams p;
+    memset(&p, 0, sizeof p);
+    fill_layout(p, groups[0], ctx);
+    int tile_start = 0;
+    bool ok = true, any_tma = false;
+    for (int i = 0; i < n && ok; ++i) {
+        const GemmArgs& g = groups[i];
+        GroupEntry& e = table[i];
+        const int celt = g.c_bf16 ? 2 : 4;
+        e.C = g.C;
+        e.ldc = g.ldc;
+        e.M = g.M;
+        e.N = g.N;
+        e.K = g.K;
+        e.nkb = (g.K + BK - 1) / BK;
+        e.tiles_m = (g.M + TILE_M - 1) / TILE_M;
+        e.tiles_n = (g.N + PN - 1) / PN;
+        e.tile_start = tile_start;
+        tile_start += e.tiles_m * e.tiles_n;
+        e.epi_tma = c_takes_tma_store(g) ? 1 : 0;
+        any_tma = any_tma || e.epi_tma;
+        ok = encode_map_2d(ctx, &e.map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, PM,
+                           CU_TENSOR_MAP_SWIZZLE_128B);
+        if (g.b_col)
+            ok = ok && encode_map_2d(ctx, &e.map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, PN / 2,
+                                     CU_TENSOR_MAP_SWIZZLE_128B);
+        else
+            ok = ok && encode_map_2d(ctx, &e.map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, g.ldb * 2, 64, BK,
+                                     CU_TENSOR_MAP_SWIZZLE_128B);
+        if (e.epi_tma)
+            ok = ok && encode_map_2d(ctx, &e.map_c,
+                                     g.c_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, g.C, g.N,
+                                     g.M, g.ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    }
+    cudaError_t err = ok ? cudaSuccess : cudaErrorInvalidValue;
+    // The table travels on the launch's stream, ahead of the kernel that reads it (from pageable
+    // memory the copy is staged before the call returns, so the host array can go).
+    if (err == cudaSuccess)
+        err = cudaMemcpyAsync(ctx.workspace, table, sizeof(GroupEntry) * n, cudaMemcpyHostToDevice, stream);
+    delete[] table;
+    if (err != cudaSuccess) return err;
+    p.groups = static_cast<const GroupEntry*>(ctx.workspace);
+    p.n_groups = n;
+    p.total_tiles = tile_start;
+    p.epi_tma = any_tma ? 1 : 0;
+    p.kid = kIdTcgen05 + (any_tma ? 0 : 2) + 32 + ctx.kid_flags;
+    *kernel_id = p.kid;
+    const int64_t max_pairs = ctx.sm_count / 2;
+    const unsigned grid = 2u * static_cast<unsigned>(p.total_tiles < max_pairs ? p.total_tiles : max_pairs);
+    CUtensorMap none;
+    memset(&none, 0, sizeof none);
+    const GemmArgs& g0 = groups[0];
+    return g0.b_col ? launch<true, 2>(g0, none, none, none, p, grid, ctx.device, stream)
+                    : launch<false, 2>(g0, none, none, none, p, grid, ctx.device, stream);
 }
 
 cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
@@ -482,8 +733,8 @@ cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStrea
     *kernel_id = p.kid;
     const int64_t max_pairs = ctx.sm_count / 2;
     const unsigned grid = 2u * static_cast<unsigned>(p.total_tiles < max_pairs ? p.total_tiles : max_pairs);
-    return g.b_col ? launch<true>(g, ma, mb, mc, p, grid, ctx.device, stream)
-                   : launch<false>(g, ma, mb, mc, p, grid, ctx.device, stream);
+    return g.b_col ? launch<true, 0>(g, ma, mb, mc, p, grid, ctx.device, stream)
+                   : launch<false, 0>(g, ma, mb, mc, p, grid, ctx.device, stream);
 }
 
 }  // namespace klin
