@@ -230,14 +230,18 @@ klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype, int64_t M
  * pointers.  Groups with M*N == 0 are skipped, K == 0 zero-fills that C.  No C
  * may overlap another group's C or any A or B.
  *
- * Execution: with variant KLINEAGE_TCGEN05, TMA-loadable operands (16-byte
- * aligned bases, pitches and batch strides) and more than 256 rows per
- * problem, ONE launch of the CTA-pair kernel walks the tiles of all problems
- * (batched: the batch is the third dimension of the tensor maps; grouped: a
- * table of per-group tensor maps and sizes, built in the handle's workspace
- * and copied on `stream` ahead of the kernel; at most 256 groups per launch).
- * Every other case - lower rungs, unaligned operands, small or skinny problems
- * - runs the rung's ordinary path once per problem, in order, on `stream`.
+ * Execution: with variant KLINEAGE_TCGEN05 and TMA-loadable operands (16-byte
+ * aligned bases, pitches and batch strides), ONE launch walks the tiles of all
+ * problems (batched: the batch is the third dimension of the tensor maps;
+ * grouped: a table of per-group tensor maps and sizes, built in the handle's
+ * workspace and copied on `stream` ahead of the kernel; at most 256 groups per
+ * launch) when they fill at least half of the SMs: on the CTA-pair kernel
+ * (512 x 256 tiles) when every problem has more than 256 rows and K >= 2048,
+ * else on the single-CTA kernel (128 x 256 tiles, whose double-buffered
+ * accumulator hides the epilogue that short K exposes); a plan pinned for the
+ * shape of the (first) problem may name the kernel.  Every other case - lower
+ * rungs, unaligned operands, a K == 0 group, too few tiles - runs the rung's
+ * ordinary path once per problem, in order, on `stream`.
  * Results equal those of `batch` / `groups` separate klineage_gemm_run calls
  * with the same variant, bit for bit unless such a call would split K.
  * Errors: as klineage_gemm_run; everything is validated before the first launch.
@@ -254,6 +258,11 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups,
                                             const void* const* B, const int64_t* ldb,
                                             void* const* C, const int64_t* ldc,
                                             int variant, void* stream);
+
+/* Number of GEMM kernels the last klineage_gemm_run / _run_addmm / _run_batched /
+ * _run_grouped call on this handle enqueued (1 when a batched or grouped call took
+ * its one-launch path; zero-fill launches count, repack pre-passes do not). */
+int klineage_gemm_last_launch_count(klineage_gemm_t h);
 
 /* ---------------------------------------------------------------------------
  * Launch plans and the autotuner of the tcgen05 rung.

@@ -34,7 +34,7 @@ EXPORTED_SYMBOLS = (
     "klineage_gemm_create", "klineage_gemm_run", "klineage_gemm_destroy", "klineage_gemm_check_args",
     "klineage_gemm_get_device_status", "klineage_gemm_last_kernel_id", "klineage_status_string",
     "klineage_variant_name", "klineage_gemm_run_noalloc", "klineage_gemm_run_addmm",
-    "klineage_gemm_run_batched", "klineage_gemm_run_grouped",
+    "klineage_gemm_run_batched", "klineage_gemm_run_grouped", "klineage_gemm_last_launch_count",
     "klineage_gemm_plan_candidates", "klineage_gemm_set_plan", "klineage_gemm_get_plan", "klineage_gemm_autotune",
 )
 
@@ -99,6 +99,8 @@ def klineage_gemm_run_addmm_raw(h, M, N, K, A, lda, B, ldb, bias, C, ldc, varian
     return _lib.klineage_gemm_run_addmm(h, M, N, K, A, lda, B, ldb, bias, C, ldc, variant, stream)
 
 
+_lib.klineage_gemm_last_launch_count.restype = _int
+_lib.klineage_gemm_last_launch_count.argtypes = [_p]
 _lib.klineage_gemm_run_batched.restype = _int
 _lib.klineage_gemm_run_batched.argtypes = [_p, _i64, _i64, _i64, _i64, _p, _i64, _i64, _p, _i64, _i64, _p, _i64, _i64,
                                            _int, _p]
@@ -320,6 +322,9 @@ class Gemm:
 
     def last_kernel_id(self) -> int:
         return klineage_gemm_last_kernel_id(self._h)
+
+    def last_launch_count(self) -> int:
+        return _lib.klineage_gemm_last_launch_count(self._h)
 
     def close(self) -> None:
         if self._h is not None:

@@ -201,6 +201,14 @@ cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStrea
 bool r4_pair_batched_possible(const GemmArgs& g, const BatchArgs& b, const RunContext& ctx);
 cudaError_t launch_r4_pair_batched(const GemmArgs& g, const BatchArgs& b, RunContext& ctx, cudaStream_t stream,
                                    int* kernel_id);
+// The same two forms on the single-CTA kernel (128 x 256 tiles, double-buffered accumulator: the
+// better choice for short K, where the pair kernel's epilogue is exposed, and for small problems).
+bool r4_single_batched_possible(const GemmArgs& g, const BatchArgs& b, const RunContext& ctx);
+cudaError_t launch_r4_single_batched(const GemmArgs& g, const BatchArgs& b, RunContext& ctx, cudaStream_t stream,
+                                     int* kernel_id);
+bool r4_single_grouped_possible(const GemmArgs* groups, int n, const RunContext& ctx);
+cudaError_t launch_r4_single_grouped(const GemmArgs* groups, int n, RunContext& ctx, cudaStream_t stream,
+                                     int* kernel_id);
 // Grouped form: `groups` host descriptions (A, B, C, sizes, pitches in GemmArgs form; all with the
 // handle's B layout and C dtype).  The table is built in the handle's workspace on `stream`.
 bool r4_pair_grouped_possible(const GemmArgs* groups, int n, const RunContext& ctx);

@@ -23,6 +23,7 @@ struct klineage_gemm_s {
     int c_dtype = 0;
     unsigned* status = nullptr;   // device: 4 words (error, kernel id, detail0, detail1)
     int last_kernel_id = -1;
+    int last_launches = 0;             // GEMM kernels the last run call enqueued
     std::map<PlanKey, R4Plan> plans;   // pinned by klineage_gemm_set_plan / klineage_gemm_autotune
     bool forcing = false;              // autotune in progress: run `forced` whatever is pinned
     R4Plan forced;
@@ -297,14 +298,18 @@ static klineage_status_t run_impl(klineage_gemm_t h, int64_t M, int64_t N, int64
         return KLINEAGE_ERR_LAUNCH;
     }
     h->last_kernel_id = kid;
+    h->last_launches += 1;
     return KLINEAGE_OK;
 }
 
 extern "C" {
 
+int klineage_gemm_last_launch_count(klineage_gemm_t h) { return h ? h->last_launches : 0; }
+
 klineage_status_t klineage_gemm_run(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
                                     const void* B, int64_t ldb, void* C, int64_t ldc, int variant, void* stream)
 {
+    if (h) h->last_launches = 0;
     return run_impl(h, M, N, K, A, lda, B, ldb, nullptr, C, ldc, variant, stream);
 }
 
@@ -313,6 +318,7 @@ klineage_status_t klineage_gemm_run_addmm(klineage_gemm_t h, int64_t M, int64_t 
                                           int64_t ldc, int variant, void* stream)
 {
     if (!h) return KLINEAGE_ERR_INVALID_ARG;
+    h->last_launches = 0;
     if (M > 0 && N > 0) {
         if (!bias || reinterpret_cast<uintptr_t>(bias) % 2) return KLINEAGE_ERR_INVALID_ARG;
         if (C && N > 0 && M > 0 && ldc >= N) {
@@ -331,6 +337,7 @@ klineage_status_t klineage_gemm_run_batched(klineage_gemm_t h, int64_t batch, in
                                             void* stream)
 {
     if (!h || batch < 0 || batch > 65535) return KLINEAGE_ERR_INVALID_ARG;
+    h->last_launches = 0;
     const klineage_status_t chk = klineage_gemm_check_args(h->b_layout, h->c_dtype, M, N, K, A, lda, B, ldb, C, ldc, variant);
     if (chk != KLINEAGE_OK) return chk;
     if (batch == 0 || M == 0 || N == 0) {
@@ -360,17 +367,42 @@ klineage_status_t klineage_gemm_run_batched(klineage_gemm_t h, int64_t batch, in
         ba.stride_a = stride_a;
         ba.stride_b = stride_b;
         ba.stride_c = stride_c;
+        // The CTA-pair kernel (512 x 256 tiles, both accumulators in use) for long K; the single-CTA
+        // kernel (128 x 256 tiles, double-buffered accumulator) for short K and small problems.  A plan
+        // pinned for the per-problem shape decides the kernel when it names one.
+        const int half_sm = h->ctx.sm_count / 2;
         const int64_t pair_tiles = ((M + 511) / 512) * ((N + 255) / 256) * batch;
-        if (M > 256 && pair_tiles >= h->ctx.sm_count / 2 && r4_pair_batched_possible(g, ba, h->ctx)) {
+        const int64_t single_tiles = ((M + 127) / 128) * ((N + 255) / 256) * batch;
+        const bool pair_ok = M > 256 && pair_tiles >= half_sm && r4_pair_batched_possible(g, ba, h->ctx);
+        const bool single_ok = M > 64 && single_tiles >= half_sm && r4_single_batched_possible(g, ba, h->ctx);
+        int want = 0;   // 1 single-CTA kernel, 2 pair kernel
+        R4Plan pinned;
+        const auto it = h->plans.find(plan_key(h, M, N, K, A, lda, B, ldb, C, ldc));
+        if (it != h->plans.end()) pinned = it->second;
+        if (pinned.kernel == 2 && pair_ok)
+            want = 2;
+        else if (pinned.kernel == 1 && single_ok)
+            want = 1;
+        else if (pair_ok && K >= 2048)
+            want = 2;
+        else if (single_ok)
+            want = 1;
+        else if (pair_ok)
+            want = 2;
+        if (want != 0) {
             DeviceGuard guard(h->ctx.device);
             if (!guard.ok) return KLINEAGE_ERR_LAUNCH;
             h->ctx.plan = R4Plan();
+            h->ctx.plan.group_m = pinned.group_m;
             int kid = -1;
-            if (launch_r4_pair_batched(g, ba, h->ctx, static_cast<cudaStream_t>(stream), &kid) != cudaSuccess) {
+            const cudaError_t e = want == 2 ? launch_r4_pair_batched(g, ba, h->ctx, static_cast<cudaStream_t>(stream), &kid)
+                                            : launch_r4_single_batched(g, ba, h->ctx, static_cast<cudaStream_t>(stream), &kid);
+            if (e != cudaSuccess) {
                 cudaGetLastError();
                 return KLINEAGE_ERR_LAUNCH;
             }
             h->last_kernel_id = kid;
+            h->last_launches = 1;
             return KLINEAGE_OK;
         }
     }
@@ -390,6 +422,7 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups, const
                                             int variant, void* stream)
 {
     if (!h || groups < 0) return KLINEAGE_ERR_INVALID_ARG;
+    h->last_launches = 0;
     if (groups == 0) {
         h->last_kernel_id = -1;
         return KLINEAGE_OK;
@@ -421,30 +454,63 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups, const
         // one launch over the tiles of all groups when every non-empty group suits the CTA-pair kernel
         GemmArgs* ga = new (std::nothrow) GemmArgs[groups];
         if (!ga) return KLINEAGE_ERR_ALLOC;
-        int n = 0;
-        bool suits = true;
-        int64_t pair_tiles = 0;
+        int n = 0, first = -1;
+        bool launchable = true, all_tall = true, all_long = true;
+        int64_t pair_tiles = 0, single_tiles = 0;
         for (int i = 0; i < groups; ++i) {
             if (M[i] == 0 || N[i] == 0) continue;
-            if (K[i] == 0 || M[i] <= 256) {
-                suits = false;
+            if (K[i] == 0) {            // a zero-fill group: leave the whole call to the ordinary path
+                launchable = false;
                 break;
             }
+            if (first < 0) first = i;
             ga[n++] = make_args(h, M[i], N[i], K[i], A[i], lda[i], B[i], ldb[i], nullptr, C[i], ldc[i]);
+            all_tall = all_tall && M[i] > 256;
+            all_long = all_long && K[i] >= 2048;
             pair_tiles += ((M[i] + 511) / 512) * ((N[i] + 255) / 256);
+            single_tiles += ((M[i] + 127) / 128) * ((N[i] + 255) / 256);
         }
-        suits = suits && n >= 1 && n <= kMaxGroups && pair_tiles >= h->ctx.sm_count / 2 && r4_pair_grouped_possible(ga, n, h->ctx);
-        if (suits) {
+        launchable = launchable && n >= 1 && n <= kMaxGroups;
+        // kernel choice as for the batched call; a plan pinned for the first group's shape may name it
+        const int half_sm = h->ctx.sm_count / 2;
+        const bool pair_ok = launchable && all_tall && pair_tiles >= half_sm && r4_pair_grouped_possible(ga, n, h->ctx);
+        const bool single_ok = launchable && single_tiles >= half_sm && r4_single_grouped_possible(ga, n, h->ctx);
+        R4Plan pinned;
+        if (first >= 0) {
+            const auto it = h->plans.find(plan_key(h, M[first], N[first], K[first], A[first], lda[first], B[first],
+                                                   ldb[first], C[first], ldc[first]));
+            if (it != h->plans.end()) pinned = it->second;
+        }
+        int want = 0;
+        if (pinned.kernel == 2 && pair_ok)
+            want = 2;
+        else if (pinned.kernel == 1 && single_ok)
+            want = 1;
+        else if (pair_ok && all_long)
+            want = 2;
+        else if (single_ok)
+            want = 1;
+        else if (pair_ok)
+            want = 2;
+        if (want != 0) {
             DeviceGuard guard(h->ctx.device);
             klineage_status_t st = guard.ok ? KLINEAGE_OK : KLINEAGE_ERR_LAUNCH;
             int kid = -1;
             h->ctx.plan = R4Plan();
-            if (st == KLINEAGE_OK && launch_r4_pair_grouped(ga, n, h->ctx, static_cast<cudaStream_t>(stream), &kid) != cudaSuccess) {
-                cudaGetLastError();
-                st = KLINEAGE_ERR_LAUNCH;
+            h->ctx.plan.group_m = pinned.group_m;
+            if (st == KLINEAGE_OK) {
+                const cudaError_t e = want == 2 ? launch_r4_pair_grouped(ga, n, h->ctx, static_cast<cudaStream_t>(stream), &kid)
+                                                : launch_r4_single_grouped(ga, n, h->ctx, static_cast<cudaStream_t>(stream), &kid);
+                if (e != cudaSuccess) {
+                    cudaGetLastError();
+                    st = KLINEAGE_ERR_LAUNCH;
+                }
             }
             delete[] ga;
-            if (st == KLINEAGE_OK) h->last_kernel_id = kid;
+            if (st == KLINEAGE_OK) {
+                h->last_kernel_id = kid;
+                h->last_launches = 1;
+            }
             return st;
         }
         delete[] ga;

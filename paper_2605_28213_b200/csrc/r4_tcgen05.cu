@@ -42,6 +42,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <new>
 
 namespace klin {
 namespace {
@@ -52,7 +53,7 @@ constexpr int kBBytes = BN * BK * 2;              // 32 KiB
 constexpr int kStageBytes = kABytes + kBBytes;    // 48 KiB
 constexpr int kEpiBufBytes = 32 * 128;            // one 32-row x 128-byte staging block
 constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;   // 4 warps x 2 buffers
-constexpr int kBarBytes = 256;
+constexpr int kBarBytes = 1536;                   // barriers, TMEM slot, abort flag, grouped schedule (<= 257 ints)
 constexpr int kSmemBytes = 1024 + STAGES * kStageBytes + kEpiBytes + kBarBytes;
 constexpr int kTmemCols = 512;
 constexpr int kThreadsTma = 6 * 32, kThreadsGeneric = 10 * 32;
@@ -75,6 +76,12 @@ struct R4Params {
     int64_t full_units;     // units [0, full_units) are whole tiles; later ones are 128-column half tiles
     int64_t total_units;
     uint32_t idesc_half;    // instruction descriptor for a half tile (N = 128)
+    // several problems in one launch (MODE 1: batched over 3-D tensor maps; MODE 2: grouped, a
+    // table of per-group tensor maps and sizes in device memory); never combined with a K split
+    int tiles_per_batch;
+    int64_t stride_c_bytes;
+    const GroupEntry* groups;
+    int n_groups;
 };
 
 // One entry of the static schedule.
@@ -83,7 +90,51 @@ struct Unit {
     int m0, n0;             // first row / column of C it computes
     int ncols;              // 256, or 128 for the half tiles that fill the last wave
     int split, kb0, kb1;    // K split index and k-block range
+    // the problem the unit belongs to (MODE 1 / 2 only)
+    int M, N, z, epi_tma;
+    const CUtensorMap *ma, *mb, *mc;
+    uint8_t* C;
+    int64_t ldc;
 };
+// MODE 1 / 2: a launch-wide tile index -> its problem and its (tile_m, tile_n) there.
+template <int MODE>
+__device__ __forceinline__ void decode_multi(Unit& x, const GemmArgs& g, const R4Params& p, const int* gstart, int& hint)
+{
+    int tm, tn;
+    if (MODE == 2) {
+        const int ti = static_cast<int>(x.tile);
+        int gi = hint;
+        while (gstart[gi + 1] <= ti) ++gi;                  // gstart[n_groups] = number of tiles > ti
+        hint = gi;
+        const GroupEntry* e = p.groups + gi;
+        x.M = e->M;
+        x.N = e->N;
+        x.z = 0;
+        x.epi_tma = e->epi_tma;
+        x.ma = &e->map_a;
+        x.mb = &e->map_b;
+        x.mc = &e->map_c;
+        x.C = static_cast<uint8_t*>(e->C);
+        x.ldc = e->ldc;
+        x.kb0 = 0;
+        x.kb1 = e->nkb;
+        raster_tile(ti - gstart[gi], e->tiles_m, e->tiles_n, tm, tn, p.group_m);
+    } else {
+        const uint32_t t32 = static_cast<uint32_t>(x.tile), tpb = static_cast<uint32_t>(p.tiles_per_batch);
+        const uint32_t b = t32 / tpb;
+        x.M = g.M;
+        x.N = g.N;
+        x.z = static_cast<int>(b);
+        x.epi_tma = p.epi_tma;
+        x.C = static_cast<uint8_t*>(g.C) + static_cast<int64_t>(b) * p.stride_c_bytes;
+        x.ldc = g.ldc;
+        x.kb0 = 0;
+        x.kb1 = p.nkb;
+        raster_tile(t32 - b * tpb, p.tiles_m, p.tiles_n, tm, tn, p.group_m);
+    }
+    x.m0 = tm * BM;
+    x.n0 = tn * BN;
+}
 __device__ __forceinline__ Unit decode_unit(int64_t u, const R4Params& p)
 {
     Unit x;
@@ -142,7 +193,7 @@ __device__ __forceinline__ uint4 gather8(const uint16_t* p, int valid)
     return r;
 }
 
-template <bool BCOL, bool GENERIC, bool SWAP>
+template <bool BCOL, bool GENERIC, bool SWAP, int MODE>
 __global__ void __launch_bounds__(GENERIC ? kThreadsGeneric : kThreadsTma, 1)
 r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ CUtensorMap map_c, R4Params p)
@@ -156,6 +207,33 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     uint64_t* acc_empty = acc_full + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile uint32_t* abort_flag = tmem_slot + 1;   // [0] raised on give-up, [1] stays 0
+    int* gstart = reinterpret_cast<int*>(const_cast<uint32_t*>(abort_flag) + 2);   // MODE 2: first tile of every group
+    int group_hint = 0;     // MODE 2: a thread's units come in increasing order; its group search resumes here
+    // One unit of the schedule for this thread's role.
+    auto unit_of = [&](int64_t u) {
+        Unit x = decode_unit(u, p);
+        if (MODE != 0) {
+            const int half_cols = x.n0 % BN;                // 0, or 128 for the second half tile
+            decode_multi<MODE>(x, g, p, gstart, group_hint);
+            x.n0 += half_cols;
+        } else {
+            x.M = g.M;
+            x.N = g.N;
+            x.z = 0;
+            x.epi_tma = p.epi_tma;
+            x.ma = &map_a;
+            x.mb = &map_b;
+            x.mc = &map_c;
+            x.C = static_cast<uint8_t*>(g.C);
+            x.ldc = g.ldc;
+        }
+        if (MODE == 1) {
+            x.ma = &map_a;
+            x.mb = &map_b;
+            x.mc = &map_c;
+        }
+        return x;
+    };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Cluster mode: no CTA may touch a peer's shared memory before that peer runs.
@@ -165,18 +243,30 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     // TMA producer state (used by warp 0, lane 0 only): position in the static schedule.
     struct {
         int64_t u;
-        int kb, kb1, m0, n0;
+        int kb, kb1, m0, n0, z;
+        const CUtensorMap *ma, *mb;
         uint32_t it;
         bool live;
-    } prod = {static_cast<int64_t>(blockIdx.x), 0, 0, 0, 0, 0u, false};
+    } prod = {static_cast<int64_t>(blockIdx.x), 0, 0, 0, 0, 0, &map_a, &map_b, 0u, false};
     auto prod_enter_unit = [&]() {
         prod.live = prod.u < total_units;
         if (!prod.live) return;
-        const Unit x = decode_unit(prod.u, p);
+        const Unit x = unit_of(prod.u);
         prod.kb = x.kb0;
         prod.kb1 = x.kb1;
         prod.m0 = x.m0;
         prod.n0 = x.n0;     // a half tile still loads 256 columns from n0; its MMA reads the first 128
+        if (MODE != 0) {
+            prod.z = x.z;
+            prod.ma = x.ma;
+            prod.mb = x.mb;
+        }
+    };
+    auto load_box = [&](void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
+        if (MODE == 1)
+            ptx::tma_load_3d(dst, map, c0, c1, prod.z, bar);
+        else
+            ptx::tma_load_2d(dst, map, c0, c1, bar);
     };
     // Issues loads until `limit` k-blocks have been issued in total or the schedule ends.
     auto produce = [&](uint32_t limit) {
@@ -192,13 +282,15 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             uint8_t* sa = smem + s * kStageBytes;
             uint8_t* sb = sa + kABytes;
             ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
-            ptx::tma_load_2d(sa, &map_a, prod.kb * BK, prod.m0, &full[s]);
+            const CUtensorMap* pa = (MODE == 2) ? prod.ma : &map_a;
+            const CUtensorMap* pb = (MODE == 2) ? prod.mb : &map_b;
+            load_box(sa, pa, prod.kb * BK, prod.m0, &full[s]);
             if (BCOL) {
-                ptx::tma_load_2d(sb, &map_b, prod.kb * BK, prod.n0, &full[s]);
+                load_box(sb, pb, prod.kb * BK, prod.n0, &full[s]);
             } else {
 #pragma unroll
                 for (int cb = 0; cb < BN / 64; ++cb)
-                    ptx::tma_load_2d(sb + cb * (64 * BK * 2), &map_b, prod.n0 + cb * 64, prod.kb * BK, &full[s]);
+                    load_box(sb + cb * (64 * BK * 2), pb, prod.n0 + cb * 64, prod.kb * BK, &full[s]);
             }
             ++prod.it;
             if (++prod.kb == prod.kb1) {
@@ -220,22 +312,28 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         abort_flag[0] = 0;
         abort_flag[1] = 0;
         ptx::fence_barrier_init();
-        if (!GENERIC) {
+        if (!GENERIC && MODE != 2) {
             ptx::prefetch_tensormap(&map_a);
             ptx::prefetch_tensormap(&map_b);
         }
-        if (p.epi_tma) ptx::prefetch_tensormap(&map_c);
+        if (p.epi_tma && MODE != 2) ptx::prefetch_tensormap(&map_c);
         // The launch is a programmatic dependent one: everything above (and the TMEM
         // allocation in warp 1) may overlap the tail of the previous kernel in the stream;
         // nothing below the wait touches global memory before that kernel has completed.
-        if (!GENERIC) prod_enter_unit();           // schedule arithmetic only
+        if (!GENERIC && MODE != 2) prod_enter_unit();           // schedule arithmetic only
         ptx::grid_dependency_wait();
-        if (!GENERIC) {
+        if (!GENERIC && MODE != 2) {
             // The first ring fill needs nothing from the other warps: start it before the
             // set-up barrier so that TMEM allocation hides behind the first loads' latency.
             produce(STAGES);
         }
         if (blockIdx.x == 0) g.status[1] = p.kid;
+    }
+    if (MODE == 2 && warp >= 2) {
+        // the grouped schedule's prefix sums (written on the stream before this launch)
+        ptx::grid_dependency_wait();
+        for (int i = static_cast<int>(threadIdx.x) - 64; i <= p.n_groups; i += blockDim.x - 64)
+            gstart[i] = (i < p.n_groups) ? p.groups[i].tile_start : static_cast<int>(p.full_units + (p.total_units - p.full_units) / 2);
     }
     if (warp == 1) {
         ptx::tmem_alloc(tmem_slot, kTmemCols);
@@ -252,6 +350,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (!GENERIC && lane == 0) {
+            if (MODE == 2) prod_enter_unit();      // (its group search reads the table the other warps just staged)
             produce(0xFFFFFFFFu);
             // Drain: every load issued must have landed before shared memory is released.
             const uint32_t it = prod.it;
@@ -264,7 +363,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             uint32_t it = 0, t = 0;
             bool ok = true;
             for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++t) {
-                const Unit x = decode_unit(u, p);
+                const Unit x = unit_of(u);
                 const int kb0 = x.kb0, kb1 = x.kb1;
                 const uint32_t idesc = (x.ncols == BN) ? p.idesc : p.idesc_half;
                 const uint32_t buf = t & 1;
@@ -318,7 +417,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         uint32_t nstaged = 0;                                // staging blocks written so far (buffer = parity)
         bool ok = true;
         for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++t) {
-            const Unit x = decode_unit(u, p);
+            const Unit x = unit_of(u);
             const int64_t tile = x.tile;
             const int split = x.split;
             const int m0 = x.m0, n0 = x.n0;
@@ -426,18 +525,18 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 continue;
             }
             const int row0 = m0 + q * 32;
-            if (row0 < g.M) {
+            if (row0 < x.M) {
                 const bool partial = p.splits > 1;
                 const bool out_bf16 = g.c_bf16 && !partial;
-                const bool use_tma = p.epi_tma && !partial;
+                const bool use_tma = x.epi_tma && !partial;
                 const int cpc = out_bf16 ? 64 : 32;           // columns per 128-byte staging row
-                float* dst_f = partial ? p.ws + static_cast<int64_t>(split) * g.M * p.ldw : static_cast<float*>(g.C);
-                uint16_t* dst_h = static_cast<uint16_t*>(g.C);
-                const int64_t ld = partial ? p.ldw : g.ldc;
-                const int rows = min(32, g.M - row0);
+                float* dst_f = partial ? p.ws + static_cast<int64_t>(split) * g.M * p.ldw : reinterpret_cast<float*>(x.C);
+                uint16_t* dst_h = reinterpret_cast<uint16_t*>(x.C);
+                const int64_t ld = partial ? p.ldw : x.ldc;
+                const int rows = min(32, x.M - row0);
                 for (int c = 0; c * cpc < x.ncols; ++c) {
                     const int col0 = n0 + c * cpc;
-                    if (col0 >= g.N) break;
+                    if (col0 >= x.N) break;
                     uint32_t v[32], w[32];
                     const uint32_t taddr = tmem_base + buf * BN + c * cpc + (static_cast<uint32_t>(q * 32) << 16);
                     ptx::tmem_ld_32x32b_x32(taddr, v);
@@ -446,8 +545,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         ptx::tmem_ld_32x32b_x32(taddr + 32, v2);
                         ptx::tmem_ld_wait();
                         if (g.bias) {   // lane l fetches two columns' bias, shuffles hand them round
-                            const float b0 = (col0 + lane < g.N) ? bias_at(g, col0 + lane) : 0.f;
-                            const float b1 = (col0 + 32 + lane < g.N) ? bias_at(g, col0 + 32 + lane) : 0.f;
+                            const float b0 = (col0 + lane < x.N) ? bias_at(g, col0 + lane) : 0.f;
+                            const float b1 = (col0 + 32 + lane < x.N) ? bias_at(g, col0 + 32 + lane) : 0.f;
 #pragma unroll
                             for (int i = 0; i < 32; ++i) {
                                 v[i] = __float_as_uint(__uint_as_float(v[i]) + __shfl_sync(0xFFFFFFFFu, b0, i));
@@ -462,7 +561,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     } else {
                         ptx::tmem_ld_wait();
                         if (g.bias && !partial) {
-                            const float b0 = (col0 + lane < g.N) ? bias_at(g, col0 + lane) : 0.f;
+                            const float b0 = (col0 + lane < x.N) ? bias_at(g, col0 + lane) : 0.f;
 #pragma unroll
                             for (int i = 0; i < 32; ++i)
                                 v[i] = __float_as_uint(__uint_as_float(v[i]) + __shfl_sync(0xFFFFFFFFu, b0, i));
@@ -471,7 +570,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         for (int i = 0; i < 32; ++i) w[i] = v[i];
                     }
                     uint8_t* b = stg + (nstaged++ & 1) * kEpiBufBytes;   // (bias was added above)
-                    if (use_tma) {
+                    if (MODE == 2 ? p.epi_tma != 0 : use_tma) {   // (grouped: an earlier group's store may be in flight)
                         if (lane == 0) ptx::tma_store_wait_read<1>();   // the store that last read this buffer
                         __syncwarp();
                     }
@@ -483,7 +582,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         ptx::fence_proxy_async_smem();
                         __syncwarp();
                         if (lane == 0) {
-                            ptx::tma_store_2d(&map_c, col0, row0, b);
+                            if (MODE == 1)
+                                ptx::tma_store_3d(x.mc, col0, row0, x.z, b);
+                            else
+                                ptx::tma_store_2d(x.mc, col0, row0, b);
                             ptx::tma_store_commit();
                         }
                     } else {
@@ -497,15 +599,15 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                             if (out_bf16) {
                                 const int col = col0 + 2 * lane;
                                 uint16_t* d = dst_h + row * ld + col;
-                                if (col + 1 < g.N && (reinterpret_cast<uintptr_t>(d) & 3) == 0) {
+                                if (col + 1 < x.N && (reinterpret_cast<uintptr_t>(d) & 3) == 0) {
                                     *reinterpret_cast<uint32_t*>(d) = word;
                                 } else {
-                                    if (col < g.N) d[0] = static_cast<uint16_t>(word & 0xFFFFu);
-                                    if (col + 1 < g.N) d[1] = static_cast<uint16_t>(word >> 16);
+                                    if (col < x.N) d[0] = static_cast<uint16_t>(word & 0xFFFFu);
+                                    if (col + 1 < x.N) d[1] = static_cast<uint16_t>(word >> 16);
                                 }
                             } else {
                                 const int col = col0 + lane;
-                                if (col < g.N) dst_f[row * ld + col] = __uint_as_float(word);
+                                if (col < x.N) dst_f[row * ld + col] = __uint_as_float(word);
                             }
                         }
                         __syncwarp();
@@ -763,11 +865,11 @@ bool resolve_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContext&
     return true;
 }
 
-template <bool BCOL, bool GENERIC, bool SWAP>
+template <bool BCOL, bool GENERIC, bool SWAP, int MODE = 0>
 cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
                    const R4Params& p, unsigned grid, int device, cudaStream_t stream)
 {
-    auto kern = r4_tcgen05_kernel<BCOL, GENERIC, SWAP>;
+    auto kern = r4_tcgen05_kernel<BCOL, GENERIC, SWAP, MODE>;
     static bool attr_set[64] = {};
     if (device < 0 || device >= 64 || !attr_set[device]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
@@ -994,6 +1096,175 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
 }
 
 }  // namespace
+
+namespace {
+
+// The parts of R4Params that depend only on the operand layout (128 x 256 tiles, no K split,
+// operands on TMA): shared by the batched and grouped launchers.
+void fill_multi_params(R4Params& p, const GemmArgs& g, const RunContext& ctx)
+{
+    memset(&p, 0, sizeof p);
+    p.splits = 1;
+    const uint32_t w_major = g.b_col ? 0u : 1u;
+    p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (w_major << 16) | (static_cast<uint32_t>(BN >> 3) << 17) |
+              (static_cast<uint32_t>(BM >> 4) << 24);
+    p.idesc_half = (p.idesc & ~(0x3Fu << 17)) | (static_cast<uint32_t>((BN / 2) >> 3) << 17);
+    p.b_desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    p.b_desc_lbo = g.b_col ? 1u : ((64u * BK * 2u) >> 4);
+    p.b_kstep = g.b_col ? 2u : (2048u >> 4);
+    p.n_mma = 16;
+    p.stage_tx = kABytes + kBBytes;
+    p.group_m = ctx.plan.group_m > 0 ? ctx.plan.group_m : 16;
+}
+
+// Static schedule over `tiles` whole tiles: a last wave that would leave at least half of the
+// SMs idle is cut into 128-column half tiles (when every problem is wider than 128 columns).
+unsigned finish_multi_schedule(R4Params& p, int64_t tiles, bool halves_ok, const RunContext& ctx)
+{
+    p.full_units = tiles;
+    const int64_t tail = tiles % ctx.sm_count;
+    if (halves_ok && tail != 0 && 2 * tail <= ctx.sm_count) p.full_units = tiles - tail;
+    p.total_units = p.full_units + 2 * (tiles - p.full_units);
+    return static_cast<unsigned>(p.total_units < ctx.sm_count ? p.total_units : ctx.sm_count);
+}
+
+bool c_store_by_tma(const GemmArgs& g)
+{
+    const int celt = g.c_bf16 ? 2 : 4;
+    return tma_ok(g.C, g.ldc, celt) && (static_cast<int64_t>(g.N) * celt) % 16 == 0;
+}
+
+}  // namespace
+
+bool r4_single_batched_possible(const GemmArgs& g, const BatchArgs& b, const RunContext& ctx)
+{
+    if (!ctx.encode_tiled || ctx.max_smem_optin < kSmemBytes || b.batch < 1 || b.batch > 65535) return false;
+    if (!tma_ok(g.A, g.lda, 2) || !tma_ok(g.B, g.ldb, 2)) return false;
+    auto ok = [](int64_t stride_elems) {
+        return stride_elems > 0 && (stride_elems * 2) % 16 == 0 && stride_elems * 2 < (int64_t(1) << 40);
+    };
+    if (!ok(b.stride_a) || !ok(b.stride_b)) return false;
+    const int64_t tiles = static_cast<int64_t>((g.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
+    return tiles * b.batch < 0x3FFFFFFFll;
+}
+
+cudaError_t launch_r4_single_batched(const GemmArgs& g, const BatchArgs& b, RunContext& ctx, cudaStream_t stream,
+                                     int* kernel_id)
+{
+    if (!r4_single_batched_possible(g, b, ctx)) return cudaErrorInvalidValue;
+    R4Params p;
+    fill_multi_params(p, g, ctx);
+    p.tiles_m = (g.M + BM - 1) / BM;
+    p.tiles_n = (g.N + BN - 1) / BN;
+    p.tiles_per_batch = p.tiles_m * p.tiles_n;
+    p.nkb = (g.K + BK - 1) / BK;
+    p.kb_per_split = p.nkb;
+    const int celt = g.c_bf16 ? 2 : 4;
+    p.stride_c_bytes = b.stride_c * celt;
+    p.epi_tma = (c_store_by_tma(g) && p.stride_c_bytes % 16 == 0 && p.stride_c_bytes > 0 &&
+                 p.stride_c_bytes < (int64_t(1) << 40))
+                    ? 1
+                    : 0;
+    CUtensorMap ma, mb, mc;
+    memset(&ma, 0, sizeof ma);
+    memset(&mb, 0, sizeof mb);
+    memset(&mc, 0, sizeof mc);
+    const uint64_t nb = static_cast<uint64_t>(b.batch);
+    bool ok = encode_map_3d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, nb, g.lda * 2, b.stride_a * 2, BK,
+                            BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (g.b_col)
+        ok = ok && encode_map_3d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, nb, g.ldb * 2, b.stride_b * 2,
+                                 BK, BN, CU_TENSOR_MAP_SWIZZLE_128B);
+    else
+        ok = ok && encode_map_3d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, nb, g.ldb * 2, b.stride_b * 2,
+                                 64, BK, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (p.epi_tma)
+        ok = ok && encode_map_3d(ctx, &mc, g.c_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                                 g.C, g.N, g.M, nb, g.ldc * celt, static_cast<uint64_t>(p.stride_c_bytes),
+                                 g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!ok) return cudaErrorInvalidValue;
+    p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + ctx.kid_flags;
+    *kernel_id = p.kid;
+    const unsigned grid = finish_multi_schedule(p, static_cast<int64_t>(p.tiles_per_batch) * b.batch, g.N > BN / 2, ctx);
+    return g.b_col ? launch<true, false, false, 1>(g, ma, mb, mc, p, grid, ctx.device, stream)
+                   : launch<false, false, false, 1>(g, ma, mb, mc, p, grid, ctx.device, stream);
+}
+
+bool r4_single_grouped_possible(const GemmArgs* groups, int n, const RunContext& ctx)
+{
+    if (!ctx.encode_tiled || ctx.max_smem_optin < kSmemBytes) return false;
+    if (n < 1 || n > kMaxGroups || ctx.workspace_bytes < static_cast<size_t>(n) * sizeof(GroupEntry)) return false;
+    int64_t tiles = 0;
+    for (int i = 0; i < n; ++i) {
+        const GemmArgs& g = groups[i];
+        if (g.M <= 0 || g.N <= 0 || g.K <= 0) return false;          // the caller drops empty groups
+        if (!tma_ok(g.A, g.lda, 2) || !tma_ok(g.B, g.ldb, 2)) return false;
+        tiles += static_cast<int64_t>((g.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
+    }
+    return tiles < 0x3FFFFFFFll;
+}
+
+cudaError_t launch_r4_single_grouped(const GemmArgs* groups, int n, RunContext& ctx, cudaStream_t stream,
+                                     int* kernel_id)
+{
+    if (!r4_single_grouped_possible(groups, n, ctx)) return cudaErrorInvalidValue;
+    GroupEntry* table = new (std::nothrow) GroupEntry[n];
+    if (!table) return cudaErrorMemoryAllocation;
+    memset(table, 0, sizeof(GroupEntry) * n);
+    R4Params p;
+    fill_multi_params(p, groups[0], ctx);
+    p.tiles_m = p.tiles_n = 1;      // unused by the grouped schedule; kept non-zero
+    int tile_start = 0;
+    bool ok = true, any_tma = false, halves_ok = true;
+    for (int i = 0; i < n && ok; ++i) {
+        const GemmArgs& g = groups[i];
+        GroupEntry& e = table[i];
+        const int celt = g.c_bf16 ? 2 : 4;
+        e.C = g.C;
+        e.ldc = g.ldc;
+        e.M = g.M;
+        e.N = g.N;
+        e.K = g.K;
+        e.nkb = (g.K + BK - 1) / BK;
+        e.tiles_m = (g.M + BM - 1) / BM;
+        e.tiles_n = (g.N + BN - 1) / BN;
+        e.tile_start = tile_start;
+        tile_start += e.tiles_m * e.tiles_n;
+        e.epi_tma = c_store_by_tma(g) ? 1 : 0;
+        any_tma = any_tma || e.epi_tma;
+        halves_ok = halves_ok && g.N > BN / 2;
+        ok = encode_map_2d(ctx, &e.map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, BM,
+                           CU_TENSOR_MAP_SWIZZLE_128B);
+        if (g.b_col)
+            ok = ok && encode_map_2d(ctx, &e.map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, BN,
+                                     CU_TENSOR_MAP_SWIZZLE_128B);
+        else
+            ok = ok && encode_map_2d(ctx, &e.map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, g.ldb * 2, 64, BK,
+                                     CU_TENSOR_MAP_SWIZZLE_128B);
+        if (e.epi_tma)
+            ok = ok && encode_map_2d(ctx, &e.map_c,
+                                     g.c_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, g.C, g.N,
+                                     g.M, g.ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    }
+    cudaError_t err = ok ? cudaSuccess : cudaErrorInvalidValue;
+    // The table travels on the launch's stream, ahead of the kernel that reads it (the copy from
+    // pageable memory is staged before the call returns, so the host array can go).
+    if (err == cudaSuccess)
+        err = cudaMemcpyAsync(ctx.workspace, table, sizeof(GroupEntry) * n, cudaMemcpyHostToDevice, stream);
+    delete[] table;
+    if (err != cudaSuccess) return err;
+    p.groups = static_cast<const GroupEntry*>(ctx.workspace);
+    p.n_groups = n;
+    p.epi_tma = any_tma ? 1 : 0;
+    p.kid = kIdTcgen05 + (any_tma ? 0 : 2) + ctx.kid_flags;
+    *kernel_id = p.kid;
+    const unsigned grid = finish_multi_schedule(p, tile_start, halves_ok, ctx);
+    CUtensorMap none;
+    memset(&none, 0, sizeof none);
+    const GemmArgs& g0 = groups[0];
+    return g0.b_col ? launch<true, false, false, 2>(g0, none, none, none, p, grid, ctx.device, stream)
+                    : launch<false, false, false, 2>(g0, none, none, none, p, grid, ctx.device, stream);
+}
 
 bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& pl)
 {

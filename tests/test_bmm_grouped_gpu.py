@@ -77,11 +77,17 @@ class Batch:
         return out
 
 
-def check_batch(kb, bt, variant, exact, want_pair=None):
+def check_batch(kb, bt, variant, exact, want_pair=None, one_launch=None, kernel=0):
+    """kernel: 1 / 2 pins the single-CTA / CTA-pair kernel for the per-problem shape first."""
     c0 = bt.cases[0]
     with kb.Gemm(0, b_col_major=c0.b_col_major, c_bf16=c0.c_bf16) as g:
+        if kernel:
+            g.set_plan(kb.klineage_gemm_plan_t(kernel, 1, 0, 0, 0), bt.a.ptr, bt.b.ptr, bt.c.ptr, c0.M, c0.N, c0.K,
+                       c0.lda, c0.ldb, c0.ldc)
         bt.run(g, variant)
         kid = g.last_kernel_id()
+        if one_launch is not None:
+            assert (g.last_launch_count() == 1) == one_launch, g.last_launch_count()
         res = bt.results()
         for b, case in enumerate(bt.cases):
             C_ref, S = P.oracle_rows(case, np.arange(case.M))
@@ -99,20 +105,25 @@ def check_batch(kb, bt, variant, exact, want_pair=None):
                 assert np.array_equal(bits1, res[b][1]), f"batch {b} differs bitwise from the single-problem call"
 
 
-# (batch, M, N, K, col, bf16, pad, gap) - pair tiles = ceil(M/512) ceil(N/256) batch must reach 74 for one launch
+# (batch, M, N, K, col, bf16, pad, gap): at least 74 tiles of 512 x 256 in the batch, so that both kernels qualify
 ONE_LAUNCH = [
     (7, 1100, 1104, 136, False, True, (0, 8, 8), (8, 16, 24)),      # ragged tiles, bf16 C through the 3-D TMA store
     (5, 600, 2100, 200, True, False, (8, 8, 4), (0, 0, 0)),         # column-major B, fp32 C through the TMA store
     (7, 520, 1301, 72, False, False, (0, 3, 1), (0, 0, 5)),         # odd N (pitch of B 1304): masked direct stores
+    (5, 1100, 1104, 2056, False, True, (0, 0, 0), (0, 0, 0)),       # K >= 2048: the pair kernel by default
 ]
 
 
 @pytest.mark.parametrize("cfg", ONE_LAUNCH, ids=lambda c: f"b{c[0]}-{c[1]}x{c[2]}x{c[3]}")
-def test_bmm_one_launch_on_the_pair_kernel(kb, cfg):
+@pytest.mark.parametrize("kernel", [0, 1, 2], ids=["default", "single", "pair"])
+def test_bmm_one_launch(kb, cfg, kernel):
     batch, M, N, K, col, bf, pad, gap = cfg
+    pair = (K >= 2048) if kernel == 0 else (kernel == 2)
     for dist, exact in (("integer", True), ("normal", False)):
+        if kernel and dist == "normal" and K >= 2048:
+            continue                      # (the long-K case costs the oracle most; integers cover the pinned kernels)
         bt = Batch(batch, M, N, K, col, bf, dist, seed=70, pad=pad, gap=gap)
-        check_batch(kb, bt, 4, exact, want_pair=True)
+        check_batch(kb, bt, 4, exact, want_pair=pair, one_launch=True, kernel=kernel)
 
 
 def test_bmm_problem_by_problem_paths(kb):
@@ -125,7 +136,8 @@ def test_bmm_problem_by_problem_paths(kb):
         for dist, exact in (("integer", True), ("uniform", False)):
             bt = Batch(cfg["batch"], cfg["M"], cfg["N"], cfg["K"], cfg["col"], cfg["bf"], dist, seed=80,
                        pad=cfg.get("pad", (0, 0, 0)), gap=cfg["gap"], share_a=cfg.get("share_a", False))
-            check_batch(kb, bt, 4, exact, want_pair=False if cfg["M"] <= 256 or cfg["gap"][0] % 8 else None)
+            check_batch(kb, bt, 4, exact, want_pair=False if cfg["M"] <= 256 or cfg["gap"][0] % 8 else None,
+                        one_launch=False)
 
 
 @pytest.mark.parametrize("variant", [0, 1, 2, 3, 5], ids=lambda v: VARIANT_NAMES[v])
@@ -153,11 +165,16 @@ def test_bmm_argument_rules(kb):
 
 
 # ---------------------------------------------------------------------------- grouped
-def run_grouped(kb, cases, variant, exact, want_pair=None):
+def run_grouped(kb, cases, variant, exact, want_pair=None, one_launch=None, kernel=0):
     import torch
     c0 = cases[0]
     devs = [P.DeviceCase(c) for c in cases]
     with kb.Gemm(0, b_col_major=c0.b_col_major, c_bf16=c0.c_bf16) as g:
+        if kernel:
+            first = next(i for i, c in enumerate(cases) if c.M and c.N)
+            c, d = cases[first], devs[first]
+            g.set_plan(kb.klineage_gemm_plan_t(kernel, 1, 0, 0, 0), d.a.ptr, d.b.ptr, d.c.ptr, c.M, c.N, c.K, c.lda,
+                       c.ldb, c.ldc)
         g.run_grouped([d.a.ptr for d in devs], [d.b.ptr for d in devs], [d.c.ptr for d in devs],
                       [c.M for c in cases], [c.N for c in cases], [c.K for c in cases],
                       [c.lda for c in cases], [c.ldb for c in cases], [c.ldc for c in cases], variant)
@@ -165,6 +182,8 @@ def run_grouped(kb, cases, variant, exact, want_pair=None):
         code, _ = g.device_status()
         assert code == 0
         kid = g.last_kernel_id()
+        if one_launch is not None:
+            assert (g.last_launch_count() == 1) == one_launch, g.last_launch_count()
         if want_pair is not None:
             assert bool((kid - 400) & 32) == want_pair, kid
         got = [d.result() for d in devs]
@@ -190,13 +209,28 @@ GROUP_SHAPES = [(300, 2048, 136), (1100, 1304, 200), (513, 2000, 64), (700, 1528
 
 
 @pytest.mark.parametrize("col,bf", [(False, True), (True, False)], ids=["row-bf16", "col-f32"])
-def test_grouped_one_launch_on_the_pair_kernel(kb, col, bf):
+@pytest.mark.parametrize("kernel", [0, 2], ids=["default-single", "pair"])
+def test_grouped_one_launch(kb, col, bf, kernel):
     for dist, exact in (("integer", True), ("normal", False)):
         cases = [gen.make_case(M, N, K, seed=100 + i, dist_a=dist, dist_b=dist, b_col_major=col, c_bf16=bf,
                                ldc=N + (4 if i % 2 else 0), name=f"g{i}-{M}x{N}x{K}-{dist}")
                  for i, (M, N, K) in enumerate(GROUP_SHAPES)]
-        # group 0 has M = 300 > 256; every group suits the pair kernel
-        run_grouped(kb, cases, 4, exact, want_pair=True)
+        # every group has more than 256 rows, so the pair kernel qualifies; K < 2048 makes the single-CTA kernel the default
+        run_grouped(kb, cases, 4, exact, want_pair=kernel == 2, one_launch=True, kernel=kernel)
+
+
+def test_grouped_long_k_takes_the_pair_kernel_and_small_groups_the_single_one(kb):
+    shapes = [(520, 2048, 2056), (300, 1304, 2048), (1030, 1528, 2120), (700, 2560, 2048)]      # 16 + 6 + 18 + 20
+    shapes += [(600, 2048, 2048), (513, 1024, 2048)]                                             # + 16 + 8 = 84 tiles of 512 x 256
+    cases = [gen.make_case(M, N, K, seed=140 + i, dist_a="integer", dist_b="integer", c_bf16=True, name=f"gk{i}")
+             for i, (M, N, K) in enumerate(shapes)]
+    run_grouped(kb, cases, 4, True, want_pair=True, one_launch=True)
+    # one group of 40 rows among them: the pair kernel no longer qualifies, the single-CTA kernel takes all groups
+    small = [(40, 2048, 136), (1100, 1304, 200), (64, 2000, 64), (700, 1528, 520), (129, 1304, 72), (600, 520, 328),
+             (1, 264, 8), (900, 2048, 264)]
+    cases = [gen.make_case(M, N, K, seed=150 + i, dist_a="integer", dist_b="integer", c_bf16=False, name=f"gs{i}")
+             for i, (M, N, K) in enumerate(small)]
+    run_grouped(kb, cases, 4, True, want_pair=False, one_launch=True)
 
 
 def test_grouped_with_an_odd_width_group_uses_masked_stores_for_it(kb):
@@ -206,7 +240,8 @@ def test_grouped_with_an_odd_width_group_uses_masked_stores_for_it(kb):
     for i, (M, N, K) in enumerate(shapes):
         cases.append(gen.make_case(M, N, K, seed=110 + i, dist_a="integer", dist_b="integer", c_bf16=True,
                                    ldb=(N + 7) // 8 * 8, ldc=N + 3, name=f"godd{i}"))
-    run_grouped(kb, cases, 4, True, want_pair=True)
+    run_grouped(kb, cases, 4, True, want_pair=False, one_launch=True)
+    run_grouped(kb, cases, 4, True, want_pair=True, one_launch=True, kernel=2)
 
 
 def test_grouped_problem_by_problem_paths(kb):
@@ -219,7 +254,7 @@ def test_grouped_problem_by_problem_paths(kb):
                               name=f"gl{i}-{M}x{N}x{K}")
             import dataclasses
             cases.append(dataclasses.replace(c, M=M, K=K))
-        run_grouped(kb, cases, variant, True, want_pair=False if variant == 4 else None)
+        run_grouped(kb, cases, variant, True, want_pair=False if variant == 4 else None, one_launch=False)
 
 
 def test_grouped_argument_rules(kb):
