@@ -563,9 +563,20 @@ def main():
                     help="configuration to time (default: the headline 8192^3; others are for profiling)")
     ap.add_argument("--variant", type=int, default=4, choices=range(6),
                     help="lineage rung to time (default 4 = tcgen05; 5 = the mma.sync rung 3.5)")
+    ap.add_argument("--family", action="store_true",
+                    help="time only the BMM / GroupedGEMM rows (for profiling) and print them as one JSON line")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.family:
+        import torch
+        from paper_2605_28213_b200 import binding as kb
+        from paper_2605_28213_b200 import inputs as gen
+        device = torch.device("cuda", 0)
+        torch.cuda.set_device(device)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+        print(json.dumps({"gemm_family": family_table(kb, gen, torch, device, load_peaks()[0], flush)}), flush=True)
+        return 0
     return run_gpu(args)
 
 
