@@ -546,6 +546,26 @@ def family_table(kb, gen, torch, device, peaks, flush):
                 "tflops_launch_per_problem": flops / (per * 1e-3) / 1e12, "kernel_id": kid,
                 "sane_vs_torch_on_64_rows": ok}
             del A, B, C
+        # Column-partitioned multi-GPU GEMM, one rank's share of 8192^3 at world 8 (1024 columns of B), its epilogue
+        # storing the slice into 8 full-width C matrices.  All 8 "ranks'" buffers live on this GPU here: the stores'
+        # cost is HBM's, not NVLink's; the row shows what the fused all-gather adds to the kernel.
+        from paper_2605_28213_b200 import npart
+        n, world = 8192, 8
+        A = rand_bf16((n, n), 31, 1.0)
+        Bs = rand_bf16((n, n // world), 32, n ** -0.5)
+        Cs = [torch.empty((n, n), dtype=torch.bfloat16, device=device) for _ in range(world)]
+        part = npart.NPartitionedGemm(g, world, 3, n, [c.data_ptr() for c in Cs], n)
+        fused = timed(lambda: part.run(A, Bs, n, n, n, n // world))
+        kid, launches = g.last_kernel_id(), g.last_launch_count()
+        alone = timed(lambda: g.run(A, Bs, part.dst[3], n, n // world, n, n, n // world, n, 4))
+        ok = all(bool(torch.equal(Cs[0][:, part.n0:part.n1], c[:, part.n0:part.n1])) for c in Cs[1:])
+        flops = 2.0 * n * (n // world) * n
+        out["npart_world8_rank_share_of_8192^3"] = {
+            "ms_fused_store_to_8_destinations": fused, "tflops_fused": flops / (fused * 1e-3) / 1e12,
+            "ms_one_destination": alone, "tflops_one_destination": flops / (alone * 1e-3) / 1e12,
+            "extra_bytes_stored": 7 * n * (n // world) * 2, "launches_one_call": launches, "kernel_id": kid,
+            "all_destinations_equal": ok}
+        del A, Bs, Cs
     out["note"] = ("median of 12 timed calls, each after a 256 MiB L2 flush; 'launch_per_problem' issues the "
                    "single-problem call once per batch / group on the same stream; the torch comparison is a "
                    "sanity check of the timed buffers, parity is established by the tests against the oracle")

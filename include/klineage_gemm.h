@@ -259,6 +259,27 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups,
                                             void* const* C, const int64_t* ldc,
                                             int variant, void* stream);
 
+/*
+ * One product, several destinations:  C_d <- A . B  for d in [0, n_dst), n_dst <= 16.
+ * C and ldc are HOST arrays of n_dst device pointers / pitches (read before the call
+ * returns); every destination is an M x N matrix of the handle's C dtype and may
+ * live on another GPU that this device can address (peer access enabled by the
+ * caller).  This is the fused all-gather of a GEMM partitioned by columns over
+ * several GPUs: rank r multiplies A by its column slice of B and passes, as
+ * destinations, the address of that slice inside every rank's full-width C - no
+ * operand is ever loaded from a peer, results leave through plain or TMA stores
+ * (the paper has no multi-GPU design; its hardware section is single-GPU).
+ * With variant KLINEAGE_TCGEN05, TMA-loadable A and B and a shape that needs neither
+ * a K split nor the skinny orientation, one launch writes every output block to all
+ * destinations from its epilogue; every other case computes into C_0 through the
+ * rung's ordinary path and copies that matrix to the other destinations on `stream`.
+ * Destinations must not overlap one another, A or B.  Errors: as klineage_gemm_run.
+ */
+klineage_status_t klineage_gemm_run_multi_dst(klineage_gemm_t h, int64_t M, int64_t N, int64_t K,
+                                              const void* A, int64_t lda, const void* B, int64_t ldb,
+                                              int n_dst, void* const* C, const int64_t* ldc,
+                                              int variant, void* stream);
+
 /* Number of GEMM kernels the last klineage_gemm_run / _run_addmm / _run_batched /
  * _run_grouped call on this handle enqueued (1 when a batched or grouped call took
  * its one-launch path; zero-fill launches count, repack pre-passes do not). */

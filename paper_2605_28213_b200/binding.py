@@ -35,6 +35,7 @@ EXPORTED_SYMBOLS = (
     "klineage_gemm_get_device_status", "klineage_gemm_last_kernel_id", "klineage_status_string",
     "klineage_variant_name", "klineage_gemm_run_noalloc", "klineage_gemm_run_addmm",
     "klineage_gemm_run_batched", "klineage_gemm_run_grouped", "klineage_gemm_last_launch_count",
+    "klineage_gemm_run_multi_dst",
     "klineage_gemm_plan_candidates", "klineage_gemm_set_plan", "klineage_gemm_get_plan", "klineage_gemm_autotune",
 )
 
@@ -115,6 +116,19 @@ def klineage_gemm_run_batched_raw(h, batch, M, N, K, A, lda, stride_a, B, ldb, s
     """Raw status of C_b <- A_b . B_b, b < batch (strides in elements)."""
     return _lib.klineage_gemm_run_batched(h, batch, M, N, K, A, lda, stride_a, B, ldb, stride_b, C, ldc, stride_c,
                                           variant, stream)
+
+
+_lib.klineage_gemm_run_multi_dst.restype = _int
+_lib.klineage_gemm_run_multi_dst.argtypes = [_p, _i64, _i64, _i64, _p, _i64, _p, _i64, _int, ctypes.POINTER(_p),
+                                             ctypes.POINTER(_i64), _int, _p]
+
+
+def klineage_gemm_run_multi_dst_raw(h, M, N, K, A, lda, B, ldb, C, ldc, variant, stream) -> int:
+    """Raw status of C_d <- A . B for every destination (C, ldc: sequences of device pointers / pitches)."""
+    n = len(C)
+    assert len(ldc) == n
+    return _lib.klineage_gemm_run_multi_dst(h, M, N, K, A, lda, B, ldb, n, (_p * n)(*[int(x) for x in C]),
+                                            (_i64 * n)(*[int(x) for x in ldc]), variant, stream)
 
 
 def klineage_gemm_run_grouped_raw(h, M, N, K, A, lda, B, ldb, C, ldc, variant, stream) -> int:
@@ -296,6 +310,12 @@ class Gemm:
                                            int(variant), self._stream(stream))
         if st != KLINEAGE_OK:
             raise KlineageError(st, "klineage_gemm_run_grouped")
+
+    def run_multi_dst(self, A, B, Cs, M, N, K, lda, ldb, ldcs, variant, stream=None) -> None:
+        st = klineage_gemm_run_multi_dst_raw(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb,
+                                             [self._ptr(c) for c in Cs], ldcs, int(variant), self._stream(stream))
+        if st != KLINEAGE_OK:
+            raise KlineageError(st, "klineage_gemm_run_multi_dst")
 
     def run_raw(self, A, B, C, M, N, K, lda, ldb, ldc, variant, stream=None) -> int:
         return klineage_gemm_run_raw(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(C),

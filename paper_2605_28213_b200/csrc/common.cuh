@@ -178,6 +178,16 @@ struct alignas(128) GroupEntry {
     int tile_start;                     // first tile of this group in the launch-wide schedule
     int epi_tma;                        // this group's C can take the TMA-store epilogue
 };
+// One problem, several destinations (MODE 3): the epilogue writes every output block to each of
+// `n_dst` C matrices - the fused all-gather of an N-partitioned multi-GPU GEMM, where the
+// destinations are the column slice of this rank in every rank's C (peer memory, plain stores
+// or TMA stores; never a load).
+struct alignas(128) DstEntry {
+    CUtensorMap map_c;
+    void* C;
+    int64_t ldc;
+};
+constexpr int kMaxDst = 16;
 constexpr int kMaxGroups = 256;         // groups per launch (the schedule's prefix sums live in shared memory)
 
 cudaError_t launch_r0_naive(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
@@ -209,6 +219,12 @@ cudaError_t launch_r4_single_batched(const GemmArgs& g, const BatchArgs& b, RunC
 bool r4_single_grouped_possible(const GemmArgs* groups, int n, const RunContext& ctx);
 cudaError_t launch_r4_single_grouped(const GemmArgs* groups, int n, RunContext& ctx, cudaStream_t stream,
                                      int* kernel_id);
+// Multi-destination form (either kernel, chosen as for a plain call): dst[i] = (C pointer, pitch).
+bool r4_multi_dst_possible(const GemmArgs& g, const RunContext& ctx);
+cudaError_t launch_r4_multi_dst(const GemmArgs& g, void* const* C, const int64_t* ldc, int n_dst, RunContext& ctx,
+                                cudaStream_t stream, int* kernel_id);
+cudaError_t launch_r4_pair_multi_dst(const GemmArgs& g, void* const* C, const int64_t* ldc, int n_dst, RunContext& ctx,
+                                     cudaStream_t stream, int* kernel_id);
 // Grouped form: `groups` host descriptions (A, B, C, sizes, pitches in GemmArgs form; all with the
 // handle's B layout and C dtype).  The table is built in the handle's workspace on `stream`.
 bool r4_pair_grouped_possible(const GemmArgs* groups, int n, const RunContext& ctx);

@@ -523,6 +523,62 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups, const
     return KLINEAGE_OK;
 }
 
+// ------------------------------------------------------------------ one product, several destinations
+klineage_status_t klineage_gemm_run_multi_dst(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A,
+                                              int64_t lda, const void* B, int64_t ldb, int n_dst, void* const* C,
+                                              const int64_t* ldc, int variant, void* stream)
+{
+    if (!h || n_dst < 1 || n_dst > kMaxDst || !C || !ldc) return KLINEAGE_ERR_INVALID_ARG;
+    h->last_launches = 0;
+    const size_t celt = h->c_dtype == KLINEAGE_C_BF16 ? 2 : 4;
+    for (int d = 0; d < n_dst; ++d) {
+        const klineage_status_t chk =
+            klineage_gemm_check_args(h->b_layout, h->c_dtype, M, N, K, A, lda, B, ldb, C[d], ldc[d], variant);
+        if (chk != KLINEAGE_OK) return chk;
+    }
+    if (M == 0 || N == 0) {
+        h->last_kernel_id = -1;
+        return KLINEAGE_OK;
+    }
+    for (int d = 0; d < n_dst; ++d)
+        for (int e = d + 1; e < n_dst; ++e)
+            if (ranges_overlap(C[d], (size_t(M - 1) * ldc[d] + N) * celt, C[e], (size_t(M - 1) * ldc[e] + N) * celt))
+                return KLINEAGE_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (variant == KLINEAGE_TCGEN05 && K > 0 && h->ctx.cc_major == 10) {
+        const GemmArgs g = make_args(h, M, N, K, A, lda, B, ldb, nullptr, C[0], ldc[0]);
+        h->ctx.plan = R4Plan();
+        const auto it = h->plans.find(plan_key(h, M, N, K, A, lda, B, ldb, C[0], ldc[0]));
+        if (it != h->plans.end()) h->ctx.plan = it->second;
+        if (r4_multi_dst_possible(g, h->ctx)) {
+            // one launch: the epilogue stores every output block to each destination
+            DeviceGuard guard(h->ctx.device);
+            if (!guard.ok) return KLINEAGE_ERR_LAUNCH;
+            int kid = -1;
+            if (launch_r4_multi_dst(g, C, ldc, n_dst, h->ctx, s, &kid) != cudaSuccess) {
+                cudaGetLastError();
+                return KLINEAGE_ERR_LAUNCH;
+            }
+            h->last_kernel_id = kid;
+            h->last_launches = 1;
+            return KLINEAGE_OK;
+        }
+    }
+    // every other case: the rung's ordinary path into the first destination, then strided copies
+    // of that result to the others on the same stream
+    const klineage_status_t st = run_impl(h, M, N, K, A, lda, B, ldb, nullptr, C[0], ldc[0], variant, stream);
+    if (st != KLINEAGE_OK) return st;
+    DeviceGuard guard(h->ctx.device);
+    for (int d = 1; d < n_dst; ++d) {
+        if (cudaMemcpy2DAsync(C[d], size_t(ldc[d]) * celt, C[0], size_t(ldc[0]) * celt, size_t(N) * celt, size_t(M),
+                              cudaMemcpyDefault, s) != cudaSuccess) {
+            cudaGetLastError();
+            return KLINEAGE_ERR_LAUNCH;
+        }
+    }
+    return KLINEAGE_OK;
+}
+
 // ------------------------------------------------------------------ launch plans and the autotuner
 klineage_status_t klineage_gemm_plan_candidates(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A,
                                                 int64_t lda, const void* B, int64_t ldb, const void* C, int64_t ldc,

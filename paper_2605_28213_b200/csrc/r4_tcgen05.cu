@@ -82,6 +82,9 @@ struct R4Params {
     int64_t stride_c_bytes;
     const GroupEntry* groups;
     int n_groups;
+    // MODE 3: one problem, every output block stored to each entry of a destination table
+    const DstEntry* dsts;
+    int n_dst;
 };
 
 // One entry of the static schedule.
@@ -212,7 +215,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     // One unit of the schedule for this thread's role.
     auto unit_of = [&](int64_t u) {
         Unit x = decode_unit(u, p);
-        if (MODE != 0) {
+        if (MODE == 1 || MODE == 2) {
             const int half_cols = x.n0 % BN;                // 0, or 128 for the second half tile
             decode_multi<MODE>(x, g, p, gstart, group_hint);
             x.n0 += half_cols;
@@ -256,7 +259,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         prod.kb1 = x.kb1;
         prod.m0 = x.m0;
         prod.n0 = x.n0;     // a half tile still loads 256 columns from n0; its MMA reads the first 128
-        if (MODE != 0) {
+        if (MODE == 1 || MODE == 2) {
             prod.z = x.z;
             prod.ma = x.ma;
             prod.mb = x.mb;
@@ -316,7 +319,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             ptx::prefetch_tensormap(&map_a);
             ptx::prefetch_tensormap(&map_b);
         }
-        if (p.epi_tma && MODE != 2) ptx::prefetch_tensormap(&map_c);
+        if (p.epi_tma && MODE != 2 && MODE != 3) ptx::prefetch_tensormap(&map_c);
         // The launch is a programmatic dependent one: everything above (and the TMEM
         // allocation in warp 1) may overlap the tail of the previous kernel in the stream;
         // nothing below the wait touches global memory before that kernel has completed.
@@ -582,15 +585,24 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         ptx::fence_proxy_async_smem();
                         __syncwarp();
                         if (lane == 0) {
-                            if (MODE == 1)
+                            if (MODE == 1) {
                                 ptx::tma_store_3d(x.mc, col0, row0, x.z, b);
-                            else
+                            } else if (MODE == 3) {
+                                for (int d = 0; d < p.n_dst; ++d) ptx::tma_store_2d(&p.dsts[d].map_c, col0, row0, b);
+                            } else {
                                 ptx::tma_store_2d(x.mc, col0, row0, b);
+                            }
                             ptx::tma_store_commit();
                         }
                     } else {
                         __syncwarp();
                         // lane l owns 32-bit word l of every staged row: coalesced 128-byte rows.
+                        for (int dd = 0; dd < (MODE == 3 ? p.n_dst : 1); ++dd) {
+                        if (MODE == 3) {
+                            dst_f = static_cast<float*>(p.dsts[dd].C);
+                            dst_h = static_cast<uint16_t*>(p.dsts[dd].C);
+                        }
+                        const int64_t ldd = (MODE == 3) ? p.dsts[dd].ldc : ld;
                         for (int rr = 0; rr < rows; ++rr) {
                             const uint32_t word =
                                 *reinterpret_cast<const uint32_t*>(b + rr * 128 + (((lane >> 2) ^ (rr & 7)) << 4) +
@@ -598,7 +610,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                             const int64_t row = row0 + rr;
                             if (out_bf16) {
                                 const int col = col0 + 2 * lane;
-                                uint16_t* d = dst_h + row * ld + col;
+                                uint16_t* d = dst_h + row * ldd + col;
                                 if (col + 1 < x.N && (reinterpret_cast<uintptr_t>(d) & 3) == 0) {
                                     *reinterpret_cast<uint32_t*>(d) = word;
                                 } else {
@@ -607,8 +619,9 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                                 }
                             } else {
                                 const int col = col0 + lane;
-                                if (col < x.N) dst_f[row * ld + col] = __uint_as_float(word);
+                                if (col < x.N) dst_f[row * ldd + col] = __uint_as_float(word);
                             }
+                        }
                         }
                         __syncwarp();
                     }
@@ -936,7 +949,14 @@ __global__ void __launch_bounds__(256) repack_rows_kernel(const uint16_t* __rest
     }
 }
 
-cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id);
+bool c_store_by_tma(const GemmArgs& g);
+struct MultiDst {
+    void* const* C;
+    const int64_t* ldc;
+    int n;
+};
+cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id,
+                              const MultiDst* md = nullptr);
 
 }  // namespace
 
@@ -987,7 +1007,7 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
 
 namespace {
 
-cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
+cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id, const MultiDst* md)
 {
     if (ctx.max_smem_optin < kSmemBytes) return cudaErrorInvalidConfiguration;
     const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN;
@@ -1012,9 +1032,13 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     // Large aligned problems run on the CTA-pair kernel (tcgen05.mma.cta_group::2).
     if (pinned.kernel == 2 && (plan.swap || plan.splits != 1 || !r4_pair_possible(g, ctx))) return cudaErrorInvalidValue;
     const bool use_pair = pinned.kernel == 2 || (pinned.kernel == 0 && r4_pair_applicable(g, ctx));
-    if (!plan.swap && plan.splits == 1 && use_pair) return launch_r4_tcgen05_pair(g, ctx, stream, kernel_id);
+    if (md && (plan.swap || plan.splits != 1)) return cudaErrorNotSupported;
+    if (!plan.swap && plan.splits == 1 && use_pair)
+        return md ? launch_r4_pair_multi_dst(g, md->C, md->ldc, md->n, ctx, stream, kernel_id)
+                  : launch_r4_tcgen05_pair(g, ctx, stream, kernel_id);
 
     const bool generic = !(ctx.encode_tiled && tma_ok(g.A, g.lda, 2) && tma_ok(g.B, g.ldb, 2));
+    if (md && generic) return cudaErrorNotSupported;
     const int celt = g.c_bf16 ? 2 : 4;
     // Skinny mode: few activation rows -> they become the MMA's N, the weights its 128 rows.
     const bool swap = plan.swap;
@@ -1050,6 +1074,25 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     memset(&mb, 0, sizeof mb);
     memset(&mc, 0, sizeof mc);
     bool ok = true;
+    DstEntry table[kMaxDst];
+    if (md) {
+        // TMA stores only when every destination qualifies (one epilogue form per launch)
+        if (md->n < 1 || md->n > kMaxDst || ctx.workspace_bytes < sizeof(DstEntry) * md->n) return cudaErrorInvalidValue;
+        memset(table, 0, sizeof(DstEntry) * md->n);
+        p.epi_tma = ctx.encode_tiled ? 1 : 0;
+        for (int d = 0; d < md->n; ++d) {
+            GemmArgs gd = g;
+            gd.C = md->C[d];
+            gd.ldc = md->ldc[d];
+            if (!c_store_by_tma(gd)) p.epi_tma = 0;
+            table[d].C = md->C[d];
+            table[d].ldc = md->ldc[d];
+        }
+        for (int d = 0; d < md->n && p.epi_tma && ok; ++d)
+            ok = encode_map_2d(ctx, &table[d].map_c,
+                               g.c_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, table[d].C, g.N,
+                               g.M, table[d].ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    }
     // Skinny mode fetches only the activation rows the MMA reads (n_mma of them).
     const uint32_t a_box_rows = swap ? static_cast<uint32_t>(p.n_mma) : BM;
     p.stage_tx = a_box_rows * BK * 2 + kBBytes;
@@ -1063,7 +1106,7 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
             ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, g.ldb * 2, 64, BK,
                                      CU_TENSOR_MAP_SWIZZLE_128B);
     }
-    if (p.epi_tma)
+    if (p.epi_tma && !md)
         ok = ok && encode_map_2d(ctx, &mc, g.c_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
                                  g.C, g.N, g.M, g.ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return cudaErrorInvalidValue;
@@ -1085,6 +1128,15 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     const int64_t units = p.total_units;
     // A cluster handles exactly one tile, so the cluster path launches every unit as a CTA.
     const unsigned grid = static_cast<unsigned>((p.cluster || units < ctx.sm_count) ? units : ctx.sm_count);
+    if (md) {
+        // the table travels on the launch's stream, ahead of the kernel (staged before the call returns)
+        const cudaError_t e = cudaMemcpyAsync(ctx.workspace, table, sizeof(DstEntry) * md->n, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return e;
+        p.dsts = static_cast<const DstEntry*>(ctx.workspace);
+        p.n_dst = md->n;
+        return g.b_col ? launch<true, false, false, 3>(g, ma, mb, mc, p, grid, ctx.device, stream)
+                       : launch<false, false, false, 3>(g, ma, mb, mc, p, grid, ctx.device, stream);
+    }
 #define KLIN_R4_LAUNCH(BC, GE, SW) launch<BC, GE, SW>(g, ma, mb, mc, p, grid, ctx.device, stream)
     if (swap) {
         if (g.b_col) return generic ? KLIN_R4_LAUNCH(true, true, true) : KLIN_R4_LAUNCH(true, false, true);
@@ -1264,6 +1316,25 @@ cudaError_t launch_r4_single_grouped(const GemmArgs* groups, int n, RunContext& 
     const GemmArgs& g0 = groups[0];
     return g0.b_col ? launch<true, false, false, 2>(g0, none, none, none, p, grid, ctx.device, stream)
                     : launch<false, false, false, 2>(g0, none, none, none, p, grid, ctx.device, stream);
+}
+
+bool r4_multi_dst_possible(const GemmArgs& g, const RunContext& ctx)
+{
+    if (!ctx.encode_tiled || ctx.max_smem_optin < kSmemBytes || g.M <= 0 || g.N <= 0 || g.K <= 0) return false;
+    if (!tma_ok(g.A, g.lda, 2) || !tma_ok(g.B, g.ldb, 2)) return false;
+    const int64_t tiles = static_cast<int64_t>((g.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
+    const int64_t ldw = (static_cast<int64_t>(g.N) + 3) & ~int64_t(3);
+    SplitPlan sp;
+    if (!resolve_split(g.M, tiles, (g.K + BK - 1) / BK, ldw, ctx, ctx.plan, &sp)) return false;
+    return !sp.swap && sp.splits == 1;
+}
+
+cudaError_t launch_r4_multi_dst(const GemmArgs& g, void* const* C, const int64_t* ldc, int n_dst, RunContext& ctx,
+                                cudaStream_t stream, int* kernel_id)
+{
+    if (!C || !ldc || n_dst < 1 || n_dst > kMaxDst) return cudaErrorInvalidValue;
+    const MultiDst md = {C, ldc, n_dst};
+    return launch_r4_planned(g, ctx, stream, kernel_id, &md);
 }
 
 bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& pl)

@@ -68,6 +68,9 @@ struct PairParams {
     // grouped launches (MODE 2): table in device memory, one entry per group
     const GroupEntry* groups;
     int n_groups;
+    // multi-destination launches (MODE 3): every output block goes to each entry of the table
+    const DstEntry* dsts;
+    int n_dst;
 };
 
 // What a role needs to know about one tile of the schedule.
@@ -145,6 +148,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_f
 
 // MODE 0: one problem (tensor maps 2-D).  MODE 1: batched (3-D tensor maps, z = batch).
 // MODE 2: grouped (per-group tensor maps and sizes from a table in device memory).
+// MODE 3: one problem whose C goes to several destinations (table of C maps / pointers).
 template <bool BCOL, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -181,7 +185,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         if (MODE != 2) {
             ptx::prefetch_tensormap(&map_a);
             ptx::prefetch_tensormap(&map_b);
-            if (p.epi_tma) ptx::prefetch_tensormap(&map_c);
+            if (p.epi_tma && MODE != 3) ptx::prefetch_tensormap(&map_c);
         }
         if (blockIdx.x == 0) g.status[1] = p.kid;
     }
@@ -418,31 +422,41 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     ptx::fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        if (MODE == 1)
+                        if (MODE == 1) {
                             ptx::tma_store_3d(x.mc, col0, row0, x.z, b);
-                        else
+                        } else if (MODE == 3) {
+                            for (int d = 0; d < p.n_dst; ++d) ptx::tma_store_2d(&p.dsts[d].map_c, col0, row0, b);
+                        } else {
                             ptx::tma_store_2d(x.mc, col0, row0, b);
+                        }
                         ptx::tma_store_commit();
                     }
                 } else {
                     __syncwarp();
+                    for (int d = 0; d < (MODE == 3 ? p.n_dst : 1); ++d) {
+                    if (MODE == 3) {
+                        dst_f = static_cast<float*>(p.dsts[d].C);
+                        dst_h = static_cast<uint16_t*>(p.dsts[d].C);
+                    }
+                    const int64_t ldd = (MODE == 3) ? p.dsts[d].ldc : x.ldc;
                     for (int rr = 0; rr < rows; ++rr) {
                         const uint32_t word = *reinterpret_cast<const uint32_t*>(
                             b + rr * 128 + (((lane >> 2) ^ (rr & 7)) << 4) + (lane & 3) * 4);
                         const int64_t row = row0 + rr;
                         if (out_bf16) {
                             const int col = col0 + 2 * lane;
-                            uint16_t* d = dst_h + row * x.ldc + col;
-                            if (col + 1 < x.N && (reinterpret_cast<uintptr_t>(d) & 3) == 0) {
-                                *reinterpret_cast<uint32_t*>(d) = word;
+                            uint16_t* o = dst_h + row * ldd + col;
+                            if (col + 1 < x.N && (reinterpret_cast<uintptr_t>(o) & 3) == 0) {
+                                *reinterpret_cast<uint32_t*>(o) = word;
                             } else {
-                                if (col < x.N) d[0] = static_cast<uint16_t>(word & 0xFFFFu);
-                                if (col + 1 < x.N) d[1] = static_cast<uint16_t>(word >> 16);
+                                if (col < x.N) o[0] = static_cast<uint16_t>(word & 0xFFFFu);
+                                if (col + 1 < x.N) o[1] = static_cast<uint16_t>(word >> 16);
                             }
                         } else {
                             const int col = col0 + lane;
-                            if (col < x.N) dst_f[row * x.ldc + col] = __uint_as_float(word);
+                            if (col < x.N) dst_f[row * ldd + col] = __uint_as_float(word);
                         }
+                    }
                     }
                     __syncwarp();
                 }
@@ -685,7 +699,29 @@ cudaError_t launch_r4_pair_grouped(const GemmArgs* groups, int n, RunContext& ct
                     : launch<false, 2>(g0, none, none, none, p, grid, ctx.device, stream);
 }
 
+namespace {
+cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const int64_t* dst_ldc, int n_dst,
+                                    RunContext& ctx, cudaStream_t stream, int* kernel_id);
+}
+
 cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
+{
+    return launch_pair_one_problem(g, nullptr, nullptr, 0, ctx, stream, kernel_id);
+}
+
+cudaError_t launch_r4_pair_multi_dst(const GemmArgs& g, void* const* C, const int64_t* ldc, int n_dst, RunContext& ctx,
+                                     cudaStream_t stream, int* kernel_id)
+{
+    if (n_dst < 1 || n_dst > kMaxDst || !C || !ldc) return cudaErrorInvalidValue;
+    return launch_pair_one_problem(g, C, ldc, n_dst, ctx, stream, kernel_id);
+}
+
+namespace {
+
+// n_dst == 0: the plain launch (C and its pitch from g).  n_dst >= 1: the multi-destination launch;
+// g.C / g.ldc are ignored, the destination table is built in the workspace on `stream`.
+cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const int64_t* dst_ldc, int n_dst,
+                                    RunContext& ctx, cudaStream_t stream, int* kernel_id)
 {
     PairParams p;
     memset(&p, 0, sizeof p);
@@ -701,6 +737,21 @@ cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStrea
                  (static_cast<int64_t>(g.N) * celt) % 16 == 0 && g.ldc * celt < (int64_t(1) << 40))
                     ? 1
                     : 0;
+    DstEntry table[kMaxDst];
+    if (n_dst > 0) {
+        // TMA stores only when every destination qualifies (one epilogue form per launch)
+        if (ctx.workspace_bytes < sizeof(DstEntry) * n_dst) return cudaErrorInvalidValue;
+        memset(table, 0, sizeof(DstEntry) * n_dst);
+        p.epi_tma = 1;
+        for (int d = 0; d < n_dst; ++d) {
+            GemmArgs gd = g;
+            gd.C = dst_c[d];
+            gd.ldc = dst_ldc[d];
+            if (!c_takes_tma_store(gd)) p.epi_tma = 0;
+            table[d].C = dst_c[d];
+            table[d].ldc = dst_ldc[d];
+        }
+    }
     // Instruction descriptor: fp32 accumulator, bf16 A/B, A K-major, B K-major (column-major B) or
     // MN-major (row-major B), N = 256, M = 256 (128 rows in each CTA of the pair).
     const uint32_t w_major = g.b_col ? 0u : 1u;
@@ -724,17 +775,32 @@ cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStrea
     else
         ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, g.ldb * 2, 64, BK,
                                  CU_TENSOR_MAP_SWIZZLE_128B);
-    if (p.epi_tma)
+    if (p.epi_tma && n_dst == 0)
         ok = ok && encode_map_2d(ctx, &mc, g.c_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
                                  g.C, g.N, g.M, g.ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    for (int d = 0; d < n_dst && p.epi_tma && ok; ++d)
+        ok = encode_map_2d(ctx, &table[d].map_c,
+                           g.c_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, table[d].C, g.N, g.M,
+                           table[d].ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return cudaErrorInvalidValue;
 
     p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + 32 + ctx.kid_flags;
     *kernel_id = p.kid;
     const int64_t max_pairs = ctx.sm_count / 2;
     const unsigned grid = 2u * static_cast<unsigned>(p.total_tiles < max_pairs ? p.total_tiles : max_pairs);
+    if (n_dst > 0) {
+        // the table travels on the launch's stream, ahead of the kernel (staged before the call returns)
+        const cudaError_t e = cudaMemcpyAsync(ctx.workspace, table, sizeof(DstEntry) * n_dst, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return e;
+        p.dsts = static_cast<const DstEntry*>(ctx.workspace);
+        p.n_dst = n_dst;
+        return g.b_col ? launch<true, 3>(g, ma, mb, mc, p, grid, ctx.device, stream)
+                       : launch<false, 3>(g, ma, mb, mc, p, grid, ctx.device, stream);
+    }
     return g.b_col ? launch<true, 0>(g, ma, mb, mc, p, grid, ctx.device, stream)
                    : launch<false, 0>(g, ma, mb, mc, p, grid, ctx.device, stream);
 }
+
+}  // namespace
 
 }  // namespace klin
