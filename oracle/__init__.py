@@ -1,1 +1,1 @@
-"""CPU oracle for the bf16 GEMM lineage.  Test infrastructure only: never imported by the product."""
+"""CPU oracles of the bf16 GEMM lineage and of the fp16 Conv2d workload.  Test infrastructure only: never imported by the product."""

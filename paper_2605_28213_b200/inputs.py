@@ -139,3 +139,67 @@ def make_config(name: str, seed: int, integer: bool = False, c_bf16: Optional[bo
 def config_shape(name: str):
     M, N, K, lda, ldb, ldc, col, cb = _CONFIGS[name][:8]
     return dict(M=M, N=N, K=K, lda=lda, ldb=ldb, ldc=ldc, b_col_major=col, c_bf16=cb)
+
+
+# ---------------------------------------------------------------------------- Conv2d inputs (fp16)
+@dataclass
+class ConvCase:
+    """A channels-last Conv2d problem: x (N, H, W, C) and w (F, R, S, C) as fp16 bit patterns (uint16)."""
+    name: str
+    N: int
+    H: int
+    W: int
+    C: int
+    F: int
+    R: int
+    S: int
+    pad: Tuple[int, int]
+    stride: Tuple[int, int]
+    y_f16: bool
+    x: np.ndarray = field(repr=False)
+    w: np.ndarray = field(repr=False)
+
+    @property
+    def P(self) -> int:
+        return (self.H + 2 * self.pad[0] - self.R) // self.stride[0] + 1
+
+    @property
+    def Q(self) -> int:
+        return (self.W + 2 * self.pad[1] - self.S) // self.stride[1] + 1
+
+    @property
+    def K(self) -> int:
+        return self.R * self.S * self.C
+
+    @property
+    def flops(self) -> float:
+        return 2.0 * self.N * self.P * self.Q * self.F * self.K
+
+
+def draw_f16(shape, dist: str, seed: int, tensor_id: int, sigma: float = 1.0) -> np.ndarray:
+    """fp16 bit patterns drawn as in ``draw`` (fp64 -> fp32 -> fp16, round to nearest even)."""
+    g = _rng(seed, tensor_id)
+    if dist == "uniform":
+        v = (2.0 * g.random(shape) - 1.0).astype(np.float32)
+    elif dist == "normal":
+        v = (g.standard_normal(shape) * sigma).astype(np.float32)
+    elif dist == "integer":
+        v = g.integers(-4, 5, size=shape).astype(np.float32)
+    else:
+        raise ValueError(f"unknown distribution {dist!r}")
+    return v.astype(np.float16).view(np.uint16)
+
+
+def make_conv_case(N: int, H: int, W: int, C: int, F: int, R: int, S: int, seed: int, pad=(1, 1), stride=(1, 1),
+                   dist: str = "normal", y_f16: bool = True, name: str = "") -> ConvCase:
+    """x ~ dist (sigma 1), w ~ dist with sigma 1/sqrt(R*S*C) for "normal" (outputs of order 1)."""
+    sig_w = 1.0 / np.sqrt(max(R * S * C, 1)) if dist == "normal" else 1.0
+    x = draw_f16((N, H, W, C), dist, seed, 10)
+    w = draw_f16((F, R, S, C), dist, seed, 11, sig_w)
+    return ConvCase(name or f"conv{N}x{H}x{W}x{C}-f{F}-{R}x{S}", N, H, W, C, F, R, S, tuple(pad), tuple(stride), y_f16,
+                    x, w)
+
+
+def conv_benchmark_case(seed: int, integer: bool = False) -> ConvCase:
+    """The paper's Conv2d shape: N=8, C=64, 56x56, F=128, 3x3, fp16; read as padding 1, stride 1."""
+    return make_conv_case(8, 56, 56, 64, 128, 3, 3, seed, dist="integer" if integer else "normal", name="conv_t2")
