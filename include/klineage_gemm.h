@@ -49,7 +49,9 @@ typedef enum {
 
 typedef enum {
     KLINEAGE_C_F32 = 0, /* C holds the fp32 accumulator                                  */
-    KLINEAGE_C_BF16 = 1 /* C holds the accumulator rounded to bf16, round-to-nearest-even */
+    KLINEAGE_C_BF16 = 1, /* C holds the accumulator rounded to bf16, round-to-nearest-even */
+    KLINEAGE_C_F16 = 2   /* klineage_conv2d_run only: y holds the accumulator rounded to fp16 (RNE); the
+                            GEMM calls refuse a handle of this dtype with KLINEAGE_ERR_INVALID_ARG       */
 } klineage_ctype_t;
 
 /*
@@ -258,6 +260,38 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups,
                                             const void* const* B, const int64_t* ldb,
                                             void* const* C, const int64_t* ldc,
                                             int variant, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * Conv2d as an implicit GEMM on the tcgen05 rung (paper, Evaluation, Table 2: Conv2d,
+ * N=8, C=64, 56x56, F=128, 3x3, FP16; the paper fixes neither layout, padding nor
+ * stride - channels-last and "same" padding are this library's reading for that
+ * shape, the call takes any padding and stride).
+ *
+ *   y[n][p][q][f] = sum_{r,s,c} x[n][p*stride_h + r - pad_h][q*stride_w + s - pad_w][c] * w[f][r][s][c]
+ *
+ * (cross-correlation, zero outside the image), P = (H + 2 pad_h - R)/stride_h + 1,
+ * Q likewise.  x: device, fp16 bits, (N, H, W, C) contiguous; w: device, fp16 bits,
+ * (F, R, S, C) contiguous; y: device, (N, P, Q, F) contiguous, fp32 or fp16 per the
+ * handle's c_dtype (KLINEAGE_C_F32 or KLINEAGE_C_F16; the handle's B layout is not
+ * used); fp32 accumulation.  Pointers need element alignment only; 16-byte aligned x
+ * with C % 8 == 0 selects 16-byte patch loads.  variant: KLINEAGE_NAIVE (direct
+ * convolution, one thread per output) or KLINEAGE_TCGEN05 (rows = output pixels,
+ * columns = filters, k = (r, s, c); producer warps gather the patches straight into
+ * the swizzled shared-memory operand layout - no im2col buffer exists - and
+ * tcgen05.mma.kind::f16 multiplies fp16 operands into TMEM).  No output pixel
+ * (N*P*Q == 0) or F == 0: nothing is launched; C == 0: y is zero-filled.
+ * Errors: INVALID_ARG (sizes, R or S outside 1..64, padding or stride outside
+ * 0..64 / 1..64, a filter larger than the padded image, null or overlapping
+ * buffers, a handle of dtype BF16), BAD_VARIANT, UNSUPPORTED_DEVICE, LAUNCH.
+ */
+klineage_status_t klineage_conv2d_check_args(int y_dtype, int64_t N, int64_t H, int64_t W, int64_t C,
+                                             int64_t F, int64_t R, int64_t S, int64_t pad_h, int64_t pad_w,
+                                             int64_t stride_h, int64_t stride_w,
+                                             const void* x, const void* w, const void* y, int variant);
+klineage_status_t klineage_conv2d_run(klineage_gemm_t h, int64_t N, int64_t H, int64_t W, int64_t C,
+                                      int64_t F, int64_t R, int64_t S, int64_t pad_h, int64_t pad_w,
+                                      int64_t stride_h, int64_t stride_w,
+                                      const void* x, const void* w, void* y, int variant, void* stream);
 
 /*
  * One product, several destinations:  C_d <- A . B  for d in [0, n_dst), n_dst <= 16.

@@ -24,7 +24,7 @@ KLINEAGE_ERR_INTERNAL = 7
 KLINEAGE_ERR_SCRATCH_LIMIT = 8
 
 KLINEAGE_B_ROW_MAJOR, KLINEAGE_B_COL_MAJOR = 0, 1
-KLINEAGE_C_F32, KLINEAGE_C_BF16 = 0, 1
+KLINEAGE_C_F32, KLINEAGE_C_BF16, KLINEAGE_C_F16 = 0, 1, 2
 KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELINED, KLINEAGE_TCGEN05, KLINEAGE_MMA_SYNC = range(6)
 # the five-step ladder, then the intermediate legacy tensor-core rung ("3.5")
 VARIANTS = (KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELINED, KLINEAGE_TCGEN05,
@@ -35,7 +35,7 @@ EXPORTED_SYMBOLS = (
     "klineage_gemm_get_device_status", "klineage_gemm_last_kernel_id", "klineage_status_string",
     "klineage_variant_name", "klineage_gemm_run_noalloc", "klineage_gemm_run_addmm",
     "klineage_gemm_run_batched", "klineage_gemm_run_grouped", "klineage_gemm_last_launch_count",
-    "klineage_gemm_run_multi_dst",
+    "klineage_gemm_run_multi_dst", "klineage_conv2d_run", "klineage_conv2d_check_args",
     "klineage_gemm_plan_candidates", "klineage_gemm_set_plan", "klineage_gemm_get_plan", "klineage_gemm_autotune",
 )
 
@@ -139,6 +139,22 @@ def klineage_gemm_run_grouped_raw(h, M, N, K, A, lda, B, ldb, C, ldc, variant, s
     ptrs = lambda xs: (_p * n)(*[None if x is None else int(x) for x in xs])
     return _lib.klineage_gemm_run_grouped(h, n, i64s(M), i64s(N), i64s(K), ptrs(A), i64s(lda), ptrs(B), i64s(ldb),
                                           ptrs(C), i64s(ldc), variant, stream)
+
+
+_lib.klineage_conv2d_run.restype = _int
+_lib.klineage_conv2d_run.argtypes = [_p] + [_i64] * 11 + [_p, _p, _p, _int, _p]
+_lib.klineage_conv2d_check_args.restype = _int
+_lib.klineage_conv2d_check_args.argtypes = [_int] + [_i64] * 11 + [_p, _p, _p, _int]
+
+
+def klineage_conv2d_run_raw(h, N, H, W, C, F, R, S, pad_h, pad_w, stride_h, stride_w, x, w, y, variant, stream) -> int:
+    """Raw status of the channels-last fp16 Conv2d (x, w, y: device addresses)."""
+    return _lib.klineage_conv2d_run(h, N, H, W, C, F, R, S, pad_h, pad_w, stride_h, stride_w, x, w, y, variant, stream)
+
+
+def klineage_conv2d_check_args(y_dtype, N, H, W, C, F, R, S, pad_h, pad_w, stride_h, stride_w, x, w, y, variant) -> int:
+    return _lib.klineage_conv2d_check_args(y_dtype, N, H, W, C, F, R, S, pad_h, pad_w, stride_h, stride_w, x, w, y,
+                                           variant)
 
 
 class klineage_gemm_plan_t(ctypes.Structure):
@@ -345,6 +361,48 @@ class Gemm:
 
     def last_launch_count(self) -> int:
         return _lib.klineage_gemm_last_launch_count(self._h)
+
+    def close(self) -> None:
+        if self._h is not None:
+            klineage_gemm_destroy(self._h)
+            self._h = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Conv2d:
+    """Handle wrapper of the fp16 channels-last Conv2d: ``Conv2d(device, y_f16).run(x, w, y, N, H, W, C, F, R, S, ...)``.
+
+    ``x`` (N, H, W, C), ``w`` (F, R, S, C) hold fp16 values, ``y`` (N, P, Q, F) fp16 or fp32; torch CUDA tensors (only
+    ``data_ptr()`` is used) or integer device addresses.  variant 0 = direct convolution, 4 = implicit GEMM on tcgen05.
+    """
+
+    def __init__(self, device: int = 0, y_f16: bool = True):
+        self.device, self.y_f16 = int(device), bool(y_f16)
+        self._h: Optional[int] = klineage_gemm_create(self.device, KLINEAGE_B_COL_MAJOR,
+                                                      KLINEAGE_C_F16 if y_f16 else KLINEAGE_C_F32, 0)
+
+    def run(self, x, w, y, N, H, W, C, F, R, S, pad=(1, 1), stride=(1, 1), variant=4, stream=None) -> None:
+        st = klineage_conv2d_run_raw(self._h, N, H, W, C, F, R, S, pad[0], pad[1], stride[0], stride[1], Gemm._ptr(x),
+                                     Gemm._ptr(w), Gemm._ptr(y), int(variant), Gemm._stream(stream))
+        if st != KLINEAGE_OK:
+            raise KlineageError(st, "klineage_conv2d_run")
+
+    def device_status(self):
+        return klineage_gemm_get_device_status(self._h)
+
+    def last_kernel_id(self) -> int:
+        return klineage_gemm_last_kernel_id(self._h)
 
     def close(self) -> None:
         if self._h is not None:

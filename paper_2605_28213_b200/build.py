@@ -11,7 +11,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libklineage_gemm.so"
 SOURCES = ["klineage_gemm.cu", "r0_naive.cu", "r1_tiled.cu", "r2_vectorized.cu", "r3_pipelined.cu", "r35_mma_sync.cu",
-           "r4_tcgen05.cu", "r4_tcgen05_pair.cu"]
+           "r4_tcgen05.cu", "r4_tcgen05_pair.cu", "conv_naive.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

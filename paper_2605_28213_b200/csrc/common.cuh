@@ -4,6 +4,7 @@
 #include <cstdint>
 #include <cuda.h>          // CUtensorMap and its enums only; libcuda is never linked
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 namespace klin {
@@ -26,6 +27,7 @@ struct GemmArgs {
     int c_bf16;
     unsigned* status;
     const uint16_t* bias;   // optional: N bf16 values added to every row of A.B (AddMM); nullptr = plain GEMM
+    int f16 = 0;            // 1: operands are fp16 and a 2-byte C is fp16 (Conv2d as implicit GEMM); 0: bf16
 };
 
 // Device-side error codes written to status[0].
@@ -43,6 +45,8 @@ enum KernelId : int {
     kIdTcgen05 = 400,         // + 1 generic-proxy producer, + 2 direct epilogue, + 4 split-K, + 8 skinny (swapped operands), + 16 cluster reduce, + 32 CTA pair,
                               // + 64 unaligned operands repacked into the workspace first
     kIdMmaSync = 500,         // rung 3.5 (mma.sync); + 1 when the producer-thread path replaces TMA
+    kIdConvNaive = 600,       // direct convolution, one thread per output
+    kIdConvTcgen05 = 700,     // implicit GEMM on the tcgen05 rung; + 2 direct epilogue, + 1 slow gather (C % 8 != 0 or unaligned x)
     kIdZeroFill = 900,
 };
 
@@ -63,6 +67,23 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     return static_cast<uint32_t>(float_to_bf16_bits(lo)) | (static_cast<uint32_t>(float_to_bf16_bits(hi)) << 16);
 }
+
+// Two floats -> packed 16-bit pair in the output type (bf16 or fp16), round to nearest even.
+__device__ __forceinline__ uint32_t pack_out2(float lo, float hi, int f16)
+{
+    if (f16) {
+        const __half2 h = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<const uint32_t*>(&h);
+    }
+    return pack_bf16x2(lo, hi);
+}
+
+// Geometry of a channels-last Conv2d run as an implicit GEMM (paper, Evaluation, Table 2: Conv2d):
+// x (N, H, W, C), w (F, R, S, C), y (N, P, Q, F); GEMM row m = (n, p, q), column f, k = (r, s, c).
+struct ConvGeom {
+    int H, W, C, P, Q, R, S;
+    int pad_h, pad_w, stride_h, stride_w;
+};
 
 // The bias of column `col` (0 when the call has none); col must be < N.
 __device__ __forceinline__ float bias_at(const GemmArgs& g, int64_t col)
@@ -219,6 +240,12 @@ cudaError_t launch_r4_single_batched(const GemmArgs& g, const BatchArgs& b, RunC
 bool r4_single_grouped_possible(const GemmArgs* groups, int n, const RunContext& ctx);
 cudaError_t launch_r4_single_grouped(const GemmArgs* groups, int n, RunContext& ctx, cudaStream_t stream,
                                      int* kernel_id);
+// Conv2d as an implicit GEMM on the single-CTA kernel (generic-proxy producers gather the patches).
+// g: M = N*P*Q, N = F, K = R*S*C, A = x, B = w (column-major, ldb = K), C = y (ldc = F), f16 = 1.
+cudaError_t launch_r4_conv2d(const GemmArgs& g, const ConvGeom& geom, RunContext& ctx, cudaStream_t stream,
+                             int* kernel_id);
+// Direct convolution, one thread per output value (the naive rung of the same operation).
+cudaError_t launch_conv2d_naive(const GemmArgs& g, const ConvGeom& geom, cudaStream_t stream, int* kernel_id);
 // Multi-destination form (either kernel, chosen as for a plain call): dst[i] = (C pointer, pitch).
 bool r4_multi_dst_possible(const GemmArgs& g, const RunContext& ctx);
 cudaError_t launch_r4_multi_dst(const GemmArgs& g, void* const* C, const int64_t* ldc, int n_dst, RunContext& ctx,

@@ -154,7 +154,8 @@ klineage_status_t klineage_gemm_create(klineage_gemm_t* out, const klineage_gemm
     *out = nullptr;
     if (!cfg) return KLINEAGE_ERR_INVALID_ARG;
     if (cfg->b_layout != KLINEAGE_B_ROW_MAJOR && cfg->b_layout != KLINEAGE_B_COL_MAJOR) return KLINEAGE_ERR_INVALID_ARG;
-    if (cfg->c_dtype != KLINEAGE_C_F32 && cfg->c_dtype != KLINEAGE_C_BF16) return KLINEAGE_ERR_INVALID_ARG;
+    if (cfg->c_dtype != KLINEAGE_C_F32 && cfg->c_dtype != KLINEAGE_C_BF16 && cfg->c_dtype != KLINEAGE_C_F16)
+        return KLINEAGE_ERR_INVALID_ARG;
     if (cfg->flags != 0) return KLINEAGE_ERR_INVALID_ARG;
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev) {
@@ -576,6 +577,98 @@ klineage_status_t klineage_gemm_run_multi_dst(klineage_gemm_t h, int64_t M, int6
             return KLINEAGE_ERR_LAUNCH;
         }
     }
+    return KLINEAGE_OK;
+}
+
+// ------------------------------------------------------------------ Conv2d
+klineage_status_t klineage_conv2d_check_args(int y_dtype, int64_t N, int64_t H, int64_t W, int64_t C, int64_t F,
+                                             int64_t R, int64_t S, int64_t pad_h, int64_t pad_w, int64_t stride_h,
+                                             int64_t stride_w, const void* x, const void* w, const void* y, int variant)
+{
+    if (y_dtype != KLINEAGE_C_F32 && y_dtype != KLINEAGE_C_F16) return KLINEAGE_ERR_INVALID_ARG;
+    if (variant != KLINEAGE_NAIVE && variant != KLINEAGE_TCGEN05) return KLINEAGE_ERR_BAD_VARIANT;
+    const int64_t lim = int64_t(1) << 20;
+    if (N < 0 || H < 0 || W < 0 || C < 0 || F < 0 || N >= lim || H >= lim || W >= lim || C >= lim || F >= lim)
+        return KLINEAGE_ERR_INVALID_ARG;
+    if (R < 1 || S < 1 || R > 64 || S > 64 || stride_h < 1 || stride_w < 1 || stride_h > 64 || stride_w > 64 ||
+        pad_h < 0 || pad_w < 0 || pad_h > 64 || pad_w > 64)
+        return KLINEAGE_ERR_INVALID_ARG;
+    if (H + 2 * pad_h < R || W + 2 * pad_w < S) return KLINEAGE_ERR_INVALID_ARG;     // no output pixel
+    const int64_t P = (H + 2 * pad_h - R) / stride_h + 1, Q = (W + 2 * pad_w - S) / stride_w + 1;
+    const int64_t M = N * P * Q, K = R * S * C;
+    if (M >= (int64_t(1) << 31) || K >= (int64_t(1) << 31)) return KLINEAGE_ERR_INVALID_ARG;
+    if (M == 0 || F == 0) return KLINEAGE_OK;
+    const size_t yelt = y_dtype == KLINEAGE_C_F16 ? 2 : 4;
+    if (!y || reinterpret_cast<uintptr_t>(y) % yelt) return KLINEAGE_ERR_INVALID_ARG;
+    if (K > 0) {
+        if (!x || !w || reinterpret_cast<uintptr_t>(x) % 2 || reinterpret_cast<uintptr_t>(w) % 2) return KLINEAGE_ERR_INVALID_ARG;
+        const size_t xb = size_t(N) * H * W * C * 2, wb = size_t(F) * K * 2, yb = size_t(M) * F * yelt;
+        if (ranges_overlap(x, xb, y, yb) || ranges_overlap(w, wb, y, yb)) return KLINEAGE_ERR_INVALID_ARG;
+    }
+    return KLINEAGE_OK;
+}
+
+klineage_status_t klineage_conv2d_run(klineage_gemm_t h, int64_t N, int64_t H, int64_t W, int64_t C, int64_t F,
+                                      int64_t R, int64_t S, int64_t pad_h, int64_t pad_w, int64_t stride_h,
+                                      int64_t stride_w, const void* x, const void* w, void* y, int variant, void* stream)
+{
+    if (!h) return KLINEAGE_ERR_INVALID_ARG;
+    h->last_launches = 0;
+    const klineage_status_t chk = klineage_conv2d_check_args(h->c_dtype, N, H, W, C, F, R, S, pad_h, pad_w, stride_h,
+                                                             stride_w, x, w, y, variant);
+    if (chk != KLINEAGE_OK) return chk;
+    ConvGeom cv;
+    cv.H = static_cast<int>(H);
+    cv.W = static_cast<int>(W);
+    cv.C = static_cast<int>(C);
+    cv.R = static_cast<int>(R);
+    cv.S = static_cast<int>(S);
+    cv.pad_h = static_cast<int>(pad_h);
+    cv.pad_w = static_cast<int>(pad_w);
+    cv.stride_h = static_cast<int>(stride_h);
+    cv.stride_w = static_cast<int>(stride_w);
+    cv.P = static_cast<int>((H + 2 * pad_h - R) / stride_h + 1);
+    cv.Q = static_cast<int>((W + 2 * pad_w - S) / stride_w + 1);
+    const int64_t M = N * cv.P * cv.Q, K = R * S * C;
+    if (M == 0 || F == 0) {
+        h->last_kernel_id = -1;
+        return KLINEAGE_OK;
+    }
+    if (variant == KLINEAGE_TCGEN05 && h->ctx.cc_major != 10) return KLINEAGE_ERR_UNSUPPORTED_DEVICE;
+    DeviceGuard guard(h->ctx.device);
+    if (!guard.ok) return KLINEAGE_ERR_LAUNCH;
+    // the implicit GEMM: rows = output pixels, columns = filters, k = (r, s, c); the weights are its
+    // column-major B with pitch K, y its row-major C with pitch F
+    GemmArgs g;
+    g.M = static_cast<int>(M);
+    g.N = static_cast<int>(F);
+    g.K = static_cast<int>(K);
+    g.A = static_cast<const uint16_t*>(x);
+    g.lda = K;
+    g.B = static_cast<const uint16_t*>(w);
+    g.ldb = K;
+    g.C = y;
+    g.ldc = F;
+    g.b_col = 1;
+    g.c_bf16 = h->c_dtype == KLINEAGE_C_F16 ? 1 : 0;     // "2-byte C"; f16 selects the rounding
+    g.status = h->status;
+    g.bias = nullptr;
+    g.f16 = 1;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int kid = -1;
+    cudaError_t e;
+    if (K == 0)
+        e = launch_zero_fill(g, s, &kid);
+    else if (variant == KLINEAGE_NAIVE)
+        e = launch_conv2d_naive(g, cv, s, &kid);
+    else
+        e = launch_r4_conv2d(g, cv, h->ctx, s, &kid);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return KLINEAGE_ERR_LAUNCH;
+    }
+    h->last_kernel_id = kid;
+    h->last_launches = 1;
     return KLINEAGE_OK;
 }
 

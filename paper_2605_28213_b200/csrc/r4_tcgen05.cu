@@ -85,6 +85,10 @@ struct R4Params {
     // MODE 3: one problem, every output block stored to each entry of a destination table
     const DstEntry* dsts;
     int n_dst;
+    // MODE 4: Conv2d as an implicit GEMM (the A producers gather input patches)
+    ConvGeom conv;
+    int conv_fast;          // 1: C % 8 == 0 and x 16-byte aligned - an 8-k chunk is one 16-byte load
+    int half_only;          // every unit is the first 128-column half of its tile (problems with N <= 128)
 };
 
 // One entry of the static schedule.
@@ -154,7 +158,10 @@ __device__ __forceinline__ Unit decode_unit(int64_t u, const R4Params& p)
         }
     } else {
         x.split = 0;
-        if (u < p.full_units) {
+        if (p.half_only) {
+            x.tile = u;
+            x.ncols = BN / 2;
+        } else if (u < p.full_units) {
             x.tile = u;
         } else {
             const int64_t v = u - p.full_units;
@@ -558,8 +565,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         }
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
-                            w[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-                            w[16 + i] = pack_bf16x2(__uint_as_float(v2[2 * i]), __uint_as_float(v2[2 * i + 1]));
+                            w[i] = pack_out2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]), g.f16);
+                            w[16 + i] = pack_out2(__uint_as_float(v2[2 * i]), __uint_as_float(v2[2 * i + 1]), g.f16);
                         }
                     } else {
                         ptx::tmem_ld_wait();
@@ -688,6 +695,49 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 uint8_t* sb = sa + kABytes;
                 const int k0 = kb * BK;
                 // A: 128 rows x 8 chunks of 8 k (K-major, 128-byte swizzle)
+                if (MODE == 4) {
+                    // implicit GEMM: row m is the output pixel (n, p, q), k the filter tap and channel
+                    // (r, s, c); the element is x[n][p*stride_h + r - pad_h][q*stride_w + s - pad_w][c]
+                    // or zero outside the image
+                    const ConvGeom& cv = p.conv;
+                    for (int c = pt; c < BM * 8; c += kProducerThreads) {
+                        const int r = c >> 3, kc = c & 7;
+                        const int gm = m0 + r;
+                        const int gk = k0 + kc * 8;
+                        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                        if (gm < g.M && gk < g.K) {
+                            const int q = gm % cv.Q, t = gm / cv.Q;
+                            const int pp = t % cv.P, n = t / cv.P;
+                            if (p.conv_fast) {
+                                const int tap = gk / cv.C, ch = gk - tap * cv.C;
+                                const int fr = tap / cv.S, fs = tap - fr * cv.S;
+                                const int h = pp * cv.stride_h + fr - cv.pad_h, w = q * cv.stride_w + fs - cv.pad_w;
+                                if (h >= 0 && h < cv.H && w >= 0 && w < cv.W)
+                                    v = __ldg(reinterpret_cast<const uint4*>(
+                                        g.A + ((static_cast<int64_t>(n) * cv.H + h) * cv.W + w) * cv.C + ch));
+                            } else {
+                                uint16_t e8[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    const int k = gk + e;
+                                    e8[e] = 0;
+                                    if (k < g.K) {
+                                        const int tap = k / cv.C, ch = k - tap * cv.C;
+                                        const int fr = tap / cv.S, fs = tap - fr * cv.S;
+                                        const int h = pp * cv.stride_h + fr - cv.pad_h, w = q * cv.stride_w + fs - cv.pad_w;
+                                        if (h >= 0 && h < cv.H && w >= 0 && w < cv.W)
+                                            e8[e] = __ldg(g.A + ((static_cast<int64_t>(n) * cv.H + h) * cv.W + w) * cv.C + ch);
+                                    }
+                                }
+                                v.x = e8[0] | (uint32_t(e8[1]) << 16);
+                                v.y = e8[2] | (uint32_t(e8[3]) << 16);
+                                v.z = e8[4] | (uint32_t(e8[5]) << 16);
+                                v.w = e8[6] | (uint32_t(e8[7]) << 16);
+                            }
+                        }
+                        *reinterpret_cast<uint4*>(sa + r * 128 + ((kc ^ (r & 7)) << 4)) = v;
+                    }
+                } else {
 #pragma unroll 4
                 for (int c = pt; c < BM * 8; c += kProducerThreads) {
                     const int r = c >> 3, kc = c & 7;
@@ -697,10 +747,11 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     *reinterpret_cast<uint4*>(sa + r * 128 + ((kc ^ (r & 7)) << 4)) =
                         gather8(g.A + gm * g.lda + gk, valid);
                 }
+                }
                 if (BCOL) {
                     // B column-major: 256 n-rows x 8 chunks of 8 k (K-major)
 #pragma unroll 4
-                    for (int c = pt; c < BN * 8; c += kProducerThreads) {
+                    for (int c = pt; c < x.ncols * 8; c += kProducerThreads) {
                         const int n = c >> 3, kc = c & 7;
                         const int64_t gn = n0 + n;
                         const int gk = k0 + kc * 8;
@@ -1316,6 +1367,48 @@ cudaError_t launch_r4_single_grouped(const GemmArgs* groups, int n, RunContext& 
     const GemmArgs& g0 = groups[0];
     return g0.b_col ? launch<true, false, false, 2>(g0, none, none, none, p, grid, ctx.device, stream)
                     : launch<false, false, false, 2>(g0, none, none, none, p, grid, ctx.device, stream);
+}
+
+cudaError_t launch_r4_conv2d(const GemmArgs& g, const ConvGeom& geom, RunContext& ctx, cudaStream_t stream,
+                             int* kernel_id)
+{
+    if (ctx.max_smem_optin < kSmemBytes || !g.b_col || g.M <= 0 || g.N <= 0 || g.K <= 0) return cudaErrorInvalidValue;
+    R4Params p;
+    fill_multi_params(p, g, ctx);
+    if (g.f16) {   // operand format fields of the instruction descriptor: 0 = fp16, 1 = bf16
+        p.idesc &= ~((1u << 7) | (1u << 10));
+        p.idesc_half &= ~((1u << 7) | (1u << 10));
+    }
+    p.tiles_m = (g.M + BM - 1) / BM;
+    p.tiles_n = (g.N + BN - 1) / BN;
+    p.nkb = (g.K + BK - 1) / BK;
+    p.kb_per_split = p.nkb;
+    p.conv = geom;
+    p.conv_fast = (geom.C % 8 == 0 && reinterpret_cast<uintptr_t>(g.A) % 16 == 0) ? 1 : 0;
+    const int celt = g.c_bf16 ? 2 : 4;
+    p.epi_tma = (ctx.encode_tiled && c_store_by_tma(g)) ? 1 : 0;
+    CUtensorMap none, mc;
+    memset(&none, 0, sizeof none);
+    memset(&mc, 0, sizeof mc);
+    if (p.epi_tma &&
+        !encode_map_2d(ctx, &mc, g.c_bf16 ? (g.f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16)
+                                          : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                       g.C, g.N, g.M, g.ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+        return cudaErrorInvalidValue;
+    const int64_t tiles = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
+    if (tiles > 0x3FFFFFFFll) return cudaErrorInvalidValue;
+    unsigned grid;
+    if (g.N <= BN / 2) {    // one 128-column half tile per row block: the MMA runs at N = 128
+        p.half_only = 1;
+        p.full_units = 0;
+        p.total_units = tiles;
+        grid = static_cast<unsigned>(tiles < ctx.sm_count ? tiles : ctx.sm_count);
+    } else {
+        grid = finish_multi_schedule(p, tiles, true, ctx);
+    }
+    p.kid = kIdConvTcgen05 + (p.epi_tma ? 0 : 2) + (p.conv_fast ? 0 : 1);
+    *kernel_id = p.kid;
+    return launch<true, true, false, 4>(g, none, none, mc, p, grid, ctx.device, stream);
 }
 
 bool r4_multi_dst_possible(const GemmArgs& g, const RunContext& ctx)
