@@ -566,6 +566,36 @@ def family_table(kb, gen, torch, device, peaks, flush):
             "extra_bytes_stored": 7 * n * (n // world) * 2, "launches_one_call": launches, "kernel_id": kid,
             "all_destinations_equal": ok}
         del A, Bs, Cs
+    # Conv2d of the paper's workload table (N=8, C=64, 56x56, F=128, 3x3, fp16; channels-last, padding 1, stride 1)
+    cc = gen.conv_benchmark_case(1)
+    x = torch.from_numpy(cc.x.view("int16")).to(device)
+    w = torch.from_numpy(cc.w.view("int16")).to(device)
+    y = torch.empty((cc.N, cc.P, cc.Q, cc.F), dtype=torch.float16, device=device)
+    with kb.Conv2d(device.index, y_f16=True) as conv:
+        row = {}
+        for v, name in ((0, "naive"), (4, "tcgen05")):
+            t = timed(lambda: conv.run(x, w, y, cc.N, cc.H, cc.W, cc.C, cc.F, cc.R, cc.S, cc.pad, cc.stride, v))
+            for _ in range(3):
+                conv.run(x, w, y, cc.N, cc.H, cc.W, cc.C, cc.F, cc.R, cc.S, cc.pad, cc.stride, v)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(50):
+                conv.run(x, w, y, cc.N, cc.H, cc.W, cc.C, cc.F, cc.R, cc.S, cc.pad, cc.stride, v)
+            e1.record()
+            e1.synchronize()
+            loop_ms = e0.elapsed_time(e1) / 50
+            row[name] = {"us_single_after_flush": t * 1e3, "us_back_to_back": loop_ms * 1e3,
+                         "tflops_back_to_back": cc.flops / (loop_ms * 1e-3) / 1e12, "kernel_id": conv.last_kernel_id()}
+        xt = x.view(torch.float16).permute(0, 3, 1, 2)          # NCHW views of channels-last storage
+        wt = w.view(torch.float16).permute(0, 3, 1, 2)
+        lib = timed(lambda: torch.nn.functional.conv2d(xt, wt, padding=cc.pad, stride=cc.stride))
+        ref = torch.nn.functional.conv2d(xt.float(), wt.float(), padding=cc.pad, stride=cc.stride).permute(0, 2, 3, 1)
+        conv.run(x, w, y, cc.N, cc.H, cc.W, cc.C, cc.F, cc.R, cc.S, cc.pad, cc.stride, 4)
+        row["sane_vs_torch_conv2d"] = bool(torch.allclose(y.float(), ref, rtol=2e-2, atol=2e-2))
+        row["context_torch_conv2d_us_single"] = lib * 1e3
+        row["algorithmic_bytes"] = int(x.numel() * 2 + w.numel() * 2 + y.numel() * 2)
+        out["conv2d_n8_c64_56x56_f128_3x3_f16"] = row
     out["note"] = ("median of 12 timed calls, each after a 256 MiB L2 flush; 'launch_per_problem' issues the "
                    "single-problem call once per batch / group on the same stream; the torch comparison is a "
                    "sanity check of the timed buffers, parity is established by the tests against the oracle")

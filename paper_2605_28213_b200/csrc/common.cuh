@@ -46,7 +46,8 @@ enum KernelId : int {
                               // + 64 unaligned operands repacked into the workspace first
     kIdMmaSync = 500,         // rung 3.5 (mma.sync); + 1 when the producer-thread path replaces TMA
     kIdConvNaive = 600,       // direct convolution, one thread per output
-    kIdConvTcgen05 = 700,     // implicit GEMM on the tcgen05 rung; + 2 direct epilogue, + 1 slow gather (C % 8 != 0 or unaligned x)
+    kIdConvTcgen05 = 700,     // implicit GEMM on the tcgen05 rung, patches by TMA; + 4 patches gathered by producer threads,
+                              // + 1 gathered element by element (C % 8 != 0 or unaligned x), + 2 direct epilogue
     kIdZeroFill = 900,
 };
 
@@ -210,6 +211,10 @@ struct alignas(128) DstEntry {
 };
 constexpr int kMaxDst = 16;
 constexpr int kMaxGroups = 256;         // groups per launch (the schedule's prefix sums live in shared memory)
+
+// 4-D tiled map of a channels-last image tensor (dims innermost first: C, W, H, N), box c_box x w_box x 1 x 1.
+bool encode_map_nhwc(const RunContext& ctx, CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t C,
+                     uint64_t W, uint64_t H, uint64_t N, uint32_t c_box, uint32_t w_box, CUtensorMapSwizzle swz);
 
 cudaError_t launch_r0_naive(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
 cudaError_t launch_r1_tiled(const GemmArgs& g, cudaStream_t stream, int* kernel_id);

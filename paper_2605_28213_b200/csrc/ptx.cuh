@@ -93,6 +93,16 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const void* tmap, in
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
         : "memory");
 }
+// 4-D tiled load (c0 innermost).  Coordinates other than the innermost may be negative or past the
+// tensor: the box is filled with zeros there (how a convolution's padding is read).
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const void* tmap, int c0, int c1, int c2, int c3, uint64_t* bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(c3),
+        "r"(smem_u32(bar))
+        : "memory");
+}
 // 3-D tiled store shared -> global (bulk group).  Coordinates must be >= 0.
 __device__ __forceinline__ void tma_store_3d(const void* tmap, int x, int y, int z, const void* smem_src)
 {

@@ -89,6 +89,8 @@ struct R4Params {
     ConvGeom conv;
     int conv_fast;          // 1: C % 8 == 0 and x 16-byte aligned - an 8-k chunk is one 16-byte load
     int half_only;          // every unit is the first 128-column half of its tile (problems with N <= 128)
+    int conv_b_tma;         // MODE 4: the weights come by TMA (warp 0), only the patches are gathered
+    int conv_b_rows;        // rows of the weight box (128 with half_only, else 256)
 };
 
 // One entry of the static schedule.
@@ -257,7 +259,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         const CUtensorMap *ma, *mb;
         uint32_t it;
         bool live;
-    } prod = {static_cast<int64_t>(blockIdx.x), 0, 0, 0, 0, 0, &map_a, &map_b, 0u, false};
+        int cw[16], ch[16], cn[16];     // MODE 4 on TMA: input origin (w, h, n) of each 8-pixel group of the tile
+    } prod = {static_cast<int64_t>(blockIdx.x), 0, 0, 0, 0, 0, &map_a, &map_b, 0u, false, {}, {}, {}};
     auto prod_enter_unit = [&]() {
         prod.live = prod.u < total_units;
         if (!prod.live) return;
@@ -270,6 +273,17 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             prod.z = x.z;
             prod.ma = x.ma;
             prod.mb = x.mb;
+        }
+        if (MODE == 4 && !GENERIC) {
+            // Q is a multiple of 8 here, so the 8 pixels of a group share (n, p) and are consecutive in q
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int m = x.m0 + 8 * j;
+                const int q = m % p.conv.Q, t = m / p.conv.Q;
+                prod.cw[j] = q - p.conv.pad_w;
+                prod.ch[j] = t % p.conv.P - p.conv.pad_h;
+                prod.cn[j] = t / p.conv.P;          // >= N past the last pixel: the box reads zeros
+            }
         }
     };
     auto load_box = [&](void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
@@ -294,6 +308,17 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
             const CUtensorMap* pa = (MODE == 2) ? prod.ma : &map_a;
             const CUtensorMap* pb = (MODE == 2) ? prod.mb : &map_b;
+            if (MODE == 4) {
+                // Conv2d: k-block = (filter tap, 64-channel group); the A stage is 16 boxes of
+                // 8 pixels x 64 channels read at the tap's offset - outside the image the TMA unit
+                // fills zeros, which is the padding
+                const int cpb = p.conv.C >> 6;
+                const int tap = prod.kb / cpb, cg = prod.kb - tap * cpb;
+                const int fr = tap / p.conv.S, fs = tap - fr * p.conv.S;
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    ptx::tma_load_4d(sa + j * 1024, &map_a, cg * 64, prod.cw[j] + fs, prod.ch[j] + fr, prod.cn[j], &full[s]);
+            } else
             load_box(sa, pa, prod.kb * BK, prod.m0, &full[s]);
             if (BCOL) {
                 load_box(sb, pb, prod.kb * BK, prod.n0, &full[s]);
@@ -312,7 +337,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
 
     if (warp == 0 && lane == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(&full[s], GENERIC ? kProducerThreads : 1);
+            ptx::mbar_init(&full[s], GENERIC ? kProducerThreads + ((MODE == 4 && p.conv_b_tma) ? 1 : 0) : 1);
             ptx::mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -364,6 +389,27 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             produce(0xFFFFFFFFu);
             // Drain: every load issued must have landed before shared memory is released.
             const uint32_t it = prod.it;
+            const uint32_t first = it > STAGES ? it - STAGES : 0;
+            for (uint32_t j = first; j < it; ++j) ptx::mbar_wait(&full[j % STAGES], (j / STAGES) & 1, abort_flag + 1);
+        }
+        if (GENERIC && MODE == 4 && lane == 0 && p.conv_b_tma) {
+            // Conv2d: the filter block of every k-block by TMA (the patches come from warps 6..9)
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+                const Unit x = decode_unit(u, p);
+                for (int kb = x.kb0; kb < x.kb1; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
+                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x450u | s);
+                        abort_flag[0] = 1;
+                        ok = false;
+                        break;
+                    }
+                    ptx::mbar_arrive_expect_tx(&full[s], static_cast<uint32_t>(p.conv_b_rows) * 128u);
+                    ptx::tma_load_2d(smem + s * kStageBytes + kABytes, &map_b, kb * BK, x.n0, &full[s]);
+                }
+            }
             const uint32_t first = it > STAGES ? it - STAGES : 0;
             for (uint32_t j = first; j < it; ++j) ptx::mbar_wait(&full[j % STAGES], (j / STAGES) & 1, abort_flag + 1);
         }
@@ -679,6 +725,82 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         const int pt = threadIdx.x - 6 * 32;                 // 0..127
         uint32_t it = 0;
         bool ok = true;
+        if (MODE == 4 && p.conv_fast) {
+            // Conv2d, 16-byte chunks (C % 8 == 0, aligned x).  Row m of the implicit GEMM is the output
+            // pixel (n, p, q), k the filter tap and channel (r, s, c); the element is
+            // x[n][p*stride_h + r - pad_h][q*stride_w + s - pad_w][c], zero outside the image.  A thread
+            // owns chunk kc of rows (pt >> 3) + 16 j: its chunk's tap is the same for all eight rows,
+            // whose pixel origins are decoded once per tile.  The eight loads of the NEXT k-block are
+            // issued before this k-block is stored, so a load's latency hides behind the ring.
+            const ConvGeom& cv = p.conv;
+            const int kc = pt & 7;
+            for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+                const Unit x = decode_unit(u, p);
+                int h0[8], w0[8], nn[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int gm = x.m0 + (pt >> 3) + 16 * j;
+                    const int q = gm % cv.Q, t = gm / cv.Q;
+                    nn[j] = gm < g.M ? t / cv.P : -1;
+                    h0[j] = (t % cv.P) * cv.stride_h - cv.pad_h;
+                    w0[j] = q * cv.stride_w - cv.pad_w;
+                }
+                auto fetch = [&](int kb, uint4 (&v)[8]) {
+                    const int gk = kb * BK + kc * 8;
+                    const int tap = gk / cv.C, ch = gk - tap * cv.C;
+                    const int fr = tap / cv.S, fs = tap - fr * cv.S;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int h = h0[j] + fr, w = w0[j] + fs;
+                        v[j] = make_uint4(0u, 0u, 0u, 0u);
+                        if (nn[j] >= 0 && gk < g.K && h >= 0 && h < cv.H && w >= 0 && w < cv.W)
+                            v[j] = __ldg(reinterpret_cast<const uint4*>(
+                                g.A + ((static_cast<int64_t>(nn[j]) * cv.H + h) * cv.W + w) * cv.C + ch));
+                    }
+                };
+                auto commit = [&](int kb, const uint4 (&v)[8]) -> bool {
+                    const int s = it % STAGES;
+                    if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
+                        if (pt == 0) report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x460u | s);
+                        abort_flag[0] = 1;
+                        return false;
+                    }
+                    uint8_t* sa = smem + s * kStageBytes;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int r = (pt >> 3) + 16 * j;
+                        *reinterpret_cast<uint4*>(sa + r * 128 + ((kc ^ (r & 7)) << 4)) = v[j];
+                    }
+                    if (!p.conv_b_tma) {
+                        // filters [F][K], K contiguous: 8-k chunks of rows n0 .. n0 + ncols
+                        uint8_t* sb = sa + kABytes;
+#pragma unroll 4
+                        for (int c = pt; c < x.ncols * 8; c += kProducerThreads) {
+                            const int n = c >> 3, kc2 = c & 7;
+                            const int64_t gn = x.n0 + n;
+                            const int gk = kb * BK + kc2 * 8;
+                            const int valid = (gn < g.N) ? min(8, max(0, g.K - gk)) : 0;
+                            *reinterpret_cast<uint4*>(sb + n * 128 + ((kc2 ^ (n & 7)) << 4)) =
+                                gather8(g.B + gn * g.ldb + gk, valid);
+                        }
+                    }
+                    ptx::fence_proxy_async_smem();
+                    ptx::mbar_arrive(&full[s]);
+                    ++it;
+                    return true;
+                };
+                uint4 va[8], vb[8];
+                fetch(x.kb0, va);
+                for (int kb = x.kb0; kb < x.kb1 && ok; kb += 2) {
+                    if (kb + 1 < x.kb1) fetch(kb + 1, vb);
+                    ok = commit(kb, va);
+                    if (ok && kb + 1 < x.kb1) {
+                        if (kb + 2 < x.kb1) fetch(kb + 2, va);
+                        ok = commit(kb + 1, vb);
+                    }
+                }
+            }
+        } else
         for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
             const Unit x = decode_unit(u, p);
             const int kb0 = x.kb0, kb1 = x.kb1;
@@ -696,45 +818,37 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 const int k0 = kb * BK;
                 // A: 128 rows x 8 chunks of 8 k (K-major, 128-byte swizzle)
                 if (MODE == 4) {
-                    // implicit GEMM: row m is the output pixel (n, p, q), k the filter tap and channel
-                    // (r, s, c); the element is x[n][p*stride_h + r - pad_h][q*stride_w + s - pad_w][c]
-                    // or zero outside the image
+                    // (the 16-byte-chunk form has a loop of its own above)
+                    // channel counts that are not multiples of 8 (a chunk may straddle two taps) or an
+                    // unaligned x: element by element
                     const ConvGeom& cv = p.conv;
                     for (int c = pt; c < BM * 8; c += kProducerThreads) {
                         const int r = c >> 3, kc = c & 7;
                         const int gm = m0 + r;
                         const int gk = k0 + kc * 8;
-                        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                        uint16_t e8[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) e8[e] = 0;
                         if (gm < g.M && gk < g.K) {
                             const int q = gm % cv.Q, t = gm / cv.Q;
                             const int pp = t % cv.P, n = t / cv.P;
-                            if (p.conv_fast) {
-                                const int tap = gk / cv.C, ch = gk - tap * cv.C;
-                                const int fr = tap / cv.S, fs = tap - fr * cv.S;
-                                const int h = pp * cv.stride_h + fr - cv.pad_h, w = q * cv.stride_w + fs - cv.pad_w;
-                                if (h >= 0 && h < cv.H && w >= 0 && w < cv.W)
-                                    v = __ldg(reinterpret_cast<const uint4*>(
-                                        g.A + ((static_cast<int64_t>(n) * cv.H + h) * cv.W + w) * cv.C + ch));
-                            } else {
-                                uint16_t e8[8];
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) {
-                                    const int k = gk + e;
-                                    e8[e] = 0;
-                                    if (k < g.K) {
-                                        const int tap = k / cv.C, ch = k - tap * cv.C;
-                                        const int fr = tap / cv.S, fs = tap - fr * cv.S;
-                                        const int h = pp * cv.stride_h + fr - cv.pad_h, w = q * cv.stride_w + fs - cv.pad_w;
-                                        if (h >= 0 && h < cv.H && w >= 0 && w < cv.W)
-                                            e8[e] = __ldg(g.A + ((static_cast<int64_t>(n) * cv.H + h) * cv.W + w) * cv.C + ch);
-                                    }
+                            for (int e = 0; e < 8; ++e) {
+                                const int k = gk + e;
+                                if (k < g.K) {
+                                    const int tap = k / cv.C, ch = k - tap * cv.C;
+                                    const int fr = tap / cv.S, fs = tap - fr * cv.S;
+                                    const int h = pp * cv.stride_h + fr - cv.pad_h, w = q * cv.stride_w + fs - cv.pad_w;
+                                    if (h >= 0 && h < cv.H && w >= 0 && w < cv.W)
+                                        e8[e] = __ldg(g.A + ((static_cast<int64_t>(n) * cv.H + h) * cv.W + w) * cv.C + ch);
                                 }
-                                v.x = e8[0] | (uint32_t(e8[1]) << 16);
-                                v.y = e8[2] | (uint32_t(e8[3]) << 16);
-                                v.z = e8[4] | (uint32_t(e8[5]) << 16);
-                                v.w = e8[6] | (uint32_t(e8[7]) << 16);
                             }
                         }
+                        uint4 v;
+                        v.x = e8[0] | (uint32_t(e8[1]) << 16);
+                        v.y = e8[2] | (uint32_t(e8[3]) << 16);
+                        v.z = e8[4] | (uint32_t(e8[5]) << 16);
+                        v.w = e8[6] | (uint32_t(e8[7]) << 16);
                         *reinterpret_cast<uint4*>(sa + r * 128 + ((kc ^ (r & 7)) << 4)) = v;
                     }
                 } else {
@@ -1385,6 +1499,15 @@ cudaError_t launch_r4_conv2d(const GemmArgs& g, const ConvGeom& geom, RunContext
     p.kb_per_split = p.nkb;
     p.conv = geom;
     p.conv_fast = (geom.C % 8 == 0 && reinterpret_cast<uintptr_t>(g.A) % 16 == 0) ? 1 : 0;
+    p.half_only = g.N <= BN / 2 ? 1 : 0;
+    p.conv_b_rows = p.half_only ? BN / 2 : BN;
+    CUtensorMap mb;
+    memset(&mb, 0, sizeof mb);
+    p.conv_b_tma = (p.conv_fast && ctx.encode_tiled && tma_ok(g.B, g.ldb, 2) &&
+                    encode_map_2d(ctx, &mb, g.f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B,
+                                  g.K, g.N, g.ldb * 2, BK, static_cast<uint32_t>(p.conv_b_rows), CU_TENSOR_MAP_SWIZZLE_128B))
+                       ? 1
+                       : 0;
     const int celt = g.c_bf16 ? 2 : 4;
     p.epi_tma = (ctx.encode_tiled && c_store_by_tma(g)) ? 1 : 0;
     CUtensorMap none, mc;
@@ -1398,17 +1521,28 @@ cudaError_t launch_r4_conv2d(const GemmArgs& g, const ConvGeom& geom, RunContext
     const int64_t tiles = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
     if (tiles > 0x3FFFFFFFll) return cudaErrorInvalidValue;
     unsigned grid;
-    if (g.N <= BN / 2) {    // one 128-column half tile per row block: the MMA runs at N = 128
-        p.half_only = 1;
+    if (p.half_only) {      // one 128-column half tile per row block: the MMA runs at N = 128
         p.full_units = 0;
         p.total_units = tiles;
         grid = static_cast<unsigned>(tiles < ctx.sm_count ? tiles : ctx.sm_count);
     } else {
         grid = finish_multi_schedule(p, tiles, true, ctx);
     }
-    p.kid = kIdConvTcgen05 + (p.epi_tma ? 0 : 2) + (p.conv_fast ? 0 : 1);
+    // Patches by TMA: 64-channel groups (a k-block is one tap of one group), unit stride, and an output
+    // width that is a multiple of 8, so that the 8 pixels of a box never straddle an output row.
+    CUtensorMap mx;
+    memset(&mx, 0, sizeof mx);
+    const bool patch_tma = p.conv_b_tma && geom.C % 64 == 0 && geom.Q % 8 == 0 && geom.stride_h == 1 && geom.stride_w == 1 &&
+                           encode_map_nhwc(ctx, &mx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, g.A, geom.C, geom.W, geom.H,
+                                           static_cast<uint64_t>(g.M / (static_cast<int64_t>(geom.P) * geom.Q)), 64, 8,
+                                           CU_TENSOR_MAP_SWIZZLE_128B);
+    p.kid = kIdConvTcgen05 + (patch_tma ? 0 : 4) + (p.epi_tma ? 0 : 2) + (p.conv_fast ? 0 : 1);
     *kernel_id = p.kid;
-    return launch<true, true, false, 4>(g, none, none, mc, p, grid, ctx.device, stream);
+    if (patch_tma) {
+        p.stage_tx = kABytes + static_cast<uint32_t>(p.conv_b_rows) * 128u;
+        return launch<true, false, false, 4>(g, mx, mb, mc, p, grid, ctx.device, stream);
+    }
+    return launch<true, true, false, 4>(g, none, mb, mc, p, grid, ctx.device, stream);
 }
 
 bool r4_multi_dst_possible(const GemmArgs& g, const RunContext& ctx)
