@@ -39,10 +39,10 @@ WORKLOADS = {
 WORKLOAD = WORKLOADS["c4"]
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one tcgen05-rung launch at 8192^3
-# (ncu capture summarised in profiles/r4_tcgen05_c4_8192.md): 0.961 GB read + 0.132 GB written.
-R4_C4_DRAM_TRAFFIC_BYTES = 1.093e9
-# the same for the skinny shape (profiles/r4_tcgen05_c5_skinny.md): 134.6 MB read + 4.1 MB written.
-R4_C5_DRAM_TRAFFIC_BYTES = 1.387e8
+# (ncu capture summarised in profiles/r4_tcgen05_c4_8192.md): 0.882 GB read + 0.130 GB written.
+R4_C4_DRAM_TRAFFIC_BYTES = 1.012e9
+# the same for the skinny shape (profiles/r4_tcgen05_c5_skinny.md): 134.6 MB read + 3.9 MB written.
+R4_C5_DRAM_TRAFFIC_BYTES = 1.385e8
 VARIANT_NAMES = ["naive", "tiled", "vectorized", "pipelined", "tcgen05", "mma_sync"]
 LINEAGE_ORDER = [0, 1, 2, 3, 5, 4]     # rung 3.5 (mma.sync, variant id 5) sits between rungs 3 and 4
 
