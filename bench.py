@@ -439,6 +439,40 @@ def lineage_table(prob_c4, kb, gen, torch, device, peaks):
                                   "frac_hbm": gbs / peaks["hbm_gbs"], "tflops": c5.flops / (med * 1e-3) / 1e12,
                                   "kernel_id": p5.gemm.last_kernel_id()}
     out["c5_16x8192x8192"] = rows
+    # Context only (not a target, not a code path of this library): the vendor GEMM on the same buffers, timed
+    # the same way as the rows above.
+    ctx_rows = {}
+    bf = torch.bfloat16
+    A5, C5 = p5.A.view(bf), torch.empty((c5.M, c5.N), dtype=torch.float32, device=device)
+    best = []
+    for _ in range(9):
+        for i in range(4):
+            torch.matmul(A5, rot[i].view(bf)).float()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(40):
+            torch.matmul(A5, rot[i % 4].view(bf))
+        e1.record()
+        e1.synchronize()
+        best.append(e0.elapsed_time(e1) / 40)
+    med = statistics.median(best)
+    ctx_rows["c5_16x8192x8192"] = {"us_median": med * 1e3, "gbs": c5.algorithmic_bytes / (med * 1e-3) / 1e9,
+                                   "note": "bf16 output (the library's default), back-to-back over 4 weight buffers"}
+    A4, B4 = prob_c4.A.view(bf), prob_c4.B.view(bf)
+    C4 = torch.empty((c4.M, c4.N), dtype=bf, device=device)
+    times = []
+    for i in range(13):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        torch.matmul(A4, B4, out=C4)
+        e1.record()
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1))
+    med = statistics.median(times[3:])
+    ctx_rows["c4_8192^3"] = {"ms_median": med, "tflops": c4.flops / (med * 1e-3) / 1e12}
+    out["context_vendor_gemm"] = ctx_rows
+    del A5, C5, C4
     # c1 and c2 are launch- and occupancy-bound (report only): back-to-back launches, operands L2-resident.
     for name in ("c1", "c2"):
         cs = gen.make_config(name, 1)
