@@ -115,6 +115,11 @@ constexpr int kGroupM = 8;
 __host__ __device__ __forceinline__ void raster_tile(int64_t t, int tiles_m, int tiles_n, int& tm, int& tn,
                                                      int group_m = kGroupM)
 {
+    if (tiles_m == 1) {   // one tile-row (the skinny orientation): no arithmetic on the critical path of short kernels
+        tm = 0;
+        tn = static_cast<int>(t);
+        return;
+    }
     const int64_t per_group = static_cast<int64_t>(group_m) * tiles_n;
     if (t < 0x7FFFFFFFll && per_group < 0x7FFFFFFFll) {
         // the common case in 32-bit arithmetic: a 64-bit division costs hundreds of cycles on the

@@ -72,6 +72,7 @@ struct R4Params {
     int n_mma;              // skinny mode: M rounded up to 16 = the MMA's N
     uint32_t stage_tx;      // bytes one stage's TMA loads deliver (A box + B boxes)
     int cluster;            // 1: the splits of a tile are one cluster and reduce through DSMEM
+    int splits_log2;        // cluster mode: splits is 2, 4 or 8
     int group_m;            // tile raster: tile-rows per group
     int64_t full_units;     // units [0, full_units) are whole tiles; later ones are 128-column half tiles
     int64_t total_units;
@@ -149,7 +150,10 @@ __device__ __forceinline__ Unit decode_unit(int64_t u, const R4Params& p)
     Unit x;
     int half = 0;
     x.ncols = BN;
-    if (p.splits > 1) {
+    if (p.cluster) {              // splits is a power of two: no division on the critical path of short kernels
+        x.tile = u >> p.splits_log2;
+        x.split = static_cast<int>(u & (p.splits - 1));
+    } else if (p.splits > 1) {
         if (u < 0x7FFFFFFFll) {   // 32-bit division: this sits on the critical path of short kernels
             const uint32_t u32 = static_cast<uint32_t>(u), sp = static_cast<uint32_t>(p.splits);
             x.tile = u32 / sp;
@@ -381,6 +385,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     ptx::grid_dependency_wait();
     ptx::grid_launch_dependents();
     if (SWAP && p.cluster) ptx::cluster_wait_acquire();
+    // Cluster mode: what the final reduce needs, computed now, off the kernel's tail.
+    const int fin_rank = (SWAP && p.cluster) ? static_cast<int>(blockIdx.x & static_cast<unsigned>(p.splits - 1)) : 0;
+    const int fin_n0 = (SWAP && p.cluster) ? static_cast<int>(blockIdx.x >> p.splits_log2) * BN : 0;
+    const float* fin_slots = reinterpret_cast<const float*>(epi_smem) + lane;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -499,16 +507,20 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     for (int mc = 0; mc < p.n_mma; mc += 16) {
                         uint32_t v[16];
                         ptx::tmem_ld_32x32b_x16(tmem_base + buf * BN + h * 128 + mc + (static_cast<uint32_t>(q * 32) << 16), v);
-                        ptx::tmem_ld_wait();
+                        uint32_t remote = 0;
                         if (p.cluster) {
                             // block (h, q) of the tile belongs to CTA (block % splits); this CTA's
-                            // partial goes to slot [split][block / splits][m][lane] of the owner.
+                            // partial goes to slot [split][block / splits][m][lane] of the owner
+                            // (address arithmetic while the TMEM load is in flight)
                             const int bi = h * 4 + q;
-                            const uint32_t owner = static_cast<uint32_t>(bi % p.splits);
-                            const int nblk = 8 / p.splits;
+                            const uint32_t owner = static_cast<uint32_t>(bi & (p.splits - 1));
+                            const int nblk = 8 >> p.splits_log2;
                             float* slot = reinterpret_cast<float*>(epi_smem) +
-                                          ((split * nblk + bi / p.splits) * p.n_mma + mc) * 32 + lane;
-                            const uint32_t remote = ptx::map_to_cta(ptx::smem_u32(slot), owner);
+                                          ((split * nblk + (bi >> p.splits_log2)) * p.n_mma + mc) * 32 + lane;
+                            remote = ptx::map_to_cta(ptx::smem_u32(slot), owner);
+                        }
+                        ptx::tmem_ld_wait();
+                        if (p.cluster) {
 #pragma unroll
                             for (int j = 0; j < 16; ++j) ptx::st_cluster_f32(remote + j * 128, __uint_as_float(v[j]));
                         } else if (n < g.N) {
@@ -898,28 +910,32 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         ptx::cluster_arrive_release();
         ptx::cluster_wait_acquire();
         if (warp >= 2 && warp < 6 && !abort_flag[0]) {
-            const int rank = static_cast<int>(blockIdx.x % p.splits);
-            const int n0 = decode_unit(blockIdx.x, p).n0;
-            const int nblk = 8 / p.splits;
-            const float* slots = reinterpret_cast<const float*>(epi_smem);
-            // each warp takes every fourth row m of every local block, four rows per step so
-            // that their shared-memory loads are in flight together; lanes run along n
-            for (int bl = 0; bl < nblk; ++bl) {
-                const int bi = bl * p.splits + rank;
-                const int n = n0 + (bi >> 2) * 128 + (bi & 3) * 32 + lane;
-                if (n >= g.N) continue;
-                for (int mb = warp - 2; mb < g.M; mb += 16) {
-                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                    for (int src = 0; src < p.splits; ++src) {
-                        const float* sl = slots + ((src * nblk + bl) * p.n_mma + mb) * 32 + lane;
+            // This CTA owns blocks bi = bl * splits + rank of the tile; slot (src * nblk + bl) holds
+            // CTA src's partial of local block bl.  A warp takes rows mb, mb+4, mb+8, mb+12; all of a
+            // block's loads are issued before the adds (in rank order: deterministic), lanes run along n.
+            const int nblk = 8 >> p.splits_log2;
+            for (int mb = warp - 2; mb < g.M; mb += 16) {
+                for (int bl = 0; bl < nblk; ++bl) {
+                    const int bi = (bl << p.splits_log2) + fin_rank;
+                    const int n = fin_n0 + (bi >> 2) * 128 + (bi & 3) * 32 + lane;
+                    if (n >= g.N) continue;
+                    const float* sl = fin_slots + (bl * p.n_mma + mb) * 32;
+                    const int src_stride = nblk * p.n_mma * 32;
+                    float v[8][4];
+#pragma unroll
+                    for (int src = 0; src < 8; ++src)
 #pragma unroll
                         for (int r = 0; r < 4; ++r)
-                            if (mb + 4 * r < g.M) acc[r] += sl[4 * r * 32];
-                    }
+                            v[src][r] = (src < p.splits && mb + 4 * r < g.M) ? sl[src * src_stride + 4 * r * 32] : 0.f;
+                    const float bn = bias_at(g, n);
 #pragma unroll
-                    for (int r = 0; r < 4; ++r)
-                        if (mb + 4 * r < g.M)
-                            store_c(g.C, g.c_bf16, static_cast<int64_t>(mb + 4 * r) * g.ldc + n, acc[r] + bias_at(g, n));
+                    for (int r = 0; r < 4; ++r) {
+                        float acc = 0.f;
+#pragma unroll
+                        for (int src = 0; src < 8; ++src)
+                            if (src < p.splits) acc += v[src][r];
+                        if (mb + 4 * r < g.M) store_c(g.C, g.c_bf16, static_cast<int64_t>(mb + 4 * r) * g.ldc + n, acc + bn);
+                    }
                 }
             }
         }
@@ -1190,6 +1206,7 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     if (!resolve_split(g.M, tiles, p.nkb, p.ldw, ctx, pinned, &plan)) return cudaErrorInvalidValue;
     p.splits = plan.splits;
     p.cluster = plan.cluster ? 1 : 0;
+    p.splits_log2 = plan.splits >= 8 ? 3 : plan.splits >= 4 ? 2 : plan.splits >= 2 ? 1 : 0;
     p.kb_per_split = (p.nkb + p.splits - 1) / p.splits;
     p.ws = static_cast<float*>(ctx.workspace);
     p.counters = ctx.tile_counters;
