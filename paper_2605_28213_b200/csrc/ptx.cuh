@@ -165,6 +165,11 @@ __device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v)
 {
     asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
 }
+__device__ __forceinline__ void st_cluster_v4_f32(uint32_t cluster_addr, float a, float b, float c, float d)
+{
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "f"(a), "f"(b), "f"(c), "f"(d)
+                 : "memory");
+}
 // Cluster-wide barrier, split in two; every thread of every CTA of the cluster
 // executes both.  (A hardware barrier: it completes because every loop that
 // precedes it in these kernels is bounded.)

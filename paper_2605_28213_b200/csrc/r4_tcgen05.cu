@@ -388,7 +388,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     // Cluster mode: what the final reduce needs, computed now, off the kernel's tail.
     const int fin_rank = (SWAP && p.cluster) ? static_cast<int>(blockIdx.x & static_cast<unsigned>(p.splits - 1)) : 0;
     const int fin_n0 = (SWAP && p.cluster) ? static_cast<int>(blockIdx.x >> p.splits_log2) * BN : 0;
-    const float* fin_slots = reinterpret_cast<const float*>(epi_smem) + lane;
+    const float* fin_slots = reinterpret_cast<const float*>(epi_smem) + lane * 4;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -510,19 +510,22 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         uint32_t remote = 0;
                         if (p.cluster) {
                             // block (h, q) of the tile belongs to CTA (block % splits); this CTA's
-                            // partial goes to slot [split][block / splits][m][lane] of the owner
+                            // partial goes to slot [split][block / splits] of the owner, laid out
+                            // [m / 4][lane][m % 4] so that four rows travel as one 16-byte store
                             // (address arithmetic while the TMEM load is in flight)
                             const int bi = h * 4 + q;
                             const uint32_t owner = static_cast<uint32_t>(bi & (p.splits - 1));
                             const int nblk = 8 >> p.splits_log2;
                             float* slot = reinterpret_cast<float*>(epi_smem) +
-                                          ((split * nblk + (bi >> p.splits_log2)) * p.n_mma + mc) * 32 + lane;
+                                          ((split * nblk + (bi >> p.splits_log2)) * p.n_mma + mc) * 32 + lane * 4;
                             remote = ptx::map_to_cta(ptx::smem_u32(slot), owner);
                         }
                         ptx::tmem_ld_wait();
                         if (p.cluster) {
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) ptx::st_cluster_f32(remote + j * 128, __uint_as_float(v[j]));
+                            for (int j = 0; j < 16; j += 4)
+                                ptx::st_cluster_v4_f32(remote + j * 128, __uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                       __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
                         } else if (n < g.N) {
                             const float bn = partial ? 0.f : bias_at(g, n);
 #pragma unroll
@@ -911,31 +914,34 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         ptx::cluster_wait_acquire();
         if (warp >= 2 && warp < 6 && !abort_flag[0]) {
             // This CTA owns blocks bi = bl * splits + rank of the tile; slot (src * nblk + bl) holds
-            // CTA src's partial of local block bl.  A warp takes rows mb, mb+4, mb+8, mb+12; all of a
-            // block's loads are issued before the adds (in rank order: deterministic), lanes run along n.
+            // CTA src's partial of local block bl as [m / 4][lane][m % 4].  A warp takes four
+            // consecutive rows (one 16-byte load per source); all of a block's loads are issued
+            // before the adds (in rank order: deterministic), lanes run along n.
             const int nblk = 8 >> p.splits_log2;
-            for (int mb = warp - 2; mb < g.M; mb += 16) {
+            for (int m4 = (warp - 2) * 4; m4 < g.M; m4 += 16) {
                 for (int bl = 0; bl < nblk; ++bl) {
                     const int bi = (bl << p.splits_log2) + fin_rank;
                     const int n = fin_n0 + (bi >> 2) * 128 + (bi & 3) * 32 + lane;
                     if (n >= g.N) continue;
-                    const float* sl = fin_slots + (bl * p.n_mma + mb) * 32;
-                    const int src_stride = nblk * p.n_mma * 32;
-                    float v[8][4];
+                    const float4* sl = reinterpret_cast<const float4*>(fin_slots + (bl * p.n_mma + m4) * 32);
+                    const int src_stride = nblk * p.n_mma * 8;      // in float4
+                    float4 v[8];
 #pragma unroll
                     for (int src = 0; src < 8; ++src)
-#pragma unroll
-                        for (int r = 0; r < 4; ++r)
-                            v[src][r] = (src < p.splits && mb + 4 * r < g.M) ? sl[src * src_stride + 4 * r * 32] : 0.f;
+                        v[src] = (src < p.splits) ? sl[src * src_stride] : make_float4(0.f, 0.f, 0.f, 0.f);
                     const float bn = bias_at(g, n);
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        float acc = 0.f;
+                    for (int src = 0; src < 8; ++src)
+                        if (src < p.splits) {
+                            acc[0] += v[src].x;
+                            acc[1] += v[src].y;
+                            acc[2] += v[src].z;
+                            acc[3] += v[src].w;
+                        }
 #pragma unroll
-                        for (int src = 0; src < 8; ++src)
-                            if (src < p.splits) acc += v[src][r];
-                        if (mb + 4 * r < g.M) store_c(g.C, g.c_bf16, static_cast<int64_t>(mb + 4 * r) * g.ldc + n, acc + bn);
-                    }
+                    for (int r = 0; r < 4; ++r)
+                        if (m4 + r < g.M) store_c(g.C, g.c_bf16, static_cast<int64_t>(m4 + r) * g.ldc + n, acc[r] + bn);
                 }
             }
         }
