@@ -73,6 +73,17 @@ typedef enum {
                                 sits between rungs 3 and 4 in speed and completes the table's vocabulary       */
 } klineage_variant_t;
 
+/*
+ * KLINEAGE_FLAG_STATIC_B - a promise about the caller's B operands ("the weights are static"): no GPU work
+ * that is still in flight when a klineage_gemm_run* call is enqueued writes B.  The tcgen05 rung then
+ * starts streaming B for a short (single-wave) launch before it waits for the previous kernel in the
+ * stream - launches go out with programmatic stream serialization, so the kernel may start while its
+ * predecessor drains - and waits only before it reads A and before it writes C.  For back-to-back
+ * weight-streaming calls (the decode shape) this hides the kernel boundary.  Without the flag every
+ * global access waits for the previous kernel.  The paper has no counterpart; results are identical.
+ */
+#define KLINEAGE_FLAG_STATIC_B 1u
+
 /* Create-time configuration (host memory, read during create only). */
 typedef struct {
     int device;             /* CUDA device ordinal the handle is bound to                              */
@@ -80,7 +91,7 @@ typedef struct {
     int c_dtype;            /* klineage_ctype_t                                                        */
     size_t workspace_bytes; /* device scratch: split-K partial sums and aligned copies of unaligned operands
                                (rung 4); 0 selects the default (64 MiB)                                */
-    unsigned flags;         /* reserved, must be 0                                                     */
+    unsigned flags;         /* 0, or KLINEAGE_FLAG_STATIC_B                                            */
 } klineage_gemm_config_t;
 
 /*
@@ -89,7 +100,7 @@ typedef struct {
  * properties of the handle so that klineage_gemm_run keeps the BLAS-like
  * argument list).  Allocates the device workspace and status block (this is the
  * only allocating call besides destroy).  out and cfg are host pointers.
- * Errors: INVALID_ARG (null, bad enum, flags != 0, no such device), ALLOC.
+ * Errors: INVALID_ARG (null, bad enum, unknown flag bits, no such device), ALLOC.
  */
 klineage_status_t klineage_gemm_create(klineage_gemm_t* out, const klineage_gemm_config_t* cfg);
 

@@ -25,6 +25,7 @@ KLINEAGE_ERR_SCRATCH_LIMIT = 8
 
 KLINEAGE_B_ROW_MAJOR, KLINEAGE_B_COL_MAJOR = 0, 1
 KLINEAGE_C_F32, KLINEAGE_C_BF16, KLINEAGE_C_F16 = 0, 1, 2
+KLINEAGE_FLAG_STATIC_B = 1
 KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELINED, KLINEAGE_TCGEN05, KLINEAGE_MMA_SYNC = range(6)
 # the five-step ladder, then the intermediate legacy tensor-core rung ("3.5")
 VARIANTS = (KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELINED, KLINEAGE_TCGEN05,
@@ -280,13 +281,14 @@ class Gemm:
     """
 
     def __init__(self, device: int = 0, b_col_major: bool = False, c_bf16: bool = False,
-                 workspace_bytes: int = 0):
+                 workspace_bytes: int = 0, static_b: bool = False):
         self.device = int(device)
         self.b_col_major = bool(b_col_major)
         self.c_bf16 = bool(c_bf16)
         self._h: Optional[int] = klineage_gemm_create(
             self.device, KLINEAGE_B_COL_MAJOR if b_col_major else KLINEAGE_B_ROW_MAJOR,
-            KLINEAGE_C_BF16 if c_bf16 else KLINEAGE_C_F32, workspace_bytes)
+            KLINEAGE_C_BF16 if c_bf16 else KLINEAGE_C_F32, workspace_bytes,
+            KLINEAGE_FLAG_STATIC_B if static_b else 0)
 
     @staticmethod
     def _ptr(x):

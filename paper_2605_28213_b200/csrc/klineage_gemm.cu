@@ -170,7 +170,7 @@ klineage_status_t klineage_gemm_create(klineage_gemm_t* out, const klineage_gemm
     if (cfg->b_layout != KLINEAGE_B_ROW_MAJOR && cfg->b_layout != KLINEAGE_B_COL_MAJOR) return KLINEAGE_ERR_INVALID_ARG;
     if (cfg->c_dtype != KLINEAGE_C_F32 && cfg->c_dtype != KLINEAGE_C_BF16 && cfg->c_dtype != KLINEAGE_C_F16)
         return KLINEAGE_ERR_INVALID_ARG;
-    if (cfg->flags != 0) return KLINEAGE_ERR_INVALID_ARG;
+    if (cfg->flags & ~KLINEAGE_FLAG_STATIC_B) return KLINEAGE_ERR_INVALID_ARG;
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev) {
         cudaGetLastError();
@@ -185,6 +185,7 @@ klineage_status_t klineage_gemm_create(klineage_gemm_t* out, const klineage_gemm
     h->c_dtype = cfg->c_dtype;
     RunContext& c = h->ctx;
     c.device = cfg->device;
+    c.flags = cfg->flags;
     cudaDeviceGetAttribute(&c.sm_count, cudaDevAttrMultiProcessorCount, c.device);
     cudaDeviceGetAttribute(&c.cc_major, cudaDevAttrComputeCapabilityMajor, c.device);
     cudaDeviceGetAttribute(&c.cc_minor, cudaDevAttrComputeCapabilityMinor, c.device);

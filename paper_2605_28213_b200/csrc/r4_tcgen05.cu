@@ -73,6 +73,7 @@ struct R4Params {
     uint32_t stage_tx;      // bytes one stage's TMA loads deliver (A box + B boxes)
     int cluster;            // 1: the splits of a tile are one cluster and reduce through DSMEM
     int splits_log2;        // cluster mode: splits is 2, 4 or 8
+    int static_b;           // the caller promised static B: the first ring fill's B boxes go out before the dependency wait
     int group_m;            // tile raster: tile-rows per group
     int64_t full_units;     // units [0, full_units) are whole tiles; later ones are 128-column half tiles
     int64_t total_units;
@@ -360,11 +361,38 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         // allocation in warp 1) may overlap the tail of the previous kernel in the stream;
         // nothing below the wait touches global memory before that kernel has completed.
         if (!GENERIC && MODE != 2) prod_enter_unit();           // schedule arithmetic only
-        ptx::grid_dependency_wait();
-        if (!GENERIC && MODE != 2) {
-            // The first ring fill needs nothing from the other warps: start it before the
-            // set-up barrier so that TMEM allocation hides behind the first loads' latency.
-            produce(STAGES);
+        if (!GENERIC && MODE == 0 && p.static_b && prod.live && prod.kb1 - prod.kb >= STAGES) {
+            // Static B: the B boxes of the first ring fill do not depend on the previous kernel in
+            // the stream and go out at once; only A waits (C is written much later, after the wait
+            // that every thread passes below).  The fresh "empty" barriers need no wait.
+            for (int s = 0; s < STAGES; ++s) {
+                uint8_t* sb = smem + s * kStageBytes + kABytes;
+                const int kb = prod.kb + s;
+                ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
+                if (BCOL) {
+                    ptx::tma_load_2d(sb, &map_b, kb * BK, prod.n0, &full[s]);
+                } else {
+#pragma unroll
+                    for (int cb = 0; cb < BN / 64; ++cb)
+                        ptx::tma_load_2d(sb + cb * (64 * BK * 2), &map_b, prod.n0 + cb * 64, kb * BK, &full[s]);
+                }
+            }
+            ptx::grid_dependency_wait();
+            for (int s = 0; s < STAGES; ++s)
+                ptx::tma_load_2d(smem + s * kStageBytes, &map_a, (prod.kb + s) * BK, prod.m0, &full[s]);
+            prod.it = STAGES;
+            prod.kb += STAGES;
+            if (prod.kb == prod.kb1) {
+                prod.u += gridDim.x;
+                prod_enter_unit();
+            }
+        } else {
+            ptx::grid_dependency_wait();
+            if (!GENERIC && MODE != 2) {
+                // The first ring fill needs nothing from the other warps: start it before the
+                // set-up barrier so that TMEM allocation hides behind the first loads' latency.
+                produce(STAGES);
+            }
         }
         if (blockIdx.x == 0) g.status[1] = p.kid;
     }
@@ -1212,6 +1240,7 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     if (!resolve_split(g.M, tiles, p.nkb, p.ldw, ctx, pinned, &plan)) return cudaErrorInvalidValue;
     p.splits = plan.splits;
     p.cluster = plan.cluster ? 1 : 0;
+    p.static_b = (ctx.flags & 1u) ? 1 : 0;
     p.splits_log2 = plan.splits >= 8 ? 3 : plan.splits >= 4 ? 2 : plan.splits >= 2 ? 1 : 0;
     p.kb_per_split = (p.nkb + p.splits - 1) / p.splits;
     p.ws = static_cast<float*>(ctx.workspace);
