@@ -287,8 +287,9 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups,
  * used); fp32 accumulation.  Pointers need element alignment only; 16-byte aligned x
  * with C % 8 == 0 selects 16-byte patch loads.  variant: KLINEAGE_NAIVE (direct
  * convolution, one thread per output) or KLINEAGE_TCGEN05 (rows = output pixels,
- * columns = filters, k = (r, s, c); producer warps gather the patches straight into
- * the swizzled shared-memory operand layout - no im2col buffer exists - and
+ * columns = filters, k = (r, s, c); the patches reach the swizzled shared-memory operand
+ * layout as 4-D TMA boxes whose out-of-image part is zero-filled (C % 64 == 0, unit
+ * stride) or are gathered by producer warps - no im2col buffer exists - and
  * tcgen05.mma.kind::f16 multiplies fp16 operands into TMEM).  No output pixel
  * (N*P*Q == 0) or F == 0: nothing is launched; C == 0: y is zero-filled.
  * Errors: INVALID_ARG (sizes, R or S outside 1..64, padding or stride outside

@@ -217,9 +217,11 @@ struct alignas(128) DstEntry {
 constexpr int kMaxDst = 16;
 constexpr int kMaxGroups = 256;         // groups per launch (the schedule's prefix sums live in shared memory)
 
-// 4-D tiled map of a channels-last image tensor (dims innermost first: C, W, H, N), box c_box x w_box x 1 x 1.
+// 4-D tiled map of a channels-last image tensor (dims innermost first: C, W, H, N), box c_box x w_box x h_box x 1,
+// elements of `elt` bytes.
 bool encode_map_nhwc(const RunContext& ctx, CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t C,
-                     uint64_t W, uint64_t H, uint64_t N, uint32_t c_box, uint32_t w_box, CUtensorMapSwizzle swz);
+                     uint64_t W, uint64_t H, uint64_t N, uint32_t c_box, uint32_t w_box, uint32_t h_box, int elt,
+                     CUtensorMapSwizzle swz);
 
 cudaError_t launch_r0_naive(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
 cudaError_t launch_r1_tiled(const GemmArgs& g, cudaStream_t stream, int* kernel_id);

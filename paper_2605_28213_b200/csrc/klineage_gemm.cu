@@ -61,12 +61,14 @@ bool encode_map_3d(const RunContext& ctx, CUtensorMap* map, CUtensorMapDataType 
 }
 
 bool encode_map_nhwc(const RunContext& ctx, CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t C,
-                     uint64_t W, uint64_t H, uint64_t N, uint32_t c_box, uint32_t w_box, CUtensorMapSwizzle swz)
+                     uint64_t W, uint64_t H, uint64_t N, uint32_t c_box, uint32_t w_box, uint32_t h_box, int elt,
+                     CUtensorMapSwizzle swz)
 {
     if (!ctx.encode_tiled) return false;
+    const cuuint64_t e = static_cast<cuuint64_t>(elt);
     const cuuint64_t dims[4] = {C, W, H, N};
-    const cuuint64_t strides[3] = {C * 2, W * C * 2, H * W * C * 2};
-    const cuuint32_t box[4] = {c_box, w_box, 1, 1};
+    const cuuint64_t strides[3] = {C * e, W * C * e, H * W * C * e};
+    const cuuint32_t box[4] = {c_box, w_box, h_box, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     const CUresult r = ctx.encode_tiled(map, dt, 4, const_cast<void*>(base), dims, strides, box, estr,
                                         CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

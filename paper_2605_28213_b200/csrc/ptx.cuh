@@ -110,6 +110,14 @@ __device__ __forceinline__ void tma_store_3d(const void* tmap, int x, int y, int
                  ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(smem_u32(smem_src))
                  : "memory");
 }
+// 4-D tiled store shared -> global (bulk group).  Coordinates must be >= 0; the part of the box past the
+// tensor's extents is not written.
+__device__ __forceinline__ void tma_store_4d(const void* tmap, int c0, int c1, int c2, int c3, const void* smem_src)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(smem_src))
+                 : "memory");
+}
 // 2-D tiled store shared -> global (bulk group).  Coordinates must be >= 0.
 __device__ __forceinline__ void tma_store_2d(const void* tmap, int x, int y, const void* smem_src)
 {

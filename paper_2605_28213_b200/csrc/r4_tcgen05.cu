@@ -93,6 +93,8 @@ struct R4Params {
     int half_only;          // every unit is the first 128-column half of its tile (problems with N <= 128)
     int conv_b_tma;         // MODE 4: the weights come by TMA (warp 0), only the patches are gathered
     int conv_b_rows;        // rows of the weight box (128 with half_only, else 256)
+    int conv_patch;         // patches by TMA: row tile t = 8 x 16 output patch (t % tq, (t / tq) % tp) of image t / (tq tp)
+    int conv_tq, conv_tp;
 };
 
 // One entry of the static schedule.
@@ -264,8 +266,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         const CUtensorMap *ma, *mb;
         uint32_t it;
         bool live;
-        int cw[16], ch[16], cn[16];     // MODE 4 on TMA: input origin (w, h, n) of each 8-pixel group of the tile
-    } prod = {static_cast<int64_t>(blockIdx.x), 0, 0, 0, 0, 0, &map_a, &map_b, 0u, false, {}, {}, {}};
+        int cw, ch, cn;                 // MODE 4 on TMA: input origin (w, h) and image of the tile's 8 x 16 pixel patch
+    } prod = {static_cast<int64_t>(blockIdx.x), 0, 0, 0, 0, 0, &map_a, &map_b, 0u, false, 0, 0, 0};
     auto prod_enter_unit = [&]() {
         prod.live = prod.u < total_units;
         if (!prod.live) return;
@@ -280,15 +282,12 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             prod.mb = x.mb;
         }
         if (MODE == 4 && !GENERIC) {
-            // Q is a multiple of 8 here, so the 8 pixels of a group share (n, p) and are consecutive in q
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const int m = x.m0 + 8 * j;
-                const int q = m % p.conv.Q, t = m / p.conv.Q;
-                prod.cw[j] = q - p.conv.pad_w;
-                prod.ch[j] = t % p.conv.P - p.conv.pad_h;
-                prod.cn[j] = t / p.conv.P;          // >= N past the last pixel: the box reads zeros
-            }
+            // patch tiling: row tile t of the launch is the 8 x 16 output patch (pt, qt) of image n
+            const int t = x.m0 / BM;
+            const int qt = t % p.conv_tq, u2 = t / p.conv_tq;
+            prod.cw = qt * 16 - p.conv.pad_w;
+            prod.ch = (u2 % p.conv_tp) * 8 - p.conv.pad_h;
+            prod.cn = u2 / p.conv_tp;
         }
     };
     auto load_box = [&](void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
@@ -314,15 +313,13 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             const CUtensorMap* pa = (MODE == 2) ? prod.ma : &map_a;
             const CUtensorMap* pb = (MODE == 2) ? prod.mb : &map_b;
             if (MODE == 4) {
-                // Conv2d: k-block = (filter tap, 64-channel group); the A stage is 16 boxes of
-                // 8 pixels x 64 channels read at the tap's offset - outside the image the TMA unit
-                // fills zeros, which is the padding
+                // Conv2d: k-block = (filter tap, 64-channel group); the A stage is ONE box of 64 channels
+                // x 16 x 8 pixels (the tile's output patch shifted by the tap) - where it leaves the
+                // image the TMA unit fills zeros, which is the padding.  GEMM row = 16 * patch row + column.
                 const int cpb = p.conv.C >> 6;
                 const int tap = prod.kb / cpb, cg = prod.kb - tap * cpb;
                 const int fr = tap / p.conv.S, fs = tap - fr * p.conv.S;
-#pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    ptx::tma_load_4d(sa + j * 1024, &map_a, cg * 64, prod.cw[j] + fs, prod.ch[j] + fr, prod.cn[j], &full[s]);
+                ptx::tma_load_4d(sa, &map_a, cg * 64, prod.cw + fs, prod.ch + fr, prod.cn, &full[s]);
             } else
             load_box(sa, pa, prod.kb * BK, prod.m0, &full[s]);
             if (BCOL) {
@@ -633,7 +630,19 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 uint16_t* dst_h = reinterpret_cast<uint16_t*>(x.C);
                 const int64_t ld = partial ? p.ldw : x.ldc;
                 const int rows = min(32, x.M - row0);
-                for (int c = 0; c * cpc < x.ncols; ++c) {
+                // Conv2d with patch tiling: this warp's 32 rows are patch rows 2q, 2q+1 (16 pixels each) of
+                // the 8 x 16 output patch (pt, qt) of image cn
+                int cq0 = 0, cp0 = 0, cimg = 0;
+                bool below = false;
+                if (MODE == 4 && !GENERIC) {
+                    const int t = m0 / BM;
+                    const int qt = t % p.conv_tq, u2 = t / p.conv_tq;
+                    cq0 = qt * 16;
+                    cp0 = (u2 % p.conv_tp) * 8 + 2 * q;
+                    cimg = u2 / p.conv_tp;
+                    below = cp0 >= p.conv.P;                      // the patch rows of this warp lie below the image
+                }
+                for (int c = 0; c * cpc < x.ncols && !below; ++c) {
                     const int col0 = n0 + c * cpc;
                     if (col0 >= x.N) break;
                     uint32_t v[32], w[32];
@@ -683,6 +692,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         if (lane == 0) {
                             if (MODE == 1) {
                                 ptx::tma_store_3d(x.mc, col0, row0, x.z, b);
+                            } else if (MODE == 4 && !GENERIC) {
+                                ptx::tma_store_4d(x.mc, col0, cq0, cp0, cimg, b);   // box: columns x 16 x 2 pixels, clipped at the image
                             } else if (MODE == 3) {
                                 for (int d = 0; d < p.n_dst; ++d) ptx::tma_store_2d(&p.dsts[d].map_c, col0, row0, b);
                             } else {
@@ -703,7 +714,12 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                             const uint32_t word =
                                 *reinterpret_cast<const uint32_t*>(b + rr * 128 + (((lane >> 2) ^ (rr & 7)) << 4) +
                                                                    (lane & 3) * 4);
-                            const int64_t row = row0 + rr;
+                            int64_t row = row0 + rr;
+                            if (MODE == 4 && !GENERIC) {     // staged row rr = pixel (cp0 + rr / 16, cq0 + rr % 16)
+                                const int pp = cp0 + (rr >> 4), qq = cq0 + (rr & 15);
+                                if (pp >= p.conv.P || qq >= p.conv.Q) continue;
+                                row = (static_cast<int64_t>(cimg) * p.conv.P + pp) * p.conv.Q + qq;
+                            }
                             if (out_bf16) {
                                 const int col = col0 + 2 * lane;
                                 uint16_t* d = dst_h + row * ldd + col;
@@ -1580,19 +1596,42 @@ cudaError_t launch_r4_conv2d(const GemmArgs& g, const ConvGeom& geom, RunContext
     } else {
         grid = finish_multi_schedule(p, tiles, true, ctx);
     }
-    // Patches by TMA: 64-channel groups (a k-block is one tap of one group), unit stride, and an output
-    // width that is a multiple of 8, so that the 8 pixels of a box never straddle an output row.
+    // Patches by TMA: 64-channel groups (a k-block is one tap of one group) and unit stride.  The rows are
+    // then tiled as 8 x 16 pixel patches of the output (one 16 KiB TMA box per k-block, clipped stores at the
+    // image edges) instead of 128 consecutive pixels.
     CUtensorMap mx;
     memset(&mx, 0, sizeof mx);
-    const bool patch_tma = p.conv_b_tma && geom.C % 64 == 0 && geom.Q % 8 == 0 && geom.stride_h == 1 && geom.stride_w == 1 &&
-                           encode_map_nhwc(ctx, &mx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, g.A, geom.C, geom.W, geom.H,
-                                           static_cast<uint64_t>(g.M / (static_cast<int64_t>(geom.P) * geom.Q)), 64, 8,
-                                           CU_TENSOR_MAP_SWIZZLE_128B);
+    const int64_t n_img = g.M / (static_cast<int64_t>(geom.P) * geom.Q);
+    const int tq = (geom.Q + 15) / 16, tp = (geom.P + 7) / 8;
+    const int64_t patch_tiles = n_img * tp * tq * p.tiles_n;
+    bool patch_tma = p.conv_b_tma && geom.C % 64 == 0 && geom.stride_h == 1 && geom.stride_w == 1 &&
+                     patch_tiles < 0x3FFFFFFFll / BM &&
+                     encode_map_nhwc(ctx, &mx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, g.A, geom.C, geom.W, geom.H,
+                                     static_cast<uint64_t>(n_img), 64, 16, 8, 2, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (patch_tma && p.epi_tma)     // y as a 4-D tensor (F, Q, P, N): a warp stores 2 patch rows x 16 pixels per box
+        patch_tma = encode_map_nhwc(ctx, &mc, g.c_bf16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                                    g.C, g.N, geom.Q, geom.P, static_cast<uint64_t>(n_img), g.c_bf16 ? 64 : 32, 16, 2, celt,
+                                    CU_TENSOR_MAP_SWIZZLE_128B);
     p.kid = kIdConvTcgen05 + (patch_tma ? 0 : 4) + (p.epi_tma ? 0 : 2) + (p.conv_fast ? 0 : 1);
     *kernel_id = p.kid;
     if (patch_tma) {
+        // the schedule runs over patch tiles: a virtual row count of 128 per patch (clipping happens in the stores)
+        GemmArgs gp = g;
+        gp.M = static_cast<int>(n_img * tp * tq * BM);
+        p.conv_patch = 1;
+        p.conv_tq = tq;
+        p.conv_tp = tp;
+        p.tiles_m = static_cast<int>(n_img * tp * tq);
         p.stage_tx = kABytes + static_cast<uint32_t>(p.conv_b_rows) * 128u;
-        return launch<true, false, false, 4>(g, mx, mb, mc, p, grid, ctx.device, stream);
+        unsigned pgrid;
+        if (p.half_only) {
+            p.full_units = 0;
+            p.total_units = patch_tiles;
+            pgrid = static_cast<unsigned>(patch_tiles < ctx.sm_count ? patch_tiles : ctx.sm_count);
+        } else {
+            pgrid = finish_multi_schedule(p, patch_tiles, true, ctx);
+        }
+        return launch<true, false, false, 4>(gp, mx, mb, mc, p, pgrid, ctx.device, stream);
     }
     return launch<true, true, false, 4>(g, none, mb, mc, p, grid, ctx.device, stream);
 }
