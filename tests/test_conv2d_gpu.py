@@ -71,6 +71,9 @@ SHAPES = [  # N, H, W, C, F, R, S, pad, stride
     (2, 6, 5, 5, 9, 2, 3, (0, 2), (1, 1)),           # C % 8 != 0: element-wise patch gather
     (1, 20, 20, 32, 300, 3, 3, (1, 1), (1, 1)),      # more than one column tile, half-tile tail
     (1, 3, 3, 8, 8, 3, 3, (0, 0), (1, 1)),           # a single output pixel
+    (2, 13, 21, 64, 100, 3, 3, (1, 1), (1, 1)),      # patch tiling, P and Q ragged; F * 2 % 16 != 0: masked stores by pixel
+    (1, 17, 35, 64, 328, 3, 3, (0, 2), (1, 1)),      # patch tiling, two column tiles (one a half tile), asymmetric padding
+    (3, 8, 16, 192, 64, 1, 1, (0, 0), (1, 1)),       # patch tiling, 1x1 filter over three 64-channel groups, exact patches
 ]
 
 
