@@ -73,6 +73,7 @@ struct R4Params {
     uint32_t stage_tx;      // bytes one stage's TMA loads deliver (A box + B boxes)
     int cluster;            // 1: the splits of a tile are one cluster and reduce through DSMEM
     int splits_log2;        // cluster mode: splits is 2, 4 or 8
+    int b_box3d;            // row-major B whose four 64-column blocks of a stage arrive as ONE 3-D box
     int static_b;           // the caller promised static B: the first ring fill's B boxes go out before the dependency wait
     int group_m;            // tile raster: tile-rows per group
     int64_t full_units;     // units [0, full_units) are whole tiles; later ones are 128-column half tiles
@@ -324,6 +325,13 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             load_box(sa, pa, prod.kb * BK, prod.m0, &full[s]);
             if (BCOL) {
                 load_box(sb, pb, prod.kb * BK, prod.n0, &full[s]);
+            } else if (MODE == 1 && p.b_box3d) {
+                ptx::tma_load_4d(sb, pb, 0, prod.kb * BK, prod.n0 >> 6, prod.z, &full[s]);   // the same box, batch as 4th coordinate
+            } else if ((MODE == 0 || MODE == 3) && p.b_box3d) {
+                // B viewed as (64 columns, K rows, N / 64 column blocks): one box of 64 x 64 x 4 lands as the
+                // four consecutive 8 KiB blocks the MN-major descriptor expects - one TMA instruction, not four
+                // (a producer thread issues a TMA instruction every ~110 cycles)
+                ptx::tma_load_3d(sb, pb, 0, prod.kb * BK, prod.n0 >> 6, &full[s]);
             } else {
 #pragma unroll
                 for (int cb = 0; cb < BN / 64; ++cb)
@@ -999,6 +1007,20 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     }
 }
 
+// Row-major B (K x N, N a multiple of 64) as a 3-D tensor: 64 columns innermost, the K rows, then the
+// N / 64 column blocks (128 bytes apart); the box takes `blocks` column blocks of 64 x BK.
+bool encode_b_blocks_3d(const RunContext& ctx, CUtensorMap* map, const GemmArgs& g, uint32_t blocks)
+{
+    if (!ctx.encode_tiled) return false;
+    const cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(g.K), static_cast<cuuint64_t>(g.N / 64)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(g.ldb) * 2, 128};
+    const cuuint32_t box[3] = {64, BK, blocks};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return ctx.encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<uint16_t*>(g.B), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool tma_ok(const void* base, int64_t ld_elems, int elt)
 {
     return reinterpret_cast<uintptr_t>(base) % 16 == 0 && (ld_elems * elt) % 16 == 0 &&
@@ -1335,6 +1357,8 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
         if (g.b_col)
             ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, BN,
                                      CU_TENSOR_MAP_SWIZZLE_128B);
+        else if (g.N % 64 == 0 && !p.static_b && encode_b_blocks_3d(ctx, &mb, g, BN / 64))
+            p.b_box3d = 1;
         else
             ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, g.ldb * 2, 64, BK,
                                      CU_TENSOR_MAP_SWIZZLE_128B);
@@ -1460,7 +1484,17 @@ cudaError_t launch_r4_single_batched(const GemmArgs& g, const BatchArgs& b, RunC
     if (g.b_col)
         ok = ok && encode_map_3d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, nb, g.ldb * 2, b.stride_b * 2,
                                  BK, BN, CU_TENSOR_MAP_SWIZZLE_128B);
-    else
+    else if (g.N % 64 == 0 && ctx.encode_tiled) {
+        // the four 64-column blocks of a stage as one box: B as (64 columns, K rows, N / 64 blocks, batch)
+        const cuuint64_t dims[4] = {64, static_cast<cuuint64_t>(g.K), static_cast<cuuint64_t>(g.N / 64), nb};
+        const cuuint64_t strides[3] = {static_cast<cuuint64_t>(g.ldb) * 2, 128, static_cast<cuuint64_t>(b.stride_b) * 2};
+        const cuuint32_t box[4] = {64, BK, BN / 64, 1};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        ok = ok && ctx.encode_tiled(&mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<uint16_t*>(g.B), dims, strides, box,
+                                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+        p.b_box3d = 1;
+    } else
         ok = ok && encode_map_3d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, nb, g.ldb * 2, b.stride_b * 2,
                                  64, BK, CU_TENSOR_MAP_SWIZZLE_128B);
     if (p.epi_tma)
