@@ -89,8 +89,9 @@ typedef struct {
     int device;             /* CUDA device ordinal the handle is bound to                              */
     int b_layout;           /* klineage_layout_t                                                       */
     int c_dtype;            /* klineage_ctype_t                                                        */
-    size_t workspace_bytes; /* device scratch: split-K partial sums and aligned copies of unaligned operands
-                               (rung 4); 0 selects the default (64 MiB)                                */
+    size_t workspace_bytes; /* device scratch of rung 4: split-K partial sums, aligned copies of unaligned
+                               operands, the tables of grouped / multi-destination launches; 0 selects
+                               the default (64 MiB).  Calls on one handle share it: one stream at a time */
     unsigned flags;         /* 0, or KLINEAGE_FLAG_STATIC_B                                            */
 } klineage_gemm_config_t;
 
