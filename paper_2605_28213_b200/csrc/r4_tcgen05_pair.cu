@@ -384,7 +384,9 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 ptx::tmem_ld_32x32b_x32(tbase + u * cpc, r0);
                 if (out_bf16) ptx::tmem_ld_32x32b_x32(tbase + u * cpc + 32, r1);
             };
-            auto finish = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32]) {
+            // pack: bias and rounding of one unit (r0, r1 -> 32 words of output); stage_store: the words
+            // go through the warp's staging block to global memory
+            auto pack = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32], uint32_t (&w)[32]) {
                 const int col0 = n0 + u * cpc;
                 if (g.bias) {   // AddMM: this unit's columns get their bias in fp32, before any rounding
                     // lane l fetches the bias of columns col0 + l and col0 + 32 + l; a shuffle hands column i's
@@ -397,7 +399,6 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                         if (out_bf16) r1[i] = __float_as_uint(__uint_as_float(r1[i]) + __shfl_sync(0xFFFFFFFFu, b1, i));
                     }
                 }
-                uint32_t w[32];
                 if (out_bf16) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
@@ -408,6 +409,9 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
 #pragma unroll
                     for (int i = 0; i < 32; ++i) w[i] = r0[i];
                 }
+            };
+            auto stage_store = [&](int u, const uint32_t (&w)[32]) {
+                const int col0 = n0 + u * cpc;
                 // (a warp's staging buffer may still be read by its previous TMA store, possibly of
                 // another group's tile: wait whenever any tile of the launch can take that path)
                 if (p.epi_tma) {
@@ -461,12 +465,40 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     __syncwarp();
                 }
             };
+            auto finish = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32]) {
+                uint32_t w[32];
+                pack(u, r0, r1, w);
+                stage_store(u, w);
+            };
 
             if (nunits == 0) {
                 release();
                 continue;
             }
             uint32_t a0[32], a1[32], c0[32], c1[32];
+            if (out_bf16 && nunits == 4) {
+                // Full-width bf16 tile: the accumulator is handed back before anything is staged or stored.
+                // Rounding (F2F, 16 results per clock and SM) is what the drain costs, so the first two units
+                // are rounded while the last two are read, the accumulator is released, and staging and the
+                // TMA stores run while the next tile's MMAs already fill it again.
+                uint32_t w0[32], w1[32];
+                issue(0, a0, a1);
+                issue(1, c0, c1);
+                ptx::tmem_ld_wait();
+                pack(0, a0, a1, w0);
+                issue(2, a0, a1);
+                pack(1, c0, c1, w1);
+                issue(3, c0, c1);
+                ptx::tmem_ld_wait();
+                release();
+                stage_store(0, w0);
+                stage_store(1, w1);
+                pack(2, a0, a1, w0);
+                stage_store(2, w0);
+                pack(3, c0, c1, w1);
+                stage_store(3, w1);
+                continue;
+            }
             issue(0, a0, a1);
             for (int u = 0; u < nunits; u += 2) {
                 ptx::tmem_ld_wait();
