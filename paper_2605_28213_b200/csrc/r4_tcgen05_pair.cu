@@ -51,7 +51,14 @@ constexpr int kEpiBytes = 8 * kEpiBufBytes;       // one staging block per epilo
 constexpr int kBarBytes = 1536;                 // barriers, TMEM slot, abort flag, grouped schedule (<= 257 ints)
 constexpr int kSmemBytes = 1024 + STAGES * kStageBytes + kEpiBytes + kBarBytes;
 constexpr int kTmemCols = 512;
-constexpr int kThreads = 10 * 32;                // producer, MMA issuer, 2 x 4 epilogue warps
+constexpr int kThreads = 12 * 32;                // warp group 0: producer, MMA issuer, two idle warps; groups 1, 2: 2 x 4 epilogue warps
+constexpr int kEpiWarp0 = 4;                     // first epilogue warp
+// Registers: the kernel is compiled for 168 per thread (three warps share a 16 K-register scheduler
+// partition); the first warp group gives its surplus back (setmaxnreg.dec) and the epilogue groups
+// take it (setmaxnreg.inc), so that three fp32 units of the accumulator fit in registers at once.
+// The two amounts must balance (the pool the increase draws from holds only what was released:
+// with 48 instead of 40 the increase never completed and the launch hung).
+constexpr int kRegsLean = 40, kRegsEpilogue = 232;   // balanced: 128 x (168 - 40) released = 256 x (232 - 168) taken
 
 struct PairParams {
     int tiles_m2, tiles_n;      // 512-row x 256-column tiles
@@ -135,6 +142,16 @@ __device__ __forceinline__ void tma_load_3d_pair(void* smem_dst, const void* tma
         "r"(cluster_bar_addr)
         : "memory");
 }
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec()
+{
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc()
+{
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar_addr)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar_addr) : "memory");
@@ -189,8 +206,8 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         }
         if (blockIdx.x == 0) g.status[1] = p.kid;
     }
-    if (MODE == 2 && warp >= 2) {
-        for (int i = threadIdx.x - 64; i <= p.n_groups; i += kThreads - 64)
+    if (MODE == 2 && warp >= kEpiWarp0) {
+        for (int i = threadIdx.x - kEpiWarp0 * 32; i <= p.n_groups; i += kThreads - kEpiWarp0 * 32)
             gstart[i] = (i < p.n_groups) ? p.groups[i].tile_start : static_cast<int>(p.total_tiles);
     }
     if (warp == 1) {
@@ -259,6 +276,10 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             tma_load_2d_pair(dst, map, c0, c1, bar);
     };
 
+    if (warp < kEpiWarp0) {
+    // One instruction for the whole first warp group (the register release is warp-group wide), ahead of
+    // the producer and MMA code, which run within the reduced budget.
+    setmaxnreg_dec<kRegsLean>();
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -345,15 +366,17 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 }
             }
         }
+    }
     } else {
         // ------------------------------------------------------------ epilogue
-        // Warps 2..5 drain the first row block's accumulator, warps 6..9 the second; a warp
+        setmaxnreg_inc<kRegsEpilogue>();
+        // Warps 4..7 drain the first row block's accumulator, warps 8..11 the second; a warp
         // reads the TMEM lane quarter (warp & 3).  TMEM loads of the next 128-byte unit are in
         // flight while the current one is converted, staged and stored, and the accumulator is
         // handed back as soon as its last load has landed.
         const int q = warp & 3;
-        const int mb = (warp - 2) >> 2;
-        uint8_t* b = epi_smem + (warp - 2) * kEpiBufBytes;
+        const int mb = (warp - kEpiWarp0) >> 2;
+        uint8_t* b = epi_smem + (warp - kEpiWarp0) * kEpiBufBytes;
         const bool out_bf16 = g.c_bf16 != 0;
         const int cpc = out_bf16 ? 64 : 32;                   // columns per 128-byte staging row
         uint32_t tcount = 0;
@@ -478,25 +501,26 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             uint32_t a0[32], a1[32], c0[32], c1[32];
             if (out_bf16 && nunits == 4) {
                 // Full-width bf16 tile: the accumulator is handed back before anything is staged or stored.
-                // Rounding (F2F, 16 results per clock and SM) is what the drain costs, so the first two units
-                // are rounded while the last two are read, the accumulator is released, and staging and the
-                // TMA stores run while the next tile's MMAs already fill it again.
-                uint32_t w0[32], w1[32];
+                // Rounding (F2F, 16 results per clock and SM) is what the drain costs: three units are read
+                // raw (192 registers), one is rounded to make room for the fourth, the accumulator is
+                // released, and the other roundings, staging and the TMA stores run while the next tile's
+                // MMAs already fill it again.
+                uint32_t d0[32], d1[32], w0[32];
                 issue(0, a0, a1);
                 issue(1, c0, c1);
+                issue(2, d0, d1);
                 ptx::tmem_ld_wait();
-                pack(0, a0, a1, w0);
-                issue(2, a0, a1);
-                pack(1, c0, c1, w1);
-                issue(3, c0, c1);
+                pack(0, a0, a1, w0);           // frees a0, a1 for the fourth unit
+                issue(3, a0, a1);
                 ptx::tmem_ld_wait();
                 release();
                 stage_store(0, w0);
-                stage_store(1, w1);
-                pack(2, a0, a1, w0);
+                pack(1, c0, c1, w0);
+                stage_store(1, w0);
+                pack(2, d0, d1, w0);
                 stage_store(2, w0);
-                pack(3, c0, c1, w1);
-                stage_store(3, w1);
+                pack(3, a0, a1, w0);
+                stage_store(3, w0);
                 continue;
             }
             issue(0, a0, a1);
