@@ -39,8 +39,8 @@ WORKLOADS = {
 WORKLOAD = WORKLOADS["c4"]
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one tcgen05-rung launch at 8192^3
-# (ncu capture summarised in profiles/r4_tcgen05_c4_8192.md): 0.882 GB read + 0.130 GB written.
-R4_C4_DRAM_TRAFFIC_BYTES = 1.012e9
+# (ncu capture summarised in profiles/r4_tcgen05_c4_8192.md): 0.884 GB read + 0.141 GB written.
+R4_C4_DRAM_TRAFFIC_BYTES = 1.026e9
 # the same for the skinny shape (profiles/r4_tcgen05_c5_skinny.md): 134.6 MB read + 3.9 MB written.
 R4_C5_DRAM_TRAFFIC_BYTES = 1.385e8
 VARIANT_NAMES = ["naive", "tiled", "vectorized", "pipelined", "tcgen05", "mma_sync"]
