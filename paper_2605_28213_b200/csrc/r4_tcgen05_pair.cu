@@ -17,9 +17,13 @@
 //               (cp.async.bulk.tensor ... .cta_group::2 lets the barrier live in
 //               the partner), which expects the bytes of both
 //   warp 1      even CTA: MMA issuer; idle in the odd CTA
-//   warps 2..9  epilogue: four warps per row block drain its accumulator (TMEM
-//               loads software-pipelined against convert / stage / TMA store or
-//               masked stores) and hand it back right after the last load
+//   warps 2..3  idle: they complete the first warp group, which as a whole hands most of its
+//               registers to the epilogue groups (setmaxnreg)
+//   warps 4..11 epilogue: four warps per row block drain its accumulator.  A full-width bf16
+//               tile reads three of its four 64-column units raw into registers, rounds one to
+//               make room for the fourth, releases the accumulator and only then rounds the
+//               rest, stages and stores (TMA store or masked stores); other tiles go unit by
+//               unit, software-pipelined, and release after the last load
 // "Stage free" and "accumulator ready" reach both CTAs through two plain
 // tcgen05.commit instructions (own barrier, peer's barrier), never the
 // cluster-wide broadcast form.  All waits are bounded; both CTAs pass a cluster barrier
