@@ -527,6 +527,39 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 stage_store(3, w0);
                 continue;
             }
+            if (!out_bf16 && nunits == 8) {
+                // Full-width fp32 tile (eight 32-column units, nothing to round): six units are read raw, two
+                // are staged and stored to make room for the last two, then the accumulator is released.
+                uint32_t d0[32], d1[32];
+                issue(0, a0, a1);
+                issue(1, a1, a0);          // (a unit is one 32-column load here: the second array is unused)
+                issue(2, c0, c1);
+                issue(3, c1, c0);
+                issue(4, d0, d1);
+                issue(5, d1, d0);
+                ptx::tmem_ld_wait();
+                if (g.bias) pack(0, a0, a0, a0);
+                stage_store(0, a0);
+                issue(6, a0, a0);
+                if (g.bias) pack(1, a1, a1, a1);
+                stage_store(1, a1);
+                issue(7, a1, a1);
+                ptx::tmem_ld_wait();
+                release();
+                if (g.bias) pack(2, c0, c0, c0);
+                stage_store(2, c0);
+                if (g.bias) pack(3, c1, c1, c1);
+                stage_store(3, c1);
+                if (g.bias) pack(4, d0, d0, d0);
+                stage_store(4, d0);
+                if (g.bias) pack(5, d1, d1, d1);
+                stage_store(5, d1);
+                if (g.bias) pack(6, a0, a0, a0);
+                stage_store(6, a0);
+                if (g.bias) pack(7, a1, a1, a1);
+                stage_store(7, a1);
+                continue;
+            }
             issue(0, a0, a1);
             for (int u = 0; u < nunits; u += 2) {
                 ptx::tmem_ld_wait();

@@ -108,3 +108,25 @@ def test_addmm_argument_errors(kb):
         assert raw(c.data_ptr() + 8) == kb.KLINEAGE_ERR_INVALID_ARG          # bias overlaps C
         assert raw(a.data_ptr() + 2) == kb.KLINEAGE_OK
         torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("bf", [False, True], ids=["f32", "bf16"])
+def test_addmm_on_the_pair_kernel_full_width_tiles(kb, bf):
+    # full-width tiles of the CTA-pair kernel hand the accumulator back before they stage and store:
+    # the bias must still reach every unit, for both output types
+    import torch
+    M, N, K = 600, 776, 136
+    for dist, exact in (("integer", True), ("normal", False)):
+        case = gen.make_case(M, N, K, seed=260, dist_a=dist, dist_b=dist, c_bf16=bf, name=f"addmm-pair-{dist}")
+        bias = gen.draw((1, N), dist, 261, 2)[0]
+        C_ref, S = reference(case, bias, np.arange(M))
+        dev = P.DeviceCase(case)
+        bbuf = P.DeviceBuffer(bias.size * 2).upload(bias)
+        with kb.Gemm(0, c_bf16=bf) as g:
+            g.set_plan(kb.klineage_gemm_plan_t(2, 1, 0, 0, 0), dev.a.ptr, dev.b.ptr, dev.c.ptr, M, N, K, case.lda, case.ldb,
+                       case.ldc)
+            g.run_addmm(dev.a.ptr, dev.b.ptr, bbuf.ptr, dev.c.ptr, M, N, K, case.lda, case.ldb, case.ldc, 4)
+            torch.cuda.synchronize()
+            assert g.device_status()[0] == 0 and (g.last_kernel_id() - 400) & 32
+        vals, bits = dev.result()
+        P.assert_matches_oracle(case, vals, bits, C_ref, S, exact=exact, what=f"{case.name} bf16={bf}")
