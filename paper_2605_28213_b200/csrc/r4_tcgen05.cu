@@ -1179,14 +1179,29 @@ namespace {
 // buffer whose pitch is a multiple of 8 elements, zero-filling the pitch padding: the
 // precondition repair that lets an unaligned operand use the TMA / tcgen05 path.  One
 // 16-byte store per thread; consecutive threads take consecutive 8-element groups.
-__global__ void __launch_bounds__(256) repack_rows_kernel(const uint16_t* __restrict__ src, int64_t ld_src,
-                                                          uint16_t* __restrict__ dst, int64_t ld_dst, int64_t rows,
-                                                          int cols)
+// Both operands of a call go through ONE launch: blocks [0, blocks_first) copy the first matrix, the rest
+// the second (a matrix with rows == 0 has no blocks).
+struct RepackJob {
+    const uint16_t* src;
+    int64_t ld_src;
+    uint16_t* dst;
+    int64_t ld_dst, rows;
+    int cols;
+};
+__global__ void __launch_bounds__(256) repack_rows_kernel(RepackJob first, RepackJob second, unsigned blocks_first)
 {
+    const bool is_first = blockIdx.x < blocks_first;
+    const RepackJob& j = is_first ? first : second;
+    const unsigned block = is_first ? blockIdx.x : blockIdx.x - blocks_first;
+    const unsigned nblocks = is_first ? blocks_first : gridDim.x - blocks_first;
+    const uint16_t* __restrict__ src = j.src;
+    uint16_t* __restrict__ dst = j.dst;
+    const int64_t ld_src = j.ld_src, ld_dst = j.ld_dst;
+    const int cols = j.cols;
     const int64_t groups_per_row = ld_dst >> 3;
-    const int64_t total = rows * groups_per_row;
-    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
-         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t total = j.rows * groups_per_row;
+    for (int64_t i = block * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(nblocks) * blockDim.x) {
         const int64_t r = i / groups_per_row;
         const int c0 = static_cast<int>(i - r * groups_per_row) * 8;
         const uint16_t* s = src + r * ld_src + c0;
@@ -1231,25 +1246,27 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
 
     GemmArgs g2 = g;
     uint8_t* ws = static_cast<uint8_t*>(ctx.workspace);
-    auto repack = [&](const uint16_t* src, int64_t ld_src, uint16_t* dst, int64_t ld_dst, int64_t rows, int cols) {
-        const int64_t groups = rows * (ld_dst >> 3);
-        const int64_t blocks = (groups + 255) / 256;
-        repack_rows_kernel<<<static_cast<unsigned>(blocks < 8 * 148 ? blocks : 8 * 148), 256, 0, stream>>>(
-            src, ld_src, dst, ld_dst, rows, cols);
-        return cudaGetLastError();
+    RepackJob ja = {nullptr, 0, nullptr, 8, 0, 0}, jb = ja;
+    auto blocks_of = [](const RepackJob& j) {
+        const int64_t blocks = (j.rows * (j.ld_dst >> 3) + 255) / 256;
+        return static_cast<unsigned>(blocks < 8 * 148 ? blocks : 8 * 148);
     };
     if (bad_a) {
-        cudaError_t e = repack(g.A, g.lda, reinterpret_cast<uint16_t*>(ws), lda2, g.M, g.K);
-        if (e != cudaSuccess) return e;
+        ja = {g.A, g.lda, reinterpret_cast<uint16_t*>(ws), lda2, g.M, g.K};
         g2.A = reinterpret_cast<const uint16_t*>(ws);
         g2.lda = lda2;
     }
     if (bad_b) {
         uint16_t* dst = reinterpret_cast<uint16_t*>(ws + ((bytes_a + 255) & ~size_t(255)));
-        cudaError_t e = repack(g.B, g.ldb, dst, ldb2, b_rows, static_cast<int>(b_cols));
-        if (e != cudaSuccess) return e;
+        jb = {g.B, g.ldb, dst, ldb2, b_rows, static_cast<int>(b_cols)};
         g2.B = dst;
         g2.ldb = ldb2;
+    }
+    {
+        const unsigned na = blocks_of(ja), nb = blocks_of(jb);
+        repack_rows_kernel<<<na + nb, 256, 0, stream>>>(ja, jb, na);
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
     }
     RunContext c2 = ctx;
     c2.workspace = ws + used;
