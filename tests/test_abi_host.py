@@ -105,3 +105,52 @@ def test_product_never_imports_the_oracle():
     for f in (ROOT / "oracle").glob("*"):
         if f.suffix in (".py", ".c"):
             assert not back.search(f.read_text()), f"{f} reaches into the product"
+
+
+def test_conv2d_check_args_rules(kb):
+    # host-only: the geometry and aliasing rules of the Conv2d call need no GPU
+    chk = kb.klineage_conv2d_check_args
+    X, Wt, Y = 0x100000, 0x200000, 0x400000
+
+    def call(**kw):
+        return chk(kw.get("dt", kb.KLINEAGE_C_F16), kw.get("N", 1), kw.get("H", 8), kw.get("W", 8), kw.get("C", 8),
+                   kw.get("F", 8), kw.get("R", 3), kw.get("S", 3), kw.get("ph", 1), kw.get("pw", 1), kw.get("sh", 1),
+                   kw.get("sw", 1), kw.get("x", X), kw.get("w", Wt), kw.get("y", Y), kw.get("v", kb.KLINEAGE_TCGEN05))
+
+    assert call() == kb.KLINEAGE_OK
+    assert call(dt=kb.KLINEAGE_C_F32) == kb.KLINEAGE_OK
+    assert call(dt=kb.KLINEAGE_C_BF16) == kb.KLINEAGE_ERR_INVALID_ARG      # bf16 is not a Conv2d output type
+    assert call(v=kb.KLINEAGE_NAIVE) == kb.KLINEAGE_OK
+    for v in (1, 2, 3, 5, 6, -1):
+        assert call(v=v) == kb.KLINEAGE_ERR_BAD_VARIANT
+    assert call(R=0) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert call(S=65) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert call(sh=0) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert call(pw=-1) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert call(H=1, ph=0) == kb.KLINEAGE_ERR_INVALID_ARG                  # filter taller than the padded image
+    assert call(H=1, ph=1) == kb.KLINEAGE_OK                               # ... but not with padding 1: P = 1
+    assert call(y=None) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert call(x=None) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert call(y=X) == kb.KLINEAGE_ERR_INVALID_ARG                        # y aliases x
+    assert call(y=Wt + 2) == kb.KLINEAGE_ERR_INVALID_ARG                   # y overlaps w
+    assert call(y=Y + 1) == kb.KLINEAGE_ERR_INVALID_ARG                    # fp16 y must be 2-byte aligned
+    assert call(dt=kb.KLINEAGE_C_F32, y=Y + 2) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert call(N=0, y=None, x=None, w=None) == kb.KLINEAGE_OK             # nothing to compute
+    assert call(F=0, y=None) == kb.KLINEAGE_OK
+    assert call(C=0) == kb.KLINEAGE_OK                                     # K = 0: y is zero-filled, x and w unused
+    assert call(N=1 << 21) == kb.KLINEAGE_ERR_INVALID_ARG
+
+
+def test_null_handles_are_refused_everywhere(kb):
+    P = 0x100000
+    assert kb.klineage_gemm_run_raw(None, 8, 8, 8, P, 8, P * 2, 8, P * 3, 8, 4, None) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert kb.klineage_gemm_run_addmm_raw(None, 8, 8, 8, P, 8, P * 2, 8, P * 4, P * 3, 8, 4, None) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert kb.klineage_gemm_run_batched_raw(None, 2, 8, 8, 8, P, 8, 64, P * 2, 8, 64, P * 3, 8, 64, 4, None) == \
+        kb.KLINEAGE_ERR_INVALID_ARG
+    assert kb.klineage_gemm_run_grouped_raw(None, [8], [8], [8], [P], [8], [P * 2], [8], [P * 3], [8], 4, None) == \
+        kb.KLINEAGE_ERR_INVALID_ARG
+    assert kb.klineage_gemm_run_multi_dst_raw(None, 8, 8, 8, P, 8, P * 2, 8, [P * 3], [8], 4, None) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert kb.klineage_conv2d_run_raw(None, 1, 8, 8, 8, 8, 3, 3, 1, 1, 1, 1, P, P * 2, P * 3, 4, None) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert kb.klineage_gemm_set_plan_raw(None, 8, 8, 8, P, 8, P * 2, 8, P * 3, 8, None) == kb.KLINEAGE_ERR_INVALID_ARG
+    assert kb._lib.klineage_gemm_last_launch_count(None) == 0
+    assert kb.klineage_gemm_last_kernel_id(None) == -1
