@@ -626,10 +626,22 @@ bool r4_pair_possible(const GemmArgs& g, const RunContext& ctx)
 
 bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx)
 {
-    if (!r4_pair_possible(g, ctx)) return false;
-    // worthwhile only when the pairs fill the machine: at least one 512 x 256 tile per SM pair
-    const int64_t tiles = static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * ((g.N + PN - 1) / PN);
-    return g.M > 2 * PM && tiles >= ctx.sm_count / 2;
+    if (!r4_pair_possible(g, ctx) || g.M <= 2 * PM) return false;
+    // Which kernel finishes first?  Estimated tensor-pipe cycles of either schedule, from measured rates:
+    // a 512 x 256 pair tile takes 1024 cycles per k-block (two accumulators alternate: full rate) plus
+    // ~5 k cycles per tile that the main loop does not hide (ring fill, accumulator drain and store); a 128 x 256
+    // tile of the single-CTA kernel takes 636 per k-block (one accumulator: 159 per MMA) with its epilogue
+    // hidden, and a last wave of at most half of the SMs is cut into half tiles worth ~0.75 of a wave.
+    // Fitted to both kernels timed at 2048^3 .. 4096^3 (steps of 256), 2048 x 4096 x 4096 and 3072 x 2048 x 8192.
+    const int64_t nkb = (g.K + BK - 1) / BK;
+    const int64_t pairs = ctx.sm_count / 2;
+    const int64_t tiles2 = static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * ((g.N + PN - 1) / PN);
+    const double t_pair = static_cast<double>((tiles2 + pairs - 1) / pairs) * (nkb * 1024.0 + 5000.0);
+    const int64_t tiles1 = static_cast<int64_t>((g.M + PM - 1) / PM) * ((g.N + PN - 1) / PN);
+    const int64_t full = tiles1 / ctx.sm_count, tail = tiles1 % ctx.sm_count;
+    const double waves = full + (tail == 0 ? 0.0 : (2 * tail <= ctx.sm_count && g.N > PN / 2 ? 0.75 : 1.0));
+    const double t_single = waves * nkb * 636.0;
+    return t_pair < t_single;
 }
 
 namespace {

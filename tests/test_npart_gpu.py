@@ -36,6 +36,9 @@ def run_world(kb, case, world, variant, quantum=8, expect_one_launch=None, expec
                 Bs = np.full((case.K, ldb), 0x7FC0, np.uint16)
                 Bs[:, :part.n_local] = case.B[:, part.n0:part.n1]
             b = P.DeviceBuffer(Bs.size * 2).upload(Bs)
+            if expect_pair:             # pin the CTA-pair kernel for this rank's slice (short K would take the other kernel)
+                g.set_plan(kb.klineage_gemm_plan_t(2, 1, 0, 0, 0), a.ptr, b.ptr, part.dst[0], case.M, part.n_local, case.K,
+                           case.lda, ldb, case.ldc)
             part.run(a.ptr, b.ptr, case.M, case.K, case.lda, ldb, variant)
             torch.cuda.synchronize()
             code, _ = g.device_status()

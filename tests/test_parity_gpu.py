@@ -43,9 +43,19 @@ def handles_tiny_ws(kb):
         h.close()
 
 
-def run_and_check(handles, case, variant, C_ref=None, S=None, rows=None, exact=False, offsets=(0, 0, 0)):
+def run_and_check(handles, case, variant, C_ref=None, S=None, rows=None, exact=False, offsets=(0, 0, 0), pin=None):
+    """pin: a launch plan (kernel, splits, split_via, group_m, half_tail) pinned for this shape during the call."""
     dev = P.DeviceCase(case, *offsets)
-    dev.run(handles[(case.b_col_major, case.c_bf16)], variant)
+    g = handles[(case.b_col_major, case.c_bf16)]
+    shape = (dev.a.ptr, dev.b.ptr, dev.c.ptr, case.M, case.N, case.K, case.lda, case.ldb, case.ldc)
+    if pin is not None:
+        from paper_2605_28213_b200 import binding as kb
+        g.set_plan(kb.klineage_gemm_plan_t(*pin), *shape)
+    try:
+        dev.run(g, variant)
+    finally:
+        if pin is not None:
+            g.set_plan(None, *shape)
     vals, bits = dev.result()
     if C_ref is None:
         rows = np.arange(case.M)
@@ -181,6 +191,7 @@ def test_tcgen05_skinny_modes(handles, col):
 
 
 # ------------------------------------------------------------------ CTA-pair form of the top rung
+PAIR = (2, 1, 0, 0, 0)      # launch plan: the CTA-pair kernel, no K split
 @pytest.mark.parametrize("col", [False, True], ids=["Brow", "Bcol"])
 def test_tcgen05_cta_pair_ragged(handles, col):
     """Large aligned shapes run on tcgen05.mma.cta_group::2 (512 x 256 pair tiles); tails in M, N and K."""
@@ -191,14 +202,16 @@ def test_tcgen05_cta_pair_ragged(handles, col):
                              name="pair-ragged-row-end")
         rows = P.sample_rows(case.M)
         C_ref, S = P.oracle_rows(case, rows)
-        run_and_check(handles, case, 4, C_ref, S, rows, exact=True)
-    for idx, (M, N, K) in enumerate([(5000, 5200, 1000), (4608, 4352, 72)]):
+        run_and_check(handles, case, 4, C_ref, S, rows, exact=True, pin=PAIR)
+        assert (handles[(col, bf)].last_kernel_id() - 400) & 32
+    # (the pair kernel is pinned: for short K the dispatch prefers the single-CTA kernel, whose epilogue is hidden)
+    for idx, (M, N, K) in enumerate([(5000, 5200, 1000), (4608, 4352, 72), (4200, 4352, 136)]):
         for bf in (False, True):
             case = gen.make_case(M, N, K, seed=60 + idx, dist_a="integer", dist_b="integer", b_col_major=col,
                                  c_bf16=bf, name=f"pair{M}x{N}x{K}-int")
             rows = P.sample_rows(M)
             C_ref, S = P.oracle_rows(case, rows)
-            vals, _ = run_and_check(handles, case, 4, C_ref, S, rows, exact=True)
+            vals, _ = run_and_check(handles, case, 4, C_ref, S, rows, exact=True, pin=PAIR)
             assert (handles[(col, bf)].last_kernel_id() - 400) & 32, "expected the CTA-pair kernel"
             if not bf:
                 assert P.integer_checksums_match(case, vals)
@@ -206,7 +219,20 @@ def test_tcgen05_cta_pair_ragged(handles, col):
                              name=f"pair{M}x{N}x{K}")
         rows = P.sample_rows(M)
         C_ref, S = P.oracle_rows(case, rows)
-        run_and_check(handles, case, 4, C_ref, S, rows)
+        run_and_check(handles, case, 4, C_ref, S, rows, pin=PAIR)
+
+
+def test_dispatch_between_the_two_kernels(handles):
+    """Long K and enough 512 x 256 tiles: the pair kernel; short K or few tiles: the single-CTA kernel."""
+    for (M, N, K), want_pair in (((2048, 4096, 4096), True), ((3072, 2048, 8192), True), ((2816, 2816, 2816), True),
+                                 ((2048, 2048, 2048), False), ((4608, 4352, 72), False), ((3584, 3584, 3584), False),
+                                 ((2304, 2304, 2304), False)):
+        case = gen.make_case(M, N, K, seed=70, dist_a="integer", dist_b="integer", c_bf16=True, name=f"disp{M}x{N}x{K}")
+        rows = P.sample_rows(M)[::8]
+        C_ref, S = P.oracle_rows(case, rows)
+        run_and_check(handles, case, 4, C_ref, S, rows, exact=True)
+        kid = handles[(False, True)].last_kernel_id()
+        assert bool((kid - 400) & 32) == want_pair, (M, N, K, kid)
 
 
 # ------------------------------------------------------------------ mid-size shapes: every scheduling mode of the top rung
