@@ -410,7 +410,7 @@ def lineage_table(prob_c4, kb, gen, torch, device, peaks):
                       "tflops_heuristic": c.flops / (heur_us * 1e-6) / 1e12}
     tune["note"] = "microseconds per launch in back-to-back loops of 10 launches, minimum of two passes"
     out["autotune"] = tune
-    del p3, p2k
+    del p2k
 
     out["gemm_family"] = family_table(kb, gen, torch, device, peaks, flush)
 
@@ -489,8 +489,21 @@ def lineage_table(prob_c4, kb, gen, torch, device, peaks):
         times.append(e0.elapsed_time(e1))
     med = statistics.median(times[3:])
     ctx_rows["c4_8192^3"] = {"ms_median": med, "tflops": c4.flops / (med * 1e-3) / 1e12}
+    A3, B3 = p3.A.view(bf).view(c3.M, c3.lda), p3.B.view(bf).view(c3.N, c3.ldb)        # B stored N x K: pass its transpose
+    C3 = torch.empty((c3.M, c3.N), dtype=bf, device=device)
+    times = []
+    for i in range(23):
+        flush.fill_(i)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        torch.matmul(A3, B3.t(), out=C3)
+        e1.record()
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1))
+    med = statistics.median(times[3:])
+    ctx_rows["c3_4096^3_Bcol"] = {"ms_median": med, "tflops": c3.flops / (med * 1e-3) / 1e12}
     out["context_vendor_gemm"] = ctx_rows
-    del A5, C5, C4
+    del A5, C5, C4, A3, B3, C3, p3
     # c1 and c2 are launch- and occupancy-bound (report only): back-to-back launches, operands L2-resident.
     for name in ("c1", "c2"):
         cs = gen.make_config(name, 1)
@@ -515,6 +528,25 @@ def lineage_table(prob_c4, kb, gen, torch, device, peaks):
                                       "tflops": cs.flops / (med * 1e-3) / 1e12, "kernel_id": ps.gemm.last_kernel_id()}
         out[f"{name}_{cs.M}x{cs.N}x{cs.K}"] = rows
         del ps
+        # context: the vendor library on a product of the same shape and pitches (fp32 / bf16 result as it gives it)
+        ta = torch.randn(cs.M, cs.K, device=device).to(torch.bfloat16)
+        tb = torch.randn(cs.K, cs.N, device=device).to(torch.bfloat16)
+        tc = torch.empty(cs.M, cs.N, device=device, dtype=torch.bfloat16)
+        for _ in range(3):
+            torch.matmul(ta, tb, out=tc)
+        torch.cuda.synchronize()
+        best = []
+        for _ in range(5):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(200):
+                torch.matmul(ta, tb, out=tc)
+            e1.record()
+            e1.synchronize()
+            best.append(e0.elapsed_time(e1) / 200)
+        ctx_rows[f"{name}_{cs.M}x{cs.N}x{cs.K}"] = {"us_median": statistics.median(best) * 1e3,
+                                                   "note": "bf16 output, back-to-back, L2-resident"}
+        del ta, tb, tc
     out["note"] = ("c4, c3: single launches timed with CUDA events (c3 after a 256 MiB L2 flush; c4 operands exceed "
                    "L2); c5: back-to-back launches rotating over 4 distinct weight buffers (512 MiB > L2), time per "
                    "launch; c1, c2: back-to-back launches, operands L2-resident (launch/occupancy bound, report only)")
