@@ -55,8 +55,9 @@ typedef enum {
 } klineage_ctype_t;
 
 /*
- * The lineage rungs (paper: Introduction, "tiling, shared-memory staging,
- * vectorized loads, software pipelining, or hardware intrinsics"; Table 1).
+ * The lineage rungs (paper: the Introduction's list of optimization intents -
+ * tiles, staging through shared memory, wide loads, a software pipeline, matrix
+ * instructions - and the transition vocabulary of Table 1).
  */
 typedef enum {
     KLINEAGE_NAIVE = 0,      /* K_0: one thread per C element, K-loop over global memory                     */
@@ -120,8 +121,8 @@ klineage_status_t klineage_gemm_create(klineage_gemm_t* out, const klineage_gemm
  *             ldc is never written.  A and B must not overlap C.
  *   Pointers need only element alignment (2 bytes bf16, 4 bytes fp32); wider
  *   alignment is detected per call and selects the vector / TMA sub-paths
- *   (paper, Introduction: "vectorized loads require alignment and valid tail
- *   handling").  Buffers stay owned by the caller.
+ *   (paper, Introduction: a wide load is valid only on aligned addresses and
+ *   with its tail handled).  Buffers stay owned by the caller.
  *
  * Errors: INVALID_ARG, BAD_VARIANT, UNSUPPORTED_DEVICE (variant 3, 4 or 5 on a
  * device without sm_100 TMA/tcgen05), LAUNCH.  Device-side give-ups (a bounded
@@ -331,6 +332,54 @@ klineage_status_t klineage_gemm_run_multi_dst(klineage_gemm_t h, int64_t M, int6
  * _run_grouped call on this handle enqueued (1 when a batched or grouped call took
  * its one-launch path; zero-fill launches count, repack pre-passes do not). */
 int klineage_gemm_last_launch_count(klineage_gemm_t h);
+
+/* ---------------------------------------------------------------------------
+ * The product with HOST operands: copies and kernels overlapped by the library.
+ *
+ * The paper times kernels with their operands already on the device
+ * (Evaluation, Setup); a caller whose matrices live in host memory pays the
+ * transfers as well, and a GEMM splits by rows of A and C so that they overlap
+ * the arithmetic.  klineage_gemm_run_host computes the same C = A . B as
+ * klineage_gemm_run, through the same rung kernels, with A, B and C in HOST memory:
+ *
+ *   copy stream   B (whole), then A row slab by row slab        (host -> device)
+ *   `stream`      slab i of C = slab i of A . B, on `variant`   (after its A slab landed)
+ *   store stream  slab i of C                                   (device -> host, after its kernel)
+ *
+ * so that, after B, the link carries A while earlier slabs are multiplied and
+ * their results travel back in the other direction.  Slabs are whole multiples
+ * of 128 rows, at most 16 per call.
+ *
+ *   A, B, C    HOST pointers; same shapes, pitches (elements, any value >= the
+ *              row length) and element types as in klineage_gemm_run.  Page-locked
+ *              memory makes the copies asynchronous and lets them overlap; pageable
+ *              memory is accepted and gives the same result without the overlap.
+ *              Only the M x N (M x K, ...) elements are read or written, padding
+ *              up to the pitch is not touched.  The buffers must stay valid, and A
+ *              and B unmodified, until work enqueued on `stream` after this call
+ *              has been reached (for instance until the stream is synchronised).
+ *   scratch    DEVICE memory on the handle's GPU, owned by the caller, at least
+ *              klineage_gemm_host_scratch_bytes(...) bytes, 256-byte aligned.  It
+ *              holds the device copies of A, B and C (pitches rounded up to 16
+ *              bytes, so the TMA sub-paths always apply) and may be reused by the
+ *              caller once `stream` has passed this call.
+ *   stream     work enqueued on it before the call precedes every copy, work
+ *              enqueued after the call follows the last copy back to the host.
+ *
+ * The first call on a handle creates the two internal streams and their events
+ * (no device memory); destroy releases them.  M == 0 or N == 0: OK, nothing is
+ * done.  K == 0: C_host <- 0.  Errors: as klineage_gemm_run, plus INVALID_ARG for a
+ * missing, misaligned or too small scratch and for host ranges of A or B that
+ * overlap C; LAUNCH when a copy cannot be enqueued.
+ * klineage_gemm_last_launch_count then reports the slab kernels of the call.
+ */
+size_t klineage_gemm_host_scratch_bytes(int b_layout, int c_dtype, int64_t M, int64_t N, int64_t K);
+
+klineage_status_t klineage_gemm_run_host(klineage_gemm_t h, int64_t M, int64_t N, int64_t K,
+                                         const void* A_host, int64_t lda, const void* B_host, int64_t ldb,
+                                         void* C_host, int64_t ldc,
+                                         void* scratch_device, size_t scratch_bytes,
+                                         int variant, void* stream);
 
 /* ---------------------------------------------------------------------------
  * Launch plans and the autotuner of the tcgen05 rung.

@@ -38,6 +38,7 @@ EXPORTED_SYMBOLS = (
     "klineage_gemm_run_batched", "klineage_gemm_run_grouped", "klineage_gemm_last_launch_count",
     "klineage_gemm_run_multi_dst", "klineage_conv2d_run", "klineage_conv2d_check_args",
     "klineage_gemm_plan_candidates", "klineage_gemm_set_plan", "klineage_gemm_get_plan", "klineage_gemm_autotune",
+    "klineage_gemm_host_scratch_bytes", "klineage_gemm_run_host",
 )
 
 
@@ -90,6 +91,24 @@ def klineage_gemm_run_noalloc(b_layout, c_dtype, M, N, K, A, lda, B, ldb, C, ldc
     one-stream-at-a-time rule.
     """
     return _lib.klineage_gemm_run_noalloc(b_layout, c_dtype, M, N, K, A, lda, B, ldb, C, ldc, stream)
+
+
+_lib.klineage_gemm_host_scratch_bytes.restype = ctypes.c_size_t
+_lib.klineage_gemm_host_scratch_bytes.argtypes = [_int, _int, _i64, _i64, _i64]
+_lib.klineage_gemm_run_host.restype = _int
+_lib.klineage_gemm_run_host.argtypes = [_p, _i64, _i64, _i64, _p, _i64, _p, _i64, _p, _i64, _p, ctypes.c_size_t, _int, _p]
+
+
+def klineage_gemm_host_scratch_bytes(b_layout, c_dtype, M, N, K) -> int:
+    """Device scratch (bytes) that klineage_gemm_run_host needs for this shape; 0 for an empty or invalid one."""
+    return int(_lib.klineage_gemm_host_scratch_bytes(b_layout, c_dtype, M, N, K))
+
+
+def klineage_gemm_run_host_raw(h, M, N, K, A_host, lda, B_host, ldb, C_host, ldc, scratch, scratch_bytes, variant,
+                               stream) -> int:
+    """Raw status of C = A.B with A, B, C in HOST memory (integer addresses) and a device scratch buffer."""
+    return _lib.klineage_gemm_run_host(h, M, N, K, A_host, lda, B_host, ldb, C_host, ldc, scratch, scratch_bytes,
+                                       variant, stream)
 
 
 _lib.klineage_gemm_run_addmm.restype = _int
@@ -308,6 +327,19 @@ class Gemm:
     def run(self, A, B, C, M, N, K, lda, ldb, ldc, variant, stream=None) -> None:
         klineage_gemm_run(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(C), ldc,
                           int(variant), self._stream(stream))
+
+    def host_scratch_bytes(self, M, N, K) -> int:
+        return klineage_gemm_host_scratch_bytes(KLINEAGE_B_COL_MAJOR if self.b_col_major else KLINEAGE_B_ROW_MAJOR,
+                                                KLINEAGE_C_BF16 if self.c_bf16 else KLINEAGE_C_F32, M, N, K)
+
+    def run_host(self, A_host, B_host, C_host, M, N, K, lda, ldb, ldc, scratch, scratch_bytes, variant,
+                 stream=None) -> None:
+        """A_host, B_host, C_host: CPU tensors (pinned for overlap) or integer host addresses; scratch: device."""
+        st = klineage_gemm_run_host_raw(self._h, M, N, K, self._ptr(A_host), lda, self._ptr(B_host), ldb,
+                                        self._ptr(C_host), ldc, self._ptr(scratch), int(scratch_bytes), int(variant),
+                                        self._stream(stream))
+        if st != KLINEAGE_OK:
+            raise KlineageError(st, "klineage_gemm_run_host")
 
     def run_addmm(self, A, B, bias, C, M, N, K, lda, ldb, ldc, variant, stream=None) -> None:
         st = klineage_gemm_run_addmm_raw(self._h, M, N, K, self._ptr(A), lda, self._ptr(B), ldb, self._ptr(bias),

@@ -27,6 +27,11 @@ struct klineage_gemm_s {
     std::map<PlanKey, R4Plan> plans;   // pinned by klineage_gemm_set_plan / klineage_gemm_autotune
     bool forcing = false;              // autotune in progress: run `forced` whatever is pinned
     R4Plan forced;
+    // klineage_gemm_run_host: copy streams and events, created by its first call
+    static constexpr int kMaxSlabs = 16;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_out = nullptr, ev_in[kMaxSlabs] = {}, ev_done[kMaxSlabs] = {};
+    bool pipe_ready = false;
 };
 
 namespace klin {
@@ -160,6 +165,69 @@ bool ranges_overlap(const void* a, size_t a_bytes, const void* b, size_t b_bytes
     return a0 < b0 + b_bytes && b0 < a0 + a_bytes;
 }
 
+// Device copies of host operands (klineage_gemm_run_host): pitches rounded up to 8 elements (16 bytes for bf16, 32 for
+// fp32), every matrix at a 256-byte offset of the caller's scratch.
+struct HostLayout {
+    int64_t lda2, ldb2, ldc2, b_rows, b_cols;
+    size_t off_a, off_b, off_c, total;
+};
+
+HostLayout host_layout(int b_layout, int c_dtype, int64_t M, int64_t N, int64_t K)
+{
+    HostLayout L;
+    const bool bcol = b_layout == KLINEAGE_B_COL_MAJOR;
+    const size_t celt = c_dtype == KLINEAGE_C_BF16 ? 2 : 4;
+    auto up8 = [](int64_t v) { return v > 0 ? (v + 7) & ~int64_t(7) : int64_t(8); };
+    auto up256 = [](size_t v) { return (v + 255) & ~size_t(255); };
+    L.b_rows = bcol ? N : K;
+    L.b_cols = bcol ? K : N;
+    L.lda2 = up8(K);
+    L.ldb2 = up8(L.b_cols);
+    L.ldc2 = up8(N);
+    L.off_a = 0;
+    L.off_b = up256(static_cast<size_t>(M) * L.lda2 * 2);
+    L.off_c = L.off_b + up256(static_cast<size_t>(L.b_rows) * L.ldb2 * 2);
+    L.total = L.off_c + up256(static_cast<size_t>(M) * L.ldc2 * celt);
+    return L;
+}
+
+void release_host_pipe(klineage_gemm_s* h)
+{
+    if (h->copy_in) cudaStreamDestroy(h->copy_in);
+    if (h->copy_out) cudaStreamDestroy(h->copy_out);
+    if (h->ev_start) cudaEventDestroy(h->ev_start);
+    if (h->ev_out) cudaEventDestroy(h->ev_out);
+    for (int i = 0; i < klineage_gemm_s::kMaxSlabs; ++i) {
+        if (h->ev_in[i]) cudaEventDestroy(h->ev_in[i]);
+        if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
+        h->ev_in[i] = h->ev_done[i] = nullptr;
+    }
+    h->copy_in = h->copy_out = nullptr;
+    h->ev_start = h->ev_out = nullptr;
+    h->pipe_ready = false;
+}
+
+// Streams that do not synchronise with the legacy default stream: every ordering is an explicit event.
+bool ensure_host_pipe(klineage_gemm_s* h)
+{
+    if (h->pipe_ready) return true;
+    bool ok = cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&h->ev_out, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < klineage_gemm_s::kMaxSlabs; ++i) {
+        ok = cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming) == cudaSuccess;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        release_host_pipe(h);
+        return false;
+    }
+    h->pipe_ready = true;
+    return true;
+}
+
 }  // namespace
 
 extern "C" {
@@ -228,6 +296,7 @@ klineage_status_t klineage_gemm_destroy(klineage_gemm_t h)
         if (h->ctx.workspace) cudaFree(h->ctx.workspace);
         if (h->ctx.tile_counters) cudaFree(h->ctx.tile_counters);
         if (h->status) cudaFree(h->status);
+        release_host_pipe(h);
     }
     delete h;
     return KLINEAGE_OK;
@@ -329,6 +398,94 @@ klineage_status_t klineage_gemm_run(klineage_gemm_t h, int64_t M, int64_t N, int
 {
     if (h) h->last_launches = 0;
     return run_impl(h, M, N, K, A, lda, B, ldb, nullptr, C, ldc, variant, stream);
+}
+
+size_t klineage_gemm_host_scratch_bytes(int b_layout, int c_dtype, int64_t M, int64_t N, int64_t K)
+{
+    if (b_layout != KLINEAGE_B_ROW_MAJOR && b_layout != KLINEAGE_B_COL_MAJOR) return 0;
+    if (c_dtype != KLINEAGE_C_F32 && c_dtype != KLINEAGE_C_BF16) return 0;
+    const int64_t lim = int64_t(1) << 31;
+    if (M <= 0 || N <= 0 || K < 0 || M >= lim || N >= lim || K >= lim) return 0;
+    return host_layout(b_layout, c_dtype, M, N, K).total;
+}
+
+klineage_status_t klineage_gemm_run_host(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A_host,
+                                         int64_t lda, const void* B_host, int64_t ldb, void* C_host, int64_t ldc,
+                                         void* scratch_device, size_t scratch_bytes, int variant, void* stream)
+{
+    if (!h) return KLINEAGE_ERR_INVALID_ARG;
+    h->last_launches = 0;
+    // shapes, pitches, element alignment and overlap follow the rules of the device call
+    const klineage_status_t chk =
+        klineage_gemm_check_args(h->b_layout, h->c_dtype, M, N, K, A_host, lda, B_host, ldb, C_host, ldc, variant);
+    if (chk != KLINEAGE_OK) return chk;
+    if (M == 0 || N == 0) {
+        h->last_kernel_id = -1;
+        return KLINEAGE_OK;
+    }
+    if ((variant == KLINEAGE_PIPELINED || variant == KLINEAGE_TCGEN05 || variant == KLINEAGE_MMA_SYNC) &&
+        h->ctx.cc_major != 10)
+        return KLINEAGE_ERR_UNSUPPORTED_DEVICE;
+    const HostLayout L = host_layout(h->b_layout, h->c_dtype, M, N, K);
+    if (!scratch_device || reinterpret_cast<uintptr_t>(scratch_device) % 256 || scratch_bytes < L.total)
+        return KLINEAGE_ERR_INVALID_ARG;
+
+    DeviceGuard guard(h->ctx.device);
+    if (!guard.ok) return KLINEAGE_ERR_LAUNCH;
+    if (!ensure_host_pipe(h)) return KLINEAGE_ERR_ALLOC;
+
+    const size_t celt = h->c_dtype == KLINEAGE_C_BF16 ? 2 : 4;
+    uint8_t* base = static_cast<uint8_t*>(scratch_device);
+    uint8_t *dA = base + L.off_a, *dB = base + L.off_b, *dC = base + L.off_c;
+    const uint8_t* hA = static_cast<const uint8_t*>(A_host);
+    uint8_t* hC = static_cast<uint8_t*>(C_host);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    // row slabs: multiples of 128 rows, about 512 rows each, at most kMaxSlabs
+    int64_t n_slabs = (M + 511) / 512;
+    if (n_slabs > klineage_gemm_s::kMaxSlabs) n_slabs = klineage_gemm_s::kMaxSlabs;
+    const int64_t slab = ((M + n_slabs - 1) / n_slabs + 127) / 128 * 128;
+    n_slabs = (M + slab - 1) / slab;
+
+    bool ok = cudaEventRecord(h->ev_start, s) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(h->copy_in, h->ev_start, 0) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(h->copy_out, h->ev_start, 0) == cudaSuccess;
+    if (ok && K > 0)
+        ok = cudaMemcpy2DAsync(dB, static_cast<size_t>(L.ldb2) * 2, B_host, static_cast<size_t>(ldb) * 2,
+                               static_cast<size_t>(L.b_cols) * 2, static_cast<size_t>(L.b_rows), cudaMemcpyHostToDevice,
+                               h->copy_in) == cudaSuccess;
+    klineage_status_t st = KLINEAGE_OK;
+    int launches = 0;
+    for (int64_t i = 0; ok && i < n_slabs; ++i) {
+        const int64_t r0 = i * slab, rows = (M - r0 < slab) ? M - r0 : slab;
+        uint8_t* dA_i = dA + static_cast<size_t>(r0) * L.lda2 * 2;
+        uint8_t* dC_i = dC + static_cast<size_t>(r0) * L.ldc2 * celt;
+        if (K > 0)
+            ok = cudaMemcpy2DAsync(dA_i, static_cast<size_t>(L.lda2) * 2, hA + static_cast<size_t>(r0) * lda * 2,
+                                   static_cast<size_t>(lda) * 2, static_cast<size_t>(K) * 2, static_cast<size_t>(rows),
+                                   cudaMemcpyHostToDevice, h->copy_in) == cudaSuccess;
+        ok = ok && cudaEventRecord(h->ev_in[i], h->copy_in) == cudaSuccess;
+        ok = ok && cudaStreamWaitEvent(s, h->ev_in[i], 0) == cudaSuccess;
+        if (!ok) break;
+        st = run_impl(h, rows, N, K, dA_i, L.lda2, dB, L.ldb2, nullptr, dC_i, L.ldc2, variant, stream);
+        if (st != KLINEAGE_OK) break;
+        launches = h->last_launches;
+        ok = cudaEventRecord(h->ev_done[i], s) == cudaSuccess;
+        ok = ok && cudaStreamWaitEvent(h->copy_out, h->ev_done[i], 0) == cudaSuccess;
+        ok = ok && cudaMemcpy2DAsync(hC + static_cast<size_t>(r0) * ldc * celt, static_cast<size_t>(ldc) * celt, dC_i,
+                                     static_cast<size_t>(L.ldc2) * celt, static_cast<size_t>(N) * celt,
+                                     static_cast<size_t>(rows), cudaMemcpyDeviceToHost, h->copy_out) == cudaSuccess;
+    }
+    // whatever happened, `stream` continues only after both copy streams have drained what was enqueued
+    const bool j1 = cudaEventRecord(h->ev_out, h->copy_out) == cudaSuccess && cudaStreamWaitEvent(s, h->ev_out, 0) == cudaSuccess;
+    const bool j2 = cudaEventRecord(h->ev_start, h->copy_in) == cudaSuccess && cudaStreamWaitEvent(s, h->ev_start, 0) == cudaSuccess;
+    h->last_launches = launches;
+    if (st != KLINEAGE_OK) return st;
+    if (!ok || !j1 || !j2) {
+        cudaGetLastError();
+        return KLINEAGE_ERR_LAUNCH;
+    }
+    return KLINEAGE_OK;
 }
 
 klineage_status_t klineage_gemm_run_addmm(klineage_gemm_t h, int64_t M, int64_t N, int64_t K, const void* A,

@@ -1,6 +1,6 @@
 // Rung 2 - "vectorize_global" (paper, Table 1; precondition: 128-bit aligned
-// access; Introduction: "vectorized loads require alignment and valid tail
-// handling").  Same 128 x 128 x 16 tiling as rung 1, but
+// access; Introduction: a wide load needs aligned addresses and a handled
+// tail).  Same 128 x 128 x 16 tiling as rung 1, but
 //   * A and B move in 16-byte groups of 8 bf16 whenever the operand's base
 //     and leading dimension are 16-byte aligned (checked per call, per operand);
 //     a group that crosses the M/N/K edge is loaded element by element under a

@@ -1,6 +1,6 @@
 // Rung 3 - "cp.async + pipeline" / "tma_load" (paper, Table 1; preconditions:
 // data movement is shared-memory staged, the TMA descriptor is encoded;
-// Introduction: "pipelining assumes staged data movement").
+// Introduction: a pipeline presupposes that data movement is staged).
 //
 // 128 x 128 x 32 tiles, a ring of 4 shared-memory stages holding RAW bf16, a
 // full/empty mbarrier pair per stage with phase parity.  Loads for k-block

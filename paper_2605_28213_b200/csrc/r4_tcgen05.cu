@@ -1,6 +1,6 @@
 // Rung 4 - the expert kernel K_n of the lineage: "warp_specialize" plus matrix
-// intrinsics (paper, Table 1; Introduction: "matrix intrinsics require
-// compatible tile shapes, layouts, and hardware support").  On sm_100a the
+// intrinsics (paper, Table 1; Introduction: a matrix instruction is valid only
+// for tile shapes, layouts and hardware that fit it).  On sm_100a the
 // intrinsic is tcgen05.mma with the accumulator in tensor memory (TMEM); the
 // table's wgmma does not exist on this architecture.
 //

@@ -29,8 +29,8 @@
 // cluster-wide broadcast form.  All waits are bounded; both CTAs pass a cluster barrier
 // before exit so that no remote arrive can hit shared memory of a finished CTA.
 //
-// Preconditions (paper, Introduction: intrinsics "require compatible tile
-// shapes, layouts, and hardware support"): A, B TMA-loadable (16-byte aligned
+// Preconditions (paper, Introduction: a matrix instruction is valid only for
+// tile shapes, layouts and hardware that fit it): A, B TMA-loadable (16-byte aligned
 // base and pitch), no K split, not the skinny orientation.  Everything else
 // runs on the single-CTA kernel of r4_tcgen05.cu.
 #include "common.cuh"

@@ -154,3 +154,28 @@ def test_null_handles_are_refused_everywhere(kb):
     assert kb.klineage_gemm_set_plan_raw(None, 8, 8, 8, P, 8, P * 2, 8, P * 3, 8, None) == kb.KLINEAGE_ERR_INVALID_ARG
     assert kb._lib.klineage_gemm_last_launch_count(None) == 0
     assert kb.klineage_gemm_last_kernel_id(None) == -1
+
+
+def test_host_scratch_bytes_follows_the_documented_layout(kb):
+    """Three matrices, pitches rounded up to 8 elements, each at a 256-byte offset; 0 for empty or invalid shapes."""
+    def expect(col, bf16, M, N, K):
+        up8 = lambda v: (v + 7) // 8 * 8 if v > 0 else 8
+        up256 = lambda v: (v + 255) // 256 * 256
+        b_rows, b_cols = (N, K) if col else (K, N)
+        return up256(M * up8(K) * 2) + up256(b_rows * up8(b_cols) * 2) + up256(M * up8(N) * (2 if bf16 else 4))
+
+    for col in (False, True):
+        for bf16 in (False, True):
+            for (M, N, K) in ((1000, 1001, 999), (1, 1, 1), (8192, 8192, 8192), (16, 8192, 8192), (70, 33, 0)):
+                got = kb.klineage_gemm_host_scratch_bytes(int(col), int(bf16), M, N, K)
+                assert got == expect(col, bf16, M, N, K), (col, bf16, M, N, K, got)
+    assert kb.klineage_gemm_host_scratch_bytes(0, 0, 1000, 1001, 999) == 2000128 + 2014208 + 4032000   # worked by hand
+    assert kb.klineage_gemm_host_scratch_bytes(0, 0, 0, 8, 8) == 0
+    assert kb.klineage_gemm_host_scratch_bytes(0, 0, 8, 0, 8) == 0
+    assert kb.klineage_gemm_host_scratch_bytes(0, 0, 8, 8, -1) == 0
+    assert kb.klineage_gemm_host_scratch_bytes(2, 0, 8, 8, 8) == 0
+    assert kb.klineage_gemm_host_scratch_bytes(0, 5, 8, 8, 8) == 0
+    assert kb.klineage_gemm_host_scratch_bytes(0, 0, 1 << 31, 8, 8) == 0
+    P = 0x100000
+    assert kb.klineage_gemm_run_host_raw(None, 8, 8, 8, P, 8, P * 2, 8, P * 3, 8, P * 4, 1 << 20, 4, None) == \
+        kb.KLINEAGE_ERR_INVALID_ARG

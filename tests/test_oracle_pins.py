@@ -1,7 +1,7 @@
 """Pins for the CPU oracle: each test fixes it to something other than itself.
 
-The paper (Evaluation, Setup) says only that correctness is checked "at three
-random seeds" against a vendor reference and prints no GEMM values, so the
+The paper (Evaluation, Setup) says only that correctness is checked with three
+random seeds against a vendor reference and prints no GEMM values, so the
 pins are mathematics: exact rational arithmetic, closed forms, invariants, a
 hand-worked example and library routines used as cross-checks.
 """

@@ -2,7 +2,7 @@
 
 Bit-exact on integer-valued inputs; within K * 2^-23 * (|A|.|B|)_ij on random
 bf16 inputs (fp32 C), widened by one bf16 rounding for bf16 C.  The paper's own
-gate is "correctness at three random seeds" (Evaluation, Setup); seeds 1..3 are
+gate is a correctness check with three random seeds (Evaluation, Setup); seeds 1..3 are
 used on the small configurations.
 """
 import numpy as np
