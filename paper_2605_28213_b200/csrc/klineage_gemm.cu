@@ -191,6 +191,15 @@ HostLayout host_layout(int b_layout, int c_dtype, int64_t M, int64_t N, int64_t 
     return L;
 }
 
+// A pitched copy; one linear copy when both sides are dense (the copy engines then see a single long transfer).
+cudaError_t copy_rows(void* dst, size_t dpitch, const void* src, size_t spitch, size_t width, size_t rows,
+                      cudaMemcpyKind kind, cudaStream_t s)
+{
+    if (rows == 0 || width == 0) return cudaSuccess;
+    if (dpitch == width && spitch == width) return cudaMemcpyAsync(dst, src, width * rows, kind, s);
+    return cudaMemcpy2DAsync(dst, dpitch, src, spitch, width, rows, kind, s);
+}
+
 void release_host_pipe(klineage_gemm_s* h)
 {
     if (h->copy_in) cudaStreamDestroy(h->copy_in);
@@ -451,9 +460,9 @@ klineage_status_t klineage_gemm_run_host(klineage_gemm_t h, int64_t M, int64_t N
     ok = ok && cudaStreamWaitEvent(h->copy_in, h->ev_start, 0) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(h->copy_out, h->ev_start, 0) == cudaSuccess;
     if (ok && K > 0)
-        ok = cudaMemcpy2DAsync(dB, static_cast<size_t>(L.ldb2) * 2, B_host, static_cast<size_t>(ldb) * 2,
-                               static_cast<size_t>(L.b_cols) * 2, static_cast<size_t>(L.b_rows), cudaMemcpyHostToDevice,
-                               h->copy_in) == cudaSuccess;
+        ok = copy_rows(dB, static_cast<size_t>(L.ldb2) * 2, B_host, static_cast<size_t>(ldb) * 2,
+                       static_cast<size_t>(L.b_cols) * 2, static_cast<size_t>(L.b_rows), cudaMemcpyHostToDevice,
+                       h->copy_in) == cudaSuccess;
     klineage_status_t st = KLINEAGE_OK;
     int launches = 0;
     for (int64_t i = 0; ok && i < n_slabs; ++i) {
@@ -461,9 +470,9 @@ klineage_status_t klineage_gemm_run_host(klineage_gemm_t h, int64_t M, int64_t N
         uint8_t* dA_i = dA + static_cast<size_t>(r0) * L.lda2 * 2;
         uint8_t* dC_i = dC + static_cast<size_t>(r0) * L.ldc2 * celt;
         if (K > 0)
-            ok = cudaMemcpy2DAsync(dA_i, static_cast<size_t>(L.lda2) * 2, hA + static_cast<size_t>(r0) * lda * 2,
-                                   static_cast<size_t>(lda) * 2, static_cast<size_t>(K) * 2, static_cast<size_t>(rows),
-                                   cudaMemcpyHostToDevice, h->copy_in) == cudaSuccess;
+            ok = copy_rows(dA_i, static_cast<size_t>(L.lda2) * 2, hA + static_cast<size_t>(r0) * lda * 2,
+                           static_cast<size_t>(lda) * 2, static_cast<size_t>(K) * 2, static_cast<size_t>(rows),
+                           cudaMemcpyHostToDevice, h->copy_in) == cudaSuccess;
         ok = ok && cudaEventRecord(h->ev_in[i], h->copy_in) == cudaSuccess;
         ok = ok && cudaStreamWaitEvent(s, h->ev_in[i], 0) == cudaSuccess;
         if (!ok) break;
@@ -472,9 +481,9 @@ klineage_status_t klineage_gemm_run_host(klineage_gemm_t h, int64_t M, int64_t N
         launches = h->last_launches;
         ok = cudaEventRecord(h->ev_done[i], s) == cudaSuccess;
         ok = ok && cudaStreamWaitEvent(h->copy_out, h->ev_done[i], 0) == cudaSuccess;
-        ok = ok && cudaMemcpy2DAsync(hC + static_cast<size_t>(r0) * ldc * celt, static_cast<size_t>(ldc) * celt, dC_i,
-                                     static_cast<size_t>(L.ldc2) * celt, static_cast<size_t>(N) * celt,
-                                     static_cast<size_t>(rows), cudaMemcpyDeviceToHost, h->copy_out) == cudaSuccess;
+        ok = ok && copy_rows(hC + static_cast<size_t>(r0) * ldc * celt, static_cast<size_t>(ldc) * celt, dC_i,
+                             static_cast<size_t>(L.ldc2) * celt, static_cast<size_t>(N) * celt,
+                             static_cast<size_t>(rows), cudaMemcpyDeviceToHost, h->copy_out) == cudaSuccess;
     }
     // whatever happened, `stream` continues only after both copy streams have drained what was enqueued
     const bool j1 = cudaEventRecord(h->ev_out, h->copy_out) == cudaSuccess && cudaStreamWaitEvent(s, h->ev_out, 0) == cudaSuccess;
