@@ -63,6 +63,25 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     return false;
 }
 
+// The same wait on a barrier given by its shared-window address (role loops that step through a ring keep the
+// address in a register instead of converting a pointer every iteration).
+__device__ __forceinline__ bool mbar_wait_addr(uint32_t bar_addr, uint32_t parity, volatile uint32_t* abort_flag)
+{
+    for (uint32_t i = 0; i < kMbarPollLimit; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.b32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar_addr), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if ((i & 1023u) == 1023u && *abort_flag) return false;
+    }
+    return false;
+}
+
 // ------------------------------------------------------------------- fences
 // Orders generic-proxy shared-memory writes before async-proxy reads (TMA
 // store, tcgen05.mma operand fetch).
@@ -101,6 +120,26 @@ __device__ __forceinline__ void tma_load_4d(void* smem_dst, const void* tmap, in
         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(c3),
         "r"(smem_u32(bar))
+        : "memory");
+}
+// The same loads and the expect-tx arrive with shared-window addresses (lean producer loops).
+__device__ __forceinline__ void mbar_arrive_expect_tx_addr(uint32_t bar_addr, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_addr(uint32_t smem_dst, const void* tmap, int x, int y, uint32_t bar_addr)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar_addr)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_addr(uint32_t smem_dst, const void* tmap, int c0, int c1, int c2, int c3,
+                                                 uint32_t bar_addr)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar_addr)
         : "memory");
 }
 // 3-D tiled store shared -> global (bulk group).  Coordinates must be >= 0.
@@ -233,6 +272,10 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
+}
+__device__ __forceinline__ void umma_commit_addr(uint32_t bar_addr)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_addr) : "memory");
 }
 // Each thread of the warp reads 32 consecutive fp32 columns of ITS lane
 // (lane = TMEM lane base of the warp's quarter + lane id).

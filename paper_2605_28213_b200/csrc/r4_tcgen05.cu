@@ -51,6 +51,12 @@ constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
 constexpr int kABytes = BM * BK * 2;              // 16 KiB
 constexpr int kBBytes = BN * BK * 2;              // 32 KiB
 constexpr int kStageBytes = kABytes + kBBytes;    // 48 KiB
+// Conv2d by TMA with at most 128 filters: a stage is a 16 KiB patch box plus a 16 KiB filter block, so the ring
+// area holds six stages instead of four (their barriers live in the grouped schedule's space, unused in that mode).
+constexpr int kConvFilterBytes = (BN / 2) * BK * 2;                                  // 16 KiB
+constexpr int kConvStageBytes = kABytes + kConvFilterBytes;                          // 32 KiB
+constexpr int kConvStages = 6;
+static_assert(kConvStages * kConvStageBytes <= STAGES * kStageBytes, "conv ring exceeds the ring area");
 constexpr int kEpiBufBytes = 32 * 128;            // one 32-row x 128-byte staging block
 constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;   // 4 warps x 2 buffers
 constexpr int kBarBytes = 1536;                   // barriers, TMEM slot, abort flag, grouped schedule (<= 257 ints)
@@ -92,6 +98,7 @@ struct R4Params {
     ConvGeom conv;
     int conv_fast;          // 1: C % 8 == 0 and x 16-byte aligned - an 8-k chunk is one 16-byte load
     int half_only;          // every unit is the first 128-column half of its tile (problems with N <= 128)
+    int conv_ring6;         // Conv2d by TMA, F <= 128: six 32 KiB stages with their own barriers and a lean producer loop
     int conv_b_tma;         // MODE 4: the weights come by TMA (warp 0), only the patches are gathered
     int conv_b_rows;        // rows of the weight box (128 with half_only, else 256)
     int conv_patch;         // patches by TMA: row tile t = 8 x 16 output patch (t % tq, (t / tq) % tp) of image t / (tq tp)
@@ -228,6 +235,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile uint32_t* abort_flag = tmem_slot + 1;   // [0] raised on give-up, [1] stays 0
     int* gstart = reinterpret_cast<int*>(const_cast<uint32_t*>(abort_flag) + 2);   // MODE 2: first tile of every group
+    // MODE 4 with the six-stage ring: its full / empty barriers (the group table's space is free there)
+    uint64_t* cfull = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(gstart) + 7) & ~uintptr_t(7));
+    uint64_t* cempty = cfull + kConvStages;
+    const bool ring6 = MODE == 4 && !GENERIC && p.conv_ring6;
     int group_hint = 0;     // MODE 2: a thread's units come in increasing order; its group search resumes here
     // One unit of the schedule for this thread's role.
     auto unit_of = [&](int64_t u) {
@@ -354,6 +365,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             ptx::mbar_init(&acc_full[b], 1);
             ptx::mbar_init(&acc_empty[b], 4);
         }
+        if (ring6)
+            for (int i = 0; i < 2 * kConvStages; ++i) ptx::mbar_init(&cfull[i], 1);
         abort_flag[0] = 0;
         abort_flag[1] = 0;
         ptx::fence_barrier_init();
@@ -396,7 +409,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             if (!GENERIC && MODE != 2) {
                 // The first ring fill needs nothing from the other warps: start it before the
                 // set-up barrier so that TMEM allocation hides behind the first loads' latency.
-                produce(STAGES);
+                if (!ring6) produce(STAGES);
             }
         }
         if (blockIdx.x == 0) g.status[1] = p.kid;
@@ -425,7 +438,50 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
-        if (!GENERIC && lane == 0) {
+        if (ring6 && lane == 0) {
+            // Conv2d, six-stage ring.  With k-blocks this short (four N = 128 MMAs) the producer's own instruction
+            // stream bounds the kernel, so this loop carries everything it needs instead of deriving it: stage
+            // addresses and parity, the tap (fr, fs) and channel group of the k-block, all by increments.
+            const uint32_t ring0 = ptx::smem_u32(smem), cfull0 = ptx::smem_u32(cfull), cempty0 = ptx::smem_u32(cempty);
+            const int cpb = p.conv.C >> 6, fS = p.conv.S, nkb = p.nkb;
+            uint32_t st = 0, ph = 1;                  // stage and the parity its "empty" barrier is waited with
+            while (prod.live) {
+                const int cw = prod.cw, ch = prod.ch, cn = prod.cn, n0 = prod.n0;
+                int cg = 0, fs = 0, fr = 0;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!ptx::mbar_wait_addr(cempty0 + 8 * st, ph, abort_flag)) {
+                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x460u | st);
+                        abort_flag[0] = 1;
+                        prod.live = false;
+                        break;
+                    }
+                    const uint32_t dst = ring0 + st * kConvStageBytes, bar = cfull0 + 8 * st;
+                    ptx::mbar_arrive_expect_tx_addr(bar, static_cast<uint32_t>(kConvStageBytes));
+                    ptx::tma_load_4d_addr(dst, &map_a, cg * 64, cw + fs, ch + fr, cn, bar);
+                    ptx::tma_load_2d_addr(dst + kABytes, &map_b, kb * BK, n0, bar);
+                    if (++cg == cpb) {
+                        cg = 0;
+                        if (++fs == fS) {
+                            fs = 0;
+                            ++fr;
+                        }
+                    }
+                    if (++st == kConvStages) {
+                        st = 0;
+                        ph ^= 1u;
+                    }
+                    ++prod.it;
+                }
+                if (!prod.live) break;
+                prod.u += gridDim.x;
+                prod_enter_unit();
+            }
+            // Drain: every load issued must have landed before shared memory is released.
+            const uint32_t it = prod.it;
+            const uint32_t first = it > kConvStages ? it - kConvStages : 0;
+            for (uint32_t j = first; j < it; ++j)
+                ptx::mbar_wait(&cfull[j % kConvStages], (j / kConvStages) & 1, abort_flag + 1);
+        } else if (!GENERIC && lane == 0) {
             if (MODE == 2) prod_enter_unit();      // (its group search reads the table the other warps just staged)
             produce(0xFFFFFFFFu);
             // Drain: every load issued must have landed before shared memory is released.
@@ -457,8 +513,21 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            uint32_t it = 0, t = 0;
+            uint32_t t = 0;
             bool ok = true;
+            // The ring position (stage s, phase ph) is carried instead of derived, barriers are addressed by their
+            // shared-window address, and a stage's descriptors are the first stage's plus s * (stage bytes >> 4)
+            // in the 14-bit start-address field (the ring ends below 256 KiB: no carry out of the field).
+            // (Measured: the length of this instruction stream does not bound the kernel - trimming it changed no
+            // timing, and releasing stages in pairs to halve the commits was slower, because the ring got shallower.)
+            uint32_t s = 0, ph = 0;
+            const uint32_t full0 = ptx::smem_u32(ring6 ? cfull : full), empty0 = ptx::smem_u32(ring6 ? cempty : empty);
+            const uint32_t n_stages = ring6 ? kConvStages : STAGES;
+            const uint32_t stage_step = (ring6 ? kConvStageBytes : kStageBytes) >> 4;
+            const uint64_t a_desc0 = make_desc(ptx::smem_u32(smem), 16, 1024);
+            const uint32_t a_lo0 = static_cast<uint32_t>(a_desc0), a_hi = static_cast<uint32_t>(a_desc0 >> 32);
+            const uint32_t b_lo0 = (((ptx::smem_u32(smem) + kABytes) >> 4) & 0x3FFFu) | (p.b_desc_lbo << 16);
+            const uint32_t b_hi = p.b_desc_hi, kstep = p.b_kstep;
             for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++t) {
                 const Unit x = unit_of(u);
                 const int kb0 = x.kb0, kb1 = x.kb1;
@@ -471,37 +540,38 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 }
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    if (!ptx::mbar_wait(&full[s], (it / STAGES) & 1, abort_flag)) {
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    if (!ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag)) {
                         report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x420u | s);
                         abort_flag[0] = 1;
                         ok = false;
                         break;
                     }
                     ptx::tc_fence_after_sync();
-                    const uint32_t sa = ptx::smem_u32(smem + s * kStageBytes);
-                    const uint32_t sb = sa + kABytes;
-                    const uint64_t a_desc = make_desc(sa, 16, 1024);
-                    const uint64_t b_desc = (static_cast<uint64_t>(p.b_desc_hi) << 32) |
-                                            (((sb >> 4) & 0x3FFFu) | (p.b_desc_lbo << 16));
+                    const uint32_t a_lo = a_lo0 + s * stage_step, b_lo = b_lo0 + s * stage_step;
 #pragma unroll
                     for (int k4 = 0; k4 < BK / 16; ++k4) {
                         // K-major operand: +32 bytes per 16 k inside the 128-byte swizzle row.
                         const uint32_t acc = (kb > kb0 || k4 > 0) ? 1u : 0u;
+                        const uint64_t a_desc = (static_cast<uint64_t>(a_hi) << 32) | (a_lo + 2u * k4);
                         if (SWAP) {
                             // weights are the 128-row operand (two halves of the tile's 256 columns,
                             // 16 KiB apart in the stage), activations the N operand
 #pragma unroll
                             for (int h = 0; h < 2; ++h)
-                                ptx::umma_f16(d_tmem + h * 128, b_desc + static_cast<uint64_t>(h * (16384 >> 4) + k4 * p.b_kstep),
-                                              a_desc + static_cast<uint64_t>(k4 * 2), idesc, acc);
+                                ptx::umma_f16(d_tmem + h * 128,
+                                              (static_cast<uint64_t>(b_hi) << 32) | (b_lo + h * (16384u >> 4) + k4 * kstep),
+                                              a_desc, idesc, acc);
                         } else {
-                            ptx::umma_f16(d_tmem, a_desc + static_cast<uint64_t>(k4 * 2),
-                                          b_desc + static_cast<uint64_t>(k4 * p.b_kstep), idesc, acc);
+                            ptx::umma_f16(d_tmem, a_desc, (static_cast<uint64_t>(b_hi) << 32) | (b_lo + k4 * kstep), idesc,
+                                          acc);
                         }
                     }
-                    ptx::umma_commit(&empty[s]);
+                    ptx::umma_commit_addr(empty0 + 8 * s);
+                    if (++s == n_stages) {
+                        s = 0;
+                        ph ^= 1u;
+                    }
                 }
                 if (ok) ptx::umma_commit(&acc_full[buf]);
             }
@@ -1674,6 +1744,7 @@ cudaError_t launch_r4_conv2d(const GemmArgs& g, const ConvGeom& geom, RunContext
         p.conv_tp = tp;
         p.tiles_m = static_cast<int>(n_img * tp * tq);
         p.stage_tx = kABytes + static_cast<uint32_t>(p.conv_b_rows) * 128u;
+        p.conv_ring6 = p.half_only;         // 16 KiB filter blocks: six stages fit where four full ones do
         unsigned pgrid;
         if (p.half_only) {
             p.full_units = 0;
