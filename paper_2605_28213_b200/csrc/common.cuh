@@ -48,6 +48,7 @@ enum KernelId : int {
     kIdConvNaive = 600,       // direct convolution, one thread per output
     kIdConvTcgen05 = 700,     // implicit GEMM on the tcgen05 rung, patches by TMA; + 4 patches gathered by producer threads,
                               // + 1 gathered element by element (C % 8 != 0 or unaligned x), + 2 direct epilogue
+                              // 708: transposed orientation (F <= 128: filters as the 128-row operand, two patch tiles per unit)
     kIdZeroFill = 900,
 };
 

@@ -99,6 +99,9 @@ struct R4Params {
     int conv_fast;          // 1: C % 8 == 0 and x 16-byte aligned - an 8-k chunk is one 16-byte load
     int half_only;          // every unit is the first 128-column half of its tile (problems with N <= 128)
     int conv_ring6;         // Conv2d by TMA, F <= 128: six 32 KiB stages with their own barriers and a lean producer loop
+    int conv_t;             // Conv2d by TMA, F <= 128, transposed: filters are the 128-row MMA operand, a unit is TWO patch
+                            // tiles (256 pixels as the N operand: full-width MMAs), the epilogue stores y transposed
+    int conv_nimg;          // images (conv_t: a unit's second patch tile may lie past the last image)
     int conv_b_tma;         // MODE 4: the weights come by TMA (warp 0), only the patches are gathered
     int conv_b_rows;        // rows of the weight box (128 with half_only, else 256)
     int conv_patch;         // patches by TMA: row tile t = 8 x 16 output patch (t % tq, (t / tq) % tp) of image t / (tq tp)
@@ -409,7 +412,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             if (!GENERIC && MODE != 2) {
                 // The first ring fill needs nothing from the other warps: start it before the
                 // set-up barrier so that TMEM allocation hides behind the first loads' latency.
-                if (!ring6) produce(STAGES);
+                if (!ring6 && !(MODE == 4 && p.conv_t)) produce(STAGES);
             }
         }
         if (blockIdx.x == 0) g.status[1] = p.kid;
@@ -438,7 +441,57 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
-        if (ring6 && lane == 0) {
+        if (MODE == 4 && !GENERIC && p.conv_t && lane == 0) {
+            // Conv2d, transposed orientation: per k-block the filter block goes to the 16 KiB slot of the 128-row
+            // operand and the patch boxes of the unit's two patch tiles to the two halves of the 256-row slot
+            // (a tile past the last image reads zeros: out-of-range coordinates).  Lean loop as below.
+            const uint32_t ring0 = ptx::smem_u32(smem), full0 = ptx::smem_u32(full), empty0 = ptx::smem_u32(empty);
+            const int cpb = p.conv.C >> 6, fS = p.conv.S, nkb = p.nkb, tq = p.conv_tq, tp = p.conv_tp;
+            uint32_t st = 0, ph = 1;
+            while (prod.live) {
+                int cw[2], ch[2], cn[2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int t = 2 * (prod.m0 / BM) + h;
+                    const int qt = t % tq, u2 = t / tq;
+                    cw[h] = qt * 16 - p.conv.pad_w;
+                    ch[h] = (u2 % tp) * 8 - p.conv.pad_h;
+                    cn[h] = u2 / tp;
+                }
+                int cg = 0, fs = 0, fr = 0;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!ptx::mbar_wait_addr(empty0 + 8 * st, ph, abort_flag)) {
+                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x470u | st);
+                        abort_flag[0] = 1;
+                        prod.live = false;
+                        break;
+                    }
+                    const uint32_t dst = ring0 + st * kStageBytes, bar = full0 + 8 * st;
+                    ptx::mbar_arrive_expect_tx_addr(bar, static_cast<uint32_t>(kStageBytes));
+                    ptx::tma_load_2d_addr(dst, &map_b, kb * BK, 0, bar);
+                    ptx::tma_load_4d_addr(dst + kABytes, &map_a, cg * 64, cw[0] + fs, ch[0] + fr, cn[0], bar);
+                    ptx::tma_load_4d_addr(dst + kABytes + kABytes, &map_a, cg * 64, cw[1] + fs, ch[1] + fr, cn[1], bar);
+                    if (++cg == cpb) {
+                        cg = 0;
+                        if (++fs == fS) {
+                            fs = 0;
+                            ++fr;
+                        }
+                    }
+                    if (++st == STAGES) {
+                        st = 0;
+                        ph ^= 1u;
+                    }
+                    ++prod.it;
+                }
+                if (!prod.live) break;
+                prod.u += gridDim.x;
+                prod_enter_unit();
+            }
+            const uint32_t it = prod.it;
+            const uint32_t first = it > STAGES ? it - STAGES : 0;
+            for (uint32_t j = first; j < it; ++j) ptx::mbar_wait(&full[j % STAGES], (j / STAGES) & 1, abort_flag + 1);
+        } else if (ring6 && lane == 0) {
             // Conv2d, six-stage ring.  With k-blocks this short (four N = 128 MMAs) the producer's own instruction
             // stream bounds the kernel, so this loop carries everything it needs instead of deriving it: stage
             // addresses and parity, the tap (fr, fs) and channel group of the k-block, all by increments.
@@ -696,6 +749,48 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         }
                     }
                 }
+                continue;
+            }
+            if (MODE == 4 && !GENERIC && p.conv_t) {
+                // Transposed Conv2d tile: TMEM lane = filter, column = pixel (128 per patch tile, 16 per patch row).
+                // A warp owns 32 filters: per step it stages 64 pixels x 32 filters (64-byte rows, its private 4 KiB
+                // block) and stores them as ONE 4-D box of y (32 filters x 16 x 4 pixels, clipped at the image).
+                const bool f_live = q * 32 < g.N;                    // (warp-uniform) filters of this warp exist
+#pragma unroll 1
+                for (int hc = 0; hc < 4; ++hc) {                     // (patch tile h, 4-row half c)
+                    const int h = hc >> 1, c = hc & 1;
+                    const int tt = 2 * (m0 / BM) + h;
+                    const int qt = tt % p.conv_tq, u2 = tt / p.conv_tq;
+                    const int cq0 = qt * 16, cp0 = (u2 % p.conv_tp) * 8 + c * 4, cimg = u2 / p.conv_tp;
+                    if (!f_live || cimg >= p.conv_nimg || cp0 >= p.conv.P) continue;
+                    uint32_t v[32], v2[32];
+                    const uint32_t taddr = tmem_base + buf * BN + h * 128 + c * 64 + (static_cast<uint32_t>(q * 32) << 16);
+                    ptx::tmem_ld_32x32b_x32(taddr, v);
+                    ptx::tmem_ld_32x32b_x32(taddr + 32, v2);
+                    uint8_t* b = stg + (nstaged++ & 1) * kEpiBufBytes;
+                    if (lane == 0) ptx::tma_store_wait_read<1>();    // the store that last read this block
+                    __syncwarp();
+                    ptx::tmem_ld_wait();
+                    uint16_t* row = reinterpret_cast<uint16_t*>(b) + lane;     // [pixel][32 filters]
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        const uint32_t w0 = pack_out2(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), g.f16);
+                        const uint32_t w1 = pack_out2(__uint_as_float(v2[j]), __uint_as_float(v2[j + 1]), g.f16);
+                        row[j * 32] = static_cast<uint16_t>(w0 & 0xFFFFu);
+                        row[(j + 1) * 32] = static_cast<uint16_t>(w0 >> 16);
+                        row[(j + 32) * 32] = static_cast<uint16_t>(w1 & 0xFFFFu);
+                        row[(j + 33) * 32] = static_cast<uint16_t>(w1 >> 16);
+                    }
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::tma_store_4d(&map_c, q * 32, cq0, cp0, cimg, b);
+                        ptx::tma_store_commit();
+                    }
+                }
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
                 continue;
             }
             const int row0 = m0 + q * 32;
@@ -1699,14 +1794,9 @@ cudaError_t launch_r4_conv2d(const GemmArgs& g, const ConvGeom& geom, RunContext
                        : 0;
     const int celt = g.c_bf16 ? 2 : 4;
     p.epi_tma = (ctx.encode_tiled && c_store_by_tma(g)) ? 1 : 0;
-    CUtensorMap none, mc;
+    CUtensorMap none, mc;          // (every tensor map is encoded only on the path that uses it: an encode costs ~1 us of host time)
     memset(&none, 0, sizeof none);
     memset(&mc, 0, sizeof mc);
-    if (p.epi_tma &&
-        !encode_map_2d(ctx, &mc, g.c_bf16 ? (g.f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16)
-                                          : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
-                       g.C, g.N, g.M, g.ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B))
-        return cudaErrorInvalidValue;
     const int64_t tiles = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
     if (tiles > 0x3FFFFFFFll) return cudaErrorInvalidValue;
     unsigned grid;
@@ -1729,10 +1819,21 @@ cudaError_t launch_r4_conv2d(const GemmArgs& g, const ConvGeom& geom, RunContext
                      patch_tiles < 0x3FFFFFFFll / BM &&
                      encode_map_nhwc(ctx, &mx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, g.A, geom.C, geom.W, geom.H,
                                      static_cast<uint64_t>(n_img), 64, 16, 8, 2, CU_TENSOR_MAP_SWIZZLE_128B);
-    if (patch_tma && p.epi_tma)     // y as a 4-D tensor (F, Q, P, N): a warp stores 2 patch rows x 16 pixels per box
+    CUtensorMap my;
+    memset(&my, 0, sizeof my);
+    const bool transposed = patch_tma && p.half_only && patch_tiles >= 2 && g.c_bf16 && p.epi_tma &&
+                            encode_map_nhwc(ctx, &my, g.f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                                            g.C, g.N, geom.Q, geom.P, static_cast<uint64_t>(n_img), 32, 16, 4, 2,
+                                            CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (patch_tma && p.epi_tma && !transposed)   // y as a 4-D tensor (F, Q, P, N): a warp stores 2 patch rows x 16 pixels per box
         patch_tma = encode_map_nhwc(ctx, &mc, g.c_bf16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
                                     g.C, g.N, geom.Q, geom.P, static_cast<uint64_t>(n_img), g.c_bf16 ? 64 : 32, 16, 2, celt,
                                     CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!patch_tma && p.epi_tma &&
+        !encode_map_2d(ctx, &mc, g.c_bf16 ? (g.f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16)
+                                          : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                       g.C, g.N, g.M, g.ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+        return cudaErrorInvalidValue;
     p.kid = kIdConvTcgen05 + (patch_tma ? 0 : 4) + (p.epi_tma ? 0 : 2) + (p.conv_fast ? 0 : 1);
     *kernel_id = p.kid;
     if (patch_tma) {
@@ -1745,6 +1846,25 @@ cudaError_t launch_r4_conv2d(const GemmArgs& g, const ConvGeom& geom, RunContext
         p.tiles_m = static_cast<int>(n_img * tp * tq);
         p.stage_tx = kABytes + static_cast<uint32_t>(p.conv_b_rows) * 128u;
         p.conv_ring6 = p.half_only;         // 16 KiB filter blocks: six stages fit where four full ones do
+        if (transposed) {
+            // At most 128 filters: run the product transposed (filters = the 128-row operand, two patch tiles =
+            // 256 pixels as the N operand), so that every MMA is full width; the epilogue stores y transposed.
+            const int64_t units = (patch_tiles + 1) / 2;
+            p.conv_t = 1;
+            p.conv_ring6 = 0;
+            p.conv_nimg = static_cast<int>(n_img);
+            p.half_only = 0;
+            p.epi_tma = 1;                 // (the kernel end waits for its stores; the map is this mode's own)
+            p.tiles_m = static_cast<int>(units);
+            p.tiles_n = 1;
+            p.full_units = p.total_units = units;
+            p.stage_tx = kStageBytes;
+            gp.M = static_cast<int>(units * BM);
+            p.kid = kIdConvTcgen05 + 8;
+            *kernel_id = p.kid;
+            const unsigned tgrid = static_cast<unsigned>(units < ctx.sm_count ? units : ctx.sm_count);
+            return launch<true, false, false, 4>(gp, mx, mb, my, p, tgrid, ctx.device, stream);
+        }
         unsigned pgrid;
         if (p.half_only) {
             p.full_units = 0;

@@ -85,7 +85,7 @@ def test_conv2d_matches_the_oracle(kb, variant, shape):
         for dist, exact in (("integer", True), ("normal", False)):
             c = gen.make_conv_case(N, H, W, C, F, R, S, seed=180, pad=pad, stride=stride, dist=dist, y_f16=y_f16)
             vals, bits, kid = run_conv(kb, c, variant)
-            assert kid == 600 if variant == 0 else 700 <= kid < 708, kid
+            assert kid == 600 if variant == 0 else 700 <= kid <= 708, kid
             check(c, vals, bits, exact, f"{c.name} variant {variant} f16={y_f16} {dist}")
 
 
@@ -96,7 +96,24 @@ def test_benchmark_shape_both_rungs(kb):
             vals, bits, kid = run_conv(kb, c, variant)
             check(c, vals, bits, exact, f"conv_t2 variant {variant} {dist}")
             if variant == 4:
-                assert kid == 700, kid          # patches and filters by TMA, TMA-store epilogue
+                assert kid == 708, kid          # patches and filters by TMA, transposed orientation (F <= 128)
+
+
+@pytest.mark.parametrize("shape", [(3, 8, 16, 192, 64, 1, 1, (0, 0)),       # 3 patch tiles: the last unit's second tile lies past the images
+                                   (2, 10, 26, 128, 72, 5, 3, (2, 0)),      # F = 72: the third warp's filter box is clipped, the fourth idles
+                                   (5, 20, 33, 64, 128, 3, 3, (1, 1)),      # 3 x 3 patch tiles per image, ragged in P and Q, 45 tiles
+                                   (1, 9, 16, 64, 8, 3, 3, (1, 1))],        # 8 filters; 2 patch tiles (the second: one pixel row)
+                         ids=lambda s: "x".join(map(str, s[:7])))
+def test_at_most_128_filters_run_transposed(kb, shape):
+    # fp16 y with at most 128 filters: filters are the 128-row MMA operand, a unit is two patch tiles (kernel id 708);
+    # fp32 y keeps the pixel-row orientation (700)
+    N, H, W, C, F, R, S, pad = shape
+    for y_f16, want_kid in ((True, 708), (False, 700)):
+        for dist, exact in (("integer", True), ("normal", False)):
+            c = gen.make_conv_case(N, H, W, C, F, R, S, seed=185, pad=pad, dist=dist, y_f16=y_f16)
+            vals, bits, kid = run_conv(kb, c, 4)
+            assert kid == want_kid, kid
+            check(c, vals, bits, exact, f"{c.name} f16={y_f16} {dist}")
 
 
 def test_unaligned_bases_take_the_slow_gather_and_direct_stores(kb):
