@@ -686,6 +686,44 @@ def family_table(kb, gen, torch, device, peaks, flush):
         ref = torch.nn.functional.conv2d(xt.float(), wt.float(), padding=cc.pad, stride=cc.stride).permute(0, 2, 3, 1)
         conv.run(x, w, y, cc.N, cc.H, cc.W, cc.C, cc.F, cc.R, cc.S, cc.pad, cc.stride, 4)
         row["sane_vs_torch_conv2d"] = bool(torch.allclose(y.float(), ref, rtol=2e-2, atol=2e-2))
+
+        # device-bound: 20 launches captured into a CUDA graph and replayed (in a plain loop both libraries are
+        # bound by their host path at this size), also at a larger batch of the same layer
+        def in_graph(fn):
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                for _ in range(3):
+                    fn()
+            torch.cuda.synchronize()
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr, stream=side):
+                for _ in range(20):
+                    fn()
+            gr.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                gr.replay()
+            e1.record()
+            e1.synchronize()
+            return e0.elapsed_time(e1) / 200 * 1e3
+
+        row["tcgen05"]["us_in_graph"] = in_graph(
+            lambda: conv.run(x, w, y, cc.N, cc.H, cc.W, cc.C, cc.F, cc.R, cc.S, cc.pad, cc.stride, 4))
+        row["tcgen05"]["tflops_in_graph"] = cc.flops / (row["tcgen05"]["us_in_graph"] * 1e-6) / 1e12
+        row["context_torch_conv2d_us_in_graph"] = in_graph(
+            lambda: torch.nn.functional.conv2d(xt, wt, padding=cc.pad, stride=cc.stride))
+        c64 = gen.make_conv_case(64, cc.H, cc.W, cc.C, cc.F, cc.R, cc.S, seed=1)
+        x64 = torch.from_numpy(c64.x.view("int16")).to(device)
+        y64 = torch.empty((c64.N, c64.P, c64.Q, c64.F), dtype=torch.float16, device=device)
+        x64t = x64.view(torch.float16).permute(0, 3, 1, 2)
+        us64 = in_graph(lambda: conv.run(x64, w, y64, c64.N, c64.H, c64.W, c64.C, c64.F, c64.R, c64.S, c64.pad, c64.stride, 4))
+        row["batch64_same_layer"] = {
+            "us_in_graph": us64, "tflops_in_graph": c64.flops / (us64 * 1e-6) / 1e12, "kernel_id": conv.last_kernel_id(),
+            "context_torch_conv2d_us_in_graph": in_graph(
+                lambda: torch.nn.functional.conv2d(x64t, wt, padding=cc.pad, stride=cc.stride))}
+        del x64, y64
         row["context_torch_conv2d_us_single"] = lib * 1e3
         row["algorithmic_bytes"] = int(x.numel() * 2 + w.numel() * 2 + y.numel() * 2)
         out["conv2d_n8_c64_56x56_f128_3x3_f16"] = row
