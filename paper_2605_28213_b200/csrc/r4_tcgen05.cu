@@ -874,6 +874,18 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                             }
                             ptx::tma_store_commit();
                         }
+                    } else if (partial) {
+                        __syncwarp();
+                        // K-split partial sums to the workspace (fp32 rows, 16-byte aligned): eight lanes cover a
+                        // staged 128-byte row with one 16-byte chunk each, four rows per step.
+                        for (int r4 = 0; r4 < rows; r4 += 4) {
+                            const int rr = r4 + (lane >> 3), j = lane & 7;
+                            const int col = col0 + j * 4;
+                            if (rr < rows && col < x.N)
+                                *reinterpret_cast<uint4*>(dst_f + (row0 + rr) * ld + col) =
+                                    *reinterpret_cast<const uint4*>(b + rr * 128 + ((j ^ (rr & 7)) << 4));
+                        }
+                        __syncwarp();
                     } else {
                         __syncwarp();
                         // lane l owns 32-bit word l of every staged row: coalesced 128-byte rows.
@@ -929,22 +941,79 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     __threadfence();
                     const int rows = min(32, g.M - row0);
                     const int64_t plane = static_cast<int64_t>(g.M) * p.ldw;
-                    for (int rr = 0; rr < rows; ++rr) {
-                        const int64_t row = row0 + rr;
-                        for (int cc = lane * 4; cc < BN; cc += 128) {
-                            const int col = n0 + cc;
-                            if (col >= g.N) break;
-                            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                            const float* src = p.ws + row * p.ldw + col;   // ldw % 4 == 0: 16-byte aligned
-                            for (int sp = 0; sp < p.splits; ++sp) {
-                                const float4 x = __ldcg(reinterpret_cast<const float4*>(src + sp * plane));
-                                acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
-                            }
-                            const float o[4] = {acc.x, acc.y, acc.z, acc.w};
+                    // Four rows x both 128-column passes x two splits per step: sixteen independent 16-byte loads
+                    // per lane are in flight before the first add (one load at a time made this reduce cost as
+                    // much as a hundred k-blocks).  Every element still adds its partials in split order.
+                    for (int r4 = 0; r4 < rows; r4 += 4) {
+                        float4 acc[4][2];
 #pragma unroll
-                            for (int e = 0; e < 4; ++e)
-                                if (col + e < g.N) store_c(g.C, g.c_bf16, row * g.ldc + col + e, o[e] + bias_at(g, col + e));
+                        for (int i = 0; i < 4; ++i)
+#pragma unroll
+                            for (int c = 0; c < 2; ++c) acc[i][c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        // (rows and columns past the matrix are clamped to valid addresses and never stored, the
+                        // odd last split is read twice and added once: the loads stay unconditional, so that all
+                        // sixteen are issued before the first use)
+                        const float* base[4][2];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+#pragma unroll
+                            for (int c = 0; c < 2; ++c) {
+                                const int col = min(n0 + lane * 4 + c * 128, static_cast<int>(p.ldw) - 4);
+                                base[i][c] = p.ws + (row0 + min(r4 + i, rows - 1)) * p.ldw + col;
+                            }
+                        for (int sp = 0; sp < p.splits; sp += 2) {
+                            float4 x[2][4][2];
+                            const int64_t off1 = (sp + 1 < p.splits ? sp + 1 : sp) * plane;
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                                for (int c = 0; c < 2; ++c) {
+                                    x[0][i][c] = __ldcg(reinterpret_cast<const float4*>(base[i][c] + sp * plane));
+                                    x[1][i][c] = __ldcg(reinterpret_cast<const float4*>(base[i][c] + off1));
+                                }
+                            if (sp + 1 >= p.splits) {
+#pragma unroll
+                                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                                    for (int c = 0; c < 2; ++c) x[1][i][c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            }
+#pragma unroll
+                            for (int s2 = 0; s2 < 2; ++s2)
+#pragma unroll
+                                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                                    for (int c = 0; c < 2; ++c) {
+                                        acc[i][c].x += x[s2][i][c].x;
+                                        acc[i][c].y += x[s2][i][c].y;
+                                        acc[i][c].z += x[s2][i][c].z;
+                                        acc[i][c].w += x[s2][i][c].w;
+                                    }
                         }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+#pragma unroll
+                            for (int c = 0; c < 2; ++c) {
+                                const int col = n0 + lane * 4 + c * 128;
+                                const int64_t row = row0 + r4 + i;
+                                if (r4 + i >= rows) continue;
+                                if (col >= g.N) continue;
+                                float o[4] = {acc[i][c].x, acc[i][c].y, acc[i][c].z, acc[i][c].w};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    if (col + e < g.N) o[e] += bias_at(g, col + e);
+                                const int64_t idx = row * g.ldc + col;
+                                if (col + 3 < g.N && g.c_bf16 && (reinterpret_cast<uintptr_t>(static_cast<uint16_t*>(g.C) + idx) & 7) == 0) {
+                                    *reinterpret_cast<uint2*>(static_cast<uint16_t*>(g.C) + idx) =
+                                        make_uint2(pack_bf16x2(o[0], o[1]), pack_bf16x2(o[2], o[3]));
+                                } else if (col + 3 < g.N && !g.c_bf16 &&
+                                           (reinterpret_cast<uintptr_t>(static_cast<float*>(g.C) + idx) & 15) == 0) {
+                                    *reinterpret_cast<float4*>(static_cast<float*>(g.C) + idx) = make_float4(o[0], o[1], o[2], o[3]);
+                                } else {
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e)
+                                        if (col + e < g.N) store_c(g.C, g.c_bf16, idx + e, o[e]);
+                                }
+                            }
                     }
                     __syncwarp();
                     if (lane == 0) *cnt = 0;   // ready for the next launch
