@@ -224,6 +224,12 @@ __device__ __forceinline__ void cluster_arrive_release()
 {
     asm volatile("barrier.cluster.arrive.release;" ::: "memory");
 }
+// The arrive of a kernel's FIRST cluster barrier, which only tells the peers that this CTA runs (its shared memory
+// exists): there are no earlier writes to publish, so the arrive need not be a release.
+__device__ __forceinline__ void cluster_arrive_relaxed()
+{
+    asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory");
+}
 __device__ __forceinline__ void cluster_wait_acquire()
 {
     asm volatile("barrier.cluster.wait.acquire;" ::: "memory");

@@ -271,7 +271,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Cluster mode: no CTA may touch a peer's shared memory before that peer runs.
-    if (SWAP && p.cluster) ptx::cluster_arrive_release();
+    if (SWAP && p.cluster) ptx::cluster_arrive_relaxed();
     const int64_t total_units = p.total_units;
 
     // TMA producer state (used by warp 0, lane 0 only): position in the static schedule.
