@@ -1263,11 +1263,13 @@ bool tma_ok(const void* base, int64_t ld_elems, int elt)
 
 // Chooses the number of K splits: minimise waves x (k-blocks per unit + fixed
 // per-unit cost), within the workspace and counter budgets.
-// `fixed` is the per-unit cost of splitting in k-block times: small for the skinny orientation
-// (coalesced partial stores, batched reduce), large for 128-row tiles, whose last arriver
-// re-reads splits x 32 x 256 floats per warp (measured: ~45 us at 1000^3, i.e. splitting
-// only pays for very long K).
-int choose_splits(int64_t tiles, int nkb, int sm, int64_t M, int64_t ldw, const RunContext& ctx, int fixed)
+// `fixed` is the per-unit cost of splitting in k-block times, `per_split` what every further split adds to it:
+// small for the skinny orientation (coalesced partial stores, batched reduce), large for 128-row tiles, whose
+// partial tile goes through the workspace and whose last arriver reads it back for every split (measured at
+// 256 x 256 x 8192 in 2 .. 16 splits: overhead = 17 us + 2.1 us per split, a k-block being 0.35 us - i.e.
+// splitting only pays for long K).
+int choose_splits(int64_t tiles, int nkb, int sm, int64_t M, int64_t ldw, const RunContext& ctx, int fixed,
+                  int per_split)
 {
     if (tiles * 2 > sm || nkb < 8 || tiles * 4 > ctx.n_tile_counters) return 1;
     const int kFixed = fixed;
@@ -1278,7 +1280,7 @@ int choose_splits(int64_t tiles, int nkb, int sm, int64_t M, int64_t ldw, const 
         const int eff = (nkb + per - 1) / per;        // splits that actually get work
         if (eff != s) continue;
         if (static_cast<size_t>(s) * M * ldw * sizeof(float) > ctx.workspace_bytes) break;
-        const int64_t cost = ((tiles * s + sm - 1) / sm) * (per + kFixed);
+        const int64_t cost = ((tiles * s + sm - 1) / sm) * (per + kFixed + per_split * s);
         if (cost < best_cost) {
             best_cost = cost;
             best = s;
@@ -1327,7 +1329,7 @@ SplitPlan plan_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContex
             return sp;
         }
     }
-    sp.splits = choose_splits(tiles, nkb, ctx.sm_count, M, ldw, ctx, sp.swap ? 6 : 100);
+    sp.splits = choose_splits(tiles, nkb, ctx.sm_count, M, ldw, ctx, sp.swap ? 6 : 48, sp.swap ? 0 : 6);
     return sp;
 }
 
@@ -1475,8 +1477,8 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     const size_t bytes_a = bad_a ? static_cast<size_t>(g.M) * lda2 * 2 : 0;
     const size_t bytes_b = bad_b ? static_cast<size_t>(b_rows) * ldb2 * 2 : 0;
     const size_t used = ((bytes_a + 255) & ~size_t(255)) + ((bytes_b + 255) & ~size_t(255));
-    // keep at least half of the workspace for split-K partial sums
-    if (used > ctx.workspace_bytes / 2) return launch_r4_planned(g, ctx, stream, kernel_id);
+    // keep at least a quarter of the workspace for split-K partial sums (the split heuristic sees what is left)
+    if (used > ctx.workspace_bytes / 4 * 3) return launch_r4_planned(g, ctx, stream, kernel_id);
 
     GemmArgs g2 = g;
     uint8_t* ws = static_cast<uint8_t*>(ctx.workspace);
