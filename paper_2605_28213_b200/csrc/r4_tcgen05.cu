@@ -850,6 +850,18 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
 #pragma unroll
                         for (int i = 0; i < 32; ++i) w[i] = v[i];
                     }
+                    if (partial) {
+                        // K-split partial sums to the workspace straight from registers: a lane holds 32 consecutive
+                        // fp32 columns of its row (128 bytes, 16-byte aligned) - eight 16-byte stores, no staging
+                        if (lane < rows) {
+                            float* prow = dst_f + (row0 + lane) * ld + col0;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                if (col0 + 4 * j < x.N)
+                                    *reinterpret_cast<uint4*>(prow + 4 * j) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                        }
+                        continue;
+                    }
                     uint8_t* b = stg + (nstaged++ & 1) * kEpiBufBytes;   // (bias was added above)
                     if (MODE == 2 ? p.epi_tma != 0 : use_tma) {   // (grouped: an earlier group's store may be in flight)
                         if (lane == 0) ptx::tma_store_wait_read<1>();   // the store that last read this buffer
@@ -874,18 +886,6 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                             }
                             ptx::tma_store_commit();
                         }
-                    } else if (partial) {
-                        __syncwarp();
-                        // K-split partial sums to the workspace (fp32 rows, 16-byte aligned): eight lanes cover a
-                        // staged 128-byte row with one 16-byte chunk each, four rows per step.
-                        for (int r4 = 0; r4 < rows; r4 += 4) {
-                            const int rr = r4 + (lane >> 3), j = lane & 7;
-                            const int col = col0 + j * 4;
-                            if (rr < rows && col < x.N)
-                                *reinterpret_cast<uint4*>(dst_f + (row0 + rr) * ld + col) =
-                                    *reinterpret_cast<const uint4*>(b + rr * 128 + ((j ^ (rr & 7)) << 4));
-                        }
-                        __syncwarp();
                     } else {
                         __syncwarp();
                         // lane l owns 32-bit word l of every staged row: coalesced 128-byte rows.
@@ -944,6 +944,17 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     // Four rows x both 128-column passes x two splits per step: sixteen independent 16-byte loads
                     // per lane are in flight before the first add (one load at a time made this reduce cost as
                     // much as a hundred k-blocks).  Every element still adds its partials in split order.
+                    const int celt_out = g.c_bf16 ? 2 : 4;
+                    const bool fast = n0 + BN <= g.N && (reinterpret_cast<uintptr_t>(g.C) % (4 * celt_out)) == 0 &&
+                                      (g.ldc * celt_out) % (4 * celt_out) == 0;
+                    float4 bias4[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+                    if (fast && g.bias) {
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            const int col = n0 + lane * 4 + c * 128;
+                            bias4[c] = make_float4(bias_at(g, col), bias_at(g, col + 1), bias_at(g, col + 2), bias_at(g, col + 3));
+                        }
+                    }
                     for (int r4 = 0; r4 < rows; r4 += 4) {
                         float4 acc[4][2];
 #pragma unroll
@@ -988,6 +999,25 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                                         acc[i][c].z += x[s2][i][c].z;
                                         acc[i][c].w += x[s2][i][c].w;
                                     }
+                        }
+                        if (fast && r4 + 3 < rows) {
+                            // whole rows of a tile inside the matrix, C aligned for vector stores: no per-element
+                            // tests (this tail runs on one warp: its instruction count is its time)
+                            const int64_t idx0 = (row0 + r4) * g.ldc + n0 + lane * 4;
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                                for (int c = 0; c < 2; ++c) {
+                                    const int64_t idx = idx0 + i * g.ldc + c * 128;
+                                    const float4 o = make_float4(acc[i][c].x + bias4[c].x, acc[i][c].y + bias4[c].y,
+                                                                 acc[i][c].z + bias4[c].z, acc[i][c].w + bias4[c].w);
+                                    if (g.c_bf16)
+                                        *reinterpret_cast<uint2*>(static_cast<uint16_t*>(g.C) + idx) =
+                                            make_uint2(pack_bf16x2(o.x, o.y), pack_bf16x2(o.z, o.w));
+                                    else
+                                        *reinterpret_cast<float4*>(static_cast<float*>(g.C) + idx) = o;
+                                }
+                            continue;
                         }
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
@@ -1266,7 +1296,7 @@ bool tma_ok(const void* base, int64_t ld_elems, int elt)
 // `fixed` is the per-unit cost of splitting in k-block times, `per_split` what every further split adds to it:
 // small for the skinny orientation (coalesced partial stores, batched reduce), large for 128-row tiles, whose
 // partial tile goes through the workspace and whose last arriver reads it back for every split (measured at
-// 256 x 256 x 8192 in 2 .. 16 splits: overhead = 17 us + 2.1 us per split, a k-block being 0.35 us - i.e.
+// 256 x 256 x 8192 in 2 .. 16 splits: overhead = 10 us + 2.2 us per split, a k-block being 0.34 us - i.e.
 // splitting only pays for long K).
 int choose_splits(int64_t tiles, int nkb, int sm, int64_t M, int64_t ldw, const RunContext& ctx, int fixed,
                   int per_split)
@@ -1329,7 +1359,7 @@ SplitPlan plan_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContex
             return sp;
         }
     }
-    sp.splits = choose_splits(tiles, nkb, ctx.sm_count, M, ldw, ctx, sp.swap ? 6 : 48, sp.swap ? 0 : 6);
+    sp.splits = choose_splits(tiles, nkb, ctx.sm_count, M, ldw, ctx, sp.swap ? 6 : 30, sp.swap ? 0 : 6);
     return sp;
 }
 
