@@ -96,6 +96,22 @@ def test_addmm_large_tensor_core_paths(kb):
                 assert (kid - 400) & flag, (kid, flag)
 
 
+@pytest.mark.parametrize("shape", [(256, 512, 8192, 0), (200, 700, 9000, 0), (130, 264, 12000, 1)],
+                         ids=lambda s: "x".join(map(str, s[:3])))
+def test_addmm_through_the_workspace_split(kb, shape):
+    # few tiles, long K: the heuristic splits K through the workspace; the bias must be added once, by the
+    # reduce - on its test-free path (whole rows of tiles inside an aligned C) and on the general one
+    M, N, K, pad = shape
+    for bf in (False, True):
+        case = gen.make_case(M, N, K, seed=270, dist_a="integer", dist_b="integer", c_bf16=bf, ldc=N + pad,
+                             name=f"addmm-split{M}x{N}x{K}")
+        bias = gen.draw((1, N), "integer", 271, 2)[0]
+        C_ref, S = reference(case, bias, np.arange(M))
+        vals, bits, kid = run_addmm(kb, case, bias, 4)
+        assert (kid - 400) & 4, kid
+        P.assert_matches_oracle(case, vals, bits, C_ref, S, exact=True, what=case.name)
+
+
 def test_addmm_argument_errors(kb):
     import torch
     a = torch.zeros(64 * 64, dtype=torch.int16, device="cuda")
