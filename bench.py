@@ -419,8 +419,7 @@ def lineage_table(prob_c4, kb, gen, torch, device, peaks):
         with kb.Gemm(device.index, b_col_major=c.b_col_major, c_bf16=c.c_bf16) as tg:
             n_cand = len(tg.plan_candidates(pr.A, pr.B, pr.C, c.M, c.N, c.K, c.lda, c.ldb, c.ldc))
             plan, best_us, heur_us = tg.autotune(pr.A, pr.B, pr.C, c.M, c.N, c.K, c.lda, c.ldb, c.ldc, iters=10)
-        tune[name] = {"candidates": n_cand, "pinned_plan": dict(zip(("kernel", "splits", "split_via", "group_m",
-                                                                      "half_tail"), plan.as_tuple())),
+        tune[name] = {"candidates": n_cand, "pinned_plan": plan.as_dict(),
                       "us_pinned": best_us, "us_heuristic": heur_us,
                       "tflops_pinned": c.flops / (best_us * 1e-6) / 1e12,
                       "tflops_heuristic": c.flops / (heur_us * 1e-6) / 1e12}

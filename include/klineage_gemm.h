@@ -85,6 +85,19 @@ typedef enum {
  */
 #define KLINEAGE_FLAG_STATIC_B 1u
 
+/*
+ * KLINEAGE_FLAG_TEST_GIVE_UP - a test hook for the boundary's error path (KLINEAGE_ERR_TIMEOUT,
+ * klineage_gemm_get_device_status).  The FIRST klineage_gemm_run(..., KLINEAGE_TCGEN05, ...) call on the
+ * handle that takes the single-CTA, non-cluster, TMA-fed kernel with more than two k-blocks per tile makes
+ * that launch give up in the permitted way: its TMA producer stops after two k-blocks and the MMA issuer's
+ * bounded wait for the third runs out after about a millisecond, whereupon every CTA records the error,
+ * raises its abort flag, lets its other roles leave their loops, frees its tensor memory and RETURNS
+ * NORMALLY - no trap, no fault, nothing unbounded; C is not written.  Every later call on the handle runs
+ * normally.  The paper's gate (Method: a candidate must compile, be correct and be profiled) needs failures
+ * to surface as statuses, which is what this flag lets a test observe.
+ */
+#define KLINEAGE_FLAG_TEST_GIVE_UP 2u
+
 /* Create-time configuration (host memory, read during create only). */
 typedef struct {
     int device;             /* CUDA device ordinal the handle is bound to                              */
@@ -93,7 +106,7 @@ typedef struct {
     size_t workspace_bytes; /* device scratch of rung 4: split-K partial sums, aligned copies of unaligned
                                operands, the tables of grouped / multi-destination launches; 0 selects
                                the default (64 MiB).  Calls on one handle share it: one stream at a time */
-    unsigned flags;         /* 0, or KLINEAGE_FLAG_STATIC_B                                            */
+    unsigned flags;         /* 0, or an OR of KLINEAGE_FLAG_STATIC_B, KLINEAGE_FLAG_TEST_GIVE_UP              */
 } klineage_gemm_config_t;
 
 /*
@@ -166,10 +179,22 @@ klineage_status_t klineage_gemm_destroy(klineage_gemm_t h);
  * the stream).  *code_out receives KLINEAGE_OK or KLINEAGE_ERR_TIMEOUT;
  * *kernel_id_out (may be NULL) receives the id the last finished kernel wrote
  * on the device, which identifies rung and sub-path (see
- * klineage_gemm_last_kernel_id).  The error code is cleared by the read.
+ * klineage_gemm_last_kernel_id).  The error code is cleared by the read; after a
+ * give-up the handle's split-K arrival counters are reset as well, so that the
+ * next call starts clean.
  * The paper's gate (Method: compile, correctness, profile) is what this serves.
  */
 klineage_status_t klineage_gemm_get_device_status(klineage_gemm_t h, int* code_out, int* kernel_id_out);
+
+/*
+ * Where the last device-side give-up reported by klineage_gemm_get_device_status on this
+ * handle happened: *block_out the CTA, *where_out the role and barrier -
+ *   0x400|s producer / "stage s free",  0x410|b MMA issuer / "accumulator b drained",
+ *   0x420|s MMA issuer / "operand stage s landed",  0x430|b epilogue / "accumulator b complete",
+ *   0x440..0x470|s gathering producers and the Conv2d producers,  0x500.. the CTA-pair kernel's roles.
+ * Both are 0 when no give-up has been read.  Either pointer may be NULL.
+ */
+klineage_status_t klineage_gemm_last_give_up(klineage_gemm_t h, unsigned* block_out, unsigned* where_out);
 
 /*
  * Host-side record of the kernel the last successful run enqueued:
@@ -217,8 +242,15 @@ int klineage_gemm_last_kernel_id(klineage_gemm_t h);
  *     kernel.  Two calls that overlap on the GPU (different streams, or several
  *     host threads) race on the array: keep calls to one stream at a time.
  *   - Device-side give-ups (bounded waits) cannot be read back through this call.
- * Results are bit-identical to klineage_gemm_run(..., KLINEAGE_TCGEN05, ...) with a
- * default handle for every accepted shape.
+ * Results: for operands that satisfy TMA's alignment rules (16-byte aligned base
+ * and pitch of A and B) the call runs the same kernels with the same schedule as
+ * klineage_gemm_run(..., KLINEAGE_TCGEN05, ...) on a default handle and gives the
+ * same bits.  Unaligned operands take another sub-path here (the handle copies
+ * them into its workspace first, this call gathers them tile by tile, and the two
+ * may split K differently): the result then carries the library's usual
+ * guarantee - bit-exact where fp32 sums are exact, else within
+ * K * 2^-23 * (|A| . |B|)_ij of the exact product - not bit equality with the
+ * handle path.
  * Errors: as klineage_gemm_run, plus KLINEAGE_ERR_SCRATCH_LIMIT.
  */
 klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype, int64_t M, int64_t N, int64_t K,
@@ -411,6 +443,9 @@ typedef struct {
     int split_via;
     int group_m;
     int half_tail;
+    int tile_n;
+    int tail_n;
+    int stages;
 } klineage_gemm_plan_t;
 
 #define KLINEAGE_MAX_PLANS 48

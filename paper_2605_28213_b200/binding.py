@@ -26,6 +26,7 @@ KLINEAGE_ERR_SCRATCH_LIMIT = 8
 KLINEAGE_B_ROW_MAJOR, KLINEAGE_B_COL_MAJOR = 0, 1
 KLINEAGE_C_F32, KLINEAGE_C_BF16, KLINEAGE_C_F16 = 0, 1, 2
 KLINEAGE_FLAG_STATIC_B = 1
+KLINEAGE_FLAG_TEST_GIVE_UP = 2
 KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELINED, KLINEAGE_TCGEN05, KLINEAGE_MMA_SYNC = range(6)
 # the five-step ladder, then the intermediate legacy tensor-core rung ("3.5")
 VARIANTS = (KLINEAGE_NAIVE, KLINEAGE_TILED, KLINEAGE_VECTORIZED, KLINEAGE_PIPELINED, KLINEAGE_TCGEN05,
@@ -38,7 +39,7 @@ EXPORTED_SYMBOLS = (
     "klineage_gemm_run_batched", "klineage_gemm_run_grouped", "klineage_gemm_last_launch_count",
     "klineage_gemm_run_multi_dst", "klineage_conv2d_run", "klineage_conv2d_check_args",
     "klineage_gemm_plan_candidates", "klineage_gemm_set_plan", "klineage_gemm_get_plan", "klineage_gemm_autotune",
-    "klineage_gemm_host_scratch_bytes", "klineage_gemm_run_host",
+    "klineage_gemm_host_scratch_bytes", "klineage_gemm_run_host", "klineage_gemm_last_give_up",
 )
 
 
@@ -179,13 +180,18 @@ def klineage_conv2d_check_args(y_dtype, N, H, W, C, F, R, S, pad_h, pad_w, strid
 
 class klineage_gemm_plan_t(ctypes.Structure):
     """Launch plan of the tcgen05 rung (0 in a field = the rung's heuristic)."""
-    _fields_ = [("kernel", _int), ("splits", _int), ("split_via", _int), ("group_m", _int), ("half_tail", _int)]
+    _fields_ = [("kernel", _int), ("splits", _int), ("split_via", _int), ("group_m", _int), ("half_tail", _int),
+                ("tile_n", _int), ("tail_n", _int), ("stages", _int)]
+    FIELDS = ("kernel", "splits", "split_via", "group_m", "half_tail", "tile_n", "tail_n", "stages")
 
     def as_tuple(self):
-        return (self.kernel, self.splits, self.split_via, self.group_m, self.half_tail)
+        return tuple(getattr(self, f) for f in self.FIELDS)
+
+    def as_dict(self):
+        return dict(zip(self.FIELDS, self.as_tuple()))
 
     def __repr__(self):
-        return ("plan(kernel=%d, splits=%d, split_via=%d, group_m=%d, half_tail=%d)" % self.as_tuple())
+        return "plan(" + ", ".join("%s=%d" % kv for kv in self.as_dict().items()) + ")"
 
 
 KLINEAGE_MAX_PLANS = 48
@@ -291,6 +297,19 @@ def klineage_gemm_last_kernel_id(h) -> int:
     return _lib.klineage_gemm_last_kernel_id(h)
 
 
+_lib.klineage_gemm_last_give_up.restype = _int
+_lib.klineage_gemm_last_give_up.argtypes = [_p, ctypes.POINTER(ctypes.c_uint), ctypes.POINTER(ctypes.c_uint)]
+
+
+def klineage_gemm_last_give_up(h):
+    """(CTA, role-and-barrier code) of the last device-side give-up read through get_device_status; (0, 0) if none."""
+    block, where = ctypes.c_uint(0), ctypes.c_uint(0)
+    st = _lib.klineage_gemm_last_give_up(h, ctypes.byref(block), ctypes.byref(where))
+    if st != KLINEAGE_OK:
+        raise KlineageError(st, "klineage_gemm_last_give_up")
+    return block.value, where.value
+
+
 class Gemm:
     """Handle wrapper: ``Gemm(device, b_col_major, c_bf16).run(A, B, C, M, N, K, lda, ldb, ldc, variant)``.
 
@@ -300,14 +319,14 @@ class Gemm:
     """
 
     def __init__(self, device: int = 0, b_col_major: bool = False, c_bf16: bool = False,
-                 workspace_bytes: int = 0, static_b: bool = False):
+                 workspace_bytes: int = 0, static_b: bool = False, test_give_up: bool = False):
         self.device = int(device)
         self.b_col_major = bool(b_col_major)
         self.c_bf16 = bool(c_bf16)
         self._h: Optional[int] = klineage_gemm_create(
             self.device, KLINEAGE_B_COL_MAJOR if b_col_major else KLINEAGE_B_ROW_MAJOR,
             KLINEAGE_C_BF16 if c_bf16 else KLINEAGE_C_F32, workspace_bytes,
-            KLINEAGE_FLAG_STATIC_B if static_b else 0)
+            (KLINEAGE_FLAG_STATIC_B if static_b else 0) | (KLINEAGE_FLAG_TEST_GIVE_UP if test_give_up else 0))
 
     @staticmethod
     def _ptr(x):
@@ -392,6 +411,9 @@ class Gemm:
 
     def last_kernel_id(self) -> int:
         return klineage_gemm_last_kernel_id(self._h)
+
+    def last_give_up(self):
+        return klineage_gemm_last_give_up(self._h)
 
     def last_launch_count(self) -> int:
         return _lib.klineage_gemm_last_launch_count(self._h)

@@ -25,6 +25,7 @@ struct klineage_gemm_s {
     int last_kernel_id = -1;
     int last_launches = 0;             // GEMM kernels the last run call enqueued
     std::map<PlanKey, R4Plan> plans;   // pinned by klineage_gemm_set_plan / klineage_gemm_autotune
+    unsigned give_up_block = 0, give_up_where = 0;   // detail of the last device-side give-up that was read
     bool forcing = false;              // autotune in progress: run `forced` whatever is pinned
     R4Plan forced;
     // klineage_gemm_run_host: copy streams and events, created by its first call
@@ -145,6 +146,9 @@ klineage_gemm_plan_t to_public(const R4Plan& p)
     o.split_via = p.split_via;
     o.group_m = p.group_m;
     o.half_tail = p.half_tail;
+    o.tile_n = p.tile_n;
+    o.tail_n = p.tail_n;
+    o.stages = p.stages;
     return o;
 }
 
@@ -156,6 +160,9 @@ R4Plan from_public(const klineage_gemm_plan_t& p)
     o.split_via = p.split_via;
     o.group_m = p.group_m;
     o.half_tail = p.half_tail;
+    o.tile_n = p.tile_n;
+    o.tail_n = p.tail_n;
+    o.stages = p.stages;
     return o;
 }
 
@@ -249,7 +256,7 @@ klineage_status_t klineage_gemm_create(klineage_gemm_t* out, const klineage_gemm
     if (cfg->b_layout != KLINEAGE_B_ROW_MAJOR && cfg->b_layout != KLINEAGE_B_COL_MAJOR) return KLINEAGE_ERR_INVALID_ARG;
     if (cfg->c_dtype != KLINEAGE_C_F32 && cfg->c_dtype != KLINEAGE_C_BF16 && cfg->c_dtype != KLINEAGE_C_F16)
         return KLINEAGE_ERR_INVALID_ARG;
-    if (cfg->flags & ~KLINEAGE_FLAG_STATIC_B) return KLINEAGE_ERR_INVALID_ARG;
+    if (cfg->flags & ~(KLINEAGE_FLAG_STATIC_B | KLINEAGE_FLAG_TEST_GIVE_UP)) return KLINEAGE_ERR_INVALID_ARG;
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev) {
         cudaGetLastError();
@@ -865,6 +872,7 @@ klineage_status_t klineage_gemm_plan_candidates(klineage_gemm_t h, int64_t M, in
         klineage_gemm_check_args(h->b_layout, h->c_dtype, M, N, K, A, lda, B, ldb, C, ldc, KLINEAGE_TCGEN05);
     if (chk != KLINEAGE_OK) return chk;
     const GemmArgs g = make_args(h, M, N, K, A, lda, B, ldb, nullptr, const_cast<void*>(C), ldc);
+    DeviceGuard guard(h->ctx.device);      // (the planner may ask the runtime how many clusters the device holds)
     R4Plan tmp[KLINEAGE_MAX_PLANS];
     const int n = r4_enumerate_plans(g, h->ctx, tmp, KLINEAGE_MAX_PLANS);
     *count = n;
@@ -887,6 +895,7 @@ klineage_status_t klineage_gemm_set_plan(klineage_gemm_t h, int64_t M, int64_t N
     }
     const R4Plan pl = from_public(*plan);
     const GemmArgs g = make_args(h, M, N, K, A, lda, B, ldb, nullptr, const_cast<void*>(C), ldc);
+    DeviceGuard guard(h->ctx.device);
     if (!r4_plan_valid(g, h->ctx, pl)) return KLINEAGE_ERR_INVALID_ARG;
     h->plans[key] = pl;
     return KLINEAGE_OK;
@@ -1012,12 +1021,25 @@ klineage_status_t klineage_gemm_get_device_status(klineage_gemm_t h, int* code_o
     if (kernel_id_out) *kernel_id_out = static_cast<int>(w[1]);
     if (w[0] != kDevOk) {
         fprintf(stderr, "klineage_gemm: device-side give-up code=%u block=%u where=0x%x\n", w[0], w[2], w[3]);
+        h->give_up_block = w[2];
+        h->give_up_where = w[3];
         if (cudaMemset(h->status, 0, sizeof(unsigned)) != cudaSuccess) cudaGetLastError();
+        // A CTA that gave up may have left split-K arrival counters short of their self-reset; a later split
+        // launch would then see a wrong last arriver.  The stream is idle by contract: start them from zero.
+        if (cudaMemset(h->ctx.tile_counters, 0, sizeof(unsigned) * h->ctx.n_tile_counters) != cudaSuccess) cudaGetLastError();
     }
     return KLINEAGE_OK;
 }
 
 int klineage_gemm_last_kernel_id(klineage_gemm_t h) { return h ? h->last_kernel_id : -1; }
+
+klineage_status_t klineage_gemm_last_give_up(klineage_gemm_t h, unsigned* block_out, unsigned* where_out)
+{
+    if (!h) return KLINEAGE_ERR_INVALID_ARG;
+    if (block_out) *block_out = h->give_up_block;
+    if (where_out) *where_out = h->give_up_where;
+    return KLINEAGE_OK;
+}
 
 const char* klineage_status_string(int status)
 {

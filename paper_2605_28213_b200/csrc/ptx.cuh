@@ -65,9 +65,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 
 // The same wait on a barrier given by its shared-window address (role loops that step through a ring keep the
 // address in a register instead of converting a pointer every iteration).
-__device__ __forceinline__ bool mbar_wait_addr(uint32_t bar_addr, uint32_t parity, volatile uint32_t* abort_flag)
+__device__ __forceinline__ bool mbar_wait_addr(uint32_t bar_addr, uint32_t parity, volatile uint32_t* abort_flag,
+                                               uint32_t limit = kMbarPollLimit)
 {
-    for (uint32_t i = 0; i < kMbarPollLimit; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"

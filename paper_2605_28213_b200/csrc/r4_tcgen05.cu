@@ -106,6 +106,11 @@ struct R4Params {
     int conv_b_rows;        // rows of the weight box (128 with half_only, else 256)
     int conv_patch;         // patches by TMA: row tile t = 8 x 16 output patch (t % tq, (t / tq) % tp) of image t / (tq tp)
     int conv_tq, conv_tp;
+    // Give-up test hook (KLINEAGE_FLAG_TEST_GIVE_UP, one launch): the TMA producer stops after this many k-blocks
+    // and the MMA issuer's wait for the next operand stage runs out after test_poll_limit polls, so that the
+    // kernel's give-up path - error word, abort flag, every role leaving its loop, TMEM freed - really runs.
+    int test_stop_after;
+    uint32_t test_poll_limit;
 };
 
 // One entry of the static schedule.
@@ -315,6 +320,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     auto produce = [&](uint32_t limit) {
         while (prod.live && prod.it < limit) {
             const uint32_t it = prod.it;
+            if (p.test_stop_after > 0 && it == static_cast<uint32_t>(p.test_stop_after)) {   // test hook: a stage never arrives
+                prod.live = false;
+                break;
+            }
             const int s = it % STAGES;
             if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
                 report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x400u | s);
@@ -581,6 +590,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             const uint32_t a_lo0 = static_cast<uint32_t>(a_desc0), a_hi = static_cast<uint32_t>(a_desc0 >> 32);
             const uint32_t b_lo0 = (((ptx::smem_u32(smem) + kABytes) >> 4) & 0x3FFFu) | (p.b_desc_lbo << 16);
             const uint32_t b_hi = p.b_desc_hi, kstep = p.b_kstep;
+            const uint32_t full_limit = p.test_poll_limit ? p.test_poll_limit : ptx::kMbarPollLimit;
             for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++t) {
                 const Unit x = unit_of(u);
                 const int kb0 = x.kb0, kb1 = x.kb1;
@@ -594,7 +604,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag)) {
+                    if (!ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag, full_limit)) {
                         report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x420u | s);
                         abort_flag[0] = 1;
                         ok = false;
@@ -793,6 +803,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
                 continue;
             }
+            if (MODE == 0 && p.cluster) continue;     // drained after the cluster-wide barrier below
             const int row0 = m0 + q * 32;
             if (row0 < x.M) {
                 const bool partial = p.splits > 1;
@@ -1050,7 +1061,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 }
             }
                 }
-        if (p.epi_tma && lane == 0) ptx::tma_store_wait_all<0>();
+        // shared memory may go once the stores have read it; their writes complete with the grid
+        if (p.epi_tma && lane == 0) ptx::tma_store_wait_read<0>();
     } else if (GENERIC) {
         // ------------------------------------------------------------ generic-proxy producers
         const int pt = threadIdx.x - 6 * 32;                 // 0..127
@@ -1223,6 +1235,180 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         }
     }
 
+    if (!SWAP && MODE == 0 && p.cluster) {
+        // K split of a 128-row tile inside a thread-block cluster (2, 4 or 8 CTAs, one K range each).  The tile
+        // is cut into (32-row lane quarter, store unit of 128 bytes per row) pairs: 16 for a 2-byte C, 32 for
+        // fp32; CTA r owns pairs [r * per, (r + 1) * per).  After a first cluster barrier - every CTA's MMAs have
+        // completed, so every operand ring is idle - each CTA sends the 32 x 32 blocks of its partial tile that
+        // it does not own to their owners (plain st.shared::cluster into the owner's ring), laid out
+        // [column / 4][row][column % 4] so that a lane's four columns travel as one conflict-free 16-byte
+        // store.  After a second barrier the owner adds the partials in rank order (deterministic; its own
+        // comes straight from TMEM), adds the bias once, rounds and stores its pairs.  No workspace, no
+        // atomics, no trip through L2.
+        const uint32_t rank = ptx::cluster_ctarank();
+        ptx::cluster_arrive_release();
+        ptx::cluster_wait_acquire();
+        const bool epi_warp = warp >= 2 && warp < 6;
+        const bool out_bf16 = g.c_bf16 != 0;
+        const int sub_log2 = out_bf16 ? 1 : 0;                          // 32-column blocks per store unit
+        const int per_log2 = (out_bf16 ? 4 : 5) - p.splits_log2;        // pairs per CTA
+        const int q = warp & 3;                                         // TMEM lane quarter of this warp
+        const uint32_t tlane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+        float* recv = reinterpret_cast<float*>(smem);
+        // slot of 32-column block c (of lane quarter qq) sent by CTA `src`, inside its owner's ring
+        auto slot_of = [&](int src, int c, int qq) {
+            const int idx = ((c >> sub_log2) << 2) + qq;
+            const int lp = idx & ((1 << per_log2) - 1);
+            return recv + ((((src << per_log2) + lp) << sub_log2) + (c & ((1 << sub_log2) - 1))) * 1024 + lane * 4;
+        };
+        if (epi_warp && !abort_flag[0]) {
+            ptx::tc_fence_after_sync();
+            // two blocks per step: both TMEM loads are in flight before the first remote store
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; c += 2) {
+                const uint32_t own0 = static_cast<uint32_t>((((c >> sub_log2) << 2) + q) >> per_log2);
+                const uint32_t own1 = static_cast<uint32_t>(((((c + 1) >> sub_log2) << 2) + q) >> per_log2);
+                if (own0 == rank && own1 == rank) continue;
+                uint32_t v0[32], v1[32];
+                ptx::tmem_ld_32x32b_x32(tlane + c * 32, v0);
+                ptx::tmem_ld_32x32b_x32(tlane + c * 32 + 32, v1);
+                const uint32_t r0 = ptx::map_to_cta(ptx::smem_u32(slot_of(static_cast<int>(rank), c, q)), own0);
+                const uint32_t r1 = ptx::map_to_cta(ptx::smem_u32(slot_of(static_cast<int>(rank), c + 1, q)), own1);
+                ptx::tmem_ld_wait();
+                if (own0 != rank) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        ptx::st_cluster_v4_f32(r0 + j * 512, __uint_as_float(v0[4 * j]), __uint_as_float(v0[4 * j + 1]),
+                                               __uint_as_float(v0[4 * j + 2]), __uint_as_float(v0[4 * j + 3]));
+                }
+                if (own1 != rank) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        ptx::st_cluster_v4_f32(r1 + j * 512, __uint_as_float(v1[4 * j]), __uint_as_float(v1[4 * j + 1]),
+                                               __uint_as_float(v1[4 * j + 2]), __uint_as_float(v1[4 * j + 3]));
+                }
+            }
+        }
+        ptx::cluster_arrive_release();
+        ptx::cluster_wait_acquire();
+        if (epi_warp && !abort_flag[0]) {
+            const Unit x = decode_unit(static_cast<int64_t>(blockIdx.x), p);
+            uint8_t* stg = epi_smem + (warp - 2) * 2 * kEpiBufBytes;
+            const int cpc = out_bf16 ? 64 : 32;
+            uint32_t nstaged = 0;
+            // a warp takes the pairs of its own TMEM lane quarter (this CTA's partial is read from TMEM)
+#pragma unroll 1
+            for (int lp = 0; lp < (1 << per_log2); ++lp) {
+                const int idx = (static_cast<int>(rank) << per_log2) + lp;
+                if ((idx & 3) != q) continue;
+                const int u = idx >> 2;
+                const int row0 = x.m0 + q * 32, col0 = x.n0 + u * cpc;
+                if (row0 >= g.M || col0 >= g.N) continue;
+                const int rows = min(32, g.M - row0);
+                uint32_t own[2][32];
+                ptx::tmem_ld_32x32b_x32(tlane + (u << sub_log2) * 32, own[0]);
+                if (out_bf16) ptx::tmem_ld_32x32b_x32(tlane + (u << sub_log2) * 32 + 32, own[1]);
+                float acc[2][32];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) acc[h][i] = 0.f;
+                }
+                bool own_added = false;
+                for (int src = 0; src < p.splits; ++src) {
+                    if (src == static_cast<int>(rank)) {
+                        ptx::tmem_ld_wait();
+                        own_added = true;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            if (h > sub_log2) continue;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) acc[h][i] += __uint_as_float(own[h][i]);
+                        }
+                        continue;
+                    }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (h > sub_log2) continue;
+                        const float4* sl = reinterpret_cast<const float4*>(slot_of(src, (u << sub_log2) + h, q));
+                        float4 t[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) t[j] = sl[j * 32];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            acc[h][4 * j] += t[j].x;
+                            acc[h][4 * j + 1] += t[j].y;
+                            acc[h][4 * j + 2] += t[j].z;
+                            acc[h][4 * j + 3] += t[j].w;
+                        }
+                    }
+                }
+                if (!own_added) ptx::tmem_ld_wait();
+                if (g.bias) {   // lane l fetches the bias of columns col0 + l (and + 32), shuffles hand them round
+                    const float b0 = (col0 + lane < g.N) ? bias_at(g, col0 + lane) : 0.f;
+                    const float b1 = (out_bf16 && col0 + 32 + lane < g.N) ? bias_at(g, col0 + 32 + lane) : 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        acc[0][i] += __shfl_sync(0xFFFFFFFFu, b0, i);
+                        acc[1][i] += __shfl_sync(0xFFFFFFFFu, b1, i);
+                    }
+                }
+                uint32_t w[32];
+                if (out_bf16) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        w[i] = pack_bf16x2(acc[0][2 * i], acc[0][2 * i + 1]);
+                        w[16 + i] = pack_bf16x2(acc[1][2 * i], acc[1][2 * i + 1]);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(acc[0][i]);
+                }
+                uint8_t* b = stg + (nstaged++ & 1) * kEpiBufBytes;
+                if (p.epi_tma) {
+                    if (lane == 0) ptx::tma_store_wait_read<1>();   // the store that last read this buffer
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    *reinterpret_cast<uint4*>(b + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                        make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                if (p.epi_tma) {
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::tma_store_2d(&map_c, col0, row0, b);
+                        ptx::tma_store_commit();
+                    }
+                } else {
+                    __syncwarp();
+                    // lane l owns 32-bit word l of every staged row: coalesced 128-byte rows
+                    for (int rr = 0; rr < rows; ++rr) {
+                        const uint32_t word = *reinterpret_cast<const uint32_t*>(
+                            b + rr * 128 + (((lane >> 2) ^ (rr & 7)) << 4) + (lane & 3) * 4);
+                        const int64_t row = row0 + rr;
+                        if (out_bf16) {
+                            const int col = col0 + 2 * lane;
+                            uint16_t* d = static_cast<uint16_t*>(g.C) + row * g.ldc + col;
+                            if (col + 1 < g.N && (reinterpret_cast<uintptr_t>(d) & 3) == 0) {
+                                *reinterpret_cast<uint32_t*>(d) = word;
+                            } else {
+                                if (col < g.N) d[0] = static_cast<uint16_t>(word & 0xFFFFu);
+                                if (col + 1 < g.N) d[1] = static_cast<uint16_t>(word >> 16);
+                            }
+                        } else {
+                            const int col = col0 + lane;
+                            if (col < g.N) static_cast<float*>(g.C)[row * g.ldc + col] = __uint_as_float(word);
+                        }
+                    }
+                    __syncwarp();
+                }
+            }
+            // shared memory may go once the stores have read it; their writes complete with the grid
+            if (p.epi_tma && lane == 0) ptx::tma_store_wait_read<0>();
+        }
+    }
+
     if (SWAP && p.cluster) {
         // Every thread of every CTA of the cluster arrives; after the wait all partial
         // blocks sent to this CTA are visible in its shared memory.
@@ -1339,6 +1525,40 @@ int choose_cluster_splits(int64_t tiles, int nkb, int sm)
     return best;
 }
 
+// 128-row tiles split inside a cluster: what the two cluster barriers, the exchange of the partial tile through
+// the operand rings and the owner's reduce cost, in k-block times (0.31 us), measured in CUDA-graph replay on
+// products of 1 .. 64 tiles: 4.0 / 5.0 / 6.6 us for 2 / 4 / 8 CTAs, about 2 us more when the launch fills
+// most of the GPU.  A launch never exceeds one wave of clusters: a CTA runs exactly one unit, and a second
+// wave would pay the kernel's set-up again (measured: 2048^3 in 4 splits 54 us against 17 us unsplit).
+int cluster_fixed_cost(int s, int64_t ctas, int sm)
+{
+    const int base = s == 2 ? 13 : s == 4 ? 16 : 22;
+    return base + (ctas * 3 > static_cast<int64_t>(sm) * 2 ? 6 : 0);
+}
+// Clusters of `s` CTAs of this kernel that the device can hold at once (GPC boundaries make this less than
+// SMs / s for large clusters); asked of the runtime once per size and device.
+int max_resident_clusters(int s, const RunContext& ctx);
+
+// K splits of the cluster route for a regular-orientation problem and their estimated cost (k-block times);
+// 1 when no split fits or pays.
+int choose_regular_cluster_splits(int64_t tiles, int nkb, const RunContext& ctx, int64_t* cost_out)
+{
+    int best = 1;
+    int64_t best_cost = ((tiles + ctx.sm_count - 1) / ctx.sm_count) * static_cast<int64_t>(nkb);
+    for (int s = 2; s <= 8 && s * 2 <= nkb; s *= 2) {
+        const int per = (nkb + s - 1) / s;
+        if ((nkb + per - 1) / per != s) continue;
+        if (tiles > max_resident_clusters(s, ctx)) continue;
+        const int64_t cost = per + cluster_fixed_cost(s, tiles * s, ctx.sm_count);
+        if (cost < best_cost) {
+            best_cost = cost;
+            best = s;
+        }
+    }
+    *cost_out = best_cost;
+    return best;
+}
+
 // How a shape is split along K: not at all, through the global workspace, or
 // through a cluster.  One function so that every caller plans the same way.
 struct SplitPlan {
@@ -1346,6 +1566,7 @@ struct SplitPlan {
     bool cluster;
     bool swap;
 };
+
 SplitPlan plan_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContext& ctx)
 {
     SplitPlan sp;
@@ -1360,6 +1581,21 @@ SplitPlan plan_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContex
         }
     }
     sp.splits = choose_splits(tiles, nkb, ctx.sm_count, M, ldw, ctx, sp.swap ? 6 : 30, sp.swap ? 0 : 6);
+    if (!sp.swap) {
+        // 128-row tiles: the cluster route against the workspace route chosen above and against no split
+        int64_t cost_c = 0;
+        const int sc = choose_regular_cluster_splits(tiles, nkb, ctx, &cost_c);
+        if (sc > 1) {
+            const int sm = ctx.sm_count;
+            const int per_w = (nkb + sp.splits - 1) / sp.splits;
+            const int64_t cost_w = sp.splits > 1 ? ((tiles * sp.splits + sm - 1) / sm) * static_cast<int64_t>(per_w + 30 + 6 * sp.splits)
+                                                 : ((tiles + sm - 1) / sm) * static_cast<int64_t>(nkb);
+            if (cost_c <= cost_w) {
+                sp.splits = sc;
+                sp.cluster = true;
+            }
+        }
+    }
     return sp;
 }
 
@@ -1371,7 +1607,10 @@ bool split_feasible(int M, int64_t tiles, int nkb, int64_t ldw, const RunContext
     if (splits < 1 || splits > 64 || splits > nkb) return false;
     const int per = (nkb + splits - 1) / splits;
     if ((nkb + per - 1) / per != splits) return false;
-    if (cluster) return M <= 32 && (splits == 2 || splits == 4 || splits == 8);
+    if (cluster) {
+        if (splits != 2 && splits != 4 && splits != 8) return false;
+        return M <= 32 || (M > 64 && tiles <= max_resident_clusters(splits, ctx));   // 128-row tiles: one wave of clusters
+    }
     if (tiles * 4 > ctx.n_tile_counters) return false;
     return static_cast<size_t>(splits) * M * ldw * sizeof(float) <= ctx.workspace_bytes;
 }
@@ -1389,8 +1628,7 @@ bool resolve_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContext&
         else if (pl.split_via == 1)
             sp.cluster = false;
         else
-            sp.cluster = sp.swap && M <= 32 && (pl.splits == 2 || pl.splits == 4 || pl.splits == 8);
-        if (sp.cluster && !sp.swap) return false;
+            sp.cluster = (M <= 32 || !sp.swap) && (pl.splits == 2 || pl.splits == 4 || pl.splits == 8);
         if (!split_feasible(M, tiles, nkb, ldw, ctx, sp.splits, sp.cluster)) return false;
     }
     *out = sp;
@@ -1435,6 +1673,36 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
     cfg.attrs = attrs;
     cfg.numAttrs = na;
     return cudaLaunchKernelEx(&cfg, kern, g, ma, mb, mc, p);
+}
+
+int max_resident_clusters(int s, const RunContext& ctx)
+{
+    static int cache[64][4] = {};      // [device][log2 s], 0 = not asked yet
+    const int l2 = s == 2 ? 1 : s == 4 ? 2 : 3;
+    const bool cacheable = ctx.device >= 0 && ctx.device < 64;
+    if (cacheable && cache[ctx.device][l2] != 0) return cache[ctx.device][l2];
+    auto kern = r4_tcgen05_kernel<false, false, false, 0>;
+    int n = 0;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(static_cast<unsigned>(ctx.sm_count / s * s));
+    cfg.blockDim = dim3(kThreadsTma);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = static_cast<unsigned>(s);
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        n = ctx.sm_count / (2 * s);    // the runtime would not say: assume half
+        if (n < 1) n = 1;
+    }
+    if (cacheable) cache[ctx.device][l2] = n;
+    return n;
 }
 
 }  // namespace
@@ -1538,6 +1806,9 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     c2.workspace = ws + used;
     c2.workspace_bytes = ctx.workspace_bytes - used;
     c2.kid_flags = 64;
+    // The promise "no in-flight work writes B" is about the caller's B; the copy just enqueued IS in-flight
+    // work that writes the B this launch reads, so its loads must wait for it like every other access.
+    if (bad_b) c2.flags &= ~1u;
     return launch_r4_planned(g2, c2, stream, kernel_id);
 }
 
@@ -1584,7 +1855,7 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     // TMA store needs C 16-byte aligned with a 16-byte-multiple pitch, and a row length that is a
     // multiple of 16 bytes: measured on B200, a store box that ends inside a 16-byte unit at the
     // right edge of the tensor writes that whole unit, i.e. up to 12 bytes of row padding.
-    p.epi_tma = (!swap && p.splits == 1 && ctx.encode_tiled && tma_ok(g.C, g.ldc, celt) &&
+    p.epi_tma = (!swap && (p.splits == 1 || p.cluster) && ctx.encode_tiled && tma_ok(g.C, g.ldc, celt) &&
                  (static_cast<int64_t>(g.N) * celt) % 16 == 0)
                     ? 1
                     : 0;
@@ -1676,6 +1947,13 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
         p.n_dst = md->n;
         return g.b_col ? launch<true, false, false, 3>(g, ma, mb, mc, p, grid, ctx.device, stream)
                        : launch<false, false, false, 3>(g, ma, mb, mc, p, grid, ctx.device, stream);
+    }
+    if ((ctx.flags & 2u) && !generic && !p.cluster && !swap && p.kb_per_split > 2) {
+        // give-up test hook, this one launch only (never on a cluster or CTA-pair launch: there a CTA that gives
+        // up leaves its peers waiting for their own limits)
+        p.test_stop_after = 2;
+        p.test_poll_limit = 1u << 14;
+        ctx.flags &= ~2u;
     }
 #define KLIN_R4_LAUNCH(BC, GE, SW) launch<BC, GE, SW>(g, ma, mb, mc, p, grid, ctx.device, stream)
     if (swap) {
@@ -2001,8 +2279,15 @@ cudaError_t launch_r4_multi_dst(const GemmArgs& g, void* const* C, const int64_t
 bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& pl)
 {
     if (pl.kernel < 0 || pl.kernel > 2 || pl.splits < 0 || pl.split_via < 0 || pl.split_via > 2 || pl.group_m < 0 ||
-        pl.group_m > 1024 || pl.half_tail < 0 || pl.half_tail > 2)
+        pl.group_m > 1024 || pl.half_tail < 0 || pl.half_tail > 2 || pl.tile_n < 0 || pl.tail_n < 0 || pl.stages < 0)
         return false;
+    // tile widths: the pair kernel takes multiples of 64 columns (and a second, narrower width for the tiles
+    // that balance its last wave)
+    if (pl.tile_n != 0 && (pl.tile_n < 64 || pl.tile_n > 256 || pl.tile_n % 64 != 0)) return false;
+    if (pl.tail_n != 0 && (pl.tail_n < 64 || pl.tail_n > 256 || pl.tail_n % 64 != 0 || pl.tail_n > (pl.tile_n ? pl.tile_n : 256)))
+        return false;
+    if ((pl.tile_n != 0 || pl.tail_n != 0) && pl.kernel != 2) return false;
+    if (pl.stages != 0) return false;
     if (g.M <= 0 || g.N <= 0 || g.K <= 0) return true;   // nothing to launch; any plan is moot
     const int64_t tiles = static_cast<int64_t>((g.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
     const int nkb = (g.K + BK - 1) / BK;
@@ -2023,7 +2308,8 @@ int r4_enumerate_plans(const GemmArgs& g, const RunContext& ctx, R4Plan* out, in
         if (n >= cap || !r4_plan_valid(g, ctx, pl)) return;
         for (int i = 0; i < n; ++i)
             if (out[i].kernel == pl.kernel && out[i].splits == pl.splits && out[i].split_via == pl.split_via &&
-                out[i].group_m == pl.group_m && out[i].half_tail == pl.half_tail)
+                out[i].group_m == pl.group_m && out[i].half_tail == pl.half_tail && out[i].tile_n == pl.tile_n &&
+                out[i].tail_n == pl.tail_n && out[i].stages == pl.stages)
                 return;
         out[n++] = pl;
     };
@@ -2066,7 +2352,7 @@ int r4_enumerate_plans(const GemmArgs& g, const RunContext& ctx, R4Plan* out, in
             pl.splits = s;
             pl.split_via = 1;
             push(pl);
-            if (swap && g.M <= 32 && (s == 2 || s == 4 || s == 8)) {
+            if ((!swap || g.M <= 32) && (s == 2 || s == 4 || s == 8)) {
                 pl.split_via = 2;
                 push(pl);
             }
@@ -2174,10 +2460,17 @@ extern "C" klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype
         cudaGetLastError();
         return KLINEAGE_ERR_INVALID_ARG;
     }
+    // (before the symbol lookup: the library image holds sm_100a code only, so on any other device the
+    // lookup itself fails and would hide the real reason)
+    int cc_major = 0;
+    if (cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess) {
+        cudaGetLastError();
+        return KLINEAGE_ERR_INTERNAL;
+    }
+    if (cc_major != 10) return KLINEAGE_ERR_UNSUPPORTED_DEVICE;
     NoAllocDevice* d = nullptr;
     const klineage_status_t st = noalloc_setup(device, &d);
     if (st != KLINEAGE_OK) return st;
-    if (d->ctx.cc_major != 10) return KLINEAGE_ERR_UNSUPPORTED_DEVICE;
 
     GemmArgs g;
     g.M = static_cast<int>(M);

@@ -71,6 +71,15 @@ struct PairParams {
     int kid;
     int group_m;
     int64_t total_tiles;
+    // Column tiling of a single problem (MODE 0 / 3): per tile row, n_wide tiles of tile_n columns followed by
+    // n_narrow tiles of tile_n2 columns (the last one clipped by N).  Wide tiles come first in the schedule and
+    // the pairs walk it back and forth, so that a pair's turns add up to about the same work (see
+    // plan_columns): the narrow tiles fill what would otherwise be an under-filled last wave.
+    int tile_n, n_wide, tile_n2, n_narrow;
+    int64_t wide_tiles;         // tiles_m2 * n_wide
+    int snake;                  // 1: odd rounds of the schedule run over the pairs in reverse order
+    uint32_t stage_tx;          // bytes the loads of both CTAs deliver per stage
+    int b_boxes;                // row-major B: 64-column boxes per CTA and stage (1 or 2)
     uint32_t idesc;
     uint32_t b_desc_hi, b_desc_lbo, b_kstep;
     // batched launches (MODE 1): the schedule runs over batch x tiles_per_batch
@@ -87,6 +96,7 @@ struct PairParams {
 // What a role needs to know about one tile of the schedule.
 struct TileInfo {
     int m0, n0;                 // first row of this CTA's first row block / first column of the pair tile
+    int width;                  // columns of the tile (the MMA's N): a multiple of 64, at most 256
     int M, N, nkb;              // extent of the problem the tile belongs to
     int z;                      // batch index (third tensor-map coordinate), 0 otherwise
     int epi_tma;
@@ -247,6 +257,8 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             x.C = static_cast<uint8_t*>(e->C);
             x.ldc = e->ldc;
             raster_tile(ti - gstart[gi], e->tiles_m, e->tiles_n, tm, tn, p.group_m);
+            x.n0 = tn * PN;
+            x.width = PN;
         } else {
             x.M = g.M;
             x.N = g.N;
@@ -262,15 +274,32 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 x.z = static_cast<int>(b);
                 x.C = static_cast<uint8_t*>(g.C) + static_cast<int64_t>(b) * p.stride_c_bytes;
                 raster_tile(t32 - b * tpb, p.tiles_m2, p.tiles_n, tm, tn, p.group_m);
+                x.n0 = tn * PN;
+                x.width = PN;
             } else {
                 x.z = 0;
                 x.C = static_cast<uint8_t*>(g.C);
-                raster_tile(t, p.tiles_m2, p.tiles_n, tm, tn, p.group_m);
+                if (t < p.wide_tiles) {
+                    raster_tile(t, p.tiles_m2, p.n_wide, tm, tn, p.group_m);
+                    x.n0 = tn * p.tile_n;
+                    x.width = p.tile_n;
+                } else {
+                    raster_tile(t - p.wide_tiles, p.tiles_m2, p.n_narrow, tm, tn, p.group_m);
+                    x.n0 = p.n_wide * p.tile_n + tn * p.tile_n2;
+                    x.width = p.tile_n2;
+                }
+                // a tile clipped by the matrix edge runs a narrower MMA
+                x.width = min(x.width, (g.N - x.n0 + 63) & ~63);
             }
         }
         x.m0 = tm * TILE_M + static_cast<int>(rank) * PM;   // this CTA's rows: m0 + [0,128) and m0 + 256 + [0,128)
-        x.n0 = tn * PN;
         return x;
+    };
+    // The r-th tile of this pair (-1: the schedule has ended).  Odd rounds run over the pairs in reverse
+    // when the schedule mixes tile widths: a pair that took an early (wide) tile takes a late (narrow) one next.
+    auto tile_at = [&](uint32_t r) -> int64_t {
+        const int64_t idx = static_cast<int64_t>(r) * n_pairs + ((p.snake && (r & 1u)) ? n_pairs - 1 - pair_id : pair_id);
+        return idx < p.total_tiles ? idx : -1;
     };
     // One operand box of a stage; completion is counted on the even CTA's barrier.
     auto load_box = [&](void* dst, const CUtensorMap* map, int c0, int c1, int z, uint32_t bar) {
@@ -289,10 +318,12 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int64_t t = pair_id; t < p.total_tiles && ok; t += n_pairs) {
+            for (uint32_t r = 0; ok; ++r) {
+                const int64_t t = tile_at(r);
+                if (t < 0) break;
                 const TileInfo x = tile_info(t);
                 const int m0 = x.m0;
-                const int nb = x.n0 + static_cast<int>(rank) * (PN / 2);    // this CTA's half of B
+                const int nb = x.n0 + static_cast<int>(rank) * (x.width >> 1);    // this CTA's half of B
                 for (int kb = 0; kb < x.nkb; ++kb, ++it) {
                     const int s = it % STAGES;
                     if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
@@ -304,7 +335,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     uint8_t* sa = smem + s * kStageBytes;
                     uint8_t* sb = sa + kABytes;
                     // The even CTA's barrier counts the bytes of both CTAs' loads of this stage.
-                    if (rank == 0) ptx::mbar_arrive_expect_tx(&full[s], 2 * kStageBytes);
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
                     const uint32_t bar = ptx::map_to_cta(ptx::smem_u32(&full[s]), 0);
                     load_box(sa, x.ma, kb * BK, m0, x.z, bar);
                     load_box(sa + kABlockBytes, x.ma, kb * BK, m0 + 2 * PM, x.z, bar);
@@ -312,7 +343,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                         load_box(sb, x.mb, kb * BK, nb, x.z, bar);
                     } else {
                         load_box(sb, x.mb, nb, kb * BK, x.z, bar);
-                        load_box(sb + 64 * BK * 2, x.mb, nb + 64, kb * BK, x.z, bar);
+                        if (p.b_boxes > 1) load_box(sb + 64 * BK * 2, x.mb, nb + 64, kb * BK, x.z, bar);
                     }
                 }
             }
@@ -329,7 +360,9 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             // -------------------------------------------------------- MMA issuer (even CTA)
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            for (int64_t t = pair_id; t < p.total_tiles && ok; t += n_pairs, ++tcount) {
+            for (;ok; ++tcount) {
+                const int64_t t = tile_at(tcount);
+                if (t < 0) break;
                 // Both accumulators are rewritten: wait until both CTAs' epilogues drained the last tile.
                 if (!ptx::mbar_wait(&acc_empty[0], (tcount & 1) ^ 1, abort_flag)) {
                     report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x520u);
@@ -337,7 +370,10 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     break;
                 }
                 ptx::tc_fence_after_sync();
-                const int nkb = (MODE == 2) ? tile_info(t).nkb : p.nkb;
+                const TileInfo x = tile_info(t);
+                const int nkb = x.nkb;
+                // the MMA's N is the tile's width
+                const uint32_t idesc = (p.idesc & ~(0x3Fu << 17)) | (static_cast<uint32_t>(x.width >> 3) << 17);
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t par = (it / STAGES) & 1;
@@ -357,9 +393,9 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                         const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
                         // alternate the two row blocks: consecutive MMAs never share an accumulator
                         umma_f16_pair(tmem_base, a_desc + static_cast<uint64_t>(k4 * 2),
-                                      b_desc + static_cast<uint64_t>(k4 * p.b_kstep), p.idesc, acc);
+                                      b_desc + static_cast<uint64_t>(k4 * p.b_kstep), idesc, acc);
                         umma_f16_pair(tmem_base + PN, a_desc + static_cast<uint64_t>((kABlockBytes >> 4) + k4 * 2),
-                                      b_desc + static_cast<uint64_t>(k4 * p.b_kstep), p.idesc, acc);
+                                      b_desc + static_cast<uint64_t>(k4 * p.b_kstep), idesc, acc);
                     }
                     umma_commit_pair(ptx::smem_u32(&empty[s]));
                     umma_commit_pair(ptx::map_to_cta(ptx::smem_u32(&empty[s]), 1));
@@ -385,7 +421,9 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         const int cpc = out_bf16 ? 64 : 32;                   // columns per 128-byte staging row
         uint32_t tcount = 0;
         bool ok = true;
-        for (int64_t t = pair_id; t < p.total_tiles && ok; t += n_pairs, ++tcount) {
+        for (; ok; ++tcount) {
+            const int64_t t = tile_at(tcount);
+            if (t < 0) break;
             const TileInfo x = tile_info(t);
             const int m0 = x.m0, n0 = x.n0;
             float* dst_f = reinterpret_cast<float*>(x.C);
@@ -399,7 +437,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             ptx::tc_fence_after_sync();
             const int row0 = m0 + mb * 2 * PM + q * 32;
             const int rows = min(32, x.M - row0);
-            const int nunits = (row0 < x.M) ? (min(PN, x.N - n0) + cpc - 1) / cpc : 0;
+            const int nunits = (row0 < x.M) ? (min(x.width, x.N - n0) + cpc - 1) / cpc : 0;
             const uint32_t tbase = tmem_base + mb * PN + (static_cast<uint32_t>(q * 32) << 16);
 
             auto release = [&]() {
@@ -572,7 +610,8 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 }
             }
         }
-        if (p.epi_tma && lane == 0) ptx::tma_store_wait_all<0>();
+        // shared memory may go once the stores have read it; their writes complete with the grid
+        if (p.epi_tma && lane == 0) ptx::tma_store_wait_read<0>();
     }
 
     // No CTA leaves while its partner may still signal into its shared memory.
@@ -695,6 +734,8 @@ cudaError_t launch_r4_pair_batched(const GemmArgs& g, const BatchArgs& b, RunCon
     p.tiles_n = (g.N + PN - 1) / PN;
     p.tiles_per_batch = p.tiles_m2 * p.tiles_n;
     p.total_tiles = static_cast<int64_t>(p.tiles_per_batch) * b.batch;
+    p.stage_tx = 2 * kStageBytes;
+    p.b_boxes = 2;
     p.nkb = (g.K + BK - 1) / BK;
     const int celt = g.c_bf16 ? 2 : 4;
     p.stride_c_bytes = b.stride_c * celt;
@@ -792,6 +833,8 @@ cudaError_t launch_r4_pair_grouped(const GemmArgs* groups, int n, RunContext& ct
     p.groups = static_cast<const GroupEntry*>(ctx.workspace);
     p.n_groups = n;
     p.total_tiles = tile_start;
+    p.stage_tx = 2 * kStageBytes;
+    p.b_boxes = 2;
     p.epi_tma = any_tma ? 1 : 0;
     p.kid = kIdTcgen05 + (any_tma ? 0 : 2) + 32 + ctx.kid_flags;
     *kernel_id = p.kid;
@@ -807,6 +850,78 @@ cudaError_t launch_r4_pair_grouped(const GemmArgs* groups, int n, RunContext& ct
 namespace {
 cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const int64_t* dst_ldc, int n_dst,
                                     RunContext& ctx, cudaStream_t stream, int* kernel_id);
+
+// Column tiling of one problem on the pair kernel (paper, Table 1 `templatize` / `autotune`: the tile shape is a
+// recipe parameter).  tile_n == 0: the pinned widths cannot run.
+struct PairColumns {
+    int tile_n, n_wide, tile_n2, n_narrow;
+    double cycles;      // estimated tensor-pipe cycles of the launch
+};
+
+// Tensor-pipe cycles of one k-block of a 512-row pair tile `w` columns wide (eight MMAs, two accumulators
+// alternating), measured with uniform-width launches.
+double pair_kblock_cycles(int w)
+{
+    return w >= 128 ? 4.0 * w : 512.0;
+}
+
+// Makespan (cycles) of the static schedule: tiles in schedule order (all wide ones, then the narrow ones),
+// dealt to `pairs` CTA pairs round by round, odd rounds in reverse order when widths are mixed.
+double pair_makespan(int64_t n_wide_tiles, int64_t n_narrow_tiles, double c_wide, double c_narrow, int64_t pairs)
+{
+    const int64_t total = n_wide_tiles + n_narrow_tiles;
+    const bool snake = n_wide_tiles > 0 && n_narrow_tiles > 0;
+    double worst = 0.0;
+    // a pair's load depends only on its position; positions 0, pairs-1 and those next to the wide / narrow
+    // boundary of each round bound the maximum, but the count is small: evaluate every pair
+    for (int64_t q = 0; q < pairs; ++q) {
+        double t = 0.0;
+        for (int64_t r = 0; r * pairs < total; ++r) {
+            const int64_t idx = r * pairs + ((snake && (r & 1)) ? pairs - 1 - q : q);
+            if (idx >= total) break;
+            t += idx < n_wide_tiles ? c_wide : c_narrow;
+        }
+        if (t > worst) worst = t;
+    }
+    return worst;
+}
+
+PairColumns plan_columns(const GemmArgs& g, const RunContext& ctx)
+{
+    const int64_t tiles_m2 = (g.M + TILE_M - 1) / TILE_M;
+    const int64_t nkb = (g.K + BK - 1) / BK;
+    const int64_t pairs = ctx.sm_count / 2 > 0 ? ctx.sm_count / 2 : 1;
+    const double per_tile = 5000.0;        // cycles per tile that the main loop does not hide
+    auto valid_w = [](int w) { return w >= 64 && w <= PN && w % 64 == 0; };   // whole 128-byte store units in either C type
+    const int wide = ctx.plan.tile_n > 0 ? ctx.plan.tile_n : PN;
+    PairColumns best = {0, 0, 0, 0, 0.0};
+    if (!valid_w(wide)) return best;
+    auto consider = [&](int n_wide, int w2) {
+        const int64_t rest = static_cast<int64_t>(g.N) - static_cast<int64_t>(n_wide) * wide;
+        const int n_narrow = rest > 0 ? static_cast<int>((rest + w2 - 1) / w2) : 0;
+        if (n_wide + n_narrow > 0x3FFFFF) return;
+        const double cw = nkb * pair_kblock_cycles(wide) + per_tile, cn = nkb * pair_kblock_cycles(w2) + per_tile;
+        const double t = pair_makespan(tiles_m2 * n_wide, tiles_m2 * n_narrow, cw, cn, pairs);
+        // (a mixed schedule has to win by 2 %: its narrow MMAs run below the full rate and it re-reads more of B)
+        const double score = (n_narrow > 0 && n_wide > 0) ? t * 1.02 : t;
+        if (best.tile_n == 0 || score < best.cycles) best = {wide, n_wide, n_narrow > 0 ? w2 : 0, n_narrow, score};
+    };
+    const int all_wide = static_cast<int>((static_cast<int64_t>(g.N) + wide - 1) / wide);
+    consider(all_wide, wide);              // uniform tiles
+    if (ctx.plan.tail_n == wide) return best;
+    if (ctx.plan.tail_n > 0 && !valid_w(ctx.plan.tail_n)) return PairColumns{0, 0, 0, 0, 0.0};
+    if (ctx.plan.tail_n > 0) best.tile_n = 0;        // a pinned narrow width must be used
+    for (int w2 = 128; w2 < wide; w2 += 64) {
+        if (ctx.plan.tail_n > 0 && w2 != ctx.plan.tail_n) continue;
+        if (tiles_m2 * all_wide <= pairs && ctx.plan.tail_n == 0) break;      // one round: nothing to balance
+        const int lo = all_wide > 24 ? all_wide - 24 : 0;
+        for (int n_wide = all_wide - 1; n_wide >= lo; --n_wide) consider(n_wide, w2);
+    }
+    if (ctx.plan.tail_n > 0 && ctx.plan.tail_n < 128 && best.tile_n == 0) {
+        for (int n_wide = all_wide - 1; n_wide >= 0 && n_wide >= all_wide - 24; --n_wide) consider(n_wide, ctx.plan.tail_n);
+    }
+    return best;
+}
 }
 
 cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
@@ -831,9 +946,22 @@ cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const
     PairParams p;
     memset(&p, 0, sizeof p);
     p.tiles_m2 = (g.M + TILE_M - 1) / TILE_M;
-    p.tiles_n = (g.N + PN - 1) / PN;
-    p.total_tiles = static_cast<int64_t>(p.tiles_m2) * p.tiles_n;
     p.nkb = (g.K + BK - 1) / BK;
+    const PairColumns cols = plan_columns(g, ctx);
+    if (cols.tile_n == 0) return cudaErrorInvalidValue;
+    p.tile_n = cols.tile_n;
+    p.n_wide = cols.n_wide;
+    p.tile_n2 = cols.tile_n2;
+    p.n_narrow = cols.n_narrow;
+    p.tiles_n = cols.n_wide + cols.n_narrow;
+    p.wide_tiles = static_cast<int64_t>(p.tiles_m2) * p.n_wide;
+    p.total_tiles = static_cast<int64_t>(p.tiles_m2) * p.tiles_n;
+    p.snake = cols.n_narrow > 0 && cols.n_wide > 0 ? 1 : 0;
+    // every tile loads a B box as wide as the widest tile's half (a narrower tile ignores the rest)
+    const int widest = cols.n_wide > 0 ? cols.tile_n : cols.tile_n2;
+    const uint32_t b_box_rows = static_cast<uint32_t>(widest / 2);
+    p.b_boxes = (widest / 2 + 63) / 64;
+    p.stage_tx = 2u * (kABytes + (g.b_col ? b_box_rows * 128u : static_cast<uint32_t>(p.b_boxes) * 8192u));
     p.group_m = ctx.plan.group_m > 0 ? ctx.plan.group_m : 4;   // default: 4 x 512 rows per raster group
     const int celt = g.c_bf16 ? 2 : 4;
     // (row length a multiple of 16 bytes too: a store box ending inside a 16-byte unit at the tensor's
@@ -875,7 +1003,7 @@ cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const
     bool ok = encode_map_2d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, PM,
                             CU_TENSOR_MAP_SWIZZLE_128B);
     if (g.b_col)
-        ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, PN / 2,
+        ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, b_box_rows,
                                  CU_TENSOR_MAP_SWIZZLE_128B);
     else
         ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, g.ldb * 2, 64, BK,

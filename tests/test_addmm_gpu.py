@@ -24,11 +24,14 @@ def kb():
     return binding
 
 
-def run_addmm(kb, case, bias_bits, variant, workspace_bytes=0):
+def run_addmm(kb, case, bias_bits, variant, workspace_bytes=0, pin=None):
     import torch
     dev = P.DeviceCase(case)
     bias = P.DeviceBuffer(bias_bits.size * 2, 2).upload(bias_bits)       # element-aligned only
     with kb.Gemm(0, b_col_major=case.b_col_major, c_bf16=case.c_bf16, workspace_bytes=workspace_bytes) as g:
+        if pin is not None:
+            g.set_plan(kb.klineage_gemm_plan_t(*pin), dev.a.ptr, dev.b.ptr, dev.c.ptr, case.M, case.N, case.K, case.lda,
+                       case.ldb, case.ldc)
         g.run_addmm(dev.a.ptr, dev.b.ptr, bias.ptr, dev.c.ptr, case.M, case.N, case.K, case.lda, case.ldb,
                     case.ldc, variant)
         torch.cuda.synchronize()
@@ -99,7 +102,7 @@ def test_addmm_large_tensor_core_paths(kb):
 @pytest.mark.parametrize("shape", [(256, 512, 8192, 0), (200, 700, 9000, 0), (130, 264, 12000, 1)],
                          ids=lambda s: "x".join(map(str, s[:3])))
 def test_addmm_through_the_workspace_split(kb, shape):
-    # few tiles, long K: the heuristic splits K through the workspace; the bias must be added once, by the
+    # few tiles, long K, K split through the workspace (pinned): the bias must be added once, by the
     # reduce - on its test-free path (whole rows of tiles inside an aligned C) and on the general one
     M, N, K, pad = shape
     for bf in (False, True):
@@ -107,9 +110,26 @@ def test_addmm_through_the_workspace_split(kb, shape):
                              name=f"addmm-split{M}x{N}x{K}")
         bias = gen.draw((1, N), "integer", 271, 2)[0]
         C_ref, S = reference(case, bias, np.arange(M))
-        vals, bits, kid = run_addmm(kb, case, bias, 4)
-        assert (kid - 400) & 4, kid
+        vals, bits, kid = run_addmm(kb, case, bias, 4, pin=(1, 6, 1))
+        assert (kid - 400) & ~(3 | 64) == 4, kid
         P.assert_matches_oracle(case, vals, bits, C_ref, S, exact=True, what=case.name)
+
+
+@pytest.mark.parametrize("shape", [(256, 512, 8192, 0), (200, 700, 9000, 0), (130, 264, 12000, 1)],
+                         ids=lambda s: "x".join(map(str, s[:3])))
+def test_addmm_through_the_cluster_split(kb, shape):
+    # the same shapes with the K splits of a tile as a cluster: the owner CTA of a block adds the bias once, after
+    # the partial sums; TMA-stored and masked-store forms, the heuristic's own choice and pinned cluster sizes
+    M, N, K, pad = shape
+    for bf in (False, True):
+        case = gen.make_case(M, N, K, seed=272, dist_a="integer", dist_b="integer", c_bf16=bf, ldc=N + pad,
+                             name=f"addmm-csplit{M}x{N}x{K}")
+        bias = gen.draw((1, N), "integer", 273, 2)[0]
+        C_ref, S = reference(case, bias, np.arange(M))
+        for pin in (None, (1, 2, 2), (1, 4, 2), (1, 8, 2)):
+            vals, bits, kid = run_addmm(kb, case, bias, 4, pin=pin)
+            assert (kid - 400) & ~(3 | 64) == (4 | 16), (kid, pin)
+            P.assert_matches_oracle(case, vals, bits, C_ref, S, exact=True, what=f"{case.name} {pin}")
 
 
 def test_addmm_argument_errors(kb):

@@ -58,7 +58,7 @@ def test_every_candidate_plan_matches_the_oracle(kb, shape):
         dev = P.DeviceCase(case)
         with kb.Gemm(0, b_col_major=col, c_bf16=bf) as g:
             plans = g.plan_candidates(*shape_args(case, dev))
-            assert len(plans) >= 2 and plans[0].as_tuple() == (0, 0, 0, 0, 0)
+            assert len(plans) >= 2 and not any(plans[0].as_tuple())
             assert len({p.as_tuple() for p in plans}) == len(plans), "duplicate candidates"
             unsplit = {}
             kernels = set()
@@ -100,7 +100,7 @@ def test_autotune_pins_a_candidate_and_later_calls_use_it(kb):
         torch.cuda.synchronize()
         assert best.as_tuple() in plans
         assert 0.0 < best_us <= heur_us
-        if best.as_tuple() != (0, 0, 0, 0, 0):
+        if any(best.as_tuple()):
             assert best_us <= 0.99 * heur_us, "a non-default plan must beat the heuristic by more than the noise"
         got, pinned = g.get_plan(*args)
         assert pinned and got.as_tuple() == best.as_tuple()
@@ -132,7 +132,9 @@ def test_plans_that_cannot_run_are_refused(kb):
                                                          case.ldb, dev.c.ptr, case.ldc, plan)
         bad = [Plan(2, 1, 0, 0, 0),      # pair kernel: pitch of A (260 elements) is not 16-byte aligned
                Plan(1, 9, 1, 0, 0),      # 9 splits of 5 k-blocks
-               Plan(1, 2, 2, 0, 0),      # cluster reduce needs the skinny orientation
+               Plan(1, 3, 2, 0, 0),      # a cluster reduce runs in 2, 4 or 8 CTAs
+               Plan(1, 1, 0, 0, 0, 96),  # tile widths are multiples of 64 columns
+               Plan(1, 1, 0, 0, 0, 0, 0, 5),   # ring depths: 0 (automatic), 4 or 6
                Plan(3, 0, 0, 0, 0), Plan(0, -1, 0, 0, 0), Plan(0, 0, 3, 0, 0), Plan(0, 0, 0, 0, 3)]
         for plan in bad:
             assert raw(plan) == kb.KLINEAGE_ERR_INVALID_ARG, plan

@@ -165,7 +165,7 @@ SKINNY = [  # (M, N, K, expected flags of kernel id - 400: 4 split-K, 8 swapped 
     (32, 1000, 4096, 4 | 8 | 16),      # M = 32: largest cluster-reduced M, ragged N
     (33, 1000, 4096, 4 | 8),           # M = 33: swapped, split through the global workspace
     (64, 520, 2048, 4 | 8),            # M = 64: last swapped M
-    (65, 520, 32768, 4),               # M = 65: regular orientation, K long enough for split-K with row-block reduce
+    (65, 520, 32768, 4 | 16),          # M = 65: regular orientation, K long enough for a split: cluster of 8, reduce through the rings
     (16, 256, 64, 8),                  # one tile, one k-block: no split
     (1, 8192, 8192, 4 | 8 | 16),       # GEMV
 ]
@@ -188,6 +188,49 @@ def test_tcgen05_skinny_modes(handles, col):
                          ldb=(4099 if col else 1001) + 2, ldc=1003, name="skinny-unaligned")
     run_and_check(handles, case, 4, exact=True, offsets=(1, 1, 1))
     assert (handles[(col, False)].last_kernel_id() - 400) & 64, "unaligned operands that fit are repacked"
+
+
+# ------------------------------------------------------------------ K splits of 128-row tiles
+REGULAR_SPLIT = [  # (M, N, K, (pad of lda, ldb, ldc)): few 128-row tiles, K long enough to split
+    (256, 256, 8192, (0, 0, 0)),       # two whole tiles, C stored by TMA
+    (384, 512, 1536, (0, 0, 0)),       # six tiles
+    (130, 300, 1000, (0, 0, 0)),       # ragged M, N and K; a bf16 row ends inside a 16-byte unit: masked stores
+    (200, 700, 3000, (8, 8, 1)),       # odd pitch of C: masked stores for both C types
+    (65, 520, 4096, (0, 0, 0)),        # first M of the regular orientation: three of four row blocks empty
+    (128, 256, 16384, (0, 0, 0)),      # one tile, very long K
+]
+
+
+@pytest.mark.parametrize("col", [False, True], ids=["Brow", "Bcol"])
+def test_tcgen05_regular_split_routes(handles, handles_tiny_ws, col):
+    """The K splits of a 128-row tile as a cluster (partials exchanged through the operand rings, owner CTAs reduce
+    in rank order) in 2, 4 and 8 CTAs, and through the global workspace; every route bit-exact on integers."""
+    for idx, (M, N, K, (pa, pb, pc)) in enumerate(REGULAR_SPLIT):
+        for bf in (False, True):
+            case = gen.make_case(M, N, K, seed=300 + idx, dist_a="integer", dist_b="integer", b_col_major=col,
+                                 c_bf16=bf, lda=K + pa, ldb=(K if col else N) + pb, ldc=N + pc,
+                                 name=f"rsplit{M}x{N}x{K}-int")
+            C_ref, S = P.oracle_rows(case, np.arange(M))
+            for splits, via in ((2, 2), (4, 2), (8, 2), (3, 1), (4, 1)):
+                run_and_check(handles, case, 4, C_ref, S, np.arange(M), exact=True, pin=(1, splits, via))
+                got = (handles[(col, bf)].last_kernel_id() - 400) & ~(3 | 64)
+                assert got == (4 | (16 if via == 2 else 0)), (M, N, K, splits, via, got)
+        # random values: inside the bound, and two runs of the cluster route agree bit for bit
+        case = gen.make_case(M, N, K, seed=300 + idx, dist_a="normal", dist_b="uniform", b_col_major=col,
+                             lda=K + pa, ldb=(K if col else N) + pb, ldc=N + pc, name=f"rsplit{M}x{N}x{K}")
+        C_ref, S = P.oracle_rows(case, np.arange(M))
+        _, b1 = run_and_check(handles, case, 4, C_ref, S, np.arange(M), pin=(1, 4, 2))
+        _, b2 = run_and_check(handles, case, 4, C_ref, S, np.arange(M), pin=(1, 4, 2))
+        assert np.array_equal(b1, b2), "two runs of the cluster reduce differ"
+    # unpinned: the heuristic takes the cluster route for few tiles and long K
+    case = gen.make_case(256, 256, 8192, seed=310, dist_a="integer", dist_b="integer", b_col_major=col, c_bf16=True)
+    run_and_check(handles, case, 4, exact=True)
+    assert (handles[(col, True)].last_kernel_id() - 400) & ~3 == (4 | 16)
+    # unaligned operands and no room to repack them: the gathering producers feed the cluster route too
+    case = gen.make_case(130, 270, 2100, seed=311, dist_a="integer", dist_b="integer", b_col_major=col, lda=2101,
+                         ldb=(2101 if col else 271), ldc=271, name="rsplit-generic")
+    run_and_check(handles_tiny_ws, case, 4, exact=True, offsets=(1, 1, 1), pin=(1, 4, 2))
+    assert (handles_tiny_ws[(col, False)].last_kernel_id() - 400) == (1 | 2 | 4 | 16)
 
 
 # ------------------------------------------------------------------ CTA-pair form of the top rung
@@ -240,7 +283,7 @@ MIDSIZE = [  # (M, N, K): what the shape exercises on the tcgen05 rung
     (1500, 2100, 333),    # 12 x 9 tiles on 148 SMs: single under-filled wave cut into half tiles, N tail inside a half
     (2304, 5120, 200),    # 360 tiles: two full waves + a 64-tile tail cut into half tiles
     (3000, 2900, 150),    # 24 x 12 = 288 tiles: 140-tile tail, too full for half tiles
-    (200, 700, 30000),    # 2 x 3 tiles, very long K: split-K through the workspace, row-block reduce, M tail
+    (200, 700, 30000),    # 2 x 3 tiles, very long K: split along K (a cluster per tile), M tail
     (130, 8192, 1024),    # 2 x 32 tiles of 128 rows, half tiles
     (4200, 4352, 136),    # CTA pairs: last 512-row tile has 104 rows (second row block and odd CTA empty)
     (1024, 9000, 96),     # wide N with a tail, K tail

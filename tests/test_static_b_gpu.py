@@ -10,13 +10,17 @@ from tests import parity as P
 
 pytestmark = pytest.mark.gpu
 
-SHAPES = [  # M, N, K, col, bf16
-    (16, 2048, 4096, False, False),     # skinny, cluster reduce, single wave
-    (48, 1024, 8192, True, True),       # skinny, workspace split
-    (300, 520, 1024, False, True),      # single wave of 128 x 256 tiles
-    (1100, 2100, 264, True, False),     # more tiles than SMs would take in one wave? (45 tiles: one wave)
-    (2100, 4200, 136, False, True),     # multi-wave: the flag changes nothing there
-    (130, 263, 70, False, False),       # unaligned: repacked operands (the repack kernels precede the GEMM)
+SHAPES = [  # M, N, K, col, bf16, (pad of lda, ldb, ldc)
+    (16, 2048, 4096, False, False, (0, 0, 0)),     # skinny, cluster reduce, single wave
+    (48, 1024, 8192, True, True, (0, 0, 0)),       # skinny, workspace split
+    (300, 520, 1024, False, True, (0, 0, 0)),      # single wave of 128 x 256 tiles
+    (1100, 2100, 264, True, False, (0, 0, 0)),     # more tiles than SMs would take in one wave? (45 tiles: one wave)
+    (2100, 4200, 136, False, True, (0, 0, 0)),     # multi-wave: the flag changes nothing there
+    (130, 263, 70, False, False, (1, 1, 1)),       # unaligned: repacked operands (the repack kernels precede the GEMM)
+    # only B unaligned, K long enough for the early first ring fill, one wave: the library's own aligned copy of B
+    # is written by the repack kernel just ahead of the GEMM, so the early loads must not run ahead of it
+    (16, 2047, 4096, False, False, (0, 2, 0)),
+    (200, 519, 1024, True, True, (0, 3, 0)),
 ]
 
 
@@ -28,10 +32,9 @@ def kb():
 
 @pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s[:3])))
 def test_static_b_changes_no_bit(kb, shape):
-    M, N, K, col, bf = shape
-    pad = 1 if (M, N, K) == (130, 263, 70) else 0
+    M, N, K, col, bf, (pa, pb, pc) = shape
     case = gen.make_case(M, N, K, seed=190, dist_a="normal", dist_b="normal", b_col_major=col, c_bf16=bf,
-                         lda=K + pad, ldb=(K if col else N) + pad, ldc=N + pad, name=f"static{M}x{N}x{K}")
+                         lda=K + pa, ldb=(K if col else N) + pb, ldc=N + pc, name=f"static{M}x{N}x{K}")
     C_ref, S = P.oracle_rows(case, np.arange(M))
     out = []
     for static in (False, True):
@@ -41,6 +44,8 @@ def test_static_b_changes_no_bit(kb, shape):
                 dev.run(g, kb.KLINEAGE_TCGEN05, check=False)
             dev.run(g, kb.KLINEAGE_TCGEN05)
             vals, bits = dev.result()
+            if pb:
+                assert (g.last_kernel_id() - 400) & 64, "the unaligned B must have been repacked for this test to bite"
         P.assert_matches_oracle(case, vals, bits, C_ref, S, exact=False, what=f"{case.name} static_b={static}")
         out.append(bits)
     assert np.array_equal(out[0], out[1])
@@ -78,4 +83,4 @@ def test_a_produced_by_the_previous_call_is_waited_for(kb):
 
 def test_unknown_flag_bits_are_refused(kb):
     with pytest.raises(kb.KlineageError):
-        kb.klineage_gemm_create(0, kb.KLINEAGE_B_ROW_MAJOR, kb.KLINEAGE_C_F32, 0, 2)
+        kb.klineage_gemm_create(0, kb.KLINEAGE_B_ROW_MAJOR, kb.KLINEAGE_C_F32, 0, 4)

@@ -66,11 +66,52 @@ def test_no_alloc_matches_handle_path_on_two_calls_in_a_row():
             assert np.array_equal(got, want), case.name
 
 
+def test_no_alloc_unaligned_operands_empty_shapes_and_no_allocation():
+    """What the entry point promises beyond the aligned case: unaligned operands are accepted (gathered tile by
+    tile, where the handle path repacks them first) and give the exact result on integer-valued inputs; K == 0
+    zero-fills; M == 0 does nothing; and the device's free memory is the same after a call as before it."""
+    import torch
+    from paper_2605_28213_b200 import binding as kb
+    stream = torch.cuda.current_stream().cuda_stream
+    for (M, N, K, col, bf, offs) in ((130, 263, 1070, False, False, (1, 1, 1)), (300, 520, 200, True, True, (1, 0, 0))):
+        case = gen.make_case(M, N, K, seed=9, dist_a="integer", dist_b="integer", b_col_major=col, c_bf16=bf,
+                             lda=K + 1, ldb=(K if col else N) + 1, ldc=N + 1, name="no-alloc unaligned")
+        with kb.Gemm(0, b_col_major=col, c_bf16=bf) as g:
+            dev = P.DeviceCase(case, *offs)
+            dev.run(g, kb.KLINEAGE_TCGEN05)
+            _, want = dev.result()
+        d2 = P.DeviceCase(case, *offs)
+        args = (kb.KLINEAGE_B_COL_MAJOR if col else kb.KLINEAGE_B_ROW_MAJOR, kb.KLINEAGE_C_BF16 if bf else kb.KLINEAGE_C_F32,
+                M, N, K, d2.a.ptr, case.lda, d2.b.ptr, case.ldb, d2.c.ptr, case.ldc, stream)
+        assert kb.klineage_gemm_run_noalloc(*args) == kb.KLINEAGE_OK
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        assert kb.klineage_gemm_run_noalloc(*args) == kb.KLINEAGE_OK
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before, "the allocation-free call changed the free device memory"
+        vals, bits = d2.result()
+        C_ref, S = P.oracle_rows(case, np.arange(M))
+        P.assert_matches_oracle(case, vals, bits, C_ref, S, exact=True, what=case.name)
+        assert np.array_equal(bits, want), "exact sums: both paths must give the same bits"
+    # K == 0: C <- 0 through this entry point too; M == 0: nothing is written
+    case = gen.make_case(40, 50, 3, seed=1, ldc=53)
+    d3 = P.DeviceCase(case)
+    assert kb.klineage_gemm_run_noalloc(0, 0, 40, 50, 0, d3.a.ptr, 3, d3.b.ptr, 50, d3.c.ptr, 53, stream) == kb.KLINEAGE_OK
+    torch.cuda.synchronize()
+    assert np.all(d3.result()[1] == 0)
+    d4 = P.DeviceCase(case)
+    before = d4.c.download().copy()
+    assert kb.klineage_gemm_run_noalloc(0, 0, 0, 50, 3, d4.a.ptr, 3, d4.b.ptr, 50, d4.c.ptr, 53, stream) == kb.KLINEAGE_OK
+    torch.cuda.synchronize()
+    assert np.array_equal(d4.c.download(), before) and d4.c.guards_intact()
+
+
 def test_no_alloc_refuses_shapes_beyond_its_fixed_scratch():
     import torch
     from paper_2605_28213_b200 import binding as kb
-    # a K long enough to be split, and splits x 2048 x 1024 fp32 partial sums >= 16 MiB > the 8 MiB reserved
-    M, N, K = 2048, 1024, 65536
+    # 64 rows (partial sums go through global memory), K long enough for 9 splits:
+    # 9 x 64 x 4096 fp32 partial sums = 9 MiB > the 8 MiB reserved
+    M, N, K = 64, 4096, 32768
     A = torch.zeros(M * K, dtype=torch.int16, device="cuda")
     B = torch.zeros(K * N, dtype=torch.int16, device="cuda")
     C = torch.full((M * N,), 7.0, dtype=torch.float32, device="cuda")
