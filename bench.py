@@ -38,11 +38,21 @@ WORKLOADS = {
 }
 WORKLOAD = WORKLOADS["c4"]
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one tcgen05-rung launch at 8192^3
-# (ncu capture summarised in profiles/r4_tcgen05_c4_8192.md): 0.884 GB read + 0.141 GB written.
-R4_C4_DRAM_TRAFFIC_BYTES = 1.026e9
-# the same for the skinny shape (profiles/r4_tcgen05_c5_skinny.md): 134.6 MB read + 3.9 MB written.
-R4_C5_DRAM_TRAFFIC_BYTES = 1.385e8
+
+
+def measured_traffic(workload: str, variant: int):
+    """DRAM bytes per launch of the dominant kernel from the stored profiler capture of this workload, or None.
+
+    The figure is not measured by this program (it never runs under a profiler): it is read from the record kept
+    beside the profiler summaries, which names the capture and the commit it was taken at."""
+    try:
+        rec = json.loads((ROOT / "profiles" / "traffic.json").read_text()).get(workload)
+        if rec and int(rec.get("variant", -1)) == variant:
+            return float(rec["dram_bytes_per_launch"])
+    except Exception:
+        pass
+    return None
+
 VARIANT_NAMES = ["naive", "tiled", "vectorized", "pipelined", "tcgen05", "mma_sync"]
 LINEAGE_ORDER = [0, 1, 2, 3, 5, 4]     # rung 3.5 (mma.sync, variant id 5) sits between rungs 3 and 4
 
@@ -342,13 +352,13 @@ def run_gpu(args):
     if args.workload == "c5":
         gbs = case.algorithmic_bytes / (ms_per_step * 1e-3) / 1e9
         line["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                            "frac": gbs / peaks["hbm_gbs"], "traffic": R4_C5_DRAM_TRAFFIC_BYTES if V == 4 else None,
+                            "frac": gbs / peaks["hbm_gbs"], "traffic": measured_traffic("c5", V),
                             "peak_source": f"{peak_kind} (copy bandwidth)", "frac_of_nominal_8000": gbs / 8000.0,
                             "algorithmic_bytes_per_launch": case.algorithmic_bytes}
     else:
         line["roofline"] = {"bound": "tensor", "achieved": per_gpu, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                             "frac": per_gpu / peaks["bf16_tflops"],
-                            "traffic": R4_C4_DRAM_TRAFFIC_BYTES if (args.workload, V) == ("c4", 4) else None,
+                            "traffic": measured_traffic(args.workload, V),
                             "peak_source": f"{peak_kind} (burst cuBLAS bf16)",
                             "frac_of_sustained": per_gpu / peaks["bf16_tflops_sustained"],
                             "frac_of_nominal_2250": per_gpu / 2250.0,
@@ -363,6 +373,94 @@ def run_gpu(args):
     if rank == 0:
         print(json.dumps(line), flush=True)
     return 0 if (parity_ok and e2e_ok and code == 0) else 1
+
+
+def run_partitioned(args):
+    """--partition n: ONE GEMM partitioned by columns over the ranks, all-gather fused into the epilogue.
+
+    Every rank holds A and its column slice of B, multiplies them on the tcgen05 rung and its epilogue stores the
+    result slice into every rank's full-width C (peer stores only; no operand is loaded from a peer, no collective
+    follows).  Strong scaling: the job is one product whatever the number of ranks.  A step ends, for the timing,
+    when every rank's launch has completed (barrier + synchronize after the loop); every rank then checks sampled
+    rows of ITS OWN C - which all ranks wrote - against the oracle."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from oracle import gemm_oracle as orc
+    from paper_2605_28213_b200 import binding as kb
+    from paper_2605_28213_b200 import inputs as gen
+    from paper_2605_28213_b200 import npart
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    peaks, peak_kind = load_peaks()
+    case = gen.make_config(args.workload, 1)                  # the same problem on every rank
+    n0, n1 = npart.column_slice(case.N, world, rank)
+    B_slice = np.ascontiguousarray(case.B[n0:n1, :] if case.b_col_major else case.B[:, n0:n1])
+    ldb = case.K if case.b_col_major else max(n1 - n0, 1)
+    A = torch.from_numpy(case.A.view("int16")).to(device)
+    Bs = torch.from_numpy(B_slice.view("int16")).to(device)
+    shared = npart.SharedC(case.M, case.ldc, torch.int16 if case.c_bf16 else torch.float32, device, world, rank)
+    shared.local.zero_()
+    gemm = kb.Gemm(local, b_col_major=case.b_col_major, c_bf16=case.c_bf16)
+    part = npart.NPartitionedGemm(gemm, world, rank, case.N, shared.ptrs, case.ldc)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    barrier()
+    for _ in range(max(3, args.warmup)):
+        npart.partitioned_step(part, A, Bs, case.M, case.K, case.lda, ldb, args.variant)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        e0.record()
+        for _ in range(args.steps):
+            npart.partitioned_step(part, A, Bs, case.M, case.K, case.lda, ldb, args.variant)
+        e1.record()
+        barrier()
+    ms = max_over_ranks(e0.elapsed_time(e1), world, device) / args.steps
+    code, kid = gemm.device_status()
+    rows = np.array(sorted({(r * 977 + 13 + 31 * rank) % case.M for r in range(8)}))
+    C_ref, S = orc.gemm(len(rows), case.N, case.K, np.ascontiguousarray(case.A[rows]), case.lda, case.B, case.ldb,
+                        case.b_col_major)
+    got = shared.local[rows.tolist()][:, :case.N].cpu().numpy()
+    vals = gen.bf16_bits_to_f32(got.view(np.uint16)).astype(np.float64) if case.c_bf16 else got.astype(np.float64)
+    bound = orc.bound_bf16(case.K, S, C_ref) if case.c_bf16 else orc.bound_f32(case.K, S)
+    ok = bool(np.all(np.abs(vals - C_ref) <= bound)) and code == 0
+    ok_all = max_over_ranks(0.0 if ok else 1.0, world, device) == 0.0
+    tflops = case.flops / (ms * 1e-3) / 1e12
+    celt = 2 if case.c_bf16 else 4
+    line = {
+        "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "strong",
+        "vs_baseline": None, "dtype": "bf16 inputs, fp32 accumulate (tcgen05.mma kind::f16), bf16 C", "data": "synthetic",
+        "config": {"workload": WORKLOADS[args.workload], "variant": f"{VARIANT_NAMES[args.variant]} (rung {args.variant})",
+                   "parallelism": f"one GEMM partitioned by columns over {world} ranks; every rank's epilogue stores its "
+                                  f"slice into all {world} C matrices (peer stores, rendezvous: {shared.how})",
+                   "l2": "A + B slice + C exceed the L2; no flush between iterations"},
+        "clocks": clocks.summary(), "gpu_launches": args.steps * world, "parity_checked": ok_all, "device_status": code,
+        "kernel_id": kid, "e2e": None,
+        "exchange": {"bytes_stored_to_peers_per_rank_per_step": int((world - 1) * case.M * (n1 - n0) * celt),
+                     "bound_note": "stores leave over NVLink at <= 770 GB/s per direction (measured peer copy)"},
+        "roofline": {"bound": "tensor", "achieved": tflops / world, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": tflops / world / peaks["bf16_tflops"], "traffic": None,
+                     "peak_source": f"{peak_kind} (burst cuBLAS bf16)", "flops_per_launch": case.flops / world},
+    }
+    if world > 1:
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    return 0 if ok_all else 1
 
 
 def lineage_table(prob_c4, kb, gen, torch, device, peaks):
@@ -750,6 +848,9 @@ def main():
                     help="configuration to time (default: the headline 8192^3; others are for profiling)")
     ap.add_argument("--variant", type=int, default=4, choices=range(6),
                     help="lineage rung to time (default 4 = tcgen05; 5 = the mma.sync rung 3.5)")
+    ap.add_argument("--partition", default="replicas", choices=["replicas", "n"],
+                    help="N > 1: 'replicas' = independent GEMMs (default, weak scaling); 'n' = ONE GEMM partitioned by "
+                         "columns over the ranks with the all-gather fused into the epilogue (strong scaling)")
     ap.add_argument("--family", action="store_true",
                     help="time only the BMM / GroupedGEMM rows (for profiling) and print them as one JSON line")
     args = ap.parse_args()
@@ -764,6 +865,8 @@ def main():
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
         print(json.dumps({"gemm_family": family_table(kb, gen, torch, device, load_peaks()[0], flush)}), flush=True)
         return 0
+    if args.partition == "n":
+        return run_partitioned(args)
     return run_gpu(args)
 
 

@@ -424,12 +424,20 @@ klineage_status_t klineage_gemm_run_host(klineage_gemm_t h, int64_t M, int64_t N
  *   kernel     1 single-CTA kernel (128 x 256 tiles), 2 CTA-pair kernel (512 x 256 tiles)
  *   splits     number of K splits (1 = none)
  *   split_via  with splits > 1: 1 partial sums through the global workspace,
- *              2 through a thread-block cluster (M <= 32, splits 2 / 4 / 8)
+ *              2 through a thread-block cluster (splits 2 / 4 / 8; M <= 32 or M > 64)
  *   group_m    tile-rows per raster group (L2 reuse pattern)
  *   half_tail  1 cut the last wave into 128-column half tiles, 2 never
+ *   tile_n     columns per output tile (needs `kernel`): single-CTA kernel 256 or 128; CTA-pair kernel a
+ *              multiple of 64 up to 256
+ *   tail_n     CTA-pair kernel only: tile_n = every tile of that width; a smaller multiple of 64 = tile rows
+ *              start with tile_n-wide tiles and end with tiles of this width, dealt to the CTA pairs back and
+ *              forth so that wide and narrow turns balance a last, under-filled wave
+ *   stages     single-CTA kernel only: depth of the operand ring - 4, or 6 with 128-column tiles (32 KiB stages)
  * Every plan computes the same C up to fp32 summation order (plans that differ
- * only in kernel / group_m / half_tail are bit-identical; K splits change the
- * order of the partial sums and stay within the parity bound).
+ * only in kernel / group_m / half_tail / tile shape / stages are bit-identical; K
+ * splits change the order of the partial sums and stay within the parity bound).
+ *   split_via  2 also covers 128-row tiles (M > 64): the K splits of a tile then run as one cluster whose
+ *              CTAs exchange their partial tiles through the idle operand rings (one wave of clusters at most)
  *
  * A plan is pinned per handle for one (M, N, K) and alignment class of the
  * operands (16-byte alignment of base and pitch of A, B, C; the pointers are

@@ -56,6 +56,7 @@ constexpr int kStageBytes = kABytes + kBBytes;    // 48 KiB
 constexpr int kConvFilterBytes = (BN / 2) * BK * 2;                                  // 16 KiB
 constexpr int kConvStageBytes = kABytes + kConvFilterBytes;                          // 32 KiB
 constexpr int kConvStages = 6;
+constexpr int kMaxStages = 6;                     // deepest ring (32 KiB stages of 128-column tiles)
 static_assert(kConvStages * kConvStageBytes <= STAGES * kStageBytes, "conv ring exceeds the ring area");
 constexpr int kEpiBufBytes = 32 * 128;            // one 32-row x 128-byte staging block
 constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;   // 4 warps x 2 buffers
@@ -111,6 +112,11 @@ struct R4Params {
     // kernel's give-up path - error word, abort flag, every role leaving its loop, TMEM freed - really runs.
     int test_stop_after;
     uint32_t test_poll_limit;
+    // Tile width and ring depth (MODE 0, TMA-fed, regular orientation; every other form runs 256 columns and 4
+    // stages): 256 columns with four 48 KiB stages, or 128 columns with four or six 32 KiB stages.
+    int tile_n;
+    int n_stages;
+    uint32_t stage_bytes;
 };
 
 // One entry of the static schedule.
@@ -168,7 +174,8 @@ __device__ __forceinline__ Unit decode_unit(int64_t u, const R4Params& p)
 {
     Unit x;
     int half = 0;
-    x.ncols = BN;
+    const int tile_n = p.tile_n;
+    x.ncols = tile_n;
     if (p.cluster) {              // splits is a power of two: no division on the critical path of short kernels
         x.tile = u >> p.splits_log2;
         x.split = static_cast<int>(u & (p.splits - 1));
@@ -185,20 +192,20 @@ __device__ __forceinline__ Unit decode_unit(int64_t u, const R4Params& p)
         x.split = 0;
         if (p.half_only) {
             x.tile = u;
-            x.ncols = BN / 2;
+            x.ncols = tile_n / 2;
         } else if (u < p.full_units) {
             x.tile = u;
         } else {
             const int64_t v = u - p.full_units;
             x.tile = p.full_units + (v >> 1);
             half = static_cast<int>(v & 1);
-            x.ncols = BN / 2;
+            x.ncols = tile_n / 2;
         }
     }
     int tm, tn;
     raster_tile(x.tile, p.tiles_m, p.tiles_n, tm, tn, p.group_m);
     x.m0 = tm * BM;
-    x.n0 = tn * BN + half * (BN / 2);
+    x.n0 = tn * tile_n + half * (tile_n / 2);
     x.kb0 = x.split * p.kb_per_split;
     x.kb1 = min(p.nkb, x.kb0 + p.kb_per_split);
     return x;
@@ -237,8 +244,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* epi_smem = smem + STAGES * kStageBytes;
     uint64_t* full = reinterpret_cast<uint64_t*>(epi_smem + kEpiBytes);
-    uint64_t* empty = full + STAGES;
-    uint64_t* acc_full = empty + STAGES;
+    uint64_t* empty = full + kMaxStages;
+    uint64_t* acc_full = empty + kMaxStages;
     uint64_t* acc_empty = acc_full + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile uint32_t* abort_flag = tmem_slot + 1;   // [0] raised on give-up, [1] stays 0
@@ -247,6 +254,11 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     uint64_t* cfull = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(gstart) + 7) & ~uintptr_t(7));
     uint64_t* cempty = cfull + kConvStages;
     const bool ring6 = MODE == 4 && !GENERIC && p.conv_ring6;
+    // Ring geometry: a parameter of the plain TMA-fed GEMM only, the constants everywhere else
+    constexpr bool kTunable = MODE == 0 && !GENERIC && !SWAP;
+    const uint32_t NS = kTunable ? static_cast<uint32_t>(p.n_stages) : static_cast<uint32_t>(STAGES);
+    const uint32_t SB = kTunable ? p.stage_bytes : static_cast<uint32_t>(kStageBytes);
+    const int TN = kTunable ? p.tile_n : BN;
     int group_hint = 0;     // MODE 2: a thread's units come in increasing order; its group search resumes here
     // One unit of the schedule for this thread's role.
     auto unit_of = [&](int64_t u) {
@@ -287,7 +299,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         uint32_t it;
         bool live;
         int cw, ch, cn;                 // MODE 4 on TMA: input origin (w, h) and image of the tile's 8 x 16 pixel patch
-    } prod = {static_cast<int64_t>(blockIdx.x), 0, 0, 0, 0, 0, &map_a, &map_b, 0u, false, 0, 0, 0};
+        uint32_t st, ph;                // ring stage of load `it` and the parity its "empty" barrier is waited with
+    } prod = {static_cast<int64_t>(blockIdx.x), 0, 0, 0, 0, 0, &map_a, &map_b, 0u, false, 0, 0, 0, 0u, 1u};
     auto prod_enter_unit = [&]() {
         prod.live = prod.u < total_units;
         if (!prod.live) return;
@@ -324,14 +337,14 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 prod.live = false;
                 break;
             }
-            const int s = it % STAGES;
-            if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
+            const uint32_t s = prod.st;
+            if (!ptx::mbar_wait(&empty[s], prod.ph, abort_flag)) {
                 report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x400u | s);
                 abort_flag[0] = 1;
                 prod.live = false;
                 break;
             }
-            uint8_t* sa = smem + s * kStageBytes;
+            uint8_t* sa = smem + s * SB;
             uint8_t* sb = sa + kABytes;
             ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
             const CUtensorMap* pa = (MODE == 2) ? prod.ma : &map_a;
@@ -358,9 +371,13 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             } else {
 #pragma unroll
                 for (int cb = 0; cb < BN / 64; ++cb)
-                    load_box(sb + cb * (64 * BK * 2), pb, prod.n0 + cb * 64, prod.kb * BK, &full[s]);
+                    if (cb * 64 < TN) load_box(sb + cb * (64 * BK * 2), pb, prod.n0 + cb * 64, prod.kb * BK, &full[s]);
             }
             ++prod.it;
+            if (++prod.st == NS) {
+                prod.st = 0;
+                prod.ph ^= 1u;
+            }
             if (++prod.kb == prod.kb1) {
                 prod.u += gridDim.x;
                 prod_enter_unit();
@@ -369,7 +386,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     };
 
     if (warp == 0 && lane == 0) {
-        for (int s = 0; s < STAGES; ++s) {
+        for (uint32_t s = 0; s < NS; ++s) {
             ptx::mbar_init(&full[s], GENERIC ? kProducerThreads + ((MODE == 4 && p.conv_b_tma) ? 1 : 0) : 1);
             ptx::mbar_init(&empty[s], 1);
         }
@@ -410,7 +427,9 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             ptx::grid_dependency_wait();
             for (int s = 0; s < STAGES; ++s)
                 ptx::tma_load_2d(smem + s * kStageBytes, &map_a, (prod.kb + s) * BK, prod.m0, &full[s]);
-            prod.it = STAGES;
+            prod.it = STAGES;          // (the host grants this path to the 4-stage, 256-column form only)
+            prod.st = 0;
+            prod.ph ^= 1u;
             prod.kb += STAGES;
             if (prod.kb == prod.kb1) {
                 prod.u += gridDim.x;
@@ -421,7 +440,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             if (!GENERIC && MODE != 2) {
                 // The first ring fill needs nothing from the other warps: start it before the
                 // set-up barrier so that TMEM allocation hides behind the first loads' latency.
-                if (!ring6 && !(MODE == 4 && p.conv_t)) produce(STAGES);
+                if (!ring6 && !(MODE == 4 && p.conv_t)) produce(NS);
             }
         }
         if (blockIdx.x == 0) g.status[1] = p.kid;
@@ -548,8 +567,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             produce(0xFFFFFFFFu);
             // Drain: every load issued must have landed before shared memory is released.
             const uint32_t it = prod.it;
-            const uint32_t first = it > STAGES ? it - STAGES : 0;
-            for (uint32_t j = first; j < it; ++j) ptx::mbar_wait(&full[j % STAGES], (j / STAGES) & 1, abort_flag + 1);
+            const uint32_t first = it > NS ? it - NS : 0;
+            for (uint32_t j = first; j < it; ++j) ptx::mbar_wait(&full[j % NS], (j / NS) & 1, abort_flag + 1);
         }
         if (GENERIC && MODE == 4 && lane == 0 && p.conv_b_tma) {
             // Conv2d: the filter block of every k-block by TMA (the patches come from warps 6..9)
@@ -584,8 +603,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             // timing, and releasing stages in pairs to halve the commits was slower, because the ring got shallower.)
             uint32_t s = 0, ph = 0;
             const uint32_t full0 = ptx::smem_u32(ring6 ? cfull : full), empty0 = ptx::smem_u32(ring6 ? cempty : empty);
-            const uint32_t n_stages = ring6 ? kConvStages : STAGES;
-            const uint32_t stage_step = (ring6 ? kConvStageBytes : kStageBytes) >> 4;
+            const uint32_t n_stages = ring6 ? kConvStages : NS;
+            const uint32_t stage_step = (ring6 ? static_cast<uint32_t>(kConvStageBytes) : SB) >> 4;
             const uint64_t a_desc0 = make_desc(ptx::smem_u32(smem), 16, 1024);
             const uint32_t a_lo0 = static_cast<uint32_t>(a_desc0), a_hi = static_cast<uint32_t>(a_desc0 >> 32);
             const uint32_t b_lo0 = (((ptx::smem_u32(smem) + kABytes) >> 4) & 0x3FFFu) | (p.b_desc_lbo << 16);
@@ -594,7 +613,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             for (int64_t u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++t) {
                 const Unit x = unit_of(u);
                 const int kb0 = x.kb0, kb1 = x.kb1;
-                const uint32_t idesc = (x.ncols == BN) ? p.idesc : p.idesc_half;
+                const uint32_t idesc = (x.ncols == TN) ? p.idesc : p.idesc_half;
                 const uint32_t buf = t & 1;
                 if (!ptx::mbar_wait(&acc_empty[buf], ((t >> 1) & 1) ^ 1, abort_flag)) {
                     report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x410u | buf);
@@ -1251,7 +1270,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         const bool epi_warp = warp >= 2 && warp < 6;
         const bool out_bf16 = g.c_bf16 != 0;
         const int sub_log2 = out_bf16 ? 1 : 0;                          // 32-column blocks per store unit
-        const int per_log2 = (out_bf16 ? 4 : 5) - p.splits_log2;        // pairs per CTA
+        const int per_log2 = (out_bf16 ? 4 : 5) - (TN == BN ? 0 : 1) - p.splits_log2;   // pairs per CTA
         const int q = warp & 3;                                         // TMEM lane quarter of this warp
         const uint32_t tlane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
         float* recv = reinterpret_cast<float*>(smem);
@@ -1265,7 +1284,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             ptx::tc_fence_after_sync();
             // two blocks per step: both TMEM loads are in flight before the first remote store
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; c += 2) {
+            for (int c = 0; c < TN / 32; c += 2) {
                 const uint32_t own0 = static_cast<uint32_t>((((c >> sub_log2) << 2) + q) >> per_log2);
                 const uint32_t own1 = static_cast<uint32_t>(((((c + 1) >> sub_log2) << 2) + q) >> per_log2);
                 if (own0 == rank && own1 == rank) continue;
@@ -1530,9 +1549,10 @@ int choose_cluster_splits(int64_t tiles, int nkb, int sm)
 // products of 1 .. 64 tiles: 4.0 / 5.0 / 6.6 us for 2 / 4 / 8 CTAs, about 2 us more when the launch fills
 // most of the GPU.  A launch never exceeds one wave of clusters: a CTA runs exactly one unit, and a second
 // wave would pay the kernel's set-up again (measured: 2048^3 in 4 splits 54 us against 17 us unsplit).
-int cluster_fixed_cost(int s, int64_t ctas, int sm)
+int cluster_fixed_cost(int s, int64_t ctas, int sm, int tile_n)
 {
-    const int base = s == 2 ? 13 : s == 4 ? 16 : 22;
+    // (128-column tiles exchange half as much: 1.7 / 2.0 / 2.5 us less)
+    const int base = tile_n == BN ? (s == 2 ? 13 : s == 4 ? 16 : 22) : (s == 2 ? 8 : s == 4 ? 10 : 14);
     return base + (ctas * 3 > static_cast<int64_t>(sm) * 2 ? 6 : 0);
 }
 // Clusters of `s` CTAs of this kernel that the device can hold at once (GPC boundaries make this less than
@@ -1541,7 +1561,7 @@ int max_resident_clusters(int s, const RunContext& ctx);
 
 // K splits of the cluster route for a regular-orientation problem and their estimated cost (k-block times);
 // 1 when no split fits or pays.
-int choose_regular_cluster_splits(int64_t tiles, int nkb, const RunContext& ctx, int64_t* cost_out)
+int choose_regular_cluster_splits(int64_t tiles, int nkb, const RunContext& ctx, int tile_n, int64_t* cost_out)
 {
     int best = 1;
     int64_t best_cost = ((tiles + ctx.sm_count - 1) / ctx.sm_count) * static_cast<int64_t>(nkb);
@@ -1549,7 +1569,7 @@ int choose_regular_cluster_splits(int64_t tiles, int nkb, const RunContext& ctx,
         const int per = (nkb + s - 1) / s;
         if ((nkb + per - 1) / per != s) continue;
         if (tiles > max_resident_clusters(s, ctx)) continue;
-        const int64_t cost = per + cluster_fixed_cost(s, tiles * s, ctx.sm_count);
+        const int64_t cost = per + cluster_fixed_cost(s, tiles * s, ctx.sm_count, tile_n);
         if (cost < best_cost) {
             best_cost = cost;
             best = s;
@@ -1565,13 +1585,15 @@ struct SplitPlan {
     int splits;
     bool cluster;
     bool swap;
+    int64_t cost;       // the heuristic's estimate for its own choice, in k-block times (0 when not computed)
 };
 
-SplitPlan plan_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContext& ctx)
+SplitPlan plan_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContext& ctx, int tile_n = BN)
 {
     SplitPlan sp;
     sp.swap = M <= 64;
     sp.cluster = false;
+    sp.cost = 0;
     if (sp.swap && M <= 32) {
         const int s = choose_cluster_splits(tiles, nkb, ctx.sm_count);
         if (s > 1) {
@@ -1580,20 +1602,20 @@ SplitPlan plan_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContex
             return sp;
         }
     }
-    sp.splits = choose_splits(tiles, nkb, ctx.sm_count, M, ldw, ctx, sp.swap ? 6 : 30, sp.swap ? 0 : 6);
+    // (the workspace reduce of 128-row tiles is written for 256-column tiles)
+    sp.splits = (sp.swap || tile_n == BN) ? choose_splits(tiles, nkb, ctx.sm_count, M, ldw, ctx, sp.swap ? 6 : 30, sp.swap ? 0 : 6) : 1;
     if (!sp.swap) {
         // 128-row tiles: the cluster route against the workspace route chosen above and against no split
+        const int sm = ctx.sm_count;
+        const int per_w = (nkb + sp.splits - 1) / sp.splits;
+        sp.cost = sp.splits > 1 ? ((tiles * sp.splits + sm - 1) / sm) * static_cast<int64_t>(per_w + 30 + 6 * sp.splits)
+                                : ((tiles + sm - 1) / sm) * static_cast<int64_t>(nkb);
         int64_t cost_c = 0;
-        const int sc = choose_regular_cluster_splits(tiles, nkb, ctx, &cost_c);
-        if (sc > 1) {
-            const int sm = ctx.sm_count;
-            const int per_w = (nkb + sp.splits - 1) / sp.splits;
-            const int64_t cost_w = sp.splits > 1 ? ((tiles * sp.splits + sm - 1) / sm) * static_cast<int64_t>(per_w + 30 + 6 * sp.splits)
-                                                 : ((tiles + sm - 1) / sm) * static_cast<int64_t>(nkb);
-            if (cost_c <= cost_w) {
-                sp.splits = sc;
-                sp.cluster = true;
-            }
+        const int sc = choose_regular_cluster_splits(tiles, nkb, ctx, tile_n, &cost_c);
+        if (sc > 1 && cost_c <= sp.cost) {
+            sp.splits = sc;
+            sp.cluster = true;
+            sp.cost = cost_c;
         }
     }
     return sp;
@@ -1616,10 +1638,12 @@ bool split_feasible(int M, int64_t tiles, int nkb, int64_t ldw, const RunContext
 }
 
 // The heuristic plan with the pinned fields of `pl` applied; false when they cannot run.
-bool resolve_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContext& ctx, const R4Plan& pl, SplitPlan* out)
+bool resolve_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContext& ctx, const R4Plan& pl, SplitPlan* out,
+                   int tile_n = BN)
 {
-    SplitPlan sp = plan_split(M, tiles, nkb, ldw, ctx);
+    SplitPlan sp = plan_split(M, tiles, nkb, ldw, ctx, tile_n);
     if (pl.splits > 0) {
+        sp.cost = 0;
         sp.splits = pl.splits;
         if (pl.splits == 1)
             sp.cluster = false;
@@ -1752,6 +1776,65 @@ __global__ void __launch_bounds__(256) repack_rows_kernel(RepackJob first, Repac
 }
 
 bool c_store_by_tma(const GemmArgs& g);
+// Tile width, ring depth and K split of a single-CTA launch (paper, Table 1 `templatize` / `autotune`; Appendix D:
+// block size, stages and split are recipe parameters swept on a fixed kernel structure).  One function, so
+// that the launcher, the plan checks and the allocation-free entry point all plan the same way.
+struct LaunchPlan {
+    int tile_n, stages;
+    SplitPlan split;
+};
+bool plan_launch(const GemmArgs& g, const RunContext& ctx, bool generic, bool multi_dst, LaunchPlan* out)
+{
+    const R4Plan& pl = ctx.plan;
+    const int nkb = (g.K + BK - 1) / BK;
+    const int64_t ldw = (static_cast<int64_t>(g.N) + 3) & ~int64_t(3);
+    const int64_t tiles_m = (g.M + BM - 1) / BM;
+    // 128-column tiles and deeper rings: the plain TMA-fed GEMM in the regular orientation only
+    const bool tunable = !generic && !multi_dst && g.M > 64 && ctx.encode_tiled != nullptr;
+    auto try_shape = [&](int tn, int st, LaunchPlan* lp) {
+        lp->tile_n = tn;
+        lp->stages = st;
+        const int64_t tiles = tiles_m * ((g.N + tn - 1) / tn);
+        if (tiles > 0x3FFFFFFFll) return false;
+        if (!resolve_split(g.M, tiles, nkb, ldw, ctx, pl, &lp->split, tn)) return false;
+        return tn == BN || lp->split.splits == 1 || lp->split.cluster;
+    };
+    if (pl.kernel != 2 && (pl.tile_n != 0 || pl.stages != 0)) {        // pinned (the pair kernel reads the fields its own way)
+        const int tn = pl.tile_n != 0 ? pl.tile_n : BN;
+        const int st = pl.stages != 0 ? pl.stages : STAGES;
+        const bool ok = (tn == BN && st == STAGES) || (tunable && tn == BN / 2 && (st == 4 || st == 6));
+        return ok && try_shape(tn, st, out);
+    }
+    LaunchPlan wide;
+    const bool wide_ok = try_shape(BN, STAGES, &wide);
+    if (!tunable || g.N <= BN / 2 || pl.half_tail != 0 || pl.kernel == 2) {
+        *out = wide;
+        return wide_ok;
+    }
+    LaunchPlan narrow;
+    const int64_t tiles256 = tiles_m * ((g.N + BN - 1) / BN);
+    if (!try_shape(BN / 2, STAGES, &narrow)) {
+        *out = wide;
+        return wide_ok;
+    }
+    if (!wide_ok) {
+        *out = narrow;
+        return true;
+    }
+    // Measured (CUDA-graph replay): a cluster split with 128-column tiles exchanges half as much and wins at equal
+    // splits; unsplit, 128-column tiles match the half-tile tail when one under-filled wave is all there is (they load
+    // only the columns they use) and lose once the tiles no longer fit one wave.
+    bool take_narrow;
+    if (pl.splits > 0)
+        take_narrow = narrow.split.cluster || (narrow.split.splits == 1 && tiles256 * 2 <= ctx.sm_count);
+    else if (narrow.split.cost != wide.split.cost)
+        take_narrow = narrow.split.cost < wide.split.cost;
+    else
+        take_narrow = narrow.split.splits > 1 || tiles256 * 2 <= ctx.sm_count;
+    if (take_narrow && narrow.split.cluster) narrow.stages = 6;
+    *out = take_narrow ? narrow : wide;
+    return true;
+}
 struct MultiDst {
     void* const* C;
     const int64_t* ldc;
@@ -1817,22 +1900,28 @@ namespace {
 cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id, const MultiDst* md)
 {
     if (ctx.max_smem_optin < kSmemBytes) return cudaErrorInvalidConfiguration;
-    const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN;
+    const R4Plan& pinned = ctx.plan;
+    const bool generic = !(ctx.encode_tiled && tma_ok(g.A, g.lda, 2) && tma_ok(g.B, g.ldb, 2));
+    // Tile width and ring depth of the single-CTA kernel (plain TMA-fed GEMM in the regular orientation only).
+    LaunchPlan shape;
+    if (!plan_launch(g, ctx, generic, md != nullptr, &shape)) return cudaErrorInvalidValue;
+    const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + shape.tile_n - 1) / shape.tile_n;
     const int64_t tiles = tiles_m * tiles_n;
     if (tiles > 0x3FFFFFFFll) return cudaErrorInvalidConfiguration;
 
     R4Params p;
     memset(&p, 0, sizeof p);
+    p.tile_n = shape.tile_n;
+    p.n_stages = shape.stages;
+    p.stage_bytes = static_cast<uint32_t>(kABytes + shape.tile_n * BK * 2);
     p.tiles_m = static_cast<int>(tiles_m);
     p.tiles_n = static_cast<int>(tiles_n);
     p.nkb = (g.K + BK - 1) / BK;
     p.ldw = (static_cast<int64_t>(g.N) + 3) & ~int64_t(3);
-    const R4Plan& pinned = ctx.plan;
-    SplitPlan plan;
-    if (!resolve_split(g.M, tiles, p.nkb, p.ldw, ctx, pinned, &plan)) return cudaErrorInvalidValue;
+    const SplitPlan plan = shape.split;
     p.splits = plan.splits;
     p.cluster = plan.cluster ? 1 : 0;
-    p.static_b = (ctx.flags & 1u) ? 1 : 0;
+    p.static_b = ((ctx.flags & 1u) && shape.tile_n == BN && shape.stages == STAGES) ? 1 : 0;
     p.splits_log2 = plan.splits >= 8 ? 3 : plan.splits >= 4 ? 2 : plan.splits >= 2 ? 1 : 0;
     p.kb_per_split = (p.nkb + p.splits - 1) / p.splits;
     p.ws = static_cast<float*>(ctx.workspace);
@@ -1846,7 +1935,6 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
         return md ? launch_r4_pair_multi_dst(g, md->C, md->ldc, md->n, ctx, stream, kernel_id)
                   : launch_r4_tcgen05_pair(g, ctx, stream, kernel_id);
 
-    const bool generic = !(ctx.encode_tiled && tma_ok(g.A, g.lda, 2) && tma_ok(g.B, g.ldb, 2));
     if (md && generic) return cudaErrorNotSupported;
     const int celt = g.c_bf16 ? 2 : 4;
     // Skinny mode: few activation rows -> they become the MMA's N, the weights its 128 rows.
@@ -1868,7 +1956,7 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
         p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (w_major << 15) | (static_cast<uint32_t>(p.n_mma >> 3) << 17) |
                   (static_cast<uint32_t>(128 >> 4) << 24);
     else
-        p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (w_major << 16) | (static_cast<uint32_t>(BN >> 3) << 17) |
+        p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (w_major << 16) | (static_cast<uint32_t>(shape.tile_n >> 3) << 17) |
                   (static_cast<uint32_t>(BM >> 4) << 24);
     // Shared-memory descriptor of B (version 1, 128-byte swizzle):
     //   K-major : 8-row groups 1024 bytes apart; +32 bytes per 16 k
@@ -1904,14 +1992,14 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     }
     // Skinny mode fetches only the activation rows the MMA reads (n_mma of them).
     const uint32_t a_box_rows = swap ? static_cast<uint32_t>(p.n_mma) : BM;
-    p.stage_tx = a_box_rows * BK * 2 + kBBytes;
+    p.stage_tx = a_box_rows * BK * 2 + static_cast<uint32_t>(shape.tile_n) * BK * 2;
     if (!generic) {
         ok = encode_map_2d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, a_box_rows,
                            CU_TENSOR_MAP_SWIZZLE_128B);
         if (g.b_col)
-            ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, BN,
-                                     CU_TENSOR_MAP_SWIZZLE_128B);
-        else if (g.N % 64 == 0 && !p.static_b && encode_b_blocks_3d(ctx, &mb, g, BN / 64))
+            ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK,
+                                     static_cast<uint32_t>(shape.tile_n), CU_TENSOR_MAP_SWIZZLE_128B);
+        else if (g.N % 64 == 0 && !p.static_b && encode_b_blocks_3d(ctx, &mb, g, static_cast<uint32_t>(shape.tile_n / 64)))
             p.b_box3d = 1;
         else
             ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, g.ldb * 2, 64, BK,
@@ -1929,13 +2017,13 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     // SMs idle is cut into 128-column half tiles (twice as many units, half as long).
     p.group_m = pinned.group_m > 0 ? pinned.group_m : 16;   // measured: 16 tile-rows per group re-read least from HBM at 8192^3
     p.full_units = tiles;
-    if (p.splits == 1 && !swap && pinned.half_tail != 2) {
+    if (p.splits == 1 && !swap && pinned.half_tail != 2 && shape.tile_n == BN) {
         const int64_t tail = tiles % ctx.sm_count;
         const bool pays = 2 * tail <= ctx.sm_count;
         if (tail != 0 && (pays || pinned.half_tail == 1) && g.N > BN / 2) p.full_units = tiles - tail;
     }
     p.total_units = p.splits > 1 ? tiles * p.splits : p.full_units + 2 * (tiles - p.full_units);
-    p.idesc_half = (p.idesc & ~(0x3Fu << 17)) | (static_cast<uint32_t>((BN / 2) >> 3) << 17);
+    p.idesc_half = (p.idesc & ~(0x3Fu << 17)) | (static_cast<uint32_t>((shape.tile_n / 2) >> 3) << 17);
     const int64_t units = p.total_units;
     // A cluster handles exactly one tile, so the cluster path launches every unit as a CTA.
     const unsigned grid = static_cast<unsigned>((p.cluster || units < ctx.sm_count) ? units : ctx.sm_count);
@@ -1985,6 +2073,9 @@ void fill_multi_params(R4Params& p, const GemmArgs& g, const RunContext& ctx)
     p.n_mma = 16;
     p.stage_tx = kABytes + kBBytes;
     p.group_m = ctx.plan.group_m > 0 ? ctx.plan.group_m : 16;
+    p.tile_n = BN;
+    p.n_stages = STAGES;
+    p.stage_bytes = kStageBytes;
 }
 
 // Static schedule over `tiles` whole tiles: a last wave that would leave at least half of the
@@ -2261,11 +2352,9 @@ bool r4_multi_dst_possible(const GemmArgs& g, const RunContext& ctx)
 {
     if (!ctx.encode_tiled || ctx.max_smem_optin < kSmemBytes || g.M <= 0 || g.N <= 0 || g.K <= 0) return false;
     if (!tma_ok(g.A, g.lda, 2) || !tma_ok(g.B, g.ldb, 2)) return false;
-    const int64_t tiles = static_cast<int64_t>((g.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
-    const int64_t ldw = (static_cast<int64_t>(g.N) + 3) & ~int64_t(3);
-    SplitPlan sp;
-    if (!resolve_split(g.M, tiles, (g.K + BK - 1) / BK, ldw, ctx, ctx.plan, &sp)) return false;
-    return !sp.swap && sp.splits == 1;
+    LaunchPlan lp;
+    if (!plan_launch(g, ctx, false, true, &lp)) return false;
+    return !lp.split.swap && lp.split.splits == 1;
 }
 
 cudaError_t launch_r4_multi_dst(const GemmArgs& g, void* const* C, const int64_t* ldc, int n_dst, RunContext& ctx,
@@ -2286,14 +2375,23 @@ bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& pl)
     if (pl.tile_n != 0 && (pl.tile_n < 64 || pl.tile_n > 256 || pl.tile_n % 64 != 0)) return false;
     if (pl.tail_n != 0 && (pl.tail_n < 64 || pl.tail_n > 256 || pl.tail_n % 64 != 0 || pl.tail_n > (pl.tile_n ? pl.tile_n : 256)))
         return false;
-    if ((pl.tile_n != 0 || pl.tail_n != 0) && pl.kernel != 2) return false;
-    if (pl.stages != 0) return false;
+    if (pl.tail_n != 0 && pl.kernel != 2) return false;
+    if (pl.kernel == 2 && pl.stages != 0) return false;
+    if (pl.kernel != 2 && (pl.tile_n != 0 || pl.stages != 0)) {
+        // single-CTA kernel: 256 columns x 4 stages, or 128 columns x 4 or 6 stages (plain TMA-fed GEMM, M > 64)
+        if (pl.tile_n != 0 && pl.tile_n != BN && pl.tile_n != BN / 2) return false;
+        if (pl.stages != 0 && pl.stages != 4 && pl.stages != 6) return false;
+    }
+    // a tile shape is a property of one of the two kernels: name the kernel with it
+    if ((pl.tile_n != 0 || pl.tail_n != 0 || pl.stages != 0) && pl.kernel == 0) return false;
     if (g.M <= 0 || g.N <= 0 || g.K <= 0) return true;   // nothing to launch; any plan is moot
-    const int64_t tiles = static_cast<int64_t>((g.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
-    const int nkb = (g.K + BK - 1) / BK;
-    const int64_t ldw = (static_cast<int64_t>(g.N) + 3) & ~int64_t(3);
-    SplitPlan sp;
-    if (!resolve_split(g.M, tiles, nkb, ldw, ctx, pl, &sp)) return false;
+    RunContext c2 = ctx;
+    c2.plan = pl;
+    // (unaligned operands that the launch repacks into the workspace run the TMA-fed kernel)
+    const bool aligned = ctx.encode_tiled && tma_ok(g.A, g.lda, 2) && tma_ok(g.B, g.ldb, 2);
+    LaunchPlan lp;
+    if (!plan_launch(g, c2, !aligned && !ctx.allow_repack, false, &lp)) return false;
+    const SplitPlan& sp = lp.split;
     if (pl.kernel == 2 && (sp.swap || sp.splits != 1 || !r4_pair_possible(g, ctx))) return false;
     return true;
 }
@@ -2329,6 +2427,32 @@ int r4_enumerate_plans(const GemmArgs& g, const RunContext& ctx, R4Plan* out, in
                 pl.group_m = gm;
                 push(pl);
             }
+        if (r4_pair_possible(g, ctx) && g.M > BM) {
+            // tile widths of the pair kernel: uniform 192 / 128 columns, and 256 with a narrow tail
+            for (int w : {192, 128}) {
+                R4Plan pl;
+                pl.kernel = 2;
+                pl.splits = 1;
+                pl.tile_n = w;
+                pl.tail_n = w;
+                push(pl);
+            }
+            R4Plan pl;
+            pl.kernel = 2;
+            pl.splits = 1;
+            pl.tile_n = 256;
+            pl.tail_n = 192;
+            push(pl);
+        }
+        // tile shapes of the single-CTA kernel: 128 columns on a 4- or 6-stage ring
+        for (int st : {4, 6}) {
+            R4Plan pl;
+            pl.kernel = 1;
+            pl.splits = 1;
+            pl.tile_n = BN / 2;
+            pl.stages = st;
+            push(pl);
+        }
         for (int gm : {4, 8, 16, 32}) {
             if (gm > 4 && gm / 2 >= tiles_m) continue;
             for (int ht : {1, 2}) {
@@ -2355,6 +2479,11 @@ int r4_enumerate_plans(const GemmArgs& g, const RunContext& ctx, R4Plan* out, in
             if ((!swap || g.M <= 32) && (s == 2 || s == 4 || s == 8)) {
                 pl.split_via = 2;
                 push(pl);
+                if (!swap) {
+                    pl.tile_n = BN / 2;
+                    pl.stages = 6;
+                    push(pl);
+                }
             }
         }
         R4Plan pl;
@@ -2493,15 +2622,18 @@ extern "C" klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype
 
     // Refuse, rather than quietly change the schedule, when the K split this
     // shape would get needs more partial-sum space than the fixed array holds.
-    const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
-    const int nkb = static_cast<int>((K + BK - 1) / BK);
     const int64_t ldw = (N + 3) & ~int64_t(3);
     RunContext unlimited = d->ctx;
     unlimited.workspace_bytes = ~size_t(0);
+    unlimited.plan = R4Plan();
     SplitPlan plan;
     plan.splits = 1;
     plan.cluster = false;
-    if (tiles <= 0x3FFFFFFFll) plan = plan_split(static_cast<int>(M), tiles, nkb, ldw, unlimited);
+    {
+        const bool generic = !(unlimited.encode_tiled && tma_ok(g.A, g.lda, 2) && tma_ok(g.B, g.ldb, 2));
+        LaunchPlan lp;
+        if (plan_launch(g, unlimited, generic, false, &lp)) plan = lp.split;
+    }
     const size_t need =
         (plan.splits > 1 && !plan.cluster) ? static_cast<size_t>(plan.splits) * M * ldw * sizeof(float) : 0;
     if (need > kNoAllocPartialBytes) {

@@ -5,9 +5,12 @@ lets the kernel's epilogue store the result slice into EVERY rank's full-width C
 operand crosses NVLink, no collective follows, the only traffic is the result leaving through stores to peer memory.
 The paper describes no multi-GPU design; this is the partitioning the GEMM admits without any exchange during compute.
 
-The rendezvous that makes a rank's C addressable by its peers is plumbing and stays outside the library: pass the list
-of per-rank C base pointers (for instance the ``buffer_ptrs`` of a ``torch.distributed._symmetric_memory`` rendezvous,
-or pointers opened from CUDA IPC handles).  On one GPU the "ranks" may simply be different buffers.
+The rendezvous that makes a rank's C addressable by its peers is plumbing and stays outside the C library, which takes
+plain pointers: ``SharedC`` below does it with ``torch.distributed`` (symmetric memory, else CUDA IPC handles passed
+over the process group), ``exchange`` is the underlying all-gather of Python objects, and ``partitioned_step`` is one
+step of a rank (launch, nothing else: the caller owns barriers and timing).  On one GPU the "ranks" may simply be
+different buffers.  The rendezvous has run on CPU ranks only (gloo, with a stand-in for the launch): this build had
+one GPU per run.
 """
 from __future__ import annotations
 
@@ -58,3 +61,67 @@ class NPartitionedGemm:
             return
         self.gemm.run_multi_dst(A, B_slice, self.dst, M, self.n_local, K, lda, ldb, [self.ldc] * self.world, variant,
                                 stream)
+
+
+def exchange(obj, world: int, group=None) -> list:
+    """Every rank's ``obj`` in rank order (``torch.distributed.all_gather_object``); ``[obj]`` for one rank."""
+    if world <= 1:
+        return [obj]
+    import torch.distributed as dist
+    out = [None] * world
+    dist.all_gather_object(out, obj, group=group)
+    return out
+
+
+class SharedC:
+    """This rank's full-width C plus the address of every rank's C as seen from this GPU.
+
+    how="symm": the buffer comes from ``torch.distributed._symmetric_memory`` and its rendezvous yields the peers'
+    mapped addresses.  how="ipc": an ordinary CUDA tensor whose storage is exported as a CUDA IPC handle, gathered
+    over the process group and opened on every peer (what ``torch.multiprocessing`` does for shared CUDA tensors).
+    how="auto" tries the first and falls back to the second.  Peers are only ever STORED to through these
+    addresses (the kernel's epilogue); nothing is loaded from a peer.
+    """
+
+    def __init__(self, M: int, ldc: int, dtype, device, world: int, rank: int, group=None, how: str = "auto"):
+        import torch
+        self.world, self.rank = int(world), int(rank)
+        self._keep = []
+        self.how = "local"
+        if world <= 1:
+            self.local = torch.empty((M, ldc), dtype=dtype, device=device)
+            self.ptrs = [self.local.data_ptr()]
+            return
+        import torch.distributed as dist
+        group = group if group is not None else dist.group.WORLD
+        if how in ("auto", "symm"):
+            try:
+                import torch.distributed._symmetric_memory as symm
+                self.local = symm.empty((M, ldc), dtype=dtype, device=device)
+                hdl = symm.rendezvous(self.local, group)
+                self.ptrs = [int(p) for p in hdl.buffer_ptrs]
+                self._keep.append(hdl)
+                self.how = "symm"
+                return
+            except Exception:
+                if how == "symm":
+                    raise
+        self.local = torch.empty((M, ldc), dtype=dtype, device=device)
+        info = self.local.untyped_storage()._share_cuda_()
+        offset = self.local.storage_offset() * self.local.element_size()
+        infos = exchange((info, offset), world, group)
+        self.ptrs = []
+        for r, (peer_info, peer_off) in enumerate(infos):
+            if r == rank:
+                self.ptrs.append(self.local.data_ptr())
+                continue
+            st = torch.UntypedStorage._new_shared_cuda(*peer_info)
+            self._keep.append(st)
+            self.ptrs.append(st.data_ptr() + peer_off)
+        self.how = "ipc"
+
+
+def partitioned_step(part: "NPartitionedGemm", A, B_slice, M: int, K: int, lda: int, ldb: int, variant: int = 4,
+                     stream=None) -> None:
+    """One step of this rank: its column slice of A . B, stored by the epilogue into every rank's C."""
+    part.run(A, B_slice, M, K, lda, ldb, variant, stream)

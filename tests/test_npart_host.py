@@ -95,3 +95,62 @@ def test_two_gloo_ranks_assemble_c_from_their_column_slices(tmp_path):
     res = [json.loads((tmp_path / f"rank{k}.json").read_text()) for k in range(2)]
     assert all(x["ok"] for x in res)
     assert res[0]["slice"][0] == 0 and res[0]["slice"][1] == res[1]["slice"][0] and res[1]["slice"][1] == 203
+
+
+DRIVER_WORKER = textwrap.dedent("""
+    import os, sys, json
+    sys.path.insert(0, os.environ["KL_ROOT"])
+    import numpy as np, torch.distributed as dist
+    from paper_2605_28213_b200 import inputs as gen, npart
+    from oracle import gemm_oracle as orc
+    dist.init_process_group("gloo")
+    rank, world = dist.get_rank(), dist.get_world_size()
+    out = os.environ["KL_OUT"]
+    M, N, K, ldc = 37, 203, 64, 208
+    case = gen.make_case(M, N, K, seed=5, dist_a="integer", dist_b="integer", name="npart")
+    # every rank's "C" is a file that all ranks can map; its "address" is (rank + 1) << 40
+    mine = np.lib.format.open_memmap(os.path.join(out, f"c{rank}.npy"), mode="w+", dtype=np.float32, shape=(M, ldc))
+    mine[:] = -1.0
+    mine.flush()
+    ptrs = npart.exchange((rank + 1) << 40, world)            # the rendezvous: everybody learns everybody's address
+    dist.barrier()
+
+    class FileGemm:                                            # stand-in for the launch: stores the slice to every C
+        c_bf16 = False
+        def run_multi_dst(self, A, B, Cs, M_, N_, K_, lda, ldb, ldcs, variant, stream):
+            C_slice, _ = orc.gemm(M_, N_, K_, A, lda, B, ldb, False)
+            for dst, ld in zip(Cs, ldcs):
+                r, off = (dst >> 40) - 1, (dst & ((1 << 40) - 1)) // 4
+                tgt = np.load(os.path.join(out, f"c{r}.npy"), mmap_mode="r+")
+                assert ld == ldc and off % 1 == 0
+                tgt[:, off:off + N_] = np.asarray(C_slice, dtype=np.float32)
+                tgt.flush()
+
+    part = npart.NPartitionedGemm(FileGemm(), world, rank, N, ptrs, ldc)
+    B_slice = np.ascontiguousarray(case.B[:, part.n0:part.n1])
+    npart.partitioned_step(part, case.A, B_slice, M, K, case.lda, part.n_local)
+    dist.barrier()                                             # a step ends when every rank's stores have landed
+    got = np.load(os.path.join(out, f"c{rank}.npy"), mmap_mode="r")
+    C_ref, _ = orc.gemm(M, N, K, case.A, case.lda, case.B, case.ldb, False)
+    ok = bool(np.array_equal(np.asarray(got[:, :N], dtype=np.float64), np.asarray(C_ref))) and bool(np.all(got[:, N:] == -1.0))
+    dist.barrier()
+    dist.destroy_process_group()
+    open(os.path.join(out, f"drv{rank}.json"), "w").write(json.dumps({"ok": ok, "ptrs": ptrs, "dst": part.dst}))
+""")
+
+
+def test_two_gloo_ranks_drive_the_fused_all_gather_with_a_stand_in_launch(tmp_path):
+    """The multi-rank driver's host logic: address exchange over the process group, slice table, every rank's launch
+    writing its slice into every rank's C, and each rank finding the whole product in its own C afterwards."""
+    script = tmp_path / "driver.py"
+    script.write_text(DRIVER_WORKER)
+    env = dict(os.environ, KL_ROOT=str(ROOT), KL_OUT=str(tmp_path))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", "29541", str(script)]
+    r = subprocess.run(cmd, capture_output=True, text=True, env=env, timeout=240)
+    assert r.returncode == 0, r.stderr[-2000:]
+    import json
+    res = [json.loads((tmp_path / f"drv{k}.json").read_text()) for k in range(2)]
+    assert all(x["ok"] for x in res)
+    assert res[0]["ptrs"] == res[1]["ptrs"] == [1 << 40, 2 << 40]
+    assert res[1]["dst"] == [p + 104 * 4 for p in res[1]["ptrs"]]          # rank 1's slice starts at column 104

@@ -67,9 +67,13 @@ def run_and_check(handles, case, variant, C_ref=None, S=None, rows=None, exact=F
 
 # ------------------------------------------------------------------ the five configurations
 @pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_NAMES)
-@pytest.mark.parametrize("name,seeds", [("c1", (1, 2, 3)), ("c2", (1, 2, 3)), ("c2pad", (1,)), ("c5", (1,)),
-                                        ("c3", (1,)), ("c4", (1,))])
+@pytest.mark.parametrize("name,seeds", [("c1", (1, 2, 3)), ("c2", (1, 2, 3)), ("c2pad", (1, 2, 3)), ("c5", (1, 2, 3)),
+                                        ("c3", (1, 2, 3)), ("c4", (1, 2, 3))])
 def test_config_random_within_bound(handles, variant, name, seeds):
+    # three seeds everywhere (the paper's gate); at 4096^3 and 8192^3 the rungs without tensor cores, which take up to a
+    # second per run there, keep to the first seed
+    if name in ("c3", "c4") and variant not in (4, 5):
+        seeds = seeds[:1]
     for seed in seeds:
         case, rows, C_ref, S = P.cached_reference(name, seed, False)
         run_and_check(handles, case, variant, C_ref, S, rows)
