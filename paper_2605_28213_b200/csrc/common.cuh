@@ -229,6 +229,9 @@ bool encode_map_nhwc(const RunContext& ctx, CUtensorMap* map, CUtensorMapDataTyp
                      uint64_t W, uint64_t H, uint64_t N, uint32_t c_box, uint32_t w_box, uint32_t h_box, int elt,
                      CUtensorMapSwizzle swz);
 
+// Edge of the square block tile the staged rungs (1, 2, 3) use for a problem: the largest of 128 / 64 / 32 whose
+// grid still has a CTA for every SM of the current device, else 32.
+int staged_tile_edge(const GemmArgs& g);
 cudaError_t launch_r0_naive(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
 cudaError_t launch_r1_tiled(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
 cudaError_t launch_r2_vectorized(const GemmArgs& g, cudaStream_t stream, int* kernel_id);

@@ -1,39 +1,52 @@
 // Rung 1 - "tile / sm_stage" (paper, Table 1; precondition: loops over the
-// output).  A 128 x 128 block tile of C per CTA; A and B k-slabs of depth 16 are
-// staged in shared memory as fp32 (converted from bf16 on the way in) and each
-// of the 256 threads keeps an 8 x 8 register tile.  Loads are scalar and masked
-// element by element, so every M/N/K tail and every alignment is handled the
-// same way; nothing is vectorized or overlapped yet.
+// output).  A T x T block tile of C per CTA (T = 128, 64 or 32); A and B k-slabs
+// of depth 16 are staged in shared memory as fp32 (converted from bf16 on the way
+// in) and each of the 256 threads keeps a (T/16) x (T/16) register tile.  Loads
+// are scalar and masked element by element, so every M/N/K tail and every
+// alignment is handled the same way; nothing is vectorized or overlapped yet.
+//
+// A thread's rows are ty + 16 i and its columns tx + 16 j: the 16 threads of a
+// half warp read 16 consecutive words of a shared-memory row (no bank conflict;
+// with columns tx * 8 + j the reads of B were four-way conflicts and the rung ran
+// at a quarter of the fp32 pipe), and a half warp's stores to C are 16 consecutive
+// elements.
+//
+// The tile is the largest of the three that still gives every SM a CTA: a
+// 256^3 product is 4 tiles of 128 x 128 but 64 of 32 x 32, and a rung that
+// stages through shared memory should not be slower than the naive kernel just
+// because most of the GPU has nothing to do.
 #include "common.cuh"
 
 namespace klin {
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 16, TM = 8, TN = 8, NT = 256;
+constexpr int BK = 16, NT = 256;
 
-template <bool BCOL>
+template <bool BCOL, int T>
 __global__ void __launch_bounds__(NT) r1_tiled_kernel(GemmArgs g, int tiles_m, int tiles_n)
 {
-    __shared__ float As[BK][BM + 1];
-    __shared__ float Bs[BK][BN + 1];
+    constexpr int TT = T / 16;                 // register tile edge
+    // (row pitch = 2 mod 32 words: the k-fastest fill - 16 k values of 2 rows per warp - then hits 32 different banks)
+    __shared__ float As[BK][T + 2];
+    __shared__ float Bs[BK][T + 2];
     if (blockIdx.x == 0 && threadIdx.x == 0) g.status[1] = kIdTiled;
 
     int tm, tn;
     raster_tile(blockIdx.x, tiles_m, tiles_n, tm, tn);
-    const int m0 = tm * BM, n0 = tn * BN;
+    const int m0 = tm * T, n0 = tn * T;
     const int t = threadIdx.x;
     const int tx = t % 16, ty = t / 16;
 
-    float acc[TM][TN];
+    float acc[TT][TT];
 #pragma unroll
-    for (int i = 0; i < TM; ++i)
+    for (int i = 0; i < TT; ++i)
 #pragma unroll
-        for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
+        for (int j = 0; j < TT; ++j) acc[i][j] = 0.f;
 
     for (int k0 = 0; k0 < g.K; k0 += BK) {
-        // A slab: 128 rows x 16 k, one element per thread per step, k fastest.
+        // A slab: T rows x 16 k, one element per thread per step, k fastest.
 #pragma unroll
-        for (int e = t; e < BM * BK; e += NT) {
+        for (int e = t; e < T * BK; e += NT) {
             const int k = e % BK, m = e / BK;
             const int64_t gm = m0 + m;
             const int gk = k0 + k;
@@ -41,7 +54,7 @@ __global__ void __launch_bounds__(NT) r1_tiled_kernel(GemmArgs g, int tiles_m, i
         }
         if (BCOL) {
 #pragma unroll
-            for (int e = t; e < BN * BK; e += NT) {
+            for (int e = t; e < T * BK; e += NT) {
                 const int k = e % BK, n = e / BK;
                 const int64_t gn = n0 + n;
                 const int gk = k0 + k;
@@ -49,8 +62,8 @@ __global__ void __launch_bounds__(NT) r1_tiled_kernel(GemmArgs g, int tiles_m, i
             }
         } else {
 #pragma unroll
-            for (int e = t; e < BN * BK; e += NT) {
-                const int n = e % BN, k = e / BN;
+            for (int e = t; e < T * BK; e += NT) {
+                const int n = e % T, k = e / T;
                 const int64_t gn = n0 + n;
                 const int64_t gk = k0 + k;
                 Bs[k][n] = (gn < g.N && gk < g.K) ? bf16_bits_to_float(g.B[gk * g.ldb + gn]) : 0.f;
@@ -59,44 +72,78 @@ __global__ void __launch_bounds__(NT) r1_tiled_kernel(GemmArgs g, int tiles_m, i
         __syncthreads();
 #pragma unroll
         for (int k = 0; k < BK; ++k) {
-            float a[TM], b[TN];
+            float a[TT], b[TT];
 #pragma unroll
-            for (int i = 0; i < TM; ++i) a[i] = As[k][ty * TM + i];
+            for (int i = 0; i < TT; ++i) a[i] = As[k][ty + 16 * i];
 #pragma unroll
-            for (int j = 0; j < TN; ++j) b[j] = Bs[k][tx * TN + j];
+            for (int j = 0; j < TT; ++j) b[j] = Bs[k][tx + 16 * j];
 #pragma unroll
-            for (int i = 0; i < TM; ++i)
+            for (int i = 0; i < TT; ++i)
 #pragma unroll
-                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+                for (int j = 0; j < TT; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
         }
         __syncthreads();
     }
 
 #pragma unroll
-    for (int i = 0; i < TM; ++i) {
-        const int64_t gm = m0 + ty * TM + i;
+    for (int i = 0; i < TT; ++i) {
+        const int64_t gm = m0 + ty + 16 * i;
         if (gm >= g.M) continue;
 #pragma unroll
-        for (int j = 0; j < TN; ++j) {
-            const int64_t gn = n0 + tx * TN + j;
+        for (int j = 0; j < TT; ++j) {
+            const int64_t gn = n0 + tx + 16 * j;
             if (gn < g.N) store_c(g.C, g.c_bf16, gm * g.ldc + gn, acc[i][j] + bias_at(g, gn));
         }
     }
 }
 
-}  // namespace
-
-cudaError_t launch_r1_tiled(const GemmArgs& g, cudaStream_t stream, int* kernel_id)
+template <int T>
+cudaError_t launch_tile(const GemmArgs& g, cudaStream_t stream)
 {
-    const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN;
+    const int64_t tiles_m = (g.M + T - 1) / T, tiles_n = (g.N + T - 1) / T;
     if (tiles_m * tiles_n > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;
     const unsigned grid = static_cast<unsigned>(tiles_m * tiles_n);
     if (g.b_col)
-        r1_tiled_kernel<true><<<grid, NT, 0, stream>>>(g, (int)tiles_m, (int)tiles_n);
+        r1_tiled_kernel<true, T><<<grid, NT, 0, stream>>>(g, (int)tiles_m, (int)tiles_n);
     else
-        r1_tiled_kernel<false><<<grid, NT, 0, stream>>>(g, (int)tiles_m, (int)tiles_n);
-    *kernel_id = kIdTiled;
+        r1_tiled_kernel<false, T><<<grid, NT, 0, stream>>>(g, (int)tiles_m, (int)tiles_n);
     return cudaGetLastError();
+}
+
+}  // namespace
+
+// Edge of the square block tile the staged rungs (1 to 3) use for a problem: the largest of 128 / 64 / 32
+// whose grid still has a CTA for every SM, else 32.
+int staged_tile_edge(const GemmArgs& g)
+{
+    int sms = 148;
+    int dev = 0;
+    static int cached_sms[64] = {};
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
+        if (cached_sms[dev] == 0 &&
+            cudaDeviceGetAttribute(&cached_sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            cudaGetLastError();
+            cached_sms[dev] = 148;
+        }
+        sms = cached_sms[dev];
+    } else {
+        cudaGetLastError();
+    }
+    for (int t : {128, 64}) {
+        const int64_t tiles = static_cast<int64_t>((g.M + t - 1) / t) * ((g.N + t - 1) / t);
+        if (tiles >= sms) return t;
+    }
+    return 32;
+}
+
+cudaError_t launch_r1_tiled(const GemmArgs& g, cudaStream_t stream, int* kernel_id)
+{
+    *kernel_id = kIdTiled;
+    switch (staged_tile_edge(g)) {
+        case 128: return launch_tile<128>(g, stream);
+        case 64: return launch_tile<64>(g, stream);
+        default: return launch_tile<32>(g, stream);
+    }
 }
 
 }  // namespace klin

@@ -2,12 +2,13 @@
 // "mma (m16n8k16)" (paper, Table 1; preconditions: the tile fits the mma shape,
 // fragments come from swizzled shared memory).  It sits between the CUDA-core
 // pipeline of rung 3 and the tcgen05 rung: the same 4-stage TMA / mbarrier ring
-// (128 x 128 x 32 tiles of raw bf16), but the multiply is
+// (T x T x 32 tiles of raw bf16; T = 128, or 64 when 128 x 128 tiles would leave SMs
+// without a CTA), but the multiply is
 // mma.sync.aligned.m16n8k16 on fragments fetched with ldmatrix from shared
 // memory laid out with TMA's swizzle patterns (64-byte swizzle for K-contiguous
 // operands, 128-byte swizzle for the N-contiguous row-major B, read with
-// ldmatrix.trans).  8 warps as 2 x 4, each a 64 x 32 warp tile (4 x 4 mma tiles,
-// fp32 accumulators in registers).  On sm_100a this path compiles and runs but
+// ldmatrix.trans).  8 warps as 2 x 4, each a (T/2) x (T/4) warp tile (4 x 4 or 2 x 2 mma
+// tiles, fp32 accumulators in registers).  On sm_100a this path compiles and runs but
 // cannot reach tcgen05 throughput: it is kept as the lineage's intermediate step.
 // Operands that break TMA's alignment rules take the producer-thread path of
 // rung 3 (masked scalar loads written into the same swizzled layout).
@@ -18,9 +19,8 @@
 namespace klin {
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 32, STAGES = 4, NT = 256;
-constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2, kStageBytes = kABytes + kBBytes;
-constexpr int kSmemBytes = STAGES * kStageBytes + 1024 /*alignment slack*/ + 128 /*barriers*/;
+constexpr int BK = 32, STAGES = 4, NT = 256;
+constexpr int smem_bytes(int T) { return STAGES * (2 * T * BK * 2) + 1024 /*alignment slack*/ + 128 /*barriers*/; }
 
 // Byte offsets of a 16-byte chunk (8 bf16) inside a stage.
 //   K-contiguous operand (A; column-major B): [row][32 k], 64-byte rows, chunk index XORed
@@ -68,11 +68,17 @@ __device__ __forceinline__ uint4 gather8(const uint16_t* p, int valid)
     return r;
 }
 
-template <bool BCOL, bool TMA>
+template <bool BCOL, bool TMA, int T>
 __global__ void __launch_bounds__(NT)
 r35_mma_sync_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     int tiles_m, int tiles_n, int c_vec, int kid)
 {
+    constexpr int BM = T, BN = T;
+    constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2, kStageBytes = kABytes + kBBytes;
+    constexpr int MI = T / 32;                         // m16 tiles per warp (warp tile T/2 rows)
+    constexpr int NJJ = T / 64;                        // pairs of n8 tiles per warp (warp tile T/4 columns)
+    constexpr int kChunks = T * BK / 8;                // 16-byte chunks of one operand block
+    constexpr int kPer = (kChunks + NT - 1) / NT;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * kStageBytes);
@@ -81,7 +87,7 @@ r35_mma_sync_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
 
     const int t = threadIdx.x;
     const int warp = t >> 5, lane = t & 31;
-    const int wm = (warp >> 2) * 64, wn = (warp & 3) * 32;   // origin of the warp tile inside the block tile
+    const int wm = (warp >> 2) * (T / 2), wn = (warp & 3) * (T / 4);   // origin of the warp tile inside the block tile
     if (blockIdx.x == 0 && t == 0) g.status[1] = kid;
 
     int tm, tn;
@@ -116,36 +122,38 @@ r35_mma_sync_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
             ptx::tma_load_2d(sa + kABytes, &map_b, kb * BK, n0, &full[s]);
         } else {
             ptx::tma_load_2d(sa + kABytes, &map_b, n0, kb * BK, &full[s]);
-            ptx::tma_load_2d(sa + kABytes + 4096, &map_b, n0 + 64, kb * BK, &full[s]);
+            if (BN > 64) ptx::tma_load_2d(sa + kABytes + 4096, &map_b, n0 + 64, kb * BK, &full[s]);
         }
         issued = kb + 1;
     };
 
-    // Producer-thread path: 4 chunks of 8 bf16 per thread and stage.
-    uint4 pre[4];
+    // Producer-thread path: up to kPer 16-byte chunks of A and of B per thread and stage.
+    uint4 pre[2 * kPer];
     auto fetch_regs = [&](int kb) {
         const int k0 = kb * BK;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int c = t + NT * (q & 1);
-            if (q < 2) {                       // A: row c/4, k-chunk c%4
+        for (int q = 0; q < kPer; ++q) {
+            const int c = t + NT * q;
+            if (c >= kChunks) break;
+            {                                  // A: row c/4, k-chunk c%4
                 const int r = c >> 2, kc = c & 3;
                 const int64_t gm = m0 + r;
                 const int gk = k0 + kc * 8;
                 const int valid = (gm < g.M) ? min(8, max(0, g.K - gk)) : 0;
                 pre[q] = gather8(g.A + gm * g.lda + gk, valid);
-            } else if (BCOL) {                 // B column-major: column c/4, k-chunk c%4
+            }
+            if (BCOL) {                        // B column-major: column c/4, k-chunk c%4
                 const int n = c >> 2, kc = c & 3;
                 const int64_t gn = n0 + n;
                 const int gk = k0 + kc * 8;
                 const int valid = (gn < g.N) ? min(8, max(0, g.K - gk)) : 0;
-                pre[q] = gather8(g.B + gn * g.ldb + gk, valid);
-            } else {                           // B row-major: k-row c/16, n-chunk c%16
-                const int k = c >> 4, nc = c & 15;
+                pre[kPer + q] = gather8(g.B + gn * g.ldb + gk, valid);
+            } else {                           // B row-major: k-row c / (T/8), n-chunk c % (T/8)
+                const int k = c / (BN / 8), nc = c % (BN / 8);
                 const int64_t gk = k0 + k;
                 const int gn = n0 + nc * 8;
                 const int valid = (gk < g.K) ? min(8, max(0, g.N - gn)) : 0;
-                pre[q] = gather8(g.B + gk * g.ldb + gn, valid);
+                pre[kPer + q] = gather8(g.B + gk * g.ldb + gn, valid);
             }
         }
     };
@@ -153,14 +161,14 @@ r35_mma_sync_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
         uint8_t* sa = smem + (kb % STAGES) * kStageBytes;
         uint8_t* sb = sa + kABytes;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int c = t + NT * (q & 1);
-            if (q < 2)
-                *reinterpret_cast<uint4*>(sa + kmajor_chunk_off(c >> 2, c & 3)) = pre[q];
-            else if (BCOL)
-                *reinterpret_cast<uint4*>(sb + kmajor_chunk_off(c >> 2, c & 3)) = pre[q];
+        for (int q = 0; q < kPer; ++q) {
+            const int c = t + NT * q;
+            if (c >= kChunks) break;
+            *reinterpret_cast<uint4*>(sa + kmajor_chunk_off(c >> 2, c & 3)) = pre[q];
+            if (BCOL)
+                *reinterpret_cast<uint4*>(sb + kmajor_chunk_off(c >> 2, c & 3)) = pre[kPer + q];
             else
-                *reinterpret_cast<uint4*>(sb + brow_chunk_off(c >> 4, c & 15)) = pre[q];
+                *reinterpret_cast<uint4*>(sb + brow_chunk_off(c / (BN / 8), c % (BN / 8))) = pre[kPer + q];
         }
         ptx::mbar_arrive(&full[kb % STAGES]);
     };
@@ -176,11 +184,11 @@ r35_mma_sync_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
         }
     }
 
-    float acc[4][4][4];   // [m16 tile][n8 tile][fragment register]
+    float acc[MI][2 * NJJ][4];   // [m16 tile][n8 tile][fragment register]
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < MI; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
+        for (int j = 0; j < 2 * NJJ; ++j)
 #pragma unroll
             for (int r = 0; r < 4; ++r) acc[i][j][r] = 0.f;
 
@@ -214,14 +222,14 @@ r35_mma_sync_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
         const uint32_t sb = sa + kABytes;
 #pragma unroll
         for (int k16 = 0; k16 < BK / 16; ++k16) {
-            uint32_t af[4][4], bf[2][4];
+            uint32_t af[MI][4], bf[NJJ][4];
             // A fragments: lanes 0-15 address rows 0-15 at k chunk 2*k16, lanes 16-31 the same rows at the next chunk
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < MI; ++i)
                 ldmatrix_x4(sa + kmajor_chunk_off(wm + i * 16 + (lane & 15), k16 * 2 + (lane >> 4)), af[i]);
             // B fragments, two n8 tiles per ldmatrix.x4: registers {b0, b1} of tile 2*jj, then of tile 2*jj+1
 #pragma unroll
-            for (int jj = 0; jj < 2; ++jj) {
+            for (int jj = 0; jj < NJJ; ++jj) {
                 if (BCOL) {
                     const int n = wn + jj * 16 + ((lane >> 4) << 3) + (lane & 7);
                     ldmatrix_x4(sb + kmajor_chunk_off(n, k16 * 2 + ((lane >> 3) & 1)), bf[jj]);
@@ -231,9 +239,9 @@ r35_mma_sync_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
                 }
             }
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < MI; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
+                for (int j = 0; j < 2 * NJJ; ++j)
                     mma_m16n8k16(acc[i][j], af[i], bf[j >> 1][(j & 1) * 2], bf[j >> 1][(j & 1) * 2 + 1]);
         }
         __syncwarp();
@@ -263,13 +271,13 @@ r35_mma_sync_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
 
     // Epilogue: fragment register r of tile (i, j) is C[wm + 16 i + lane/4 + 8 (r/2)][wn + 8 j + 2 (lane%4) + r%2].
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < MI; ++i)
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int64_t gm = m0 + wm + i * 16 + (lane >> 2) + h * 8;
             if (gm >= g.M) continue;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < 2 * NJJ; ++j) {
                 const int gn = n0 + wn + j * 8 + (lane & 3) * 2;
                 const float v0 = acc[i][j][h * 2] + (gn < g.N ? bias_at(g, gn) : 0.f);
                 const float v1 = acc[i][j][h * 2 + 1] + (gn + 1 < g.N ? bias_at(g, gn + 1) : 0.f);
@@ -294,33 +302,32 @@ r35_mma_sync_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
         }
 }
 
-template <bool BCOL, bool TMA>
+template <bool BCOL, bool TMA, int T>
 cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& mb, int tiles_m, int tiles_n, int c_vec,
                    int kid, int device, cudaStream_t stream)
 {
-    auto kern = r35_mma_sync_kernel<BCOL, TMA>;
+    auto kern = r35_mma_sync_kernel<BCOL, TMA, T>;
     static bool attr_set[64] = {};   // per instantiation and device
     if (device < 0 || device >= 64 || !attr_set[device]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(T));
         if (e != cudaSuccess) return e;
         if (device >= 0 && device < 64) attr_set[device] = true;
     }
-    kern<<<static_cast<unsigned>(tiles_m) * tiles_n, NT, kSmemBytes, stream>>>(g, ma, mb, tiles_m, tiles_n, c_vec, kid);
+    kern<<<static_cast<unsigned>(tiles_m) * tiles_n, NT, smem_bytes(T), stream>>>(g, ma, mb, tiles_m, tiles_n, c_vec, kid);
     return cudaGetLastError();
 }
 
-}  // namespace
-
 // TMA's rules for a 2-D bf16 operand: 16-byte aligned base, row pitch a
 // multiple of 16 bytes and below 2^40.
-static bool tma_ok35(const void* base, int64_t ld_elems)
+bool tma_ok35(const void* base, int64_t ld_elems)
 {
     return reinterpret_cast<uintptr_t>(base) % 16 == 0 && (ld_elems * 2) % 16 == 0 && ld_elems * 2 < (1ll << 40);
 }
 
-cudaError_t launch_r35_mma_sync(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
+template <int T>
+cudaError_t launch_tile(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
 {
-    const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN;
+    const int64_t tiles_m = (g.M + T - 1) / T, tiles_n = (g.N + T - 1) / T;
     if (tiles_m * tiles_n > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;
     const bool tma = ctx.encode_tiled && tma_ok35(g.A, g.lda) && tma_ok35(g.B, g.ldb);
     const int c_vec = (reinterpret_cast<uintptr_t>(g.C) % 16 == 0) && (g.ldc % (g.c_bf16 ? 8 : 4) == 0);
@@ -328,10 +335,10 @@ cudaError_t launch_r35_mma_sync(const GemmArgs& g, RunContext& ctx, cudaStream_t
     memset(&ma, 0, sizeof ma);
     memset(&mb, 0, sizeof mb);
     if (tma) {
-        bool ok = encode_map_2d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, BM,
+        bool ok = encode_map_2d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, T,
                                 CU_TENSOR_MAP_SWIZZLE_64B);
         if (g.b_col)
-            ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, BN,
+            ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, T,
                                      CU_TENSOR_MAP_SWIZZLE_64B);
         else
             ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, g.ldb * 2, 64, BK,
@@ -342,10 +349,19 @@ cudaError_t launch_r35_mma_sync(const GemmArgs& g, RunContext& ctx, cudaStream_t
     *kernel_id = kid;
     const int tmi = static_cast<int>(tiles_m), tni = static_cast<int>(tiles_n);
     if (g.b_col)
-        return tma ? launch<true, true>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream)
-                   : launch<true, false>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream);
-    return tma ? launch<false, true>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream)
-               : launch<false, false>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream);
+        return tma ? launch<true, true, T>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream)
+                   : launch<true, false, T>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream);
+    return tma ? launch<false, true, T>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream)
+               : launch<false, false, T>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream);
+}
+
+}  // namespace
+
+cudaError_t launch_r35_mma_sync(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
+{
+    // 64 x 64 tiles when 128 x 128 tiles would leave SMs without a CTA (the rule of the staged rungs)
+    return staged_tile_edge(g) == 128 ? launch_tile<128>(g, ctx, stream, kernel_id)
+                                      : launch_tile<64>(g, ctx, stream, kernel_id);
 }
 
 }  // namespace klin

@@ -2,7 +2,8 @@
 // data movement is shared-memory staged, the TMA descriptor is encoded;
 // Introduction: a pipeline presupposes that data movement is staged).
 //
-// 128 x 128 x 32 tiles, a ring of 4 shared-memory stages holding RAW bf16, a
+// T x T x 32 tiles (T = 128, 64 or 32: the largest whose grid still gives every SM a CTA,
+// as in rungs 1 and 2), a ring of 4 shared-memory stages holding RAW bf16, a
 // full/empty mbarrier pair per stage with phase parity.  Loads for k-block
 // kb+3 are in flight while k-block kb is multiplied (fp32 FMA on CUDA cores,
 // bf16 -> fp32 widening when a value is read from shared memory).  With no
@@ -26,9 +27,9 @@
 namespace klin {
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 32, STAGES = 4, NT = 256;
-constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2, kStageBytes = kABytes + kBBytes;
-constexpr int kSmemBytes = STAGES * kStageBytes + 1024 /*alignment slack*/ + 128 /*barriers*/;
+constexpr int BK = 32, STAGES = 4, NT = 256;
+// Shared memory of a T x T tile: STAGES x (A block + B block of T x 32 bf16 each), alignment slack, barriers.
+constexpr int smem_bytes(int T) { return STAGES * (2 * T * BK * 2) + 1024 + 128; }
 
 // Byte offset of B element group inside a stage's B block.
 //   row-major   B: [k][128 n] dense, 256-byte rows
@@ -49,11 +50,17 @@ __device__ __forceinline__ uint4 gather8(const uint16_t* p, int valid)
     return r;
 }
 
-template <bool BCOL, bool TMA>
+template <bool BCOL, bool TMA, int T>
 __global__ void __launch_bounds__(NT)
 r3_pipelined_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     int tiles_m, int tiles_n, int c_vec, int kid)
 {
+    constexpr int BM = T, BN = T;
+    constexpr int TT = T / 16;                         // register tile edge: rows ty + 16 i, TT columns per thread
+    constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2, kStageBytes = kABytes + kBBytes;
+    constexpr int kChunks = T * BK / 8;                // 16-byte chunks of one operand block
+    constexpr int kPer = (kChunks + NT - 1) / NT;      // chunks of each operand a thread moves on the producer-thread path
+    constexpr int kBRow = BN * 2;                      // bytes of one k-row of a row-major B block
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * kStageBytes);
@@ -99,31 +106,33 @@ r3_pipelined_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
         issued = kb + 1;
     };
 
-    // Producer-thread path: 4 chunks of 8 bf16 per thread and stage.
-    uint4 pre[4];
+    // Producer-thread path: up to kPer 16-byte chunks of A and of B per thread and stage.
+    uint4 pre[2 * kPer];
     auto fetch_regs = [&](int kb) {
         const int k0 = kb * BK;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int c = t + NT * (q & 1);
-            if (q < 2) {                       // A: row c/4, k-chunk c%4
+        for (int q = 0; q < kPer; ++q) {
+            const int c = t + NT * q;
+            if (c >= kChunks) break;
+            {                                  // A: row c/4, k-chunk c%4
                 const int r = c >> 2, kc = c & 3;
                 const int64_t gm = m0 + r;
                 const int gk = k0 + kc * 8;
                 const int valid = (gm < g.M) ? min(8, max(0, g.K - gk)) : 0;
                 pre[q] = gather8(g.A + gm * g.lda + gk, valid);
-            } else if (BCOL) {                 // B column-major: column c/4, k-chunk c%4
+            }
+            if (BCOL) {                        // B column-major: column c/4, k-chunk c%4
                 const int n = c >> 2, kc = c & 3;
                 const int64_t gn = n0 + n;
                 const int gk = k0 + kc * 8;
                 const int valid = (gn < g.N) ? min(8, max(0, g.K - gk)) : 0;
-                pre[q] = gather8(g.B + gn * g.ldb + gk, valid);
-            } else {                           // B row-major: k-row c/16, n-chunk c%16
-                const int k = c >> 4, nc = c & 15;
+                pre[kPer + q] = gather8(g.B + gn * g.ldb + gk, valid);
+            } else {                           // B row-major: k-row c / (T/8), n-chunk c % (T/8)
+                const int k = c / (BN / 8), nc = c % (BN / 8);
                 const int64_t gk = k0 + k;
                 const int gn = n0 + nc * 8;
                 const int valid = (gk < g.K) ? min(8, max(0, g.N - gn)) : 0;
-                pre[q] = gather8(g.B + gk * g.ldb + gn, valid);
+                pre[kPer + q] = gather8(g.B + gk * g.ldb + gn, valid);
             }
         }
     };
@@ -131,14 +140,14 @@ r3_pipelined_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
         uint8_t* sa = smem + (kb % STAGES) * kStageBytes;
         uint8_t* sb = sa + kABytes;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int c = t + NT * (q & 1);
-            if (q < 2)
-                *reinterpret_cast<uint4*>(sa + (c >> 2) * 64 + (c & 3) * 16) = pre[q];
-            else if (BCOL)
-                *reinterpret_cast<uint4*>(sb + b_col_chunk_off(c >> 2, c & 3)) = pre[q];
+        for (int q = 0; q < kPer; ++q) {
+            const int c = t + NT * q;
+            if (c >= kChunks) break;
+            *reinterpret_cast<uint4*>(sa + (c >> 2) * 64 + (c & 3) * 16) = pre[q];
+            if (BCOL)
+                *reinterpret_cast<uint4*>(sb + b_col_chunk_off(c >> 2, c & 3)) = pre[kPer + q];
             else
-                *reinterpret_cast<uint4*>(sb + (c >> 4) * 256 + (c & 15) * 16) = pre[q];
+                *reinterpret_cast<uint4*>(sb + (c / (BN / 8)) * kBRow + (c % (BN / 8)) * 16) = pre[kPer + q];
         }
         ptx::mbar_arrive(&full[kb % STAGES]);
     };
@@ -154,11 +163,11 @@ r3_pipelined_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
         }
     }
 
-    float2 acc2[8][4];   // acc2[i][jp] = accumulators of columns 2*jp and 2*jp+1 of row i
+    float2 acc2[TT][TT / 2];   // acc2[i][jp] = accumulators of columns 2*jp and 2*jp+1 of row i
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < TT; ++i)
 #pragma unroll
-        for (int jp = 0; jp < 4; ++jp) acc2[i][jp] = make_float2(0.f, 0.f);
+        for (int jp = 0; jp < TT / 2; ++jp) acc2[i][jp] = make_float2(0.f, 0.f);
 
     for (int kb = 0; kb < nkb && ok; ++kb) {
         const int s = kb % STAGES;
@@ -190,47 +199,59 @@ r3_pipelined_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
         const uint8_t* sb = sa + kABytes;
 #pragma unroll
         for (int kk = 0; kk < BK / 8; ++kk) {
-            uint32_t aw[8][4];
+            uint32_t aw[TT][4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < TT; ++i) {
                 const uint4 v = *reinterpret_cast<const uint4*>(sa + (ty + 16 * i) * 64 + kk * 16);
                 aw[i][0] = v.x; aw[i][1] = v.y; aw[i][2] = v.z; aw[i][3] = v.w;
             }
             if (BCOL) {
-                uint32_t bw[8][4];
+                uint32_t bw[TT][4];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
+                for (int j = 0; j < TT; ++j) {
                     const uint4 v = *reinterpret_cast<const uint4*>(sb + b_col_chunk_off(tx + 16 * j, kk));
                     bw[j][0] = v.x; bw[j][1] = v.y; bw[j][2] = v.z; bw[j][3] = v.w;
                 }
 #pragma unroll
                 for (int k8 = 0; k8 < 8; ++k8) {
-                    float2 b2[4];
+                    float2 b2[TT / 2];
 #pragma unroll
-                    for (int jp = 0; jp < 4; ++jp) {
+                    for (int jp = 0; jp < TT / 2; ++jp) {
                         b2[jp].x = (k8 & 1) ? bf16_hi(bw[2 * jp][k8 >> 1]) : bf16_lo(bw[2 * jp][k8 >> 1]);
                         b2[jp].y = (k8 & 1) ? bf16_hi(bw[2 * jp + 1][k8 >> 1]) : bf16_lo(bw[2 * jp + 1][k8 >> 1]);
                     }
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
+                    for (int i = 0; i < TT; ++i) {
                         const float a = (k8 & 1) ? bf16_hi(aw[i][k8 >> 1]) : bf16_lo(aw[i][k8 >> 1]);
                         const float2 a2 = make_float2(a, a);
 #pragma unroll
-                        for (int jp = 0; jp < 4; ++jp) acc2[i][jp] = __ffma2_rn(a2, b2[jp], acc2[i][jp]);
+                        for (int jp = 0; jp < TT / 2; ++jp) acc2[i][jp] = __ffma2_rn(a2, b2[jp], acc2[i][jp]);
                     }
                 }
             } else {
 #pragma unroll
                 for (int k8 = 0; k8 < 8; ++k8) {
-                    const uint4 v = *reinterpret_cast<const uint4*>(sb + (kk * 8 + k8) * 256 + tx * 16);
-                    const float2 b2[4] = {make_float2(bf16_lo(v.x), bf16_hi(v.x)), make_float2(bf16_lo(v.y), bf16_hi(v.y)),
-                                          make_float2(bf16_lo(v.z), bf16_hi(v.z)), make_float2(bf16_lo(v.w), bf16_hi(v.w))};
+                    // this thread's TT consecutive columns of k-row kk * 8 + k8: 16, 8 or 4 bytes
+                    uint32_t w[TT / 2];
+                    const uint8_t* src = sb + (kk * 8 + k8) * kBRow + tx * (TT * 2);
+                    if constexpr (TT == 8) {
+                        const uint4 v = *reinterpret_cast<const uint4*>(src);
+                        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+                    } else if constexpr (TT == 4) {
+                        const uint2 v = *reinterpret_cast<const uint2*>(src);
+                        w[0] = v.x; w[1] = v.y;
+                    } else {
+                        w[0] = *reinterpret_cast<const uint32_t*>(src);
+                    }
+                    float2 b2[TT / 2];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
+                    for (int jp = 0; jp < TT / 2; ++jp) b2[jp] = make_float2(bf16_lo(w[jp]), bf16_hi(w[jp]));
+#pragma unroll
+                    for (int i = 0; i < TT; ++i) {
                         const float a = (k8 & 1) ? bf16_hi(aw[i][k8 >> 1]) : bf16_lo(aw[i][k8 >> 1]);
                         const float2 a2 = make_float2(a, a);
 #pragma unroll
-                        for (int jp = 0; jp < 4; ++jp) acc2[i][jp] = __ffma2_rn(a2, b2[jp], acc2[i][jp]);
+                        for (int jp = 0; jp < TT / 2; ++jp) acc2[i][jp] = __ffma2_rn(a2, b2[jp], acc2[i][jp]);
                     }
                 }
             }
@@ -260,82 +281,96 @@ r3_pipelined_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const
         return;
     }
 
-    // Epilogue: rows ty + 16 i; columns tx*8 + j (row-major B) or tx + 16 j.
-    float acc[8][8];
+    // Epilogue: rows ty + 16 i; columns tx * TT + j (row-major B) or tx + 16 j.
+    float acc[TT][TT];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < TT; ++i)
 #pragma unroll
-        for (int jp = 0; jp < 4; ++jp) {
+        for (int jp = 0; jp < TT / 2; ++jp) {
             acc[i][2 * jp] = acc2[i][jp].x;
             acc[i][2 * jp + 1] = acc2[i][jp].y;
         }
-    if (g.bias) {   // AddMM: the bias of each of this thread's 8 columns
+    if (g.bias) {   // AddMM: the bias of each of this thread's columns
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int gn = n0 + (BCOL ? tx + 16 * j : tx * 8 + j);
+        for (int j = 0; j < TT; ++j) {
+            const int gn = n0 + (BCOL ? tx + 16 * j : tx * TT + j);
             const float b = gn < g.N ? bias_at(g, gn) : 0.f;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) acc[i][j] += b;
+            for (int i = 0; i < TT; ++i) acc[i][j] += b;
         }
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < TT; ++i) {
         const int64_t gm = m0 + ty + 16 * i;
         if (gm >= g.M) continue;
         if (BCOL) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+            for (int j = 0; j < TT; ++j) {
                 const int gn = n0 + tx + 16 * j;
                 if (gn < g.N) store_c(g.C, g.c_bf16, gm * g.ldc + gn, acc[i][j]);
             }
         } else {
-            const int gn = n0 + tx * 8;
-            if (c_vec && gn + 8 <= g.N) {
-                if (g.c_bf16) {
-                    uint4 w = make_uint4(pack_bf16x2(acc[i][0], acc[i][1]), pack_bf16x2(acc[i][2], acc[i][3]),
-                                         pack_bf16x2(acc[i][4], acc[i][5]), pack_bf16x2(acc[i][6], acc[i][7]));
-                    *reinterpret_cast<uint4*>(static_cast<uint16_t*>(g.C) + gm * g.ldc + gn) = w;
-                } else {
-                    float* p = static_cast<float*>(g.C) + gm * g.ldc + gn;
-                    *reinterpret_cast<float4*>(p) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-                    *reinterpret_cast<float4*>(p + 4) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+            const int gn = n0 + tx * TT;
+            bool done = false;
+            if constexpr (TT == 8) {
+                if (c_vec && gn + 8 <= g.N) {
+                    if (g.c_bf16) {
+                        uint4 w = make_uint4(pack_bf16x2(acc[i][0], acc[i][1]), pack_bf16x2(acc[i][2], acc[i][3]),
+                                             pack_bf16x2(acc[i][4], acc[i][5]), pack_bf16x2(acc[i][6], acc[i][7]));
+                        *reinterpret_cast<uint4*>(static_cast<uint16_t*>(g.C) + gm * g.ldc + gn) = w;
+                    } else {
+                        float* p = static_cast<float*>(g.C) + gm * g.ldc + gn;
+                        *reinterpret_cast<float4*>(p) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                        *reinterpret_cast<float4*>(p + 4) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+                    }
+                    done = true;
                 }
-            } else {
+            } else if constexpr (TT == 4) {
+                if (c_vec && gn + 4 <= g.N) {      // (C 16-byte aligned, pitch a multiple of 16 bytes: 4 columns are 8 / 16 bytes)
+                    if (g.c_bf16)
+                        *reinterpret_cast<uint2*>(static_cast<uint16_t*>(g.C) + gm * g.ldc + gn) =
+                            make_uint2(pack_bf16x2(acc[i][0], acc[i][1]), pack_bf16x2(acc[i][2], acc[i][3]));
+                    else
+                        *reinterpret_cast<float4*>(static_cast<float*>(g.C) + gm * g.ldc + gn) =
+                            make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                    done = true;
+                }
+            }
+            if (!done) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
+                for (int j = 0; j < TT; ++j)
                     if (gn + j < g.N) store_c(g.C, g.c_bf16, gm * g.ldc + gn + j, acc[i][j]);
             }
         }
     }
 }
 
-template <bool BCOL, bool TMA>
+template <bool BCOL, bool TMA, int T>
 cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& mb, int tiles_m, int tiles_n, int c_vec,
                    int kid, int device, cudaStream_t stream)
 {
-    auto kern = r3_pipelined_kernel<BCOL, TMA>;
+    auto kern = r3_pipelined_kernel<BCOL, TMA, T>;
     static bool attr_set[64] = {};   // per instantiation and device
     if (device < 0 || device >= 64 || !attr_set[device]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(T));
         if (e != cudaSuccess) return e;
         if (device >= 0 && device < 64) attr_set[device] = true;
     }
-    kern<<<static_cast<unsigned>(tiles_m) * tiles_n, NT, kSmemBytes, stream>>>(g, ma, mb, tiles_m, tiles_n, c_vec, kid);
+    kern<<<static_cast<unsigned>(tiles_m) * tiles_n, NT, smem_bytes(T), stream>>>(g, ma, mb, tiles_m, tiles_n, c_vec, kid);
     return cudaGetLastError();
 }
 
-}  // namespace
-
 // TMA's rules for a 2-D bf16 operand: 16-byte aligned base, row pitch a
 // multiple of 16 bytes and below 2^40.
-static bool tma_ok(const void* base, int64_t ld_elems)
+bool tma_ok(const void* base, int64_t ld_elems)
 {
     return reinterpret_cast<uintptr_t>(base) % 16 == 0 && (ld_elems * 2) % 16 == 0 && ld_elems * 2 < (1ll << 40);
 }
 
-cudaError_t launch_r3_pipelined(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
+template <int T>
+cudaError_t launch_tile(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
 {
-    const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN;
+    const int64_t tiles_m = (g.M + T - 1) / T, tiles_n = (g.N + T - 1) / T;
     if (tiles_m * tiles_n > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;
     const bool tma = ctx.encode_tiled && tma_ok(g.A, g.lda) && tma_ok(g.B, g.ldb);
     const int c_vec = (reinterpret_cast<uintptr_t>(g.C) % 16 == 0) && (g.ldc % (g.c_bf16 ? 8 : 4) == 0);
@@ -343,13 +378,13 @@ cudaError_t launch_r3_pipelined(const GemmArgs& g, RunContext& ctx, cudaStream_t
     memset(&ma, 0, sizeof ma);
     memset(&mb, 0, sizeof mb);
     if (tma) {
-        bool ok = encode_map_2d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, BM,
+        bool ok = encode_map_2d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, T,
                                 CU_TENSOR_MAP_SWIZZLE_NONE);
         if (g.b_col)
-            ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, BN,
+            ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.K, g.N, g.ldb * 2, BK, T,
                                      CU_TENSOR_MAP_SWIZZLE_64B);
         else
-            ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, g.ldb * 2, BN, BK,
+            ok = ok && encode_map_2d(ctx, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.B, g.N, g.K, g.ldb * 2, T, BK,
                                      CU_TENSOR_MAP_SWIZZLE_NONE);
         if (!ok) return cudaErrorInvalidValue;
     }
@@ -357,10 +392,21 @@ cudaError_t launch_r3_pipelined(const GemmArgs& g, RunContext& ctx, cudaStream_t
     *kernel_id = kid;
     const int tmi = static_cast<int>(tiles_m), tni = static_cast<int>(tiles_n);
     if (g.b_col)
-        return tma ? launch<true, true>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream)
-                   : launch<true, false>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream);
-    return tma ? launch<false, true>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream)
-               : launch<false, false>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream);
+        return tma ? launch<true, true, T>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream)
+                   : launch<true, false, T>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream);
+    return tma ? launch<false, true, T>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream)
+               : launch<false, false, T>(g, ma, mb, tmi, tni, c_vec, kid, ctx.device, stream);
+}
+
+}  // namespace
+
+cudaError_t launch_r3_pipelined(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
+{
+    switch (staged_tile_edge(g)) {
+        case 128: return launch_tile<128>(g, ctx, stream, kernel_id);
+        case 64: return launch_tile<64>(g, ctx, stream, kernel_id);
+        default: return launch_tile<32>(g, ctx, stream, kernel_id);
+    }
 }
 
 }  // namespace klin
