@@ -67,7 +67,9 @@ __device__ __forceinline__ uint16_t float_to_bf16_bits(float f)
 // Two floats -> packed bf16x2 (lo in bits 0..15), round to nearest even.
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
-    return static_cast<uint32_t>(float_to_bf16_bits(lo)) | (static_cast<uint32_t>(float_to_bf16_bits(hi)) << 16);
+    // one packed conversion instruction (cvt.rn.bf16x2.f32) instead of two scalar ones and a merge
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
 }
 
 // Two floats -> packed 16-bit pair in the output type (bf16 or fp16), round to nearest even.

@@ -59,10 +59,11 @@ constexpr int kThreads = 12 * 32;                // warp group 0: producer, MMA 
 constexpr int kEpiWarp0 = 4;                     // first epilogue warp
 // Registers: the kernel is compiled for 168 per thread (three warps share a 16 K-register scheduler
 // partition); the first warp group gives its surplus back (setmaxnreg.dec) and the epilogue groups
-// take it (setmaxnreg.inc), so that three fp32 units of the accumulator fit in registers at once.
+// take it (setmaxnreg.inc), so that three fp32 units of the accumulator fit in registers at once
+// (the compiler allocates each region against its own limit: at 40 / 232 the epilogue spilled).
 // The two amounts must balance (the pool the increase draws from holds only what was released:
 // with 48 instead of 40 the increase never completed and the launch hung).
-constexpr int kRegsLean = 40, kRegsEpilogue = 232;   // balanced: 128 x (168 - 40) released = 256 x (232 - 168) taken
+constexpr int kRegsLean = 24, kRegsEpilogue = 240;   // balanced: 128 x (168 - 24) released = 256 x (240 - 168) taken
 
 struct PairParams {
     int tiles_m2, tiles_n;      // 512-row x 256-column tiles
