@@ -202,6 +202,7 @@ klineage_status_t klineage_gemm_last_give_up(klineage_gemm_t h, unsigned* block_
  *   300 TMA pipeline, 301 producer-thread pipeline
  *   400 + 1*(generic-proxy producer) + 2*(direct epilogue) + 4*(split-K) + 8*(skinny mode)
  *       + 16*(cluster reduce) + 32*(CTA-pair MMA) + 64*(unaligned operands repacked into the workspace)
+ *       + 128*(last wave of CTA-pair tiles streamed along K)
  *   500 mma.sync rung on the TMA ring, 501 on producer threads
  *   900 zero fill (K == 0); -1 before the first run or after a no-op.
  */
@@ -424,7 +425,11 @@ klineage_status_t klineage_gemm_run_host(klineage_gemm_t h, int64_t M, int64_t N
  *   kernel     1 single-CTA kernel (128 x 256 tiles), 2 CTA-pair kernel (512 x 256 tiles)
  *   splits     number of K splits (1 = none)
  *   split_via  with splits > 1: 1 partial sums through the global workspace,
- *              2 through a thread-block cluster (splits 2 / 4 / 8; M <= 32 or M > 64)
+ *              2 through a thread-block cluster (splits 2 / 4 / 8; M <= 32 or M > 64);
+ *              with kernel 2 and splits 1: 3 streams the under-filled last wave of pair tiles along K (the
+ *              k-blocks of its tiles are dealt out evenly over all CTA pairs; pieces that do not hold a tile's
+ *              first k-block pass their fp32 partial tile through the workspace, the piece that does adds them
+ *              in k order - a fixed order, so results repeat bit for bit), 1 never does
  *   group_m    tile-rows per raster group (L2 reuse pattern)
  *   half_tail  1 cut the last wave into 128-column half tiles, 2 never
  *   tile_n     columns per output tile (needs `kernel`): single-CTA kernel 256 or 128; CTA-pair kernel a

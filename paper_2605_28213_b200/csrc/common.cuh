@@ -43,7 +43,7 @@ enum KernelId : int {
     kIdVectorized = 200,      // + 1 (A vector loads) + 2 (B vector loads) + 4 (C vector stores)
     kIdPipelined = 300,       // + 1 when the producer-thread path replaces TMA
     kIdTcgen05 = 400,         // + 1 generic-proxy producer, + 2 direct epilogue, + 4 split-K, + 8 skinny (swapped operands), + 16 cluster reduce, + 32 CTA pair,
-                              // + 64 unaligned operands repacked into the workspace first
+                              // + 64 unaligned operands repacked into the workspace first, + 128 last wave of pair tiles streamed along K
     kIdMmaSync = 500,         // rung 3.5 (mma.sync); + 1 when the producer-thread path replaces TMA
     kIdConvNaive = 600,       // direct convolution, one thread per output
     kIdConvTcgen05 = 700,     // implicit GEMM on the tcgen05 rung, patches by TMA; + 4 patches gathered by producer threads,
@@ -157,7 +157,8 @@ typedef CUresult (*TensorMapEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cu
 struct R4Plan {
     int kernel = 0;      // 0 auto, 1 single-CTA kernel, 2 CTA-pair kernel
     int splits = 0;      // 0 auto, 1 no K split, n > 1 K splits
-    int split_via = 0;   // with splits > 1: 0 auto, 1 global workspace, 2 cluster (distributed shared memory)
+    int split_via = 0;   // with splits > 1: 0 auto, 1 global workspace, 2 cluster (distributed shared memory);
+                         // pair kernel (splits == 1): 0 auto, 1 whole tiles only, 3 stream the last wave along K
     int group_m = 0;     // 0 auto, else tile-rows per raster group
     int half_tail = 0;   // 0 auto, 1 cut the last wave into half tiles, 2 never
     int tile_n = 0;      // 0 auto, else columns per output tile (pair kernel: a multiple of 64, at most 256;
@@ -176,6 +177,9 @@ struct RunContext {
     TensorMapEncodeTiledFn encode_tiled = nullptr;   // from cudaGetDriverEntryPoint
     void* workspace = nullptr;                       // split-K partial sums (fp32)
     size_t workspace_bytes = 0;
+    unsigned* sk_flags = nullptr;                    // streamed last wave of the pair kernel: one flag per (pair, CTA,
+                                                     // epilogue warp), holding the epoch of the launch that wrote it
+    unsigned sk_epoch = 0;                           // bumped by every launch that streams its last wave
     unsigned* tile_counters = nullptr;               // split-K arrival counters, zero between calls
     int n_tile_counters = 0;
     unsigned flags = 0;
@@ -245,6 +249,9 @@ cudaError_t launch_zero_fill(const GemmArgs& g, cudaStream_t stream, int* kernel
 bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx);
 // Hard preconditions of the CTA-pair kernel only (operands TMA-loadable), without the size heuristic.
 bool r4_pair_possible(const GemmArgs& g, const RunContext& ctx);
+// Whether the pair kernel can stream this problem's last wave along K (enough k-blocks per piece, workspace for the
+// partial tiles, every pair of the grid resident).
+bool r4_pair_stream_k_possible(const GemmArgs& g, const RunContext& ctx);
 // True when `plan` can run this problem on the tcgen05 rung (the launcher refuses it otherwise).
 bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& plan);
 // Candidate plans of a problem, the all-zero heuristic plan first; returns how many were written.

@@ -292,6 +292,9 @@ klineage_status_t klineage_gemm_create(klineage_gemm_t* out, const klineage_gemm
     bool ok = cudaMalloc(&c.workspace, c.workspace_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(reinterpret_cast<void**>(&c.tile_counters), sizeof(unsigned) * kTileCounters) == cudaSuccess;
     ok = ok && cudaMalloc(reinterpret_cast<void**>(&h->status), 4 * sizeof(unsigned)) == cudaSuccess;
+    const size_t n_sk_flags = static_cast<size_t>(c.sm_count > 0 ? c.sm_count : 1) * 8;     // (SMs / 2 pairs) x 2 CTAs x 8 warps
+    ok = ok && cudaMalloc(reinterpret_cast<void**>(&c.sk_flags), n_sk_flags * sizeof(unsigned)) == cudaSuccess;
+    ok = ok && cudaMemset(c.sk_flags, 0, n_sk_flags * sizeof(unsigned)) == cudaSuccess;
     ok = ok && cudaMemset(c.tile_counters, 0, sizeof(unsigned) * kTileCounters) == cudaSuccess;
     ok = ok && cudaMemset(h->status, 0, 4 * sizeof(unsigned)) == cudaSuccess;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
@@ -311,6 +314,7 @@ klineage_status_t klineage_gemm_destroy(klineage_gemm_t h)
         DeviceGuard guard(h->ctx.device);
         if (h->ctx.workspace) cudaFree(h->ctx.workspace);
         if (h->ctx.tile_counters) cudaFree(h->ctx.tile_counters);
+        if (h->ctx.sk_flags) cudaFree(h->ctx.sk_flags);
         if (h->status) cudaFree(h->status);
         release_host_pipe(h);
     }

@@ -1892,7 +1892,10 @@ cudaError_t launch_r4_tcgen05(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     // The promise "no in-flight work writes B" is about the caller's B; the copy just enqueued IS in-flight
     // work that writes the B this launch reads, so its loads must wait for it like every other access.
     if (bad_b) c2.flags &= ~1u;
-    return launch_r4_planned(g2, c2, stream, kernel_id);
+    const cudaError_t e = launch_r4_planned(g2, c2, stream, kernel_id);
+    ctx.sk_epoch = c2.sk_epoch;          // (state the launch advanced lives in the caller's context)
+    ctx.flags &= c2.flags | 1u;          // a one-shot test hook that fired stays fired
+    return e;
 }
 
 namespace {
@@ -2367,7 +2370,7 @@ cudaError_t launch_r4_multi_dst(const GemmArgs& g, void* const* C, const int64_t
 
 bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& pl)
 {
-    if (pl.kernel < 0 || pl.kernel > 2 || pl.splits < 0 || pl.split_via < 0 || pl.split_via > 2 || pl.group_m < 0 ||
+    if (pl.kernel < 0 || pl.kernel > 2 || pl.splits < 0 || pl.split_via < 0 || pl.split_via > 3 || pl.group_m < 0 ||
         pl.group_m > 1024 || pl.half_tail < 0 || pl.half_tail > 2 || pl.tile_n < 0 || pl.tail_n < 0 || pl.stages < 0)
         return false;
     // tile widths: the pair kernel takes multiples of 64 columns (and a second, narrower width for the tiles
@@ -2376,6 +2379,7 @@ bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& pl)
     if (pl.tail_n != 0 && (pl.tail_n < 64 || pl.tail_n > 256 || pl.tail_n % 64 != 0 || pl.tail_n > (pl.tile_n ? pl.tile_n : 256)))
         return false;
     if (pl.tail_n != 0 && pl.kernel != 2) return false;
+    if (pl.split_via == 3 && (pl.kernel != 2 || pl.splits > 1)) return false;     // streaming the last wave is the pair kernel's
     if (pl.kernel == 2 && pl.stages != 0) return false;
     if (pl.kernel != 2 && (pl.tile_n != 0 || pl.stages != 0)) {
         // single-CTA kernel: 256 columns x 4 stages, or 128 columns x 4 or 6 stages (plain TMA-fed GEMM, M > 64)
@@ -2393,6 +2397,8 @@ bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& pl)
     if (!plan_launch(g, c2, !aligned && !ctx.allow_repack, false, &lp)) return false;
     const SplitPlan& sp = lp.split;
     if (pl.kernel == 2 && (sp.swap || sp.splits != 1 || !r4_pair_possible(g, ctx))) return false;
+    if (pl.split_via == 3 && (pl.tile_n % 256 != 0 || (pl.tail_n != 0 && pl.tail_n != 256) || !r4_pair_stream_k_possible(g, ctx)))
+        return false;
     return true;
 }
 
@@ -2443,6 +2449,14 @@ int r4_enumerate_plans(const GemmArgs& g, const RunContext& ctx, R4Plan* out, in
             pl.tile_n = 256;
             pl.tail_n = 192;
             push(pl);
+            // last wave streamed along K, and never streamed
+            for (int via : {3, 1}) {
+                R4Plan ps;
+                ps.kernel = 2;
+                ps.splits = 1;
+                ps.split_via = via;
+                push(ps);
+            }
         }
         // tile shapes of the single-CTA kernel: 128 columns on a 4- or 6-stage ring
         for (int st : {4, 6}) {

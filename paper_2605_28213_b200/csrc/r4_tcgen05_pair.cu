@@ -81,6 +81,22 @@ struct PairParams {
     int snake;                  // 1: odd rounds of the schedule run over the pairs in reverse order
     uint32_t stage_tx;          // bytes the loads of both CTAs deliver per stage
     int b_boxes;                // row-major B: 64-column boxes per CTA and stage (1 or 2)
+    // Streamed last wave (MODE 0, uniform 256-column tiles).  Tiles [0, sk_first) run whole, sk_rounds of them per
+    // pair; the k-blocks of the remaining tiles - one under-filled wave - are laid end to end (sk_work of them) and
+    // pair q takes the contiguous range [q * sk_work / pairs, (q + 1) * sk_work / pairs).  A range that starts
+    // inside a tile begins with a piece that does not hold the tile's first k-block: the pair computes it FIRST,
+    // writes the fp32 partial tile to its slot of the workspace and raises the slot's flags; the piece that holds
+    // a tile's first k-block comes after it in its pair's order, reads the partials of the pairs after it (whose
+    // first pieces are shorter than this pair's two) in k order, adds them and stores the tile; the whole tiles
+    // come last.  No pair ever waits for work that has not been started, sums are added in a fixed order,
+    // nothing is atomic.
+    int sk;                     // 1: the schedule above
+    int sk_rounds;
+    int64_t sk_first;
+    int64_t sk_work;
+    float* sk_slots;            // [pair][128 blocks of 32 rows x 32 columns] fp32, a block laid out [column / 4][row][column % 4]
+    unsigned* sk_flags;         // [pair][CTA of the pair][epilogue warp]: the launch's epoch once the warp's rows are written
+    unsigned sk_epoch;
     uint32_t idesc;
     uint32_t b_desc_hi, b_desc_lbo, b_kstep;
     // batched launches (MODE 1): the schedule runs over batch x tiles_per_batch
@@ -302,6 +318,66 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         const int64_t idx = static_cast<int64_t>(r) * n_pairs + ((p.snake && (r & 1u)) ? n_pairs - 1 - pair_id : pair_id);
         return idx < p.total_tiles ? idx : -1;
     };
+    // One item of this pair's work list: a tile and the k-blocks [kb0, kb1) of it.  kind 0: the whole tile;
+    // 1: a piece without the tile's first k-block - its partial sums go to this pair's workspace slot;
+    // 2: a piece with the first but not the last k-block - it adds the partial sums of the pairs after it.
+    struct Work {
+        int64_t tile;
+        int kb0, kb1, kind;
+    };
+    struct WorkState {
+        uint32_t i;             // whole-tile rounds handed out so far
+        int64_t pos, end;       // streamed range still to hand out (k-blocks of the streamed region)
+        bool first_done;
+    };
+    auto work_init = [&]() {
+        WorkState st = {0u, 0, 0, false};
+        if (MODE == 0 && p.sk) {
+            st.pos = pair_id * p.sk_work / n_pairs;
+            st.end = (pair_id + 1) * p.sk_work / n_pairs;
+        }
+        return st;
+    };
+    auto next_work = [&](WorkState& st, Work& w) -> bool {
+        if (!(MODE == 0 && p.sk)) {
+            const int64_t t = tile_at(st.i++);
+            if (t < 0) return false;
+            w.tile = t;
+            w.kb0 = 0;
+            w.kb1 = -1;         // the tile's own k-block count
+            w.kind = 0;
+            return true;
+        }
+        const int nkb = p.nkb;
+        if (!st.first_done) {   // first: the piece that starts inside a tile
+            st.first_done = true;
+            const int off = static_cast<int>(st.pos % nkb);
+            if (off != 0 && st.pos < st.end) {
+                w.tile = p.sk_first + st.pos / nkb;
+                w.kb0 = off;
+                w.kb1 = static_cast<int>(min(static_cast<int64_t>(nkb), off + (st.end - st.pos)));
+                w.kind = 1;
+                st.pos += w.kb1 - w.kb0;
+                return true;
+            }
+        }
+        if (st.pos < st.end) {  // then the rest of the range, tile by tile (it starts at a tile's first k-block)
+            w.tile = p.sk_first + st.pos / nkb;
+            w.kb0 = 0;
+            w.kb1 = static_cast<int>(min(static_cast<int64_t>(nkb), st.end - st.pos));
+            w.kind = w.kb1 == nkb ? 0 : 2;
+            st.pos += w.kb1;
+            return true;
+        }
+        if (st.i < static_cast<uint32_t>(p.sk_rounds)) {       // last the whole tiles of the full rounds: the adding of
+            w.tile = static_cast<int64_t>(st.i++) * n_pairs + pair_id;   // partial sums above hides behind their MMAs
+            w.kb0 = 0;
+            w.kb1 = nkb;
+            w.kind = 0;
+            return true;
+        }
+        return false;
+    };
     // One operand box of a stage; completion is counted on the even CTA's barrier.
     auto load_box = [&](void* dst, const CUtensorMap* map, int c0, int c1, int z, uint32_t bar) {
         if (MODE == 1)
@@ -319,13 +395,14 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (uint32_t r = 0; ok; ++r) {
-                const int64_t t = tile_at(r);
-                if (t < 0) break;
-                const TileInfo x = tile_info(t);
+            WorkState ws = work_init();
+            Work wk;
+            while (ok && next_work(ws, wk)) {
+                const TileInfo x = tile_info(wk.tile);
                 const int m0 = x.m0;
                 const int nb = x.n0 + static_cast<int>(rank) * (x.width >> 1);    // this CTA's half of B
-                for (int kb = 0; kb < x.nkb; ++kb, ++it) {
+                const int kb_end = wk.kb1 < 0 ? x.nkb : wk.kb1;
+                for (int kb = wk.kb0; kb < kb_end; ++kb, ++it) {
                     const int s = it % STAGES;
                     if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
                         report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x500u | s);
@@ -361,9 +438,10 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             // -------------------------------------------------------- MMA issuer (even CTA)
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            for (;ok; ++tcount) {
-                const int64_t t = tile_at(tcount);
-                if (t < 0) break;
+            WorkState ws = work_init();
+            Work wk;
+            for (; ok && next_work(ws, wk); ++tcount) {
+                const int64_t t = wk.tile;
                 // Both accumulators are rewritten: wait until both CTAs' epilogues drained the last tile.
                 if (!ptx::mbar_wait(&acc_empty[0], (tcount & 1) ^ 1, abort_flag)) {
                     report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x520u);
@@ -372,10 +450,10 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 }
                 ptx::tc_fence_after_sync();
                 const TileInfo x = tile_info(t);
-                const int nkb = x.nkb;
+                const int kb_first = wk.kb0, kb_end = wk.kb1 < 0 ? x.nkb : wk.kb1;
                 // the MMA's N is the tile's width
                 const uint32_t idesc = (p.idesc & ~(0x3Fu << 17)) | (static_cast<uint32_t>(x.width >> 3) << 17);
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                for (int kb = kb_first; kb < kb_end; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t par = (it / STAGES) & 1;
                     if (!ptx::mbar_wait(&full[s], par, abort_flag)) {
@@ -391,7 +469,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     const uint64_t b_desc = make_desc(sb, p.b_desc_lbo, p.b_desc_hi);
 #pragma unroll
                     for (int k4 = 0; k4 < BK / 16; ++k4) {
-                        const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
+                        const uint32_t acc = (kb > kb_first || k4 > 0) ? 1u : 0u;
                         // alternate the two row blocks: consecutive MMAs never share an accumulator
                         umma_f16_pair(tmem_base, a_desc + static_cast<uint64_t>(k4 * 2),
                                       b_desc + static_cast<uint64_t>(k4 * p.b_kstep), idesc, acc);
@@ -422,10 +500,10 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         const int cpc = out_bf16 ? 64 : 32;                   // columns per 128-byte staging row
         uint32_t tcount = 0;
         bool ok = true;
-        for (; ok; ++tcount) {
-            const int64_t t = tile_at(tcount);
-            if (t < 0) break;
-            const TileInfo x = tile_info(t);
+        WorkState ws = work_init();
+        Work wk;
+        for (; ok && next_work(ws, wk); ++tcount) {
+            const TileInfo x = tile_info(wk.tile);
             const int m0 = x.m0, n0 = x.n0;
             float* dst_f = reinterpret_cast<float*>(x.C);
             uint16_t* dst_h = reinterpret_cast<uint16_t*>(x.C);
@@ -440,6 +518,8 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             const int rows = min(32, x.M - row0);
             const int nunits = (row0 < x.M) ? (min(x.width, x.N - n0) + cpc - 1) / cpc : 0;
             const uint32_t tbase = tmem_base + mb * PN + (static_cast<uint32_t>(q * 32) << 16);
+            // first 4 KiB block of this warp's rows inside a partial-tile slot: (CTA, row block, lane quarter) x 8 column blocks
+            const int64_t sk_block = ((static_cast<int64_t>(rank) * 2 + mb) * 4 + q) * (PN / 32);
 
             auto release = [&]() {
                 ptx::tc_fence_before_sync();
@@ -531,18 +611,107 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     __syncwarp();
                 }
             };
-            auto finish = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32]) {
-                uint32_t w[32];
-                pack(u, r0, r1, w);
-                stage_store(u, w);
+            if (MODE == 0 && wk.kind == 1) {
+                // A piece without the tile's first k-block: this warp's 32 rows of the raw fp32 partial tile go to the
+                // pair's workspace slot, as 4 KiB blocks of 32 rows x 32 columns laid out [column / 4][row][column % 4]
+                // (a warp's store instruction writes 512 contiguous bytes); then the accumulator is handed back and
+                // the warp's flag tells the owner its rows are there.
+                uint4* dst = reinterpret_cast<uint4*>(p.sk_slots + pair_id * (TILE_M * PN) + sk_block * 1024) + lane;
+                uint32_t v0[32], v1[32];
+#pragma unroll 1
+                for (int c = 0; c < PN / 32; c += 2) {
+                    ptx::tmem_ld_32x32b_x32(tbase + c * 32, v0);
+                    ptx::tmem_ld_32x32b_x32(tbase + c * 32 + 32, v1);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        __stcg(dst + c * 256 + j * 32, make_uint4(v0[4 * j], v0[4 * j + 1], v0[4 * j + 2], v0[4 * j + 3]));
+                        __stcg(dst + (c + 1) * 256 + j * 32, make_uint4(v1[4 * j], v1[4 * j + 1], v1[4 * j + 2], v1[4 * j + 3]));
+                    }
+                }
+                release();
+                __threadfence();
+                __syncwarp();
+                if (lane == 0)
+                    *reinterpret_cast<volatile unsigned*>(p.sk_flags + (pair_id * 2 + rank) * 8 + (warp - kEpiWarp0)) = p.sk_epoch;
+                continue;
+            }
+            // A piece with the tile's first but not its last k-block: the pairs after this one hold the rest of the
+            // tile's K range, each as one partial tile in its slot, in k order.  They computed those pieces first of
+            // all, so the flags are long up; the wait is bounded all the same.
+            int n_part = 0;
+            if (MODE == 0 && wk.kind == 2) {
+                const int64_t rel = wk.tile - p.sk_first;
+                for (int64_t j = pair_id + 1; j < n_pairs; ++j) {
+                    const int64_t sj = j * p.sk_work / n_pairs;
+                    if (sj % p.nkb == 0 || sj / p.nkb != rel) break;
+                    ++n_part;
+                }
+                bool seen = true;
+                if (lane == 0) {
+                    for (int j = 1; j <= n_part && seen; ++j) {
+                        const volatile unsigned* f = p.sk_flags + ((pair_id + j) * 2 + rank) * 8 + (warp - kEpiWarp0);
+                        seen = false;
+                        for (uint32_t i = 0; i < ptx::kMbarPollLimit; ++i) {
+                            if (*f == p.sk_epoch) {
+                                seen = true;
+                                break;
+                            }
+                            if ((i & 1023u) == 1023u && abort_flag[0]) break;
+                        }
+                    }
+                    if (!seen) {
+                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x560u);
+                        abort_flag[0] = 1;
+                    }
+                }
+                seen = __shfl_sync(0xFFFFFFFFu, seen ? 1 : 0, 0) != 0;
+                __threadfence();
+                if (!seen) {       // give up: hand the accumulator back so that the other roles drain, store nothing
+                    release();
+                    ok = false;
+                    break;
+                }
+            }
+            // adds the partial sums of unit u (this lane's row, the unit's columns) to r0 / r1, in k order
+            auto add_partials = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32]) {
+                for (int j = 1; j <= n_part; ++j) {
+                    // unit u = 32-column blocks u * (cpc / 32) and, for a 2-byte C, the next one
+                    const float4* src = reinterpret_cast<const float4*>(p.sk_slots + (pair_id + j) * (TILE_M * PN) + sk_block * 1024) +
+                                        u * (cpc / 32) * 256 + lane;
+                    float4 t[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) t[i] = __ldcg(src + i * 32);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        r0[4 * i] = __float_as_uint(__uint_as_float(r0[4 * i]) + t[i].x);
+                        r0[4 * i + 1] = __float_as_uint(__uint_as_float(r0[4 * i + 1]) + t[i].y);
+                        r0[4 * i + 2] = __float_as_uint(__uint_as_float(r0[4 * i + 2]) + t[i].z);
+                        r0[4 * i + 3] = __float_as_uint(__uint_as_float(r0[4 * i + 3]) + t[i].w);
+                    }
+                    if (out_bf16) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) t[i] = __ldcg(src + 256 + i * 32);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            r1[4 * i] = __float_as_uint(__uint_as_float(r1[4 * i]) + t[i].x);
+                            r1[4 * i + 1] = __float_as_uint(__uint_as_float(r1[4 * i + 1]) + t[i].y);
+                            r1[4 * i + 2] = __float_as_uint(__uint_as_float(r1[4 * i + 2]) + t[i].z);
+                            r1[4 * i + 3] = __float_as_uint(__uint_as_float(r1[4 * i + 3]) + t[i].w);
+                        }
+                    }
+                }
             };
-
             if (nunits == 0) {
                 release();
                 continue;
             }
             uint32_t a0[32], a1[32], c0[32], c1[32];
-            if (out_bf16 && nunits == 4) {
+            auto pack_p = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32], uint32_t (&w)[32]) {
+                if (MODE == 0 && n_part > 0) add_partials(u, r0, r1);
+                pack(u, r0, r1, w);
+            };
+            if (out_bf16 && nunits == 4 && n_part == 0) {
                 // Full-width bf16 tile: the accumulator is handed back before anything is staged or stored.
                 // Rounding (F2F, 16 results per clock and SM) is what the drain costs: three units are read
                 // raw (192 registers), one is rounded to make room for the fourth, the accumulator is
@@ -566,7 +735,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 stage_store(3, w0);
                 continue;
             }
-            if (!out_bf16 && nunits == 8) {
+            if (!out_bf16 && nunits == 8 && n_part == 0) {
                 // Full-width fp32 tile (eight 32-column units, nothing to round): six units are read raw, two
                 // are staged and stored to make room for the last two, then the accumulator is released.
                 uint32_t d0[32], d1[32];
@@ -599,15 +768,22 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 stage_store(7, a1);
                 continue;
             }
+            // (a tile that adds partial sums takes this path whatever its width)
             issue(0, a0, a1);
             for (int u = 0; u < nunits; u += 2) {
                 ptx::tmem_ld_wait();
                 if (u + 1 < nunits) issue(u + 1, c0, c1); else release();
-                finish(u, a0, a1);
+                {
+                    uint32_t w[32];
+                    pack_p(u, a0, a1, w);
+                    stage_store(u, w);
+                }
                 if (u + 1 < nunits) {
                     ptx::tmem_ld_wait();
                     if (u + 2 < nunits) issue(u + 2, a0, a1); else release();
-                    finish(u + 1, c0, c1);
+                    uint32_t w[32];
+                    pack_p(u + 1, c0, c1, w);
+                    stage_store(u + 1, w);
                 }
             }
         }
@@ -887,6 +1063,69 @@ double pair_makespan(int64_t n_wide_tiles, int64_t n_narrow_tiles, double c_wide
     return worst;
 }
 
+// Whether and how the last, under-filled wave of pair tiles is streamed along K (see PairParams).
+struct StreamK {
+    bool on;
+    int rounds;
+    int64_t first, work;
+};
+// CTA pairs of this kernel that the device holds at once (asked of the runtime once per device): a streamed wave
+// has pairs waiting on one another's partial tiles, so every pair of the grid must be resident.
+int resident_pairs(const RunContext& ctx)
+{
+    static int cache[64] = {};
+    const bool cacheable = ctx.device >= 0 && ctx.device < 64;
+    if (cacheable && cache[ctx.device] != 0) return cache[ctx.device];
+    auto kern = r4_pair_kernel<false, 0>;
+    int n = 0;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(static_cast<unsigned>(ctx.sm_count / 2 * 2));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 0) {
+        cudaGetLastError();
+        n = 0;
+    }
+    if (cacheable) cache[ctx.device] = n > 0 ? n : -1;
+    return n > 0 ? n : -1;
+}
+
+StreamK plan_stream_k(int64_t tiles, int nkb, int64_t pairs, const RunContext& ctx, bool forced)
+{
+    StreamK sk = {false, 0, 0, 0};
+    if (!ctx.sk_flags || pairs < 2 || tiles <= 0) return sk;
+    if (resident_pairs(ctx) < pairs) return sk;
+    const int64_t rounds = tiles / pairs, rem = tiles % pairs;
+    if (rem == 0) return sk;
+    const int64_t work = rem * nkb;
+    const int64_t share = (work + pairs - 1) / pairs;             // k-blocks of the streamed wave per pair
+    // every piece at least 8 k-blocks deep on average, and no tile cut into more than 6 pieces
+    if (share < 8 || share * 6 < nkb || work / pairs < 1) return sk;
+    if (static_cast<size_t>(pairs) * TILE_M * PN * sizeof(float) > ctx.workspace_bytes) return sk;
+    if (rounds > 0x7FFFFFFF) return sk;
+    // Not chosen unless a plan asks for it.  Measured on B200 (single launches after an L2 flush): 4096^3 107 us
+    // streamed against 92 us in whole tiles, 3072 x 2048 x 8192 91 against 87, 2048 x 4096 x 4096 71 against 52 -
+    // although the schedule alone (partial tiles neither written nor read) would take 89 / 75 / 54 us.  The pair
+    // kernel's main loop already draws about 9 TB/s from the L2; the partial tiles' trip through it (1 MiB per
+    // pair) comes on top, and a power-capped part clocks lower with every SM busy.  The autotuner times the
+    // candidate and may pin it where it wins.
+    if (!forced) return sk;
+    sk.on = true;
+    sk.rounds = static_cast<int>(rounds);
+    sk.first = rounds * pairs;
+    sk.work = work;
+    return sk;
+}
+
 PairColumns plan_columns(const GemmArgs& g, const RunContext& ctx)
 {
     const int64_t tiles_m2 = (g.M + TILE_M - 1) / TILE_M;
@@ -923,6 +1162,13 @@ PairColumns plan_columns(const GemmArgs& g, const RunContext& ctx)
     }
     return best;
 }
+}
+
+bool r4_pair_stream_k_possible(const GemmArgs& g, const RunContext& ctx)
+{
+    if (!r4_pair_possible(g, ctx) || g.M <= 0 || g.N <= 0 || g.K <= 0) return false;
+    const int64_t tiles = static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * ((g.N + PN - 1) / PN);
+    return plan_stream_k(tiles, (g.K + BK - 1) / BK, ctx.sm_count / 2, ctx, true).on;
 }
 
 cudaError_t launch_r4_tcgen05_pair(const GemmArgs& g, RunContext& ctx, cudaStream_t stream, int* kernel_id)
@@ -1018,10 +1264,28 @@ cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const
                            table[d].ldc * celt, g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return cudaErrorInvalidValue;
 
-    p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + 32 + ctx.kid_flags;
-    *kernel_id = p.kid;
     const int64_t max_pairs = ctx.sm_count / 2;
-    const unsigned grid = 2u * static_cast<unsigned>(p.total_tiles < max_pairs ? p.total_tiles : max_pairs);
+    unsigned grid = 2u * static_cast<unsigned>(p.total_tiles < max_pairs ? p.total_tiles : max_pairs);
+    // Stream the under-filled last wave along K?  (one problem, one destination, uniform 256-column tiles)
+    if (n_dst == 0 && cols.n_narrow == 0 && cols.tile_n == PN && ctx.plan.split_via != 1) {
+        const StreamK sk = plan_stream_k(p.total_tiles, p.nkb, max_pairs, ctx, ctx.plan.split_via == 3);
+        if (sk.on) {
+            p.sk = 1;
+            p.sk_rounds = sk.rounds;
+            p.sk_first = sk.first;
+            p.sk_work = sk.work;
+            p.sk_slots = static_cast<float*>(ctx.workspace);
+            p.sk_flags = ctx.sk_flags;
+            p.sk_epoch = ++ctx.sk_epoch;
+            grid = 2u * static_cast<unsigned>(max_pairs);
+        } else if (ctx.plan.split_via == 3) {
+            return cudaErrorInvalidValue;
+        }
+    } else if (ctx.plan.split_via == 3) {
+        return cudaErrorInvalidValue;
+    }
+    p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + 32 + (p.sk ? 128 : 0) + ctx.kid_flags;
+    *kernel_id = p.kid;
     if (n_dst > 0) {
         // the table travels on the launch's stream, ahead of the kernel (staged before the call returns)
         const cudaError_t e = cudaMemcpyAsync(ctx.workspace, table, sizeof(DstEntry) * n_dst, cudaMemcpyHostToDevice, stream);

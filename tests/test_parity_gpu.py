@@ -269,6 +269,45 @@ def test_tcgen05_cta_pair_ragged(handles, col):
         run_and_check(handles, case, 4, C_ref, S, rows, pin=PAIR)
 
 
+STREAMED = (2, 1, 3)        # launch plan: the CTA-pair kernel, last wave streamed along K
+@pytest.mark.parametrize("col", [False, True], ids=["Brow", "Bcol"])
+def test_tcgen05_cta_pair_streamed_last_wave(handles, col):
+    """The under-filled last wave of pair tiles cut along K: pieces without a tile's first k-block leave their fp32
+    partial tile in the workspace, the piece with it adds them in k order.  Bit-exact on integers, identical to the
+    whole-tile schedule, for fewer tiles than pairs, for one and for several full rounds before the streamed wave."""
+    for idx, (M, N, K) in enumerate([(2048, 4096, 2048),     # 64 tiles on 74 pairs: everything is streamed
+                                     (4096, 4096, 1024),     # 128 tiles: one full round, then 54 streamed tiles
+                                     (5000, 5200, 1104),     # 10 x 21 = 210 tiles: two rounds + 62 tiles, ragged M, N, K
+                                     (1536, 2048, 4096)]):   # 24 tiles: every tile cut into three or four pieces
+        for bf in (False, True):
+            case = gen.make_case(M, N, K, seed=320 + idx, dist_a="integer", dist_b="integer", b_col_major=col,
+                                 c_bf16=bf, name=f"streamed{M}x{N}x{K}-int")
+            rows = P.sample_rows(M)
+            C_ref, S = P.oracle_rows(case, rows)
+            vals, bits = run_and_check(handles, case, 4, C_ref, S, rows, exact=True, pin=STREAMED)
+            flags = handles[(col, bf)].last_kernel_id() - 400
+            assert (flags & 32) and (flags & 128), (M, N, K, flags)
+            _, whole = run_and_check(handles, case, 4, C_ref, S, rows, exact=True, pin=(2, 1, 1))
+            assert not ((handles[(col, bf)].last_kernel_id() - 400) & 128)
+            assert np.array_equal(bits, whole), "streamed and whole-tile schedules differ"
+            if not bf:
+                assert P.integer_checksums_match(case, vals)
+        case = gen.make_case(M, N, K, seed=320 + idx, dist_a="normal", dist_b="uniform", b_col_major=col,
+                             name=f"streamed{M}x{N}x{K}")
+        rows = P.sample_rows(M)
+        C_ref, S = P.oracle_rows(case, rows)
+        _, b1 = run_and_check(handles, case, 4, C_ref, S, rows, pin=STREAMED)
+        _, b2 = run_and_check(handles, case, 4, C_ref, S, rows, pin=STREAMED)
+        assert np.array_equal(b1, b2), "two streamed runs differ"
+    # a shape whose streamed pieces would be too short: the plan is refused
+    case = gen.make_case(4200, 4352, 136, seed=330, dist_a="integer", dist_b="integer", b_col_major=col)
+    dev = P.DeviceCase(case)
+    g = handles[(col, False)]
+    from paper_2605_28213_b200 import binding as kb
+    assert kb.klineage_gemm_set_plan_raw(g._h, case.M, case.N, case.K, dev.a.ptr, case.lda, dev.b.ptr, case.ldb, dev.c.ptr,
+                                         case.ldc, kb.klineage_gemm_plan_t(*STREAMED)) == kb.KLINEAGE_ERR_INVALID_ARG
+
+
 def test_dispatch_between_the_two_kernels(handles):
     """Long K and enough 512 x 256 tiles: the pair kernel; short K or few tiles: the single-CTA kernel."""
     for (M, N, K), want_pair in (((2048, 4096, 4096), True), ((3072, 2048, 8192), True), ((2816, 2816, 2816), True),
@@ -394,7 +433,7 @@ def test_each_variant_reports_its_own_kernel(handles, kb):
             code, dev_id = g.device_status()
             assert code == 0 and dev_id == g.last_kernel_id()
             if v == 4:
-                assert 400 <= dev_id < 528
+                assert 400 <= dev_id < 656
                 # unaligned operands are repacked into the workspace (flag 64), never gathered, when they fit
                 assert ((dev_id - 400) & 1) == 0 and bool((dev_id - 400) & 64) == (case.name == "c2")
             else:
