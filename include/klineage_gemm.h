@@ -432,12 +432,12 @@ klineage_status_t klineage_gemm_run_host(klineage_gemm_t h, int64_t M, int64_t N
  *              in k order - a fixed order, so results repeat bit for bit), 1 never does
  *   group_m    tile-rows per raster group (L2 reuse pattern)
  *   half_tail  1 cut the last wave into 128-column half tiles, 2 never
- *   tile_n     columns per output tile (needs `kernel`): single-CTA kernel 256 or 128; CTA-pair kernel a
+ *   tile_n     columns per output tile (needs `kernel`): single-CTA kernel 256, 128 or 64; CTA-pair kernel a
  *              multiple of 64 up to 256
  *   tail_n     CTA-pair kernel only: tile_n = every tile of that width; a smaller multiple of 64 = tile rows
  *              start with tile_n-wide tiles and end with tiles of this width, dealt to the CTA pairs back and
  *              forth so that wide and narrow turns balance a last, under-filled wave
- *   stages     single-CTA kernel only: depth of the operand ring - 4, or 6 with 128-column tiles (32 KiB stages)
+ *   stages     single-CTA kernel only: depth of the operand ring - 4, or 6 with 128- or 64-column tiles
  * Every plan computes the same C up to fp32 summation order (plans that differ
  * only in kernel / group_m / half_tail / tile shape / stages are bit-identical; K
  * splits change the order of the partial sums and stay within the parity bound).

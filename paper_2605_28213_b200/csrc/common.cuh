@@ -162,7 +162,7 @@ struct R4Plan {
     int group_m = 0;     // 0 auto, else tile-rows per raster group
     int half_tail = 0;   // 0 auto, 1 cut the last wave into half tiles, 2 never
     int tile_n = 0;      // 0 auto, else columns per output tile (pair kernel: a multiple of 64, at most 256;
-                         // single-CTA kernel: 128 or 256)
+                         // single-CTA kernel: 64, 128 or 256)
     int tail_n = 0;      // pair kernel: 0 auto, tile_n = uniform tiles, else the width of the narrow tiles that
                          // follow the wide ones in every tile row and balance the last wave
     int stages = 0;      // 0 auto, else depth of the operand ring

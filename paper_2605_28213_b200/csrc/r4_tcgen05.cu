@@ -113,7 +113,7 @@ struct R4Params {
     int test_stop_after;
     uint32_t test_poll_limit;
     // Tile width and ring depth (MODE 0, TMA-fed, regular orientation; every other form runs 256 columns and 4
-    // stages): 256 columns with four 48 KiB stages, or 128 columns with four or six 32 KiB stages.
+    // stages): 256 columns with four 48 KiB stages, or 128 / 64 columns with four or six 32 / 24 KiB stages.
     int tile_n;
     int n_stages;
     uint32_t stage_bytes;
@@ -1270,7 +1270,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         const bool epi_warp = warp >= 2 && warp < 6;
         const bool out_bf16 = g.c_bf16 != 0;
         const int sub_log2 = out_bf16 ? 1 : 0;                          // 32-column blocks per store unit
-        const int per_log2 = (out_bf16 ? 4 : 5) - (TN == BN ? 0 : 1) - p.splits_log2;   // pairs per CTA
+        const int per_log2 = (out_bf16 ? 4 : 5) - (TN == BN ? 0 : TN == BN / 2 ? 1 : 2) - p.splits_log2;   // pairs per CTA
         const int q = warp & 3;                                         // TMEM lane quarter of this warp
         const uint32_t tlane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
         float* recv = reinterpret_cast<float*>(smem);
@@ -1802,7 +1802,7 @@ bool plan_launch(const GemmArgs& g, const RunContext& ctx, bool generic, bool mu
     if (pl.kernel != 2 && (pl.tile_n != 0 || pl.stages != 0)) {        // pinned (the pair kernel reads the fields its own way)
         const int tn = pl.tile_n != 0 ? pl.tile_n : BN;
         const int st = pl.stages != 0 ? pl.stages : STAGES;
-        const bool ok = (tn == BN && st == STAGES) || (tunable && tn == BN / 2 && (st == 4 || st == 6));
+        const bool ok = (tn == BN && st == STAGES) || (tunable && (tn == BN / 2 || tn == BN / 4) && (st == 4 || st == 6));
         return ok && try_shape(tn, st, out);
     }
     LaunchPlan wide;
@@ -1832,6 +1832,13 @@ bool plan_launch(const GemmArgs& g, const RunContext& ctx, bool generic, bool mu
     else
         take_narrow = narrow.split.splits > 1 || tiles256 * 2 <= ctx.sm_count;
     if (take_narrow && narrow.split.cluster) narrow.stages = 6;
+    if (take_narrow && narrow.split.splits == 1 && g.N > BN / 4) {
+        // still at most half a wave of 128-column tiles: 64 columns (measured 0.4 - 0.5 us off a 5 - 7 us launch at
+        // 256^3, 512^3 and 300 x 520 x 200: an MMA takes as long whatever its width, the epilogue of a tile shrinks)
+        const int64_t tiles128 = tiles_m * ((g.N + BN / 2 - 1) / (BN / 2));
+        LaunchPlan tiny;
+        if (tiles128 * 2 <= ctx.sm_count && try_shape(BN / 4, STAGES, &tiny) && tiny.split.splits == 1) narrow = tiny;
+    }
     *out = take_narrow ? narrow : wide;
     return true;
 }
@@ -2382,8 +2389,8 @@ bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& pl)
     if (pl.split_via == 3 && (pl.kernel != 2 || pl.splits > 1)) return false;     // streaming the last wave is the pair kernel's
     if (pl.kernel == 2 && pl.stages != 0) return false;
     if (pl.kernel != 2 && (pl.tile_n != 0 || pl.stages != 0)) {
-        // single-CTA kernel: 256 columns x 4 stages, or 128 columns x 4 or 6 stages (plain TMA-fed GEMM, M > 64)
-        if (pl.tile_n != 0 && pl.tile_n != BN && pl.tile_n != BN / 2) return false;
+        // single-CTA kernel: 256 columns x 4 stages, or 128 / 64 columns x 4 or 6 stages (plain TMA-fed GEMM, M > 64)
+        if (pl.tile_n != 0 && pl.tile_n != BN && pl.tile_n != BN / 2 && pl.tile_n != BN / 4) return false;
         if (pl.stages != 0 && pl.stages != 4 && pl.stages != 6) return false;
     }
     // a tile shape is a property of one of the two kernels: name the kernel with it
@@ -2465,6 +2472,14 @@ int r4_enumerate_plans(const GemmArgs& g, const RunContext& ctx, R4Plan* out, in
             pl.splits = 1;
             pl.tile_n = BN / 2;
             pl.stages = st;
+            push(pl);
+        }
+        if (tiles * 2 <= ctx.sm_count) {     // few tiles: 64 columns
+            R4Plan pl;
+            pl.kernel = 1;
+            pl.splits = 1;
+            pl.tile_n = BN / 4;
+            pl.stages = 4;
             push(pl);
         }
         for (int gm : {4, 8, 16, 32}) {
