@@ -463,6 +463,37 @@ def run_partitioned(args):
     return 0 if ok_all else 1
 
 
+def run_shape(args):
+    """--shape MxNxK: one ad-hoc product (row-major bf16 operands N(0, 1/sqrt(K)), bf16 C) through the chosen rung;
+    a profiling aid - the profiler summaries of shapes outside the five configurations name this command."""
+    import numpy as np
+    import torch
+    from paper_2605_28213_b200 import binding as kb
+    from paper_2605_28213_b200 import inputs as gen
+    M, N, K = (int(x) for x in args.shape.lower().split("x"))
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    case = gen.make_case(M, N, K, seed=1, dist_a="normal", dist_b="normal", sigma_b=K ** -0.5, c_bf16=True,
+                         name=f"shape{M}x{N}x{K}")
+    prob = DeviceProblem(case, kb, torch, device)
+    ok = smoke_check(prob, args.variant)
+    for _ in range(max(3, args.warmup)):
+        prob.run(args.variant)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        prob.run(args.variant)
+    e1.record()
+    e1.synchronize()
+    us = e0.elapsed_time(e1) / args.steps * 1e3
+    code, kid = prob.gemm.device_status()
+    print(json.dumps({"shape": [M, N, K], "variant": VARIANT_NAMES[args.variant], "us_per_launch_back_to_back": us,
+                      "tflops": case.flops / us / 1e6, "kernel_id": kid, "device_status": code, "parity_checked": ok}),
+          flush=True)
+    return 0 if ok and code == 0 else 1
+
+
 def lineage_table(prob_c4, kb, gen, torch, device, peaks):
     """Per-rung throughput at 8192^3 and 4096^3, and the HBM-bound skinny shape for every rung."""
     out = {}
@@ -851,6 +882,7 @@ def main():
     ap.add_argument("--partition", default="replicas", choices=["replicas", "n"],
                     help="N > 1: 'replicas' = independent GEMMs (default, weak scaling); 'n' = ONE GEMM partitioned by "
                          "columns over the ranks with the all-gather fused into the epilogue (strong scaling)")
+    ap.add_argument("--shape", default=None, help="MxNxK: time one ad-hoc product (profiling aid) and print a short JSON line")
     ap.add_argument("--family", action="store_true",
                     help="time only the BMM / GroupedGEMM rows (for profiling) and print them as one JSON line")
     args = ap.parse_args()
@@ -865,6 +897,8 @@ def main():
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
         print(json.dumps({"gemm_family": family_table(kb, gen, torch, device, load_peaks()[0], flush)}), flush=True)
         return 0
+    if args.shape:
+        return run_shape(args)
     if args.partition == "n":
         return run_partitioned(args)
     return run_gpu(args)
