@@ -197,11 +197,15 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_f
 // MODE 0: one problem (tensor maps 2-D).  MODE 1: batched (3-D tensor maps, z = batch).
 // MODE 2: grouped (per-group tensor maps and sizes from a table in device memory).
 // MODE 3: one problem whose C goes to several destinations (table of C maps / pointers).
-template <bool BCOL, int MODE>
+// MODE 5: MODE 0 with its last wave streamed along K (a separate instantiation, so that the plain kernel does not carry
+// the work-list arithmetic in its 24-register producer and MMA threads).
+template <bool BCOL, int MODE_>
 __global__ void __launch_bounds__(kThreads, 1)
 r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c, PairParams p)
 {
+    constexpr bool SK = MODE_ == 5;
+    constexpr int MODE = SK ? 0 : MODE_;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* epi_smem = smem + STAGES * kStageBytes;
@@ -332,14 +336,14 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
     };
     auto work_init = [&]() {
         WorkState st = {0u, 0, 0, false};
-        if (MODE == 0 && p.sk) {
+        if (SK) {
             st.pos = pair_id * p.sk_work / n_pairs;
             st.end = (pair_id + 1) * p.sk_work / n_pairs;
         }
         return st;
     };
     auto next_work = [&](WorkState& st, Work& w) -> bool {
-        if (!(MODE == 0 && p.sk)) {
+        if (!SK) {
             const int64_t t = tile_at(st.i++);
             if (t < 0) return false;
             w.tile = t;
@@ -611,7 +615,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     __syncwarp();
                 }
             };
-            if (MODE == 0 && wk.kind == 1) {
+            if (SK && wk.kind == 1) {
                 // A piece without the tile's first k-block: this warp's 32 rows of the raw fp32 partial tile go to the
                 // pair's workspace slot, as 4 KiB blocks of 32 rows x 32 columns laid out [column / 4][row][column % 4]
                 // (a warp's store instruction writes 512 contiguous bytes); then the accumulator is handed back and
@@ -640,7 +644,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             // tile's K range, each as one partial tile in its slot, in k order.  They computed those pieces first of
             // all, so the flags are long up; the wait is bounded all the same.
             int n_part = 0;
-            if (MODE == 0 && wk.kind == 2) {
+            if (SK && wk.kind == 2) {
                 const int64_t rel = wk.tile - p.sk_first;
                 for (int64_t j = pair_id + 1; j < n_pairs; ++j) {
                     const int64_t sj = j * p.sk_work / n_pairs;
@@ -708,7 +712,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             }
             uint32_t a0[32], a1[32], c0[32], c1[32];
             auto pack_p = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32], uint32_t (&w)[32]) {
-                if (MODE == 0 && n_part > 0) add_partials(u, r0, r1);
+                if (SK && n_part > 0) add_partials(u, r0, r1);
                 pack(u, r0, r1, w);
             };
             if (out_bf16 && nunits == 4 && n_part == 0) {
@@ -1209,7 +1213,9 @@ cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const
     const uint32_t b_box_rows = static_cast<uint32_t>(widest / 2);
     p.b_boxes = (widest / 2 + 63) / 64;
     p.stage_tx = 2u * (kABytes + (g.b_col ? b_box_rows * 128u : static_cast<uint32_t>(p.b_boxes) * 8192u));
-    p.group_m = ctx.plan.group_m > 0 ? ctx.plan.group_m : 4;   // default: 4 x 512 rows per raster group
+    // default raster group: 4 x 512 rows; 8 when the problem has at least 16 tile rows (measured at 8192^3 in rested
+    // 10-launch bursts: 672-674 us against 676-678 us for 4 and 684-686 us for 1, 2, 3 or 16)
+    p.group_m = ctx.plan.group_m > 0 ? ctx.plan.group_m : (p.tiles_m2 >= 16 ? 8 : 4);
     const int celt = g.c_bf16 ? 2 : 4;
     // (row length a multiple of 16 bytes too: a store box ending inside a 16-byte unit at the tensor's
     // right edge writes the whole unit)
@@ -1295,6 +1301,9 @@ cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const
         return g.b_col ? launch<true, 3>(g, ma, mb, mc, p, grid, ctx.device, stream)
                        : launch<false, 3>(g, ma, mb, mc, p, grid, ctx.device, stream);
     }
+    if (p.sk)
+        return g.b_col ? launch<true, 5>(g, ma, mb, mc, p, grid, ctx.device, stream)
+                       : launch<false, 5>(g, ma, mb, mc, p, grid, ctx.device, stream);
     return g.b_col ? launch<true, 0>(g, ma, mb, mc, p, grid, ctx.device, stream)
                    : launch<false, 0>(g, ma, mb, mc, p, grid, ctx.device, stream);
 }
