@@ -287,4 +287,19 @@ cudaError_t launch_r4_pair_multi_dst(const GemmArgs& g, void* const* C, const in
 bool r4_pair_grouped_possible(const GemmArgs* groups, int n, const RunContext& ctx);
 cudaError_t launch_r4_pair_grouped(const GemmArgs* groups, int n, RunContext& ctx, cudaStream_t stream, int* kernel_id);
 
+
+// Timeline stamps for tuning (compiled in only with -DKLIN_TRACE; the shipped library carries none of it).
+// A translation unit that stamps defines KLIN_TRACE_BUF as its own static __device__ array of
+// kTraceSlots x (CTAs) 64-bit words; slot s of CTA b receives the SM's cycle counter.
+#ifdef KLIN_TRACE
+constexpr int kTraceSlots = 64, kTraceCtas = 160;
+#define KLIN_T(slot)                                                                                  \
+    do {                                                                                              \
+        if ((slot) >= 0 && (slot) < klin::kTraceSlots && blockIdx.x < klin::kTraceCtas)               \
+            KLIN_TRACE_BUF[blockIdx.x * klin::kTraceSlots + (slot)] = static_cast<unsigned long long>(clock64()); \
+    } while (0)
+#else
+#define KLIN_T(slot) ((void)0)
+#endif
+
 }  // namespace klin

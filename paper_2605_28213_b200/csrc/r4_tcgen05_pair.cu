@@ -38,6 +38,19 @@
 #include <cstring>
 #include <new>
 
+#ifdef KLIN_TRACE
+static __device__ unsigned long long klin_trace_pair[klin::kTraceSlots * klin::kTraceCtas];
+#define KLIN_TRACE_BUF klin_trace_pair
+extern "C" int klin_trace_dump_pair(unsigned long long* host)
+{
+    cudaDeviceSynchronize();
+    const cudaError_t e = cudaMemcpyFromSymbol(host, klin_trace_pair, sizeof klin_trace_pair);
+    void* dev = nullptr;
+    if (cudaGetSymbolAddress(&dev, klin_trace_pair) == cudaSuccess) cudaMemset(dev, 0, sizeof klin_trace_pair);
+    return static_cast<int>(e);
+}
+#endif
+
 namespace klin {
 namespace {
 
@@ -155,21 +168,21 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t cluster_bar_addr)
 }
 // 2-D tiled load whose completion is counted on a barrier that may live in the
 // partner CTA (shared::cluster address); the data lands in this CTA.
-__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const void* tmap, int x, int y, uint32_t cluster_bar_addr)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t smem_dst, const void* tmap, int x, int y, uint32_t cluster_bar_addr)
 {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, "
         "%3}], [%4];"
-        ::"r"(ptx::smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(cluster_bar_addr)
+        ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(cluster_bar_addr)
         : "memory");
 }
-__device__ __forceinline__ void tma_load_3d_pair(void* smem_dst, const void* tmap, int x, int y, int z,
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t smem_dst, const void* tmap, int x, int y, int z,
                                                  uint32_t cluster_bar_addr)
 {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, "
         "%3, %4}], [%5];"
-        ::"r"(ptx::smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z),
+        ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z),
         "r"(cluster_bar_addr)
         : "memory");
 }
@@ -223,6 +236,14 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
     const int64_t n_pairs = gridDim.x >> 1;
 
     if (warp == 0 && lane == 0) {
+        KLIN_T(0);
+#ifdef KLIN_TRACE
+        {
+            unsigned long long ns;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+            if (blockIdx.x < kTraceCtas) KLIN_TRACE_BUF[blockIdx.x * kTraceSlots + 5] = ns;
+        }
+#endif
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(&full[s], 1);
             ptx::mbar_init(&empty[s], 1);
@@ -234,6 +255,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         abort_flag[0] = 0;
         abort_flag[1] = 0;
         ptx::fence_barrier_init();
+        KLIN_T(24);
         if (MODE != 2) {
             ptx::prefetch_tensormap(&map_a);
             ptx::prefetch_tensormap(&map_b);
@@ -250,12 +272,15 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         tmem_relinquish_pair();
     }
     ptx::tc_fence_before_sync();
+    if (threadIdx.x == 32) KLIN_T(25);      // TMEM allocated
     __syncthreads();
+    if (threadIdx.x == 0) KLIN_T(26);
     // Both CTAs' barriers exist before anyone signals across the pair.
     ptx::cluster_arrive_release();
     ptx::cluster_wait_acquire();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) KLIN_T(1);
 
     int group_hint = 0;     // MODE 2: a thread's tiles come in increasing order, so its search resumes here
     auto tile_info = [&](int64_t t) {
@@ -383,7 +408,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         return false;
     };
     // One operand box of a stage; completion is counted on the even CTA's barrier.
-    auto load_box = [&](void* dst, const CUtensorMap* map, int c0, int c1, int z, uint32_t bar) {
+    auto load_box = [&](uint32_t dst, const CUtensorMap* map, int c0, int c1, int z, uint32_t bar) {
         if (MODE == 1)
             tma_load_3d_pair(dst, map, c0, c1, z, bar);
         else
@@ -394,38 +419,59 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
     // One instruction for the whole first warp group (the register release is warp-group wide), ahead of
     // the producer and MMA code, which run within the reduced budget.
     setmaxnreg_dec<kRegsLean>();
+    if (threadIdx.x == 0) KLIN_T(27);
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
+        // (One thread issues all of a stage's loads.  Measured: three threads - one per operand block, each
+        // waiting for "stage free" on its own - made the main loop 4 % SLOWER, 1120 against 1077 clocks per
+        // k-block: the loop is not waiting for the producer.  A k-block moves 48 KiB into shared memory and its
+        // eight MMAs read 64 KiB from it, 112 of the 128 bytes per clock a CTA's shared memory delivers.)
         if (lane == 0) {
-            uint32_t it = 0;
+            // The ring position (stage s, parity ph of its "empty" barrier) is carried, barriers and stages are
+            // addressed by their shared-window addresses, and everything a stage's loads need is in registers
+            // before the wait: what follows the wait is the expect-tx arrive and the loads themselves.  (The time
+            // from "stage free" to "loads issued" is part of every stage's round trip: four stages of 1024 MMA
+            // clocks hide about 4 k clocks of it, and a load takes about 3 k to land.)
+            uint32_t it = 0, s = 0, ph = 1;
             bool ok = true;
+            const uint32_t smem0 = ptx::smem_u32(smem), empty0 = ptx::smem_u32(empty), full0 = ptx::smem_u32(full);
+            const uint32_t full_even0 = ptx::map_to_cta(full0, 0);   // the even CTA's barriers (consecutive words)
+            const uint32_t stage_tx = p.stage_tx;
+            const bool two_boxes = !BCOL && p.b_boxes > 1;
             WorkState ws = work_init();
             Work wk;
             while (ok && next_work(ws, wk)) {
                 const TileInfo x = tile_info(wk.tile);
-                const int m0 = x.m0;
+                const int m0 = x.m0, z = x.z;
+                const CUtensorMap *ma = x.ma, *mb = x.mb;
                 const int nb = x.n0 + static_cast<int>(rank) * (x.width >> 1);    // this CTA's half of B
                 const int kb_end = wk.kb1 < 0 ? x.nkb : wk.kb1;
+                if (it == 0) KLIN_T(28);
                 for (int kb = wk.kb0; kb < kb_end; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    if (!ptx::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag)) {
+                    const uint32_t sa = smem0 + s * kStageBytes, sb = sa + kABytes;
+                    const uint32_t bar = full_even0 + 8 * s;
+                    const int kx = kb * BK;
+                    if (!ptx::mbar_wait_addr(empty0 + 8 * s, ph, abort_flag)) {
                         report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x500u | s);
                         abort_flag[0] = 1;
                         ok = false;
                         break;
                     }
-                    uint8_t* sa = smem + s * kStageBytes;
-                    uint8_t* sb = sa + kABytes;
                     // The even CTA's barrier counts the bytes of both CTAs' loads of this stage.
-                    if (rank == 0) ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
-                    const uint32_t bar = ptx::map_to_cta(ptx::smem_u32(&full[s]), 0);
-                    load_box(sa, x.ma, kb * BK, m0, x.z, bar);
-                    load_box(sa + kABlockBytes, x.ma, kb * BK, m0 + 2 * PM, x.z, bar);
+                    if (rank == 0) ptx::mbar_arrive_expect_tx_addr(full0 + 8 * s, stage_tx);
+                    load_box(sa, ma, kx, m0, z, bar);
+                    load_box(sa + kABlockBytes, ma, kx, m0 + 2 * PM, z, bar);
                     if (BCOL) {
-                        load_box(sb, x.mb, kb * BK, nb, x.z, bar);
+                        load_box(sb, mb, kx, nb, z, bar);
                     } else {
-                        load_box(sb, x.mb, nb, kb * BK, x.z, bar);
-                        if (p.b_boxes > 1) load_box(sb + 64 * BK * 2, x.mb, nb + 64, kb * BK, x.z, bar);
+                        load_box(sb, mb, nb, kx, z, bar);
+                        if (two_boxes) load_box(sb + 64 * BK * 2, mb, nb + 64, kx, z, bar);
+                    }
+                    if (it == 0) KLIN_T(2);
+                    if (it == STAGES - 1) KLIN_T(3);
+                    if (++s == STAGES) {
+                        s = 0;
+                        ph ^= 1u;
                     }
                 }
             }
@@ -440,12 +486,24 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
             // -------------------------------------------------------- MMA issuer (even CTA)
-            uint32_t it = 0, tcount = 0;
+            // Ring position carried, barriers by shared-window address, a stage's descriptors = the first stage's
+            // plus s * (stage bytes >> 4) in the 14-bit start-address field (the ring ends below 256 KiB).  The next
+            // tile's coordinates are worked out BEFORE the wait for the drained accumulators, not after it.
+            uint32_t tcount = 0, s = 0, ph = 0;
             bool ok = true;
+            const uint32_t full0 = ptx::smem_u32(full), empty0 = ptx::smem_u32(empty);
+            const uint32_t empty_odd0 = ptx::map_to_cta(empty0, 1);
+            const uint32_t accf = ptx::smem_u32(&acc_full[0]), accf_odd = ptx::map_to_cta(accf, 1);
+            const uint64_t a_desc0 = make_desc(ptx::smem_u32(smem), 1, (1024u >> 4) | (1u << 14) | (2u << 29));
+            const uint64_t b_desc0 = make_desc(ptx::smem_u32(smem) + kABytes, p.b_desc_lbo, p.b_desc_hi);
+            const uint32_t kstep = p.b_kstep;
             WorkState ws = work_init();
             Work wk;
             for (; ok && next_work(ws, wk); ++tcount) {
-                const int64_t t = wk.tile;
+                const TileInfo x = tile_info(wk.tile);
+                const int kb_first = wk.kb0, kb_end = wk.kb1 < 0 ? x.nkb : wk.kb1;
+                // the MMA's N is the tile's width
+                const uint32_t idesc = (p.idesc & ~(0x3Fu << 17)) | (static_cast<uint32_t>(x.width >> 3) << 17);
                 // Both accumulators are rewritten: wait until both CTAs' epilogues drained the last tile.
                 if (!ptx::mbar_wait(&acc_empty[0], (tcount & 1) ^ 1, abort_flag)) {
                     report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x520u);
@@ -453,39 +511,39 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     break;
                 }
                 ptx::tc_fence_after_sync();
-                const TileInfo x = tile_info(t);
-                const int kb_first = wk.kb0, kb_end = wk.kb1 < 0 ? x.nkb : wk.kb1;
-                // the MMA's N is the tile's width
-                const uint32_t idesc = (p.idesc & ~(0x3Fu << 17)) | (static_cast<uint32_t>(x.width >> 3) << 17);
-                for (int kb = kb_first; kb < kb_end; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    const uint32_t par = (it / STAGES) & 1;
-                    if (!ptx::mbar_wait(&full[s], par, abort_flag)) {
+                KLIN_T(tcount < 4 ? 8 + 4 * static_cast<int>(tcount) : -1);
+                for (int kb = kb_first; kb < kb_end; ++kb) {
+                    if (!ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag)) {
                         report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x530u | s);
                         abort_flag[0] = 1;
                         ok = false;
                         break;
                     }
                     ptx::tc_fence_after_sync();
-                    const uint32_t sa = ptx::smem_u32(smem + s * kStageBytes);
-                    const uint32_t sb = sa + kABytes;
-                    const uint64_t a_desc = make_desc(sa, 1, (1024u >> 4) | (1u << 14) | (2u << 29));
-                    const uint64_t b_desc = make_desc(sb, p.b_desc_lbo, p.b_desc_hi);
+                    if (kb == kb_first) KLIN_T(tcount < 4 ? 9 + 4 * static_cast<int>(tcount) : -1);
+                    if (kb == kb_end - 1) KLIN_T(tcount < 4 ? 10 + 4 * static_cast<int>(tcount) : -1);
+                    const uint64_t a_desc = a_desc0 + s * static_cast<uint32_t>(kStageBytes >> 4);
+                    const uint64_t b_desc = b_desc0 + s * static_cast<uint32_t>(kStageBytes >> 4);
 #pragma unroll
                     for (int k4 = 0; k4 < BK / 16; ++k4) {
                         const uint32_t acc = (kb > kb_first || k4 > 0) ? 1u : 0u;
                         // alternate the two row blocks: consecutive MMAs never share an accumulator
                         umma_f16_pair(tmem_base, a_desc + static_cast<uint64_t>(k4 * 2),
-                                      b_desc + static_cast<uint64_t>(k4 * p.b_kstep), idesc, acc);
+                                      b_desc + static_cast<uint64_t>(k4 * kstep), idesc, acc);
                         umma_f16_pair(tmem_base + PN, a_desc + static_cast<uint64_t>((kABlockBytes >> 4) + k4 * 2),
-                                      b_desc + static_cast<uint64_t>(k4 * p.b_kstep), idesc, acc);
+                                      b_desc + static_cast<uint64_t>(k4 * kstep), idesc, acc);
                     }
-                    umma_commit_pair(ptx::smem_u32(&empty[s]));
-                    umma_commit_pair(ptx::map_to_cta(ptx::smem_u32(&empty[s]), 1));
+                    umma_commit_pair(empty0 + 8 * s);
+                    umma_commit_pair(empty_odd0 + 8 * s);
+                    if (++s == STAGES) {
+                        s = 0;
+                        ph ^= 1u;
+                    }
                 }
                 if (ok) {
-                    umma_commit_pair(ptx::smem_u32(&acc_full[0]));
-                    umma_commit_pair(ptx::map_to_cta(ptx::smem_u32(&acc_full[0]), 1));
+                    umma_commit_pair(accf);
+                    umma_commit_pair(accf_odd);
+                    KLIN_T(tcount < 4 ? 11 + 4 * static_cast<int>(tcount) : -1);
                 }
             }
         }
@@ -511,6 +569,50 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             const int m0 = x.m0, n0 = x.n0;
             float* dst_f = reinterpret_cast<float*>(x.C);
             uint16_t* dst_h = reinterpret_cast<uint16_t*>(x.C);
+            const int row0 = m0 + mb * 2 * PM + q * 32;
+            const int rows = min(32, x.M - row0);
+            const int nunits = (row0 < x.M) ? (min(x.width, x.N - n0) + cpc - 1) / cpc : 0;
+            const uint32_t tbase = tmem_base + mb * PN + (static_cast<uint32_t>(q * 32) << 16);
+            // first 4 KiB block of this warp's rows inside a partial-tile slot: (CTA, row block, lane quarter) x 8 column blocks
+            const int64_t sk_block = ((static_cast<int64_t>(rank) * 2 + mb) * 4 + q) * (PN / 32);
+
+            // A piece with the tile's first but not its last k-block: the pairs after this one hold the rest of the
+            // tile's K range, each as one partial tile in its slot, in k order.  They computed those pieces first of
+            // all, so the flags are up long before this piece's own MMAs end: the (bounded) wait for them happens
+            // here, ahead of the wait for the accumulator.
+            int n_part = 0;
+            if (SK && wk.kind == 2) {
+                const int64_t rel = wk.tile - p.sk_first;
+                for (int64_t j = pair_id + 1; j < n_pairs; ++j) {
+                    const int64_t sj = j * p.sk_work / n_pairs;
+                    if (sj % p.nkb == 0 || sj / p.nkb != rel) break;
+                    ++n_part;
+                }
+                bool seen = true;
+                if (lane == 0) {
+                    for (int j = 1; j <= n_part && seen; ++j) {
+                        const volatile unsigned* f = p.sk_flags + ((pair_id + j) * 2 + rank) * 8 + (warp - kEpiWarp0);
+                        seen = false;
+                        for (uint32_t i = 0; i < ptx::kMbarPollLimit; ++i) {
+                            if (*f == p.sk_epoch) {
+                                seen = true;
+                                break;
+                            }
+                            if ((i & 1023u) == 1023u && abort_flag[0]) break;
+                        }
+                    }
+                    if (!seen) {
+                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x560u);
+                        abort_flag[0] = 1;
+                    }
+                }
+                seen = __shfl_sync(0xFFFFFFFFu, seen ? 1 : 0, 0) != 0;
+                __threadfence();
+                if (!seen) {       // give up: nothing is stored; the raised flag ends the other roles' waits
+                    ok = false;
+                    break;
+                }
+            }
             if (!ptx::mbar_wait(&acc_full[0], tcount & 1, abort_flag)) {
                 if (lane == 0) report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x540u);
                 abort_flag[0] = 1;
@@ -518,12 +620,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 break;
             }
             ptx::tc_fence_after_sync();
-            const int row0 = m0 + mb * 2 * PM + q * 32;
-            const int rows = min(32, x.M - row0);
-            const int nunits = (row0 < x.M) ? (min(x.width, x.N - n0) + cpc - 1) / cpc : 0;
-            const uint32_t tbase = tmem_base + mb * PN + (static_cast<uint32_t>(q * 32) << 16);
-            // first 4 KiB block of this warp's rows inside a partial-tile slot: (CTA, row block, lane quarter) x 8 column blocks
-            const int64_t sk_block = ((static_cast<int64_t>(rank) * 2 + mb) * 4 + q) * (PN / 32);
+            if (warp == kEpiWarp0 && lane == 0) KLIN_T(tcount < 8 ? 40 + 3 * static_cast<int>(tcount) : -1);
 
             auto release = [&]() {
                 ptx::tc_fence_before_sync();
@@ -640,52 +737,26 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     *reinterpret_cast<volatile unsigned*>(p.sk_flags + (pair_id * 2 + rank) * 8 + (warp - kEpiWarp0)) = p.sk_epoch;
                 continue;
             }
-            // A piece with the tile's first but not its last k-block: the pairs after this one hold the rest of the
-            // tile's K range, each as one partial tile in its slot, in k order.  They computed those pieces first of
-            // all, so the flags are long up; the wait is bounded all the same.
-            int n_part = 0;
-            if (SK && wk.kind == 2) {
-                const int64_t rel = wk.tile - p.sk_first;
-                for (int64_t j = pair_id + 1; j < n_pairs; ++j) {
-                    const int64_t sj = j * p.sk_work / n_pairs;
-                    if (sj % p.nkb == 0 || sj / p.nkb != rel) break;
-                    ++n_part;
-                }
-                bool seen = true;
-                if (lane == 0) {
-                    for (int j = 1; j <= n_part && seen; ++j) {
-                        const volatile unsigned* f = p.sk_flags + ((pair_id + j) * 2 + rank) * 8 + (warp - kEpiWarp0);
-                        seen = false;
-                        for (uint32_t i = 0; i < ptx::kMbarPollLimit; ++i) {
-                            if (*f == p.sk_epoch) {
-                                seen = true;
-                                break;
-                            }
-                            if ((i & 1023u) == 1023u && abort_flag[0]) break;
-                        }
-                    }
-                    if (!seen) {
-                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x560u);
-                        abort_flag[0] = 1;
-                    }
-                }
-                seen = __shfl_sync(0xFFFFFFFFu, seen ? 1 : 0, 0) != 0;
-                __threadfence();
-                if (!seen) {       // give up: hand the accumulator back so that the other roles drain, store nothing
-                    release();
-                    ok = false;
-                    break;
-                }
+            if (nunits == 0) {
+                release();
+                continue;
             }
-            // adds the partial sums of unit u (this lane's row, the unit's columns) to r0 / r1, in k order
+            uint32_t a0[32], a1[32], c0[32], c1[32];
+            // adds the partial sums of unit u (this lane's row, the unit's columns) to r0 / r1, slot by slot = in k order;
+            // all of a slot's loads for the unit (eight, or sixteen for a 2-byte C) are in flight together
             auto add_partials = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32]) {
+#pragma unroll 1
                 for (int j = 1; j <= n_part; ++j) {
                     // unit u = 32-column blocks u * (cpc / 32) and, for a 2-byte C, the next one
                     const float4* src = reinterpret_cast<const float4*>(p.sk_slots + (pair_id + j) * (TILE_M * PN) + sk_block * 1024) +
                                         u * (cpc / 32) * 256 + lane;
-                    float4 t[8];
+                    float4 t[8], t2[8];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) t[i] = __ldcg(src + i * 32);
+                    // (unconditional: values defined on one side of a branch only cost the register allocator
+                    // dearly here - 1.4 KB of spills; a 4-byte C re-reads its block and ignores the copy)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) t2[i] = __ldcg(src + (out_bf16 ? 256 : 0) + i * 32);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         r0[4 * i] = __float_as_uint(__uint_as_float(r0[4 * i]) + t[i].x);
@@ -695,26 +766,33 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     }
                     if (out_bf16) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) t[i] = __ldcg(src + 256 + i * 32);
-#pragma unroll
                         for (int i = 0; i < 8; ++i) {
-                            r1[4 * i] = __float_as_uint(__uint_as_float(r1[4 * i]) + t[i].x);
-                            r1[4 * i + 1] = __float_as_uint(__uint_as_float(r1[4 * i + 1]) + t[i].y);
-                            r1[4 * i + 2] = __float_as_uint(__uint_as_float(r1[4 * i + 2]) + t[i].z);
-                            r1[4 * i + 3] = __float_as_uint(__uint_as_float(r1[4 * i + 3]) + t[i].w);
+                            r1[4 * i] = __float_as_uint(__uint_as_float(r1[4 * i]) + t2[i].x);
+                            r1[4 * i + 1] = __float_as_uint(__uint_as_float(r1[4 * i + 1]) + t2[i].y);
+                            r1[4 * i + 2] = __float_as_uint(__uint_as_float(r1[4 * i + 2]) + t2[i].z);
+                            r1[4 * i + 3] = __float_as_uint(__uint_as_float(r1[4 * i + 3]) + t2[i].w);
                         }
                     }
                 }
             };
-            if (nunits == 0) {
-                release();
+            if (SK && n_part > 0) {
+                // The owner of a streamed tile, unit by unit: the accumulator's values plus the partial sums of the
+                // later k ranges.  (One unit of the accumulator in registers at a time: the registers go to the
+                // sixteen loads per lane that are in flight for every slot.)
+#pragma unroll 1
+                for (int u = 0; u < nunits; ++u) {
+                    issue(u, a0, a1);
+                    ptx::tmem_ld_wait();
+                    if (u == nunits - 1) release();
+                    if (warp == kEpiWarp0 && lane == 0) KLIN_T(48 + 3 * u);
+                    add_partials(u, a0, a1);
+                    if (warp == kEpiWarp0 && lane == 0) KLIN_T(49 + 3 * u);
+                    pack(u, a0, a1, c0);
+                    stage_store(u, c0);
+                    if (warp == kEpiWarp0 && lane == 0) KLIN_T(50 + 3 * u);
+                }
                 continue;
             }
-            uint32_t a0[32], a1[32], c0[32], c1[32];
-            auto pack_p = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32], uint32_t (&w)[32]) {
-                if (SK && n_part > 0) add_partials(u, r0, r1);
-                pack(u, r0, r1, w);
-            };
             if (out_bf16 && nunits == 4 && n_part == 0) {
                 // Full-width bf16 tile: the accumulator is handed back before anything is staged or stored.
                 // Rounding (F2F, 16 results per clock and SM) is what the drain costs: three units are read
@@ -723,13 +801,14 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 // MMAs already fill it again.
                 uint32_t d0[32], d1[32], w0[32];
                 issue(0, a0, a1);
+                ptx::tmem_ld_wait();
                 issue(1, c0, c1);
                 issue(2, d0, d1);
-                ptx::tmem_ld_wait();
-                pack(0, a0, a1, w0);           // frees a0, a1 for the fourth unit
+                pack(0, a0, a1, w0);           // (while units 1 and 2 are on their way) frees a0, a1 for the fourth unit
                 issue(3, a0, a1);
                 ptx::tmem_ld_wait();
                 release();
+                if (warp == kEpiWarp0 && lane == 0) KLIN_T(tcount < 8 ? 41 + 3 * static_cast<int>(tcount) : -1);
                 stage_store(0, w0);
                 pack(1, c0, c1, w0);
                 stage_store(1, w0);
@@ -737,6 +816,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 stage_store(2, w0);
                 pack(3, a0, a1, w0);
                 stage_store(3, w0);
+                if (warp == kEpiWarp0 && lane == 0) KLIN_T(tcount < 8 ? 42 + 3 * static_cast<int>(tcount) : -1);
                 continue;
             }
             if (!out_bf16 && nunits == 8 && n_part == 0) {
@@ -772,21 +852,20 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 stage_store(7, a1);
                 continue;
             }
-            // (a tile that adds partial sums takes this path whatever its width)
             issue(0, a0, a1);
             for (int u = 0; u < nunits; u += 2) {
                 ptx::tmem_ld_wait();
                 if (u + 1 < nunits) issue(u + 1, c0, c1); else release();
                 {
                     uint32_t w[32];
-                    pack_p(u, a0, a1, w);
+                    pack(u, a0, a1, w);
                     stage_store(u, w);
                 }
                 if (u + 1 < nunits) {
                     ptx::tmem_ld_wait();
                     if (u + 2 < nunits) issue(u + 2, a0, a1); else release();
                     uint32_t w[32];
-                    pack_p(u + 1, c0, c1, w);
+                    pack(u + 1, c0, c1, w);
                     stage_store(u + 1, w);
                 }
             }
@@ -800,6 +879,14 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
     __syncthreads();
     ptx::cluster_arrive_release();
     ptx::cluster_wait_acquire();
+    if (threadIdx.x == 0) KLIN_T(4);
+#ifdef KLIN_TRACE
+    if (threadIdx.x == 0) {
+        unsigned long long ns;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+        if (blockIdx.x < kTraceCtas) KLIN_TRACE_BUF[blockIdx.x * kTraceSlots + 6] = ns;
+    }
+#endif
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         tmem_dealloc_pair(tmem_base, kTmemCols);
