@@ -83,6 +83,32 @@ __device__ __forceinline__ bool mbar_wait_addr(uint32_t bar_addr, uint32_t parit
     return false;
 }
 
+// Named barrier `id` of the CTA, split in two: threads that only signal (arrive) and threads that wait (sync) for
+// `threads` participants in total (a multiple of the warp size; every thread of a warp executes the same one).
+__device__ __forceinline__ void named_barrier_arrive(uint32_t id, uint32_t threads)
+{
+    asm volatile("barrier.cta.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t threads)
+{
+    asm volatile("barrier.cta.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// One non-blocking look at a barrier's phase (mbarrier.test_wait never suspends the thread): role loops probe the
+// NEXT stage's barrier before they issue the current stage's work, so that the answer is there when they need it.
+__device__ __forceinline__ uint32_t mbar_test_addr(uint32_t bar_addr, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_addr), "r"(parity)
+        : "memory");
+    return ok;
+}
+
 // ------------------------------------------------------------------- fences
 // Orders generic-proxy shared-memory writes before async-proxy reads (TMA
 // store, tcgen05.mma operand fetch).

@@ -44,6 +44,32 @@
 #include <mutex>
 #include <new>
 
+#ifdef KLIN_TRACE
+static __device__ unsigned long long klin_trace_single[klin::kTraceSlots * klin::kTraceCtas];
+#define KLIN_TRACE_BUF klin_trace_single
+extern "C" int klin_trace_dump_single(unsigned long long* host)
+{
+    cudaDeviceSynchronize();
+    const cudaError_t e = cudaMemcpyFromSymbol(host, klin_trace_single, sizeof klin_trace_single);
+    void* dev = nullptr;
+    if (cudaGetSymbolAddress(&dev, klin_trace_single) == cudaSuccess) cudaMemset(dev, 0, sizeof klin_trace_single);
+    return static_cast<int>(e);
+}
+static __device__ int klin_trace_knob;      // experiments: MMAs issued per k-block (0 = all four)
+extern "C" int klin_trace_set_knob(int v)
+{
+    return static_cast<int>(cudaMemcpyToSymbol(klin_trace_knob, &v, sizeof v));
+}
+#define KLIN_TNS(slot)                                                                             \
+    do {                                                                                           \
+        unsigned long long ns_;                                                                    \
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns_));                                    \
+        if (blockIdx.x < klin::kTraceCtas) KLIN_TRACE_BUF[blockIdx.x * klin::kTraceSlots + (slot)] = ns_; \
+    } while (0)
+#else
+#define KLIN_TNS(slot) ((void)0)
+#endif
+
 namespace klin {
 namespace {
 
@@ -56,7 +82,7 @@ constexpr int kStageBytes = kABytes + kBBytes;    // 48 KiB
 constexpr int kConvFilterBytes = (BN / 2) * BK * 2;                                  // 16 KiB
 constexpr int kConvStageBytes = kABytes + kConvFilterBytes;                          // 32 KiB
 constexpr int kConvStages = 6;
-constexpr int kMaxStages = 6;                     // deepest ring (32 KiB stages of 128-column tiles)
+constexpr int kMaxStages = 8;                     // deepest ring (24 KiB stages of 64-column tiles; 6 x 32 KiB with 128 columns)
 static_assert(kConvStages * kConvStageBytes <= STAGES * kStageBytes, "conv ring exceeds the ring area");
 constexpr int kEpiBufBytes = 32 * 128;            // one 32-row x 128-byte staging block
 constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;   // 4 warps x 2 buffers
@@ -259,6 +285,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     const uint32_t NS = kTunable ? static_cast<uint32_t>(p.n_stages) : static_cast<uint32_t>(STAGES);
     const uint32_t SB = kTunable ? p.stage_bytes : static_cast<uint32_t>(kStageBytes);
     const int TN = kTunable ? p.tile_n : BN;
+    // (Measured: a tcgen05.mma of this kernel issues every ~159 clocks whatever its N - 64, 128 or 256 - and
+    // whether or not consecutive ones share an accumulator: letting a narrow tile's k-steps alternate between
+    // two or four accumulators, summed by the epilogue, left the main loop at 636 clocks per k-block and only made
+    // the epilogue longer.  What a narrow tile buys is a shorter epilogue and more CTAs, not cheaper MMAs.)
     int group_hint = 0;     // MODE 2: a thread's units come in increasing order; its group search resumes here
     // One unit of the schedule for this thread's role.
     auto unit_of = [&](int64_t u) {
@@ -329,6 +359,38 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         else
             ptx::tma_load_2d(dst, map, c0, c1, bar);
     };
+    // The expect-tx arrive and the loads of one stage: k-block kb of the tile at (m0, n0) of the producer's unit.
+    auto stage_loads = [&](uint32_t s, int kb, int m0, int n0) {
+        uint8_t* sa = smem + s * SB;
+        uint8_t* sb = sa + kABytes;
+        ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
+        const CUtensorMap* pa = (MODE == 2) ? prod.ma : &map_a;
+        const CUtensorMap* pb = (MODE == 2) ? prod.mb : &map_b;
+        if (MODE == 4) {
+            // Conv2d: k-block = (filter tap, 64-channel group); the A stage is ONE box of 64 channels
+            // x 16 x 8 pixels (the tile's output patch shifted by the tap) - where it leaves the
+            // image the TMA unit fills zeros, which is the padding.  GEMM row = 16 * patch row + column.
+            const int cpb = p.conv.C >> 6;
+            const int tap = kb / cpb, cg = kb - tap * cpb;
+            const int fr = tap / p.conv.S, fs = tap - fr * p.conv.S;
+            ptx::tma_load_4d(sa, &map_a, cg * 64, prod.cw + fs, prod.ch + fr, prod.cn, &full[s]);
+        } else
+            load_box(sa, pa, kb * BK, m0, &full[s]);
+        if (BCOL) {
+            load_box(sb, pb, kb * BK, n0, &full[s]);
+        } else if (MODE == 1 && p.b_box3d) {
+            ptx::tma_load_4d(sb, pb, 0, kb * BK, n0 >> 6, prod.z, &full[s]);   // the same box, batch as 4th coordinate
+        } else if ((MODE == 0 || MODE == 3) && p.b_box3d) {
+            // B viewed as (64 columns, K rows, N / 64 column blocks): one box of 64 x 64 x 4 lands as the
+            // four consecutive 8 KiB blocks the MN-major descriptor expects - one TMA instruction, not four
+            // (a producer thread issues a TMA instruction every ~110 cycles)
+            ptx::tma_load_3d(sb, pb, 0, kb * BK, n0 >> 6, &full[s]);
+        } else {
+#pragma unroll
+            for (int cb = 0; cb < BN / 64; ++cb)
+                if (cb * 64 < TN) load_box(sb + cb * (64 * BK * 2), pb, n0 + cb * 64, kb * BK, &full[s]);
+        }
+    };
     // Issues loads until `limit` k-blocks have been issued in total or the schedule ends.
     auto produce = [&](uint32_t limit) {
         while (prod.live && prod.it < limit) {
@@ -344,35 +406,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 prod.live = false;
                 break;
             }
-            uint8_t* sa = smem + s * SB;
-            uint8_t* sb = sa + kABytes;
-            ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
-            const CUtensorMap* pa = (MODE == 2) ? prod.ma : &map_a;
-            const CUtensorMap* pb = (MODE == 2) ? prod.mb : &map_b;
-            if (MODE == 4) {
-                // Conv2d: k-block = (filter tap, 64-channel group); the A stage is ONE box of 64 channels
-                // x 16 x 8 pixels (the tile's output patch shifted by the tap) - where it leaves the
-                // image the TMA unit fills zeros, which is the padding.  GEMM row = 16 * patch row + column.
-                const int cpb = p.conv.C >> 6;
-                const int tap = prod.kb / cpb, cg = prod.kb - tap * cpb;
-                const int fr = tap / p.conv.S, fs = tap - fr * p.conv.S;
-                ptx::tma_load_4d(sa, &map_a, cg * 64, prod.cw + fs, prod.ch + fr, prod.cn, &full[s]);
-            } else
-            load_box(sa, pa, prod.kb * BK, prod.m0, &full[s]);
-            if (BCOL) {
-                load_box(sb, pb, prod.kb * BK, prod.n0, &full[s]);
-            } else if (MODE == 1 && p.b_box3d) {
-                ptx::tma_load_4d(sb, pb, 0, prod.kb * BK, prod.n0 >> 6, prod.z, &full[s]);   // the same box, batch as 4th coordinate
-            } else if ((MODE == 0 || MODE == 3) && p.b_box3d) {
-                // B viewed as (64 columns, K rows, N / 64 column blocks): one box of 64 x 64 x 4 lands as the
-                // four consecutive 8 KiB blocks the MN-major descriptor expects - one TMA instruction, not four
-                // (a producer thread issues a TMA instruction every ~110 cycles)
-                ptx::tma_load_3d(sb, pb, 0, prod.kb * BK, prod.n0 >> 6, &full[s]);
-            } else {
-#pragma unroll
-                for (int cb = 0; cb < BN / 64; ++cb)
-                    if (cb * 64 < TN) load_box(sb + cb * (64 * BK * 2), pb, prod.n0 + cb * 64, prod.kb * BK, &full[s]);
-            }
+            stage_loads(s, prod.kb, prod.m0, prod.n0);
             ++prod.it;
             if (++prod.st == NS) {
                 prod.st = 0;
@@ -385,29 +419,111 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         }
     };
 
-    if (warp == 0 && lane == 0) {
-        for (uint32_t s = 0; s < NS; ++s) {
-            ptx::mbar_init(&full[s], GENERIC ? kProducerThreads + ((MODE == 4 && p.conv_b_tma) ? 1 : 0) : 1);
-            ptx::mbar_init(&empty[s], 1);
+    // The rest of the schedule after the first ring fill, for the TMA-fed GEMM forms: the ring position is carried in
+    // registers and a unit's k-blocks run in a loop of their own - wait, expect-tx arrive, loads, nothing else.  (Short
+    // k-blocks are bound by the round trip "stage freed -> loads issued -> data landed", about 2 k clocks of TMA
+    // latency under load plus this thread's own instruction stream: the general loop above spent 500 clocks per
+    // stage on itself.)
+    auto produce_rest = [&]() {
+        uint32_t st = prod.st, ph = prod.ph, it = prod.it;
+        const uint32_t empty0 = ptx::smem_u32(empty);
+        uint32_t ready = 0;     // the current stage's "empty" barrier was seen complete by the look-ahead probe
+        while (prod.live) {
+            const int m0 = prod.m0, n0 = prod.n0, kb1 = prod.kb1;
+            for (int kb = prod.kb; kb < kb1; ++kb, ++it) {
+                if (it == 8) KLIN_T(20);
+                if (it == 9) KLIN_T(23);
+                if (!ready && !ptx::mbar_wait_addr(empty0 + 8 * st, ph, abort_flag)) {
+                    report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x400u | st);
+                    abort_flag[0] = 1;
+                    prod.live = false;
+                    break;
+                }
+                if (it == 8) KLIN_T(21);
+                if (it == 9) KLIN_T(24);
+                const uint32_t st_next = (st + 1 == NS) ? 0u : st + 1, ph_next = (st + 1 == NS) ? ph ^ 1u : ph;
+                ready = ptx::mbar_test_addr(empty0 + 8 * st_next, ph_next);
+                stage_loads(st, kb, m0, n0);
+                if (it == 8) KLIN_T(22);
+                if (it == 9) KLIN_T(25);
+                st = st_next;
+                ph = ph_next;
+            }
+            if (!prod.live) break;
+            prod.u += gridDim.x;
+            prod_enter_unit();
         }
-        for (int b = 0; b < 2; ++b) {
-            ptx::mbar_init(&acc_full[b], 1);
-            ptx::mbar_init(&acc_empty[b], 4);
+        prod.it = it;
+    };
+
+    // Set-up.  In the TMA-fed GEMM forms warp 0 does not wait for the other warps: it initialises the barriers,
+    // signals (a named barrier the others wait on) and goes straight on to the first ring fill, while warp 1
+    // allocates TMEM and the MMA and epilogue threads work out their first unit.  (The fill used to come before a
+    // CTA-wide barrier that every warp waited on: on 256^3 the first MMA was issued 4.9 k clocks after the CTA's
+    // start, 2.2 k of them spent issuing four stages of loads one after the other.)
+    constexpr bool kEarlyProducer = !GENERIC && (MODE == 0 || MODE == 1 || MODE == 3);
+    // The first ring fill in one pass of the instruction stream: lane l issues stage l (plain GEMM forms).
+    constexpr bool kLockstepFill = !GENERIC && (MODE == 0 || MODE == 3);
+    if (warp == 0) {
+        if (lane == 0) {
+            KLIN_T(0);
+            KLIN_TNS(6);
+            for (uint32_t s = 0; s < NS; ++s) {
+                ptx::mbar_init(&full[s], GENERIC ? kProducerThreads + ((MODE == 4 && p.conv_b_tma) ? 1 : 0) : 1);
+                ptx::mbar_init(&empty[s], 1);
+            }
+            for (int b = 0; b < 2; ++b) {
+                ptx::mbar_init(&acc_full[b], 1);
+                ptx::mbar_init(&acc_empty[b], 4);
+            }
+            if (ring6)
+                for (int i = 0; i < 2 * kConvStages; ++i) ptx::mbar_init(&cfull[i], 1);
+            abort_flag[0] = 0;
+            abort_flag[1] = 0;
+            ptx::fence_barrier_init();
+            if (!GENERIC && MODE != 2) {
+                ptx::prefetch_tensormap(&map_a);
+                ptx::prefetch_tensormap(&map_b);
+            }
+            if (p.epi_tma && MODE != 2 && MODE != 3) ptx::prefetch_tensormap(&map_c);
+            KLIN_T(1);
         }
-        if (ring6)
-            for (int i = 0; i < 2 * kConvStages; ++i) ptx::mbar_init(&cfull[i], 1);
-        abort_flag[0] = 0;
-        abort_flag[1] = 0;
-        ptx::fence_barrier_init();
-        if (!GENERIC && MODE != 2) {
-            ptx::prefetch_tensormap(&map_a);
-            ptx::prefetch_tensormap(&map_b);
+        if (kEarlyProducer) {
+            __syncwarp();
+            ptx::named_barrier_arrive(1, blockDim.x);
         }
-        if (p.epi_tma && MODE != 2 && MODE != 3) ptx::prefetch_tensormap(&map_c);
         // The launch is a programmatic dependent one: everything above (and the TMEM
         // allocation in warp 1) may overlap the tail of the previous kernel in the stream;
         // nothing below the wait touches global memory before that kernel has completed.
-        if (!GENERIC && MODE != 2) prod_enter_unit();           // schedule arithmetic only
+        if (lane == 0 && !GENERIC && MODE != 2) prod_enter_unit();           // schedule arithmetic only
+        if (lane == 0) KLIN_T(2);
+        const bool lockstep = kLockstepFill && !ring6 && !p.static_b && p.test_stop_after == 0;
+        if (lockstep) {
+            const int kb = __shfl_sync(0xFFFFFFFFu, prod.kb, 0), kb1 = __shfl_sync(0xFFFFFFFFu, prod.kb1, 0);
+            const int m0 = __shfl_sync(0xFFFFFFFFu, prod.m0, 0), n0 = __shfl_sync(0xFFFFFFFFu, prod.n0, 0);
+            const int live = __shfl_sync(0xFFFFFFFFu, prod.live ? 1 : 0, 0);
+            const int nfill = live ? min(static_cast<int>(NS), kb1 - kb) : 0;
+            ptx::grid_dependency_wait();
+            if (lane == 0) KLIN_T(3);
+            // (the "empty" barriers are fresh: the first NS loads wait for nothing)
+            if (lane < nfill) stage_loads(static_cast<uint32_t>(lane), kb + lane, m0, n0);
+            __syncwarp();
+            if (lane == 0 && nfill > 0) {
+                prod.it = static_cast<uint32_t>(nfill);
+                if (static_cast<uint32_t>(nfill) == NS) {
+                    prod.st = 0;
+                    prod.ph ^= 1u;
+                } else {
+                    prod.st = static_cast<uint32_t>(nfill);
+                }
+                prod.kb += nfill;
+                if (prod.kb == prod.kb1) {
+                    prod.u += gridDim.x;
+                    prod_enter_unit();
+                }
+            }
+            if (lane == 0) KLIN_T(4);
+        } else if (lane == 0) {
         if (!GENERIC && MODE == 0 && p.static_b && prod.live && prod.kb1 - prod.kb >= STAGES) {
             // Static B: the B boxes of the first ring fill do not depend on the previous kernel in
             // the stream and go out at once; only A waits (C is written much later, after the wait
@@ -437,13 +553,16 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             }
         } else {
             ptx::grid_dependency_wait();
+            KLIN_T(3);
             if (!GENERIC && MODE != 2) {
                 // The first ring fill needs nothing from the other warps: start it before the
                 // set-up barrier so that TMEM allocation hides behind the first loads' latency.
                 if (!ring6 && !(MODE == 4 && p.conv_t)) produce(NS);
             }
+            KLIN_T(4);
         }
-        if (blockIdx.x == 0) g.status[1] = p.kid;
+        }
+        if (lane == 0 && blockIdx.x == 0) g.status[1] = p.kid;
     }
     if (MODE == 2 && warp >= 2) {
         // the grouped schedule's prefix sums (written on the stream before this launch)
@@ -456,9 +575,15 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before_sync();
-    __syncthreads();
+    if (threadIdx.x == 32) KLIN_T(16);
+    if (kEarlyProducer) {
+        if (warp != 0) ptx::named_barrier_sync(1, blockDim.x);
+    } else {
+        __syncthreads();
+    }
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) KLIN_T(5);
     ptx::grid_dependency_wait();
     ptx::grid_launch_dependents();
     if (SWAP && p.cluster) ptx::cluster_wait_acquire();
@@ -564,7 +689,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 ptx::mbar_wait(&cfull[j % kConvStages], (j / kConvStages) & 1, abort_flag + 1);
         } else if (!GENERIC && lane == 0) {
             if (MODE == 2) prod_enter_unit();      // (its group search reads the table the other warps just staged)
-            produce(0xFFFFFFFFu);
+            if (MODE == 4 || p.test_stop_after > 0)
+                produce(0xFFFFFFFFu);
+            else
+                produce_rest();
             // Drain: every load issued must have landed before shared memory is released.
             const uint32_t it = prod.it;
             const uint32_t first = it > NS ? it - NS : 0;
@@ -602,6 +730,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             // (Measured: the length of this instruction stream does not bound the kernel - trimming it changed no
             // timing, and releasing stages in pairs to halve the commits was slower, because the ring got shallower.)
             uint32_t s = 0, ph = 0;
+            uint32_t ready = 0;     // the current stage's "full" barrier was seen complete by the look-ahead probe
+#ifdef KLIN_TRACE
+            const int trace_knob = klin_trace_knob > 0 ? klin_trace_knob : 4;
+#endif
             const uint32_t full0 = ptx::smem_u32(ring6 ? cfull : full), empty0 = ptx::smem_u32(ring6 ? cempty : empty);
             const uint32_t n_stages = ring6 ? kConvStages : NS;
             const uint32_t stage_step = (ring6 ? static_cast<uint32_t>(kConvStageBytes) : SB) >> 4;
@@ -621,18 +753,35 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     break;
                 }
                 ptx::tc_fence_after_sync();
+                if (t == 0) KLIN_T(8);
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag, full_limit)) {
+                    if (t == 0 && kb == kb0 + 8) KLIN_T(26);
+                    if (t == 0 && kb == kb0 + 9) KLIN_T(29);
+                    if (!ready && !ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag, full_limit)) {
                         report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x420u | s);
                         abort_flag[0] = 1;
                         ok = false;
                         break;
                     }
-                    ptx::tc_fence_after_sync();
+                    // (TMA-fed operands need no tcgen05 fence here: they were written through the async proxy, which
+                    // is also how the MMA reads them.)
+                    if (GENERIC) ptx::tc_fence_after_sync();
+                    // The
+                    // next stage's barrier is probed now: a passing wait costs ~250 clocks of latency when it is
+                    // asked for only at the top of the next iteration.
+                    const uint32_t s_next = (s + 1 == n_stages) ? 0u : s + 1, ph_next = (s + 1 == n_stages) ? ph ^ 1u : ph;
+                    ready = ptx::mbar_test_addr(full0 + 8 * s_next, ph_next);
+                    if (t == 0 && kb == kb0) KLIN_T(9);
+                    if (t == 0 && kb == kb1 - 1) KLIN_T(10);
+                    if (t == 0 && kb == kb0 + 8) KLIN_T(27);
+                    if (t == 0 && kb == kb0 + 9) KLIN_T(30);
                     const uint32_t a_lo = a_lo0 + s * stage_step, b_lo = b_lo0 + s * stage_step;
 #pragma unroll
                     for (int k4 = 0; k4 < BK / 16; ++k4) {
+#ifdef KLIN_TRACE
+                        if (k4 >= trace_knob) continue;
+#endif
                         // K-major operand: +32 bytes per 16 k inside the 128-byte swizzle row.
                         const uint32_t acc = (kb > kb0 || k4 > 0) ? 1u : 0u;
                         const uint64_t a_desc = (static_cast<uint64_t>(a_hi) << 32) | (a_lo + 2u * k4);
@@ -650,12 +799,13 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         }
                     }
                     ptx::umma_commit_addr(empty0 + 8 * s);
-                    if (++s == n_stages) {
-                        s = 0;
-                        ph ^= 1u;
-                    }
+                    if (t == 0 && kb == kb0 + 8) KLIN_T(28);
+                    if (t == 0 && kb == kb0 + 9) KLIN_T(31);
+                    s = s_next;
+                    ph = ph_next;
                 }
                 if (ok) ptx::umma_commit(&acc_full[buf]);
+                if (t == 0) KLIN_T(11);
             }
         }
     } else if (warp < 6) {
@@ -678,6 +828,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 break;
             }
             ptx::tc_fence_after_sync();
+            if (t == 0 && warp == 2 && lane == 0) KLIN_T(12);
             if (SWAP) {
                 // lane = weight column n, registers = activation rows m
                 const bool partial = p.splits > 1 && !p.cluster;
@@ -958,6 +1109,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
+            if (t == 0 && warp == 2 && lane == 0) KLIN_T(13);
 
             if (p.splits > 1 && row0 < g.M) {
                 // Arrival per (tile, 32-row block); the last arriver adds the partials in split order.
@@ -1468,8 +1620,13 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         }
     }
 
+    if (warp == 2 && lane == 0) KLIN_T(14);
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (threadIdx.x == 0) {
+        KLIN_T(15);
+        KLIN_TNS(7);
+    }
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
@@ -1802,7 +1959,8 @@ bool plan_launch(const GemmArgs& g, const RunContext& ctx, bool generic, bool mu
     if (pl.kernel != 2 && (pl.tile_n != 0 || pl.stages != 0)) {        // pinned (the pair kernel reads the fields its own way)
         const int tn = pl.tile_n != 0 ? pl.tile_n : BN;
         const int st = pl.stages != 0 ? pl.stages : STAGES;
-        const bool ok = (tn == BN && st == STAGES) || (tunable && (tn == BN / 2 || tn == BN / 4) && (st == 4 || st == 6));
+        const bool ok = (tn == BN && st == STAGES) ||
+                        (tunable && ((tn == BN / 2 && (st == 4 || st == 6)) || (tn == BN / 4 && (st == 4 || st == 6 || st == 8))));
         return ok && try_shape(tn, st, out);
     }
     LaunchPlan wide;
@@ -2389,9 +2547,9 @@ bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& pl)
     if (pl.split_via == 3 && (pl.kernel != 2 || pl.splits > 1)) return false;     // streaming the last wave is the pair kernel's
     if (pl.kernel == 2 && pl.stages != 0) return false;
     if (pl.kernel != 2 && (pl.tile_n != 0 || pl.stages != 0)) {
-        // single-CTA kernel: 256 columns x 4 stages, or 128 / 64 columns x 4 or 6 stages (plain TMA-fed GEMM, M > 64)
+        // single-CTA kernel: 256 columns x 4 stages, 128 columns x 4 or 6, 64 columns x 4, 6 or 8 (plain TMA-fed GEMM, M > 64)
         if (pl.tile_n != 0 && pl.tile_n != BN && pl.tile_n != BN / 2 && pl.tile_n != BN / 4) return false;
-        if (pl.stages != 0 && pl.stages != 4 && pl.stages != 6) return false;
+        if (pl.stages != 0 && pl.stages != 4 && pl.stages != 6 && !(pl.stages == 8 && pl.tile_n == BN / 4)) return false;
     }
     // a tile shape is a property of one of the two kernels: name the kernel with it
     if ((pl.tile_n != 0 || pl.tail_n != 0 || pl.stages != 0) && pl.kernel == 0) return false;
@@ -2475,12 +2633,14 @@ int r4_enumerate_plans(const GemmArgs& g, const RunContext& ctx, R4Plan* out, in
             push(pl);
         }
         if (tiles * 2 <= ctx.sm_count) {     // few tiles: 64 columns
-            R4Plan pl;
-            pl.kernel = 1;
-            pl.splits = 1;
-            pl.tile_n = BN / 4;
-            pl.stages = 4;
-            push(pl);
+            for (int st : {4, 8}) {
+                R4Plan pl;
+                pl.kernel = 1;
+                pl.splits = 1;
+                pl.tile_n = BN / 4;
+                pl.stages = st;
+                push(pl);
+            }
         }
         for (int gm : {4, 8, 16, 32}) {
             if (gm > 4 && gm / 2 >= tiles_m) continue;

@@ -490,13 +490,19 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             // plus s * (stage bytes >> 4) in the 14-bit start-address field (the ring ends below 256 KiB).  The next
             // tile's coordinates are worked out BEFORE the wait for the drained accumulators, not after it.
             uint32_t tcount = 0, s = 0, ph = 0;
+            uint32_t ready = 0;     // the current stage's "full" barrier was seen complete by the look-ahead probe
             bool ok = true;
             const uint32_t full0 = ptx::smem_u32(full), empty0 = ptx::smem_u32(empty);
             const uint32_t empty_odd0 = ptx::map_to_cta(empty0, 1);
             const uint32_t accf = ptx::smem_u32(&acc_full[0]), accf_odd = ptx::map_to_cta(accf, 1);
+            // descriptors: the high words never change, the low words step by 16-byte units (no carry out of the
+            // 14-bit address field inside the ring)
             const uint64_t a_desc0 = make_desc(ptx::smem_u32(smem), 1, (1024u >> 4) | (1u << 14) | (2u << 29));
             const uint64_t b_desc0 = make_desc(ptx::smem_u32(smem) + kABytes, p.b_desc_lbo, p.b_desc_hi);
+            const uint32_t a_lo0 = static_cast<uint32_t>(a_desc0), a_hi = static_cast<uint32_t>(a_desc0 >> 32);
+            const uint32_t b_lo0 = static_cast<uint32_t>(b_desc0), b_hi = static_cast<uint32_t>(b_desc0 >> 32);
             const uint32_t kstep = p.b_kstep;
+            auto desc = [](uint32_t hi, uint32_t lo) { return (static_cast<uint64_t>(hi) << 32) | lo; };
             WorkState ws = work_init();
             Work wk;
             for (; ok && next_work(ws, wk); ++tcount) {
@@ -513,32 +519,35 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 ptx::tc_fence_after_sync();
                 KLIN_T(tcount < 4 ? 8 + 4 * static_cast<int>(tcount) : -1);
                 for (int kb = kb_first; kb < kb_end; ++kb) {
-                    if (!ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag)) {
+                    if (!ready && !ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag)) {
                         report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x530u | s);
                         abort_flag[0] = 1;
                         ok = false;
                         break;
                     }
-                    ptx::tc_fence_after_sync();
+                    // (no tcgen05 fence: the operands came through the async proxy, which is how the MMA reads them.)
+                    // This thread's instruction stream bounds the main loop - eight MMAs at ~85 clocks of issue each
+                    // plus what surrounds them, against the 1024 clocks the tensor pipe needs - so the next
+                    // stage's barrier is probed here, a k-block ahead of the wait that would use the answer.
+                    const uint32_t s_next = (s + 1 == STAGES) ? 0u : s + 1, ph_next = (s + 1 == STAGES) ? ph ^ 1u : ph;
+                    ready = ptx::mbar_test_addr(full0 + 8 * s_next, ph_next);
                     if (kb == kb_first) KLIN_T(tcount < 4 ? 9 + 4 * static_cast<int>(tcount) : -1);
                     if (kb == kb_end - 1) KLIN_T(tcount < 4 ? 10 + 4 * static_cast<int>(tcount) : -1);
-                    const uint64_t a_desc = a_desc0 + s * static_cast<uint32_t>(kStageBytes >> 4);
-                    const uint64_t b_desc = b_desc0 + s * static_cast<uint32_t>(kStageBytes >> 4);
+                    const uint32_t a_lo = a_lo0 + s * static_cast<uint32_t>(kStageBytes >> 4);
+                    const uint32_t b_lo = b_lo0 + s * static_cast<uint32_t>(kStageBytes >> 4);
 #pragma unroll
                     for (int k4 = 0; k4 < BK / 16; ++k4) {
                         const uint32_t acc = (kb > kb_first || k4 > 0) ? 1u : 0u;
                         // alternate the two row blocks: consecutive MMAs never share an accumulator
-                        umma_f16_pair(tmem_base, a_desc + static_cast<uint64_t>(k4 * 2),
-                                      b_desc + static_cast<uint64_t>(k4 * kstep), idesc, acc);
-                        umma_f16_pair(tmem_base + PN, a_desc + static_cast<uint64_t>((kABlockBytes >> 4) + k4 * 2),
-                                      b_desc + static_cast<uint64_t>(k4 * kstep), idesc, acc);
+                        const uint64_t bd = desc(b_hi, b_lo + static_cast<uint32_t>(k4) * kstep);
+                        umma_f16_pair(tmem_base, desc(a_hi, a_lo + static_cast<uint32_t>(k4 * 2)), bd, idesc, acc);
+                        umma_f16_pair(tmem_base + PN, desc(a_hi, a_lo + static_cast<uint32_t>((kABlockBytes >> 4) + k4 * 2)),
+                                      bd, idesc, acc);
                     }
                     umma_commit_pair(empty0 + 8 * s);
                     umma_commit_pair(empty_odd0 + 8 * s);
-                    if (++s == STAGES) {
-                        s = 0;
-                        ph ^= 1u;
-                    }
+                    s = s_next;
+                    ph = ph_next;
                 }
                 if (ok) {
                     umma_commit_pair(accf);
