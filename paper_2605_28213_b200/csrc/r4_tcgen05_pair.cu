@@ -198,7 +198,10 @@ __device__ __forceinline__ void setmaxnreg_inc()
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar_addr) : "memory");
+    // (The arrive only says "my TMEM reads have completed" - tcgen05.wait::ld has made sure of that before - and
+    // publishes no memory.  With .release.cluster it took 1.3 k clocks per tile, on the path that keeps the next
+    // tile's MMAs waiting; the default form - release at CTA scope - is what this needs.)
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar_addr) : "memory");
 }
 
 __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_field, uint32_t hi)
@@ -633,7 +636,9 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
 
             auto release = [&]() {
                 ptx::tc_fence_before_sync();
+                if (tcount == 0 && warp == kEpiWarp0 && lane == 0) KLIN_T(60);
                 __syncwarp();
+                if (tcount == 0 && warp == kEpiWarp0 && lane == 0) KLIN_T(61);
                 if (lane == 0) mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&acc_empty[0]), 0));
             };
             auto issue = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32]) {
@@ -811,11 +816,15 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 uint32_t d0[32], d1[32], w0[32];
                 issue(0, a0, a1);
                 ptx::tmem_ld_wait();
+                if (tcount == 0 && warp == kEpiWarp0 && lane == 0) KLIN_T(56);
                 issue(1, c0, c1);
                 issue(2, d0, d1);
+                if (tcount == 0 && warp == kEpiWarp0 && lane == 0) KLIN_T(57);
                 pack(0, a0, a1, w0);           // (while units 1 and 2 are on their way) frees a0, a1 for the fourth unit
+                if (tcount == 0 && warp == kEpiWarp0 && lane == 0) KLIN_T(58);
                 issue(3, a0, a1);
                 ptx::tmem_ld_wait();
+                if (tcount == 0 && warp == kEpiWarp0 && lane == 0) KLIN_T(59);
                 release();
                 if (warp == kEpiWarp0 && lane == 0) KLIN_T(tcount < 8 ? 41 + 3 * static_cast<int>(tcount) : -1);
                 stage_store(0, w0);
@@ -944,15 +953,15 @@ bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx)
 {
     if (!r4_pair_possible(g, ctx) || g.M <= 2 * PM) return false;
     // Which kernel finishes first?  Estimated tensor-pipe cycles of either schedule, from measured rates:
-    // a 512 x 256 pair tile takes 1024 cycles per k-block (two accumulators alternate: full rate) plus
-    // ~5 k cycles per tile that the main loop does not hide (ring fill, accumulator drain and store); a 128 x 256
+    // a 512 x 256 pair tile takes ~1035 cycles per k-block (two accumulators alternate: full rate) plus
+    // ~3.6 k cycles per tile that the main loop does not hide (accumulator drain, barrier round trips); a 128 x 256
     // tile of the single-CTA kernel takes 636 per k-block (one accumulator: 159 per MMA) with its epilogue
     // hidden, and a last wave of at most half of the SMs is cut into half tiles worth ~0.75 of a wave.
     // Fitted to both kernels timed at 2048^3 .. 4096^3 (steps of 256), 2048 x 4096 x 4096 and 3072 x 2048 x 8192.
     const int64_t nkb = (g.K + BK - 1) / BK;
     const int64_t pairs = ctx.sm_count / 2;
     const int64_t tiles2 = static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * ((g.N + PN - 1) / PN);
-    const double t_pair = static_cast<double>((tiles2 + pairs - 1) / pairs) * (nkb * 1024.0 + 5000.0);
+    const double t_pair = static_cast<double>((tiles2 + pairs - 1) / pairs) * (nkb * 1035.0 + 3600.0);
     const int64_t tiles1 = static_cast<int64_t>((g.M + PM - 1) / PM) * ((g.N + PN - 1) / PN);
     const int64_t full = tiles1 / ctx.sm_count, tail = tiles1 % ctx.sm_count;
     const double waves = full + (tail == 0 ? 0.0 : (2 * tail <= ctx.sm_count && g.N > PN / 2 ? 0.75 : 1.0));
