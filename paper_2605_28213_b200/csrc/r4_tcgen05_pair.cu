@@ -278,8 +278,9 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
     if (threadIdx.x == 32) KLIN_T(25);      // TMEM allocated
     __syncthreads();
     if (threadIdx.x == 0) KLIN_T(26);
-    // Both CTAs' barriers exist before anyone signals across the pair.
-    ptx::cluster_arrive_release();
+    // Both CTAs' barriers exist before anyone signals across the pair (their initialisation was published by the
+    // mbarrier-init fence above; the arrive itself publishes nothing and need not be a release).
+    ptx::cluster_arrive_relaxed();
     ptx::cluster_wait_acquire();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
@@ -895,7 +896,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
     // No CTA leaves while its partner may still signal into its shared memory.
     ptx::tc_fence_before_sync();
     __syncthreads();
-    ptx::cluster_arrive_release();
+    ptx::cluster_arrive_relaxed();      // (an execution barrier only: no memory is handed over here)
     ptx::cluster_wait_acquire();
     if (threadIdx.x == 0) KLIN_T(4);
 #ifdef KLIN_TRACE
