@@ -1,9 +1,12 @@
 // Rung 1 - "tile / sm_stage" (paper, Table 1; precondition: loops over the
 // output).  A T x T block tile of C per CTA (T = 128, 64 or 32); A and B k-slabs
-// of depth 16 are staged in shared memory as fp32 (converted from bf16 on the way
+// of depth 16 or 32 are staged in shared memory as fp32 (converted from bf16 on the way
 // in) and each of the 256 threads keeps a (T/16) x (T/16) register tile.  Loads
 // are scalar and masked element by element, so every M/N/K tail and every
 // alignment is handled the same way; nothing is vectorized or overlapped yet.
+//
+// Two CTAs share an SM (the register tile is capped at 128 registers per thread for it): one CTA's slab fill overlaps
+// the other's arithmetic, which is all the overlap this rung has (8192^3: 20.3 -> 29.5 TFLOP/s).
 //
 // A thread's rows are ty + 16 i and its columns tx + 16 j: the 16 threads of a
 // half warp read 16 consecutive words of a shared-memory row (no bank conflict;
@@ -20,15 +23,20 @@
 namespace klin {
 namespace {
 
-constexpr int BK = 16, NT = 256;
+constexpr int NT = 256;
 
 template <bool BCOL, int T>
-__global__ void __launch_bounds__(NT) r1_tiled_kernel(GemmArgs g, int tiles_m, int tiles_n)
+__global__ void __launch_bounds__(NT, 2) r1_tiled_kernel(GemmArgs g, int tiles_m, int tiles_n)
 {
     constexpr int TT = T / 16;                 // register tile edge
-    // (row pitch = 2 mod 32 words: the k-fastest fill - 16 k values of 2 rows per warp - then hits 32 different banks)
-    __shared__ float As[BK][T + 2];
-    __shared__ float Bs[BK][T + 2];
+    // k-slab depth: 16 for the 128 tile; 32 for the smaller ones, which synchronise twice per slab for a quarter or a
+    // sixteenth of the arithmetic (measured: 16 x 8192 x 8192 535 -> 426 us, 1000 x 1001 x 999 105 -> 99 us; at 128
+    // the deeper slab was slower, 8192^3 29.5 -> 27.3 TFLOP/s)
+    constexpr int BK = T == 128 ? 16 : 32;
+    // a warp covers 16 k of 2 rows: 2 mod 32 spreads them over 32 banks; 32 k of one row with the deeper slab: 1 mod 32
+    constexpr int PITCH = BK == 16 ? T + 2 : T + 1;
+    __shared__ float As[BK][PITCH];
+    __shared__ float Bs[BK][PITCH];
     if (blockIdx.x == 0 && threadIdx.x == 0) g.status[1] = kIdTiled;
 
     int tm, tn;
