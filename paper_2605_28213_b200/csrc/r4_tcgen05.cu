@@ -1417,8 +1417,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         // comes straight from TMEM), adds the bias once, rounds and stores its pairs.  No workspace, no
         // atomics, no trip through L2.
         const uint32_t rank = ptx::cluster_ctarank();
-        ptx::cluster_arrive_release();
+        if (warp == 2 && lane == 0) KLIN_T(32);
+        ptx::cluster_arrive_relaxed();      // (an execution barrier: "my MMAs are done"; the data follows behind the second one)
         ptx::cluster_wait_acquire();
+        if (warp == 2 && lane == 0) KLIN_T(33);
         const bool epi_warp = warp >= 2 && warp < 6;
         const bool out_bf16 = g.c_bf16 != 0;
         const int sub_log2 = out_bf16 ? 1 : 0;                          // 32-column blocks per store unit
@@ -1460,8 +1462,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 }
             }
         }
+        if (warp == 2 && lane == 0) KLIN_T(34);
         ptx::cluster_arrive_release();
         ptx::cluster_wait_acquire();
+        if (warp == 2 && lane == 0) KLIN_T(35);
         if (epi_warp && !abort_flag[0]) {
             const Unit x = decode_unit(static_cast<int64_t>(blockIdx.x), p);
             uint8_t* stg = epi_smem + (warp - 2) * 2 * kEpiBufBytes;
