@@ -7,9 +7,9 @@
 // which fetch the other half of B from the peer's shared memory.  Per k-block a
 // CTA loads 48 KiB for 256 x 256 x 64 multiply-adds (half the bytes per flop of
 // the single-CTA 128 x 256 tile).  The two row blocks have separate fp32
-// accumulators in TMEM (2 x 256 columns) and their MMAs ALTERNATE: measured on
-// B200, back-to-back tcgen05.mma into the same accumulator run at 159 clocks
-// per 128 x 256 x 16 instruction, alternating accumulators at the full 128.
+// accumulators in TMEM (2 x 256 columns) and their MMAs ALTERNATE (row block 0,
+// row block 1, next k-step); eight full-width MMAs per k-block need 1024 clocks
+// of the tensor pipe, and the issuing thread keeps up with that (1033-1040 measured).
 //
 //   warp 0      TMA producer (each CTA loads its own A box and its half of B;
 //               every byte is fetched by exactly one CTA, into its own memory).  Both
@@ -956,7 +956,7 @@ bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx)
     // Which kernel finishes first?  Estimated tensor-pipe cycles of either schedule, from measured rates:
     // a 512 x 256 pair tile takes ~1035 cycles per k-block (two accumulators alternate: full rate) plus
     // ~3.6 k cycles per tile that the main loop does not hide (accumulator drain, barrier round trips); a 128 x 256
-    // tile of the single-CTA kernel takes 636 per k-block (one accumulator: 159 per MMA) with its epilogue
+    // tile of the single-CTA kernel takes 636 per k-block (its issuing thread and the shared-memory port) with its epilogue
     // hidden, and a last wave of at most half of the SMs is cut into half tiles worth ~0.75 of a wave.
     // Fitted to both kernels timed at 2048^3 .. 4096^3 (steps of 256), 2048 x 4096 x 4096 and 3072 x 2048 x 8192.
     const int64_t nkb = (g.K + BK - 1) / BK;
