@@ -437,7 +437,9 @@ klineage_status_t klineage_gemm_run_host(klineage_gemm_t h, int64_t M, int64_t N
  *   tail_n     CTA-pair kernel only: tile_n = every tile of that width; a smaller multiple of 64 = tile rows
  *              start with tile_n-wide tiles and end with tiles of this width, dealt to the CTA pairs back and
  *              forth so that wide and narrow turns balance a last, under-filled wave
- *   stages     single-CTA kernel only: depth of the operand ring - 4; 6 with 128- or 64-column tiles; 8 with 64-column tiles
+ *   stages     single-CTA kernel only: depth of the operand ring in 64-deep k-blocks - 4; 6 with 128- or 64-column
+ *              tiles; 8 with 64-column tiles.  Without a K split, 6 stages of 128-column tiles and 8 stages of
+ *              64-column tiles are filled and freed two k-blocks at a time (3 / 4 stages of 128 k)
  * Every plan computes the same C up to fp32 summation order (plans that differ
  * only in kernel / group_m / half_tail / tile shape / stages are bit-identical; K
  * splits change the order of the partial sums and stay within the parity bound).

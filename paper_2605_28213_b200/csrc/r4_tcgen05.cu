@@ -141,6 +141,7 @@ struct R4Params {
     // Tile width and ring depth (MODE 0, TMA-fed, regular orientation; every other form runs 256 columns and 4
     // stages): 256 columns with four 48 KiB stages, or 128 / 64 columns with four or six 32 / 24 KiB stages.
     int tile_n;
+    int kpair;              // 1: a stage holds TWO 64-deep k-blocks (one barrier round trip per eight MMAs); nkb counts such pairs
     int n_stages;
     uint32_t stage_bytes;
 };
@@ -285,6 +286,11 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     const uint32_t NS = kTunable ? static_cast<uint32_t>(p.n_stages) : static_cast<uint32_t>(STAGES);
     const uint32_t SB = kTunable ? p.stage_bytes : static_cast<uint32_t>(kStageBytes);
     const int TN = kTunable ? p.tile_n : BN;
+    // Narrow tiles may pair their k-blocks: a stage is two sub-stages of the usual layout, 64 k each, filled and freed
+    // together.  The issuing thread spends ~350 clocks per barrier round trip (probe, commit, descriptor step) on top
+    // of ~85 per MMA; with eight MMAs per round trip instead of four a k-block of 64 costs ~515 clocks instead of ~690.
+    const int NSUB = (kTunable && p.kpair) ? 2 : 1;
+    const uint32_t SUB = SB / static_cast<uint32_t>(NSUB);          // bytes of a sub-stage
     // (Measured: a tcgen05.mma of this kernel issues every ~159 clocks whatever its N - 64, 128 or 256 - and
     // whether or not consecutive ones share an accumulator: letting a narrow tile's k-steps alternate between
     // two or four accumulators, summed by the epilogue, left the main loop at 636 clocks per k-block and only made
@@ -360,12 +366,15 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             ptx::tma_load_2d(dst, map, c0, c1, bar);
     };
     // The expect-tx arrive and the loads of one stage: k-block kb of the tile at (m0, n0) of the producer's unit.
-    auto stage_loads = [&](uint32_t s, int kb, int m0, int n0) {
-        uint8_t* sa = smem + s * SB;
-        uint8_t* sb = sa + kABytes;
+    auto stage_loads = [&](uint32_t s, int kb_stage, int m0, int n0) {
         ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
         const CUtensorMap* pa = (MODE == 2) ? prod.ma : &map_a;
         const CUtensorMap* pb = (MODE == 2) ? prod.mb : &map_b;
+        for (int h = 0; h < NSUB; ++h) {
+        // (a sub-stage past the end of K reads zeros: out-of-range boxes are filled, and its MMAs add nothing)
+        const int kb = kb_stage * NSUB + h;
+        uint8_t* sa = smem + s * SB + h * SUB;
+        uint8_t* sb = sa + kABytes;
         if (MODE == 4) {
             // Conv2d: k-block = (filter tap, 64-channel group); the A stage is ONE box of 64 channels
             // x 16 x 8 pixels (the tile's output patch shifted by the tap) - where it leaves the
@@ -389,6 +398,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
 #pragma unroll
             for (int cb = 0; cb < BN / 64; ++cb)
                 if (cb * 64 < TN) load_box(sb + cb * (64 * BK * 2), pb, n0 + cb * 64, kb * BK, &full[s]);
+        }
         }
     };
     // Issues loads until `limit` k-blocks have been issued in total or the schedule ends.
@@ -776,27 +786,29 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     if (t == 0 && kb == kb1 - 1) KLIN_T(10);
                     if (t == 0 && kb == kb0 + 8) KLIN_T(27);
                     if (t == 0 && kb == kb0 + 9) KLIN_T(30);
-                    const uint32_t a_lo = a_lo0 + s * stage_step, b_lo = b_lo0 + s * stage_step;
+                    for (int h = 0; h < NSUB; ++h) {
+                    const uint32_t a_lo = a_lo0 + s * stage_step + h * (SUB >> 4), b_lo = b_lo0 + s * stage_step + h * (SUB >> 4);
 #pragma unroll
                     for (int k4 = 0; k4 < BK / 16; ++k4) {
 #ifdef KLIN_TRACE
                         if (k4 >= trace_knob) continue;
 #endif
                         // K-major operand: +32 bytes per 16 k inside the 128-byte swizzle row.
-                        const uint32_t acc = (kb > kb0 || k4 > 0) ? 1u : 0u;
+                        const uint32_t acc = (kb > kb0 || k4 > 0 || h > 0) ? 1u : 0u;
                         const uint64_t a_desc = (static_cast<uint64_t>(a_hi) << 32) | (a_lo + 2u * k4);
                         if (SWAP) {
                             // weights are the 128-row operand (two halves of the tile's 256 columns,
                             // 16 KiB apart in the stage), activations the N operand
 #pragma unroll
-                            for (int h = 0; h < 2; ++h)
-                                ptx::umma_f16(d_tmem + h * 128,
-                                              (static_cast<uint64_t>(b_hi) << 32) | (b_lo + h * (16384u >> 4) + k4 * kstep),
+                            for (int hh = 0; hh < 2; ++hh)
+                                ptx::umma_f16(d_tmem + hh * 128,
+                                              (static_cast<uint64_t>(b_hi) << 32) | (b_lo + hh * (16384u >> 4) + k4 * kstep),
                                               a_desc, idesc, acc);
                         } else {
                             ptx::umma_f16(d_tmem, a_desc, (static_cast<uint64_t>(b_hi) << 32) | (b_lo + k4 * kstep), idesc,
                                           acc);
                         }
+                    }
                     }
                     ptx::umma_commit_addr(empty0 + 8 * s);
                     if (t == 0 && kb == kb0 + 8) KLIN_T(28);
@@ -1993,13 +2005,15 @@ bool plan_launch(const GemmArgs& g, const RunContext& ctx, bool generic, bool mu
         take_narrow = narrow.split.cost < wide.split.cost;
     else
         take_narrow = narrow.split.splits > 1 || tiles256 * 2 <= ctx.sm_count;
-    if (take_narrow && narrow.split.cluster) narrow.stages = 6;
+    // the deepest ring: six real stages for a cluster split; unsplit, three stages of two k-blocks each (one barrier round
+    // trip per eight MMAs: 1024^3 9.1 -> 8.4 us, 1536^3 13.2 -> 11.5 in graph replay)
+    if (take_narrow && (narrow.split.cluster || narrow.split.splits == 1)) narrow.stages = 6;
     if (take_narrow && narrow.split.splits == 1 && g.N > BN / 4) {
         // still at most half a wave of 128-column tiles: 64 columns (measured 0.4 - 0.5 us off a 5 - 7 us launch at
         // 256^3, 512^3 and 300 x 520 x 200: an MMA takes as long whatever its width, the epilogue of a tile shrinks)
         const int64_t tiles128 = tiles_m * ((g.N + BN / 2 - 1) / (BN / 2));
         LaunchPlan tiny;
-        if (tiles128 * 2 <= ctx.sm_count && try_shape(BN / 4, STAGES, &tiny) && tiny.split.splits == 1) narrow = tiny;
+        if (tiles128 * 2 <= ctx.sm_count && try_shape(BN / 4, 8, &tiny) && tiny.split.splits == 1) narrow = tiny;
     }
     *out = take_narrow ? narrow : wide;
     return true;
@@ -2086,9 +2100,17 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     p.tile_n = shape.tile_n;
     p.n_stages = shape.stages;
     p.stage_bytes = static_cast<uint32_t>(kABytes + shape.tile_n * BK * 2);
+    // Unsplit narrow tiles on their deepest ring pair their k-blocks: 8 x 24 KiB -> 4 stages of two, 6 x 32 KiB -> 3
+    const bool kpair = !generic && md == nullptr && !shape.split.swap && shape.split.splits == 1 &&
+                       ((shape.tile_n == BN / 4 && shape.stages == 8) || (shape.tile_n == BN / 2 && shape.stages == 6));
+    if (kpair) {
+        p.kpair = 1;
+        p.n_stages = shape.stages / 2;
+        p.stage_bytes *= 2;
+    }
     p.tiles_m = static_cast<int>(tiles_m);
     p.tiles_n = static_cast<int>(tiles_n);
-    p.nkb = (g.K + BK - 1) / BK;
+    p.nkb = kpair ? (g.K + 2 * BK - 1) / (2 * BK) : (g.K + BK - 1) / BK;
     p.ldw = (static_cast<int64_t>(g.N) + 3) & ~int64_t(3);
     const SplitPlan plan = shape.split;
     p.splits = plan.splits;
@@ -2164,7 +2186,7 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     }
     // Skinny mode fetches only the activation rows the MMA reads (n_mma of them).
     const uint32_t a_box_rows = swap ? static_cast<uint32_t>(p.n_mma) : BM;
-    p.stage_tx = a_box_rows * BK * 2 + static_cast<uint32_t>(shape.tile_n) * BK * 2;
+    p.stage_tx = (a_box_rows * BK * 2 + static_cast<uint32_t>(shape.tile_n) * BK * 2) * (p.kpair ? 2u : 1u);
     if (!generic) {
         ok = encode_map_2d(ctx, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.A, g.K, g.M, g.lda * 2, BK, a_box_rows,
                            CU_TENSOR_MAP_SWIZZLE_128B);
