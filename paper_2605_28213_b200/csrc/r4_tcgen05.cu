@@ -1719,14 +1719,14 @@ int choose_cluster_splits(int64_t tiles, int nkb, int sm)
 
 // 128-row tiles split inside a cluster: what the two cluster barriers, the exchange of the partial tile through
 // the operand rings and the owner's reduce cost, in k-block times (0.31 us), measured in CUDA-graph replay on
-// products of 1 .. 64 tiles: 4.0 / 5.0 / 6.6 us for 2 / 4 / 8 CTAs, about 2 us more when the launch fills
-// most of the GPU.  A launch never exceeds one wave of clusters: a CTA runs exactly one unit, and a second
+// products of 1 .. 64 tiles: 4.0 / 5.0 / 6.6 us for 2 / 4 / 8 CTAs, about 4 us more when the launch fills
+// most of the GPU (768 x 768 x 3072: 72 CTAs in pairs 12.3 us, 144 CTAs in fours 14.4 us).  A launch never exceeds one wave of clusters: a CTA runs exactly one unit, and a second
 // wave would pay the kernel's set-up again (measured: 2048^3 in 4 splits 54 us against 17 us unsplit).
 int cluster_fixed_cost(int s, int64_t ctas, int sm, int tile_n)
 {
     // (128-column tiles exchange half as much: 1.7 / 2.0 / 2.5 us less)
     const int base = tile_n == BN ? (s == 2 ? 13 : s == 4 ? 16 : 22) : (s == 2 ? 8 : s == 4 ? 10 : 14);
-    return base + (ctas * 3 > static_cast<int64_t>(sm) * 2 ? 6 : 0);
+    return base + (ctas * 3 > static_cast<int64_t>(sm) * 2 ? 12 : 0);
 }
 // Clusters of `s` CTAs of this kernel that the device can hold at once (GPC boundaries make this less than
 // SMs / s for large clusters); asked of the runtime once per size and device.
@@ -1737,12 +1737,14 @@ int max_resident_clusters(int s, const RunContext& ctx);
 int choose_regular_cluster_splits(int64_t tiles, int nkb, const RunContext& ctx, int tile_n, int64_t* cost_out)
 {
     int best = 1;
-    int64_t best_cost = ((tiles + ctx.sm_count - 1) / ctx.sm_count) * static_cast<int64_t>(nkb);
+    // costs in fifths of a k-block time; a k-block of a narrow tile (paired k-blocks) takes about 0.8 of a wide one's
+    const int64_t kb_cost = tile_n == BN ? 5 : 4;
+    int64_t best_cost = ((tiles + ctx.sm_count - 1) / ctx.sm_count) * static_cast<int64_t>(nkb) * kb_cost;
     for (int s = 2; s <= 8 && s * 2 <= nkb; s *= 2) {
         const int per = (nkb + s - 1) / s;
         if ((nkb + per - 1) / per != s) continue;
         if (tiles > max_resident_clusters(s, ctx)) continue;
-        const int64_t cost = per + cluster_fixed_cost(s, tiles * s, ctx.sm_count, tile_n);
+        const int64_t cost = per * kb_cost + 5 * cluster_fixed_cost(s, tiles * s, ctx.sm_count, tile_n);
         if (cost < best_cost) {
             best_cost = cost;
             best = s;
@@ -1781,8 +1783,9 @@ SplitPlan plan_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContex
         // 128-row tiles: the cluster route against the workspace route chosen above and against no split
         const int sm = ctx.sm_count;
         const int per_w = (nkb + sp.splits - 1) / sp.splits;
-        sp.cost = sp.splits > 1 ? ((tiles * sp.splits + sm - 1) / sm) * static_cast<int64_t>(per_w + 30 + 6 * sp.splits)
-                                : ((tiles + sm - 1) / sm) * static_cast<int64_t>(nkb);
+        // (in fifths of a k-block time, like the cluster route's estimate)
+        sp.cost = sp.splits > 1 ? ((tiles * sp.splits + sm - 1) / sm) * static_cast<int64_t>(per_w + 30 + 6 * sp.splits) * 5
+                                : ((tiles + sm - 1) / sm) * static_cast<int64_t>(nkb) * (tile_n == BN ? 5 : 4);
         int64_t cost_c = 0;
         const int sc = choose_regular_cluster_splits(tiles, nkb, ctx, tile_n, &cost_c);
         if (sc > 1 && cost_c <= sp.cost) {
@@ -2101,7 +2104,11 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     p.n_stages = shape.stages;
     p.stage_bytes = static_cast<uint32_t>(kABytes + shape.tile_n * BK * 2);
     // Unsplit narrow tiles on their deepest ring pair their k-blocks: 8 x 24 KiB -> 4 stages of two, 6 x 32 KiB -> 3
-    const bool kpair = !generic && md == nullptr && !shape.split.swap && shape.split.splits == 1 &&
+    // (with a cluster split only if every split still gets work when K is counted in pairs of k-blocks)
+    const int nkb_pairs = (g.K + 2 * BK - 1) / (2 * BK);
+    const int per_pairs = (nkb_pairs + shape.split.splits - 1) / shape.split.splits;
+    const bool pairs_split_evenly = shape.split.splits == 1 || (shape.split.cluster && (nkb_pairs + per_pairs - 1) / per_pairs == shape.split.splits);
+    const bool kpair = !generic && md == nullptr && !shape.split.swap && pairs_split_evenly &&
                        ((shape.tile_n == BN / 4 && shape.stages == 8) || (shape.tile_n == BN / 2 && shape.stages == 6));
     if (kpair) {
         p.kpair = 1;

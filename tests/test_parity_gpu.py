@@ -468,3 +468,25 @@ def test_error_codes(handles, kb):
         kb.klineage_gemm_create(999, 0, 0)
     dev.run(g, 4)
     dev.result()
+
+
+# ------------------------------------------------------------------ paired k-blocks of narrow tiles
+# (kernel, splits, split_via, group_m, half_tail, tile_n, tail_n, stages): 64 columns x 8 stages and 128 columns x 6
+# stages run two 64-deep k-blocks per stage.  K below: one k-block (the stage's second half lies wholly past K), an odd
+# number of k-blocks, a ragged last k-block, many pairs; with a cluster split, K ranges counted in pairs.
+PAIRED_K = [((1, 1, 0, 0, 0, 64, 0, 8), 40), ((1, 1, 0, 0, 0, 64, 0, 8), 200), ((1, 1, 0, 0, 0, 64, 0, 8), 328),
+            ((1, 1, 0, 0, 0, 128, 0, 6), 64), ((1, 1, 0, 0, 0, 128, 0, 6), 456), ((1, 1, 0, 0, 0, 128, 0, 6), 1096),
+            ((1, 2, 2, 0, 0, 128, 0, 6), 1096), ((1, 4, 2, 0, 0, 128, 0, 6), 2056)]
+
+
+@pytest.mark.parametrize("col", [False, True], ids=["Brow", "Bcol"])
+@pytest.mark.parametrize("pin,K", PAIRED_K, ids=lambda v: "x".join(map(str, v)) if isinstance(v, tuple) else f"K{v}")
+def test_tcgen05_paired_k_blocks(handles, pin, K, col):
+    for bf in (False, True):
+        case = gen.make_case(300, 264, K, seed=77, dist_a="integer", dist_b="integer", b_col_major=col, c_bf16=bf,
+                             name=f"paired {pin} K={K}")
+        run_and_check(handles, case, 4, exact=True, pin=pin)
+        g = handles[(col, bf)]
+        flags = g.last_kernel_id() - 400
+        assert flags >= 0 and not (flags & 32), "the single-CTA kernel must have run"
+        assert bool(flags & 16) == (pin[1] > 1), "cluster split exactly when the plan asks for one"
