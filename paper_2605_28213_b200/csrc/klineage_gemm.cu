@@ -651,7 +651,7 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups, const
         if (!ga) return KLINEAGE_ERR_ALLOC;
         int n = 0, first = -1;
         bool launchable = true, all_tall = true, all_long = true;
-        int64_t pair_tiles = 0, single_tiles = 0;
+        int64_t pair_tiles = 0, single_tiles = 0, rows = 0, rows_by_256 = 0;
         for (int i = 0; i < groups; ++i) {
             if (M[i] == 0 || N[i] == 0) continue;
             if (K[i] == 0) {            // a zero-fill group: leave the whole call to the ordinary path
@@ -660,6 +660,9 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups, const
             }
             if (first < 0) first = i;
             ga[n++] = make_args(h, M[i], N[i], K[i], A[i], lda[i], B[i], ldb[i], nullptr, C[i], ldc[i]);
+            // (a pair tile with at most 256 live rows issues half of its MMAs: rows count in steps of 256)
+            rows += M[i];
+            rows_by_256 += (M[i] + 255) / 256 * 256;
             all_tall = all_tall && M[i] > 256;
             all_long = all_long && K[i] >= 1024;
             pair_tiles += ((M[i] + 511) / 512) * ((N[i] + 255) / 256);
@@ -668,7 +671,10 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups, const
         launchable = launchable && n >= 1 && n <= kMaxGroups;
         // kernel choice as for the batched call; a plan pinned for the first group's shape may name it
         const int half_sm = h->ctx.sm_count / 2;
-        const bool pair_ok = launchable && all_tall && pair_tiles >= half_sm && r4_pair_grouped_possible(ga, n, h->ctx);
+        // by default the pair kernel when every group has more than 256 rows, or - ragged groups - when rounding every
+        // group up to 256 rows adds at most a quarter (a pinned plan may ask for it whatever the groups' heights)
+        all_tall = all_tall || rows_by_256 * 4 <= rows * 5;
+        const bool pair_ok = launchable && pair_tiles >= half_sm && r4_pair_grouped_possible(ga, n, h->ctx);
         const bool single_ok = launchable && single_tiles >= half_sm && r4_single_grouped_possible(ga, n, h->ctx);
         R4Plan pinned;
         if (first >= 0) {
@@ -681,7 +687,7 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups, const
             want = 2;
         else if (pinned.kernel == 1 && single_ok)
             want = 1;
-        else if (pair_ok && all_long)
+        else if (pair_ok && all_long && all_tall)
             want = 2;
         else if (single_ok)
             want = 1;

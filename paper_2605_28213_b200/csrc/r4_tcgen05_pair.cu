@@ -514,6 +514,10 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 const int kb_first = wk.kb0, kb_end = wk.kb1 < 0 ? x.nkb : wk.kb1;
                 // the MMA's N is the tile's width
                 const uint32_t idesc = (p.idesc & ~(0x3Fu << 17)) | (static_cast<uint32_t>(x.width >> 3) << 17);
+                // A tile whose second row block lies wholly past the matrix (at most 256 live rows) issues the first
+                // block's MMAs only: this thread's instruction stream bounds the loop, so such a tile takes about
+                // half the time (its second accumulator is never read: the epilogue warps of that block have no rows).
+                const bool two_blocks = x.M - x.m0 > 2 * PM;
                 // Both accumulators are rewritten: wait until both CTAs' epilogues drained the last tile.
                 if (!ptx::mbar_wait(&acc_empty[0], (tcount & 1) ^ 1, abort_flag)) {
                     report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x520u);
@@ -545,8 +549,9 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                         // alternate the two row blocks: consecutive MMAs never share an accumulator
                         const uint64_t bd = desc(b_hi, b_lo + static_cast<uint32_t>(k4) * kstep);
                         umma_f16_pair(tmem_base, desc(a_hi, a_lo + static_cast<uint32_t>(k4 * 2)), bd, idesc, acc);
-                        umma_f16_pair(tmem_base + PN, desc(a_hi, a_lo + static_cast<uint32_t>((kABlockBytes >> 4) + k4 * 2)),
-                                      bd, idesc, acc);
+                        if (two_blocks)
+                            umma_f16_pair(tmem_base + PN, desc(a_hi, a_lo + static_cast<uint32_t>((kABlockBytes >> 4) + k4 * 2)),
+                                          bd, idesc, acc);
                     }
                     umma_commit_pair(empty0 + 8 * s);
                     umma_commit_pair(empty_odd0 + 8 * s);
