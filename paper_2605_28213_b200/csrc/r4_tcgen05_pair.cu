@@ -1078,8 +1078,46 @@ cudaError_t launch_r4_pair_grouped(const GemmArgs* groups, int n, RunContext& ct
 {
     if (!r4_pair_grouped_possible(groups, n, ctx)) return cudaErrorInvalidValue;
     static_assert(sizeof(GroupEntry) % 128 == 0, "table entries keep their tensor maps 128-byte aligned");
+    // Ragged groups: a tile row with at most 256 live rows costs about half a tile (its second row block issues no
+    // MMAs).  Such a last tile row becomes a table entry of its own (the group's A and C from that row on), all of
+    // them go to the END of the schedule, and odd rounds run over the pairs in reverse: the pairs that got a full
+    // tile in the last full round get the half tiles last.  (Dealt round-robin in group order, a G = 8 launch of
+    // 320 tiles kept some pairs busy for 5 tiles' time where 4 suffice.)
+    GemmArgs* ents = new (std::nothrow) GemmArgs[2 * n];
+    if (!ents) return cudaErrorMemoryAllocation;
+    int n_full = 0, n_half = 0;
+    GemmArgs* halves = ents + n;
+    for (int i = 0; i < n; ++i) {
+        const GemmArgs& g = groups[i];
+        const int rem = g.M % TILE_M;
+        if (rem == 0 || rem > 2 * PM) {
+            ents[n_full++] = g;
+            continue;
+        }
+        GemmArgs h = g;                       // the last (or only) tile row
+        const int64_t off = g.M - rem;
+        h.A = g.A + off * g.lda;
+        h.C = static_cast<uint8_t*>(g.C) + off * g.ldc * (g.c_bf16 ? 2 : 4);
+        h.M = rem;
+        halves[n_half++] = h;
+        if (off > 0) {
+            GemmArgs f = g;
+            f.M = static_cast<int>(off);
+            ents[n_full++] = f;
+        }
+    }
+    const bool reorder = n_half > 0 && n_full > 0 && n_full + n_half <= kMaxGroups &&
+                         ctx.workspace_bytes >= static_cast<size_t>(n_full + n_half) * sizeof(GroupEntry);
+    if (reorder) {
+        for (int i = 0; i < n_half; ++i) ents[n_full + i] = halves[i];
+        n = n_full + n_half;
+        groups = ents;
+    }
     GroupEntry* table = new (std::nothrow) GroupEntry[n];
-    if (!table) return cudaErrorMemoryAllocation;
+    if (!table) {
+        delete[] ents;
+        return cudaErrorMemoryAllocation;
+    }
     memset(table, 0, sizeof(GroupEntry) * n);
     PairParams p;
     memset(&p, 0, sizeof p);
@@ -1121,10 +1159,13 @@ cudaError_t launch_r4_pair_grouped(const GemmArgs* groups, int n, RunContext& ct
     if (err == cudaSuccess)
         err = cudaMemcpyAsync(ctx.workspace, table, sizeof(GroupEntry) * n, cudaMemcpyHostToDevice, stream);
     delete[] table;
+    const GemmArgs g0 = groups[0];
+    delete[] ents;
     if (err != cudaSuccess) return err;
     p.groups = static_cast<const GroupEntry*>(ctx.workspace);
     p.n_groups = n;
     p.total_tiles = tile_start;
+    p.snake = reorder ? 1 : 0;
     p.stage_tx = 2 * kStageBytes;
     p.b_boxes = 2;
     p.epi_tma = any_tma ? 1 : 0;
@@ -1134,7 +1175,6 @@ cudaError_t launch_r4_pair_grouped(const GemmArgs* groups, int n, RunContext& ct
     const unsigned grid = 2u * static_cast<unsigned>(p.total_tiles < max_pairs ? p.total_tiles : max_pairs);
     CUtensorMap none;
     memset(&none, 0, sizeof none);
-    const GemmArgs& g0 = groups[0];
     return g0.b_col ? launch<true, 2>(g0, none, none, none, p, grid, ctx.device, stream)
                     : launch<false, 2>(g0, none, none, none, p, grid, ctx.device, stream);
 }

@@ -276,3 +276,16 @@ def test_grouped_argument_rules(kb):
         vals, bits = d.result()
         C_ref, S = P.oracle_rows(c, np.arange(c.M))
         P.assert_matches_oracle(c, vals, bits, C_ref, S, exact=True, what=c.name)
+
+
+def test_grouped_ragged_rows_on_the_pair_kernel(kb):
+    """Groups whose last tile row has at most 256 live rows: those tile rows become table entries of their own at the
+    end of the schedule (their second row block issues no MMAs) - the result must not notice.  Heights: a multiple of
+    512, at most 256 in all, exactly 256 and 257 over a multiple, one row over."""
+    shapes = [(1024, 1304, 200), (64, 2048, 136), (256, 520, 72), (768, 1528, 328), (769, 1024, 64), (513, 2000, 264),
+              (1536, 2048, 72), (1200, 776, 136), (2, 304, 520)]       # 97 pair tiles: at least one per CTA pair
+    for col, bf in ((False, True), (True, False)):
+        cases = [gen.make_case(M, N, K, seed=170 + i, dist_a="integer", dist_b="integer", b_col_major=col, c_bf16=bf,
+                               ldc=N + (8 if i % 3 == 0 else 0), name=f"gr{i}-{M}x{N}x{K}")
+                 for i, (M, N, K) in enumerate(shapes)]
+        run_grouped(kb, cases, 4, True, want_pair=True, one_launch=True, kernel=2)
