@@ -244,6 +244,15 @@ __device__ __forceinline__ void st_cluster_v4_f32(uint32_t cluster_addr, float a
     asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "f"(a), "f"(b), "f"(c), "f"(d)
                  : "memory");
 }
+// The same store, asynchronous: its 16 bytes are counted (complete_tx) on an mbarrier of the destination CTA when
+// they have landed, so the receiver waits for exactly its data and no cluster-wide barrier is needed.
+__device__ __forceinline__ void st_async_v4_f32(uint32_t cluster_addr, float a, float b, float c, float d, uint32_t cluster_mbar)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(
+                     cluster_addr),
+                 "f"(a), "f"(b), "f"(c), "f"(d), "r"(cluster_mbar)
+                 : "memory");
+}
 // Cluster-wide barrier, split in two; every thread of every CTA of the cluster
 // executes both.  (A hardware barrier: it completes because every loop that
 // precedes it in these kernels is bounded.)

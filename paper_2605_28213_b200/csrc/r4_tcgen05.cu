@@ -323,8 +323,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // Cluster mode: no CTA may touch a peer's shared memory before that peer runs.
-    if (SWAP && p.cluster) ptx::cluster_arrive_relaxed();
+    // Cluster mode: no CTA may touch a peer's shared memory before that peer runs and has initialised the barrier
+    // its incoming partial sums are counted on (warp 0 arrives after it has done that, below).
+    if (SWAP && p.cluster && warp != 0) ptx::cluster_arrive_relaxed();
+    uint64_t* xchg_bar = cfull;      // skinny cluster mode only (the six-stage ring's barriers are another mode's)
     const int64_t total_units = p.total_units;
 
     // TMA producer state (used by warp 0, lane 0 only): position in the static schedule.
@@ -490,6 +492,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 for (int i = 0; i < 2 * kConvStages; ++i) ptx::mbar_init(&cfull[i], 1);
             abort_flag[0] = 0;
             abort_flag[1] = 0;
+            if (SWAP && p.cluster) ptx::mbar_init(xchg_bar, 1);
             ptx::fence_barrier_init();
             if (!GENERIC && MODE != 2) {
                 ptx::prefetch_tensormap(&map_a);
@@ -497,6 +500,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             }
             if (p.epi_tma && MODE != 2 && MODE != 3) ptx::prefetch_tensormap(&map_c);
             KLIN_T(1);
+        }
+        if (SWAP && p.cluster) {
+            __syncwarp();
+            ptx::cluster_arrive_relaxed();
         }
         if (kEarlyProducer) {
             __syncwarp();
@@ -822,6 +829,16 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         }
     } else if (warp < 6) {
         // ------------------------------------------------------------ epilogue
+        if (SWAP && p.cluster && warp == 2 && lane == 0) {
+            // what this CTA will receive: every source's partial of each block it owns that lies inside the matrix
+            const int nblk = 8 >> p.splits_log2;
+            uint32_t blocks = 0;
+            for (int bl = 0; bl < nblk; ++bl) {
+                const int bi = (bl << p.splits_log2) + fin_rank;
+                if (fin_n0 + (bi >> 2) * 128 + (bi & 3) * 32 < g.N) ++blocks;
+            }
+            ptx::mbar_arrive_expect_tx(xchg_bar, blocks * static_cast<uint32_t>(p.splits) * static_cast<uint32_t>(p.n_mma) * 128u);
+        }
         const int q = warp & 3;                              // TMEM lane quarter this warp may read
         uint8_t* stg = epi_smem + (warp - 2) * 2 * kEpiBufBytes;
         uint32_t t = 0;
@@ -855,7 +872,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     for (int mc = 0; mc < p.n_mma; mc += 16) {
                         uint32_t v[16];
                         ptx::tmem_ld_32x32b_x16(tmem_base + buf * BN + h * 128 + mc + (static_cast<uint32_t>(q * 32) << 16), v);
-                        uint32_t remote = 0;
+                        uint32_t remote = 0, remote_bar = 0;
                         if (p.cluster) {
                             // block (h, q) of the tile belongs to CTA (block % splits); this CTA's
                             // partial goes to slot [split][block / splits] of the owner, laid out
@@ -867,13 +884,16 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                             float* slot = reinterpret_cast<float*>(epi_smem) +
                                           ((split * nblk + (bi >> p.splits_log2)) * p.n_mma + mc) * 32 + lane * 4;
                             remote = ptx::map_to_cta(ptx::smem_u32(slot), owner);
+                            remote_bar = ptx::map_to_cta(ptx::smem_u32(xchg_bar), owner);
                         }
                         ptx::tmem_ld_wait();
                         if (p.cluster) {
+                            // asynchronous stores counted on the owner's barrier: the owner waits for its bytes, no
+                            // cluster-wide barrier stands between the last MMA and the reduce
 #pragma unroll
                             for (int j = 0; j < 16; j += 4)
-                                ptx::st_cluster_v4_f32(remote + j * 128, __uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                       __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                                ptx::st_async_v4_f32(remote + j * 128, __uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                     __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]), remote_bar);
                         } else if (n < g.N) {
                             const float bn = partial ? 0.f : bias_at(g, n);
 #pragma unroll
@@ -1597,11 +1617,17 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     }
 
     if (SWAP && p.cluster) {
-        // Every thread of every CTA of the cluster arrives; after the wait all partial
-        // blocks sent to this CTA are visible in its shared memory.
-        ptx::cluster_arrive_release();
-        ptx::cluster_wait_acquire();
-        if (warp >= 2 && warp < 6 && !abort_flag[0]) {
+        // The owner waits until every byte sent to it has landed: (splits) sources x its blocks inside the matrix
+        // x n_mma rows x 128 bytes, announced on its barrier by one thread at the start of the epilogue role.
+        bool got = true;
+        if (warp >= 2 && warp < 6) {
+            got = ptx::mbar_wait(xchg_bar, 0, abort_flag);
+            if (!got) {
+                if (lane == 0) report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x480u);
+                abort_flag[0] = 1;
+            }
+        }
+        if (warp >= 2 && warp < 6 && got && !abort_flag[0]) {
             // This CTA owns blocks bi = bl * splits + rank of the tile; slot (src * nblk + bl) holds
             // CTA src's partial of local block bl as [m / 4][lane][m % 4].  A warp takes four
             // consecutive rows (one 16-byte load per source); all of a block's loads are issued
@@ -1634,6 +1660,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 }
             }
         }
+        // No CTA leaves while a peer could still send into its shared memory (on the ordinary path every byte has
+        // been counted by now; a peer that gave up sends nothing more after it arrives here).  Execution only.
+        ptx::cluster_arrive_relaxed();
+        ptx::cluster_wait_acquire();
     }
 
     if (warp == 2 && lane == 0) KLIN_T(14);
