@@ -94,21 +94,6 @@ __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t threads
     asm volatile("barrier.cta.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
-// One non-blocking look at a barrier's phase (mbarrier.test_wait never suspends the thread): role loops probe the
-// NEXT stage's barrier before they issue the current stage's work, so that the answer is there when they need it.
-__device__ __forceinline__ uint32_t mbar_test_addr(uint32_t bar_addr, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar_addr), "r"(parity)
-        : "memory");
-    return ok;
-}
-
 // ------------------------------------------------------------------- fences
 // Orders generic-proxy shared-memory writes before async-proxy reads (TMA
 // store, tcgen05.mma operand fetch).
@@ -148,6 +133,14 @@ __device__ __forceinline__ void tma_load_4d(void* smem_dst, const void* tmap, in
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(c3),
         "r"(smem_u32(bar))
         : "memory");
+}
+// Untiled bulk copy global -> shared (both addresses 16-byte aligned, the size a multiple of 16), completion counted
+// in bytes on `bar`; no multicast.
+__device__ __forceinline__ void bulk_load_1d(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar_addr)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_dst),
+                 "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(bar_addr)
+                 : "memory");
 }
 // The same loads and the expect-tx arrive with shared-window addresses (lean producer loops).
 __device__ __forceinline__ void mbar_arrive_expect_tx_addr(uint32_t bar_addr, uint32_t bytes)

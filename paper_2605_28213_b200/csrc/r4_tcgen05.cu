@@ -372,35 +372,40 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         ptx::mbar_arrive_expect_tx(&full[s], p.stage_tx);
         const CUtensorMap* pa = (MODE == 2) ? prod.ma : &map_a;
         const CUtensorMap* pb = (MODE == 2) ? prod.mb : &map_b;
-        for (int h = 0; h < NSUB; ++h) {
-        // (a sub-stage past the end of K reads zeros: out-of-range boxes are filled, and its MMAs add nothing)
-        const int kb = kb_stage * NSUB + h;
-        uint8_t* sa = smem + s * SB + h * SUB;
-        uint8_t* sb = sa + kABytes;
-        if (MODE == 4) {
-            // Conv2d: k-block = (filter tap, 64-channel group); the A stage is ONE box of 64 channels
-            // x 16 x 8 pixels (the tile's output patch shifted by the tap) - where it leaves the
-            // image the TMA unit fills zeros, which is the padding.  GEMM row = 16 * patch row + column.
-            const int cpb = p.conv.C >> 6;
-            const int tap = kb / cpb, cg = kb - tap * cpb;
-            const int fr = tap / p.conv.S, fs = tap - fr * p.conv.S;
-            ptx::tma_load_4d(sa, &map_a, cg * 64, prod.cw + fs, prod.ch + fr, prod.cn, &full[s]);
-        } else
-            load_box(sa, pa, kb * BK, m0, &full[s]);
-        if (BCOL) {
-            load_box(sb, pb, kb * BK, n0, &full[s]);
-        } else if (MODE == 1 && p.b_box3d) {
-            ptx::tma_load_4d(sb, pb, 0, kb * BK, n0 >> 6, prod.z, &full[s]);   // the same box, batch as 4th coordinate
-        } else if ((MODE == 0 || MODE == 3) && p.b_box3d) {
-            // B viewed as (64 columns, K rows, N / 64 column blocks): one box of 64 x 64 x 4 lands as the
-            // four consecutive 8 KiB blocks the MN-major descriptor expects - one TMA instruction, not four
-            // (a producer thread issues a TMA instruction every ~110 cycles)
-            ptx::tma_load_3d(sb, pb, 0, kb * BK, n0 >> 6, &full[s]);
-        } else {
+        // the loads of one 64-deep (sub-)stage: k-block kb into the sub-stage at sa
+        auto sub_loads = [&](int kb, uint8_t* sa) {
+            uint8_t* sb = sa + kABytes;
+            if (MODE == 4) {
+                // Conv2d: k-block = (filter tap, 64-channel group); the A stage is ONE box of 64 channels
+                // x 16 x 8 pixels (the tile's output patch shifted by the tap) - where it leaves the
+                // image the TMA unit fills zeros, which is the padding.  GEMM row = 16 * patch row + column.
+                const int cpb = p.conv.C >> 6;
+                const int tap = kb / cpb, cg = kb - tap * cpb;
+                const int fr = tap / p.conv.S, fs = tap - fr * p.conv.S;
+                ptx::tma_load_4d(sa, &map_a, cg * 64, prod.cw + fs, prod.ch + fr, prod.cn, &full[s]);
+            } else
+                load_box(sa, pa, kb * BK, m0, &full[s]);
+            if (BCOL) {
+                load_box(sb, pb, kb * BK, n0, &full[s]);
+            } else if (MODE == 1 && p.b_box3d) {
+                ptx::tma_load_4d(sb, pb, 0, kb * BK, n0 >> 6, prod.z, &full[s]);   // the same box, batch as 4th coordinate
+            } else if ((MODE == 0 || MODE == 3) && p.b_box3d) {
+                // B viewed as (64 columns, K rows, N / 64 column blocks): one box of 64 x 64 x 4 lands as the
+                // four consecutive 8 KiB blocks the MN-major descriptor expects - one TMA instruction, not four
+                // (a producer thread issues a TMA instruction every ~110 cycles)
+                ptx::tma_load_3d(sb, pb, 0, kb * BK, n0 >> 6, &full[s]);
+            } else {
 #pragma unroll
-            for (int cb = 0; cb < BN / 64; ++cb)
-                if (cb * 64 < TN) load_box(sb + cb * (64 * BK * 2), pb, n0 + cb * 64, kb * BK, &full[s]);
-        }
+                for (int cb = 0; cb < BN / 64; ++cb)
+                    if (cb * 64 < TN) load_box(sb + cb * (64 * BK * 2), pb, n0 + cb * 64, kb * BK, &full[s]);
+            }
+        };
+        if (kTunable && NSUB == 2) {
+            // (a sub-stage past the end of K reads zeros: out-of-range boxes are filled, and its MMAs add nothing)
+            sub_loads(2 * kb_stage, smem + s * SB);
+            sub_loads(2 * kb_stage + 1, smem + s * SB + SUB);
+        } else {
+            sub_loads(kb_stage, smem + s * SB);
         }
     };
     // Issues loads until `limit` k-blocks have been issued in total or the schedule ends.
@@ -439,13 +444,12 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
     auto produce_rest = [&]() {
         uint32_t st = prod.st, ph = prod.ph, it = prod.it;
         const uint32_t empty0 = ptx::smem_u32(empty);
-        uint32_t ready = 0;     // the current stage's "empty" barrier was seen complete by the look-ahead probe
         while (prod.live) {
             const int m0 = prod.m0, n0 = prod.n0, kb1 = prod.kb1;
             for (int kb = prod.kb; kb < kb1; ++kb, ++it) {
                 if (it == 8) KLIN_T(20);
                 if (it == 9) KLIN_T(23);
-                if (!ready && !ptx::mbar_wait_addr(empty0 + 8 * st, ph, abort_flag)) {
+                if (!ptx::mbar_wait_addr(empty0 + 8 * st, ph, abort_flag)) {
                     report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x400u | st);
                     abort_flag[0] = 1;
                     prod.live = false;
@@ -454,7 +458,6 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 if (it == 8) KLIN_T(21);
                 if (it == 9) KLIN_T(24);
                 const uint32_t st_next = (st + 1 == NS) ? 0u : st + 1, ph_next = (st + 1 == NS) ? ph ^ 1u : ph;
-                ready = ptx::mbar_test_addr(empty0 + 8 * st_next, ph_next);
                 stage_loads(st, kb, m0, n0);
                 if (it == 8) KLIN_T(22);
                 if (it == 9) KLIN_T(25);
@@ -747,7 +750,6 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
             // (Measured: the length of this instruction stream does not bound the kernel - trimming it changed no
             // timing, and releasing stages in pairs to halve the commits was slower, because the ring got shallower.)
             uint32_t s = 0, ph = 0;
-            uint32_t ready = 0;     // the current stage's "full" barrier was seen complete by the look-ahead probe
 #ifdef KLIN_TRACE
             const int trace_knob = klin_trace_knob > 0 ? klin_trace_knob : 4;
 #endif
@@ -775,7 +777,7 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (t == 0 && kb == kb0 + 8) KLIN_T(26);
                     if (t == 0 && kb == kb0 + 9) KLIN_T(29);
-                    if (!ready && !ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag, full_limit)) {
+                    if (!ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag, full_limit)) {
                         report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x420u | s);
                         abort_flag[0] = 1;
                         ok = false;
@@ -784,39 +786,42 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     // (TMA-fed operands need no tcgen05 fence here: they were written through the async proxy, which
                     // is also how the MMA reads them.)
                     if (GENERIC) ptx::tc_fence_after_sync();
-                    // The
-                    // next stage's barrier is probed now: a passing wait costs ~250 clocks of latency when it is
-                    // asked for only at the top of the next iteration.
+                    // (A look-ahead probe of the next stage's barrier cost this kernel's long-K launches 6 %, 63.5 -> 67.6 us
+                    // at 2048 x 2048 x 8192, ahead of the MMAs and 3 % behind them: not used.)
                     const uint32_t s_next = (s + 1 == n_stages) ? 0u : s + 1, ph_next = (s + 1 == n_stages) ? ph ^ 1u : ph;
-                    ready = ptx::mbar_test_addr(full0 + 8 * s_next, ph_next);
                     if (t == 0 && kb == kb0) KLIN_T(9);
                     if (t == 0 && kb == kb1 - 1) KLIN_T(10);
                     if (t == 0 && kb == kb0 + 8) KLIN_T(27);
                     if (t == 0 && kb == kb0 + 9) KLIN_T(30);
-                    for (int h = 0; h < NSUB; ++h) {
-                    const uint32_t a_lo = a_lo0 + s * stage_step + h * (SUB >> 4), b_lo = b_lo0 + s * stage_step + h * (SUB >> 4);
+                    // the MMAs of one 64-deep (sub-)stage; `later`: not the unit's first sub-stage
+                    auto issue_sub = [&](uint32_t a_lo, uint32_t b_lo, bool later) {
 #pragma unroll
-                    for (int k4 = 0; k4 < BK / 16; ++k4) {
+                        for (int k4 = 0; k4 < BK / 16; ++k4) {
 #ifdef KLIN_TRACE
-                        if (k4 >= trace_knob) continue;
+                            if (k4 >= trace_knob) continue;
 #endif
-                        // K-major operand: +32 bytes per 16 k inside the 128-byte swizzle row.
-                        const uint32_t acc = (kb > kb0 || k4 > 0 || h > 0) ? 1u : 0u;
-                        const uint64_t a_desc = (static_cast<uint64_t>(a_hi) << 32) | (a_lo + 2u * k4);
-                        if (SWAP) {
-                            // weights are the 128-row operand (two halves of the tile's 256 columns,
-                            // 16 KiB apart in the stage), activations the N operand
+                            // K-major operand: +32 bytes per 16 k inside the 128-byte swizzle row.
+                            const uint32_t acc = (later || k4 > 0) ? 1u : 0u;
+                            const uint64_t a_desc = (static_cast<uint64_t>(a_hi) << 32) | (a_lo + 2u * k4);
+                            if (SWAP) {
+                                // weights are the 128-row operand (two halves of the tile's 256 columns,
+                                // 16 KiB apart in the stage), activations the N operand
 #pragma unroll
-                            for (int hh = 0; hh < 2; ++hh)
-                                ptx::umma_f16(d_tmem + hh * 128,
-                                              (static_cast<uint64_t>(b_hi) << 32) | (b_lo + hh * (16384u >> 4) + k4 * kstep),
-                                              a_desc, idesc, acc);
-                        } else {
-                            ptx::umma_f16(d_tmem, a_desc, (static_cast<uint64_t>(b_hi) << 32) | (b_lo + k4 * kstep), idesc,
-                                          acc);
+                                for (int hh = 0; hh < 2; ++hh)
+                                    ptx::umma_f16(d_tmem + hh * 128,
+                                                  (static_cast<uint64_t>(b_hi) << 32) | (b_lo + hh * (16384u >> 4) + k4 * kstep),
+                                                  a_desc, idesc, acc);
+                            } else {
+                                ptx::umma_f16(d_tmem, a_desc, (static_cast<uint64_t>(b_hi) << 32) | (b_lo + k4 * kstep), idesc,
+                                              acc);
+                            }
                         }
-                    }
-                    }
+                    };
+                    const uint32_t a_lo = a_lo0 + s * stage_step, b_lo = b_lo0 + s * stage_step;
+                    issue_sub(a_lo, b_lo, kb > kb0);
+                    // (the paired form is a branch of its own so that the one-k-block form keeps its straight-line code:
+                    // as a loop over the sub-stages it cost the 256-column tiles 6 % - 2048^3 16.2 -> 17.2 us)
+                    if (kTunable && NSUB == 2) issue_sub(a_lo + (SUB >> 4), b_lo + (SUB >> 4), true);
                     ptx::umma_commit_addr(empty0 + 8 * s);
                     if (t == 0 && kb == kb0 + 8) KLIN_T(28);
                     if (t == 0 && kb == kb0 + 9) KLIN_T(31);

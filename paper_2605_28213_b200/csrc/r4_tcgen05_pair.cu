@@ -232,6 +232,9 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     int* gstart = reinterpret_cast<int*>(const_cast<uint32_t*>(abort_flag) + 2);   // MODE 2: first tile of every group
+    // streamed schedule: six barriers per epilogue warp for the partial sums it streams through the idle ring (the
+    // group table's space is free there)
+    uint64_t* fix_bar = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(gstart) + 7) & ~uintptr_t(7));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();          // 0 = even CTA (issues the MMAs), 1 = odd CTA
@@ -257,6 +260,8 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         }
         abort_flag[0] = 0;
         abort_flag[1] = 0;
+        if (SK)
+            for (int i = 0; i < 8 * 6; ++i) ptx::mbar_init(&fix_bar[i], 1);
         ptx::fence_barrier_init();
         KLIN_T(24);
         if (MODE != 2) {
@@ -494,7 +499,6 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             // plus s * (stage bytes >> 4) in the 14-bit start-address field (the ring ends below 256 KiB).  The next
             // tile's coordinates are worked out BEFORE the wait for the drained accumulators, not after it.
             uint32_t tcount = 0, s = 0, ph = 0;
-            uint32_t ready = 0;     // the current stage's "full" barrier was seen complete by the look-ahead probe
             bool ok = true;
             const uint32_t full0 = ptx::smem_u32(full), empty0 = ptx::smem_u32(empty);
             const uint32_t empty_odd0 = ptx::map_to_cta(empty0, 1);
@@ -527,7 +531,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 ptx::tc_fence_after_sync();
                 KLIN_T(tcount < 4 ? 8 + 4 * static_cast<int>(tcount) : -1);
                 for (int kb = kb_first; kb < kb_end; ++kb) {
-                    if (!ready && !ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag)) {
+                    if (!ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag)) {
                         report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x530u | s);
                         abort_flag[0] = 1;
                         ok = false;
@@ -535,10 +539,9 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     }
                     // (no tcgen05 fence: the operands came through the async proxy, which is how the MMA reads them.)
                     // This thread's instruction stream bounds the main loop - eight MMAs at ~85 clocks of issue each
-                    // plus what surrounds them, against the 1024 clocks the tensor pipe needs - so the next
-                    // stage's barrier is probed here, a k-block ahead of the wait that would use the answer.
+                    // plus what surrounds them, against the 1024 clocks the tensor pipe needs - so nothing is derived
+                    // here that can be carried.  (A look-ahead probe of the next stage's barrier changed nothing.)
                     const uint32_t s_next = (s + 1 == STAGES) ? 0u : s + 1, ph_next = (s + 1 == STAGES) ? ph ^ 1u : ph;
-                    ready = ptx::mbar_test_addr(full0 + 8 * s_next, ph_next);
                     if (kb == kb_first) KLIN_T(tcount < 4 ? 9 + 4 * static_cast<int>(tcount) : -1);
                     if (kb == kb_end - 1) KLIN_T(tcount < 4 ? 10 + 4 * static_cast<int>(tcount) : -1);
                     const uint32_t a_lo = a_lo0 + s * static_cast<uint32_t>(kStageBytes >> 4);
@@ -795,8 +798,84 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     }
                 }
             };
+            if (SK && n_part > 0 && p.sk_rounds == 0) {
+                // The owner's piece is the pair's LAST work here (no whole tiles follow), its MMAs have completed and
+                // no load is in flight or to come: the operand ring is idle.  The partial sums stream through it -
+                // 4 KiB blocks by bulk copies, six in flight per warp on barriers of their own, in the order they are
+                // added (unit, half, slot) - instead of through registers, where one slot's sixteen loads per lane at
+                // a time left this epilogue, which nothing hides, at 25-28 k clocks.
+                const int wi = warp - kEpiWarp0;
+                const uint32_t buf0 = ptx::smem_u32(smem) + static_cast<uint32_t>(wi) * (6u * 4096u);
+                const uint32_t bar0 = ptx::smem_u32(fix_bar + wi * 6);
+                const int per_unit = (cpc / 32) * n_part;          // items of a unit: (half, slot), slots in k order
+                const int total = nunits * per_unit;
+                auto issue_item = [&](int i) {
+                    if (lane == 0) {
+                        const int blk = i / n_part, j = 1 + i % n_part;
+                        const float* src = p.sk_slots + (pair_id + j) * (TILE_M * PN) + (sk_block + blk) * 1024;
+                        const uint32_t slot = static_cast<uint32_t>(i % 6);
+                        ptx::fence_proxy_async_smem();             // the buffer's last readers were generic loads
+                        ptx::mbar_arrive_expect_tx_addr(bar0 + 8 * slot, 4096u);
+                        ptx::bulk_load_1d(buf0 + slot * 4096u, src, 4096u, bar0 + 8 * slot);
+                    }
+                };
+                for (int i = 0; i < total && i < 6; ++i) issue_item(i);
+                bool fine = true;
+#pragma unroll 1
+                for (int u = 0; u < nunits && fine; ++u) {
+                    issue(u, a0, a1);
+                    ptx::tmem_ld_wait();
+                    if (u == nunits - 1) release();
+#pragma unroll 1
+                    for (int k = 0; k < per_unit; ++k) {
+                        const int i = u * per_unit + k;
+                        const uint32_t slot = static_cast<uint32_t>(i % 6);
+                        if (!ptx::mbar_wait_addr(bar0 + 8 * slot, static_cast<uint32_t>(i / 6) & 1u, abort_flag)) {
+                            if (lane == 0) report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x570u | slot);
+                            abort_flag[0] = 1;
+                            fine = false;
+                            break;
+                        }
+                        const float4* sp = reinterpret_cast<const float4*>(smem + wi * (6 * 4096) + slot * 4096) + lane;
+                        float4 t[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) t[e] = sp[e * 32];
+                        if (k >= n_part) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                a1[4 * e] = __float_as_uint(__uint_as_float(a1[4 * e]) + t[e].x);
+                                a1[4 * e + 1] = __float_as_uint(__uint_as_float(a1[4 * e + 1]) + t[e].y);
+                                a1[4 * e + 2] = __float_as_uint(__uint_as_float(a1[4 * e + 2]) + t[e].z);
+                                a1[4 * e + 3] = __float_as_uint(__uint_as_float(a1[4 * e + 3]) + t[e].w);
+                            }
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                a0[4 * e] = __float_as_uint(__uint_as_float(a0[4 * e]) + t[e].x);
+                                a0[4 * e + 1] = __float_as_uint(__uint_as_float(a0[4 * e + 1]) + t[e].y);
+                                a0[4 * e + 2] = __float_as_uint(__uint_as_float(a0[4 * e + 2]) + t[e].z);
+                                a0[4 * e + 3] = __float_as_uint(__uint_as_float(a0[4 * e + 3]) + t[e].w);
+                            }
+                        }
+                        __syncwarp();
+                        if (i + 6 < total) issue_item(i + 6);
+                    }
+                    if (!fine) {
+                        if (u != nunits - 1) release();
+                        break;
+                    }
+                    pack(u, a0, a1, c0);
+                    stage_store(u, c0);
+                }
+                if (!fine) {
+                    ok = false;
+                    break;
+                }
+                continue;
+            }
             if (SK && n_part > 0) {
-                // The owner of a streamed tile, unit by unit: the accumulator's values plus the partial sums of the
+                // The owner of a streamed tile when whole tiles follow (its epilogue then hides behind their MMAs, and
+                // the ring is theirs), unit by unit: the accumulator's values plus the partial sums of the
                 // later k ranges.  (One unit of the accumulator in registers at a time: the registers go to the
                 // sixteen loads per lane that are in flight for every slot.)
 #pragma unroll 1

@@ -278,7 +278,8 @@ def test_tcgen05_cta_pair_streamed_last_wave(handles, col):
     for idx, (M, N, K) in enumerate([(2048, 4096, 2048),     # 64 tiles on 74 pairs: everything is streamed
                                      (4096, 4096, 1024),     # 128 tiles: one full round, then 54 streamed tiles
                                      (5000, 5200, 1104),     # 10 x 21 = 210 tiles: two rounds + 62 tiles, ragged M, N, K
-                                     (1536, 2048, 4096)]):   # 24 tiles: every tile cut into three or four pieces
+                                     (1536, 2048, 4096),     # 24 tiles: every tile cut into three or four pieces
+                                     (2500, 2120, 1104)]):   # 5 x 9 = 45 tiles, all streamed, ragged M, N and K
         for bf in (False, True):
             case = gen.make_case(M, N, K, seed=320 + idx, dist_a="integer", dist_b="integer", b_col_major=col,
                                  c_bf16=bf, name=f"streamed{M}x{N}x{K}-int")
