@@ -1273,7 +1273,9 @@ struct PairColumns {
 // alternating), measured with uniform-width launches.
 double pair_kblock_cycles(int w)
 {
-    return w >= 128 ? 4.0 * w : 512.0;
+    // (single under-filled waves at K = 8192: 256 / 192 / 128 columns 90.1 / 84.0 / 81 us per tile - the issuing thread
+    // and the A operand's bytes do not shrink with the width)
+    return w >= 256 ? 1035.0 : w >= 192 ? 960.0 : w >= 128 ? 930.0 : 900.0;
 }
 
 // Makespan (cycles) of the static schedule: tiles in schedule order (all wide ones, then the narrow ones),
@@ -1382,6 +1384,17 @@ PairColumns plan_columns(const GemmArgs& g, const RunContext& ctx)
     };
     const int all_wide = static_cast<int>((static_cast<int64_t>(g.N) + wide - 1) / wide);
     consider(all_wide, wide);              // uniform tiles
+    if (ctx.plan.tile_n == 0 && ctx.plan.tail_n == 0 && ctx.plan.split_via != 3 && tiles_m2 * all_wide <= pairs) {
+        // One under-filled round: narrower uniform tiles that still fit one round finish sooner (a tile's time falls by
+        // 7-10 %, nothing else changes): 3072 x 2048 x 8192 90.1 -> 84.0 us with 192 columns.
+        for (int w : {192, 128}) {
+            const int64_t cols = (static_cast<int64_t>(g.N) + w - 1) / w;
+            if (tiles_m2 * cols > pairs) continue;
+            const double t = nkb * pair_kblock_cycles(w) + per_tile;
+            if (t < best.cycles * 0.97) best = {w, static_cast<int>(cols), 0, 0, t};
+        }
+        return best;
+    }
     if (ctx.plan.tail_n == wide) return best;
     if (ctx.plan.tail_n > 0 && !valid_w(ctx.plan.tail_n)) return PairColumns{0, 0, 0, 0, 0.0};
     if (ctx.plan.tail_n > 0) best.tile_n = 0;        // a pinned narrow width must be used
