@@ -284,10 +284,13 @@ klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype, int64_t M
  * grouped: a table of per-group tensor maps and sizes, built in the handle's
  * workspace and copied on `stream` ahead of the kernel; at most 256 groups per
  * launch) when they fill at least half of the SMs: on the CTA-pair kernel
- * (512 x 256 tiles) when every problem has more than 256 rows and K >= 2048,
- * else on the single-CTA kernel (128 x 256 tiles, whose double-buffered
- * accumulator hides the epilogue that short K exposes); a plan pinned for the
- * shape of the (first) problem may name the kernel.  Every other case - lower
+ * (512 x 256 tiles) when K >= 1024 and either every problem has more than 256
+ * rows or rounding every group's rows up to a multiple of 256 adds at most a
+ * quarter (a pair tile with at most 256 live rows does half the work; such
+ * last tile rows of the groups are scheduled last), else on the single-CTA
+ * kernel (128 x 256 tiles, whose double-buffered accumulator hides the epilogue
+ * that short K exposes); a plan pinned for the shape of the (first) problem
+ * may name the kernel.  Every other case - lower
  * rungs, unaligned operands, a K == 0 group, too few tiles - runs the rung's
  * ordinary path once per problem, in order, on `stream`.
  * Results equal those of `batch` / `groups` separate klineage_gemm_run calls
