@@ -125,6 +125,7 @@ struct R4Params {
     ConvGeom conv;
     int conv_fast;          // 1: C % 8 == 0 and x 16-byte aligned - an 8-k chunk is one 16-byte load
     int half_only;          // every unit is the first 128-column half of its tile (problems with N <= 128)
+    int one_wave;           // whole unsplit tiles, at most one per CTA: unit u is tile (u / tiles_n, u % tiles_n)
     int conv_ring6;         // Conv2d by TMA, F <= 128: six 32 KiB stages with their own barriers and a lean producer loop
     int conv_t;             // Conv2d by TMA, F <= 128, transposed: filters are the 128-row MMA operand, a unit is TWO patch
                             // tiles (256 pixels as the N operand: full-width MMAs), the epilogue stores y transposed
@@ -203,6 +204,19 @@ __device__ __forceinline__ Unit decode_unit(int64_t u, const R4Params& p)
     int half = 0;
     const int tile_n = p.tile_n;
     x.ncols = tile_n;
+    if (p.one_wave) {
+        // One wave of whole tiles: the order they are dealt in does not matter, so the unit decodes with one 32-bit
+        // division (this arithmetic is the first thing every role runs: cold code on the critical path of short kernels).
+        const uint32_t u32 = static_cast<uint32_t>(u), tn_count = static_cast<uint32_t>(p.tiles_n);
+        const uint32_t tm = u32 / tn_count, tn = u32 - tm * tn_count;
+        x.tile = u;
+        x.split = 0;
+        x.m0 = static_cast<int>(tm) * BM;
+        x.n0 = static_cast<int>(tn) * tile_n;
+        x.kb0 = 0;
+        x.kb1 = p.nkb;
+        return x;
+    }
     if (p.cluster) {              // splits is a power of two: no division on the critical path of short kernels
         x.tile = u >> p.splits_log2;
         x.split = static_cast<int>(u & (p.splits - 1));
@@ -2261,6 +2275,7 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
     p.total_units = p.splits > 1 ? tiles * p.splits : p.full_units + 2 * (tiles - p.full_units);
     p.idesc_half = (p.idesc & ~(0x3Fu << 17)) | (static_cast<uint32_t>((shape.tile_n / 2) >> 3) << 17);
     const int64_t units = p.total_units;
+    p.one_wave = (p.splits == 1 && !p.cluster && p.full_units == tiles && units <= ctx.sm_count && tiles_m > 1) ? 1 : 0;
     // A cluster handles exactly one tile, so the cluster path launches every unit as a CTA.
     const unsigned grid = static_cast<unsigned>((p.cluster || units < ctx.sm_count) ? units : ctx.sm_count);
     if (md) {
