@@ -36,6 +36,15 @@ def test_library_exports_every_declared_symbol(kb):
         assert name in decl or name.startswith("klineage_"), name
 
 
+def test_shipped_library_carries_no_trace_code(kb):
+    """The timeline stamps of the tcgen05 kernels exist only in builds with -DKLIN_TRACE: the shipped library exports
+    none of the trace entry points (and therefore holds no trace buffer the kernels could write to)."""
+    import ctypes
+    lib = ctypes.CDLL(str(kb.LIB_PATH))
+    for name in ("klin_trace_dump_pair", "klin_trace_dump_single", "klin_trace_set_knob"):
+        assert not hasattr(lib, name), name
+
+
 def test_status_and_variant_names(kb):
     assert kb.klineage_status_string(0) == "ok"
     assert kb.klineage_status_string(kb.KLINEAGE_ERR_BAD_VARIANT) == "bad variant"
