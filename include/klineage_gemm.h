@@ -203,6 +203,7 @@ klineage_status_t klineage_gemm_last_give_up(klineage_gemm_t h, unsigned* block_
  *   400 + 1*(generic-proxy producer) + 2*(direct epilogue) + 4*(split-K) + 8*(skinny mode)
  *       + 16*(cluster reduce) + 32*(CTA-pair MMA) + 64*(unaligned operands repacked into the workspace)
  *       + 128*(last wave of CTA-pair tiles streamed along K)
+ *       + 256*(CTA-pair MMA on 256-row tiles, two k-blocks per stage)
  *   500 mma.sync rung on the TMA ring, 501 on producer threads
  *   900 zero fill (K == 0); -1 before the first run or after a no-op.
  */
@@ -440,9 +441,13 @@ klineage_status_t klineage_gemm_run_host(klineage_gemm_t h, int64_t M, int64_t N
  *   tail_n     CTA-pair kernel only: tile_n = every tile of that width; a smaller multiple of 64 = tile rows
  *              start with tile_n-wide tiles and end with tiles of this width, dealt to the CTA pairs back and
  *              forth so that wide and narrow turns balance a last, under-filled wave
- *   stages     single-CTA kernel only: depth of the operand ring in 64-deep k-blocks - 4; 6 with 128- or 64-column
+ *   stages     single-CTA kernel: depth of the operand ring in 64-deep k-blocks - 4; 6 with 128- or 64-column
  *              tiles; 8 with 64-column tiles.  Without a K split, 6 stages of 128-column tiles and 8 stages of
- *              64-column tiles are filled and freed two k-blocks at a time (3 / 4 stages of 128 k)
+ *              64-column tiles are filled and freed two k-blocks at a time (3 / 4 stages of 128 k).
+ *              CTA-pair kernel: 3 = tiles of 256 x 256 instead of 512 x 256, three stages of two k-blocks each,
+ *              the two TMEM accumulators holding consecutive tiles of a pair (one fills while the other drains);
+ *              256-column tiles only, no narrow tail, no streamed wave.  The heuristic takes it for K >= 3072
+ *              when such tiles make one round over more than half of the CTA pairs
  * Every plan computes the same C up to fp32 summation order (plans that differ
  * only in kernel / group_m / half_tail / tile shape / stages are bit-identical; K
  * splits change the order of the partial sums and stay within the parity bound).

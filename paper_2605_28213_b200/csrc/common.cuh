@@ -165,7 +165,7 @@ struct R4Plan {
                          // single-CTA kernel: 64, 128 or 256)
     int tail_n = 0;      // pair kernel: 0 auto, tile_n = uniform tiles, else the width of the narrow tiles that
                          // follow the wide ones in every tile row and balance the last wave
-    int stages = 0;      // 0 auto, else depth of the operand ring
+    int stages = 0;      // 0 auto, else depth of the operand ring (pair kernel: 3 = 256-row tiles, two k-blocks per stage)
 };
 
 // Host-side state of a handle that the TMA rungs need.
@@ -247,6 +247,8 @@ cudaError_t launch_r35_mma_sync(const GemmArgs& g, RunContext& ctx, cudaStream_t
 cudaError_t launch_zero_fill(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
 // CTA-pair (cta_group::2) form of rung 4 and the test of its preconditions.
 bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx);
+// Whether an unpinned single-destination launch takes the pair kernel's k-paired 256-row tiles.
+bool r4_pair_k_paired_auto(const GemmArgs& g, const RunContext& ctx);
 // Hard preconditions of the CTA-pair kernel only (operands TMA-loadable), without the size heuristic.
 bool r4_pair_possible(const GemmArgs& g, const RunContext& ctx);
 // Whether the pair kernel can stream this problem's last wave along K (enough k-blocks per piece, workspace for the

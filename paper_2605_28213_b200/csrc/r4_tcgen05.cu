@@ -336,7 +336,8 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         return x;
     };
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // (the warp index by a broadcast: the compiler then knows it, and every role branch, to be uniform across the warp)
+    const int warp = __shfl_sync(0xFFFFFFFFu, static_cast<int>(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     // Cluster mode: no CTA may touch a peer's shared memory before that peer runs and has initialised the barrier
     // its incoming partial sums are counted on (warp 0 arrives after it has done that, below).
     if (SWAP && p.cluster && warp != 0) ptx::cluster_arrive_relaxed();
@@ -755,7 +756,12 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // The whole warp walks the schedule and waits on the barriers; lane 0 alone issues the MMAs and commits.  (With
+        // the loop inside a one-lane branch every descriptor is a per-thread value that has to be moved into the uniform
+        // registers the MMA instruction reads, instruction by instruction; in converged code the compiler keeps ring
+        // position and descriptors there from the start.)
+        {
+            const bool issuer = lane == 0;
             uint32_t t = 0;
             bool ok = true;
             // The ring position (stage s, phase ph) is carried instead of derived, barriers are addressed by their
@@ -781,19 +787,23 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                 const uint32_t idesc = (x.ncols == TN) ? p.idesc : p.idesc_half;
                 const uint32_t buf = t & 1;
                 if (!ptx::mbar_wait(&acc_empty[buf], ((t >> 1) & 1) ^ 1, abort_flag)) {
-                    report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x410u | buf);
-                    abort_flag[0] = 1;
+                    if (issuer) {
+                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x410u | buf);
+                        abort_flag[0] = 1;
+                    }
                     break;
                 }
                 ptx::tc_fence_after_sync();
-                if (t == 0) KLIN_T(8);
+                if (issuer && t == 0) KLIN_T(8);
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    if (t == 0 && kb == kb0 + 8) KLIN_T(26);
-                    if (t == 0 && kb == kb0 + 9) KLIN_T(29);
+                    if (issuer && t == 0 && kb == kb0 + 8) KLIN_T(26);
+                    if (issuer && t == 0 && kb == kb0 + 9) KLIN_T(29);
                     if (!ptx::mbar_wait_addr(full0 + 8 * s, ph, abort_flag, full_limit)) {
-                        report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x420u | s);
-                        abort_flag[0] = 1;
+                        if (issuer) {
+                            report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x420u | s);
+                            abort_flag[0] = 1;
+                        }
                         ok = false;
                         break;
                     }
@@ -803,10 +813,10 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                     // (A look-ahead probe of the next stage's barrier cost this kernel's long-K launches 6 %, 63.5 -> 67.6 us
                     // at 2048 x 2048 x 8192, ahead of the MMAs and 3 % behind them: not used.)
                     const uint32_t s_next = (s + 1 == n_stages) ? 0u : s + 1, ph_next = (s + 1 == n_stages) ? ph ^ 1u : ph;
-                    if (t == 0 && kb == kb0) KLIN_T(9);
-                    if (t == 0 && kb == kb1 - 1) KLIN_T(10);
-                    if (t == 0 && kb == kb0 + 8) KLIN_T(27);
-                    if (t == 0 && kb == kb0 + 9) KLIN_T(30);
+                    if (issuer && t == 0 && kb == kb0) KLIN_T(9);
+                    if (issuer && t == 0 && kb == kb1 - 1) KLIN_T(10);
+                    if (issuer && t == 0 && kb == kb0 + 8) KLIN_T(27);
+                    if (issuer && t == 0 && kb == kb0 + 9) KLIN_T(30);
                     // the MMAs of one 64-deep (sub-)stage; `later`: not the unit's first sub-stage
                     auto issue_sub = [&](uint32_t a_lo, uint32_t b_lo, bool later) {
 #pragma unroll
@@ -832,18 +842,20 @@ r4_tcgen05_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const _
                         }
                     };
                     const uint32_t a_lo = a_lo0 + s * stage_step, b_lo = b_lo0 + s * stage_step;
-                    issue_sub(a_lo, b_lo, kb > kb0);
-                    // (the paired form is a branch of its own so that the one-k-block form keeps its straight-line code:
-                    // as a loop over the sub-stages it cost the 256-column tiles 6 % - 2048^3 16.2 -> 17.2 us)
-                    if (kTunable && NSUB == 2) issue_sub(a_lo + (SUB >> 4), b_lo + (SUB >> 4), true);
-                    ptx::umma_commit_addr(empty0 + 8 * s);
-                    if (t == 0 && kb == kb0 + 8) KLIN_T(28);
-                    if (t == 0 && kb == kb0 + 9) KLIN_T(31);
+                    if (issuer) {
+                        issue_sub(a_lo, b_lo, kb > kb0);
+                        // (the paired form is a branch of its own so that the one-k-block form keeps its straight-line
+                        // code: as a loop over the sub-stages it cost the 256-column tiles 6 % - 2048^3 16.2 -> 17.2 us)
+                        if (kTunable && NSUB == 2) issue_sub(a_lo + (SUB >> 4), b_lo + (SUB >> 4), true);
+                        ptx::umma_commit_addr(empty0 + 8 * s);
+                    }
+                    if (issuer && t == 0 && kb == kb0 + 8) KLIN_T(28);
+                    if (issuer && t == 0 && kb == kb0 + 9) KLIN_T(31);
                     s = s_next;
                     ph = ph_next;
                 }
-                if (ok) ptx::umma_commit(&acc_full[buf]);
-                if (t == 0) KLIN_T(11);
+                if (ok && issuer) ptx::umma_commit(&acc_full[buf]);
+                if (issuer && t == 0) KLIN_T(11);
             }
         }
     } else if (warp < 6) {
@@ -2179,7 +2191,7 @@ cudaError_t launch_r4_planned(const GemmArgs& g, RunContext& ctx, cudaStream_t s
 
     // Large aligned problems run on the CTA-pair kernel (tcgen05.mma.cta_group::2).
     if (pinned.kernel == 2 && (plan.swap || plan.splits != 1 || !r4_pair_possible(g, ctx))) return cudaErrorInvalidValue;
-    const bool use_pair = pinned.kernel == 2 || (pinned.kernel == 0 && r4_pair_applicable(g, ctx));
+    const bool use_pair = pinned.kernel == 2 || (pinned.kernel == 0 && (r4_pair_applicable(g, ctx) || (!md && plan.splits == 1 && !plan.swap && r4_pair_k_paired_auto(g, ctx))));
     if (md && (plan.swap || plan.splits != 1)) return cudaErrorNotSupported;
     if (!plan.swap && plan.splits == 1 && use_pair)
         return md ? launch_r4_pair_multi_dst(g, md->C, md->ldc, md->n, ctx, stream, kernel_id)
@@ -2628,7 +2640,10 @@ bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& pl)
         return false;
     if (pl.tail_n != 0 && pl.kernel != 2) return false;
     if (pl.split_via == 3 && (pl.kernel != 2 || pl.splits > 1)) return false;     // streaming the last wave is the pair kernel's
-    if (pl.kernel == 2 && pl.stages != 0) return false;
+    // CTA-pair kernel: stages = 3 asks for k-paired 256-row tiles (three stages of two k-blocks), 256 columns wide
+    if (pl.kernel == 2 && pl.stages != 0 &&
+        !(pl.stages == 3 && (pl.tile_n == 0 || pl.tile_n == BN) && pl.tail_n == 0 && pl.split_via != 3))
+        return false;
     if (pl.kernel != 2 && (pl.tile_n != 0 || pl.stages != 0)) {
         // single-CTA kernel: 256 columns x 4 stages, 128 columns x 4 or 6, 64 columns x 4, 6 or 8 (plain TMA-fed GEMM, M > 64)
         if (pl.tile_n != 0 && pl.tile_n != BN && pl.tile_n != BN / 2 && pl.tile_n != BN / 4) return false;
@@ -2697,6 +2712,14 @@ int r4_enumerate_plans(const GemmArgs& g, const RunContext& ctx, R4Plan* out, in
             pl.tile_n = 256;
             pl.tail_n = 192;
             push(pl);
+            // 256-row tiles, two k-blocks per stage
+            if (g.M > 2 * BM) {
+                R4Plan pk;
+                pk.kernel = 2;
+                pk.splits = 1;
+                pk.stages = 3;
+                push(pk);
+            }
             // last wave streamed along K, and never streamed
             for (int via : {3, 1}) {
                 R4Plan ps;

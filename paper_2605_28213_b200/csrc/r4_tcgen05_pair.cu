@@ -221,10 +221,19 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                const __grid_constant__ CUtensorMap map_c, PairParams p)
 {
     constexpr bool SK = MODE_ == 5;
-    constexpr int MODE = SK ? 0 : MODE_;
+    constexpr bool KP = MODE_ == 6;
+    constexpr int MODE = (SK || KP) ? 0 : MODE_;
+    // Ring and tile geometry.  The plain forms: 512-row tiles, four stages of one k-block (two row blocks of A and half
+    // of B).  KP: 256-row tiles, three stages of TWO k-blocks (A and half of B of either), eight MMAs per stage into
+    // ONE accumulator; the two accumulators belong to consecutive tiles of the pair, each drained by its own four
+    // epilogue warps while the other fills.
+    constexpr int NS = KP ? 3 : STAGES;
+    constexpr int SB = KP ? 4 * kABlockBytes : kStageBytes;
+    constexpr int TM = KP ? 2 * PM : TILE_M;
+    constexpr int KSTAGE = KP ? 2 * BK : BK;     // k per stage
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* epi_smem = smem + STAGES * kStageBytes;
+    uint8_t* epi_smem = smem + STAGES * kStageBytes;     // (= 3 x 64 KiB: the k-paired ring ends at the same place)
     uint64_t* full = reinterpret_cast<uint64_t*>(epi_smem + kEpiBytes);   // even CTA: both CTAs' loads landed
     uint64_t* empty = full + STAGES;                                      // the pair's MMAs are done with the stage
     uint64_t* acc_full = empty + STAGES;                                  // [0]: the tile's accumulators are complete
@@ -256,7 +265,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(&acc_full[b], 1);
-            ptx::mbar_init(&acc_empty[b], 16);             // 8 epilogue warps of each CTA
+            ptx::mbar_init(&acc_empty[b], KP ? 8 : 16);    // the epilogue warps of both CTAs that drain it
         }
         abort_flag[0] = 0;
         abort_flag[1] = 0;
@@ -347,7 +356,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 x.width = min(x.width, (g.N - x.n0 + 63) & ~63);
             }
         }
-        x.m0 = tm * TILE_M + static_cast<int>(rank) * PM;   // this CTA's rows: m0 + [0,128) and m0 + 256 + [0,128)
+        x.m0 = tm * TM + static_cast<int>(rank) * PM;   // this CTA's rows: m0 + [0,128) and (512-row tiles) m0 + 256 + [0,128)
         return x;
     };
     // The r-th tile of this pair (-1: the schedule has ended).  Odd rounds run over the pairs in reverse
@@ -457,9 +466,9 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 const int kb_end = wk.kb1 < 0 ? x.nkb : wk.kb1;
                 if (it == 0) KLIN_T(28);
                 for (int kb = wk.kb0; kb < kb_end; ++kb, ++it) {
-                    const uint32_t sa = smem0 + s * kStageBytes, sb = sa + kABytes;
+                    const uint32_t sa = smem0 + s * SB, sb = sa + kABytes;
                     const uint32_t bar = full_even0 + 8 * s;
-                    const int kx = kb * BK;
+                    const int kx = kb * KSTAGE;
                     if (!ptx::mbar_wait_addr(empty0 + 8 * s, ph, abort_flag)) {
                         report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x500u | s);
                         abort_flag[0] = 1;
@@ -469,6 +478,19 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     // The even CTA's barrier counts the bytes of both CTAs' loads of this stage.
                     if (rank == 0) ptx::mbar_arrive_expect_tx_addr(full0 + 8 * s, stage_tx);
                     load_box(sa, ma, kx, m0, z, bar);
+                    if (KP) {
+                        // the stage's second k-block (past the end of K the boxes read zeros and its MMAs add nothing)
+                        load_box(sa + kABlockBytes, ma, kx + BK, m0, z, bar);
+                        if (BCOL) {
+                            load_box(sb, mb, kx, nb, z, bar);
+                            load_box(sb + kBHalfBytes, mb, kx + BK, nb, z, bar);
+                        } else {
+                            load_box(sb, mb, nb, kx, z, bar);
+                            if (two_boxes) load_box(sb + 64 * BK * 2, mb, nb + 64, kx, z, bar);
+                            load_box(sb + kBHalfBytes, mb, nb, kx + BK, z, bar);
+                            if (two_boxes) load_box(sb + kBHalfBytes + 64 * BK * 2, mb, nb + 64, kx + BK, z, bar);
+                        }
+                    } else {
                     load_box(sa + kABlockBytes, ma, kx, m0 + 2 * PM, z, bar);
                     if (BCOL) {
                         load_box(sb, mb, kx, nb, z, bar);
@@ -476,9 +498,10 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                         load_box(sb, mb, nb, kx, z, bar);
                         if (two_boxes) load_box(sb + 64 * BK * 2, mb, nb + 64, kx, z, bar);
                     }
+                    }
                     if (it == 0) KLIN_T(2);
-                    if (it == STAGES - 1) KLIN_T(3);
-                    if (++s == STAGES) {
+                    if (it == NS - 1) KLIN_T(3);
+                    if (++s == NS) {
                         s = 0;
                         ph ^= 1u;
                     }
@@ -487,9 +510,9 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             // Drain: in the even CTA wait for the last fills; the odd CTA's loads are covered by
             // the same barriers (the MMAs that consumed them have completed before the epilogue ends).
             if (rank == 0) {
-                const uint32_t first = it > STAGES ? it - STAGES : 0;
+                const uint32_t first = it > NS ? it - NS : 0;
                 for (uint32_t j = first; j < it; ++j)
-                    ptx::mbar_wait(&full[j % STAGES], (j / STAGES) & 1, abort_flag + 1);
+                    ptx::mbar_wait(&full[j % NS], (j / NS) & 1, abort_flag + 1);
             }
         }
     } else if (warp == 1) {
@@ -522,8 +545,10 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 // block's MMAs only: this thread's instruction stream bounds the loop, so such a tile takes about
                 // half the time (its second accumulator is never read: the epilogue warps of that block have no rows).
                 const bool two_blocks = x.M - x.m0 > 2 * PM;
-                // Both accumulators are rewritten: wait until both CTAs' epilogues drained the last tile.
-                if (!ptx::mbar_wait(&acc_empty[0], (tcount & 1) ^ 1, abort_flag)) {
+                // Both accumulators are rewritten: wait until both CTAs' epilogues drained the last tile.  (KP: the
+                // accumulator of this tile's parity, drained of the tile before the last.)
+                const uint32_t buf = KP ? (tcount & 1u) : 0u;
+                if (!ptx::mbar_wait(&acc_empty[buf], ((KP ? tcount >> 1 : tcount) & 1) ^ 1, abort_flag)) {
                     report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x520u);
                     abort_flag[0] = 1;
                     break;
@@ -541,20 +566,31 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     // This thread's instruction stream bounds the main loop - eight MMAs at ~85 clocks of issue each
                     // plus what surrounds them, against the 1024 clocks the tensor pipe needs - so nothing is derived
                     // here that can be carried.  (A look-ahead probe of the next stage's barrier changed nothing.)
-                    const uint32_t s_next = (s + 1 == STAGES) ? 0u : s + 1, ph_next = (s + 1 == STAGES) ? ph ^ 1u : ph;
+                    const uint32_t s_next = (s + 1 == NS) ? 0u : s + 1, ph_next = (s + 1 == NS) ? ph ^ 1u : ph;
                     if (kb == kb_first) KLIN_T(tcount < 4 ? 9 + 4 * static_cast<int>(tcount) : -1);
                     if (kb == kb_end - 1) KLIN_T(tcount < 4 ? 10 + 4 * static_cast<int>(tcount) : -1);
-                    const uint32_t a_lo = a_lo0 + s * static_cast<uint32_t>(kStageBytes >> 4);
-                    const uint32_t b_lo = b_lo0 + s * static_cast<uint32_t>(kStageBytes >> 4);
+                    const uint32_t a_lo = a_lo0 + s * static_cast<uint32_t>(SB >> 4);
+                    const uint32_t b_lo = b_lo0 + s * static_cast<uint32_t>(SB >> 4);
+                    if (KP) {
+                        const uint32_t d = tmem_base + buf * PN;
 #pragma unroll
-                    for (int k4 = 0; k4 < BK / 16; ++k4) {
-                        const uint32_t acc = (kb > kb_first || k4 > 0) ? 1u : 0u;
-                        // alternate the two row blocks: consecutive MMAs never share an accumulator
-                        const uint64_t bd = desc(b_hi, b_lo + static_cast<uint32_t>(k4) * kstep);
-                        umma_f16_pair(tmem_base, desc(a_hi, a_lo + static_cast<uint32_t>(k4 * 2)), bd, idesc, acc);
-                        if (two_blocks)
-                            umma_f16_pair(tmem_base + PN, desc(a_hi, a_lo + static_cast<uint32_t>((kABlockBytes >> 4) + k4 * 2)),
-                                          bd, idesc, acc);
+                        for (int k8 = 0; k8 < 2 * (BK / 16); ++k8) {
+                            const uint32_t sub = static_cast<uint32_t>(k8 >> 2), k4 = static_cast<uint32_t>(k8 & 3);
+                            umma_f16_pair(d, desc(a_hi, a_lo + sub * (kABlockBytes >> 4) + k4 * 2u),
+                                          desc(b_hi, b_lo + sub * (kBHalfBytes >> 4) + k4 * kstep), idesc,
+                                          (kb > kb_first || k8 > 0) ? 1u : 0u);
+                        }
+                    } else {
+#pragma unroll
+                        for (int k4 = 0; k4 < BK / 16; ++k4) {
+                            const uint32_t acc = (kb > kb_first || k4 > 0) ? 1u : 0u;
+                            // alternate the two row blocks: consecutive MMAs never share an accumulator
+                            const uint64_t bd = desc(b_hi, b_lo + static_cast<uint32_t>(k4) * kstep);
+                            umma_f16_pair(tmem_base, desc(a_hi, a_lo + static_cast<uint32_t>(k4 * 2)), bd, idesc, acc);
+                            if (two_blocks)
+                                umma_f16_pair(tmem_base + PN,
+                                              desc(a_hi, a_lo + static_cast<uint32_t>((kABlockBytes >> 4) + k4 * 2)), bd, idesc, acc);
+                        }
                     }
                     umma_commit_pair(empty0 + 8 * s);
                     umma_commit_pair(empty_odd0 + 8 * s);
@@ -562,8 +598,8 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     ph = ph_next;
                 }
                 if (ok) {
-                    umma_commit_pair(accf);
-                    umma_commit_pair(accf_odd);
+                    umma_commit_pair(accf + 8 * buf);
+                    umma_commit_pair(accf_odd + 8 * buf);
                     KLIN_T(tcount < 4 ? 11 + 4 * static_cast<int>(tcount) : -1);
                 }
             }
@@ -586,11 +622,12 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         WorkState ws = work_init();
         Work wk;
         for (; ok && next_work(ws, wk); ++tcount) {
+            if (KP && (tcount & 1u) != static_cast<uint32_t>(mb)) continue;     // the other warp group's tile
             const TileInfo x = tile_info(wk.tile);
             const int m0 = x.m0, n0 = x.n0;
             float* dst_f = reinterpret_cast<float*>(x.C);
             uint16_t* dst_h = reinterpret_cast<uint16_t*>(x.C);
-            const int row0 = m0 + mb * 2 * PM + q * 32;
+            const int row0 = m0 + (KP ? 0 : mb * 2 * PM) + q * 32;
             const int rows = min(32, x.M - row0);
             const int nunits = (row0 < x.M) ? (min(x.width, x.N - n0) + cpc - 1) / cpc : 0;
             const uint32_t tbase = tmem_base + mb * PN + (static_cast<uint32_t>(q * 32) << 16);
@@ -634,7 +671,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     break;
                 }
             }
-            if (!ptx::mbar_wait(&acc_full[0], tcount & 1, abort_flag)) {
+            if (!ptx::mbar_wait(&acc_full[KP ? mb : 0], (KP ? tcount >> 1 : tcount) & 1, abort_flag)) {
                 if (lane == 0) report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x540u);
                 abort_flag[0] = 1;
                 ok = false;
@@ -648,7 +685,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 if (tcount == 0 && warp == kEpiWarp0 && lane == 0) KLIN_T(60);
                 __syncwarp();
                 if (tcount == 0 && warp == kEpiWarp0 && lane == 0) KLIN_T(61);
-                if (lane == 0) mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&acc_empty[0]), 0));
+                if (lane == 0) mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&acc_empty[KP ? mb : 0]), 0));
             };
             auto issue = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32]) {
                 ptx::tmem_ld_32x32b_x32(tbase + u * cpc, r0);
@@ -1409,6 +1446,31 @@ PairColumns plan_columns(const GemmArgs& g, const RunContext& ctx)
     }
     return best;
 }
+
+// Whether a single problem runs as k-paired 256-row tiles: when a plan asks for it (stages = 3), else - with nothing
+// pinned - by the rule of r4_pair_k_paired_auto.  Never with a tile width other than 256, a narrow tail or a streamed
+// last wave.
+bool pair_k_paired(const GemmArgs& g, const RunContext& ctx)
+{
+    const R4Plan& pl = ctx.plan;
+    if (pl.stages != 0 && pl.stages != 3) return false;
+    if ((pl.tile_n != 0 && pl.tile_n != PN) || pl.tail_n != 0 || pl.split_via == 3) return false;
+    if (pl.stages == 3) return true;
+    return pl.kernel == 0 && pl.split_via == 0 && pl.tile_n == 0 && r4_pair_k_paired_auto(g, ctx);
+}
+}
+
+// One round of 256 x 256 tiles that fills more than half of the CTA pairs, K long enough to pay for the pair kernel's
+// set-up.  Measured (single launches after an L2 flush, against the single-CTA kernel's one wave of 128 x 256 tiles):
+// 2048 x 2048 x 8192 56.2 against 61.4 us, 512 x 8192 x 8192 61.5 / 65.5, 1536 x 2048 x 4096 32.8 / 34.8, 2304 x 2048 x
+// 6144 45.6 / 49.1, 2048 x 2048 x 3072 28.2 / 28.8; with 32 tiles (1024 x 2048 x 8192) 54 against 42 for the
+// single-CTA kernel's cluster split, and in several rounds (4096^3) 100 against 94 for 512-row tiles.
+bool r4_pair_k_paired_auto(const GemmArgs& g, const RunContext& ctx)
+{
+    if (!r4_pair_possible(g, ctx) || g.M <= 2 * PM || g.K < 3072) return false;
+    const int64_t tiles = static_cast<int64_t>((g.M + 2 * PM - 1) / (2 * PM)) * ((g.N + PN - 1) / PN);
+    const int64_t pairs = ctx.sm_count / 2;
+    return tiles <= pairs && 2 * tiles > pairs;
 }
 
 bool r4_pair_stream_k_possible(const GemmArgs& g, const RunContext& ctx)
@@ -1439,9 +1501,17 @@ cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const
 {
     PairParams p;
     memset(&p, 0, sizeof p);
-    p.tiles_m2 = (g.M + TILE_M - 1) / TILE_M;
+    // k-paired 256-row tiles (see the kernel): one problem, one destination, uniform 256-column tiles, whole tiles
+    const bool kp = n_dst == 0 && pair_k_paired(g, ctx);
+    if (ctx.plan.stages == 3 && !kp) return cudaErrorInvalidValue;
+    p.tiles_m2 = kp ? (g.M + 2 * PM - 1) / (2 * PM) : (g.M + TILE_M - 1) / TILE_M;
     p.nkb = (g.K + BK - 1) / BK;
-    const PairColumns cols = plan_columns(g, ctx);
+    if (kp) p.nkb = (p.nkb + 1) / 2;        // the kernel's k-loop counts stages of two k-blocks
+    PairColumns cols = plan_columns(g, ctx);
+    if (kp) {
+        const int n_tiles = (g.N + PN - 1) / PN;
+        cols = PairColumns{PN, n_tiles, 0, 0, 0.0};
+    }
     if (cols.tile_n == 0) return cudaErrorInvalidValue;
     p.tile_n = cols.tile_n;
     p.n_wide = cols.n_wide;
@@ -1456,6 +1526,7 @@ cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const
     const uint32_t b_box_rows = static_cast<uint32_t>(widest / 2);
     p.b_boxes = (widest / 2 + 63) / 64;
     p.stage_tx = 2u * (kABytes + (g.b_col ? b_box_rows * 128u : static_cast<uint32_t>(p.b_boxes) * 8192u));
+    if (kp) p.stage_tx = 2u * (kABytes + 2u * (g.b_col ? b_box_rows * 128u : static_cast<uint32_t>(p.b_boxes) * 8192u));
     // default raster group: 4 x 512 rows; 8 when the problem has at least 16 tile rows (measured at 8192^3 in rested
     // 10-launch bursts: 672-674 us against 676-678 us for 4 and 684-686 us for 1, 2, 3 or 16)
     p.group_m = ctx.plan.group_m > 0 ? ctx.plan.group_m : (p.tiles_m2 >= 16 ? 8 : 4);
@@ -1516,7 +1587,7 @@ cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const
     const int64_t max_pairs = ctx.sm_count / 2;
     unsigned grid = 2u * static_cast<unsigned>(p.total_tiles < max_pairs ? p.total_tiles : max_pairs);
     // Stream the under-filled last wave along K?  (one problem, one destination, uniform 256-column tiles)
-    if (n_dst == 0 && cols.n_narrow == 0 && cols.tile_n == PN && ctx.plan.split_via != 1) {
+    if (n_dst == 0 && !kp && cols.n_narrow == 0 && cols.tile_n == PN && ctx.plan.split_via != 1) {
         const StreamK sk = plan_stream_k(p.total_tiles, p.nkb, max_pairs, ctx, ctx.plan.split_via == 3);
         if (sk.on) {
             p.sk = 1;
@@ -1533,7 +1604,7 @@ cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const
     } else if (ctx.plan.split_via == 3) {
         return cudaErrorInvalidValue;
     }
-    p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + 32 + (p.sk ? 128 : 0) + ctx.kid_flags;
+    p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + 32 + (p.sk ? 128 : 0) + (kp ? 256 : 0) + ctx.kid_flags;
     *kernel_id = p.kid;
     if (n_dst > 0) {
         // the table travels on the launch's stream, ahead of the kernel (staged before the call returns)
@@ -1547,6 +1618,9 @@ cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const
     if (p.sk)
         return g.b_col ? launch<true, 5>(g, ma, mb, mc, p, grid, ctx.device, stream)
                        : launch<false, 5>(g, ma, mb, mc, p, grid, ctx.device, stream);
+    if (kp)
+        return g.b_col ? launch<true, 6>(g, ma, mb, mc, p, grid, ctx.device, stream)
+                       : launch<false, 6>(g, ma, mb, mc, p, grid, ctx.device, stream);
     return g.b_col ? launch<true, 0>(g, ma, mb, mc, p, grid, ctx.device, stream)
                    : launch<false, 0>(g, ma, mb, mc, p, grid, ctx.device, stream);
 }

@@ -309,11 +309,53 @@ def test_tcgen05_cta_pair_streamed_last_wave(handles, col):
                                          case.ldc, kb.klineage_gemm_plan_t(*STREAMED)) == kb.KLINEAGE_ERR_INVALID_ARG
 
 
+K_PAIRED = (2, 1, 0, 0, 0, 0, 0, 3)     # launch plan: the CTA-pair kernel on 256-row tiles, two k-blocks per stage
+@pytest.mark.parametrize("col", [False, True], ids=["Brow", "Bcol"])
+def test_tcgen05_cta_pair_k_paired_tiles(handles, col):
+    """256 x 256 pair tiles on a ring of three two-k-block stages, the TMEM accumulators alternating between a pair's
+    consecutive tiles.  Bit-exact on integers and identical to the 512-row schedule: one round, several rounds (both
+    accumulators in flight), an odd number of k-blocks (the last stage's second half lies past K), ragged M and N,
+    a tile row with at most 128 live rows (the odd CTA has none)."""
+    for idx, (M, N, K) in enumerate([(2048, 2048, 4096),     # 64 tiles on 74 pairs, one round
+                                     (4096, 4096, 320),      # 256 tiles: 3.5 rounds, five k-blocks
+                                     (2500, 2120, 1104),     # 10 x 9 tiles, ragged M, N and K (17.25 k-blocks)
+                                     (2100, 1304, 72),       # two k-blocks, the second one 8 deep; last tile row 52 rows
+                                     (300, 520, 64)]):       # one k-block: every stage's second half is empty
+        for bf in (False, True):
+            case = gen.make_case(M, N, K, seed=340 + idx, dist_a="integer", dist_b="integer", b_col_major=col,
+                                 c_bf16=bf, name=f"kpaired{M}x{N}x{K}-int")
+            rows = P.sample_rows(M)
+            C_ref, S = P.oracle_rows(case, rows)
+            vals, bits = run_and_check(handles, case, 4, C_ref, S, rows, exact=True, pin=K_PAIRED)
+            flags = handles[(col, bf)].last_kernel_id() - 400
+            assert (flags & 32) and (flags & 256), (M, N, K, flags)
+            _, whole = run_and_check(handles, case, 4, C_ref, S, rows, exact=True, pin=(2, 1, 1))
+            assert not ((handles[(col, bf)].last_kernel_id() - 400) & 256)
+            assert np.array_equal(bits, whole), "256-row and 512-row schedules differ"
+            if not bf:
+                assert P.integer_checksums_match(case, vals)
+        case = gen.make_case(M, N, K, seed=340 + idx, dist_a="normal", dist_b="uniform", b_col_major=col,
+                             name=f"kpaired{M}x{N}x{K}")
+        rows = P.sample_rows(M)
+        C_ref, S = P.oracle_rows(case, rows)
+        run_and_check(handles, case, 4, C_ref, S, rows, pin=K_PAIRED)
+    # the form is the pair kernel's and 256 columns wide: other combinations are refused
+    case = gen.make_case(2048, 2048, 4096, seed=350, dist_a="integer", dist_b="integer", b_col_major=col)
+    dev = P.DeviceCase(case)
+    g = handles[(col, False)]
+    from paper_2605_28213_b200 import binding as kb
+    for bad in ((2, 1, 0, 0, 0, 192, 0, 3), (2, 1, 3, 0, 0, 0, 0, 3), (2, 1, 0, 0, 0, 0, 0, 4), (1, 1, 0, 0, 0, 0, 0, 3)):
+        assert kb.klineage_gemm_set_plan_raw(g._h, case.M, case.N, case.K, dev.a.ptr, case.lda, dev.b.ptr, case.ldb,
+                                             dev.c.ptr, case.ldc, kb.klineage_gemm_plan_t(*bad)) == kb.KLINEAGE_ERR_INVALID_ARG
+
+
 def test_dispatch_between_the_two_kernels(handles):
     """Long K and enough 512 x 256 tiles: the pair kernel; short K or few tiles: the single-CTA kernel."""
     for (M, N, K), want_pair in (((2048, 4096, 4096), True), ((3072, 2048, 8192), True), ((2816, 2816, 2816), True),
                                  ((2048, 2048, 2048), False), ((4608, 4352, 72), False), ((3584, 3584, 3584), False),
-                                 ((2304, 2304, 2304), False)):
+                                 ((2304, 2304, 2304), False),
+                                 ((2048, 2048, 8192), True),       # one round of 64 k-paired 256-row tiles
+                                 ((1024, 2048, 8192), False)):     # 32 such tiles: the single-CTA kernel's cluster split
         case = gen.make_case(M, N, K, seed=70, dist_a="integer", dist_b="integer", c_bf16=True, name=f"disp{M}x{N}x{K}")
         rows = P.sample_rows(M)[::8]
         C_ref, S = P.oracle_rows(case, rows)
