@@ -288,7 +288,9 @@ klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype, int64_t M
  * (512 x 256 tiles) when K >= 1024 and either every problem has more than 256
  * rows or rounding every group's rows up to a multiple of 256 adds at most a
  * quarter (a pair tile with at most 256 live rows does half the work; such
- * last tile rows of the groups are scheduled last), else on the single-CTA
+ * last tile rows of the groups are scheduled last; 256 x 256 tiles instead when
+ * twice the tiles take fewer than twice the rounds over the CTA pairs - see
+ * `stages` of the launch plan), else on the single-CTA
  * kernel (128 x 256 tiles, whose double-buffered accumulator hides the epilogue
  * that short K exposes); a plan pinned for the shape of the (first) problem
  * may name the kernel.  Every other case - lower

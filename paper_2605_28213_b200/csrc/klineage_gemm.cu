@@ -589,6 +589,10 @@ klineage_status_t klineage_gemm_run_batched(klineage_gemm_t h, int64_t batch, in
             if (!guard.ok) return KLINEAGE_ERR_LAUNCH;
             h->ctx.plan = R4Plan();
             h->ctx.plan.group_m = pinned.group_m;
+            if (want == 2 && pinned.kernel == 2) {      // the plan also says which tiles: stages 3 = 256 rows, two k-blocks per stage
+                h->ctx.plan.kernel = 2;
+                h->ctx.plan.stages = pinned.stages;
+            }
             int kid = -1;
             const cudaError_t e = want == 2 ? launch_r4_pair_batched(g, ba, h->ctx, static_cast<cudaStream_t>(stream), &kid)
                                             : launch_r4_single_batched(g, ba, h->ctx, static_cast<cudaStream_t>(stream), &kid);
@@ -699,6 +703,10 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups, const
             int kid = -1;
             h->ctx.plan = R4Plan();
             h->ctx.plan.group_m = pinned.group_m;
+            if (want == 2 && pinned.kernel == 2) {      // the plan also says which tiles: stages 3 = 256 rows, two k-blocks per stage
+                h->ctx.plan.kernel = 2;
+                h->ctx.plan.stages = pinned.stages;
+            }
             if (st == KLINEAGE_OK) {
                 const cudaError_t e = want == 2 ? launch_r4_pair_grouped(ga, n, h->ctx, static_cast<cudaStream_t>(stream), &kid)
                                                 : launch_r4_single_grouped(ga, n, h->ctx, static_cast<cudaStream_t>(stream), &kid);

@@ -35,6 +35,7 @@
 // runs on the single-CTA kernel of r4_tcgen05.cu.
 #include "common.cuh"
 #include "ptx.cuh"
+#include <algorithm>
 #include <cstring>
 #include <new>
 
@@ -213,6 +214,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_f
 // MODE 0: one problem (tensor maps 2-D).  MODE 1: batched (3-D tensor maps, z = batch).
 // MODE 2: grouped (per-group tensor maps and sizes from a table in device memory).
 // MODE 3: one problem whose C goes to several destinations (table of C maps / pointers).
+// MODE 6, 7, 8: MODE 0, 1, 2 on 256-row tiles with two k-blocks per stage (see the ring geometry in the kernel).
 // MODE 5: MODE 0 with its last wave streamed along K (a separate instantiation, so that the plain kernel does not carry
 // the work-list arithmetic in its 24-register producer and MMA threads).
 template <bool BCOL, int MODE_>
@@ -221,8 +223,8 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                const __grid_constant__ CUtensorMap map_c, PairParams p)
 {
     constexpr bool SK = MODE_ == 5;
-    constexpr bool KP = MODE_ == 6;
-    constexpr int MODE = (SK || KP) ? 0 : MODE_;
+    constexpr bool KP = MODE_ >= 6;              // 6, 7, 8: modes 0, 1, 2 on k-paired 256-row tiles
+    constexpr int MODE = SK ? 0 : KP ? MODE_ - 6 : MODE_;
     // Ring and tile geometry.  The plain forms: 512-row tiles, four stages of one k-block (two row blocks of A and half
     // of B).  KP: 256-row tiles, three stages of TWO k-blocks (A and half of B of either), eight MMAs per stage into
     // ONE accumulator; the two accumulators belong to consecutive tiles of the pair, each drained by its own four
@@ -1111,6 +1113,29 @@ void fill_layout(PairParams& p, const GemmArgs& g, const RunContext& ctx)
     p.b_kstep = g.b_col ? 2u : (2048u >> 4);
 }
 
+// Rounds of 256-row tiles against rounds of 512-row tiles.  A k-paired stage (two k-blocks of a 256 x 256 tile) takes
+// ~1100 clocks in a single round and ~1170 when the launch runs several (a third more L2 traffic per flop than 512-row
+// tiles), and a tile leaves ~1.2 k clocks unhidden - its drain overlaps the next tile's MMAs; a 512 x 256 tile takes
+// 1035 per k-block and leaves 3.6 k.  Twice the tiles in fewer than twice the rounds is what pays: 3584^3 70.7 us against
+// 77.3 (three rounds against two), 2560 x 4096 x 4096 76.8 / 84.5, BMM 32 x 1024^3 60.4 / 62.4 (seven against four),
+// ragged groups 201 / 219; with both counts a whole number of rounds (4096^3: four against two) 100 against 94.
+bool pair_k_paired_faster(int64_t tiles256, int64_t tiles512, int64_t nkb, int64_t pairs)
+{
+    if (pairs <= 0 || nkb < 16) return false;
+    const int64_t r256 = (tiles256 + pairs - 1) / pairs, r512 = (tiles512 + pairs - 1) / pairs;
+    const double t256 = static_cast<double>(r256) * (static_cast<double>((nkb + 1) / 2) * (r256 > 1 ? 1170.0 : 1100.0) + 1200.0);
+    const double t512 = static_cast<double>(r512) * (static_cast<double>(nkb) * 1035.0 + 3600.0);
+    return t256 < 0.97 * t512;
+}
+
+// Batched and grouped launches: k-paired 256-row tiles when the plan that names the pair kernel asks for them
+// (stages 3), and by the estimate above when no plan names a kernel.
+bool pair_k_paired_multi(const RunContext& ctx, int64_t tiles256, int64_t tiles512, int64_t nkb)
+{
+    if (ctx.plan.kernel == 2) return ctx.plan.stages == 3;
+    return ctx.plan.kernel == 0 && pair_k_paired_faster(tiles256, tiles512, nkb, ctx.sm_count / 2);
+}
+
 bool c_takes_tma_store(const GemmArgs& g)
 {
     const int celt = g.c_bf16 ? 2 : 4;
@@ -1138,13 +1163,17 @@ cudaError_t launch_r4_pair_batched(const GemmArgs& g, const BatchArgs& b, RunCon
     PairParams p;
     memset(&p, 0, sizeof p);
     fill_layout(p, g, ctx);
-    p.tiles_m2 = (g.M + TILE_M - 1) / TILE_M;
+    const int64_t tn = (g.N + PN - 1) / PN;
+    const bool kp = pair_k_paired_multi(ctx, (g.M + 2 * PM - 1) / (2 * PM) * tn * b.batch, (g.M + TILE_M - 1) / TILE_M * tn * b.batch,
+                                        (g.K + BK - 1) / BK);
+    p.tiles_m2 = kp ? (g.M + 2 * PM - 1) / (2 * PM) : (g.M + TILE_M - 1) / TILE_M;
     p.tiles_n = (g.N + PN - 1) / PN;
     p.tiles_per_batch = p.tiles_m2 * p.tiles_n;
     p.total_tiles = static_cast<int64_t>(p.tiles_per_batch) * b.batch;
-    p.stage_tx = 2 * kStageBytes;
+    p.stage_tx = kp ? 2 * 4 * kABlockBytes : 2 * kStageBytes;
     p.b_boxes = 2;
     p.nkb = (g.K + BK - 1) / BK;
+    if (kp) p.nkb = (p.nkb + 1) / 2;        // stages of two k-blocks
     const int celt = g.c_bf16 ? 2 : 4;
     p.stride_c_bytes = b.stride_c * celt;
     p.epi_tma = (c_takes_tma_store(g) && p.stride_c_bytes % 16 == 0 && p.stride_c_bytes > 0 &&
@@ -1169,10 +1198,13 @@ cudaError_t launch_r4_pair_batched(const GemmArgs& g, const BatchArgs& b, RunCon
                                  g.C, g.N, g.M, nb, g.ldc * celt, static_cast<uint64_t>(p.stride_c_bytes),
                                  g.c_bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return cudaErrorInvalidValue;
-    p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + 32 + ctx.kid_flags;
+    p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + 32 + (kp ? 256 : 0) + ctx.kid_flags;
     *kernel_id = p.kid;
     const int64_t max_pairs = ctx.sm_count / 2;
     const unsigned grid = 2u * static_cast<unsigned>(p.total_tiles < max_pairs ? p.total_tiles : max_pairs);
+    if (kp)
+        return g.b_col ? launch<true, 7>(g, ma, mb, mc, p, grid, ctx.device, stream)
+                       : launch<false, 7>(g, ma, mb, mc, p, grid, ctx.device, stream);
     return g.b_col ? launch<true, 1>(g, ma, mb, mc, p, grid, ctx.device, stream)
                    : launch<false, 1>(g, ma, mb, mc, p, grid, ctx.device, stream);
 }
@@ -1199,11 +1231,19 @@ cudaError_t launch_r4_pair_grouped(const GemmArgs* groups, int n, RunContext& ct
     // them go to the END of the schedule, and odd rounds run over the pairs in reverse: the pairs that got a full
     // tile in the last full round get the half tiles last.  (Dealt round-robin in group order, a G = 8 launch of
     // 320 tiles kept some pairs busy for 5 tiles' time where 4 suffice.)
+    int64_t t256 = 0, t512 = 0, nkb_max = 0;
+    for (int i = 0; i < n; ++i) {
+        const int64_t tn = (groups[i].N + PN - 1) / PN;
+        t256 += (groups[i].M + 2 * PM - 1) / (2 * PM) * tn;
+        t512 += (groups[i].M + TILE_M - 1) / TILE_M * tn;
+        nkb_max = std::max<int64_t>(nkb_max, (groups[i].K + BK - 1) / BK);
+    }
+    const bool kp = pair_k_paired_multi(ctx, t256, t512, nkb_max);        // 256-row tiles: no tile row is worth splitting off
     GemmArgs* ents = new (std::nothrow) GemmArgs[2 * n];
     if (!ents) return cudaErrorMemoryAllocation;
     int n_full = 0, n_half = 0;
     GemmArgs* halves = ents + n;
-    for (int i = 0; i < n; ++i) {
+    for (int i = 0; i < n && !kp; ++i) {
         const GemmArgs& g = groups[i];
         const int rem = g.M % TILE_M;
         if (rem == 0 || rem > 2 * PM) {
@@ -1251,6 +1291,10 @@ cudaError_t launch_r4_pair_grouped(const GemmArgs* groups, int n, RunContext& ct
         e.K = g.K;
         e.nkb = (g.K + BK - 1) / BK;
         e.tiles_m = (g.M + TILE_M - 1) / TILE_M;
+        if (kp) {
+            e.nkb = (e.nkb + 1) / 2;        // stages of two k-blocks
+            e.tiles_m = (g.M + 2 * PM - 1) / (2 * PM);
+        }
         e.tiles_n = (g.N + PN - 1) / PN;
         e.tile_start = tile_start;
         tile_start += e.tiles_m * e.tiles_n;
@@ -1282,15 +1326,18 @@ cudaError_t launch_r4_pair_grouped(const GemmArgs* groups, int n, RunContext& ct
     p.n_groups = n;
     p.total_tiles = tile_start;
     p.snake = reorder ? 1 : 0;
-    p.stage_tx = 2 * kStageBytes;
+    p.stage_tx = kp ? 2 * 4 * kABlockBytes : 2 * kStageBytes;
     p.b_boxes = 2;
     p.epi_tma = any_tma ? 1 : 0;
-    p.kid = kIdTcgen05 + (any_tma ? 0 : 2) + 32 + ctx.kid_flags;
+    p.kid = kIdTcgen05 + (any_tma ? 0 : 2) + 32 + (kp ? 256 : 0) + ctx.kid_flags;
     *kernel_id = p.kid;
     const int64_t max_pairs = ctx.sm_count / 2;
     const unsigned grid = 2u * static_cast<unsigned>(p.total_tiles < max_pairs ? p.total_tiles : max_pairs);
     CUtensorMap none;
     memset(&none, 0, sizeof none);
+    if (kp)
+        return g0.b_col ? launch<true, 8>(g0, none, none, none, p, grid, ctx.device, stream)
+                        : launch<false, 8>(g0, none, none, none, p, grid, ctx.device, stream);
     return g0.b_col ? launch<true, 2>(g0, none, none, none, p, grid, ctx.device, stream)
                     : launch<false, 2>(g0, none, none, none, p, grid, ctx.device, stream);
 }
@@ -1460,17 +1507,28 @@ bool pair_k_paired(const GemmArgs& g, const RunContext& ctx)
 }
 }
 
-// One round of 256 x 256 tiles that fills more than half of the CTA pairs, K long enough to pay for the pair kernel's
-// set-up.  Measured (single launches after an L2 flush, against the single-CTA kernel's one wave of 128 x 256 tiles):
-// 2048 x 2048 x 8192 56.2 against 61.4 us, 512 x 8192 x 8192 61.5 / 65.5, 1536 x 2048 x 4096 32.8 / 34.8, 2304 x 2048 x
-// 6144 45.6 / 49.1, 2048 x 2048 x 3072 28.2 / 28.8; with 32 tiles (1024 x 2048 x 8192) 54 against 42 for the
-// single-CTA kernel's cluster split, and in several rounds (4096^3) 100 against 94 for 512-row tiles.
+// One problem, nothing pinned.  One round of 256 x 256 tiles that fills more than half of the CTA pairs, K long enough
+// to pay for the pair kernel's set-up - measured (single launches after an L2 flush, against the single-CTA kernel's one
+// wave of 128 x 256 tiles): 2048 x 2048 x 8192 56.2 against 61.4 us, 512 x 8192 x 8192 61.5 / 65.5, 1536 x 2048 x 4096
+// 32.8 / 34.8, 2304 x 2048 x 6144 45.6 / 49.1, 2048 x 2048 x 3072 28.2 / 28.8; with 32 tiles (1024 x 2048 x 8192) 54
+// against 42 for the single-CTA kernel's cluster split.  Several rounds: when they beat the 512-row tiles' rounds
+// (pair_k_paired_faster) and the single-CTA kernel's waves at the ~700 clocks per k-block it takes with every SM busy
+// (3072 x 4096 x 2048: 46.1 against 50.2 and 52.2 us).
 bool r4_pair_k_paired_auto(const GemmArgs& g, const RunContext& ctx)
 {
-    if (!r4_pair_possible(g, ctx) || g.M <= 2 * PM || g.K < 3072) return false;
-    const int64_t tiles = static_cast<int64_t>((g.M + 2 * PM - 1) / (2 * PM)) * ((g.N + PN - 1) / PN);
+    if (!r4_pair_possible(g, ctx) || g.M <= 2 * PM) return false;
+    const int64_t tn = (g.N + PN - 1) / PN;
+    const int64_t tiles = static_cast<int64_t>((g.M + 2 * PM - 1) / (2 * PM)) * tn;
     const int64_t pairs = ctx.sm_count / 2;
-    return tiles <= pairs && 2 * tiles > pairs;
+    if (tiles <= pairs) return 2 * tiles > pairs && g.K >= 3072;
+    const int64_t nkb = (g.K + BK - 1) / BK;
+    if (!pair_k_paired_faster(tiles, static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * tn, nkb, pairs)) return false;
+    const int64_t r256 = (tiles + pairs - 1) / pairs;
+    const double t256 = static_cast<double>(r256) * (static_cast<double>((nkb + 1) / 2) * 1170.0 + 1200.0);
+    const int64_t tiles1 = static_cast<int64_t>((g.M + PM - 1) / PM) * tn;
+    const int64_t full = tiles1 / ctx.sm_count, tail = tiles1 % ctx.sm_count;
+    const double waves = full + (tail == 0 ? 0.0 : (2 * tail <= ctx.sm_count && g.N > PN / 2 ? 0.75 : 1.0));
+    return t256 < waves * static_cast<double>(nkb) * 700.0;
 }
 
 bool r4_pair_stream_k_possible(const GemmArgs& g, const RunContext& ctx)

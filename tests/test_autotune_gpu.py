@@ -66,10 +66,12 @@ def test_every_candidate_plan_matches_the_oracle(kb, shape):
                 vals, bits, kid = run_plan(kb, g, case, dev, plan)
                 P.assert_matches_oracle(case, vals, bits, C_ref, S, exact=integer, what=f"{case.name} {plan}")
                 flags = kid - 400
-                assert 0 <= flags < 128, kid
+                assert 0 <= flags < 512, kid
                 kernels.add(bool(flags & 32))
                 if plan.kernel == 2:
                     assert flags & 32, f"{plan} ran kernel {kid}"
+                    assert bool(flags & 128) == (plan.split_via == 3), f"{plan} ran kernel {kid}"
+                    assert bool(flags & 256) == (plan.stages == 3), f"{plan} ran kernel {kid}"
                 if plan.kernel == 1:
                     assert not flags & 32, f"{plan} ran kernel {kid}"
                 if plan.splits > 1:

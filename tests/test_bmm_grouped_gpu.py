@@ -77,12 +77,20 @@ class Batch:
         return out
 
 
-def check_batch(kb, bt, variant, exact, want_pair=None, one_launch=None, kernel=0):
-    """kernel: 1 / 2 pins the single-CTA / CTA-pair kernel for the per-problem shape first."""
+def plan_of(kernel):
+    """A kernel number (1 single-CTA, 2 CTA pair) or a whole plan as a tuple."""
+    return kernel if isinstance(kernel, tuple) else (kernel, 1, 0, 0, 0)
+
+
+K_PAIRED = (2, 1, 0, 0, 0, 0, 0, 3)     # the CTA-pair kernel on 256-row tiles, two k-blocks per stage
+
+
+def check_batch(kb, bt, variant, exact, want_pair=None, one_launch=None, kernel=0, want_k_paired=None):
+    """kernel: 1 / 2 pins the single-CTA / CTA-pair kernel for the per-problem shape first (a tuple: that plan)."""
     c0 = bt.cases[0]
     with kb.Gemm(0, b_col_major=c0.b_col_major, c_bf16=c0.c_bf16) as g:
         if kernel:
-            g.set_plan(kb.klineage_gemm_plan_t(kernel, 1, 0, 0, 0), bt.a.ptr, bt.b.ptr, bt.c.ptr, c0.M, c0.N, c0.K,
+            g.set_plan(kb.klineage_gemm_plan_t(*plan_of(kernel)), bt.a.ptr, bt.b.ptr, bt.c.ptr, c0.M, c0.N, c0.K,
                        c0.lda, c0.ldb, c0.ldc)
         bt.run(g, variant)
         kid = g.last_kernel_id()
@@ -95,6 +103,8 @@ def check_batch(kb, bt, variant, exact, want_pair=None, one_launch=None, kernel=
                                     what=f"{case.name} {VARIANT_NAMES[variant]} batch {b}")
         if want_pair is not None:
             assert bool((kid - 400) & 32) == want_pair, kid
+        if want_k_paired is not None:
+            assert bool((kid - 400) & 256) == want_k_paired, kid
         # the same problems one by one through klineage_gemm_run
         for b, case in enumerate(bt.cases):
             dev = P.DeviceCase(case)
@@ -124,6 +134,26 @@ def test_bmm_one_launch(kb, cfg, kernel):
             continue                      # (the long-K case costs the oracle most; integers cover the pinned kernels)
         bt = Batch(batch, M, N, K, col, bf, dist, seed=70, pad=pad, gap=gap)
         check_batch(kb, bt, 4, exact, want_pair=pair, one_launch=True, kernel=kernel)
+
+
+@pytest.mark.parametrize("cfg", [ONE_LAUNCH[0], ONE_LAUNCH[1], ONE_LAUNCH[3]], ids=lambda c: f"b{c[0]}-{c[1]}x{c[2]}x{c[3]}")
+def test_bmm_k_paired_tiles(kb, cfg):
+    """The batched launch on 256 x 256 pair tiles, two k-blocks per stage: pinned, against the oracle and bit-equal to
+    the problems one by one; K = 136 / 200 / 2056 give an odd number of k-blocks and a ragged last one."""
+    batch, M, N, K, col, bf, pad, gap = cfg
+    for dist, exact in (("integer", True),) + ((("normal", False),) if K < 2048 else ()):
+        bt = Batch(batch, M, N, K, col, bf, dist, seed=75, pad=pad, gap=gap)
+        check_batch(kb, bt, 4, exact, want_pair=True, one_launch=True, kernel=K_PAIRED, want_k_paired=True)
+
+
+def test_bmm_k_paired_tiles_by_default(kb):
+    """Twice the tiles in fewer than twice the rounds: 5 x (1100 x 1104 x 2056) is 75 tiles of 512 x 256 (two rounds on
+    74 CTA pairs) or 125 of 256 x 256 (two rounds as well) - the launch takes the 256-row tiles on its own."""
+    bt = Batch(5, 1100, 1104, 2056, False, True, "integer", seed=76)
+    check_batch(kb, bt, 4, True, want_pair=True, one_launch=True, want_k_paired=True)
+    # a pinned pair kernel without the stage count keeps the 512-row tiles
+    bt = Batch(5, 1100, 1104, 2056, False, True, "integer", seed=76)
+    check_batch(kb, bt, 4, True, want_pair=True, one_launch=True, kernel=2, want_k_paired=False)
 
 
 def test_bmm_problem_by_problem_paths(kb):
@@ -165,7 +195,7 @@ def test_bmm_argument_rules(kb):
 
 
 # ---------------------------------------------------------------------------- grouped
-def run_grouped(kb, cases, variant, exact, want_pair=None, one_launch=None, kernel=0):
+def run_grouped(kb, cases, variant, exact, want_pair=None, one_launch=None, kernel=0, want_k_paired=None):
     import torch
     c0 = cases[0]
     devs = [P.DeviceCase(c) for c in cases]
@@ -173,7 +203,7 @@ def run_grouped(kb, cases, variant, exact, want_pair=None, one_launch=None, kern
         if kernel:
             first = next(i for i, c in enumerate(cases) if c.M and c.N)
             c, d = cases[first], devs[first]
-            g.set_plan(kb.klineage_gemm_plan_t(kernel, 1, 0, 0, 0), d.a.ptr, d.b.ptr, d.c.ptr, c.M, c.N, c.K, c.lda,
+            g.set_plan(kb.klineage_gemm_plan_t(*plan_of(kernel)), d.a.ptr, d.b.ptr, d.c.ptr, c.M, c.N, c.K, c.lda,
                        c.ldb, c.ldc)
         g.run_grouped([d.a.ptr for d in devs], [d.b.ptr for d in devs], [d.c.ptr for d in devs],
                       [c.M for c in cases], [c.N for c in cases], [c.K for c in cases],
@@ -186,6 +216,8 @@ def run_grouped(kb, cases, variant, exact, want_pair=None, one_launch=None, kern
             assert (g.last_launch_count() == 1) == one_launch, g.last_launch_count()
         if want_pair is not None:
             assert bool((kid - 400) & 32) == want_pair, kid
+        if want_k_paired is not None:
+            assert bool((kid - 400) & 256) == want_k_paired, kid
         got = [d.result() for d in devs]
         for case, (vals, bits) in zip(cases, got):
             if case.M == 0 or case.N == 0:
@@ -288,4 +320,6 @@ def test_grouped_ragged_rows_on_the_pair_kernel(kb):
         cases = [gen.make_case(M, N, K, seed=170 + i, dist_a="integer", dist_b="integer", b_col_major=col, c_bf16=bf,
                                ldc=N + (8 if i % 3 == 0 else 0), name=f"gr{i}-{M}x{N}x{K}")
                  for i, (M, N, K) in enumerate(shapes)]
-        run_grouped(kb, cases, 4, True, want_pair=True, one_launch=True, kernel=2)
+        run_grouped(kb, cases, 4, True, want_pair=True, one_launch=True, kernel=2, want_k_paired=False)
+        # the same groups on 256-row tiles (no tile row is split off: every tile is one row block)
+        run_grouped(kb, cases, 4, True, want_pair=True, one_launch=True, kernel=K_PAIRED, want_k_paired=True)
