@@ -624,7 +624,11 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
         WorkState ws = work_init();
         Work wk;
         for (; ok && next_work(ws, wk); ++tcount) {
-            if (KP && (tcount & 1u) != static_cast<uint32_t>(mb)) continue;     // the other warp group's tile
+            // KP: a tile belongs to the warp group of its parity - except the pair's LAST tile, which both groups drain,
+            // the owner the first half of its 128-byte units and the other group (idle by then) the second half.
+            const int ab = KP ? static_cast<int>(tcount & 1u) : mb;           // the accumulator (KP) / row block read here
+            const bool helper = KP && ab != mb;
+            if (helper && tile_at(ws.i) >= 0) continue;
             const TileInfo x = tile_info(wk.tile);
             const int m0 = x.m0, n0 = x.n0;
             float* dst_f = reinterpret_cast<float*>(x.C);
@@ -632,7 +636,10 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             const int row0 = m0 + (KP ? 0 : mb * 2 * PM) + q * 32;
             const int rows = min(32, x.M - row0);
             const int nunits = (row0 < x.M) ? (min(x.width, x.N - n0) + cpc - 1) / cpc : 0;
-            const uint32_t tbase = tmem_base + mb * PN + (static_cast<uint32_t>(q * 32) << 16);
+            const uint32_t tbase = tmem_base + ab * PN + (static_cast<uint32_t>(q * 32) << 16);
+            const bool shared = KP && nunits >= 2 && tile_at(ws.i) < 0;       // both warp groups drain this tile
+            if (helper && !shared) continue;
+            const int u_lo = (shared && helper) ? nunits / 2 : 0, u_hi = (shared && !helper) ? nunits / 2 : nunits;
             // first 4 KiB block of this warp's rows inside a partial-tile slot: (CTA, row block, lane quarter) x 8 column blocks
             const int64_t sk_block = ((static_cast<int64_t>(rank) * 2 + mb) * 4 + q) * (PN / 32);
 
@@ -673,7 +680,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     break;
                 }
             }
-            if (!ptx::mbar_wait(&acc_full[KP ? mb : 0], (KP ? tcount >> 1 : tcount) & 1, abort_flag)) {
+            if (!ptx::mbar_wait(&acc_full[KP ? ab : 0], (KP ? tcount >> 1 : tcount) & 1, abort_flag)) {
                 if (lane == 0) report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x540u);
                 abort_flag[0] = 1;
                 ok = false;
@@ -687,7 +694,8 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 if (tcount == 0 && warp == kEpiWarp0 && lane == 0) KLIN_T(60);
                 __syncwarp();
                 if (tcount == 0 && warp == kEpiWarp0 && lane == 0) KLIN_T(61);
-                if (lane == 0) mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&acc_empty[KP ? mb : 0]), 0));
+                // (a shared tile is the pair's last: nobody waits for its accumulator)
+                if (lane == 0 && !shared) mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&acc_empty[KP ? ab : 0]), 0));
             };
             auto issue = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32]) {
                 ptx::tmem_ld_32x32b_x32(tbase + u * cpc, r0);
@@ -931,7 +939,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 }
                 continue;
             }
-            if (out_bf16 && nunits == 4 && n_part == 0) {
+            if (out_bf16 && nunits == 4 && n_part == 0 && !shared) {
                 // Full-width bf16 tile: the accumulator is handed back before anything is staged or stored.
                 // Rounding (F2F, 16 results per clock and SM) is what the drain costs: three units are read
                 // raw (192 registers), one is rounded to make room for the fourth, the accumulator is
@@ -961,7 +969,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 if (warp == kEpiWarp0 && lane == 0) KLIN_T(tcount < 8 ? 42 + 3 * static_cast<int>(tcount) : -1);
                 continue;
             }
-            if (!out_bf16 && nunits == 8 && n_part == 0) {
+            if (!out_bf16 && nunits == 8 && n_part == 0 && !shared) {
                 // Full-width fp32 tile (eight 32-column units, nothing to round): six units are read raw, two
                 // are staged and stored to make room for the last two, then the accumulator is released.
                 uint32_t d0[32], d1[32];
@@ -994,18 +1002,18 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 stage_store(7, a1);
                 continue;
             }
-            issue(0, a0, a1);
-            for (int u = 0; u < nunits; u += 2) {
+            if (u_lo < u_hi) issue(u_lo, a0, a1);
+            for (int u = u_lo; u < u_hi; u += 2) {
                 ptx::tmem_ld_wait();
-                if (u + 1 < nunits) issue(u + 1, c0, c1); else release();
+                if (u + 1 < u_hi) issue(u + 1, c0, c1); else release();
                 {
                     uint32_t w[32];
                     pack(u, a0, a1, w);
                     stage_store(u, w);
                 }
-                if (u + 1 < nunits) {
+                if (u + 1 < u_hi) {
                     ptx::tmem_ld_wait();
-                    if (u + 2 < nunits) issue(u + 2, a0, a1); else release();
+                    if (u + 2 < u_hi) issue(u + 2, a0, a1); else release();
                     uint32_t w[32];
                     pack(u + 1, c0, c1, w);
                     stage_store(u + 1, w);
