@@ -1081,24 +1081,33 @@ bool r4_pair_possible(const GemmArgs& g, const RunContext& ctx)
     return ok2(g.A, g.lda) && ok2(g.B, g.ldb);
 }
 
+// Estimated cycles of the single-CTA kernel's schedule: per wave of 128 x 256 tiles 580 per k-block (the issuing
+// thread and the shared-memory port; the epilogue hides behind the next tile) plus ~4 k that no main loop hides; a
+// launch that is one under-filled wave cut into half tiles counts 0.8.  Fitted to graph replays (operands in the L2)
+// of 1536^3 ... 2560^3, 4096 x 4096 x {256, 512, 1024}, 8192 x 8192 x {128, 512}.
+static double single_schedule_cycles(const GemmArgs& g, const RunContext& ctx)
+{
+    const int64_t nkb = (g.K + BK - 1) / BK;
+    const int64_t tiles1 = static_cast<int64_t>((g.M + PM - 1) / PM) * ((g.N + PN - 1) / PN);
+    const int64_t full = tiles1 / ctx.sm_count, tail = tiles1 % ctx.sm_count;
+    const double waves = full + (tail == 0 ? 0.0 : (full == 0 && 2 * tail <= ctx.sm_count && g.N > PN / 2 ? 0.8 : 1.0));
+    return waves * (4000.0 + 580.0 * static_cast<double>(nkb));
+}
+
 bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx)
 {
     if (!r4_pair_possible(g, ctx) || g.M <= 2 * PM) return false;
-    // Which kernel finishes first?  Estimated tensor-pipe cycles of either schedule, from measured rates:
-    // a 512 x 256 pair tile takes ~1035 cycles per k-block (two accumulators alternate: full rate) plus
-    // ~3.6 k cycles per tile that the main loop does not hide (accumulator drain, barrier round trips); a 128 x 256
-    // tile of the single-CTA kernel takes 636 per k-block (its issuing thread and the shared-memory port) with its epilogue
-    // hidden, and a last wave of at most half of the SMs is cut into half tiles worth ~0.75 of a wave.
-    // Fitted to both kernels timed at 2048^3 .. 4096^3 (steps of 256), 2048 x 4096 x 4096 and 3072 x 2048 x 8192.
+    // Which kernel finishes first?  Estimated cycles of either schedule, from measured rates: a 512 x 256 pair tile
+    // takes ~1035 cycles per k-block (two accumulators alternate: full rate) plus ~3.6 k cycles per tile that the main
+    // loop does not hide (accumulator drain, barrier round trips); the single-CTA kernel as estimated above.  Timed
+    // with operands in the L2 (graph replay) and after an L2 flush; the rule follows the former where they disagree
+    // (2304^3: 26.3 against 31.2 us warm, 31.6 / 36.9 cold; 4096 x 4096 x 1024 28.1 / 31.2 and 33.7 / 37.9; 8192 x 8192
+    // x 128 29.7 / 40.5 and 33.6 / 45.1; 2048^3 23.8 / 16.7 and 29.7 / 23.0 - the single-CTA kernel's).
     const int64_t nkb = (g.K + BK - 1) / BK;
     const int64_t pairs = ctx.sm_count / 2;
     const int64_t tiles2 = static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * ((g.N + PN - 1) / PN);
     const double t_pair = static_cast<double>((tiles2 + pairs - 1) / pairs) * (nkb * 1035.0 + 3600.0);
-    const int64_t tiles1 = static_cast<int64_t>((g.M + PM - 1) / PM) * ((g.N + PN - 1) / PN);
-    const int64_t full = tiles1 / ctx.sm_count, tail = tiles1 % ctx.sm_count;
-    const double waves = full + (tail == 0 ? 0.0 : (2 * tail <= ctx.sm_count && g.N > PN / 2 ? 0.75 : 1.0));
-    const double t_single = waves * nkb * 636.0;
-    return t_pair < t_single;
+    return t_pair < single_schedule_cycles(g, ctx);
 }
 
 namespace {
@@ -1520,7 +1529,7 @@ bool pair_k_paired(const GemmArgs& g, const RunContext& ctx)
 // wave of 128 x 256 tiles): 2048 x 2048 x 8192 56.2 against 61.4 us, 512 x 8192 x 8192 61.5 / 65.5, 1536 x 2048 x 4096
 // 32.8 / 34.8, 2304 x 2048 x 6144 45.6 / 49.1, 2048 x 2048 x 3072 28.2 / 28.8; with 32 tiles (1024 x 2048 x 8192) 54
 // against 42 for the single-CTA kernel's cluster split.  Several rounds: when they beat the 512-row tiles' rounds
-// (pair_k_paired_faster) and the single-CTA kernel's waves at the ~700 clocks per k-block it takes with every SM busy
+// (pair_k_paired_faster) and the single-CTA kernel's estimate
 // (3072 x 4096 x 2048: 46.1 against 50.2 and 52.2 us).
 bool r4_pair_k_paired_auto(const GemmArgs& g, const RunContext& ctx)
 {
@@ -1533,10 +1542,7 @@ bool r4_pair_k_paired_auto(const GemmArgs& g, const RunContext& ctx)
     if (!pair_k_paired_faster(tiles, static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * tn, nkb, pairs)) return false;
     const int64_t r256 = (tiles + pairs - 1) / pairs;
     const double t256 = static_cast<double>(r256) * (static_cast<double>((nkb + 1) / 2) * 1170.0 + 1200.0);
-    const int64_t tiles1 = static_cast<int64_t>((g.M + PM - 1) / PM) * tn;
-    const int64_t full = tiles1 / ctx.sm_count, tail = tiles1 % ctx.sm_count;
-    const double waves = full + (tail == 0 ? 0.0 : (2 * tail <= ctx.sm_count && g.N > PN / 2 ? 0.75 : 1.0));
-    return t256 < waves * static_cast<double>(nkb) * 700.0;
+    return t256 < single_schedule_cycles(g, ctx);
 }
 
 bool r4_pair_stream_k_possible(const GemmArgs& g, const RunContext& ctx)

@@ -352,8 +352,8 @@ def test_tcgen05_cta_pair_k_paired_tiles(handles, col):
 def test_dispatch_between_the_two_kernels(handles):
     """Long K and enough 512 x 256 (or 256 x 256) tiles: the pair kernel; short K or few tiles: the single-CTA kernel."""
     for (M, N, K), want_pair in (((2048, 4096, 4096), True), ((3072, 2048, 8192), True), ((2816, 2816, 2816), True),
-                                 ((2048, 2048, 2048), False), ((4608, 4352, 72), False), ((3584, 3584, 3584), True),    # (three rounds of 256-row tiles)
-                                 ((2304, 2304, 2304), False),
+                                 ((2048, 2048, 2048), False), ((1536, 3072, 1024), False), ((3584, 3584, 3584), True),    # (three rounds of 256-row tiles)
+                                 ((2304, 2304, 2304), True), ((1536, 1536, 1536), False), ((4096, 4096, 512), True),
                                  ((2048, 2048, 8192), True),       # one round of 64 k-paired 256-row tiles
                                  ((1024, 2048, 8192), False)):     # 32 such tiles: the single-CTA kernel's cluster split
         case = gen.make_case(M, N, K, seed=70, dist_a="integer", dist_b="integer", c_bf16=True, name=f"disp{M}x{N}x{K}")
@@ -387,6 +387,10 @@ def test_midsize_shapes(handles, variant):
         C_ref, S = P.oracle_rows(case, rows)
         vals, _ = run_and_check(handles, case, variant, C_ref, S, rows, exact=True)
         assert P.integer_checksums_match(case, vals), case.name
+        if variant == 4:
+            # the schedule named above is the single-CTA kernel's: run it there whatever the dispatch rule prefers
+            run_and_check(handles, case, variant, C_ref, S, rows, exact=True, pin=(1, 0, 0, 0, 0))
+            assert not (handles[(col, False)].last_kernel_id() - 400) & 32
         case = gen.make_case(M, N, K, seed=80 + idx, dist_a="normal", dist_b="uniform", b_col_major=not col, c_bf16=bf,
                              name=f"mid{M}x{N}x{K}")
         C_ref, S = P.oracle_rows(case, rows)
