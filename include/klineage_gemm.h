@@ -285,14 +285,15 @@ klineage_status_t klineage_gemm_run_noalloc(int b_layout, int c_dtype, int64_t M
  * grouped: a table of per-group tensor maps and sizes, built in the handle's
  * workspace and copied on `stream` ahead of the kernel; at most 256 groups per
  * launch) when they fill at least half of the SMs: on the CTA-pair kernel
- * (512 x 256 tiles) when K >= 1024 and either every problem has more than 256
- * rows or rounding every group's rows up to a multiple of 256 adds at most a
- * quarter (a pair tile with at most 256 live rows does half the work; such
- * last tile rows of the groups are scheduled last; 256 x 256 tiles instead when
- * twice the tiles take fewer than twice the rounds over the CTA pairs - see
- * `stages` of the launch plan), else on the single-CTA
- * kernel (128 x 256 tiles, whose double-buffered accumulator hides the epilogue
- * that short K exposes); a plan pinned for the shape of the (first) problem
+ * (512 x 256 tiles, or 256 x 256 tiles when twice the tiles take fewer than
+ * twice the rounds over the CTA pairs - see `stages` of the launch plan) or on
+ * the single-CTA kernel (128 x 256 tiles, whose double-buffered accumulator
+ * hides the epilogue), whichever schedule the rung's cycle estimate makes the
+ * shorter over all problems of the call; grouped calls take the pair kernel
+ * only when every problem has more than 256 rows or rounding every group's
+ * rows up to a multiple of 256 adds at most a quarter (with 512-row tiles, a
+ * tile with at most 256 live rows does half the work and such last tile rows
+ * of the groups are scheduled last).  A plan pinned for the shape of the (first) problem
  * may name the kernel.  Every other case - lower
  * rungs, unaligned operands, a K == 0 group, too few tiles - runs the rung's
  * ordinary path once per problem, in order, on `stream`.

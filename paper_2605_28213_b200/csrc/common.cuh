@@ -247,6 +247,8 @@ cudaError_t launch_r35_mma_sync(const GemmArgs& g, RunContext& ctx, cudaStream_t
 cudaError_t launch_zero_fill(const GemmArgs& g, cudaStream_t stream, int* kernel_id);
 // CTA-pair (cta_group::2) form of rung 4 and the test of its preconditions.
 bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx);
+// The same estimate for a batched or grouped launch, on its tile counts (128 x 256 / 256 x 256 / 512 x 256) and longest K.
+bool r4_pair_faster_multi(int64_t tiles128, int64_t tiles256, int64_t tiles512, int64_t nkb, const RunContext& ctx);
 // Whether an unpinned single-destination launch takes the pair kernel's k-paired 256-row tiles.
 bool r4_pair_k_paired_auto(const GemmArgs& g, const RunContext& ctx);
 // Hard preconditions of the CTA-pair kernel only (operands TMA-loadable), without the size heuristic.

@@ -562,9 +562,9 @@ klineage_status_t klineage_gemm_run_batched(klineage_gemm_t h, int64_t batch, in
         ba.stride_a = stride_a;
         ba.stride_b = stride_b;
         ba.stride_c = stride_c;
-        // The CTA-pair kernel (512 x 256 tiles, both accumulators in use) for K of 1024 and more; the single-CTA
-        // kernel (128 x 256 tiles, double-buffered accumulator) for short K and small problems.  A plan
-        // pinned for the per-problem shape decides the kernel when it names one.
+        // The CTA-pair kernel (512 x 256 or 256 x 256 tiles) or the single-CTA kernel (128 x 256 tiles), whichever the
+        // cycle estimate of the two schedules favours over the whole batch.  A plan pinned for the per-problem shape
+        // decides the kernel when it names one.
         const int half_sm = h->ctx.sm_count / 2;
         const int64_t pair_tiles = ((M + 511) / 512) * ((N + 255) / 256) * batch;
         const int64_t single_tiles = ((M + 127) / 128) * ((N + 255) / 256) * batch;
@@ -578,7 +578,7 @@ klineage_status_t klineage_gemm_run_batched(klineage_gemm_t h, int64_t batch, in
             want = 2;
         else if (pinned.kernel == 1 && single_ok)
             want = 1;
-        else if (pair_ok && K >= 1024)     // (measured 32 x 1024^3: 66.6 us against 68.6; 64 x 512^3: 31.7 against 29.7)
+        else if (pair_ok && r4_pair_faster_multi(single_tiles, ((M + 255) / 256) * ((N + 255) / 256) * batch, pair_tiles, (K + 63) / 64, h->ctx))
             want = 2;
         else if (single_ok)
             want = 1;
@@ -654,8 +654,9 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups, const
         GemmArgs* ga = new (std::nothrow) GemmArgs[groups];
         if (!ga) return KLINEAGE_ERR_ALLOC;
         int n = 0, first = -1;
-        bool launchable = true, all_tall = true, all_long = true;
-        int64_t pair_tiles = 0, single_tiles = 0, rows = 0, rows_by_256 = 0;
+        bool launchable = true, all_tall = true;
+        int64_t k_max = 0;
+        int64_t pair_tiles = 0, kp_tiles = 0, single_tiles = 0, rows = 0, rows_by_256 = 0;
         for (int i = 0; i < groups; ++i) {
             if (M[i] == 0 || N[i] == 0) continue;
             if (K[i] == 0) {            // a zero-fill group: leave the whole call to the ordinary path
@@ -668,8 +669,9 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups, const
             rows += M[i];
             rows_by_256 += (M[i] + 255) / 256 * 256;
             all_tall = all_tall && M[i] > 256;
-            all_long = all_long && K[i] >= 1024;
+            k_max = K[i] > k_max ? K[i] : k_max;
             pair_tiles += ((M[i] + 511) / 512) * ((N[i] + 255) / 256);
+            kp_tiles += ((M[i] + 255) / 256) * ((N[i] + 255) / 256);
             single_tiles += ((M[i] + 127) / 128) * ((N[i] + 255) / 256);
         }
         launchable = launchable && n >= 1 && n <= kMaxGroups;
@@ -691,7 +693,7 @@ klineage_status_t klineage_gemm_run_grouped(klineage_gemm_t h, int groups, const
             want = 2;
         else if (pinned.kernel == 1 && single_ok)
             want = 1;
-        else if (pair_ok && all_long && all_tall)
+        else if (pair_ok && all_tall && r4_pair_faster_multi(single_tiles, kp_tiles, pair_tiles, (k_max + 63) / 64, h->ctx))
             want = 2;
         else if (single_ok)
             want = 1;

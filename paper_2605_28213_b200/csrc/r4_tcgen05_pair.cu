@@ -1085,13 +1085,30 @@ bool r4_pair_possible(const GemmArgs& g, const RunContext& ctx)
 // thread and the shared-memory port; the epilogue hides behind the next tile) plus ~4 k that no main loop hides; a
 // launch that is one under-filled wave cut into half tiles counts 0.8.  Fitted to graph replays (operands in the L2)
 // of 1536^3 ... 2560^3, 4096 x 4096 x {256, 512, 1024}, 8192 x 8192 x {128, 512}.
+static double single_schedule_cycles(int64_t tiles1, int64_t nkb, bool halves, const RunContext& ctx)
+{
+    const int64_t full = tiles1 / ctx.sm_count, tail = tiles1 % ctx.sm_count;
+    const double waves = full + (tail == 0 ? 0.0 : (full == 0 && 2 * tail <= ctx.sm_count && halves ? 0.8 : 1.0));
+    return waves * (4000.0 + 580.0 * static_cast<double>(nkb));
+}
 static double single_schedule_cycles(const GemmArgs& g, const RunContext& ctx)
 {
-    const int64_t nkb = (g.K + BK - 1) / BK;
-    const int64_t tiles1 = static_cast<int64_t>((g.M + PM - 1) / PM) * ((g.N + PN - 1) / PN);
-    const int64_t full = tiles1 / ctx.sm_count, tail = tiles1 % ctx.sm_count;
-    const double waves = full + (tail == 0 ? 0.0 : (full == 0 && 2 * tail <= ctx.sm_count && g.N > PN / 2 ? 0.8 : 1.0));
-    return waves * (4000.0 + 580.0 * static_cast<double>(nkb));
+    return single_schedule_cycles(static_cast<int64_t>((g.M + PM - 1) / PM) * ((g.N + PN - 1) / PN), (g.K + BK - 1) / BK,
+                                  g.N > PN / 2, ctx);
+}
+
+// Batched and grouped launches: the same comparison on the launch's tile counts (128 x 256 and 512 x 256 tiles over all
+// problems, the longest K).  Measured cold / warm in us, single-CTA against pair: BMM 32 x 1024 x 1024 x 512 41.8 / 37.6
+// against 41.7 / 36.8, 16 x 2048 x 2048 x 512 69.7 / 69.3 against 62.4 / 62.8, 32 x 1024 x 1024 x 256 31.7 / 27.0 against
+// 28.7 / 24.2, 24 x 768 x 3072 x 768 85.0 / 83.9 against 82.9 / 84.5 (73.8 / 77.6 on 256-row tiles).
+bool r4_pair_faster_multi(int64_t tiles128, int64_t tiles256, int64_t tiles512, int64_t nkb, const RunContext& ctx)
+{
+    const int64_t pairs = ctx.sm_count / 2;
+    if (pairs <= 0) return false;
+    // the pair kernel's better form: 512-row tiles, or 256-row tiles at 1170 per stage of two k-blocks + 1.2 k per tile
+    const double t512 = static_cast<double>((tiles512 + pairs - 1) / pairs) * (nkb * 1035.0 + 3600.0);
+    const double t256 = static_cast<double>((tiles256 + pairs - 1) / pairs) * (((nkb + 1) / 2) * 1170.0 + 1200.0);
+    return (t512 < t256 ? t512 : t256) < single_schedule_cycles(tiles128, nkb, false, ctx);
 }
 
 bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx)
@@ -1130,18 +1147,19 @@ void fill_layout(PairParams& p, const GemmArgs& g, const RunContext& ctx)
     p.b_kstep = g.b_col ? 2u : (2048u >> 4);
 }
 
-// Rounds of 256-row tiles against rounds of 512-row tiles.  A k-paired stage (two k-blocks of a 256 x 256 tile) takes
-// ~1100 clocks in a single round and ~1170 when the launch runs several (a third more L2 traffic per flop than 512-row
-// tiles), and a tile leaves ~1.2 k clocks unhidden - its drain overlaps the next tile's MMAs; a 512 x 256 tile takes
-// 1035 per k-block and leaves 3.6 k.  Twice the tiles in fewer than twice the rounds is what pays: 3584^3 70.7 us against
+// Rounds of 256-row tiles against rounds of 512-row tiles, for launches of several rounds.  Per tile, fitted to graph
+// replays of batched and single launches (K = 128 ... 4096): 2.4 k + 1350 per stage of two k-blocks for a 256 x 256 tile
+// (its drain overlaps the next tile's MMAs; a third more L2 traffic per flop than the 512-row tile), 3.9 k + 1257 per
+// k-block for a 512 x 256 tile.  Twice the tiles in fewer than twice the rounds is what pays: 3584^3 70.7 us against
 // 77.3 (three rounds against two), 2560 x 4096 x 4096 76.8 / 84.5, BMM 32 x 1024^3 60.4 / 62.4 (seven against four),
-// ragged groups 201 / 219; with both counts a whole number of rounds (4096^3: four against two) 100 against 94.
+// 24 x 768 x 3072 x 768 73.8 / 82.9, ragged groups 201 / 219; with both counts a whole number of rounds (4096^3: four
+// against two) 100 against 94, 8192 x 8192 x 128 32.8 against 29.7.
 bool pair_k_paired_faster(int64_t tiles256, int64_t tiles512, int64_t nkb, int64_t pairs)
 {
-    if (pairs <= 0 || nkb < 16) return false;
+    if (pairs <= 0 || nkb < 1) return false;
     const int64_t r256 = (tiles256 + pairs - 1) / pairs, r512 = (tiles512 + pairs - 1) / pairs;
-    const double t256 = static_cast<double>(r256) * (static_cast<double>((nkb + 1) / 2) * (r256 > 1 ? 1170.0 : 1100.0) + 1200.0);
-    const double t512 = static_cast<double>(r512) * (static_cast<double>(nkb) * 1035.0 + 3600.0);
+    const double t256 = static_cast<double>(r256) * (static_cast<double>((nkb + 1) / 2) * 1350.0 + 2400.0);
+    const double t512 = static_cast<double>(r512) * (static_cast<double>(nkb) * 1257.0 + 3900.0);
     return t256 < 0.97 * t512;
 }
 

@@ -128,7 +128,10 @@ ONE_LAUNCH = [
 @pytest.mark.parametrize("kernel", [0, 1, 2], ids=["default", "single", "pair"])
 def test_bmm_one_launch(kb, cfg, kernel):
     batch, M, N, K, col, bf, pad, gap = cfg
-    pair = (K >= 2048) if kernel == 0 else (kernel == 2)
+    # unpinned: the cycle estimate of the schedules decides - rounds of 512 x 256 or 256 x 256 pair tiles beat the waves
+    # of 128 x 256 tiles at all four shapes (measured: 15.4 against 17.4 us at 5 x 600 x 2104 x 200, 39.8 against 43.0 at
+    # 5 x 1100 x 1104 x 2056)
+    pair = True if kernel == 0 else (kernel == 2)
     for dist, exact in (("integer", True), ("normal", False)):
         if kernel and dist == "normal" and K >= 2048:
             continue                      # (the long-K case costs the oracle most; integers cover the pinned kernels)
@@ -241,14 +244,15 @@ GROUP_SHAPES = [(300, 2048, 136), (1100, 1304, 200), (513, 2000, 64), (700, 1528
 
 
 @pytest.mark.parametrize("col,bf", [(False, True), (True, False)], ids=["row-bf16", "col-f32"])
-@pytest.mark.parametrize("kernel", [0, 2], ids=["default-single", "pair"])
+@pytest.mark.parametrize("kernel", [0, 1, 2], ids=["default", "single", "pair"])
 def test_grouped_one_launch(kb, col, bf, kernel):
     for dist, exact in (("integer", True), ("normal", False)):
         cases = [gen.make_case(M, N, K, seed=100 + i, dist_a=dist, dist_b=dist, b_col_major=col, c_bf16=bf,
                                ldc=N + (4 if i % 2 else 0), name=f"g{i}-{M}x{N}x{K}-{dist}")
                  for i, (M, N, K) in enumerate(GROUP_SHAPES)]
-        # every group has more than 256 rows, so the pair kernel qualifies; K < 2048 makes the single-CTA kernel the default
-        run_grouped(kb, cases, 4, exact, want_pair=kernel == 2, one_launch=True, kernel=kernel)
+        # every group has more than 256 rows, so the pair kernel qualifies, and the cycle estimate prefers it (two rounds
+        # of 256 x 256 tiles against two waves of 128 x 256 tiles)
+        run_grouped(kb, cases, 4, exact, want_pair=kernel != 1, one_launch=True, kernel=kernel)
 
 
 def test_grouped_long_k_takes_the_pair_kernel_and_small_groups_the_single_one(kb):
@@ -272,8 +276,9 @@ def test_grouped_with_an_odd_width_group_uses_masked_stores_for_it(kb):
     for i, (M, N, K) in enumerate(shapes):
         cases.append(gen.make_case(M, N, K, seed=110 + i, dist_a="integer", dist_b="integer", c_bf16=True,
                                    ldb=(N + 7) // 8 * 8, ldc=N + 3, name=f"godd{i}"))
-    run_grouped(kb, cases, 4, True, want_pair=False, one_launch=True)
+    run_grouped(kb, cases, 4, True, want_pair=False, one_launch=True, kernel=1)
     run_grouped(kb, cases, 4, True, want_pair=True, one_launch=True, kernel=2)
+    run_grouped(kb, cases, 4, True, one_launch=True)
 
 
 def test_grouped_problem_by_problem_paths(kb):
