@@ -6,13 +6,14 @@
 // alignment is handled the same way; nothing is vectorized or overlapped yet.
 //
 // Two CTAs share an SM (the register tile is capped at 128 registers per thread for it): one CTA's slab fill overlaps
-// the other's arithmetic, which is all the overlap this rung has (8192^3: 20.3 -> 29.5 TFLOP/s).
+// the other's arithmetic, which is all the overlap this rung has (8192^3: 20.3 -> 29.5 TFLOP/s at the time).
 //
-// A thread's rows are ty + 16 i and its columns tx + 16 j: the 16 threads of a
-// half warp read 16 consecutive words of a shared-memory row (no bank conflict;
-// with columns tx * 8 + j the reads of B were four-way conflicts and the rung ran
-// at a quarter of the fp32 pipe), and a half warp's stores to C are 16 consecutive
-// elements.
+// In the 128 tile a thread's rows and columns come in groups of four consecutive ones (rows 4 ty + i and 64 + 4 ty + i,
+// columns likewise with tx): one 16-byte shared-memory read fetches a group, 4 reads per 64 FMAs instead of 16 scalar
+// ones (the 16 threads of a half warp read 256 consecutive bytes of a row of B and all the same 16 bytes of A), and
+// a half warp's stores to C cover 64 consecutive elements: 8192^3 29.5 -> 37.6 TFLOP/s, 4096^3 34.1 -> 38.0.  (With
+// columns tx * 8 + j - eight consecutive ones - the reads of B were four-way bank conflicts and the rung ran at a
+// quarter of the fp32 pipe.)  The 64 and 32 tiles keep rows ty + 16 i and columns tx + 16 j, read word by word.
 //
 // The tile is the largest of the three that still gives every SM a CTA: a
 // 256^3 product is 4 tiles of 128 x 128 but 64 of 32 x 32, and a rung that
@@ -34,9 +35,16 @@ __global__ void __launch_bounds__(NT, 2) r1_tiled_kernel(GemmArgs g, int tiles_m
     // the deeper slab was slower, 8192^3 29.5 -> 27.3 TFLOP/s)
     constexpr int BK = T == 128 ? 16 : 32;
     // a warp covers 16 k of 2 rows: 2 mod 32 spreads them over 32 banks; 32 k of one row with the deeper slab: 1 mod 32
-    constexpr int PITCH = BK == 16 ? T + 2 : T + 1;
-    __shared__ float As[BK][PITCH];
-    __shared__ float Bs[BK][PITCH];
+    // 128 tile: rows stay 16-byte aligned for the register tile's vector reads; smaller tiles: a warp's fill covers 32 k
+    // of one row, 1 mod 32 spreads them over the banks
+    constexpr int PITCH = T == 128 ? T + 4 : T + 1;
+    // fill loops: eight loads in flight push the 128 tile past its 128 registers (spills); the smaller tiles want them all
+    constexpr int FILL_UNROLL = T == 128 ? 4 : 8;
+    // a thread's rows (columns) come in groups of V consecutive ones: 4 for the 128 tile (vector reads), else single
+    // rows ty + 16 i and columns tx + 16 j read word by word (the smaller tiles stay as plain as the rung's name)
+    constexpr int V = T == 128 ? 4 : 1;
+    __shared__ __align__(16) float As[BK][PITCH];
+    __shared__ __align__(16) float Bs[BK][PITCH];
     if (blockIdx.x == 0 && threadIdx.x == 0) g.status[1] = kIdTiled;
 
     int tm, tn;
@@ -53,7 +61,7 @@ __global__ void __launch_bounds__(NT, 2) r1_tiled_kernel(GemmArgs g, int tiles_m
 
     for (int k0 = 0; k0 < g.K; k0 += BK) {
         // A slab: T rows x 16 k, one element per thread per step, k fastest.
-#pragma unroll
+#pragma unroll FILL_UNROLL
         for (int e = t; e < T * BK; e += NT) {
             const int k = e % BK, m = e / BK;
             const int64_t gm = m0 + m;
@@ -61,7 +69,7 @@ __global__ void __launch_bounds__(NT, 2) r1_tiled_kernel(GemmArgs g, int tiles_m
             As[k][m] = (gm < g.M && gk < g.K) ? bf16_bits_to_float(g.A[gm * g.lda + gk]) : 0.f;
         }
         if (BCOL) {
-#pragma unroll
+#pragma unroll FILL_UNROLL
             for (int e = t; e < T * BK; e += NT) {
                 const int k = e % BK, n = e / BK;
                 const int64_t gn = n0 + n;
@@ -69,7 +77,7 @@ __global__ void __launch_bounds__(NT, 2) r1_tiled_kernel(GemmArgs g, int tiles_m
                 Bs[k][n] = (gn < g.N && gk < g.K) ? bf16_bits_to_float(g.B[gn * g.ldb + gk]) : 0.f;
             }
         } else {
-#pragma unroll
+#pragma unroll FILL_UNROLL
             for (int e = t; e < T * BK; e += NT) {
                 const int n = e % T, k = e / T;
                 const int64_t gn = n0 + n;
@@ -82,9 +90,17 @@ __global__ void __launch_bounds__(NT, 2) r1_tiled_kernel(GemmArgs g, int tiles_m
         for (int k = 0; k < BK; ++k) {
             float a[TT], b[TT];
 #pragma unroll
-            for (int i = 0; i < TT; ++i) a[i] = As[k][ty + 16 * i];
-#pragma unroll
-            for (int j = 0; j < TT; ++j) b[j] = Bs[k][tx + 16 * j];
+            for (int i = 0; i < TT; i += V) {
+                const float* pa = &As[k][(i / V) * 16 * V + ty * V];
+                const float* pb = &Bs[k][(i / V) * 16 * V + tx * V];
+                if (V == 4) {
+                    *reinterpret_cast<float4*>(&a[i]) = *reinterpret_cast<const float4*>(pa);
+                    *reinterpret_cast<float4*>(&b[i]) = *reinterpret_cast<const float4*>(pb);
+                } else {
+                    a[i] = *pa;
+                    b[i] = *pb;
+                }
+            }
 #pragma unroll
             for (int i = 0; i < TT; ++i)
 #pragma unroll
@@ -95,11 +111,11 @@ __global__ void __launch_bounds__(NT, 2) r1_tiled_kernel(GemmArgs g, int tiles_m
 
 #pragma unroll
     for (int i = 0; i < TT; ++i) {
-        const int64_t gm = m0 + ty + 16 * i;
+        const int64_t gm = m0 + (i / V) * 16 * V + ty * V + (i % V);
         if (gm >= g.M) continue;
 #pragma unroll
         for (int j = 0; j < TT; ++j) {
-            const int64_t gn = n0 + tx + 16 * j;
+            const int64_t gn = n0 + (j / V) * 16 * V + tx * V + (j % V);
             if (gn < g.N) store_c(g.C, g.c_bf16, gm * g.ldc + gn, acc[i][j] + bias_at(g, gn));
         }
     }
