@@ -93,6 +93,7 @@ struct PairParams {
     int tile_n, n_wide, tile_n2, n_narrow;
     int64_t wide_tiles;         // tiles_m2 * n_wide
     int snake;                  // 1: odd rounds of the schedule run over the pairs in reverse order
+    int one_round;              // 1 (one problem): uniform tiles, at most one per pair - tile t is (t / n_wide, t % n_wide)
     uint32_t stage_tx;          // bytes the loads of both CTAs deliver per stage
     int b_boxes;                // row-major B: 64-column boxes per CTA and stage (1 or 2)
     // Streamed last wave (MODE 0, uniform 256-column tiles).  Tiles [0, sk_first) run whole, sk_rounds of them per
@@ -345,7 +346,15 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             } else {
                 x.z = 0;
                 x.C = static_cast<uint8_t*>(g.C);
-                if (t < p.wide_tiles) {
+                if (p.one_round) {
+                    // one round of uniform tiles, at most one per pair: their order does not matter, and the first
+                    // decode is on the critical path of a short launch - one 32-bit division, row-major
+                    const uint32_t t32 = static_cast<uint32_t>(t), per_row = static_cast<uint32_t>(p.n_wide);
+                    tm = static_cast<int>(t32 / per_row);
+                    tn = static_cast<int>(t32 - static_cast<uint32_t>(tm) * per_row);
+                    x.n0 = tn * p.tile_n;
+                    x.width = p.tile_n;
+                } else if (t < p.wide_tiles) {
                     raster_tile(t, p.tiles_m2, p.n_wide, tm, tn, p.group_m);
                     x.n0 = tn * p.tile_n;
                     x.width = p.tile_n;
@@ -1542,8 +1551,8 @@ bool pair_k_paired(const GemmArgs& g, const RunContext& ctx)
 }
 }
 
-// One problem, nothing pinned.  One round of 256 x 256 tiles that fills more than half of the CTA pairs, K long enough
-// to pay for the pair kernel's set-up - measured (single launches after an L2 flush, against the single-CTA kernel's one
+// One problem, nothing pinned.  One round of 256 x 256 tiles that fills more than half of the CTA pairs, K >= 2048 to
+// pay for the pair kernel's set-up (2048^3 in graph replay: 15.9 against 16.1 us; 2048 x 2048 x 1024 11.7 against 11.0) - measured (single launches after an L2 flush, against the single-CTA kernel's one
 // wave of 128 x 256 tiles): 2048 x 2048 x 8192 56.2 against 61.4 us, 512 x 8192 x 8192 61.5 / 65.5, 1536 x 2048 x 4096
 // 32.8 / 34.8, 2304 x 2048 x 6144 45.6 / 49.1, 2048 x 2048 x 3072 28.2 / 28.8; with 32 tiles (1024 x 2048 x 8192) 54
 // against 42 for the single-CTA kernel's cluster split.  Several rounds: when they beat the 512-row tiles' rounds
@@ -1555,7 +1564,7 @@ bool r4_pair_k_paired_auto(const GemmArgs& g, const RunContext& ctx)
     const int64_t tn = (g.N + PN - 1) / PN;
     const int64_t tiles = static_cast<int64_t>((g.M + 2 * PM - 1) / (2 * PM)) * tn;
     const int64_t pairs = ctx.sm_count / 2;
-    if (tiles <= pairs) return 2 * tiles > pairs && g.K >= 3072;
+    if (tiles <= pairs) return 2 * tiles > pairs && g.K >= 2048;
     const int64_t nkb = (g.K + BK - 1) / BK;
     if (!pair_k_paired_faster(tiles, static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * tn, nkb, pairs)) return false;
     const int64_t r256 = (tiles + pairs - 1) / pairs;
@@ -1694,6 +1703,7 @@ cudaError_t launch_pair_one_problem(const GemmArgs& g, void* const* dst_c, const
     } else if (ctx.plan.split_via == 3) {
         return cudaErrorInvalidValue;
     }
+    p.one_round = (!p.sk && cols.n_narrow == 0 && p.total_tiles <= max_pairs && p.tiles_m2 > 1) ? 1 : 0;
     p.kid = kIdTcgen05 + (p.epi_tma ? 0 : 2) + 32 + (p.sk ? 128 : 0) + (kp ? 256 : 0) + ctx.kid_flags;
     *kernel_id = p.kid;
     if (n_dst > 0) {

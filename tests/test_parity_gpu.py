@@ -352,7 +352,7 @@ def test_tcgen05_cta_pair_k_paired_tiles(handles, col):
 def test_dispatch_between_the_two_kernels(handles):
     """Long K and enough 512 x 256 (or 256 x 256) tiles: the pair kernel; short K or few tiles: the single-CTA kernel."""
     for (M, N, K), want_pair in (((2048, 4096, 4096), True), ((3072, 2048, 8192), True), ((2816, 2816, 2816), True),
-                                 ((2048, 2048, 2048), False), ((1536, 3072, 1024), False), ((3584, 3584, 3584), True),    # (three rounds of 256-row tiles)
+                                 ((2048, 2048, 1024), False), ((1536, 3072, 1024), False), ((3584, 3584, 3584), True),    # (three rounds of 256-row tiles)
                                  ((2304, 2304, 2304), True), ((1536, 1536, 1536), False), ((4096, 4096, 512), True),
                                  ((2048, 2048, 8192), True),       # one round of 64 k-paired 256-row tiles
                                  ((1024, 2048, 8192), False)):     # 32 such tiles: the single-CTA kernel's cluster split
