@@ -689,6 +689,11 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                     break;
                 }
             }
+            // AddMM: this lane's bias values of the tile's eight 32-column blocks, fetched while the MMAs still run (inside
+            // the drain their ~600-clock loads stood in the way of every unit: 4096^3 with bias 97.2 us against 95.0 without)
+            float pb[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) pb[k] = (g.bias && n0 + 32 * k + lane < x.N) ? bias_at(g, n0 + 32 * k + lane) : 0.f;
             if (!ptx::mbar_wait(&acc_full[KP ? ab : 0], (KP ? tcount >> 1 : tcount) & 1, abort_flag)) {
                 if (lane == 0) report_error(g.status, kDevBarrierTimeout, blockIdx.x, 0x540u);
                 abort_flag[0] = 1;
@@ -712,13 +717,21 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
             };
             // pack: bias and rounding of one unit (r0, r1 -> 32 words of output); stage_store: the words
             // go through the warp's staging block to global memory
-            auto pack = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32], uint32_t (&w)[32]) {
+            // (`pre`: u is a literal at the call site - the prefetched values are picked at compile time; the general
+            // loops, whose u is a variable, fetch the unit's bias here)
+            auto pack = [&](int u, uint32_t (&r0)[32], uint32_t (&r1)[32], uint32_t (&w)[32], bool pre = false) {
                 const int col0 = n0 + u * cpc;
                 if (g.bias) {   // AddMM: this unit's columns get their bias in fp32, before any rounding
-                    // lane l fetches the bias of columns col0 + l and col0 + 32 + l; a shuffle hands column i's
+                    // lane l holds the bias of columns col0 + l and col0 + 32 + l; a shuffle hands column i's
                     // value to every lane (every lane holds a different row of the same columns)
-                    const float b0 = (col0 + lane < x.N) ? bias_at(g, col0 + lane) : 0.f;
-                    const float b1 = (out_bf16 && col0 + 32 + lane < x.N) ? bias_at(g, col0 + 32 + lane) : 0.f;
+                    float b0, b1;
+                    if (pre) {
+                        b0 = out_bf16 ? pb[(2 * u) & 7] : pb[u & 7];
+                        b1 = out_bf16 ? pb[(2 * u + 1) & 7] : 0.f;
+                    } else {
+                        b0 = (col0 + lane < x.N) ? bias_at(g, col0 + lane) : 0.f;
+                        b1 = (out_bf16 && col0 + 32 + lane < x.N) ? bias_at(g, col0 + 32 + lane) : 0.f;
+                    }
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         r0[i] = __float_as_uint(__uint_as_float(r0[i]) + __shfl_sync(0xFFFFFFFFu, b0, i));
@@ -961,7 +974,7 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 issue(1, c0, c1);
                 issue(2, d0, d1);
                 if (tcount == 0 && warp == kEpiWarp0 && lane == 0) KLIN_T(57);
-                pack(0, a0, a1, w0);           // (while units 1 and 2 are on their way) frees a0, a1 for the fourth unit
+                pack(0, a0, a1, w0, true);     // (while units 1 and 2 are on their way) frees a0, a1 for the fourth unit
                 if (tcount == 0 && warp == kEpiWarp0 && lane == 0) KLIN_T(58);
                 issue(3, a0, a1);
                 ptx::tmem_ld_wait();
@@ -969,11 +982,11 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 release();
                 if (warp == kEpiWarp0 && lane == 0) KLIN_T(tcount < 8 ? 41 + 3 * static_cast<int>(tcount) : -1);
                 stage_store(0, w0);
-                pack(1, c0, c1, w0);
+                pack(1, c0, c1, w0, true);
                 stage_store(1, w0);
-                pack(2, d0, d1, w0);
+                pack(2, d0, d1, w0, true);
                 stage_store(2, w0);
-                pack(3, a0, a1, w0);
+                pack(3, a0, a1, w0, true);
                 stage_store(3, w0);
                 if (warp == kEpiWarp0 && lane == 0) KLIN_T(tcount < 8 ? 42 + 3 * static_cast<int>(tcount) : -1);
                 continue;
@@ -989,25 +1002,25 @@ r4_pair_kernel(GemmArgs g, const __grid_constant__ CUtensorMap map_a, const __gr
                 issue(4, d0, d1);
                 issue(5, d1, d0);
                 ptx::tmem_ld_wait();
-                if (g.bias) pack(0, a0, a0, a0);
+                if (g.bias) pack(0, a0, a0, a0, true);
                 stage_store(0, a0);
                 issue(6, a0, a0);
-                if (g.bias) pack(1, a1, a1, a1);
+                if (g.bias) pack(1, a1, a1, a1, true);
                 stage_store(1, a1);
                 issue(7, a1, a1);
                 ptx::tmem_ld_wait();
                 release();
-                if (g.bias) pack(2, c0, c0, c0);
+                if (g.bias) pack(2, c0, c0, c0, true);
                 stage_store(2, c0);
-                if (g.bias) pack(3, c1, c1, c1);
+                if (g.bias) pack(3, c1, c1, c1, true);
                 stage_store(3, c1);
-                if (g.bias) pack(4, d0, d0, d0);
+                if (g.bias) pack(4, d0, d0, d0, true);
                 stage_store(4, d0);
-                if (g.bias) pack(5, d1, d1, d1);
+                if (g.bias) pack(5, d1, d1, d1, true);
                 stage_store(5, d1);
-                if (g.bias) pack(6, a0, a0, a0);
+                if (g.bias) pack(6, a0, a0, a0, true);
                 stage_store(6, a0);
-                if (g.bias) pack(7, a1, a1, a1);
+                if (g.bias) pack(7, a1, a1, a1, true);
                 stage_store(7, a1);
                 continue;
             }
