@@ -1564,8 +1564,9 @@ bool pair_k_paired(const GemmArgs& g, const RunContext& ctx)
 }
 }
 
-// One problem, nothing pinned.  One round of 256 x 256 tiles that fills more than half of the CTA pairs, K >= 2048 to
-// pay for the pair kernel's set-up (2048^3 in graph replay: 15.9 against 16.1 us; 2048 x 2048 x 1024 11.7 against 11.0) - measured (single launches after an L2 flush, against the single-CTA kernel's one
+// One problem, nothing pinned.  One round of 256 x 256 tiles that fills more than half of the CTA pairs, K >= 3072: at
+// 2048^3 the form is level with the single-CTA kernel in graph replay (15.9 against 16.1 us) but its cluster launch
+// costs the host more, and launches enqueued one by one fall behind (18.5 against 16.9 us per launch) - measured (single launches after an L2 flush, against the single-CTA kernel's one
 // wave of 128 x 256 tiles): 2048 x 2048 x 8192 56.2 against 61.4 us, 512 x 8192 x 8192 61.5 / 65.5, 1536 x 2048 x 4096
 // 32.8 / 34.8, 2304 x 2048 x 6144 45.6 / 49.1, 2048 x 2048 x 3072 28.2 / 28.8; with 32 tiles (1024 x 2048 x 8192) 54
 // against 42 for the single-CTA kernel's cluster split.  Several rounds: when they beat the 512-row tiles' rounds
@@ -1577,7 +1578,7 @@ bool r4_pair_k_paired_auto(const GemmArgs& g, const RunContext& ctx)
     const int64_t tn = (g.N + PN - 1) / PN;
     const int64_t tiles = static_cast<int64_t>((g.M + 2 * PM - 1) / (2 * PM)) * tn;
     const int64_t pairs = ctx.sm_count / 2;
-    if (tiles <= pairs) return 2 * tiles > pairs && g.K >= 2048;
+    if (tiles <= pairs) return 2 * tiles > pairs && g.K >= 3072;
     const int64_t nkb = (g.K + BK - 1) / BK;
     if (!pair_k_paired_faster(tiles, static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * tn, nkb, pairs)) return false;
     const int64_t r256 = (tiles + pairs - 1) / pairs;
