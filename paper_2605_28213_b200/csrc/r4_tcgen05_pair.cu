@@ -1503,7 +1503,32 @@ StreamK plan_stream_k(int64_t tiles, int nkb, int64_t pairs, const RunContext& c
     return sk;
 }
 
+PairColumns plan_columns_uncached(const GemmArgs& g, const RunContext& ctx);
+
+// The search below evaluates up to fifty schedules of seventy-four pairs each: 8-20 us of host time, which a launch of a
+// dozen microseconds enqueued in a loop cannot hide (4096 x 4096 x 256: 21.5 us per call against 13.4 for the single-CTA
+// kernel's launch).  Its result depends on the sizes and the plan only: the last few are remembered per thread.
 PairColumns plan_columns(const GemmArgs& g, const RunContext& ctx)
+{
+    struct Entry {
+        int64_t M, N, K;
+        int sm, tile_n, tail_n, split_via;
+        bool used;
+        PairColumns cols;
+    };
+    static thread_local Entry memo[8] = {};
+    static thread_local unsigned next = 0;
+    for (const Entry& e : memo)
+        if (e.used && e.M == g.M && e.N == g.N && e.K == g.K && e.sm == ctx.sm_count && e.tile_n == ctx.plan.tile_n &&
+            e.tail_n == ctx.plan.tail_n && e.split_via == ctx.plan.split_via)
+            return e.cols;
+    Entry& e = memo[next++ % 8];
+    e = Entry{g.M, g.N, g.K, ctx.sm_count, ctx.plan.tile_n, ctx.plan.tail_n, ctx.plan.split_via, true,
+              plan_columns_uncached(g, ctx)};
+    return e.cols;
+}
+
+PairColumns plan_columns_uncached(const GemmArgs& g, const RunContext& ctx)
 {
     const int64_t tiles_m2 = (g.M + TILE_M - 1) / TILE_M;
     const int64_t nkb = (g.K + BK - 1) / BK;
