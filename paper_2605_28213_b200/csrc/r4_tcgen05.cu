@@ -1787,7 +1787,12 @@ int cluster_fixed_cost(int s, int64_t ctas, int sm, int tile_n)
 {
     // (128-column tiles exchange half as much: 1.7 / 2.0 / 2.5 us less)
     const int base = tile_n == BN ? (s == 2 ? 13 : s == 4 ? 16 : 22) : (s == 2 ? 8 : s == 4 ? 10 : 14);
-    return base + (ctas * 3 > static_cast<int64_t>(sm) * 2 ? 12 : 0);
+    // (a launch of fours or eights over most of the GPU: 35 k-block times measured at 768 x 768 x 3072 and at 1024 x 1024 x
+    // 4096 - 16.3 us in fours against 14.4 in pairs - where 16 + 12 said 28)
+    // 256-column tiles pay it from a third of the GPU on: 1024 x 1024 x 4096 in pairs of 256-column tiles (64 CTAs) 17.9 us
+    // = 26 k-block times over its 32 k-blocks, in pairs of 128-column tiles (128 CTAs) 14.4 us.
+    const bool crowded = tile_n == BN ? ctas * 3 > static_cast<int64_t>(sm) : ctas * 3 > static_cast<int64_t>(sm) * 2;
+    return base + (crowded ? (s >= 4 && ctas * 3 > static_cast<int64_t>(sm) * 2 ? 19 : 12) : 0);
 }
 // Clusters of `s` CTAs of this kernel that the device can hold at once (GPC boundaries make this less than
 // SMs / s for large clusters); asked of the runtime once per size and device.
