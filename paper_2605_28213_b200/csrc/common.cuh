@@ -249,6 +249,9 @@ cudaError_t launch_zero_fill(const GemmArgs& g, cudaStream_t stream, int* kernel
 bool r4_pair_applicable(const GemmArgs& g, const RunContext& ctx);
 // The same estimate for a batched or grouped launch, on its tile counts (128 x 256 / 256 x 256 / 512 x 256) and longest K.
 bool r4_pair_faster_multi(int64_t tiles128, int64_t tiles256, int64_t tiles512, int64_t nkb, const RunContext& ctx);
+// One wave of 128 x 128 tiles whose columns are at least 8 points fuller than those of 256-column tiles (N = 1064: 0.92
+// against 0.83): the single-CTA kernel then runs its 128-column tiles, and the pair kernel's 256-column forms stand back.
+bool r4_narrow_tiles_fill_better(int64_t M, int64_t N, int sm_count);
 // Whether an unpinned single-destination launch takes the pair kernel's k-paired 256-row tiles.
 bool r4_pair_k_paired_auto(const GemmArgs& g, const RunContext& ctx);
 // Hard preconditions of the CTA-pair kernel only (operands TMA-loadable), without the size heuristic.

@@ -1800,12 +1800,21 @@ int max_resident_clusters(int s, const RunContext& ctx);
 
 // K splits of the cluster route for a regular-orientation problem and their estimated cost (k-block times);
 // 1 when no split fits or pays.
+// A k-block of an UNSPLIT launch in fifths of a wide tile's k-block time: 128-column tiles take 4 (paired k-blocks) while
+// the launch is small and 5 once a third of the SMs or more are at work (1208 x 992 x 4936, 80 such tiles: 0.32 us per
+// k-block, 28.9 us against 24.6 in pairs; 592 x 1688 x 2744, 70 tiles: 18.4 against 15.2).  The splits themselves keep 4:
+// 160 x 4016 x 4000 in pairs of 128-column tiles runs 0.27 us per k-block on 128 CTAs.
+int64_t unsplit_kb_cost(int tile_n, int64_t tiles, int sm)
+{
+    return (tile_n == BN || tiles * 3 > sm) ? 5 : 4;
+}
+
 int choose_regular_cluster_splits(int64_t tiles, int nkb, const RunContext& ctx, int tile_n, int64_t* cost_out)
 {
     int best = 1;
     // costs in fifths of a k-block time; a k-block of a narrow tile (paired k-blocks) takes about 0.8 of a wide one's
     const int64_t kb_cost = tile_n == BN ? 5 : 4;
-    int64_t best_cost = ((tiles + ctx.sm_count - 1) / ctx.sm_count) * static_cast<int64_t>(nkb) * kb_cost;
+    int64_t best_cost = ((tiles + ctx.sm_count - 1) / ctx.sm_count) * static_cast<int64_t>(nkb) * unsplit_kb_cost(tile_n, tiles, ctx.sm_count);
     for (int s = 2; s <= 8 && s * 2 <= nkb; s *= 2) {
         const int per = (nkb + s - 1) / s;
         if ((nkb + per - 1) / per != s) continue;
@@ -1851,7 +1860,7 @@ SplitPlan plan_split(int M, int64_t tiles, int nkb, int64_t ldw, const RunContex
         const int per_w = (nkb + sp.splits - 1) / sp.splits;
         // (in fifths of a k-block time, like the cluster route's estimate)
         sp.cost = sp.splits > 1 ? ((tiles * sp.splits + sm - 1) / sm) * static_cast<int64_t>(per_w + 30 + 6 * sp.splits) * 5
-                                : ((tiles + sm - 1) / sm) * static_cast<int64_t>(nkb) * (tile_n == BN ? 5 : 4);
+                                : ((tiles + sm - 1) / sm) * static_cast<int64_t>(nkb) * unsplit_kb_cost(tile_n, tiles, sm);
         int64_t cost_c = 0;
         const int sc = choose_regular_cluster_splits(tiles, nkb, ctx, tile_n, &cost_c);
         if (sc > 1 && cost_c <= sp.cost) {
@@ -2068,6 +2077,15 @@ bool plan_launch(const GemmArgs& g, const RunContext& ctx, bool generic, bool mu
     // splits; unsplit, 128-column tiles match the half-tile tail when one under-filled wave is all there is (they load
     // only the columns they use) and lose once the tiles no longer fit one wave.
     bool take_narrow;
+    // Columns that 256-wide tiles fill badly (N just above a multiple of 256) while one wave of 128-wide tiles fills
+    // them well: measured unsplit, 128 against 256 columns, 1912 x 1064 x 3544 25.6 against 37.1 us, 3104 x 528 x 4784
+    // 24.1 / 34.1, 3632 x 616 x 816 9.2 / 12.0, 4848 x 304 x 1144 10.4 / 13.4, 1808 x 1112 x 320 6.3 / 7.7.
+    if (pl.splits == 0 && pl.split_via == 0 && wide.split.splits == 1 && narrow.split.splits == 1 &&
+        r4_narrow_tiles_fill_better(g.M, g.N, ctx.sm_count)) {
+        narrow.stages = nkb >= 16 ? 6 : 4;       // (short K: the plain four-stage ring was the faster one in those runs)
+        *out = narrow;
+        return true;
+    }
     if (pl.splits > 0)
         take_narrow = narrow.split.cluster || (narrow.split.splits == 1 && tiles256 * 2 <= ctx.sm_count);
     else if (narrow.split.cost != wide.split.cost)
@@ -2631,6 +2649,16 @@ cudaError_t launch_r4_multi_dst(const GemmArgs& g, void* const* C, const int64_t
     if (!C || !ldc || n_dst < 1 || n_dst > kMaxDst) return cudaErrorInvalidValue;
     const MultiDst md = {C, ldc, n_dst};
     return launch_r4_planned(g, ctx, stream, kernel_id, &md);
+}
+
+bool r4_narrow_tiles_fill_better(int64_t M, int64_t N, int sm_count)
+{
+    if (M <= 0 || N <= 0) return false;
+    const int64_t tm = (M + BM - 1) / BM, wide = (N + BN - 1) / BN, narrow = (N + BN / 2 - 1) / (BN / 2);
+    if (tm * narrow > sm_count) return false;
+    const double fill_wide = static_cast<double>(N) / static_cast<double>(wide * BN);
+    const double fill_narrow = static_cast<double>(N) / static_cast<double>(narrow * (BN / 2));
+    return fill_narrow >= fill_wide + 0.08;
 }
 
 bool r4_plan_valid(const GemmArgs& g, const RunContext& ctx, const R4Plan& pl)

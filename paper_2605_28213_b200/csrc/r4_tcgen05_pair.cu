@@ -1603,7 +1603,17 @@ bool r4_pair_k_paired_auto(const GemmArgs& g, const RunContext& ctx)
     const int64_t tn = (g.N + PN - 1) / PN;
     const int64_t tiles = static_cast<int64_t>((g.M + 2 * PM - 1) / (2 * PM)) * tn;
     const int64_t pairs = ctx.sm_count / 2;
-    if (tiles <= pairs) return 2 * tiles > pairs && g.K >= 3072;
+    if (tiles <= pairs) {
+        // (not where one wave of the single-CTA kernel's 128-column tiles fills the matrix's columns much better: at
+        // 1912 x 1064 x 3544 - the fifth 256-column tile holds 40 columns - they take 25.7 us against 29.2, at 3104 x
+        // 528 x 4784 24.0 against 28.8)
+        // K: from 3072 on; from 1280 on where the single-CTA kernel's wave of 128 x 256 tiles would be less than 85 % full
+        // (launches enqueued one by one, us: 1328 x 1944 x 2128 18.6 against 22.9, 544 x 5896 x 1776 18.0 / 20.2, 1472 x 2040 x
+        // 1496 18.4 / 19.7; at 2048^3 - 128 tiles on 148 SMs - 18.5 against 16.9)
+        const int64_t tiles1 = static_cast<int64_t>((g.M + PM - 1) / PM) * tn;
+        const bool k_ok = g.K >= 3072 || (g.K >= 1280 && tiles1 * 100 < static_cast<int64_t>(ctx.sm_count) * 85);
+        return 2 * tiles > pairs && k_ok && !r4_narrow_tiles_fill_better(g.M, g.N, ctx.sm_count);
+    }
     const int64_t nkb = (g.K + BK - 1) / BK;
     if (!pair_k_paired_faster(tiles, static_cast<int64_t>((g.M + TILE_M - 1) / TILE_M) * tn, nkb, pairs)) return false;
     const int64_t r256 = (tiles + pairs - 1) / pairs;
