@@ -2080,13 +2080,11 @@ bool plan_launch(const GemmArgs& g, const RunContext& ctx, bool generic, bool mu
     // Columns that 256-wide tiles fill badly (N just above a multiple of 256) while one wave of 128-wide tiles fills
     // them well: measured unsplit, 128 against 256 columns, 1912 x 1064 x 3544 25.6 against 37.1 us, 3104 x 528 x 4784
     // 24.1 / 34.1, 3632 x 616 x 816 9.2 / 12.0, 4848 x 304 x 1144 10.4 / 13.4, 1808 x 1112 x 320 6.3 / 7.7.
-    if (pl.splits == 0 && pl.split_via == 0 && wide.split.splits == 1 && narrow.split.splits == 1 &&
-        r4_narrow_tiles_fill_better(g.M, g.N, ctx.sm_count)) {
-        narrow.stages = nkb >= 16 ? 6 : 4;       // (short K: the plain four-stage ring was the faster one in those runs)
-        *out = narrow;
-        return true;
-    }
-    if (pl.splits > 0)
+    const bool fuller = pl.splits == 0 && pl.split_via == 0 && wide.split.splits == 1 && narrow.split.splits == 1 &&
+                        r4_narrow_tiles_fill_better(g.M, g.N, ctx.sm_count);
+    if (fuller)
+        take_narrow = true;
+    else if (pl.splits > 0)
         take_narrow = narrow.split.cluster || (narrow.split.splits == 1 && tiles256 * 2 <= ctx.sm_count);
     else if (narrow.split.cost != wide.split.cost)
         take_narrow = narrow.split.cost < wide.split.cost;
@@ -2095,6 +2093,7 @@ bool plan_launch(const GemmArgs& g, const RunContext& ctx, bool generic, bool mu
     // the deepest ring: six real stages for a cluster split; unsplit, three stages of two k-blocks each (one barrier round
     // trip per eight MMAs: 1024^3 9.1 -> 8.4 us, 1536^3 13.2 -> 11.5 in graph replay)
     if (take_narrow && (narrow.split.cluster || narrow.split.splits == 1)) narrow.stages = 6;
+    if (fuller && nkb < 16) narrow.stages = 4;      // (short K: the plain four-stage ring was the faster one in those runs)
     if (take_narrow && narrow.split.splits == 1 && g.N > BN / 4) {
         // still at most half a wave of 128-column tiles: 64 columns (measured 0.4 - 0.5 us off a 5 - 7 us launch at
         // 256^3, 512^3 and 300 x 520 x 200: an MMA takes as long whatever its width, the epilogue of a tile shrinks)
