@@ -449,8 +449,10 @@ klineage_status_t klineage_gemm_run_host(klineage_gemm_t h, int64_t M, int64_t N
  *              64-column tiles are filled and freed two k-blocks at a time (3 / 4 stages of 128 k).
  *              CTA-pair kernel: 3 = tiles of 256 x 256 instead of 512 x 256, three stages of two k-blocks each,
  *              the two TMEM accumulators holding consecutive tiles of a pair (one fills while the other drains);
- *              256-column tiles only, no narrow tail, no streamed wave.  The heuristic takes it for K >= 3072
- *              when such tiles make one round over more than half of the CTA pairs
+ *              256-column tiles only, no narrow tail, no streamed wave.  The heuristic takes it when such
+ *              tiles make one round over more than half of the CTA pairs (K >= 3072, or K >= 1280 where the
+ *              single-CTA kernel's wave would be less than 85 % full) or several rounds that its cycle estimate
+ *              puts ahead of the 512-row tiles' rounds
  * Every plan computes the same C up to fp32 summation order (plans that differ
  * only in kernel / group_m / half_tail / tile shape / stages are bit-identical; K
  * splits change the order of the partial sums and stay within the parity bound).
