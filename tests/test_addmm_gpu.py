@@ -147,11 +147,16 @@ def test_addmm_argument_errors(kb):
 
 
 @pytest.mark.parametrize("bf", [False, True], ids=["f32", "bf16"])
-def test_addmm_on_the_pair_kernel_full_width_tiles(kb, bf):
-    # full-width tiles of the CTA-pair kernel hand the accumulator back before they stage and store:
-    # the bias must still reach every unit, for both output types
+@pytest.mark.parametrize("plan,shape", [((2, 1, 0, 0, 0), (600, 776, 136)),
+                                        ((2, 1, 0, 0, 0, 0, 0, 3), (600, 776, 136)),        # 256-row tiles, one per pair
+                                        ((2, 1, 0, 0, 0, 0, 0, 3), (2100, 2056, 200))],     # 81 of them: two for some pairs
+                         ids=["512-row", "256-row", "256-row-two-rounds"])
+def test_addmm_on_the_pair_kernel_full_width_tiles(kb, bf, plan, shape):
+    # full-width tiles of the CTA-pair kernel hand the accumulator back before they stage and store, and a lane fetches
+    # its bias values before the accumulator is complete: the bias must still reach every unit, for both output types
+    # and both tile heights
     import torch
-    M, N, K = 600, 776, 136
+    M, N, K = shape
     for dist, exact in (("integer", True), ("normal", False)):
         case = gen.make_case(M, N, K, seed=260, dist_a=dist, dist_b=dist, c_bf16=bf, name=f"addmm-pair-{dist}")
         bias = gen.draw((1, N), dist, 261, 2)[0]
@@ -159,10 +164,11 @@ def test_addmm_on_the_pair_kernel_full_width_tiles(kb, bf):
         dev = P.DeviceCase(case)
         bbuf = P.DeviceBuffer(bias.size * 2).upload(bias)
         with kb.Gemm(0, c_bf16=bf) as g:
-            g.set_plan(kb.klineage_gemm_plan_t(2, 1, 0, 0, 0), dev.a.ptr, dev.b.ptr, dev.c.ptr, M, N, K, case.lda, case.ldb,
+            g.set_plan(kb.klineage_gemm_plan_t(*plan), dev.a.ptr, dev.b.ptr, dev.c.ptr, M, N, K, case.lda, case.ldb,
                        case.ldc)
             g.run_addmm(dev.a.ptr, dev.b.ptr, bbuf.ptr, dev.c.ptr, M, N, K, case.lda, case.ldb, case.ldc, 4)
             torch.cuda.synchronize()
-            assert g.device_status()[0] == 0 and (g.last_kernel_id() - 400) & 32
+            flags = g.last_kernel_id() - 400
+            assert g.device_status()[0] == 0 and flags & 32 and bool(flags & 256) == (len(plan) == 8)
         vals, bits = dev.result()
         P.assert_matches_oracle(case, vals, bits, C_ref, S, exact=exact, what=f"{case.name} bf16={bf}")
